@@ -1,0 +1,353 @@
+"""Pins for the CPU oracle: what the paper and the mathematics fix, checked without a GPU."""
+import math
+import os
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import a3_oracle as O
+from paper_2511_17560_b200 import workloads as W
+from tests.helpers import make_request, oracle_model, oracle_weights
+
+GOLDEN = os.path.join(os.path.dirname(__file__), "golden")
+
+
+# ------------------------------------------------------------------ RoPE (Eq. 2)
+
+
+def test_rope_d4_matrix_written_out():
+    """The printed 4x4 rotation, multiplied out by hand (tests/golden/rope_d4.txt)."""
+    for line in open(os.path.join(GOLDEN, "rope_d4.txt")):
+        if line.startswith("#"):
+            continue
+        v = [float(t) for t in line.split()]
+        base, m, x, y = v[0], int(v[1]), np.array(v[2:6]), np.array(v[6:10])
+        got = O.rope_rotate(x.reshape(1, 1, 4), np.array([m]), base, layout=1)[0, 0]
+        np.testing.assert_allclose(got, y, rtol=0, atol=1e-12)
+        # half-split layout is the same rotation on pairs (0,2),(1,3)
+        xs = x[[0, 2, 1, 3]]
+        got2 = O.rope_rotate(xs.reshape(1, 1, 4), np.array([m]), base, layout=0)[0, 0]
+        np.testing.assert_allclose(got2, y[[0, 2, 1, 3]], rtol=0, atol=1e-12)
+
+
+@pytest.mark.parametrize("D", [64, 128])
+@pytest.mark.parametrize("theta", [1e4, 5e5, 1e6])
+@pytest.mark.parametrize("layout", [0, 1])
+@pytest.mark.parametrize("dtype,tol", [(np.float64, 1e-9), (np.float32, 1e-5)])
+def test_rope_composition_identity(D, theta, layout, dtype, tol):
+    """R(delta) R(m) x == R(m + delta) x; R(0) = I; the rotation keeps the norm."""
+    rng = np.random.default_rng(1)
+    T = 33
+    x = rng.standard_normal((T, 3, D)).astype(dtype)
+    m = rng.integers(0, 2048, size=T)
+    for delta in (0, 1, 511, 512, 5120, 32256):
+        d = np.full(T, delta)
+        two = O.rope_rotate(O.rope_rotate(x, m, theta, layout), d, theta, layout)
+        one = O.rope_rotate(x, m + d, theta, layout)
+        assert np.abs(two - one).max() <= tol * max(1.0, np.abs(x).max())
+        np.testing.assert_allclose(np.linalg.norm(one, axis=-1), np.linalg.norm(x, axis=-1), rtol=1e-5 if dtype == np.float32 else 1e-12)
+    np.testing.assert_array_equal(O.rope_rotate(x, np.zeros(T, dtype=np.int64), theta, layout), x)
+
+
+def test_rope_relative_property():
+    """<R(m)q, R(n)k> depends on m-n only (the reason position recovery is possible)."""
+    rng = np.random.default_rng(2)
+    q = rng.standard_normal((1, 1, 128))
+    k = rng.standard_normal((1, 1, 128))
+    def dot(m, n):
+        return float((O.rope_rotate(q, np.array([m]), 5e5) * O.rope_rotate(k, np.array([n]), 5e5)).sum())
+    assert abs(dot(700, 650) - dot(50, 0)) < 1e-9
+    assert abs(dot(32000, 31000) - dot(1000, 0)) < 1e-9
+    assert abs(dot(50, 0) - dot(51, 0)) > 1e-6
+
+
+def test_rope_frequencies_definition():
+    th = O.rope_frequencies(128, 10000.0)
+    assert th.shape == (64,)
+    assert th[0] == 1.0
+    assert abs(th[32] - 10000.0 ** (-0.5)) < 1e-15
+    assert abs(th[63] - 10000.0 ** (-126.0 / 128.0)) < 1e-15
+
+
+def test_position_recovery_offsets_and_value_copy():
+    m = W.TINY_GQA
+    model = oracle_model(m)
+    lens = (5, 1, 9)
+    ks, vs = zip(*[W.make_cache_like(m, t, 0, c) for c, t in enumerate(lens)])
+    offs = (0, 5, 6)
+    Kf, Vf = O.position_recovery(ks, vs, offs, 17, model)
+    for c, (o, t) in enumerate(zip(offs, lens)):
+        np.testing.assert_array_equal(Vf[:, o:o + t], vs[c])
+        # rotating by the offset == encoding un-rotated keys directly at the global position
+        for l in range(m.n_layers):
+            raw = O.rope_rotate(ks[c][l].astype(np.float64), -np.arange(t), m.rope_theta)  # strip local position
+            direct = O.rope_rotate(raw, o + np.arange(t), m.rope_theta)
+            np.testing.assert_allclose(Kf[l, o:o + t], direct, atol=1e-9)
+    np.testing.assert_array_equal(Kf[:, 0:5], ks[0])  # offset 0: identity
+    assert not Kf[:, 15:].any() and not Vf[:, 15:].any()
+
+
+# ------------------------------------------------------------------ small building blocks against library routines
+
+
+def test_round_bf16_matches_torch():
+    rng = np.random.default_rng(3)
+    x = np.concatenate([rng.standard_normal(4096) * 3, [0.0, -0.0, 1.0, 1.00390625, 1.01171875, 65504.0, 1e-30]]).astype(np.float32)
+    ref = torch.from_numpy(x).to(torch.bfloat16).to(torch.float32).numpy()
+    np.testing.assert_array_equal(O.round_bf16(x), ref)
+    np.testing.assert_array_equal(O.round_bf16(x.astype(np.float64)), ref.astype(np.float64))
+
+
+def test_block_pieces_match_torch():
+    rng = np.random.default_rng(4)
+    x = rng.standard_normal((7, 64))
+    g = rng.standard_normal(64)
+    ref = torch.nn.functional.rms_norm(torch.from_numpy(x), (64,), torch.from_numpy(g), eps=1e-5).numpy()
+    np.testing.assert_allclose(O.rmsnorm(x, g, 1e-5), ref, atol=1e-12)
+    np.testing.assert_allclose(O.silu(x), torch.nn.functional.silu(torch.from_numpy(x)).numpy(), atol=1e-12)
+
+
+def test_attention_matches_torch_sdpa_mha_and_gqa():
+    """Hq == Hkv reduces to textbook multi-head attention; GQA to repeated KV heads."""
+    rng = np.random.default_rng(5)
+    for Hq, Hkv, D in ((4, 4, 64), (8, 2, 128), (7, 1, 128)):
+        model = O.Model(1, Hq * D, Hq, Hkv, D, 128)
+        n = 37
+        q = rng.standard_normal((n, Hq, D))
+        K = rng.standard_normal((n, Hkv, D))
+        V = rng.standard_normal((n, Hkv, D))
+        o, lse = O.attention_rows(q, np.arange(n), K, V, model)
+        tq = torch.from_numpy(q).permute(1, 0, 2)[None]
+        tk = torch.from_numpy(K).permute(1, 0, 2).repeat_interleave(Hq // Hkv, dim=0)[None]
+        tv = torch.from_numpy(V).permute(1, 0, 2).repeat_interleave(Hq // Hkv, dim=0)[None]
+        ref = torch.nn.functional.scaled_dot_product_attention(tq, tk, tv, is_causal=True)[0].permute(1, 0, 2).numpy()
+        np.testing.assert_allclose(o, ref, atol=1e-10)
+        # sparse rows: rows [3, 20, 36] of the same problem give the same outputs
+        rows = np.array([3, 20, 36])
+        o2, lse2 = O.attention_rows(q[rows], rows, K, V, model)
+        np.testing.assert_allclose(o2, ref[rows], atol=1e-10)
+        np.testing.assert_allclose(lse2, lse[rows], atol=1e-10)
+
+
+def test_attention_causality():
+    rng = np.random.default_rng(6)
+    model = O.Model(1, 256, 4, 2, 64, 128)
+    n = 50
+    q = rng.standard_normal((3, 4, 64))
+    pos = np.array([4, 17, 30])
+    K = rng.standard_normal((n, 2, 64))
+    V = rng.standard_normal((n, 2, 64))
+    o1, _ = O.attention_rows(q, pos, K, V, model)
+    K2, V2 = K.copy(), V.copy()
+    K2[31:] += 100.0
+    V2[31:] -= 100.0
+    o2, _ = O.attention_rows(q, pos, K2, V2, model)
+    np.testing.assert_array_equal(o1, o2)
+    K2[17] += 1.0
+    o3, _ = O.attention_rows(q, pos, K2, V2, model)
+    np.testing.assert_array_equal(o1[0], o3[0])
+    assert np.abs(o1[1] - o3[1]).max() > 0
+
+
+# ------------------------------------------------------------------ scores (Eq. 3)
+
+
+def test_scores_softmax_rows_and_mass():
+    rng = np.random.default_rng(7)
+    model = O.Model(1, 512, 8, 2, 64, 128)
+    n_ctx, nq = 90, 6
+    n = n_ctx + nq
+    K = rng.standard_normal((n, 2, 64))
+    q = rng.standard_normal((nq, 8, 64))
+    qpos = np.arange(n_ctx, n)
+    for h in range(8):
+        P = O.attention_probs(q, qpos, K, model, h)
+        np.testing.assert_allclose(P.sum(axis=1), 1.0, atol=1e-12)
+        for j in range(nq):
+            assert not P[j, n_ctx + j + 1:].any()
+    s = O.query_scores(q, qpos, K, model, 5, n_ctx)
+    assert s.shape == (n,) and not s[:5].any() and not s[n_ctx:].any()
+    # total mass = |Q|*Hq minus what the question rows put on system-prompt and question keys
+    missing = 0.0
+    for h in range(8):
+        P = O.attention_probs(q, qpos, K, model, h)
+        missing += P[:, :5].sum() + P[:, n_ctx:].sum()
+    assert abs(s.sum() + missing - nq * 8) < 1e-9
+    assert s.sum() < nq * 8
+
+
+def test_scores_single_head_single_query_is_textbook_softmax():
+    rng = np.random.default_rng(8)
+    model = O.Model(1, 64, 1, 1, 64, 128)
+    K = rng.standard_normal((21, 1, 64))
+    q = rng.standard_normal((1, 1, 64))
+    s = O.query_scores(q, np.array([20]), K, model, 0, 20)
+    logits = torch.from_numpy(K[:, 0, :] @ q[0, 0] / 8.0)
+    np.testing.assert_allclose(s[:20], torch.softmax(logits, 0).numpy()[:20], atol=1e-12)
+
+
+def test_scores_uniform_keys_closed_form():
+    """All keys equal => every visible key gets 1/(#visible): s_i = Hq * sum_j 1/(n_ctx + j + 1)."""
+    model = O.Model(1, 512, 8, 2, 64, 128)
+    n_ctx, nq = 40, 5
+    K = np.ones((n_ctx + nq, 2, 64)) * 0.3
+    q = np.random.default_rng(9).standard_normal((nq, 8, 64))
+    s = O.query_scores(q, np.arange(n_ctx, n_ctx + nq), K, model, 0, n_ctx)
+    expect = 8 * sum(1.0 / (n_ctx + j + 1) for j in range(nq))
+    np.testing.assert_allclose(s[:n_ctx], expect, rtol=1e-12)
+
+
+# ------------------------------------------------------------------ top-p (Eq. 3)
+
+
+def test_topk_bruteforce_small():
+    rng = np.random.default_rng(10)
+    for trial in range(200):
+        n = int(rng.integers(1, 40))
+        b = int(rng.integers(0, n))
+        e = int(rng.integers(b, n + 1))
+        s = rng.integers(0, 6, size=n).astype(np.float64) / 4.0  # many exact ties
+        k = int(rng.integers(0, e - b + 2))
+        got = O.topk_select(s, b, e, k)
+        # brute force: repeatedly take the best remaining (max score, then min index)
+        remaining = list(range(b, e))
+        want = []
+        for _ in range(min(k, e - b)):
+            best = remaining[0]
+            for i in remaining:
+                if s[i] > s[best]:
+                    best = i
+            want.append(best)
+            remaining.remove(best)
+        assert got.tolist() == sorted(want)
+        assert len(set(got.tolist())) == len(got)
+        if len(got) and remaining:
+            assert s[got].min() >= max(s[i] for i in remaining)
+
+
+def test_topk_edges_and_ties():
+    s = np.array([0.5, 0.5, 0.5, 0.5, 0.1])
+    assert O.topk_select(s, 0, 5, 2).tolist() == [0, 1]
+    assert O.topk_select(s, 1, 5, 2).tolist() == [1, 2]
+    assert O.topk_select(s, 0, 5, 0).tolist() == []
+    assert O.topk_select(s, 0, 5, 5).tolist() == [0, 1, 2, 3, 4]
+    assert O.topk_select(s, 0, 5, 99).tolist() == [0, 1, 2, 3, 4]
+    assert O.recompute_count(0.15, 5152, 5120) == 772
+    assert O.recompute_count(0.15, 528, 512) == 79
+    assert O.recompute_count(1.0, 528, 512) == 512
+    assert O.recompute_count(0.0, 528, 512) == 0
+    assert O.recompute_count(0.3, 10, 10) == 3  # 0.3*10 = 2.9999999999999996 in binary
+
+
+# ------------------------------------------------------------------ whole-path identities
+
+
+@pytest.fixture(scope="module")
+def tiny3():
+    m, r = W.request_for("tiny3")
+    # wider weights/embeddings than N(0, 0.02) so that later layers depend visibly on context
+    model, weights, x0, ck, cv = make_request(m, r, seed=0, emb_std=1.0, w_std=0.05)
+    Kv, Vv, Xv = O.full_prefill(x0, weights, model)
+    return m, r, model, weights, x0, ck, cv, Kv, Vv, Xv
+
+
+def test_layer0_and_chunk0_exactness(tiny3):
+    m, r, model, weights, x0, ck, cv, Kv, Vv, Xv = tiny3
+    Kf, Vf = O.position_recovery(ck, cv, r.offsets, r.n, model)
+    # layer-0 K, V depend on the token alone, so recovered == full prefill for every chunk
+    np.testing.assert_allclose(Kf[0, :r.n_ctx], Kv[0, :r.n_ctx], atol=1e-10)
+    np.testing.assert_allclose(Vf[0, :r.n_ctx], Vv[0, :r.n_ctx], atol=1e-10)
+    # the chunk at offset 0 is a true causal prefix: exact at every layer
+    t0 = r.chunk_lens[0]
+    np.testing.assert_allclose(Kf[:, :t0], Kv[:, :t0], atol=1e-10)
+    np.testing.assert_allclose(Vf[:, :t0], Vv[:, :t0], atol=1e-10)
+    # later chunks at later layers are NOT exact (the missing cross-chunk attention)
+    assert np.abs(Vf[2, t0:r.n_ctx] - Vv[2, t0:r.n_ctx]).max() > 1e-3
+
+
+@pytest.mark.parametrize("select_layer", [0, 1])
+def test_ratio_one_is_full_prefill(tiny3, select_layer):
+    m, r, model, weights, x0, ck, cv, Kv, Vv, Xv = tiny3
+    res = O.fuse_request(ck, cv, x0, r.n_question, weights, model, ratio=1.0, select_layer=select_layer)
+    assert res.Re.tolist() == list(range(r.n_ctx))
+    np.testing.assert_allclose(res.K, Kv, atol=1e-9)
+    np.testing.assert_allclose(res.V, Vv, atol=1e-9)
+    np.testing.assert_allclose(res.X, Xv, atol=1e-8)
+
+
+def test_ratio_zero_is_position_recovered_concatenation(tiny3):
+    m, r, model, weights, x0, ck, cv, Kv, Vv, Xv = tiny3
+    Kf, Vf = O.position_recovery(ck, cv, r.offsets, r.n, model)
+    nc = r.n_ctx
+    res0 = O.fuse_request(ck, cv, x0, r.n_question, weights, model, ratio=0.0, select_layer=0)
+    assert res0.Re.size == 0 and res0.R.tolist() == list(range(nc, r.n))
+    # selection at layer 0 rewrites layer 0 with true values, which there equal the recovered ones
+    np.testing.assert_allclose(res0.K[0, :nc], Kf[0, :nc], atol=1e-10)
+    np.testing.assert_array_equal(res0.K[1:, :nc], Kf[1:, :nc])
+    np.testing.assert_array_equal(res0.V[1:, :nc], Vf[1:, :nc])
+    # question rows are a plain forward over the recovered cache
+    X = x0[nc:].astype(np.float64)
+    K2, V2 = Kf.copy(), Vf.copy()
+    for l in range(m.n_layers):
+        X = O.recompute_layer(X, np.arange(nc, r.n), weights[l], model, K2[l], V2[l])
+    np.testing.assert_allclose(res0.X, X, atol=1e-10)
+    np.testing.assert_allclose(res0.K[:, nc:], K2[:, nc:], atol=1e-10)
+    # selection at layer 1: layers 0 and 1 carry true values, layer 2 stays the recovered concatenation
+    res1 = O.fuse_request(ck, cv, x0, r.n_question, weights, model, ratio=0.0, select_layer=1)
+    np.testing.assert_allclose(res1.K[:2], Kv[:2], atol=1e-9)
+    np.testing.assert_array_equal(res1.K[2, :nc], Kf[2, :nc])
+    np.testing.assert_array_equal(res1.V[2, :nc], Vf[2, :nc])
+    assert np.abs(res1.V[1, :nc] - Vf[1, :nc]).max() > 1e-3
+
+
+def test_partial_ratio_properties(tiny3):
+    m, r, model, weights, x0, ck, cv, Kv, Vv, Xv = tiny3
+    Kf, Vf = O.position_recovery(ck, cv, r.offsets, r.n, model)
+    nc = r.n_ctx
+    prev, errs = None, []
+    for ratio in (0.05, 0.10, 0.15, 0.30, 0.6):
+        res = O.fuse_request(ck, cv, x0, r.n_question, weights, model, ratio=ratio, select_layer=1)
+        p = O.recompute_count(ratio, r.n, nc)
+        assert res.Re.size == p and np.all(np.diff(res.Re) > 0) and res.Re.max() < nc
+        if prev is not None:
+            assert set(prev.tolist()) <= set(res.Re.tolist())  # nested selections
+        prev = res.Re
+        # min selected >= max unselected
+        mask = np.ones(nc, bool)
+        mask[res.Re] = False
+        assert res.scores[res.Re].min() >= res.scores[:nc][mask].max()
+        # rows outside R at layers after the selection layer are untouched, bit for bit
+        np.testing.assert_array_equal(res.K[2, :nc][mask], Kf[2, :nc][mask])
+        np.testing.assert_array_equal(res.V[2, :nc][mask], Vf[2, :nc][mask])
+        # selected rows of chunk 0 recompute to the cached (exact) values
+        sel0 = res.Re[res.Re < r.chunk_lens[0]]
+        if sel0.size:
+            np.testing.assert_allclose(res.K[2, sel0], Kf[2, sel0], atol=1e-9)
+            np.testing.assert_allclose(res.V[2, sel0], Vf[2, sel0], atol=1e-9)
+        errs.append(np.abs(res.X[-r.n_question:] - Xv[-r.n_question:]).mean())
+    r1 = O.fuse_request(ck, cv, x0, r.n_question, weights, model, ratio=1.0, select_layer=1)
+    assert np.abs(r1.X[-r.n_question:] - Xv[-r.n_question:]).mean() < 1e-9
+    # soft check (unpinned claim on random weights): more recomputation does not make things worse overall
+    assert errs[-1] < errs[0]
+
+
+def test_forced_selection_and_system_prompt(tiny3):
+    m, r, model, weights, x0, ck, cv, Kv, Vv, Xv = tiny3
+    forced = np.array([130, 131, 400])
+    res = O.fuse_request(ck, cv, x0, r.n_question, weights, model, ratio=0.15, select_layer=1, forced_Re=forced)
+    assert res.R.tolist() == forced.tolist() + list(range(r.n_ctx, r.n))
+    res = O.fuse_request(ck, cv, x0, r.n_question, weights, model, ratio=0.15, select_layer=1, n_system=128)
+    assert res.Re.min() >= 128 and not res.scores[:128].any()
+    assert res.Re.size == O.recompute_count(0.15, r.n, r.n_ctx - 128)
+
+
+def test_bf16_mirrored_oracle_stays_close_to_exact(tiny3):
+    """Rounding at the storage points perturbs, but does not change, what is computed (shallow stack)."""
+    m, r, model, weights, x0, ck, cv, Kv, Vv, Xv = tiny3
+    a = O.fuse_request(ck, cv, x0, r.n_question, weights, model, ratio=0.15, select_layer=1)
+    b = O.fuse_request(ck, cv, x0, r.n_question, weights, model, ratio=0.15, select_layer=1, rnd=O.round_bf16, forced_Re=a.Re)
+    assert np.abs(a.K - b.K).max() < 0.25 and np.abs(a.K - b.K).mean() < 2e-2
+    c = O.fuse_request(ck, cv, x0, r.n_question, weights, model, ratio=0.15, select_layer=1, dtype=np.float32)
+    assert c.Re.tolist() == a.Re.tolist()
+    assert np.abs(a.K - c.K).max() < 1e-3
