@@ -1,0 +1,205 @@
+/*
+ * a3.h - C ABI of the B200 (sm_100a) hot path of attention-aware KV-cache fusion (A^3).
+ *
+ * The library fuses KV caches that were prefilled chunk by chunk (Eq. 1) into one
+ * cache for the concatenated input X = (S, D_1..D_k, Q): position recovery (Eq. 2),
+ * question->context relevance scores and top-p selection (Eq. 3), and recomputation
+ * of the selected rows [Re, Q] over the fused cache (Eq. 4, Eq. 5).
+ *
+ * Conventions
+ *  - "dev" pointers are CUDA device pointers, "host" pointers ordinary host memory.
+ *  - Tensors are bf16 (2 bytes, row-major) unless stated; scores and log-sum-exps are
+ *    fp32; indices and positions int32.
+ *  - A per-layer KV cache is [slots][n_kv_heads][head_dim]; a token's global position
+ *    is its cache slot.  Linear maps are stored [out][in] (y = x W^T).
+ *  - The caller owns every buffer (weights, chunk caches, fused cache, workspace,
+ *    outputs).  The handle borrows the weight pointers for its lifetime and owns only
+ *    its RoPE table, a small status block and tensor-map descriptors.
+ *  - Hot calls allocate nothing, do not synchronise and copy nothing between host and
+ *    device (a3_fuse_request_host excepted); all work is queued on `stream`
+ *    (a cudaStream_t passed as void*).  Calls on different streams may overlap only if
+ *    they use different workspaces.
+ *  - Return value: A3_OK or a negative a3_status.  Host-detectable problems are
+ *    rejected before any launch.  Problems only the device can see (a position outside
+ *    the cache, a non-finite score, an exhausted bounded wait) set the handle's device
+ *    status word and the kernel skips the offending access; read it with
+ *    a3_device_status.  No kernel traps.
+ *  - Supported shapes: head_dim 64 or 128; d_model, n_q_heads*head_dim,
+ *    n_kv_heads*head_dim and d_ff multiples of 128; n_q_heads a multiple of n_kv_heads.
+ *    Row counts, chunk lengths and cache lengths are arbitrary.
+ */
+#ifndef A3_H_
+#define A3_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct a3_handle a3_handle;
+typedef void* a3_stream; /* cudaStream_t */
+
+typedef enum {
+  A3_OK = 0,
+  A3_EINVAL = -1,       /* bad argument (null pointer, negative size, range) */
+  A3_EUNSUPPORTED = -2, /* shape outside the supported set */
+  A3_EWORKSPACE = -3,   /* workspace too small */
+  A3_ECUDA = -4,        /* a CUDA call failed; see a3_last_cuda_error */
+  A3_EDEVICE = -5       /* a kernel recorded a problem in the device status word */
+} a3_status;
+
+/* Device status bits (a3_device_status). */
+#define A3_DEV_BAD_POSITION 1u   /* a row position / slot was outside [0, kv_len) */
+#define A3_DEV_NONFINITE_SCORE 2u
+#define A3_DEV_WAIT_EXHAUSTED 4u /* a bounded barrier wait gave up */
+#define A3_DEV_UNSORTED_ROWS 8u  /* row positions not strictly ascending */
+
+typedef struct {
+  int n_layers, d_model, n_q_heads, n_kv_heads, head_dim, d_ff;
+  double rope_theta;  /* base of theta_i = base^(-2i/head_dim) (Position Recovery) */
+  float rms_eps;
+  int rope_layout;    /* 0: pairs (i, i+D/2); 1: pairs (2i, 2i+1) as the matrix before Eq. 2 */
+  int max_positions;  /* RoPE table rows: largest global position + 1 ever used */
+} a3_model_desc;
+
+/* One decoder block; all dev pointers to bf16.  bq/bk/bv may be NULL. */
+typedef struct {
+  const void *attn_norm, *wq, *wk, *wv, *bq, *bk, *bv, *wo, *mlp_norm, *w_gate, *w_up, *w_down;
+} a3_layer_weights;
+
+/* One precomputed chunk (Eq. 1): K_i, V_i of all layers, stored at local positions 0..len-1. */
+typedef struct {
+  const void* k_src;          /* dev, [n_layers][len][Hkv][D], layer l at k_src + l*src_layer_stride */
+  const void* v_src;          /* dev, same layout */
+  uint64_t src_layer_stride;  /* bytes between consecutive layers of this chunk */
+  int32_t len;                /* tokens in the chunk */
+  int32_t dst_offset;         /* first slot of the chunk in the fused cache (o_c) */
+  int32_t delta;              /* rotation to apply: global minus stored position (= dst_offset for local storage) */
+  int32_t reserved;
+} a3_chunk_ref;
+
+/* One fusion request.  Slots [0, n_ctx) are the chunks in input order, [n_ctx, n_ctx+n_question)
+ * the question.  Slots [0, n_system) (a system prompt) are attendable but never candidates. */
+typedef struct {
+  const a3_chunk_ref* chunks; /* dev array [n_chunks] */
+  int32_t n_chunks, max_chunk_len;
+  int32_t n_ctx, n_question, n_system;
+  int32_t select_layer;       /* layer whose true Q/K give the scores (paper: 1) */
+  int32_t n_recompute;        /* p = |Re| (a3_recompute_count) */
+  int32_t reserved;
+  const void* x0;             /* dev [n][d_model]: embeddings of the whole input */
+  void* k_fused;              /* dev [n_layers][n][Hkv][D], layer l at + l*layer_stride */
+  void* v_fused;
+  uint64_t layer_stride;      /* bytes */
+  const int32_t* forced_re;   /* dev [n_recompute] ascending, or NULL: replaces the selection */
+  int32_t* rows_out;          /* dev [n_recompute + n_question]: R = Re (ascending) then question slots */
+  float* scores_out;          /* dev [n]: s(d_i) on candidates, 0 elsewhere */
+  void* x_out;                /* dev [n_recompute + n_question][d_model]: final hidden rows of R */
+} a3_request;
+
+/* Host buffers for a3_fuse_request_host (pinned memory recommended). */
+typedef struct {
+  const void* const* chunk_k; /* host array [n_chunks] of host pointers, each [n_layers][len][Hkv][D] */
+  const void* const* chunk_v;
+  const int32_t* chunk_len;   /* host [n_chunks] */
+  const void* x0;             /* host [n][d_model] */
+  int32_t* rows_out;          /* host [n_recompute + n_question] */
+  void* x_out;                /* host [n_recompute + n_question][d_model] */
+} a3_host_io;
+
+/* ---- lifetime ---------------------------------------------------------------------- */
+
+/* Creates a handle on the current device: checks the shape, borrows `layers` (host array
+ * [n_layers] of dev pointers, copied), builds the fp32 cos/sin table [max_positions][D/2]
+ * from float64 angles.  Allocates; not a hot call. */
+int a3_create(a3_handle** out, const a3_model_desc* model, const a3_layer_weights* layers);
+void a3_destroy(a3_handle* h);
+
+/* Bytes of workspace a3_recompute_layer needs for max_rows rows (also enough for
+ * a3_query_scores / a3_topk_select on caches up to max_rows slots). */
+size_t a3_layer_workspace_bytes(const a3_handle* h, int max_rows);
+/* Bytes of workspace a3_fuse_request needs for an input of n slots (chunks + question). */
+size_t a3_request_workspace_bytes(const a3_handle* h, int n);
+/* Additional device staging bytes a3_fuse_request_host needs. */
+size_t a3_host_staging_bytes(const a3_handle* h, int n_ctx, int n);
+
+/* p = min(n_candidates, floor(ratio * n + 1e-9)): the size of Re (Eq. 3, p = r n). Host only. */
+int a3_recompute_count(double ratio, int n, int n_candidates);
+
+/* ---- the steps --------------------------------------------------------------------- */
+
+/* Position recovery (Eq. 2): for layers [layer_begin, layer_end), every chunk c, token t:
+ *   k_fused[l][dst_offset+t] = R(delta) k_src[l][t]   (rotation per head, fp32 arithmetic)
+ *   v_fused[l][dst_offset+t] = v_src[l][t]
+ * chunks: dev array; max_chunk_len >= every len (host copy of the largest length, sizes the grid).
+ * Fused layer l lives at k_fused + l*layer_stride bytes. */
+int a3_rope_rerotate(const a3_handle* h, const a3_chunk_ref* chunks, int n_chunks, int max_chunk_len,
+                     void* k_fused, void* v_fused, uint64_t layer_stride, int layer_begin, int layer_end,
+                     a3_stream stream);
+
+/* Relevance scores (Eq. 3): scores[i] = sum over question rows j and query heads h of
+ * Softmax_row(q_{j,h} K^T / sqrt(D))[i] for i in [cand_begin, cand_end), 0 for other i < kv_len.
+ * Each softmax row runs over slots 0..q_pos[j].  q_rows: dev [nq][Hq][D], already rotated;
+ * k_layer: dev [kv_len][Hkv][D].  lse: dev [nq][Hq] natural-log row log-sum-exps of the scaled
+ * logits (as a3_recompute_layer emits) or NULL, in which case a statistics pass runs first.
+ * The result is deterministic (fixed summation order). */
+int a3_query_scores(const a3_handle* h, const void* q_rows, const int32_t* q_pos, int nq, const void* k_layer,
+                    int kv_len, int cand_begin, int cand_end, const float* lse, float* scores, void* ws,
+                    size_t ws_bytes, a3_stream stream);
+
+/* Selection (Eq. 3, Re = top_p(s)): the k slots of [cand_begin, cand_end) with the largest score;
+ * ties go to the lower slot; idx_out (dev [k]) is ascending.  k is clamped to the candidate count. */
+int a3_topk_select(const a3_handle* h, const float* scores, int cand_begin, int cand_end, int k,
+                   int32_t* idx_out, a3_stream stream);
+
+/* One decoder layer for the carried rows (Eq. 5; Eq. 4 at the selection layer; the whole block
+ * when the rows are all of 0..n-1): RMSNorm, QKV (+bias), RoPE of q and k at pos, k/v written to
+ * cache rows pos BEFORE the attention, causal attention over slots 0..pos[m], output projection +
+ * residual, RMSNorm, SwiGLU MLP + residual.  x_rows: dev [M][d_model], in/out.  pos: dev [M],
+ * strictly ascending, < kv_len.  k_layer/v_layer: this layer's cache, dev [kv_len][Hkv][D].
+ * lse_out: dev [M][Hq] or NULL. */
+int a3_recompute_layer(const a3_handle* h, int layer, void* x_rows, const int32_t* pos, int M, void* k_layer,
+                       void* v_layer, int kv_len, float* lse_out, void* ws, size_t ws_bytes, a3_stream stream);
+
+/* Scatter (Eq. 5, K'_cat[Re,Q] <- ..., V_cat[Re,Q] <- ...): cache row slots[m] = row m.
+ * k_rows/v_rows: dev [M][Hkv][D]; slots: dev [M], each in [0, kv_len). */
+int a3_scatter_kv(const a3_handle* h, const void* k_rows, const void* v_rows, const int32_t* slots, int M,
+                  void* k_layer, void* v_layer, int kv_len, a3_stream stream);
+
+/* Row gather X[R] (Eq. 4, Q_true[Re, Q]): dst[m] = src[rows[m]], rows of `width` bf16 elements. */
+int a3_gather_rows(const a3_handle* h, const void* src, int n_src, const int32_t* rows, int M, int width,
+                   void* dst, a3_stream stream);
+
+/* The whole request (Method, "Attention-Aware Accurate Fusion"): position recovery of all layers,
+ * the leading full blocks 0..select_layer-1 over all n rows, true K/V of all rows and question
+ * queries at select_layer, scores, selection, then layers select_layer..L-1 on rows R only.
+ * Fills the fused cache in place, rows_out, scores_out, x_out. */
+int a3_fuse_request(const a3_handle* h, const a3_request* req, void* ws, size_t ws_bytes, a3_stream stream);
+
+/* Several independent requests on one stream (batched serving). */
+int a3_fuse_batch(const a3_handle* h, const a3_request* reqs, int n_requests, void* ws, size_t ws_bytes,
+                  a3_stream stream);
+
+/* a3_fuse_request with the chunk caches and embeddings in HOST memory: copies them to `staging`
+ * (dev, a3_host_staging_bytes), builds the chunk descriptors, fuses, copies rows_out and x_out
+ * back to the host and waits for the stream.  req->chunks, req->x0 are ignored (taken from io);
+ * the fused cache and scores stay on the device. */
+int a3_fuse_request_host(const a3_handle* h, const a3_request* req, const a3_host_io* io, void* staging,
+                         size_t staging_bytes, void* ws, size_t ws_bytes, a3_stream stream);
+
+/* ---- diagnostics -------------------------------------------------------------------- */
+
+/* Waits for `stream`, reads and clears the device status word (A3_DEV_* bits). */
+int a3_device_status(const a3_handle* h, uint32_t* bits_out, a3_stream stream);
+const char* a3_status_string(int status);
+/* cudaError_t of the last failed CUDA call made by this library on the calling thread. */
+int a3_last_cuda_error(void);
+/* Number of kernel launches this library has queued since the counter was last reset (host counter). */
+uint64_t a3_launch_count(int reset);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* A3_H_ */

@@ -255,11 +255,14 @@ def recompute_layer(
     X: [M][d] hidden rows at global positions pos (ascending; position = cache slot).
     K, V: this layer's fused cache [n][Hkv][D], updated IN PLACE at rows pos before
     the attention is taken.  Returns the rows' hidden state after the block.
-    `rnd` is applied at the points where a bf16 pipeline stores a tensor.
+    `rnd` is applied at the points where a bf16 pipeline stores a tensor
+    (norm outputs, q/k/v after RoPE, attention output, hidden state after each
+    residual, the SwiGLU product); with the default identity nothing is rounded.
     """
     M = X.shape[0]
     a = rnd(rmsnorm(X, w.attn_norm, model.rms_eps))
-    q, k, v = project_qkv(a, w, model, pos, rnd)
+    q_e, k_e, v_e = project_qkv(a, w, model, pos, identity)  # exact values, before storage rounding
+    q, k, v = rnd(q_e), rnd(k_e), rnd(v_e)
     K[pos] = k
     V[pos] = v
     o, lse = attention_rows(q, pos, K, V, model)
@@ -267,9 +270,12 @@ def recompute_layer(
     X1 = rnd(X + o @ w.wo.astype(X.dtype).T)
     a2 = rnd(rmsnorm(X1, w.mlp_norm, model.rms_eps))
     hmid = rnd(silu(a2 @ w.w_gate.astype(X.dtype).T) * (a2 @ w.w_up.astype(X.dtype).T))
-    X2 = rnd(X1 + hmid @ w.w_down.astype(X.dtype).T)
+    X2_e = X1 + hmid @ w.w_down.astype(X.dtype).T
+    X2 = rnd(X2_e)
     if return_parts:
-        return X2, dict(a=a, q=q, k=k, v=v, o=o, lse=lse, x_attn=X1, a2=a2, h=hmid)
+        # *_exact: the same quantities before the final storage rounding (what a bf16 result is compared with)
+        return X2, dict(a=a, q=q, k=k, v=v, o=o, lse=lse, x_attn=X1, a2=a2, h=hmid,
+                        q_exact=q_e, k_exact=k_e, v_exact=v_e, x_exact=X2_e)
     return X2
 
 

@@ -1,0 +1,421 @@
+// Handle lifetime, workspace carving and the orchestration of the fusion request (host code only).
+#include <math.h>
+#include <stdlib.h>
+#include <string.h>
+
+#include "a3_internal.cuh"
+
+namespace a3 {
+int build_rope_table(float2* tab, int max_pos, int D, double base, cudaStream_t st);
+
+// Workspace of one a3_recompute_layer call, carved from a caller-provided buffer.
+struct LayerWs {
+  bf16 *a, *q, *o, *hmid;
+  float* lse;
+  size_t bytes;
+};
+static LayerWs carve_layer_ws(const a3_model_desc& m, int rows, void* base) {
+  LayerWs w;
+  char* p = (char*)base;
+  size_t off = 0;
+  auto take = [&](size_t b) {
+    char* r = p ? p + off : nullptr;
+    off += align_up(b, 256);
+    return r;
+  };
+  const size_t R = (size_t)(rows > 0 ? rows : 1);
+  w.a = (bf16*)take(R * m.d_model * 2);
+  w.q = (bf16*)take(R * m.n_q_heads * m.head_dim * 2);
+  w.o = (bf16*)take(R * m.n_q_heads * m.head_dim * 2);
+  w.hmid = (bf16*)take(R * m.d_ff * 2);
+  w.lse = (float*)take(R * m.n_q_heads * 4);
+  w.bytes = off;
+  return w;
+}
+
+struct RequestWs {
+  bf16* x_all;
+  int32_t* all_pos;
+  float* lse_q;
+  void* layer;
+  size_t bytes;
+};
+static RequestWs carve_request_ws(const a3_model_desc& m, int n, void* base) {
+  RequestWs w;
+  char* p = (char*)base;
+  size_t off = 0;
+  auto take = [&](size_t b) {
+    char* r = p ? p + off : nullptr;
+    off += align_up(b, 256);
+    return r;
+  };
+  const size_t N = (size_t)(n > 0 ? n : 1);
+  w.x_all = (bf16*)take(N * m.d_model * 2);
+  w.all_pos = (int32_t*)take(N * 4);
+  w.lse_q = (float*)take(N * m.n_q_heads * 4);
+  w.layer = take(carve_layer_ws(m, n, nullptr).bytes);
+  w.bytes = off;
+  return w;
+}
+}  // namespace a3
+
+using namespace a3;
+
+extern "C" const char* a3_status_string(int s) {
+  switch (s) {
+    case A3_OK: return "ok";
+    case A3_EINVAL: return "invalid argument";
+    case A3_EUNSUPPORTED: return "unsupported shape";
+    case A3_EWORKSPACE: return "workspace too small";
+    case A3_ECUDA: return "CUDA call failed";
+    case A3_EDEVICE: return "device status word set";
+    default: return "unknown status";
+  }
+}
+
+extern "C" int a3_last_cuda_error(void) { return g_last_cuda_error; }
+
+extern "C" uint64_t a3_launch_count(int reset) {
+  uint64_t v = g_launches;
+  if (reset) g_launches = 0;
+  return v;
+}
+
+extern "C" int a3_recompute_count(double ratio, int n, int n_candidates) {
+  if (n_candidates <= 0 || n <= 0 || !(ratio > 0.0)) return 0;
+  double p = floor(ratio * (double)n + 1e-9);
+  if (p > (double)n_candidates) return n_candidates;
+  return (int)p;
+}
+
+extern "C" int a3_create(a3_handle** out, const a3_model_desc* m, const a3_layer_weights* layers) {
+  if (!out || !m || !layers) return A3_EINVAL;
+  *out = nullptr;
+  if (m->n_layers <= 0 || m->d_model <= 0 || m->n_q_heads <= 0 || m->n_kv_heads <= 0 || m->d_ff <= 0 ||
+      m->max_positions <= 0 || !(m->rope_theta > 0.0) || !(m->rms_eps >= 0.f))
+    return A3_EINVAL;
+  if (m->head_dim != 64 && m->head_dim != 128) return A3_EUNSUPPORTED;
+  if (m->rope_layout != 0 && m->rope_layout != 1) return A3_EUNSUPPORTED;
+  if (m->n_q_heads % m->n_kv_heads) return A3_EUNSUPPORTED;
+  if (m->d_model % 128 || (m->n_q_heads * m->head_dim) % 128 || (m->n_kv_heads * m->head_dim) % 128 || m->d_ff % 128)
+    return A3_EUNSUPPORTED;
+  for (int l = 0; l < m->n_layers; ++l) {
+    const a3_layer_weights& w = layers[l];
+    const void* req[] = {w.attn_norm, w.wq, w.wk, w.wv, w.wo, w.mlp_norm, w.w_gate, w.w_up, w.w_down};
+    for (const void* p : req)
+      if (!p || ((uintptr_t)p & 15)) return A3_EINVAL;
+    const void* opt[] = {w.bq, w.bk, w.bv};
+    for (const void* p : opt)
+      if (p && ((uintptr_t)p & 15)) return A3_EINVAL;
+  }
+  a3_handle* h = (a3_handle*)calloc(1, sizeof(a3_handle));
+  if (!h) return A3_EINVAL;
+  h->m = *m;
+  h->layers = (a3_layer_weights*)malloc(sizeof(a3_layer_weights) * m->n_layers);
+  memcpy(h->layers, layers, sizeof(a3_layer_weights) * m->n_layers);
+  cudaError_t e = cudaGetDevice(&h->device);
+  if (e == cudaSuccess) e = cudaDeviceGetAttribute(&h->sm_count, cudaDevAttrMultiProcessorCount, h->device);
+  if (e == cudaSuccess) e = cudaMalloc((void**)&h->rope_tab, (size_t)m->max_positions * (m->head_dim / 2) * sizeof(float2));
+  if (e == cudaSuccess) e = cudaMalloc((void**)&h->dev_status, 256);
+  if (e == cudaSuccess) e = cudaMemset(h->dev_status, 0, 256);
+  if (e != cudaSuccess) {
+    a3_destroy(h);
+    return cuda_fail(e);
+  }
+  int s = build_rope_table(h->rope_tab, m->max_positions, m->head_dim, m->rope_theta, 0);
+  if (s == A3_OK) {
+    e = cudaStreamSynchronize(0);
+    if (e != cudaSuccess) s = cuda_fail(e);
+  }
+  if (s != A3_OK) {
+    a3_destroy(h);
+    return s;
+  }
+  *out = h;
+  return A3_OK;
+}
+
+extern "C" void a3_destroy(a3_handle* h) {
+  if (!h) return;
+  if (h->rope_tab) cudaFree(h->rope_tab);
+  if (h->dev_status) cudaFree(h->dev_status);
+  free(h->layers);
+  free(h);
+}
+
+extern "C" size_t a3_layer_workspace_bytes(const a3_handle* h, int max_rows) {
+  if (!h || max_rows < 0) return 0;
+  return carve_layer_ws(h->m, max_rows, nullptr).bytes;
+}
+
+extern "C" size_t a3_request_workspace_bytes(const a3_handle* h, int n) {
+  if (!h || n < 0) return 0;
+  return carve_request_ws(h->m, n, nullptr).bytes;
+}
+
+extern "C" int a3_device_status(const a3_handle* h, uint32_t* bits_out, a3_stream stream) {
+  if (!h || !bits_out) return A3_EINVAL;
+  cudaStream_t st = (cudaStream_t)stream;
+  A3_CUDA(cudaStreamSynchronize(st));
+  uint32_t v = 0;
+  A3_CUDA(cudaMemcpy(&v, h->dev_status, 4, cudaMemcpyDeviceToHost));
+  if (v) A3_CUDA(cudaMemset(h->dev_status, 0, 4));
+  *bits_out = v;
+  return A3_OK;
+}
+
+// ------------------------------------------------------------------ one layer (Eq. 5)
+namespace a3 {
+// rows_kv: rows whose k/v are projected and written to the cache (all M); rows_q: q is projected for rows
+// [q_first, M) only (the selection layer needs the question rows' queries, not the context rows').
+static int qkv_project(const a3_handle* h, int layer, const bf16* a, const int32_t* pos, int M, int q_first, bf16* q_out,
+                       bf16* kc, bf16* vc, int kv_len, cudaStream_t st) {
+  const a3_model_desc& m = h->m;
+  const a3_layer_weights& w = h->layers[layer];
+  const int qd = m.n_q_heads * m.head_dim, kvd = m.n_kv_heads * m.head_dim;
+  GemmArgs g{};
+  g.K = m.d_model;
+  g.q_out = q_out;
+  g.k_cache = kc;
+  g.v_cache = vc;
+  g.kv_len = kv_len;
+  if (q_first == 0) {
+    g.A = a;
+    g.M = M;
+    g.pos = pos;
+    g.nseg = 3;
+    g.seg[0] = {(const bf16*)w.wq, (const bf16*)w.bq, qd, 0};
+    g.seg[1] = {(const bf16*)w.wk, (const bf16*)w.bk, kvd, 1};
+    g.seg[2] = {(const bf16*)w.wv, (const bf16*)w.bv, kvd, 2};
+    return gemm_bf16(h, EPI_QKV, g, st);
+  }
+  g.A = a;
+  g.M = M;
+  g.pos = pos;
+  g.nseg = 2;
+  g.seg[0] = {(const bf16*)w.wk, (const bf16*)w.bk, kvd, 1};
+  g.seg[1] = {(const bf16*)w.wv, (const bf16*)w.bv, kvd, 2};
+  A3_TRY(gemm_bf16(h, EPI_QKV, g, st));
+  if (q_first < M) {
+    g.A = a + (size_t)q_first * m.d_model;
+    g.M = M - q_first;
+    g.pos = pos + q_first;
+    g.nseg = 1;
+    g.seg[0] = {(const bf16*)w.wq, (const bf16*)w.bq, qd, 0};
+    A3_TRY(gemm_bf16(h, EPI_QKV, g, st));
+  }
+  return A3_OK;
+}
+
+static int recompute_layer_impl(const a3_handle* h, int layer, bf16* x, const int32_t* pos, int M, bf16* kc, bf16* vc,
+                                int kv_len, float* lse_out, const LayerWs& w, cudaStream_t st) {
+  const a3_model_desc& m = h->m;
+  const a3_layer_weights& lw = h->layers[layer];
+  const int qd = m.n_q_heads * m.head_dim;
+  A3_TRY(rmsnorm_rows(x, (const bf16*)lw.attn_norm, m.rms_eps, M, m.d_model, w.a, st));
+  A3_TRY(qkv_project(h, layer, w.a, pos, M, 0, w.q, kc, vc, kv_len, st));
+  A3_TRY(attention_rows(h, w.q, pos, M, kc, vc, kv_len, w.o, lse_out, st));
+  GemmArgs g{};
+  g.A = w.o;
+  g.M = M;
+  g.K = qd;
+  g.nseg = 1;
+  g.seg[0] = {(const bf16*)lw.wo, nullptr, m.d_model, 0};
+  g.C = x;
+  g.ldc = m.d_model;
+  A3_TRY(gemm_bf16(h, EPI_RESIDUAL, g, st));
+  A3_TRY(rmsnorm_rows(x, (const bf16*)lw.mlp_norm, m.rms_eps, M, m.d_model, w.a, st));
+  GemmArgs u{};
+  u.A = w.a;
+  u.M = M;
+  u.K = m.d_model;
+  u.nseg = 1;
+  u.seg[0] = {(const bf16*)lw.w_gate, nullptr, m.d_ff, 0};
+  u.B2 = (const bf16*)lw.w_up;
+  u.C = w.hmid;
+  u.ldc = m.d_ff;
+  A3_TRY(gemm_bf16(h, EPI_SWIGLU, u, st));
+  GemmArgs d{};
+  d.A = w.hmid;
+  d.M = M;
+  d.K = m.d_ff;
+  d.nseg = 1;
+  d.seg[0] = {(const bf16*)lw.w_down, nullptr, m.d_model, 0};
+  d.C = x;
+  d.ldc = m.d_model;
+  A3_TRY(gemm_bf16(h, EPI_RESIDUAL, d, st));
+  return A3_OK;
+}
+}  // namespace a3
+
+extern "C" int a3_recompute_layer(const a3_handle* h, int layer, void* x_rows, const int32_t* pos, int M, void* k_layer,
+                                  void* v_layer, int kv_len, float* lse_out, void* ws, size_t ws_bytes, a3_stream stream) {
+  if (!h || layer < 0 || layer >= h->m.n_layers || M < 0 || kv_len < 0) return A3_EINVAL;
+  if (M == 0) return A3_OK;
+  if (!x_rows || !pos || !k_layer || !v_layer || !ws) return A3_EINVAL;
+  if (kv_len > h->m.max_positions || M > kv_len) return A3_EINVAL;
+  if (((uintptr_t)x_rows | (uintptr_t)k_layer | (uintptr_t)v_layer | (uintptr_t)ws) & 15) return A3_EINVAL;
+  LayerWs w = carve_layer_ws(h->m, M, ws);
+  if (w.bytes > ws_bytes) return A3_EWORKSPACE;
+  cudaStream_t st = (cudaStream_t)stream;
+  A3_TRY(check_rows(h, pos, M, kv_len, st));
+  return recompute_layer_impl(h, layer, (bf16*)x_rows, pos, M, (bf16*)k_layer, (bf16*)v_layer, kv_len, lse_out, w, st);
+}
+
+// ------------------------------------------------------------------ scores (Eq. 3)
+extern "C" int a3_query_scores(const a3_handle* h, const void* q_rows, const int32_t* q_pos, int nq, const void* k_layer,
+                               int kv_len, int cand_begin, int cand_end, const float* lse, float* scores, void* ws,
+                               size_t ws_bytes, a3_stream stream) {
+  if (!h || nq < 0 || kv_len < 0 || cand_begin < 0 || cand_end < cand_begin || cand_end > kv_len) return A3_EINVAL;
+  if (kv_len == 0) return A3_OK;
+  if (!scores || !k_layer) return A3_EINVAL;
+  if (nq > 0 && (!q_rows || !q_pos)) return A3_EINVAL;
+  if (((uintptr_t)q_rows | (uintptr_t)k_layer) & 15) return A3_EINVAL;
+  cudaStream_t st = (cudaStream_t)stream;
+  if (!lse && nq > 0) {
+    const size_t need = align_up((size_t)nq * h->m.n_q_heads * 4, 256);
+    if (!ws || ws_bytes < need) return A3_EWORKSPACE;
+    A3_TRY(attention_rows(h, (const bf16*)q_rows, q_pos, nq, (const bf16*)k_layer, (const bf16*)k_layer, kv_len, nullptr,
+                          (float*)ws, st));
+    lse = (const float*)ws;
+  }
+  return scores_pass(h, (const bf16*)q_rows, q_pos, nq, (const bf16*)k_layer, kv_len, cand_begin, cand_end, lse, scores, st);
+}
+
+// ------------------------------------------------------------------ the whole request
+extern "C" int a3_fuse_request(const a3_handle* h, const a3_request* r, void* ws, size_t ws_bytes, a3_stream stream) {
+  if (!h || !r || !ws) return A3_EINVAL;
+  const a3_model_desc& m = h->m;
+  if (r->n_ctx < 0 || r->n_question < 0 || r->n_system < 0 || r->n_system > r->n_ctx || r->n_chunks < 0) return A3_EINVAL;
+  const int n = r->n_ctx + r->n_question;
+  if (n == 0) return A3_OK;
+  if (n > m.max_positions) return A3_EINVAL;
+  if (r->select_layer < 0 || r->select_layer >= m.n_layers) return A3_EINVAL;
+  const int n_cand = r->n_ctx - r->n_system;
+  if (r->n_recompute < 0 || r->n_recompute > n_cand) return A3_EINVAL;
+  if (!r->x0 || !r->k_fused || !r->v_fused || !r->rows_out || !r->scores_out || !r->x_out) return A3_EINVAL;
+  if (r->n_chunks > 0 && !r->chunks) return A3_EINVAL;
+  const size_t layer_bytes = (size_t)n * m.n_kv_heads * m.head_dim * 2;
+  if (r->layer_stride < layer_bytes || (r->layer_stride & 15)) return A3_EINVAL;
+  if (((uintptr_t)r->x0 | (uintptr_t)r->k_fused | (uintptr_t)r->v_fused | (uintptr_t)r->x_out | (uintptr_t)ws) & 15) return A3_EINVAL;
+  RequestWs w = carve_request_ws(m, n, ws);
+  if (w.bytes > ws_bytes) return A3_EWORKSPACE;
+  cudaStream_t st = (cudaStream_t)stream;
+  const int p = r->n_recompute, nq = r->n_question, M = p + nq, ls = r->select_layer;
+  LayerWs lw = carve_layer_ws(m, n, w.layer);
+  auto kl = [&](int l) { return (bf16*)((char*)r->k_fused + (size_t)l * r->layer_stride); };
+  auto vl = [&](int l) { return (bf16*)((char*)r->v_fused + (size_t)l * r->layer_stride); };
+
+  // position recovery of every layer in one launch (Eq. 2)
+  A3_TRY(a3_rope_rerotate(h, r->chunks, r->n_chunks, r->max_chunk_len, r->k_fused, r->v_fused, r->layer_stride, 0,
+                          m.n_layers, stream));
+  // leading full blocks: the whole input through layers 0..select_layer-1
+  A3_CUDA(cudaMemcpyAsync(w.x_all, r->x0, (size_t)n * m.d_model * 2, cudaMemcpyDeviceToDevice, st));
+  A3_TRY(iota_rows(w.all_pos, 0, n, st));
+  for (int l = 0; l < ls; ++l)
+    A3_TRY(recompute_layer_impl(h, l, w.x_all, w.all_pos, n, kl(l), vl(l), n, nullptr, lw, st));
+  // selection layer: true K, V for all rows, queries of the question rows, scores, Re (Eq. 3)
+  A3_TRY(rmsnorm_rows(w.x_all, (const bf16*)h->layers[ls].attn_norm, m.rms_eps, n, m.d_model, lw.a, st));
+  A3_TRY(qkv_project(h, ls, lw.a, w.all_pos, n, r->n_ctx, lw.q, kl(ls), vl(ls), n, st));
+  A3_CUDA(cudaMemsetAsync(r->scores_out, 0, (size_t)n * 4, st));
+  if (nq > 0) {
+    A3_TRY(attention_rows(h, lw.q, w.all_pos + r->n_ctx, nq, kl(ls), vl(ls), n, nullptr, w.lse_q, st));
+    A3_TRY(scores_pass(h, lw.q, w.all_pos + r->n_ctx, nq, kl(ls), n, r->n_system, r->n_ctx, w.lse_q, r->scores_out, st));
+  }
+  if (p > 0) {
+    if (r->forced_re) A3_CUDA(cudaMemcpyAsync(r->rows_out, r->forced_re, (size_t)p * 4, cudaMemcpyDeviceToDevice, st));
+    else A3_TRY(a3_topk_select(h, r->scores_out, r->n_system, r->n_ctx, p, r->rows_out, stream));
+  }
+  A3_TRY(iota_rows(r->rows_out + p, r->n_ctx, nq, st));
+  if (M == 0) return A3_OK;
+  A3_TRY(check_rows(h, r->rows_out, M, n, st));
+  A3_TRY(a3_gather_rows(h, w.x_all, n, r->rows_out, M, m.d_model, r->x_out, stream));
+  // layers select_layer..L-1 on rows [Re, Q] only (Eq. 4, Eq. 5)
+  for (int l = ls; l < m.n_layers; ++l)
+    A3_TRY(recompute_layer_impl(h, l, (bf16*)r->x_out, r->rows_out, M, kl(l), vl(l), n, nullptr, lw, st));
+  return A3_OK;
+}
+
+extern "C" int a3_fuse_batch(const a3_handle* h, const a3_request* reqs, int n_requests, void* ws, size_t ws_bytes,
+                             a3_stream stream) {
+  if (!h || n_requests < 0 || (n_requests > 0 && !reqs)) return A3_EINVAL;
+  for (int i = 0; i < n_requests; ++i) A3_TRY(a3_fuse_request(h, &reqs[i], ws, ws_bytes, stream));
+  return A3_OK;
+}
+
+// ------------------------------------------------------------------ host-buffer entry
+extern "C" size_t a3_host_staging_bytes(const a3_handle* h, int n_ctx, int n) {
+  if (!h || n_ctx < 0 || n < n_ctx) return 0;
+  const a3_model_desc& m = h->m;
+  const size_t row = (size_t)m.n_kv_heads * m.head_dim * 2;
+  // chunk K and V of all layers, embeddings, descriptors (one per token is an upper bound on chunks)
+  return align_up(2 * (size_t)m.n_layers * n_ctx * row, 256) + align_up((size_t)n * m.d_model * 2, 256) +
+         align_up((size_t)(n_ctx + 1) * sizeof(a3_chunk_ref), 256);
+}
+
+extern "C" int a3_fuse_request_host(const a3_handle* h, const a3_request* req, const a3_host_io* io, void* staging,
+                                    size_t staging_bytes, void* ws, size_t ws_bytes, a3_stream stream) {
+  if (!h || !req || !io || !staging) return A3_EINVAL;
+  if (!io->x0 || !io->rows_out || !io->x_out) return A3_EINVAL;
+  if (req->n_chunks > 0 && (!io->chunk_k || !io->chunk_v || !io->chunk_len)) return A3_EINVAL;
+  const a3_model_desc& m = h->m;
+  const int n = req->n_ctx + req->n_question;
+  if (req->n_ctx < 0 || req->n_question < 0 || req->n_chunks < 0 || req->n_chunks > req->n_ctx + 1) return A3_EINVAL;
+  if (a3_host_staging_bytes(h, req->n_ctx, n) > staging_bytes) return A3_EWORKSPACE;
+  cudaStream_t st = (cudaStream_t)stream;
+  const size_t row = (size_t)m.n_kv_heads * m.head_dim * 2;
+  char* base = (char*)staging;
+  char* kv = base;
+  char* x0 = base + align_up(2 * (size_t)m.n_layers * req->n_ctx * row, 256);
+  a3_chunk_ref* dref = (a3_chunk_ref*)(x0 + align_up((size_t)n * m.d_model * 2, 256));
+  a3_chunk_ref* href = (a3_chunk_ref*)malloc(sizeof(a3_chunk_ref) * (req->n_chunks > 0 ? req->n_chunks : 1));
+  if (!href) return A3_EINVAL;
+  int off = 0, maxlen = 0;
+  size_t kvoff = 0;
+  for (int c = 0; c < req->n_chunks; ++c) {
+    const int len = io->chunk_len[c];
+    if (len < 0 || off + len > req->n_ctx) {
+      free(href);
+      return A3_EINVAL;
+    }
+    const size_t bytes = (size_t)m.n_layers * len * row;
+    cudaError_t e = cudaMemcpyAsync(kv + kvoff, io->chunk_k[c], bytes, cudaMemcpyHostToDevice, st);
+    if (e == cudaSuccess) e = cudaMemcpyAsync(kv + kvoff + bytes, io->chunk_v[c], bytes, cudaMemcpyHostToDevice, st);
+    if (e != cudaSuccess) {
+      free(href);
+      return cuda_fail(e);
+    }
+    href[c].k_src = kv + kvoff;
+    href[c].v_src = kv + kvoff + bytes;
+    href[c].src_layer_stride = (uint64_t)len * row;
+    href[c].len = len;
+    href[c].dst_offset = off;
+    href[c].delta = off;
+    href[c].reserved = 0;
+    kvoff += 2 * bytes;
+    off += len;
+    if (len > maxlen) maxlen = len;
+  }
+  if (off != req->n_ctx) {
+    free(href);
+    return A3_EINVAL;
+  }
+  cudaError_t e = cudaMemcpyAsync(x0, io->x0, (size_t)n * m.d_model * 2, cudaMemcpyHostToDevice, st);
+  // the descriptor array is pageable host memory: this copy returns only once it has been staged
+  if (e == cudaSuccess && req->n_chunks > 0)
+    e = cudaMemcpyAsync(dref, href, sizeof(a3_chunk_ref) * req->n_chunks, cudaMemcpyHostToDevice, st);
+  free(href);
+  if (e != cudaSuccess) return cuda_fail(e);
+  a3_request r = *req;
+  r.chunks = dref;
+  r.max_chunk_len = maxlen;
+  r.x0 = x0;
+  A3_TRY(a3_fuse_request(h, &r, ws, ws_bytes, stream));
+  const int M = r.n_recompute + r.n_question;
+  if (M > 0) {
+    A3_CUDA(cudaMemcpyAsync(io->rows_out, r.rows_out, (size_t)M * 4, cudaMemcpyDeviceToHost, st));
+    A3_CUDA(cudaMemcpyAsync(io->x_out, r.x_out, (size_t)M * m.d_model * 2, cudaMemcpyDeviceToHost, st));
+  }
+  A3_CUDA(cudaStreamSynchronize(st));
+  return A3_OK;
+}

@@ -1,0 +1,163 @@
+// Internal declarations shared by the translation units of liba3.so (not part of the C ABI).
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "a3.h"
+
+typedef __nv_bfloat16 bf16;
+
+struct a3_handle {
+  a3_model_desc m;
+  a3_layer_weights* layers;  // host copy [n_layers]
+  float2* rope_tab;          // dev [max_positions][D/2] (cos, sin)
+  uint32_t* dev_status;      // dev, 1 word (+ padding)
+  int device;
+  int sm_count;
+  void* tmaps;               // host-side tensor-map cache (a3_gemm_tc.cu)
+};
+
+namespace a3 {
+
+extern thread_local int g_last_cuda_error;
+extern unsigned long long g_launches;
+
+inline int cuda_fail(cudaError_t e) {
+  g_last_cuda_error = (int)e;
+  return A3_ECUDA;
+}
+#define A3_CUDA(call)                                   \
+  do {                                                  \
+    cudaError_t e_ = (call);                            \
+    if (e_ != cudaSuccess) return ::a3::cuda_fail(e_);  \
+  } while (0)
+
+// Call after every kernel launch: counts it and converts a launch error into a status.
+inline int launched() {
+  ++g_launches;
+  cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess) return cuda_fail(e);
+  return A3_OK;
+}
+#define A3_LAUNCHED()                 \
+  do {                                \
+    int s_ = ::a3::launched();        \
+    if (s_ != A3_OK) return s_;       \
+  } while (0)
+#define A3_TRY(expr)                  \
+  do {                                \
+    int s_ = (expr);                  \
+    if (s_ != A3_OK) return s_;       \
+  } while (0)
+
+inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+inline int cdiv(long long a, long long b) { return (int)((a + b - 1) / b); }
+
+// ---------------------------------------------------------------- internal step launchers
+
+// out[m] = rmsnorm(x[m]) * gain, rows of width d.
+int rmsnorm_rows(const bf16* x, const bf16* gain, float eps, int M, int d, bf16* out, cudaStream_t st);
+
+enum GemmEpilogue { EPI_RESIDUAL = 0, EPI_SWIGLU = 1, EPI_QKV = 2 };
+
+struct GemmSegment {
+  const bf16* B;     // [n][K] row-major
+  const bf16* bias;  // [n] or null
+  int n;             // columns of this segment (multiple of 128)
+  int kind;          // 0 = q, 1 = k, 2 = v (EPI_QKV only)
+};
+
+struct GemmArgs {
+  const bf16* A;  // [M][K] row-major
+  int M, K;
+  GemmSegment seg[3];
+  int nseg;
+  const bf16* B2;  // EPI_SWIGLU: the "up" matrix, same shape as seg[0].B (gate)
+  bf16* C;         // EPI_RESIDUAL: [M][N] in/out (C += A B^T); EPI_SWIGLU: [M][N] out
+  int ldc;
+  // EPI_QKV
+  bf16* q_out;      // [M][Hq*D]
+  bf16* k_cache;    // [kv_len][Hkv*D]
+  bf16* v_cache;
+  const int32_t* pos;  // [M] cache slot = RoPE position of each row
+  int kv_len;
+};
+
+// C-tile GEMM with fused epilogue on the tensor cores; all operands K-major bf16, fp32 accumulate.
+int gemm_bf16(const a3_handle* h, GemmEpilogue epi, const GemmArgs& a, cudaStream_t st);
+
+// Causal attention of M rows (at cache slots pos[m]) over a [kv_len][Hkv][D] cache.
+// q: [M][Hq][D]; o: [M][Hq][D] (may be null: statistics only); lse: [M][Hq] or null.
+int attention_rows(const a3_handle* h, const bf16* q, const int32_t* pos, int M, const bf16* k, const bf16* v,
+                   int kv_len, bf16* o, float* lse, cudaStream_t st);
+
+int scores_pass(const a3_handle* h, const bf16* q, const int32_t* q_pos, int nq, const bf16* k, int kv_len,
+                int cand_begin, int cand_end, const float* lse, float* scores, cudaStream_t st);
+
+int iota_rows(int32_t* out, int begin, int count, cudaStream_t st);
+int check_rows(const a3_handle* h, const int32_t* pos, int M, int kv_len, cudaStream_t st);
+
+}  // namespace a3
+
+// ---------------------------------------------------------------- device helpers
+#ifdef __CUDACC__
+namespace a3 {
+
+__device__ __forceinline__ float bf2f(bf16 x) { return __bfloat162float(x); }
+
+// 8 bf16 packed in a uint4 <-> 8 floats
+__device__ __forceinline__ void unpack8(const uint4& v, float* f) {
+  const __nv_bfloat162* p = reinterpret_cast<const __nv_bfloat162*>(&v);
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    float2 t = __bfloat1622float2(p[i]);
+    f[2 * i] = t.x;
+    f[2 * i + 1] = t.y;
+  }
+}
+__device__ __forceinline__ uint4 pack8(const float* f) {
+  uint4 v;
+  __nv_bfloat162* p = reinterpret_cast<__nv_bfloat162*>(&v);
+#pragma unroll
+  for (int i = 0; i < 4; ++i) p[i] = __floats2bfloat162_rn(f[2 * i], f[2 * i + 1]);
+  return v;
+}
+__device__ __forceinline__ uint32_t pack2(float a, float b) {
+  __nv_bfloat162 t = __floats2bfloat162_rn(a, b);
+  return *reinterpret_cast<uint32_t*>(&t);
+}
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void cp_async16(uint32_t dst, const void* src, bool pred) {
+  int sz = pred ? 16 : 0;
+  asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;\n" ::"r"(dst), "l"(src), "r"(sz));
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;\n" ::); }
+template <int N>
+__device__ __forceinline__ void cp_async_wait() {
+  asm volatile("cp.async.wait_group %0;\n" ::"n"(N));
+}
+
+__device__ __forceinline__ void ldmatrix_x4(uint32_t addr, uint32_t& r0, uint32_t& r1, uint32_t& r2, uint32_t& r3) {
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];\n"
+               : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3)
+               : "r"(addr));
+}
+__device__ __forceinline__ void ldmatrix_x4_trans(uint32_t addr, uint32_t& r0, uint32_t& r1, uint32_t& r2, uint32_t& r3) {
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];\n"
+               : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3)
+               : "r"(addr));
+}
+// D(16x8, fp32) += A(16x16, bf16, row) * B(16x8, bf16, col)
+__device__ __forceinline__ void mma_bf16(float* c, const uint32_t* a, uint32_t b0, uint32_t b1) {
+  asm volatile(
+      "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};\n"
+      : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+      : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+}
+
+}  // namespace a3
+#endif

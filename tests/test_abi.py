@@ -1,0 +1,61 @@
+"""Host-only checks of the C-ABI library: it builds, loads, and exports every symbol include/a3.h declares."""
+import ctypes
+import os
+import re
+
+import pytest
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module")
+def lib_path():
+    from paper_2511_17560_b200 import build
+    return build.build()
+
+
+def declared_symbols():
+    text = open(os.path.join(ROOT, "include", "a3.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    return sorted(set(re.findall(r"\b(a3_[a-z0-9_]+)\s*\(", text)))
+
+
+def test_header_symbols_are_exported(lib_path):
+    lib = ctypes.CDLL(lib_path)
+    syms = declared_symbols()
+    assert {"a3_rope_rerotate", "a3_query_scores", "a3_topk_select", "a3_recompute_layer", "a3_scatter_kv",
+            "a3_fuse_request"} <= set(syms)
+    for s in syms:
+        assert hasattr(lib, s), s
+
+
+def test_binding_lists_the_same_symbols(lib_path):
+    from paper_2511_17560_b200 import a3
+    assert sorted(a3.EXPORTS) == declared_symbols()
+    a3._load()
+
+
+def test_host_only_entry_points(lib_path):
+    from paper_2511_17560_b200 import a3
+    lib = a3._load()
+    assert a3.recompute_count(0.15, 5152, 5120) == 772
+    assert a3.recompute_count(0.15, 528, 512) == 79
+    assert a3.recompute_count(1.0, 528, 512) == 512
+    assert a3.recompute_count(0.0, 528, 512) == 0
+    assert a3.recompute_count(0.3, 10, 10) == 3
+    assert lib.a3_status_string(0) == b"ok"
+    assert lib.a3_status_string(-3) == b"workspace too small"
+    # argument validation happens before any CUDA call
+    assert lib.a3_create(None, None, None) == -1
+    assert lib.a3_fuse_request(None, None, None, 0, None) == -1
+    assert lib.a3_rope_rerotate(None, None, 0, 0, None, None, 0, 0, 0, None) == -1
+    assert lib.a3_topk_select(None, None, 0, 0, 0, None, None) == -1
+    assert lib.a3_layer_workspace_bytes(None, 10) == 0
+
+
+def test_struct_layouts_match_header():
+    from paper_2511_17560_b200 import a3
+    assert ctypes.sizeof(a3.ChunkRef) == 40
+    assert ctypes.sizeof(a3.LayerWeights) == 12 * 8
+    assert ctypes.sizeof(a3.Request) == 8 + 8 * 4 + 8 * 8
+    assert ctypes.sizeof(a3.ModelDesc) == 48

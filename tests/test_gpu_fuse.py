@@ -1,0 +1,199 @@
+"""Whole-request parity: a3_fuse_request against the oracle's fuse_request on the small configurations.
+
+The oracle mirrors the bf16 storage points (rnd=round_bf16).  Scores are gated at 1e-3 only in the
+teacher-forced step test; here the query/key inputs of the score step have themselves gone through two
+different bf16 pipelines, so the end-to-end score gate is looser and the selection is checked (a) exactly
+against the GPU's own scores and (b) against the oracle's modulo scores near the threshold.  Later layers
+are compared with both sides forced onto the GPU's index set.
+"""
+import numpy as np
+import pytest
+import torch
+
+from oracle import a3_oracle as O
+from paper_2511_17560_b200 import workloads as W
+from tests.helpers import oracle_model, oracle_weights
+from tests.test_gpu_steps import KV_MAX, KV_MEAN, a3mod, check_kv, dev_weights, f64, to_dev  # noqa: F401
+
+pytestmark = pytest.mark.gpu
+
+
+class Setup:
+    """A request on both sides: oracle inputs (numpy) and device copies."""
+
+    def __init__(self, a3mod, config, seed=0, emb_std=1.0, w_std=0.05, n_system=0):
+        self.m, self.r = W.request_for(config)
+        m, r = self.m, self.r
+        self.n_system = n_system
+        self.dev = torch.device("cuda:0")
+        layers = W.make_weights(m, seed, std=w_std)
+        self.model, self.weights = oracle_model(m), oracle_weights(layers)
+        self.eng = a3mod.A3(m, dev_weights(layers, self.dev), r.n + 8)
+        self.x0 = W.make_embeddings(m, r.n, seed, std=emb_std)
+        # Eq. 1 on the oracle, mirrored roundings: the stored chunk caches are bf16 values
+        self.ck, self.cv = [], []
+        for o, t in zip(r.offsets, r.chunk_lens):
+            k, v = O.precompute_chunk(self.x0[o:o + t], self.weights, self.model, rnd=O.round_bf16)
+            self.ck.append(k)
+            self.cv.append(v)
+        self.dk = [to_dev(k, self.dev) for k in self.ck]
+        self.dv = [to_dev(v, self.dev) for v in self.cv]
+        self.dx0 = to_dev(self.x0, self.dev)
+        self.tab = a3mod.chunk_table(self.dk, self.dv, r.offsets)
+
+    def fused_buffers(self):
+        m, r = self.m, self.r
+        K = torch.zeros((m.n_layers, r.n, m.n_kv_heads, m.head_dim), dtype=torch.bfloat16, device=self.dev)
+        return K, torch.zeros_like(K)
+
+    def run_gpu(self, ratio, select_layer=None, forced=None):
+        r = self.r
+        K, V = self.fused_buffers()
+        sl = r.select_layer if select_layer is None else select_layer
+        fr = None if forced is None else torch.from_numpy(np.asarray(forced, dtype=np.int32)).to(self.dev)
+        req, out = self.eng.make_request(self.tab, len(self.dk), max(r.chunk_lens), r.n_ctx, r.n_question, self.dx0, K, V,
+                                         ratio=ratio, select_layer=sl, n_system=self.n_system, forced_re=fr)
+        self.eng.fuse_request(req)
+        assert self.eng.device_status() == 0
+        return K, V, out
+
+    def run_oracle(self, ratio, select_layer=None, forced=None):
+        r = self.r
+        sl = r.select_layer if select_layer is None else select_layer
+        return O.fuse_request(self.ck, self.cv, self.x0, r.n_question, self.weights, self.model, ratio, select_layer=sl,
+                              n_system=self.n_system, rnd=O.round_bf16, forced_Re=forced)
+
+
+@pytest.mark.parametrize("config,n_system", [("tiny", 0), ("tiny3", 0), ("tiny_gqa", 100), ("tiny_g7", 0)])
+def test_fuse_request_matches_oracle(a3mod, config, n_system):
+    s = Setup(a3mod, config, n_system=n_system)
+    m, r = s.m, s.r
+    K, V, out = s.run_gpu(r.ratio)
+    p = O.recompute_count(r.ratio, r.n, r.n_ctx - n_system)
+    assert out["p"] == p == a3mod.recompute_count(r.ratio, r.n, r.n_ctx - n_system)
+    rows = out["rows"].cpu().numpy()
+    gs = out["scores"].cpu().numpy().astype(np.float64)
+    Re_gpu = rows[:p]
+    assert rows[p:].tolist() == list(range(r.n_ctx, r.n))
+    # (a) the selection is exactly top-p of the scores the GPU computed
+    assert Re_gpu.tolist() == O.topk_select(gs, n_system, r.n_ctx, p).tolist()
+    # (b) against the oracle run end to end: scores close, sets differ only at the threshold
+    ref = s.run_oracle(r.ratio)
+    cand = slice(n_system, r.n_ctx)
+    rel = np.abs(gs[cand] - ref.scores[cand]) / ref.scores[cand]
+    assert rel.max() <= 3e-2, rel.max()
+    assert not gs[:n_system].any() and not gs[r.n_ctx:].any()
+    tau = np.sort(ref.scores[cand])[-p]
+    for i in set(Re_gpu.tolist()) ^ set(ref.Re.tolist()):
+        assert abs(ref.scores[i] - tau) <= 3e-2 * tau
+    # (c) both sides on the GPU's index set: fused cache and final rows, layer by layer
+    ref = s.run_oracle(r.ratio, forced=Re_gpu)
+    gK, gV, gX = f64(K), f64(V), f64(out["x"])
+    for l in range(m.n_layers):
+        # depth amplifies rounding differences between two bf16 pipelines; the stated gates hold up to the
+        # layer after the selection layer and a looser one is recorded beyond
+        slack = 1.0 if l <= r.select_layer + 1 else 4.0
+        check_kv(gK[l], ref.K[l], f"fused K layer {l}", scale=slack)
+        check_kv(gV[l], ref.V[l], f"fused V layer {l}", scale=slack)
+    # rows outside R at layers after the selection layer are the re-rotated chunk rows, bit for bit
+    Kr, Vr = s.fused_buffers()
+    s.eng.rope_rerotate(s.tab, len(s.dk), max(r.chunk_lens), Kr, Vr)
+    mask = torch.ones(r.n, dtype=torch.bool, device=s.dev)
+    mask[out["rows"].long()] = False
+    for l in range(r.select_layer + 1, m.n_layers):
+        assert torch.equal(K[l][mask], Kr[l][mask]) and torch.equal(V[l][mask], Vr[l][mask])
+    scale = max(1.0, float(np.abs(ref.X).std()))
+    err = np.abs(gX - ref.X)
+    assert err.mean() <= 8e-3 * scale and err.max() <= 0.25 * scale, (err.mean(), err.max(), scale)
+    s.eng.close()
+
+
+def test_ratio_one_equals_gpu_full_prefill_and_ratio_zero_keeps_cache(a3mod):
+    s = Setup(a3mod, "tiny3")
+    m, r = s.m, s.r
+    # full prefill on the GPU through the per-layer call: every row, positions 0..n-1
+    Kp, Vp = s.fused_buffers()
+    X = s.dx0.clone()
+    pos = torch.arange(r.n, dtype=torch.int32, device=s.dev)
+    for l in range(m.n_layers):
+        s.eng.recompute_layer(l, X, pos, Kp[l], Vp[l])
+    K1, V1, out1 = s.run_gpu(1.0)
+    assert out1["p"] == r.n_ctx
+    assert out1["rows"].cpu().numpy().tolist() == list(range(r.n))
+    # same kernels, same rows, same order: the r = 1 fusion IS the full prefill
+    assert torch.equal(K1, Kp) and torch.equal(V1, Vp) and torch.equal(out1["x"], X)
+    # and it agrees with the oracle's full prefill
+    Ko, Vo, Xo = O.full_prefill(s.x0, s.weights, s.model, rnd=O.round_bf16)
+    check_kv(f64(Kp)[:2], Ko[:2], "prefill K")
+    # r = 0: only the question rows move; layers after the selection layer keep the re-rotated context rows
+    K0, V0, out0 = s.run_gpu(0.0)
+    assert out0["p"] == 0 and out0["rows"].cpu().numpy().tolist() == list(range(r.n_ctx, r.n))
+    Kr, Vr = s.fused_buffers()
+    s.eng.rope_rerotate(s.tab, len(s.dk), max(r.chunk_lens), Kr, Vr)
+    assert torch.equal(K0[2, :r.n_ctx], Kr[2, :r.n_ctx]) and torch.equal(V0[2, :r.n_ctx], Vr[2, :r.n_ctx])
+    assert torch.equal(K0[:2], K1[:2])  # layers up to the selection layer hold true values either way
+    # nested selections across ratios on the same request
+    prev = None
+    for ratio in (0.05, 0.10, 0.15, 0.30):
+        _, _, o = s.run_gpu(ratio)
+        cur = set(o["rows"].cpu().numpy()[: o["p"]].tolist())
+        if prev is not None:
+            assert prev <= cur
+        prev = cur
+    s.eng.close()
+
+
+def test_fuse_batch_and_host_entry_match_single_requests(a3mod):
+    s = Setup(a3mod, "tiny_gqa")
+    m, r = s.m, s.r
+    K, V, out = s.run_gpu(r.ratio)
+    # batch of two identical requests into separate buffers
+    reqs, outs, bufs = [], [], []
+    for _ in range(2):
+        Kb, Vb = s.fused_buffers()
+        rq, ob = s.eng.make_request(s.tab, len(s.dk), max(r.chunk_lens), r.n_ctx, r.n_question, s.dx0, Kb, Vb,
+                                    ratio=r.ratio, select_layer=r.select_layer)
+        reqs.append(rq)
+        outs.append(ob)
+        bufs.append((Kb, Vb))
+    s.eng.fuse_batch(reqs)
+    for (Kb, Vb), ob in zip(bufs, outs):
+        assert torch.equal(Kb, K) and torch.equal(Vb, V) and torch.equal(ob["x"], out["x"]) and torch.equal(ob["rows"], out["rows"])
+    # host entry: chunk caches and embeddings in pinned host memory
+    hk = [k.cpu().pin_memory() for k in s.dk]
+    hv = [v.cpu().pin_memory() for v in s.dv]
+    hx = s.dx0.cpu().pin_memory()
+    Kh, Vh = s.fused_buffers()
+    rq, oh = s.eng.make_request(None, len(hk), 0, r.n_ctx, r.n_question, None, Kh, Vh, ratio=r.ratio, select_layer=r.select_layer)
+    rows_h = torch.empty(oh["p"] + r.n_question, dtype=torch.int32).pin_memory()
+    x_h = torch.empty((oh["p"] + r.n_question, m.d_model), dtype=torch.bfloat16).pin_memory()
+    staging = torch.empty(s.eng.host_staging_bytes(r.n_ctx, r.n), dtype=torch.uint8, device=s.dev)
+    s.eng.fuse_request_host(rq, hk, hv, hx, rows_h, x_h, staging)
+    assert torch.equal(Kh, K) and torch.equal(Vh, V)
+    assert torch.equal(rows_h, out["rows"].cpu()) and torch.equal(x_h, out["x"].cpu())
+    assert s.eng.device_status() == 0
+    s.eng.close()
+
+
+def test_fuse_request_rejects_bad_arguments(a3mod):
+    s = Setup(a3mod, "tiny")
+    r = s.r
+    K, V = s.fused_buffers()
+    lib = a3mod._load()
+    import ctypes as C
+    def status(**kw):
+        rq, out = s.eng.make_request(s.tab, len(s.dk), max(r.chunk_lens), r.n_ctx, r.n_question, s.dx0, K, V, ratio=0.15, select_layer=0)
+        ws_bytes = kw.pop("_ws", None)
+        for k, v in kw.items():
+            setattr(rq, k, v)
+        ws = s.eng.workspace(s.eng.request_workspace_bytes(r.n))
+        return lib.a3_fuse_request(s.eng._h, C.byref(rq), ws.data_ptr(), ws.numel() if ws_bytes is None else ws_bytes, None)
+    assert status() == 0
+    assert status(select_layer=5) == -1
+    assert status(n_recompute=r.n_ctx + 1) == -1
+    assert status(x0=None) == -1
+    assert status(layer_stride=16) == -1
+    assert status(_ws=1024) == -3
+    assert lib.a3_fuse_request(None, None, None, 0, None) == -1
+    torch.cuda.synchronize()
+    s.eng.close()
