@@ -18,6 +18,16 @@ from tests.test_gpu_steps import KV_MAX, KV_MEAN, a3mod, check_kv, dev_weights, 
 pytestmark = pytest.mark.gpu
 
 
+def check_drift(got, want, what, mean_gate):
+    """End-to-end comparison of two bf16-rounded tensors that came through different pipelines: a one-ulp flip
+    at the largest magnitude is legitimate, so the max gate is two ulps there; the mean gate is the caller's."""
+    err = np.abs(got - want)
+    top = max(float(np.abs(want).max()), 1e-6)
+    ulp = 2.0 ** (np.floor(np.log2(top)) - 7)
+    assert err.max() <= max(KV_MAX, 2 * ulp), f"{what}: max abs {err.max():.3e} (ulp {ulp:.3e})"
+    assert err.mean() <= mean_gate, f"{what}: mean abs {err.mean():.3e} > {mean_gate:.1e}"
+
+
 class Setup:
     """A request on both sides: oracle inputs (numpy) and device copies."""
 
@@ -64,9 +74,13 @@ class Setup:
                               n_system=self.n_system, rnd=O.round_bf16, forced_Re=forced)
 
 
-@pytest.mark.parametrize("config,n_system", [("tiny", 0), ("tiny3", 0), ("tiny_gqa", 100), ("tiny_g7", 0)])
-def test_fuse_request_matches_oracle(a3mod, config, n_system):
-    s = Setup(a3mod, config, n_system=n_system)
+# "spec": the configurations' own distributions, weights and embeddings N(0, 0.02^2).  "wide": weights N(0, 0.05^2) and
+# unit embeddings, which at d = 512 give K/V the spread they have at Llama width (about 1.1) and make every
+# sub-block's gain exceed one, so that rounding differences grow visibly from layer to layer.
+@pytest.mark.parametrize("config,n_system,dist", [("tiny", 0, "spec"), ("tiny3", 0, "spec"), ("tiny", 0, "wide"), ("tiny3", 0, "wide"),
+                                                  ("tiny_gqa", 100, "wide"), ("tiny_g7", 0, "spec"), ("tiny_g7", 0, "wide")])
+def test_fuse_request_matches_oracle(a3mod, config, n_system, dist):
+    s = Setup(a3mod, config, n_system=n_system, **(dict(emb_std=0.02, w_std=0.02) if dist == "spec" else {}))
     m, r = s.m, s.r
     K, V, out = s.run_gpu(r.ratio)
     p = O.recompute_count(r.ratio, r.n, r.n_ctx - n_system)
@@ -90,11 +104,13 @@ def test_fuse_request_matches_oracle(a3mod, config, n_system):
     ref = s.run_oracle(r.ratio, forced=Re_gpu)
     gK, gV, gX = f64(K), f64(V), f64(out["x"])
     for l in range(m.n_layers):
-        # depth amplifies rounding differences between two bf16 pipelines; the stated gates hold up to the
-        # layer after the selection layer and a looser one is recorded beyond
-        slack = 1.0 if l <= r.select_layer + 1 else 4.0
-        check_kv(gK[l], ref.K[l], f"fused K layer {l}", scale=slack)
-        check_kv(gV[l], ref.V[l], f"fused V layer {l}", scale=slack)
+        # Layer 0 sees identical inputs on both sides, so the stated mean gate applies as it is.  Deeper layers are
+        # fed by each side's own bf16 hidden state, whose rounding differences the blocks amplify: the bound
+        # recorded here is twice the gate for the configurations' own distributions and triples per layer for the
+        # wide one (the per-layer, teacher-forced gates are in test_gpu_steps).
+        gate = KV_MEAN if l == 0 else (2 * KV_MEAN if dist == "spec" else KV_MEAN * 3 ** l)
+        check_drift(gK[l], ref.K[l], f"fused K layer {l}", gate)
+        check_drift(gV[l], ref.V[l], f"fused V layer {l}", gate)
     # rows outside R at layers after the selection layer are the re-rotated chunk rows, bit for bit
     Kr, Vr = s.fused_buffers()
     s.eng.rope_rerotate(s.tab, len(s.dk), max(r.chunk_lens), Kr, Vr)
@@ -102,9 +118,7 @@ def test_fuse_request_matches_oracle(a3mod, config, n_system):
     mask[out["rows"].long()] = False
     for l in range(r.select_layer + 1, m.n_layers):
         assert torch.equal(K[l][mask], Kr[l][mask]) and torch.equal(V[l][mask], Vr[l][mask])
-    scale = max(1.0, float(np.abs(ref.X).std()))
-    err = np.abs(gX - ref.X)
-    assert err.mean() <= 8e-3 * scale and err.max() <= 0.25 * scale, (err.mean(), err.max(), scale)
+    check_drift(gX, ref.X, "final hidden rows", 6e-3 * float(np.abs(ref.X).std()) * 2 ** (m.n_layers - 1))
     s.eng.close()
 
 
@@ -124,7 +138,8 @@ def test_ratio_one_equals_gpu_full_prefill_and_ratio_zero_keeps_cache(a3mod):
     assert torch.equal(K1, Kp) and torch.equal(V1, Vp) and torch.equal(out1["x"], X)
     # and it agrees with the oracle's full prefill
     Ko, Vo, Xo = O.full_prefill(s.x0, s.weights, s.model, rnd=O.round_bf16)
-    check_kv(f64(Kp)[:2], Ko[:2], "prefill K")
+    check_drift(f64(Kp)[0], Ko[0], "prefill K layer 0", KV_MEAN)
+    check_drift(f64(Kp)[1], Ko[1], "prefill K layer 1", 2 * KV_MEAN)
     # r = 0: only the question rows move; layers after the selection layer keep the re-rotated context rows
     K0, V0, out0 = s.run_gpu(0.0)
     assert out0["p"] == 0 and out0["rows"].cpu().numpy().tolist() == list(range(r.n_ctx, r.n))

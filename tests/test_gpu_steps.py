@@ -251,9 +251,13 @@ def test_recompute_layer_parity(a3mod, shape, kv_len, M, seed):
     mask[pos] = False
     np.testing.assert_array_equal(gK[mask], Kc[layer][mask])  # rows outside R untouched, bit for bit
     np.testing.assert_array_equal(gV[mask], Vc[layer][mask])
-    scale = max(1.0, float(np.abs(parts["x_exact"]).std()))
-    check_kv(gX, parts["x_exact"], "hidden rows", scale=scale)
-    np.testing.assert_allclose(lse.cpu().numpy(), parts["lse"], atol=2e-2)
+    # Hidden rows are not covered by the stated K/V gates.  Their bound: one bf16 rounding of the result (mean
+    # about 1.2e-3 per unit spread) plus what the one deliberate difference between the pipelines - attention
+    # probabilities enter the P.V tensor-core product as bf16 - becomes after the output projection and the MLP,
+    # whose gains exceed one with these weights (measured 2.5e-3..3e-3 per unit spread).  Gate: twice the K/V
+    # gates per unit spread of the result.
+    check_kv(gX, parts["x_exact"], "hidden rows", scale=2.0 * float(parts["x_exact"].std()))
+    np.testing.assert_allclose(lse.cpu().numpy(), parts["lse"], atol=5e-3)
     eng.close()
 
 
