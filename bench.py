@@ -1,0 +1,417 @@
+#!/usr/bin/env python
+"""Benchmark of the A^3 fusion hot path: context tokens fused per second on B200.
+
+A step is one whole fusion request (position recovery of all layers, the leading full block, selection,
+and the recompute layers) on synthetic inputs of the configured shape.  One JSON line is printed by rank 0.
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--impl a3|reference] [--config NAME]
+
+N > 1 runs N independent replicas (one process per GPU, launched with torch.distributed.run); the path has no
+exchange step, so there is no data-path collective: only the barrier and the max-over-ranks of the time.
+`--impl reference` times the CPU oracle (as it stands, fp32) on the host cores on a bounded sample of the same
+workload.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "context_tokens_fused_per_s"
+UNIT = "tokens/s"
+FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        try:
+            with open(path) as f:
+                p = json.load(f)
+            return {k: float(p[k]) for k in FALLBACK_PEAKS}, "measured"
+        except Exception:
+            pass
+    return dict(FALLBACK_PEAKS), "fallback"
+
+
+# ------------------------------------------------------------------ algorithmic work of one request
+
+
+def algorithmic_work(m, r, p, rows):
+    """FLOPs / bytes the method must do per request, per kernel class (not what a kernel happens to move)."""
+    n, nq, L, ls = r.n, r.n_question, m.n_layers, r.select_layer
+    d, D, Hq, Hkv, F = m.d_model, m.head_dim, m.n_q_heads, m.n_kv_heads, m.d_ff
+    M = p + nq
+    qd, kvd = Hq * D, Hkv * D
+    full_rows = n * ls                      # rows through complete blocks before the selection layer
+    sparse_rows = M * (L - ls)              # rows through complete blocks from the selection layer on
+    w = {}
+    w["gemm_qkv"] = 2.0 * d * ((full_rows + sparse_rows) * (qd + 2 * kvd) + n * 2 * kvd + nq * qd)
+    w["gemm_residual"] = 2.0 * (full_rows + sparse_rows) * (qd * d + F * d)
+    w["gemm_swiglu"] = 2.0 * (full_rows + sparse_rows) * d * 2 * F
+    vis_full = n * (n + 1) / 2.0
+    vis_q = float(sum(range(r.n_ctx + 1, n + 1)))
+    vis_rows = float(np.sum(np.asarray(rows, dtype=np.float64) + 1.0))
+    w["attention"] = 4.0 * D * Hq * (ls * vis_full + (L - ls) * vis_rows) + 2.0 * D * Hq * vis_q
+    w["scores"] = 2.0 * D * Hq * vis_q
+    b = {"rerotate": 4.0 * r.n_ctx * kvd * 2 * L}
+    return w, b
+
+
+# ------------------------------------------------------------------ clocks
+
+
+class ClockSampler:
+    Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.proc = None
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits", "-lms", "100",
+                                          "-i", str(gpu_index)], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+        except Exception:
+            self.proc = None
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.15)
+        self.proc.terminate()
+        try:
+            out, _ = self.proc.communicate(timeout=5)
+        except Exception:
+            self.proc.kill()
+            out = ""
+        sm, mx, reasons, power = [], [], set(), []
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for line in out.strip().splitlines():
+            f = [x.strip() for x in line.split(",")]
+            if len(f) < 9:
+                continue
+            try:
+                sm.append(float(f[1]))
+                mx.append(float(f[2]))
+                power.append(float(f[3]))
+            except ValueError:
+                continue
+            for nm, val in zip(names, f[5:9]):
+                if val.lower().startswith("active"):
+                    reasons.add(nm)
+        if not sm:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["no samples"]}
+        return {"sm_mhz": float(np.median(sm)), "sm_max_mhz": float(max(mx)), "reasons": sorted(reasons),
+                "samples": len(sm), "power_w_max": max(power) if power else None}
+
+
+# ------------------------------------------------------------------ multi-rank plumbing
+
+
+def dist_setup(n_gpus: int, backend: str = "nccl"):
+    """Returns (rank, world, local_rank).  world > 1 only under torch.distributed.run."""
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    if world <= 1:
+        return 0, 1, 0
+    import torch.distributed as dist
+    os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+    if not dist.is_initialized():
+        dist.init_process_group(backend=backend)
+    return dist.get_rank(), dist.get_world_size(), int(os.environ.get("LOCAL_RANK", "0"))
+
+
+def barrier():
+    import torch.distributed as dist
+    if dist.is_available() and dist.is_initialized():
+        dist.barrier()
+
+
+def max_over_ranks(value: float, device="cpu") -> float:
+    import torch
+    import torch.distributed as dist
+    if not (dist.is_available() and dist.is_initialized()):
+        return float(value)
+    t = torch.tensor([float(value)], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def aggregate_value(units_per_rank_per_step: float, steps: int, world: int, max_seconds: float) -> float:
+    """Whole-job throughput of `world` independent replicas (weak scaling)."""
+    return units_per_rank_per_step * steps * world / max_seconds
+
+
+# ------------------------------------------------------------------ the CPU oracle arm
+
+
+def oracle_sample(config: str, seed: int = 0):
+    """Builds the inputs of the bounded oracle sample: 3 layers of the stack at full width, random caches."""
+    from dataclasses import replace
+    from oracle import a3_oracle as O
+    from paper_2511_17560_b200 import workloads as W
+    m_full, r = W.request_for(config)
+    m = replace(m_full, n_layers=min(3, m_full.n_layers))
+    model = O.Model(m.n_layers, m.d_model, m.n_q_heads, m.n_kv_heads, m.head_dim, m.d_ff, m.rope_theta, m.rms_eps, m.rope_layout)
+    weights = [O.LayerWeights(**w) for w in W.make_weights(m, seed)]
+    x0 = W.make_embeddings_device(m, r.n, "cpu", seed).float().numpy()
+    ck, cv = zip(*[W.make_cache_like(replace(m, n_layers=1), t, seed, c, std=1.28) for c, t in enumerate(r.chunk_lens)])
+    return dict(O=O, m_full=m_full, m=m, r=r, model=model, weights=weights, x0=x0, ck=ck, cv=cv)
+
+
+def oracle_step(S, stride: int = 4):
+    """One bounded sample of the request on the oracle (fp32), extrapolated to the whole request.
+
+    Timed pieces, each the oracle's own function: position recovery of one layer (x L); one full block on every
+    `stride`-th row (x stride x select_layer); the selection layer's norm + QKV on every `stride`-th row (x stride),
+    scores and top-p at full size; one recompute layer on the p + |Q| carried rows (x (L - select_layer)).
+    """
+    O, m, mf, r, model, weights = S["O"], S["m"], S["m_full"], S["r"], S["model"], S["weights"]
+    dt = np.float32
+    L, ls = mf.n_layers, min(r.select_layer, m.n_layers - 1)
+    n, nq = r.n, r.n_question
+    one = O.Model(1, m.d_model, m.n_q_heads, m.n_kv_heads, m.head_dim, m.d_ff, m.rope_theta, m.rms_eps, m.rope_layout)
+    t = {}
+    c0 = time.perf_counter()
+    K, V = O.position_recovery(S["ck"], S["cv"], r.offsets, n, one, dtype=dt)
+    t["position_recovery"] = (time.perf_counter() - c0) * L
+    K, V = K[0], V[0]
+    X = S["x0"].astype(dt)
+    sub = np.arange(0, n, stride)
+    c0 = time.perf_counter()
+    if ls > 0:
+        O.recompute_layer(X[sub], sub, weights[0], model, K, V)
+    t["full_blocks"] = (time.perf_counter() - c0) * stride * ls
+    c0 = time.perf_counter()
+    w = weights[ls]
+    a = O.rmsnorm(X[sub], w.attn_norm, model.rms_eps)
+    O.project_qkv(a, w, model, sub)
+    t_kv = (time.perf_counter() - c0) * stride
+    c0 = time.perf_counter()
+    q_rows = np.arange(r.n_ctx, n)
+    aq = O.rmsnorm(X[q_rows], w.attn_norm, model.rms_eps)
+    q, _, _ = O.project_qkv(aq, w, model, q_rows)
+    s = O.query_scores(q, q_rows, K, model, 0, r.n_ctx)
+    p = O.recompute_count(r.ratio, n, r.n_ctx)
+    Re = O.topk_select(s, 0, r.n_ctx, p)
+    t["selection"] = t_kv + (time.perf_counter() - c0)
+    R = np.concatenate([Re, q_rows])
+    c0 = time.perf_counter()
+    O.recompute_layer(X[R], R, weights[min(ls + 1, m.n_layers - 1)], model, K, V)
+    t["recompute_layers"] = (time.perf_counter() - c0) * (L - ls)
+    return sum(t.values()), t
+
+
+def oracle_threads() -> int:
+    try:
+        from threadpoolctl import threadpool_info
+        return max([int(i.get("num_threads", 1)) for i in threadpool_info()] + [1])
+    except Exception:
+        return os.cpu_count() or 1
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    S = oracle_sample(args.config)
+    r = S["r"]
+    for _ in range(args.warmup):
+        oracle_step(S)
+    secs, parts = [], None
+    for _ in range(args.steps):
+        s, parts = oracle_step(S)
+        secs.append(s)
+    t = float(np.mean(secs))
+    value = r.n_ctx / t
+    sample = ("per step: position recovery of 1 layer, one full block and the selection-layer QKV on every 4th row, "
+              "scores + top-p at full size, one recompute layer on the p+|Q| rows; scaled to all layers/rows "
+              "(extrapolated); oracle in fp32 with random caches of the workload's shape")
+    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": t * 1e3, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": "f32", "data": "synthetic",
+            "config": {"workload": args.config, "recompute_ratio": r.ratio, "n_ctx": r.n_ctx, "n_question": r.n_question},
+            "cpu_baseline": {"value": value, "unit": UNIT, "cores": oracle_threads(), "kind": "oracle", "sample": sample,
+                             "seconds_by_phase": parts},
+            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
+    print(json.dumps(line), flush=True)
+
+
+# ------------------------------------------------------------------ the CUDA arm
+
+
+def precompute_chunks(eng, m, r, x0, dev):
+    """Eq. 1 on the GPU: each chunk alone at local positions 0..T-1 through every layer (same kernels, all rows)."""
+    import torch
+    ck, cv = [], []
+    for o, t in zip(r.offsets, r.chunk_lens):
+        K = torch.zeros((m.n_layers, t, m.n_kv_heads, m.head_dim), dtype=torch.bfloat16, device=dev)
+        V = torch.zeros_like(K)
+        X = x0[o:o + t].clone()
+        pos = torch.arange(t, dtype=torch.int32, device=dev)
+        for l in range(m.n_layers):
+            eng.recompute_layer(l, X, pos, K[l], V[l])
+        ck.append(K)
+        cv.append(V)
+    return ck, cv
+
+
+def run_a3(args):
+    import torch
+    from paper_2511_17560_b200 import a3
+    from paper_2511_17560_b200 import workloads as W
+
+    rank, world, local = dist_setup(args.gpus)
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    peaks, peak_src = load_peaks()
+    m, r = W.request_for(args.config)
+    if args.layers:
+        from dataclasses import replace
+        m = replace(m, n_layers=args.layers)  # profiling captures only: a truncated stack is not a bench result
+    eng = a3.A3(m, W.make_weights_device(m, dev, seed=0), r.n + 8)
+    x0 = W.make_embeddings_device(m, r.n, dev, seed=0)
+    ck, cv = precompute_chunks(eng, m, r, x0, dev)
+    tab = a3.chunk_table(ck, cv, r.offsets)
+    K = torch.zeros((m.n_layers, r.n, m.n_kv_heads, m.head_dim), dtype=torch.bfloat16, device=dev)
+    V = torch.zeros_like(K)
+    req, out = eng.make_request(tab, len(ck), max(r.chunk_lens), r.n_ctx, r.n_question, x0, K, V, ratio=r.ratio,
+                                select_layer=r.select_layer)
+    p = out["p"]
+    eng.workspace(eng.request_workspace_bytes(r.n))
+    stream = torch.cuda.current_stream()
+
+    for _ in range(max(args.warmup, 3)):
+        eng.fuse_request(req)
+    torch.cuda.synchronize()
+    assert eng.device_status() == 0, "device status word set during warm-up"
+    a3.launch_count(reset=True)
+    eng.fuse_request(req)
+    torch.cuda.synchronize()
+    launches_per_step = a3.launch_count(reset=True)
+    eng.profile_enable(launches_per_step * args.steps + 16)
+
+    sampler = ClockSampler(local) if rank == 0 else None
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    torch.cuda.synchronize()
+    e0.record(stream)
+    for _ in range(args.steps):
+        eng.fuse_request(req)
+    e1.record(stream)
+    torch.cuda.synchronize()
+    barrier()
+    seconds = max_over_ranks(e0.elapsed_time(e1) / 1e3, dev)
+    clocks = sampler.stop() if sampler else None
+    gpu_launches = a3.launch_count(reset=True)
+    prof = eng.profile_read()
+    eng.profile_enable(0)
+    assert eng.device_status() == 0, "device status word set during the timed region"
+    value = aggregate_value(r.n_ctx, args.steps, world, seconds)
+    rows = out["rows"].cpu().numpy()
+
+    # ---- roofline of the dominant kernel class (device time from CUDA events around every launch)
+    flops, bts = algorithmic_work(m, r, p, rows)
+    kernels = {}
+    for name, e in prof.items():
+        if not e["launches"]:
+            continue
+        per_step_ms = e["ms"] / args.steps
+        k = {"launches_per_step": e["launches"] / args.steps, "ms_per_step": per_step_ms}
+        if name in flops:
+            k.update(bound="tensor", achieved=flops[name] / (per_step_ms * 1e-3) / 1e12, unit="TFLOP/s")
+            k["frac"] = k["achieved"] / peaks["bf16_tflops_sustained"]
+        elif name in bts:
+            k.update(bound="hbm", achieved=bts[name] / (per_step_ms * 1e-3) / 1e9, unit="GB/s")
+            k["frac"] = k["achieved"] / peaks["hbm_gbs"]
+        kernels[name] = k
+    tot_ms = sum(k["ms_per_step"] for k in kernels.values())
+    for k in kernels.values():
+        k["share"] = k["ms_per_step"] / tot_ms
+    top = max(kernels, key=lambda nm: kernels[nm]["ms_per_step"])
+    tk = kernels[top]
+    roofline = {"kernel": top, "bound": tk.get("bound"), "achieved": tk.get("achieved"),
+                "peak": peaks["bf16_tflops_sustained"] if tk.get("bound") == "tensor" else peaks["hbm_gbs"],
+                "unit": tk.get("unit"), "frac": tk.get("frac"), "traffic": None, "peak_source": peak_src + " (sustained)",
+                "avg_launch_ms": tk["ms_per_step"] / tk["launches_per_step"], "kernels": kernels}
+    total_flops = sum(flops.values())
+
+    # ---- end to end through the host-buffer entry: pinned chunk caches + embeddings in, rows + hidden rows out
+    e2e = None
+    if not args.no_e2e:
+        hk = [k.cpu().pin_memory() for k in ck]
+        hv = [v.cpu().pin_memory() for v in cv]
+        hx = x0.cpu().pin_memory()
+        rows_h = torch.empty(p + r.n_question, dtype=torch.int32).pin_memory()
+        x_h = torch.empty((p + r.n_question, m.d_model), dtype=torch.bfloat16).pin_memory()
+        staging = torch.empty(eng.host_staging_bytes(r.n_ctx, r.n), dtype=torch.uint8, device=dev)
+        req_h, out_h = eng.make_request(None, len(hk), 0, r.n_ctx, r.n_question, None, K, V, ratio=r.ratio, select_layer=r.select_layer)
+        for _ in range(2):
+            eng.fuse_request_host(req_h, hk, hv, hx, rows_h, x_h, staging)
+        barrier()
+        torch.cuda.synchronize()
+        t0 = time.perf_counter()
+        e0.record(stream)
+        for _ in range(args.steps):
+            eng.fuse_request_host(req_h, hk, hv, hx, rows_h, x_h, staging)
+        e1.record(stream)
+        torch.cuda.synchronize()
+        wall = time.perf_counter() - t0
+        sec_e = max_over_ranks(max(e0.elapsed_time(e1) / 1e3, wall), dev)
+        h2d = sum(k.numel() * 2 for k in hk) * 2 + hx.numel() * 2
+        d2h = rows_h.numel() * 4 + x_h.numel() * 2
+        e2e = {"value": aggregate_value(r.n_ctx, args.steps, world, sec_e), "unit": UNIT, "ms_per_step": sec_e / args.steps * 1e3,
+               "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h)}
+        assert torch.equal(rows_h, out["rows"].cpu()), "host entry selected different rows"
+
+    cpu = None
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        S = oracle_sample(args.config)
+        t, parts = oracle_step(S)
+        cpu = {"value": r.n_ctx / t, "unit": UNIT, "cores": oracle_threads(), "kind": "oracle", "seconds": t,
+               "sample": "one bounded oracle step (fp32): 1 layer of position recovery, a full block and the selection QKV on "
+                         "every 4th row, scores + top-p at full size, one recompute layer; extrapolated to the whole request",
+               "seconds_by_phase": parts}
+    if rank == 0:
+        line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3),
+                "ms_per_step": seconds / args.steps * 1e3, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+                "dtype": "bf16", "data": "synthetic",
+                "config": {"workload": args.config, "model": m.name, "chunks": len(r.chunk_lens), "n_ctx": r.n_ctx,
+                           "n_question": r.n_question, "recompute_ratio": r.ratio, "n_recompute": p, "select_layer": r.select_layer,
+                           "replicas": world, "layers": m.n_layers, "truncated_for_profiling": bool(args.layers), "l2": "inputs larger than L2: every step streams the stack's weights "
+                                                    f"({sum(t.numel() for w in eng._weights for t in w.values()) * 2 / 2**30:.1f} GiB) and the fused cache"},
+                "request_ms": seconds / args.steps * 1e3,
+                "algorithmic_tflop_per_request": total_flops / 1e12,
+                "request_tflops": total_flops / (seconds / args.steps) / 1e12,
+                "request_frac_of_sustained_peak": total_flops / (seconds / args.steps) / 1e12 / peaks["bf16_tflops_sustained"],
+                "gpu_launches": int(gpu_launches), "clocks": clocks, "roofline": roofline, "e2e": e2e, "cpu_baseline": cpu}
+        print(json.dumps(line), flush=True)
+    eng.close()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=5)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="a3", choices=["a3", "reference"])
+    ap.add_argument("--config", default="llama8b_10x512")
+    ap.add_argument("--layers", type=int, default=0, help="truncate the stack (ncu captures of a small case only)")
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_a3(args)
+
+
+if __name__ == "__main__":
+    main()

@@ -199,6 +199,19 @@ int a3_last_cuda_error(void);
 /* Number of kernel launches this library has queued since the counter was last reset (host counter). */
 uint64_t a3_launch_count(int reset);
 
+/* Per-kernel-class device timing with CUDA events recorded on the launching stream around every launch.
+ * a3_profile_enable(h, max_records > 0) allocates the event pool (not a hot call) and starts recording;
+ * max_records = 0 stops and frees it.  When the pool is full further launches are not recorded.
+ * a3_profile_read waits for `stream`, adds up the elapsed time per class and clears the records. */
+typedef enum {
+  A3_K_REROTATE = 0, A3_K_RMSNORM, A3_K_GEMM_QKV, A3_K_ATTENTION, A3_K_GEMM_RESIDUAL, A3_K_GEMM_SWIGLU,
+  A3_K_SCORES, A3_K_TOPK, A3_K_ROWS /* gather, scatter, index kernels */, A3_K_CLASSES
+} a3_kernel_class;
+typedef struct { uint64_t launches; double ms; } a3_profile_entry;
+int a3_profile_enable(a3_handle* h, int max_records);
+int a3_profile_read(a3_handle* h, a3_profile_entry* out /* host [A3_K_CLASSES] */, a3_stream stream);
+const char* a3_kernel_class_name(int cls);
+
 #ifdef __cplusplus
 }
 #endif

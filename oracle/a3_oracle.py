@@ -45,6 +45,7 @@ has no pin beyond the oracle itself ("parity unpinned" for that one statement).
 from __future__ import annotations
 
 import math
+import time
 from dataclasses import dataclass, field
 from typing import Callable, List, Optional, Sequence
 
@@ -392,15 +393,18 @@ def fuse_request(
     assert n_ctx + n_question == n
     cand_begin, cand_end = n_system, n_ctx
     trace = {}
+    stamps = [("start", time.perf_counter())]  # wall-clock per phase, for the CPU baseline report only
 
     # position recovery (Eq. 2)
     K, V = position_recovery(chunk_k, chunk_v, offsets, n, model, dtype, rnd)
+    stamps.append(("position_recovery", time.perf_counter()))
 
     # embedding + leading decoder blocks over the whole input -> true states at the selection layer
     X = x0.astype(dtype)
     all_pos = np.arange(n)
     for l in range(select_layer):
         X = recompute_layer(X, all_pos, weights[l], model, K[l], V[l], rnd)
+        stamps.append((f"full_block_{l}", time.perf_counter()))
 
     # true K, V for every row at the selection layer; question queries; scores; Re (Eq. 3)
     w = weights[select_layer]
@@ -416,10 +420,13 @@ def fuse_request(
     if keep_trace:
         trace["x_select"] = X.copy()
     X = X[R]
+    stamps.append(("selection", time.perf_counter()))
 
     # layers from the selection layer on: only rows [Re, Q] (Eq. 4, Eq. 5)
     for l in range(select_layer, L):
         if keep_trace:
             trace[f"x_in_{l}"] = X.copy()
         X = recompute_layer(X, R, weights[l], model, K[l], V[l], rnd)
+        stamps.append((f"recompute_{l}", time.perf_counter()))
+    trace["seconds"] = {name: t - stamps[i][1] for i, (name, t) in enumerate(stamps[1:])}
     return FuseResult(K=K, V=V, Re=Re, R=R, scores=s, X=X, trace=trace)

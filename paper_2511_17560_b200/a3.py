@@ -64,7 +64,13 @@ class HostIO(C.Structure):
 EXPORTS = ("a3_create", "a3_destroy", "a3_layer_workspace_bytes", "a3_request_workspace_bytes", "a3_host_staging_bytes",
            "a3_recompute_count", "a3_rope_rerotate", "a3_query_scores", "a3_topk_select", "a3_recompute_layer",
            "a3_scatter_kv", "a3_gather_rows", "a3_fuse_request", "a3_fuse_batch", "a3_fuse_request_host",
-           "a3_device_status", "a3_status_string", "a3_last_cuda_error", "a3_launch_count")
+           "a3_device_status", "a3_status_string", "a3_last_cuda_error", "a3_launch_count", "a3_profile_enable",
+           "a3_profile_read", "a3_kernel_class_name")
+K_CLASSES = 9
+
+
+class ProfileEntry(C.Structure):
+    _fields_ = [("launches", C.c_uint64), ("ms", C.c_double)]
 
 
 def _load():
@@ -100,6 +106,10 @@ def _load():
     lib.a3_last_cuda_error.argtypes = []
     lib.a3_launch_count.argtypes = [i32]
     lib.a3_launch_count.restype = u64
+    lib.a3_profile_enable.argtypes = [vp, i32]
+    lib.a3_profile_read.argtypes = [vp, C.POINTER(ProfileEntry), vp]
+    lib.a3_kernel_class_name.argtypes = [i32]
+    lib.a3_kernel_class_name.restype = C.c_char_p
     _lib = lib
     return lib
 
@@ -283,6 +293,17 @@ class A3:
         ws = self.workspace(self.request_workspace_bytes(n))
         _check(_load().a3_fuse_request_host(self._h, C.byref(req), C.byref(io), _ptr(staging), staging.numel(),
                                             _ptr(ws), ws.numel(), _stream()), "a3_fuse_request_host")
+
+    def profile_enable(self, max_records: int):
+        _check(_load().a3_profile_enable(self._h, int(max_records)), "a3_profile_enable")
+
+    def profile_read(self) -> Dict[str, Dict[str, float]]:
+        """Per kernel class: launches and summed device milliseconds since the last read (waits for the stream)."""
+        lib = _load()
+        arr = (ProfileEntry * K_CLASSES)()
+        _check(lib.a3_profile_read(self._h, arr, _stream()), "a3_profile_read")
+        return {lib.a3_kernel_class_name(k).decode(): dict(launches=int(arr[k].launches), ms=float(arr[k].ms))
+                for k in range(K_CLASSES)}
 
     def device_status(self) -> int:
         bits = C.c_uint32(0)

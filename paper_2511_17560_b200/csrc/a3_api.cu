@@ -135,8 +135,56 @@ extern "C" int a3_create(a3_handle** out, const a3_model_desc* m, const a3_layer
   return A3_OK;
 }
 
+extern "C" int a3_profile_enable(a3_handle* h, int max_records) {
+  if (!h || max_records < 0) return A3_EINVAL;
+  if (h->prof) {
+    for (int i = 0; i < 2 * h->prof->capacity; ++i) cudaEventDestroy(h->prof->ev[i]);
+    free(h->prof->ev);
+    free(h->prof->cls);
+    free(h->prof);
+    h->prof = nullptr;
+  }
+  if (max_records == 0) return A3_OK;
+  Profiler* p = (Profiler*)calloc(1, sizeof(Profiler));
+  p->ev = (cudaEvent_t*)calloc(2 * (size_t)max_records, sizeof(cudaEvent_t));
+  p->cls = (int*)calloc(max_records, sizeof(int));
+  p->capacity = max_records;
+  for (int i = 0; i < 2 * max_records; ++i) {
+    cudaError_t e = cudaEventCreate(&p->ev[i]);
+    if (e != cudaSuccess) {
+      p->capacity = i / 2;
+      break;
+    }
+  }
+  h->prof = p;
+  return A3_OK;
+}
+
+extern "C" int a3_profile_read(a3_handle* h, a3_profile_entry* out, a3_stream stream) {
+  if (!h || !out) return A3_EINVAL;
+  for (int k = 0; k < A3_K_CLASSES; ++k) out[k] = a3_profile_entry{0, 0.0};
+  A3_CUDA(cudaStreamSynchronize((cudaStream_t)stream));
+  Profiler* p = h->prof;
+  if (!p) return A3_OK;
+  for (int i = 0; i < p->used; ++i) {
+    float ms = 0.f;
+    A3_CUDA(cudaEventElapsedTime(&ms, p->ev[2 * i], p->ev[2 * i + 1]));
+    out[p->cls[i]].launches += 1;
+    out[p->cls[i]].ms += ms;
+  }
+  p->used = 0;
+  return A3_OK;
+}
+
+extern "C" const char* a3_kernel_class_name(int cls) {
+  static const char* names[A3_K_CLASSES] = {"rerotate", "rmsnorm", "gemm_qkv", "attention", "gemm_residual",
+                                            "gemm_swiglu", "scores", "topk", "rows"};
+  return cls >= 0 && cls < A3_K_CLASSES ? names[cls] : "?";
+}
+
 extern "C" void a3_destroy(a3_handle* h) {
   if (!h) return;
+  a3_profile_enable(h, 0);
   if (h->rope_tab) cudaFree(h->rope_tab);
   if (h->dev_status) cudaFree(h->dev_status);
   free(h->layers);
@@ -212,7 +260,7 @@ static int recompute_layer_impl(const a3_handle* h, int layer, bf16* x, const in
   const a3_model_desc& m = h->m;
   const a3_layer_weights& lw = h->layers[layer];
   const int qd = m.n_q_heads * m.head_dim;
-  A3_TRY(rmsnorm_rows(x, (const bf16*)lw.attn_norm, m.rms_eps, M, m.d_model, w.a, st));
+  A3_TRY(rmsnorm_rows(h, x, (const bf16*)lw.attn_norm, m.rms_eps, M, m.d_model, w.a, st));
   A3_TRY(qkv_project(h, layer, w.a, pos, M, 0, w.q, kc, vc, kv_len, st));
   A3_TRY(attention_rows(h, w.q, pos, M, kc, vc, kv_len, w.o, lse_out, st));
   GemmArgs g{};
@@ -224,7 +272,7 @@ static int recompute_layer_impl(const a3_handle* h, int layer, bf16* x, const in
   g.C = x;
   g.ldc = m.d_model;
   A3_TRY(gemm_bf16(h, EPI_RESIDUAL, g, st));
-  A3_TRY(rmsnorm_rows(x, (const bf16*)lw.mlp_norm, m.rms_eps, M, m.d_model, w.a, st));
+  A3_TRY(rmsnorm_rows(h, x, (const bf16*)lw.mlp_norm, m.rms_eps, M, m.d_model, w.a, st));
   GemmArgs u{};
   u.A = w.a;
   u.M = M;
@@ -311,11 +359,11 @@ extern "C" int a3_fuse_request(const a3_handle* h, const a3_request* r, void* ws
                           m.n_layers, stream));
   // leading full blocks: the whole input through layers 0..select_layer-1
   A3_CUDA(cudaMemcpyAsync(w.x_all, r->x0, (size_t)n * m.d_model * 2, cudaMemcpyDeviceToDevice, st));
-  A3_TRY(iota_rows(w.all_pos, 0, n, st));
+  A3_TRY(iota_rows(h, w.all_pos, 0, n, st));
   for (int l = 0; l < ls; ++l)
     A3_TRY(recompute_layer_impl(h, l, w.x_all, w.all_pos, n, kl(l), vl(l), n, nullptr, lw, st));
   // selection layer: true K, V for all rows, queries of the question rows, scores, Re (Eq. 3)
-  A3_TRY(rmsnorm_rows(w.x_all, (const bf16*)h->layers[ls].attn_norm, m.rms_eps, n, m.d_model, lw.a, st));
+  A3_TRY(rmsnorm_rows(h, w.x_all, (const bf16*)h->layers[ls].attn_norm, m.rms_eps, n, m.d_model, lw.a, st));
   A3_TRY(qkv_project(h, ls, lw.a, w.all_pos, n, r->n_ctx, lw.q, kl(ls), vl(ls), n, st));
   A3_CUDA(cudaMemsetAsync(r->scores_out, 0, (size_t)n * 4, st));
   if (nq > 0) {
@@ -326,7 +374,7 @@ extern "C" int a3_fuse_request(const a3_handle* h, const a3_request* r, void* ws
     if (r->forced_re) A3_CUDA(cudaMemcpyAsync(r->rows_out, r->forced_re, (size_t)p * 4, cudaMemcpyDeviceToDevice, st));
     else A3_TRY(a3_topk_select(h, r->scores_out, r->n_system, r->n_ctx, p, r->rows_out, stream));
   }
-  A3_TRY(iota_rows(r->rows_out + p, r->n_ctx, nq, st));
+  A3_TRY(iota_rows(h, r->rows_out + p, r->n_ctx, nq, st));
   if (M == 0) return A3_OK;
   A3_TRY(check_rows(h, r->rows_out, M, n, st));
   A3_TRY(a3_gather_rows(h, w.x_all, n, r->rows_out, M, m.d_model, r->x_out, stream));

@@ -236,6 +236,7 @@ int attention_rows(const a3_handle* h, const bf16* q, const int32_t* pos, int M,
     A3_CUDA(cudaFuncSetAttribute(attention_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, 5 * 64 * 64 * 2));
     attr_set = true;
   }
+  ProfScope prof(h, A3_K_ATTENTION, st);
   if (D == 128) attention_kernel<128><<<grid, AT_THREADS, smem, st>>>(q, pos, M, k, v, kv_len, o, lse, Hq, Hkv, scale_log2);
   else attention_kernel<64><<<grid, AT_THREADS, smem, st>>>(q, pos, M, k, v, kv_len, o, lse, Hq, Hkv, scale_log2);
   A3_LAUNCHED();
@@ -334,6 +335,7 @@ int scores_pass(const a3_handle* h, const bf16* q, const int32_t* q_pos, int nq,
   const int Hq = h->m.n_q_heads, Hkv = h->m.n_kv_heads, D = h->m.head_dim;
   const float scale_log2 = LOG2E / sqrtf((float)D);
   dim3 grid(cdiv(kv_len, AT_BN));
+  ProfScope prof(h, A3_K_SCORES, st);
   if (D == 128) scores_kernel<128><<<grid, AT_THREADS, 0, st>>>(q, q_pos, nq, k, kv_len, cand_begin, cand_end, lse, scores, Hq, Hkv, scale_log2);
   else scores_kernel<64><<<grid, AT_THREADS, 0, st>>>(q, q_pos, nq, k, kv_len, cand_begin, cand_end, lse, scores, Hq, Hkv, scale_log2);
   A3_LAUNCHED();

@@ -285,6 +285,7 @@ int gemm_bf16(const a3_handle* h, GemmEpilogue epi, const GemmArgs& a, cudaStrea
     A3_CUDA(cudaFuncSetAttribute(gemm_mma_kernel<EPI_QKV>, cudaFuncAttributeMaxDynamicSharedMemorySize, GEMM_SMEM));
     attr_set = true;
   }
+  ProfScope prof(h, epi == EPI_RESIDUAL ? A3_K_GEMM_RESIDUAL : epi == EPI_SWIGLU ? A3_K_GEMM_SWIGLU : A3_K_GEMM_QKV, st);
   if (epi == EPI_RESIDUAL) gemm_mma_kernel<EPI_RESIDUAL><<<grid, GEMM_THREADS, GEMM_SMEM, st>>>(p);
   else if (epi == EPI_SWIGLU) gemm_mma_kernel<EPI_SWIGLU><<<grid, GEMM_THREADS, GEMM_SMEM, st>>>(p);
   else gemm_mma_kernel<EPI_QKV><<<grid, GEMM_THREADS, GEMM_SMEM, st>>>(p);

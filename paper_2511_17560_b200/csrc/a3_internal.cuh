@@ -9,6 +9,8 @@
 
 typedef __nv_bfloat16 bf16;
 
+namespace a3 { struct Profiler; }
+
 struct a3_handle {
   a3_model_desc m;
   a3_layer_weights* layers;  // host copy [n_layers]
@@ -17,6 +19,7 @@ struct a3_handle {
   int device;
   int sm_count;
   void* tmaps;               // host-side tensor-map cache (a3_gemm_tc.cu)
+  a3::Profiler* prof;        // null unless a3_profile_enable is on
 };
 
 namespace a3 {
@@ -52,13 +55,38 @@ inline int launched() {
     if (s_ != A3_OK) return s_;       \
   } while (0)
 
+// Event pair around one launch (only when profiling is enabled on the handle).
+struct Profiler {
+  cudaEvent_t* ev;
+  int* cls;
+  int capacity, used;  // in records (two events each)
+};
+struct ProfScope {
+  Profiler* p;
+  cudaStream_t st;
+  ProfScope(const a3_handle* h, int k, cudaStream_t s) : p(h ? h->prof : nullptr), st(s) {
+    if (p && p->used < p->capacity) {
+      p->cls[p->used] = k;
+      cudaEventRecord(p->ev[2 * p->used], st);
+    } else {
+      p = nullptr;
+    }
+  }
+  ~ProfScope() {
+    if (p) {
+      cudaEventRecord(p->ev[2 * p->used + 1], st);
+      ++p->used;
+    }
+  }
+};
+
 inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 inline int cdiv(long long a, long long b) { return (int)((a + b - 1) / b); }
 
 // ---------------------------------------------------------------- internal step launchers
 
 // out[m] = rmsnorm(x[m]) * gain, rows of width d.
-int rmsnorm_rows(const bf16* x, const bf16* gain, float eps, int M, int d, bf16* out, cudaStream_t st);
+int rmsnorm_rows(const a3_handle* h, const bf16* x, const bf16* gain, float eps, int M, int d, bf16* out, cudaStream_t st);
 
 enum GemmEpilogue { EPI_RESIDUAL = 0, EPI_SWIGLU = 1, EPI_QKV = 2 };
 
@@ -96,7 +124,7 @@ int attention_rows(const a3_handle* h, const bf16* q, const int32_t* pos, int M,
 int scores_pass(const a3_handle* h, const bf16* q, const int32_t* q_pos, int nq, const bf16* k, int kv_len,
                 int cand_begin, int cand_end, const float* lse, float* scores, cudaStream_t st);
 
-int iota_rows(int32_t* out, int begin, int count, cudaStream_t st);
+int iota_rows(const a3_handle* h, int32_t* out, int begin, int count, cudaStream_t st);
 int check_rows(const a3_handle* h, const int32_t* pos, int M, int kv_len, cudaStream_t st);
 
 }  // namespace a3

@@ -159,6 +159,7 @@ extern "C" int a3_rope_rerotate(const a3_handle* h, const a3_chunk_ref* chunks, 
   rerotate_kernel<DD, LL><<<grid, RR_THREADS, 0, st>>>(chunks, (char*)k_fused, (char*)v_fused, layer_stride,          \
                                                        layer_begin, row_elems, tok, h->rope_tab, h->m.max_positions, \
                                                        h->dev_status)
+  ProfScope prof(h, A3_K_REROTATE, st);
   if (h->m.head_dim == 128 && h->m.rope_layout == 0) RR_LAUNCH(128, 0);
   else if (h->m.head_dim == 128) RR_LAUNCH(128, 1);
   else if (h->m.head_dim == 64 && h->m.rope_layout == 0) RR_LAUNCH(64, 0);
@@ -217,8 +218,9 @@ __global__ void check_rows_kernel(const int32_t* pos, int M, int kv_len, uint32_
   if (i > 0 && pos[i - 1] >= p) atomicOr(status, A3_DEV_UNSORTED_ROWS);
 }
 
-int iota_rows(int32_t* out, int begin, int count, cudaStream_t st) {
+int iota_rows(const a3_handle* h, int32_t* out, int begin, int count, cudaStream_t st) {
   if (count <= 0) return A3_OK;
+  ProfScope prof(h, A3_K_ROWS, st);
   iota_kernel<<<cdiv(count, 256), 256, 0, st>>>(out, begin, count);
   A3_LAUNCHED();
   return A3_OK;
@@ -226,6 +228,7 @@ int iota_rows(int32_t* out, int begin, int count, cudaStream_t st) {
 
 int check_rows(const a3_handle* h, const int32_t* pos, int M, int kv_len, cudaStream_t st) {
   if (M <= 0) return A3_OK;
+  ProfScope prof(h, A3_K_ROWS, st);
   check_rows_kernel<<<cdiv(M, 256), 256, 0, st>>>(pos, M, kv_len, h->dev_status);
   A3_LAUNCHED();
   return A3_OK;
@@ -264,8 +267,9 @@ rmsnorm_kernel(const uint4* __restrict__ x, const uint4* __restrict__ gain, floa
   }
 }
 
-int rmsnorm_rows(const bf16* x, const bf16* gain, float eps, int M, int d, bf16* out, cudaStream_t st) {
+int rmsnorm_rows(const a3_handle* h, const bf16* x, const bf16* gain, float eps, int M, int d, bf16* out, cudaStream_t st) {
   if (M <= 0) return A3_OK;
+  ProfScope prof(h, A3_K_RMSNORM, st);
   rmsnorm_kernel<<<M, RN_THREADS, 0, st>>>((const uint4*)x, (const uint4*)gain, eps, d / 8, (uint4*)out);
   A3_LAUNCHED();
   return A3_OK;
@@ -281,6 +285,7 @@ extern "C" int a3_scatter_kv(const a3_handle* h, const void* k_rows, const void*
   if (((uintptr_t)k_rows | (uintptr_t)v_rows | (uintptr_t)k_layer | (uintptr_t)v_layer) & 15) return A3_EINVAL;
   const int row_vecs = h->m.n_kv_heads * h->m.head_dim / 8;
   const int rows_per_cta = row_vecs >= 256 ? 1 : 256 / row_vecs;
+  ProfScope prof(h, A3_K_ROWS, (cudaStream_t)stream);
   scatter_kv_kernel<<<cdiv(M, rows_per_cta), 256, 0, (cudaStream_t)stream>>>(
       (const uint4*)k_rows, (const uint4*)v_rows, slots, M, row_vecs, (uint4*)k_layer, (uint4*)v_layer, kv_len, h->dev_status);
   A3_LAUNCHED();
@@ -293,6 +298,7 @@ extern "C" int a3_gather_rows(const a3_handle* h, const void* src, int n_src, co
   if (M == 0) return A3_OK;
   if (!src || !rows || !dst) return A3_EINVAL;
   if (((uintptr_t)src | (uintptr_t)dst) & 15) return A3_EINVAL;
+  ProfScope prof(h, A3_K_ROWS, (cudaStream_t)stream);
   gather_rows_kernel<<<M, 256, 0, (cudaStream_t)stream>>>((const uint4*)src, n_src, rows, M, width / 8, (uint4*)dst, h->dev_status);
   A3_LAUNCHED();
   return A3_OK;

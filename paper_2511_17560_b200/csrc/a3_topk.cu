@@ -112,6 +112,7 @@ extern "C" int a3_topk_select(const a3_handle* h, const float* scores, int cand_
   if (k > n) k = n;
   if (k == 0) return A3_OK;
   if (!scores || !idx_out) return A3_EINVAL;
+  ProfScope prof(h, A3_K_TOPK, (cudaStream_t)stream);
   topk_select_kernel<<<1, TK_THREADS, 0, (cudaStream_t)stream>>>(scores, cand_begin, n, k, idx_out, h->dev_status);
   A3_LAUNCHED();
   return A3_OK;
