@@ -244,7 +244,7 @@ gemm_mma_kernel(const GemmDev p) {
   }
 }
 
-int gemm_bf16(const a3_handle* h, GemmEpilogue epi, const GemmArgs& a, cudaStream_t st) {
+static int gemm_bf16_mma(const a3_handle* h, GemmEpilogue epi, const GemmArgs& a, cudaStream_t st) {
   if (a.M <= 0) return A3_OK;
   if (a.K % BK) return A3_EUNSUPPORTED;
   GemmDev p{};
@@ -293,4 +293,15 @@ int gemm_bf16(const a3_handle* h, GemmEpilogue epi, const GemmArgs& a, cudaStrea
   return A3_OK;
 }
 
+int gemm_bf16_tc(const a3_handle* h, GemmEpilogue epi, const GemmArgs& a, cudaStream_t st);
+
+// 0: tcgen05 kernel (a3_gemm_tc.cu); 1: the warp-level mma.sync kernel above, kept as a cross-check for bring-up
+int g_gemm_impl = 0;
+
+int gemm_bf16(const a3_handle* h, GemmEpilogue epi, const GemmArgs& a, cudaStream_t st) {
+  return g_gemm_impl == 1 ? gemm_bf16_mma(h, epi, a, st) : gemm_bf16_tc(h, epi, a, st);
+}
+
 }  // namespace a3
+
+extern "C" void a3_internal_set_gemm_impl(int impl) { a3::g_gemm_impl = impl; }
