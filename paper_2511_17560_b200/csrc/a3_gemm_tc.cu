@@ -22,7 +22,7 @@ constexpr int TC_BM = 128, TC_BK = 64, TC_THREADS = 192;
 constexpr unsigned long long TC_WAIT_NS = 500000000ull;
 
 struct TcParams {
-  int M, K;
+  int M, K, N;
   int seg_tiles_end[3];
   int kind[3];
   const bf16* bias[3];
@@ -149,6 +149,7 @@ __global__ void __launch_bounds__(TC_THREADS)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB0,
                const __grid_constant__ CUtensorMap tmB1, const __grid_constant__ CUtensorMap tmB2, const TcParams p) {
   using L = TcLayout<BN, STAGES>;
+  constexpr int TMEM_COLS = BN <= 128 ? 128 : 256;  // allocations are powers of two
   extern __shared__ unsigned char smem_raw[];
   const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   unsigned char* base_ptr = smem_raw + (base - smem_u32(smem_raw));
@@ -186,7 +187,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
   }
   if (warp == 1) {
-    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32((const void*)tmem_slot)), "r"(BN) : "memory");
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32((const void*)tmem_slot)), "r"(TMEM_COLS) : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
   }
   tc_fence_before();
@@ -260,10 +261,11 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
           __syncwarp();
           float acc[32], old[32];
           tc_ld32(trow + c * 32, acc);
-          bf16* cp = p.C + (size_t)(row_ok ? gr : 0) * p.ldc + n0 + c * 32;
-          if (row_ok) load32_bf16(cp, old);
+          const bool col_ok = row_ok && n0 + c * 32 < p.N;  // tiles need not divide N: TMA zero-fills, stores are cut
+          bf16* cp = p.C + (size_t)(row_ok ? gr : 0) * p.ldc + (col_ok ? n0 + c * 32 : 0);
+          if (col_ok) load32_bf16(cp, old);
           tc_wait_ld();
-          if (row_ok) {
+          if (col_ok) {
 #pragma unroll
             for (int e = 0; e < 32; ++e) acc[e] += old[e];
             store32_bf16(cp, acc);
@@ -352,7 +354,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
   }
   tc_fence_before();
   __syncthreads();
-  if (warp == 1) asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(BN) : "memory");
+  if (warp == 1) asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(TMEM_COLS) : "memory");
 }
 
 // ---------------------------------------------------------------- host side
@@ -417,24 +419,65 @@ static int launch_tc(const a3_handle* h, const GemmArgs& a, const TcParams& p, i
   return A3_OK;
 }
 
+// Tile width / pipeline depth per epilogue [EPI_RESIDUAL, EPI_SWIGLU, EPI_QKV] -> {BN, STAGES}; BN = 0 lets the
+// launcher choose (a3_internal_set_gemm_cfg pins a choice for tuning runs).  Measured on B200 at Llama-8B width:
+// two co-resident CTAs per SM (256/2, 128/3) overlap one tile's epilogue with the other's main loop and win when
+// the grid has several waves; a single wave prefers the widest tile that still gives every SM at most one CTA.
+int g_tc_cfg[3][2] = {{0, 0}, {256, 2}, {0, 0}};
+
+template <int EPI>
+static int dispatch_tc(const a3_handle* h, const GemmArgs& a, const TcParams& p, int tiles, int bn, int stages, cudaStream_t st) {
+  if (bn == 256 && stages == 4) return launch_tc<EPI, 256, 4>(h, a, p, tiles, st);
+  if (bn == 256 && stages == 3) return launch_tc<EPI, 256, 3>(h, a, p, tiles, st);
+  if (bn == 256 && stages == 2) return launch_tc<EPI, 256, 2>(h, a, p, tiles, st);
+  if (bn == 224 && stages == 4) return launch_tc<EPI, 224, 4>(h, a, p, tiles, st);
+  if (bn == 192 && stages == 4) return launch_tc<EPI, 192, 4>(h, a, p, tiles, st);
+  if (bn == 128 && stages == 3) return launch_tc<EPI, 128, 3>(h, a, p, tiles, st);
+  if (bn == 128 && stages == 6) return launch_tc<EPI, 128, 6>(h, a, p, tiles, st);
+  return launch_tc<EPI, 128, 4>(h, a, p, tiles, st);
+}
+
 int gemm_bf16_tc(const a3_handle* h, GemmEpilogue epi, const GemmArgs& a, cudaStream_t st) {
   if (a.M <= 0) return A3_OK;
   if (a.K % TC_BK) return A3_EUNSUPPORTED;
-  constexpr int BN_RES = 128, BN_SWI = 256, BN_QKV = 128;
-  const int bn = epi == EPI_RESIDUAL ? BN_RES : epi == EPI_SWIGLU ? BN_SWI / 2 : BN_QKV;  // output columns per tile
+  int bn = g_tc_cfg[epi][0];
+  int stages = g_tc_cfg[epi][1];
+  if (bn == 0) {
+    const int m_tiles = cdiv(a.M, TC_BM), sms = h->sm_count > 0 ? h->sm_count : 148;
+    if (epi == EPI_RESIDUAL) {
+      // when a single wave of CTAs covers the output either way, the narrower 224-column tile shortens it
+      const int n = a.seg[0].n;
+      bn = (m_tiles * cdiv(n, 256) <= sms && m_tiles * cdiv(n, 224) <= sms) ? 224 : 256;
+      stages = 4;
+    } else {
+      bn = 256;
+      stages = 4;
+    }
+  }
+  // output columns per tile; QKV tiles must hold whole heads and divide every segment
+  int out_cols = epi == EPI_SWIGLU ? bn / 2 : bn;
+  if (epi == EPI_QKV) {
+    for (int s = 0; s < a.nseg; ++s)
+      if (a.seg[s].n % out_cols) {
+        bn = out_cols = 128;
+        stages = 3;
+      }
+  }
   TcParams p{};
   p.M = a.M;
   p.K = a.K;
   int tiles = 0;
   for (int s = 0; s < 3; ++s) {
     if (s < a.nseg) {
-      if (a.seg[s].n % bn) return A3_EUNSUPPORTED;
+      if (epi != EPI_RESIDUAL && a.seg[s].n % out_cols) return A3_EUNSUPPORTED;
+      if (a.seg[s].n % 32) return A3_EUNSUPPORTED;
       p.bias[s] = a.seg[s].bias;
       p.kind[s] = a.seg[s].kind;
-      tiles += a.seg[s].n / bn;
+      tiles += cdiv(a.seg[s].n, out_cols);
     }
     p.seg_tiles_end[s] = tiles;
   }
+  p.N = a.seg[0].n;
   p.C = a.C;
   p.ldc = a.ldc;
   p.q_out = a.q_out;
@@ -449,9 +492,16 @@ int gemm_bf16_tc(const a3_handle* h, GemmEpilogue epi, const GemmArgs& a, cudaSt
   p.max_pos = h->m.max_positions;
   p.tab = h->rope_tab;
   p.status = h->dev_status;
-  if (epi == EPI_RESIDUAL) return launch_tc<EPI_RESIDUAL, BN_RES, 4>(h, a, p, tiles, st);
-  if (epi == EPI_SWIGLU) return launch_tc<EPI_SWIGLU, BN_SWI, 4>(h, a, p, tiles, st);
-  return launch_tc<EPI_QKV, BN_QKV, 4>(h, a, p, tiles, st);
+  if (epi == EPI_RESIDUAL) return dispatch_tc<EPI_RESIDUAL>(h, a, p, tiles, bn, stages, st);
+  if (epi == EPI_SWIGLU) return dispatch_tc<EPI_SWIGLU>(h, a, p, tiles, bn, stages, st);
+  return dispatch_tc<EPI_QKV>(h, a, p, tiles, bn, stages, st);
 }
 
 }  // namespace a3
+
+extern "C" void a3_internal_set_gemm_cfg(int epi, int bn, int stages) {
+  if (epi >= 0 && epi < 3) {
+    a3::g_tc_cfg[epi][0] = bn;
+    a3::g_tc_cfg[epi][1] = stages;
+  }
+}
