@@ -47,7 +47,8 @@ typedef enum {
   A3_EUNSUPPORTED = -2, /* shape outside the supported set */
   A3_EWORKSPACE = -3,   /* workspace too small */
   A3_ECUDA = -4,        /* a CUDA call failed; see a3_last_cuda_error */
-  A3_EDEVICE = -5       /* a kernel recorded a problem in the device status word */
+  A3_EDEVICE = -5,      /* a kernel recorded a problem in the device status word */
+  A3_ETOOLARGE = -6     /* the request exceeds a fixed built-in limit (a3_query_scores_static) */
 } a3_status;
 
 /* Device status bits (a3_device_status). */
@@ -148,6 +149,21 @@ int a3_rope_rerotate(const a3_handle* h, const a3_chunk_ref* chunks, int n_chunk
 int a3_query_scores(const a3_handle* h, const void* q_rows, const int32_t* q_pos, int nq, const void* k_layer,
                     int kv_len, int cand_begin, int cand_end, const float* lse, float* scores, void* ws,
                     size_t ws_bytes, a3_stream stream);
+
+/* a3_query_scores without a workspace, for callers that cannot allocate device memory where they need the
+ * scores (for example a serving engine that gave all free HBM to its KV-cache pool at start-up, or plug-in code
+ * inside a framework that owns the allocator).  The paper has no counterpart: this is a packaging variant of the
+ * call above, with the same arguments minus lse/ws and the same result.  The row log-sum-exps go to a fixed
+ * array inside the library image: A3_STATIC_LSE_MAX floats (256 KiB) that every GPU which loads the library
+ * holds until the process exits.  nq * n_q_heads above that limit returns A3_ETOOLARGE and launches nothing.
+ * The call makes no allocation of any kind.  Its first call on a device looks up the array's device address
+ * (once per device; that device must be current and must be the handle's) and should therefore be made before
+ * any stream capture begins.  All calls share the array; it keeps the previous call's contents, and nothing in
+ * it needs clearing because each call overwrites the entries it later reads.  Calls whose kernels may overlap
+ * on the GPU race on it: order them. */
+#define A3_STATIC_LSE_MAX 65536
+int a3_query_scores_static(const a3_handle* h, const void* q_rows, const int32_t* q_pos, int nq, const void* k_layer,
+                           int kv_len, int cand_begin, int cand_end, float* scores, a3_stream stream);
 
 /* Selection (Eq. 3, Re = top_p(s)): the k slots of [cand_begin, cand_end) with the largest score;
  * ties go to the lower slot; idx_out (dev [k]) is ascending.  k is clamped to the candidate count. */

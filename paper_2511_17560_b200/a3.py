@@ -62,7 +62,7 @@ class HostIO(C.Structure):
 
 
 EXPORTS = ("a3_create", "a3_destroy", "a3_layer_workspace_bytes", "a3_request_workspace_bytes", "a3_host_staging_bytes",
-           "a3_recompute_count", "a3_rope_rerotate", "a3_query_scores", "a3_topk_select", "a3_recompute_layer",
+           "a3_recompute_count", "a3_rope_rerotate", "a3_query_scores", "a3_query_scores_static", "a3_topk_select", "a3_recompute_layer",
            "a3_scatter_kv", "a3_gather_rows", "a3_fuse_request", "a3_fuse_batch", "a3_fuse_request_host",
            "a3_device_status", "a3_status_string", "a3_last_cuda_error", "a3_launch_count", "a3_profile_enable",
            "a3_profile_read", "a3_kernel_class_name")
@@ -93,6 +93,7 @@ def _load():
     lib.a3_recompute_count.argtypes = [C.c_double, i32, i32]
     lib.a3_rope_rerotate.argtypes = [vp, vp, i32, i32, vp, vp, u64, i32, i32, vp]
     lib.a3_query_scores.argtypes = [vp, vp, vp, i32, vp, i32, i32, i32, vp, vp, vp, sz, vp]
+    lib.a3_query_scores_static.argtypes = [vp, vp, vp, i32, vp, i32, i32, i32, vp, vp]
     lib.a3_topk_select.argtypes = [vp, vp, i32, i32, i32, vp, vp]
     lib.a3_recompute_layer.argtypes = [vp, i32, vp, vp, i32, vp, vp, i32, vp, vp, sz, vp]
     lib.a3_scatter_kv.argtypes = [vp, vp, vp, vp, i32, vp, vp, i32, vp]
@@ -218,6 +219,19 @@ class A3:
         _check(_load().a3_query_scores(self._h, _ptr(q_rows), _ptr(q_pos), nq, _ptr(k_layer), kv_len, cand_begin,
                                        cand_end, _ptr(lse), _ptr(scores), _ptr(ws), ws.numel(), _stream()),
                "a3_query_scores")
+        return scores
+
+    def query_scores_static(self, q_rows, q_pos, k_layer, cand_begin, cand_end, scores=None):
+        """a3_query_scores for callers that cannot allocate: no workspace, scratch inside the library image.
+
+        Limited to q_rows.shape[0] * n_q_heads <= 65536; calls that may overlap on the GPU must be ordered by the
+        caller because they share that scratch.  Only `scores` (an output) is created here when not supplied.
+        """
+        nq, kv_len = q_rows.shape[0], k_layer.shape[0]
+        if scores is None:
+            scores = torch.empty(kv_len, dtype=torch.float32, device=k_layer.device)
+        _check(_load().a3_query_scores_static(self._h, _ptr(q_rows), _ptr(q_pos), nq, _ptr(k_layer), kv_len, cand_begin,
+                                              cand_end, _ptr(scores), _stream()), "a3_query_scores_static")
         return scores
 
     def topk_select(self, scores, cand_begin, cand_end, k, idx_out=None):

@@ -69,6 +69,7 @@ extern "C" const char* a3_status_string(int s) {
     case A3_EWORKSPACE: return "workspace too small";
     case A3_ECUDA: return "CUDA call failed";
     case A3_EDEVICE: return "device status word set";
+    case A3_ETOOLARGE: return "size exceeds a fixed built-in limit";
     default: return "unknown status";
   }
 }
