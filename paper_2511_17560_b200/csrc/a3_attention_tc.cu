@@ -1,0 +1,446 @@
+// Attention of the carried rows over the fused GQA cache (Eq. 4, Eq. 5) on the 5th-generation tensor cores.
+//
+// Row m sits at global position pos[m] and sees cache slots 0..pos[m].  The G = Hq/Hkv query heads that share one
+// KV head are packed into the row dimension (flat row r -> token r / G, head r % G); one CTA owns 128 flat rows of
+// one KV head and walks the keys in tiles of 128 up to the largest position among its rows.
+//
+//   warp 0 (one lane)   TMA producer: K and V tiles of the cache ([slots][Hkv*D] seen as a 2-D tensor, 128-byte
+//                       swizzle, two stages).
+//   warp 1 (one lane)   tcgen05.mma issuer: S = Q K^T (128 x 128 x D) into one of two TMEM buffers, and, once the
+//                       probabilities of a tile are in shared memory, O~ = P V (128 x D x 128, V as an MN-major
+//                       operand) into a third TMEM buffer.  S of tile t+1 is issued before P V of tile t, so the
+//                       tensor core works while the softmax threads do.
+//   warps 2..5          one thread per row: two passes over the row of S in TMEM (maximum, then exp2 and sum), P
+//                       written as bf16 into shared memory in the swizzled K-major layout the MMA reads, running
+//                       rescale of the output kept in registers (O = O * alpha + O~), final normalisation, stores.
+// Statistics are fp32 in the exp2 domain.  Every mbarrier wait is bounded (see a3_gemm_tc.cu); there is no block-
+// wide or named barrier inside the loops, so a role that gives up cannot strand another.
+#include <cuda.h>
+
+#include "a3_internal.cuh"
+
+namespace a3 {
+
+constexpr int ATC_THREADS = 192;
+constexpr int ATC_BM = 128, ATC_BN = 128;
+constexpr unsigned long long ATC_WAIT_NS = 500000000ull;
+constexpr float ATC_LOG2E = 1.4426950408889634f, ATC_LN2 = 0.6931471805599453f;
+
+namespace atc {
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ uint32_t mbar_try_wait(uint32_t bar, uint32_t parity) {
+  uint32_t done;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.b32 %0, 1, 0, p;\n\t}"
+      : "=r"(done)
+      : "r"(bar), "r"(parity)
+      : "memory");
+  return done;
+}
+__device__ __forceinline__ unsigned long long global_ns() {
+  unsigned long long t;
+  asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
+  return t;
+}
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, uint32_t* status) {
+  if (mbar_try_wait(bar, parity)) return true;
+  const unsigned long long t0 = global_ns();
+  for (;;) {
+#pragma unroll 1
+    for (int i = 0; i < 32; ++i)
+      if (mbar_try_wait(bar, parity)) return true;
+    if (*abort_flag) return false;
+    if (global_ns() - t0 > ATC_WAIT_NS) {
+      *abort_flag = 1;
+      atomicOr(status, A3_DEV_WAIT_EXHAUSTED);
+      return false;
+    }
+  }
+}
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int x, int y, uint32_t bar) {
+  asm volatile("cp.async.bulk.tensor.2d.shared::cta.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+               ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(bar)
+               : "memory");
+}
+__device__ __forceinline__ void fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+__device__ __forceinline__ void commit(uint32_t bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void mma_f16(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+      ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+__device__ __forceinline__ void ld32(uint32_t taddr, float* v) {
+  uint32_t* r = reinterpret_cast<uint32_t*>(v);
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+        "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]),
+        "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]),
+        "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+      : "r"(taddr)
+      : "memory");
+}
+__device__ __forceinline__ void wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+
+// K-major [rows][64] bf16 sub-tile, 128-byte swizzle, 8-row groups 1024 bytes apart
+__device__ __forceinline__ uint64_t desc_k_sw128(uint32_t saddr) {
+  return (uint64_t)((saddr & 0x3FFFFu) >> 4) | ((uint64_t)(1024u >> 4) << 32) | (1ull << 46) | (2ull << 61);
+}
+// MN-major operand stored as [k rows][64 mn elements] sub-tiles (one 128-byte row per k), 128-byte swizzle:
+// 8-k-row groups are 1024 bytes apart (SBO), successive 64-element mn atoms `lbo` bytes apart (LBO)
+__device__ __forceinline__ uint64_t desc_mn_sw128(uint32_t saddr, uint32_t lbo) {
+  return (uint64_t)((saddr & 0x3FFFFu) >> 4) | ((uint64_t)((lbo >> 4) & 0x3FFFu) << 16) | ((uint64_t)(1024u >> 4) << 32) |
+         (1ull << 46) | (2ull << 61);
+}
+// bf16 x bf16 -> fp32, M = 128, A K-major; b_mn = 1 when B is MN-major
+__host__ __device__ constexpr uint32_t idesc(int n, int b_mn) {
+  return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)b_mn << 16) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(ATC_BM >> 4) << 24);
+}
+// byte offset of element chunk (16 bytes) j of row r inside a [rows][64] bf16 sub-tile with the 128-byte swizzle
+__device__ __forceinline__ uint32_t swz(int r, int j) { return (uint32_t)(r * 128 + ((j ^ (r & 7)) << 4)); }
+}  // namespace atc
+
+template <int D>
+struct AtcLayout {
+  static constexpr int SUB = 128 * 64 * 2;           // one [128][64] bf16 sub-tile: 16 KiB
+  static constexpr int Q_BYTES = (D / 64) * SUB;
+  static constexpr int KV_STAGE = 2 * (D / 64) * SUB;  // K then V
+  static constexpr int P_BYTES = 2 * SUB;
+  static constexpr int Q_OFF = 0;
+  static constexpr int KV_OFF = Q_BYTES;
+  static constexpr int P_OFF = KV_OFF + 2 * KV_STAGE;
+  static constexpr int BAR_OFF = P_OFF + P_BYTES;
+  static constexpr int SMEM_BYTES = BAR_OFF + 256 + 1024;
+};
+
+template <int D>
+__global__ void __launch_bounds__(ATC_THREADS)
+attention_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV,
+                    const bf16* __restrict__ q, const int32_t* __restrict__ pos, int M, int kv_len, bf16* __restrict__ o,
+                    float* __restrict__ lse, int Hq, int Hkv, float scale_log2, uint32_t* status) {
+  using L = AtcLayout<D>;
+  using namespace atc;
+  extern __shared__ unsigned char smem_raw[];
+  const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+  unsigned char* base_ptr = smem_raw + (base - smem_u32(smem_raw));
+  // barriers: kv_full[2], kv_empty[2], s_full[2], o_full, p_ready, q_ready
+  const uint32_t bars = base + L::BAR_OFF;
+  auto kv_full = [&](int s) { return bars + 8u * s; };
+  auto kv_empty = [&](int s) { return bars + 8u * (2 + s); };
+  auto s_full = [&](int b) { return bars + 8u * (4 + b); };
+  const uint32_t o_full = bars + 8u * 6, p_ready = bars + 8u * 7, q_ready = bars + 8u * 8;
+  volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(base_ptr + L::BAR_OFF + 8 * 9);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(base_ptr + L::BAR_OFF + 8 * 9 + 8);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int G = Hq / Hkv;
+  const int g = blockIdx.y;
+  const int tile = gridDim.x - 1 - blockIdx.x;  // latest (longest) row tiles first
+  const int r0 = tile * ATC_BM;
+  const int rows_total = M * G;
+  const bool want_o = o != nullptr;
+
+  const int last_tok = min(M - 1, (r0 + ATC_BM - 1) / G);
+  const int maxpos = min(pos[last_tok], kv_len - 1);
+  const int minpos = pos[r0 / G];
+  const int nkt = maxpos < 0 ? 0 : maxpos / ATC_BN + 1;
+
+  if (threadIdx.x == 0) {
+    for (int i = 0; i < 2; ++i) {
+      mbar_init(kv_full(i), 1);
+      mbar_init(kv_empty(i), 1);
+      mbar_init(s_full(i), 1);
+    }
+    mbar_init(o_full, 1);
+    mbar_init(p_ready, 128);
+    mbar_init(q_ready, 128);
+    abort_flag[0] = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    fence_async_smem();
+  }
+  if (warp == 1) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32((const void*)tmem_slot)), "r"(512) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  fence_before();
+  __syncthreads();
+  fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+  const uint32_t tmem_s0 = tmem_base, tmem_o = tmem_base + 256;
+
+  if (warp == 0) {
+    // ---------------- TMA producer
+    if (lane == 0) {
+      asm volatile("prefetch.tensormap [%0];" ::"l"(&tmK) : "memory");
+      asm volatile("prefetch.tensormap [%0];" ::"l"(&tmV) : "memory");
+      for (int kt = 0; kt < nkt; ++kt) {
+        const int s = kt & 1;
+        if (!mbar_wait(kv_empty(s), ((kt >> 1) & 1) ^ 1, abort_flag, status)) break;
+        const uint32_t sk = base + L::KV_OFF + s * L::KV_STAGE, sv = sk + (D / 64) * L::SUB;
+        mbar_expect_tx(kv_full(s), L::KV_STAGE);
+#pragma unroll
+        for (int j = 0; j < D / 64; ++j) {
+          tma_load_2d(sk + j * L::SUB, &tmK, g * D + 64 * j, kt * ATC_BN, kv_full(s));
+          tma_load_2d(sv + j * L::SUB, &tmV, g * D + 64 * j, kt * ATC_BN, kv_full(s));
+        }
+      }
+    }
+  } else if (warp == 1) {
+    // ---------------- MMA issuer
+    if (lane == 0 && nkt > 0) {
+      constexpr uint32_t idesc_s = idesc(ATC_BN, 0);
+      constexpr uint32_t idesc_o = idesc(D, 1);
+      const uint32_t sq = base + L::Q_OFF, sp = base + L::P_OFF;
+      auto issue_s = [&](int kt) {
+        const uint32_t sk = base + L::KV_OFF + (kt & 1) * L::KV_STAGE;
+#pragma unroll
+        for (int k = 0; k < D / 16; ++k) {
+          const uint32_t sub = (k / 4) * L::SUB + (k % 4) * 32;
+          mma_f16(tmem_s0 + (kt & 1) * 128, desc_k_sw128(sq + sub), desc_k_sw128(sk + sub), idesc_s, k != 0);
+        }
+        commit(s_full(kt & 1));
+      };
+      bool ok = mbar_wait(q_ready, 0, abort_flag, status);
+      ok = ok && mbar_wait(kv_full(0), 0, abort_flag, status);
+      if (ok) {
+        fence_after();
+        issue_s(0);
+      }
+      for (int kt = 0; kt < nkt && ok; ++kt) {
+        if (kt + 1 < nkt) {
+          ok = mbar_wait(kv_full((kt + 1) & 1), ((kt + 1) >> 1) & 1, abort_flag, status);
+          if (!ok) break;
+          fence_after();
+          issue_s(kt + 1);
+        }
+        ok = mbar_wait(p_ready, kt & 1, abort_flag, status);
+        if (!ok) break;
+        fence_after();
+        if (want_o) {
+          const uint32_t sv = base + L::KV_OFF + (kt & 1) * L::KV_STAGE + (D / 64) * L::SUB;
+#pragma unroll
+          for (int k = 0; k < ATC_BN / 16; ++k) {
+            const uint64_t da = desc_k_sw128(sp + (k / 4) * L::SUB + (k % 4) * 32);
+            const uint64_t db = desc_mn_sw128(sv + k * 16 * 128, L::SUB);
+            mma_f16(tmem_o, da, db, idesc_o, k != 0);
+          }
+          commit(o_full);
+        }
+        commit(kv_empty(kt & 1));
+      }
+    }
+  } else {
+    // ---------------- softmax / epilogue: thread = row
+    const int quarter = warp & 3;
+    const int row = quarter * 32 + lane;
+    const int fr = r0 + row;
+    const bool row_ok = fr < rows_total;
+    const int tok = row_ok ? fr / G : 0;
+    const int hq = g * G + (row_ok ? fr % G : 0);
+    const int lim = row_ok ? min(pos[tok], kv_len - 1) : -1;
+    const uint32_t lane_addr = (uint32_t)(quarter * 32) << 16;
+
+    // Q row -> shared memory, swizzled K-major sub-tiles
+    {
+      const uint4* src = reinterpret_cast<const uint4*>(q + ((size_t)tok * Hq + hq) * D);
+#pragma unroll
+      for (int c = 0; c < D / 8; ++c) {
+        uint4 v = row_ok ? __ldg(src + c) : make_uint4(0, 0, 0, 0);
+        *reinterpret_cast<uint4*>(base_ptr + L::Q_OFF + (c / 8) * L::SUB + swz(row, c % 8)) = v;
+      }
+      fence_async_smem();
+      mbar_arrive(q_ready);
+    }
+
+    float o_reg[D];
+#pragma unroll
+    for (int e = 0; e < D; ++e) o_reg[e] = 0.f;
+    float m_run = -INFINITY, l_run = 0.f, alpha_prev = 0.f;
+    bool ok = true;
+
+    for (int kt = 0; kt < nkt; ++kt) {
+      // the result of every wait is made warp-uniform: tcgen05.ld is a warp-wide instruction
+      ok = __all_sync(0xffffffffu, mbar_wait(s_full(kt & 1), (kt >> 1) & 1, abort_flag, status));
+      if (!ok) break;
+      fence_after();
+      const uint32_t ts = tmem_s0 + (kt & 1) * 128 + lane_addr;
+      const int key0 = kt * ATC_BN;
+      const bool need_mask = key0 + ATC_BN - 1 > minpos;
+      // pass 1: row maximum of the scaled, masked logits
+      float mx = -INFINITY;
+#pragma unroll 1
+      for (int c = 0; c < 4; ++c) {
+        float s[32];
+        ld32(ts + c * 32, s);
+        wait_ld();
+#pragma unroll
+        for (int e = 0; e < 32; ++e) {
+          float x = s[e] * scale_log2;
+          if (need_mask && key0 + c * 32 + e > lim) x = -INFINITY;
+          mx = fmaxf(mx, x);
+        }
+      }
+      const float m_new = fmaxf(m_run, mx);
+      const float mref = m_new == -INFINITY ? 0.f : m_new;
+      const float alpha = exp2f(m_run - mref);
+      m_run = m_new;
+      // previous tile's P V is needed before P may be overwritten; fold it into the running output
+      if (kt > 0 && want_o) {
+        ok = __all_sync(0xffffffffu, mbar_wait(o_full, (kt - 1) & 1, abort_flag, status));
+        if (!ok) break;
+        fence_after();
+#pragma unroll
+        for (int c = 0; c < D / 32; ++c) {
+          float t[32];
+          ld32(tmem_o + lane_addr + c * 32, t);
+          wait_ld();
+#pragma unroll
+          for (int e = 0; e < 32; ++e) o_reg[c * 32 + e] = o_reg[c * 32 + e] * alpha_prev + t[e];
+        }
+      }
+      alpha_prev = alpha;
+      // pass 2: probabilities, row sum, bf16 P into shared memory
+      float lsum = 0.f;
+#pragma unroll 1
+      for (int c = 0; c < 4; ++c) {
+        float s[32];
+        ld32(ts + c * 32, s);
+        wait_ld();
+#pragma unroll
+        for (int e = 0; e < 32; ++e) {
+          float x = s[e] * scale_log2;
+          if (need_mask && key0 + c * 32 + e > lim) x = -INFINITY;
+          const float pe = exp2f(x - mref);
+          s[e] = pe;
+          lsum += pe;
+        }
+        if (want_o) {
+#pragma unroll
+          for (int i = 0; i < 4; ++i)
+            *reinterpret_cast<uint4*>(base_ptr + L::P_OFF + (c >> 1) * L::SUB + swz(row, (c & 1) * 4 + i)) = pack8(s + 8 * i);
+        }
+      }
+      l_run = l_run * alpha + lsum;
+      if (want_o && kt == nkt - 1) {
+        // slots beyond the CTA's last visible key may hold anything: they get probability zero, and zero times a
+        // non-finite value would still poison the product, so clear those V rows of the last tile
+        const int first_bad = maxpos - key0 + 1;
+        const bool landed = mbar_wait(kv_full(kt & 1), (kt >> 1) & 1, abort_flag, status);  // already complete: S of this tile was computed
+        if (landed && row >= first_bad) {
+          unsigned char* sv = base_ptr + L::KV_OFF + (kt & 1) * L::KV_STAGE + (D / 64) * L::SUB;
+#pragma unroll
+          for (int j = 0; j < D / 64; ++j)
+#pragma unroll
+            for (int c = 0; c < 8; ++c) *reinterpret_cast<uint4*>(sv + j * L::SUB + row * 128 + c * 16) = make_uint4(0, 0, 0, 0);
+        }
+      }
+      fence_async_smem();
+      fence_before();
+      mbar_arrive(p_ready);
+    }
+    if (ok && want_o && nkt > 0) {
+      ok = __all_sync(0xffffffffu, mbar_wait(o_full, (nkt - 1) & 1, abort_flag, status));
+      if (ok) {
+        fence_after();
+#pragma unroll
+        for (int c = 0; c < D / 32; ++c) {
+          float t[32];
+          ld32(tmem_o + lane_addr + c * 32, t);
+          wait_ld();
+#pragma unroll
+          for (int e = 0; e < 32; ++e) o_reg[c * 32 + e] = o_reg[c * 32 + e] * alpha_prev + t[e];
+        }
+      }
+    }
+    if (ok && row_ok) {
+      const float inv = l_run > 0.f ? 1.f / l_run : 0.f;
+      if (want_o) {
+        uint4* dst = reinterpret_cast<uint4*>(o + ((size_t)tok * Hq + hq) * D);
+#pragma unroll
+        for (int c = 0; c < D / 8; ++c) {
+          float t[8];
+#pragma unroll
+          for (int e = 0; e < 8; ++e) t[e] = o_reg[c * 8 + e] * inv;
+          dst[c] = pack8(t);
+        }
+      }
+      if (lse) lse[(size_t)tok * Hq + hq] = l_run > 0.f ? (m_run + log2f(l_run)) * ATC_LN2 : -INFINITY;
+    }
+  }
+  atc::fence_before();
+  __syncthreads();
+  if (warp == 1) asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(512) : "memory");
+}
+
+// ---------------------------------------------------------------- host side
+typedef CUresult (*EncodeTiledFn2)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                                   const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                   CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+static int make_cache_tmap(CUtensorMap* map, const void* ptr, long long rows, long long cols) {
+  static EncodeTiledFn2 fn = nullptr;
+  if (!fn) {
+    void* p = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &qres) != cudaSuccess || qres != cudaDriverEntryPointSuccess)
+      return A3_ECUDA;
+    fn = (EncodeTiledFn2)p;
+  }
+  cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
+  cuuint64_t strides[1] = {(cuuint64_t)cols * 2};
+  cuuint32_t box[2] = {64, (cuuint32_t)ATC_BN};
+  cuuint32_t estr[2] = {1, 1};
+  CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(ptr), dims, strides, box, estr,
+                  CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                  CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  if (r != CUDA_SUCCESS) {
+    g_last_cuda_error = (int)r;
+    return A3_ECUDA;
+  }
+  return A3_OK;
+}
+
+int attention_rows_tc(const a3_handle* h, const bf16* q, const int32_t* pos, int M, const bf16* k, const bf16* v,
+                      int kv_len, bf16* o, float* lse, cudaStream_t st) {
+  if (M <= 0) return A3_OK;
+  const int Hq = h->m.n_q_heads, Hkv = h->m.n_kv_heads, D = h->m.head_dim;
+  const int G = Hq / Hkv;
+  CUtensorMap tK, tV;
+  A3_TRY(make_cache_tmap(&tK, k, kv_len, (long long)Hkv * D));
+  A3_TRY(make_cache_tmap(&tV, v, kv_len, (long long)Hkv * D));
+  dim3 grid(cdiv((long long)M * G, ATC_BM), Hkv);
+  const float scale_log2 = ATC_LOG2E / sqrtf((float)D);
+  static bool attr_set = false;
+  if (!attr_set) {
+    A3_CUDA(cudaFuncSetAttribute(attention_tc_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, AtcLayout<128>::SMEM_BYTES));
+    A3_CUDA(cudaFuncSetAttribute(attention_tc_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, AtcLayout<64>::SMEM_BYTES));
+    attr_set = true;
+  }
+  ProfScope prof(h, A3_K_ATTENTION, st);
+  if (D == 128)
+    attention_tc_kernel<128><<<grid, ATC_THREADS, AtcLayout<128>::SMEM_BYTES, st>>>(tK, tV, q, pos, M, kv_len, o, lse, Hq, Hkv, scale_log2, h->dev_status);
+  else
+    attention_tc_kernel<64><<<grid, ATC_THREADS, AtcLayout<64>::SMEM_BYTES, st>>>(tK, tV, q, pos, M, kv_len, o, lse, Hq, Hkv, scale_log2, h->dev_status);
+  A3_LAUNCHED();
+  return A3_OK;
+}
+
+}  // namespace a3
