@@ -217,3 +217,45 @@ def make_cache_device(m: ModelShape, n_tokens: int, device, seed: int, stream: i
     k = (torch.randn(shape, generator=g, device=device, dtype=torch.float32) * std).to(torch.bfloat16)
     v = (torch.randn(shape, generator=g, device=device, dtype=torch.float32) * std).to(torch.bfloat16)
     return k, v
+
+
+# ------------------------------------------------------------------ planted relevance (32K-context configuration)
+
+
+def plant_embeddings(x0: torch.Tensor, r: RequestShape, planted_chunks, cosine: float = 0.5, seed: int = 0) -> torch.Tensor:
+    """Make the question rows and the rows of `planted_chunks` share a direction (cosine ~ `cosine` with it).
+
+    x0: [n][d] embeddings (any device).  Each affected row keeps its norm: e <- |e| (c u + sqrt(1-c^2) e_perp), u a
+    seeded unit vector and e_perp the row's unit component orthogonal to u.  Returns a new bf16 tensor.
+    """
+    g = torch.Generator(device="cpu")
+    g.manual_seed(seed * 15485863 + 5)
+    u = torch.randn(x0.shape[1], generator=g, dtype=torch.float32)
+    u = (u / u.norm()).to(x0.device)
+    rows = list(range(r.n_ctx, r.n))
+    for c in planted_chunks:
+        rows += list(range(r.offsets[c], r.offsets[c] + r.chunk_lens[c]))
+    idx = torch.tensor(rows, device=x0.device, dtype=torch.long)
+    e = x0[idx].float()
+    norm = e.norm(dim=1, keepdim=True)
+    perp = e - (e @ u)[:, None] * u[None, :]
+    perp = perp / perp.norm(dim=1, keepdim=True)
+    out = x0.clone()
+    out[idx] = (norm * (cosine * u[None, :] + (1.0 - cosine * cosine) ** 0.5 * perp)).to(x0.dtype)
+    return out
+
+
+def tie_keys_to_queries(w: Dict[str, torch.Tensor], m: ModelShape, rho: float = 0.7, seed: int = 0) -> None:
+    """In place: make each KV head's key projection correlate (rho) with the mean of its query heads' projections.
+
+    With independent random Wq and Wk the logit q.k has zero mean whatever the inputs share; tying them lets a
+    shared input direction show up as attention, which is what the planted configuration needs.
+    """
+    G, D = m.n_q_heads // m.n_kv_heads, m.head_dim
+    wq, wk = w["wq"], w["wk"]
+    g = torch.Generator(device="cpu")
+    g.manual_seed(seed * 32452843 + 11)
+    for h in range(m.n_kv_heads):
+        mean_q = wq[h * G * D:(h + 1) * G * D].float().view(G, D, -1).mean(dim=0) * (G ** 0.5)
+        noise = wk[h * D:(h + 1) * D].float()
+        wk[h * D:(h + 1) * D] = (rho * mean_q + (1.0 - rho * rho) ** 0.5 * noise).to(wk.dtype)

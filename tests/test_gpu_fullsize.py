@@ -1,0 +1,233 @@
+"""Parity at the benchmark configurations' full width and length, in the launch configuration bench.py times.
+
+The oracle cannot run these sizes whole in test time, so each request is checked through (a) exact properties that
+hold at any size (the selection is the top-p of the scores the GPU computed; rows outside R keep the re-rotated
+chunk values bit for bit; scores vanish outside the candidates and their mass is bounded), (b) position recovery on
+sampled rows against the oracle, and (c) one recompute layer at full width and length, teacher-forced, on sampled
+rows the oracle computes one by one.  Stacks are truncated to three layers (selection at layer 1) except for one
+full-depth run; widths, lengths, chunk structure and ratios are the configurations' own.
+"""
+from dataclasses import replace
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import a3_oracle as O
+from paper_2511_17560_b200 import workloads as W
+from tests.helpers import oracle_model
+from tests.test_gpu_steps import KV_MAX, KV_MEAN, check_kv, f64
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda:0"
+
+
+def precompute(eng, m, r, x0):
+    """Eq. 1 with the library itself: every chunk alone at local positions (all rows through every layer)."""
+    ck, cv = [], []
+    for o, t in zip(r.offsets, r.chunk_lens):
+        K = torch.zeros((m.n_layers, t, m.n_kv_heads, m.head_dim), dtype=torch.bfloat16, device=DEV)
+        V = torch.zeros_like(K)
+        X = x0[o:o + t].clone()
+        pos = torch.arange(t, dtype=torch.int32, device=DEV)
+        for l in range(m.n_layers):
+            eng.recompute_layer(l, X, pos, K[l], V[l])
+        ck.append(K)
+        cv.append(V)
+    return ck, cv
+
+
+class Case:
+    def __init__(self, config, layers=3, planted=None, emb_std=0.02, seed=0):
+        from paper_2511_17560_b200 import a3
+        self.a3 = a3
+        m, self.r = W.request_for(config)
+        self.m = m = replace(m, n_layers=layers)
+        r = self.r
+        self.weights = W.make_weights_device(m, DEV, seed)
+        self.x0 = W.make_embeddings_device(m, r.n, DEV, seed, std=emb_std)
+        if planted:
+            W.tie_keys_to_queries(self.weights[r.select_layer], m, 0.7, seed)
+            self.x0 = W.plant_embeddings(self.x0, r, planted, 0.5, seed)
+        self.eng = a3.A3(m, self.weights, r.n + 8)
+        self.ck, self.cv = precompute(self.eng, m, r, self.x0)
+        self.tab = a3.chunk_table(self.ck, self.cv, r.offsets)
+
+    def buffers(self):
+        m, r = self.m, self.r
+        K = torch.zeros((m.n_layers, r.n, m.n_kv_heads, m.head_dim), dtype=torch.bfloat16, device=DEV)
+        return K, torch.zeros_like(K)
+
+    def fuse(self, ratio=None):
+        r = self.r
+        K, V = self.buffers()
+        req, out = self.eng.make_request(self.tab, len(self.ck), max(r.chunk_lens), r.n_ctx, r.n_question, self.x0, K, V,
+                                         ratio=r.ratio if ratio is None else ratio, select_layer=r.select_layer)
+        self.eng.fuse_request(req)
+        assert self.eng.device_status() == 0
+        return K, V, out
+
+    def oracle_layer(self, l):
+        return O.LayerWeights(**{k: v.float().cpu().numpy() for k, v in self.weights[l].items()})
+
+
+def check_request_properties(c: Case, K, V, out, ratio=None):
+    """Everything about a finished request that can be checked exactly at any size."""
+    m, r = c.m, c.r
+    ratio = r.ratio if ratio is None else ratio
+    p = O.recompute_count(ratio, r.n, r.n_ctx)
+    rows = out["rows"].cpu().numpy()
+    s = out["scores"].cpu().numpy().astype(np.float64)
+    assert out["p"] == p and rows.shape[0] == p + r.n_question
+    assert rows[p:].tolist() == list(range(r.n_ctx, r.n))
+    assert np.all(np.diff(rows) > 0)
+    assert rows[:p].tolist() == O.topk_select(s, 0, r.n_ctx, p).tolist()  # bit-exact selection on the GPU's scores
+    assert np.isfinite(s).all() and (s >= 0).all() and not s[r.n_ctx:].any()
+    total = r.n_question * m.n_q_heads
+    assert 0.5 * total < s.sum() <= total * (1 + 1e-5)
+    assert torch.isfinite(out["x"].float()).all() and torch.isfinite(K.float()).all() and torch.isfinite(V.float()).all()
+    # rows outside R at layers after the selection layer: the re-rotated chunk rows, bit for bit
+    Kr, Vr = c.buffers()
+    c.eng.rope_rerotate(c.tab, len(c.ck), max(r.chunk_lens), Kr, Vr)
+    keep = torch.ones(r.n, dtype=torch.bool, device=DEV)
+    keep[out["rows"].long()] = False
+    for l in range(r.select_layer + 1, m.n_layers):
+        assert torch.equal(K[l][keep], Kr[l][keep]) and torch.equal(V[l][keep], Vr[l][keep])
+    return rows, s, Kr, Vr
+
+
+def check_position_recovery_samples(c: Case, Kr, Vr, n_samples=64, seed=0):
+    """Eq. 2 on sampled (layer, chunk, token) rows against the oracle, incl. the last chunk (largest offset)."""
+    m, r = c.m, c.r
+    rng = np.random.default_rng(seed)
+    errs = []
+    for i in range(n_samples):
+        l = int(rng.integers(0, m.n_layers))
+        ch = len(r.chunk_lens) - 1 if i % 4 == 0 else int(rng.integers(0, len(r.chunk_lens)))
+        t = int(rng.integers(0, r.chunk_lens[ch]))
+        src = c.ck[ch][l, t].float().cpu().numpy().astype(np.float64)[None]
+        want = O.rope_rotate(src, np.array([r.offsets[ch]]), m.rope_theta, m.rope_layout)[0]
+        got = f64(Kr[l, r.offsets[ch] + t])
+        errs.append(np.abs(got - want))
+        assert torch.equal(Vr[l, r.offsets[ch] + t], c.cv[ch][l, t])
+    errs = np.stack(errs)
+    assert errs.max() <= KV_MAX and errs.mean() <= KV_MEAN, (errs.max(), errs.mean())
+
+
+def check_layer_samples(c: Case, layer, rows, K_layer, V_layer, n_samples=10, seed=0):
+    """One recompute layer at full width/length, teacher-forced: the GPU runs all carried rows; the oracle recomputes
+    sampled rows one by one from the same inputs (cache taken from the GPU after its scatter)."""
+    m, r = c.m, c.r
+    M = rows.shape[0]
+    g = torch.Generator(device=DEV)
+    g.manual_seed(1234 + seed)
+    X = torch.randn((M, m.d_model), generator=g, device=DEV, dtype=torch.float32).to(torch.bfloat16)
+    Kc, Vc = K_layer.clone(), V_layer.clone()
+    pos = torch.from_numpy(rows.astype(np.int32)).to(DEV)
+    Xg = X.clone()
+    lse = torch.empty((M, m.n_q_heads), dtype=torch.float32, device=DEV)
+    c.eng.recompute_layer(layer, Xg, pos, Kc, Vc, lse_out=lse)
+    assert c.eng.device_status() == 0
+    rng = np.random.default_rng(seed)
+    sel = np.unique(np.concatenate([[0, M - 1], rng.choice(M, size=n_samples, replace=False)]))
+    w, model = c.oracle_layer(layer), oracle_model(m)
+    Ko, Vo = f64(Kc), f64(Vc)
+    Xo, parts = O.recompute_layer(f64(X[sel]), rows[sel], w, model, Ko, Vo, rnd=O.round_bf16, return_parts=True)
+    check_kv(f64(Kc[pos[sel].long()]), parts["k_exact"], "K rows at full width")
+    check_kv(f64(Vc[pos[sel].long()]), parts["v_exact"], "V rows at full width")
+    check_kv(f64(Xg[sel]), parts["x_exact"], "hidden rows at full width", scale=2.0 * float(parts["x_exact"].std()))
+    np.testing.assert_allclose(lse[sel].cpu().numpy(), parts["lse"], atol=5e-3)
+
+
+def test_llama8b_10x512_three_layers():
+    c = Case("llama8b_10x512")
+    K, V, out = c.fuse()
+    rows, s, Kr, Vr = check_request_properties(c, K, V, out)
+    assert out["p"] == 772
+    check_position_recovery_samples(c, Kr, Vr)
+    check_layer_samples(c, 2, rows, K[2], V[2])
+    # the full block: all 5152 rows at positions 0..n-1 (launch shape of the leading block), sampled rows
+    check_layer_samples(c, 0, np.arange(c.r.n), Kr[0], Vr[0], n_samples=6, seed=1)
+    c.eng.close()
+
+
+def test_llama8b_10x512_full_depth_runs_clean():
+    c = Case("llama8b_10x512", layers=32)
+    K, V, out = c.fuse()
+    check_request_properties(c, K, V, out)
+    K2, V2, out2 = c.fuse()  # same request again: bit-identical (no atomics, fixed reduction orders)
+    assert torch.equal(K, K2) and torch.equal(V, V2) and torch.equal(out["x"], out2["x"]) and torch.equal(out["scores"], out2["scores"])
+    c.eng.close()
+
+
+def test_llama8b_32k_planted_relevance():
+    planted = (20, 45)
+    c = Case("llama8b_64x512", planted=planted, emb_std=1.0)
+    K, V, out = c.fuse()
+    rows, s, Kr, Vr = check_request_properties(c, K, V, out)
+    assert out["p"] == 4920
+    Re = rows[: out["p"]]
+    share = np.mean([(r // 512) in planted for r in Re])
+    assert share >= 3 * len(planted) / 64, share  # the selection concentrates on the planted chunks
+    check_position_recovery_samples(c, Kr, Vr, seed=2)
+    check_layer_samples(c, 2, rows, K[2], V[2], n_samples=6, seed=2)
+    c.eng.close()
+
+
+def test_qwen7b_ragged_ratio_sweep():
+    c = Case("qwen7b_16xU")
+    assert len(c.r.chunk_lens) == 16 and all(256 <= t <= 2048 for t in c.r.chunk_lens)
+    prev = None
+    for ratio in (0.05, 0.10, 0.15, 0.30):
+        K, V, out = c.fuse(ratio)
+        rows, s, Kr, Vr = check_request_properties(c, K, V, out, ratio)
+        cur = set(rows[: out["p"]].tolist())
+        if prev is not None:
+            assert prev <= cur  # nested selections on the same request
+        prev = cur
+        if ratio == 0.15:
+            check_position_recovery_samples(c, Kr, Vr, seed=3)
+            check_layer_samples(c, 2, rows, K[2], V[2], n_samples=6, seed=3)  # G = 7 packing, q/k/v bias
+    c.eng.close()
+
+
+def test_batched_serving_matches_single_requests():
+    from paper_2511_17560_b200 import a3
+    m = replace(W.LLAMA8B, n_layers=3)
+    pool_lens, reqs = W.batched_requests(seed=0)
+    assert len(pool_lens) == 200 and len(reqs) == 16
+    weights = W.make_weights_device(m, DEV, 0)
+    n_max = max(sum(pool_lens[i] for i in ids) + nq for ids, nq in reqs)
+    eng = a3.A3(m, weights, n_max + 8)
+    used = sorted({i for ids, _ in reqs for i in ids})
+    pool = {}
+    for i in used:  # only the pool chunks some request uses are prefilled
+        t = pool_lens[i]
+        r1 = W.RequestShape((t,), 0, 0.15, 1)
+        x = W.make_embeddings_device(m, t, DEV, 0, stream=1000 + i)
+        ck, cv = precompute(eng, m, r1, x)
+        pool[i] = (ck[0], cv[0], x)
+    batch, singles, keep = [], [], []
+    for j, (ids, nq) in enumerate(reqs):
+        lens = tuple(pool_lens[i] for i in ids)
+        r = W.RequestShape(lens, nq, 0.15, 1)
+        xq = W.make_embeddings_device(m, nq, DEV, 0, stream=5000 + j)
+        x0 = torch.cat([pool[i][2] for i in ids] + [xq]).contiguous()
+        tab = a3.chunk_table([pool[i][0] for i in ids], [pool[i][1] for i in ids], r.offsets)
+        for dest in (batch, singles):
+            K = torch.zeros((m.n_layers, r.n, m.n_kv_heads, m.head_dim), dtype=torch.bfloat16, device=DEV)
+            V = torch.zeros_like(K)
+            req, out = eng.make_request(tab, len(ids), max(lens), r.n_ctx, nq, x0, K, V, ratio=0.15, select_layer=1)
+            dest.append((req, out, K, V))
+        keep.append((x0, tab))
+    eng.fuse_batch([b[0] for b in batch])
+    for req, out, K, V in singles:
+        eng.fuse_request(req)
+    assert eng.device_status() == 0
+    for (rb, ob, Kb, Vb), (rs, os_, Ks, Vs) in zip(batch, singles):
+        assert torch.equal(Kb, Ks) and torch.equal(Vb, Vs) and torch.equal(ob["x"], os_["x"]) and torch.equal(ob["rows"], os_["rows"])
+        s = ob["scores"].cpu().numpy().astype(np.float64)
+        p = ob["p"]
+        n_ctx = rb.n_ctx
+        assert ob["rows"].cpu().numpy()[:p].tolist() == O.topk_select(s, 0, n_ctx, p).tolist()
+    eng.close()
