@@ -8,11 +8,12 @@
 //                       swizzle, two stages).
 //   warp 1 (one lane)   tcgen05.mma issuer: S = Q K^T (128 x 128 x D) into one of two TMEM buffers, and, once the
 //                       probabilities of a tile are in shared memory, O~ = P V (128 x D x 128, V as an MN-major
-//                       operand) into a third TMEM buffer.  S of tile t+1 is issued before P V of tile t, so the
+//                       operand) accumulated into a third TMEM buffer.  S of tile t+1 is issued before P V of tile t, so the
 //                       tensor core works while the softmax threads do.
-//   warps 2..5          one thread per row: two passes over the row of S in TMEM (maximum, then exp2 and sum), P
-//                       written as bf16 into shared memory in the swizzled K-major layout the MMA reads, running
-//                       rescale of the output kept in registers (O = O * alpha + O~), final normalisation, stores.
+//   warps 2..5          one thread per row: one pass over the row of S in TMEM (exp2 against a lazily raised
+//                       reference maximum, row sum), P written as bf16 into shared memory in the swizzled K-major
+//                       layout the MMA reads; the output accumulates in TMEM across key tiles and is rescaled there
+//                       only when the reference has to be raised; final normalisation and stores.
 // Statistics are fp32 in the exp2 domain.  Every mbarrier wait is bounded (see a3_gemm_tc.cu); there is no block-
 // wide or named barrier inside the loops, so a role that gives up cannot strand another.
 #include <cuda.h>
@@ -99,6 +100,18 @@ __device__ __forceinline__ void ld32(uint32_t taddr, float* v) {
       : "memory");
 }
 __device__ __forceinline__ void wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+__device__ __forceinline__ void st32(uint32_t taddr, const float* v) {
+  const uint32_t* r = reinterpret_cast<const uint32_t*>(v);
+  asm volatile(
+      "tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16, "
+      "%17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31, %32};"
+      ::"r"(taddr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]), "r"(r[8]),
+        "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15]), "r"(r[16]), "r"(r[17]),
+        "r"(r[18]), "r"(r[19]), "r"(r[20]), "r"(r[21]), "r"(r[22]), "r"(r[23]), "r"(r[24]), "r"(r[25]), "r"(r[26]),
+        "r"(r[27]), "r"(r[28]), "r"(r[29]), "r"(r[30]), "r"(r[31])
+      : "memory");
+}
+__device__ __forceinline__ void wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 
 // K-major [rows][64] bf16 sub-tile, 128-byte swizzle, 8-row groups 1024 bytes apart
 __device__ __forceinline__ uint64_t desc_k_sw128(uint32_t saddr) {
@@ -118,37 +131,61 @@ __host__ __device__ constexpr uint32_t idesc(int n, int b_mn) {
 __device__ __forceinline__ uint32_t swz(int r, int j) { return (uint32_t)(r * 128 + ((j ^ (r & 7)) << 4)); }
 }  // namespace atc
 
+__device__ __forceinline__ float ex2_approx(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+// 32 logits of one row -> probabilities (in place), running relative maximum and four partial row sums.
+// t = s * scale - m_ref is one FMA; ex2.approx maps -inf to +0, so masked keys need no second select.
+template <bool MASK>
+__device__ __forceinline__ void softmax_chunk(float* sv, int key_base, int lim, float scale, float neg_ref, float& mx, float (&ls)[4]) {
+#pragma unroll
+  for (int e = 0; e < 32; ++e) {
+    float t = fmaf(sv[e], scale, neg_ref);
+    if (MASK && key_base + e > lim) t = -INFINITY;
+    mx = fmaxf(mx, t);
+    const float pe = ex2_approx(t);
+    sv[e] = pe;
+    ls[e & 3] += pe;
+  }
+}
+
 template <int D>
 struct AtcLayout {
   static constexpr int SUB = 128 * 64 * 2;           // one [128][64] bf16 sub-tile: 16 KiB
   static constexpr int Q_BYTES = (D / 64) * SUB;
   static constexpr int KV_STAGE = 2 * (D / 64) * SUB;  // K then V
-  static constexpr int P_BYTES = 2 * SUB;
+  static constexpr int P_BYTES = 2 * SUB;                // one P buffer; two of them alternate
   static constexpr int Q_OFF = 0;
   static constexpr int KV_OFF = Q_BYTES;
   static constexpr int P_OFF = KV_OFF + 2 * KV_STAGE;
-  static constexpr int BAR_OFF = P_OFF + P_BYTES;
+  static constexpr int BAR_OFF = P_OFF + 2 * P_BYTES;
   static constexpr int SMEM_BYTES = BAR_OFF + 256 + 1024;
 };
 
 template <int D>
-__global__ void __launch_bounds__(ATC_THREADS)
+__global__ void __launch_bounds__(ATC_THREADS, 1)
 attention_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV,
                     const bf16* __restrict__ q, const int32_t* __restrict__ pos, int M, int kv_len, bf16* __restrict__ o,
-                    float* __restrict__ lse, int Hq, int Hkv, float scale_log2, uint32_t* status) {
+                    float* __restrict__ lse, int Hq, int Hkv, float scale_log2, uint32_t* status, int dbg) {
   using L = AtcLayout<D>;
   using namespace atc;
   extern __shared__ unsigned char smem_raw[];
   const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   unsigned char* base_ptr = smem_raw + (base - smem_u32(smem_raw));
-  // barriers: kv_full[2], kv_empty[2], s_full[2], o_full, p_ready, q_ready
+  // barriers: kv_full[2], kv_empty[2], s_full[2], p_ready[2], q_ready, p_free[2]
   const uint32_t bars = base + L::BAR_OFF;
   auto kv_full = [&](int s) { return bars + 8u * s; };
   auto kv_empty = [&](int s) { return bars + 8u * (2 + s); };
   auto s_full = [&](int b) { return bars + 8u * (4 + b); };
-  const uint32_t o_full = bars + 8u * 6, p_ready = bars + 8u * 7, q_ready = bars + 8u * 8;
-  volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(base_ptr + L::BAR_OFF + 8 * 9);
-  volatile int* abort_flag = reinterpret_cast<volatile int*>(base_ptr + L::BAR_OFF + 8 * 9 + 8);
+  // p_ready alternates between two barriers: a fast warp may finish tile t+1 before a slow warp has arrived for
+  // tile t, and on a single barrier its second arrival would be counted towards tile t
+  auto p_ready = [&](int b) { return bars + 8u * (6 + b); };
+  const uint32_t q_ready = bars + 8u * 8;
+  auto p_free = [&](int b) { return bars + 8u * (9 + b); };
+  volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(base_ptr + L::BAR_OFF + 8 * 11);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(base_ptr + L::BAR_OFF + 8 * 11 + 8);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int G = Hq / Hkv;
@@ -168,9 +205,10 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
       mbar_init(kv_full(i), 1);
       mbar_init(kv_empty(i), 1);
       mbar_init(s_full(i), 1);
+      mbar_init(p_free(i), 1);
     }
-    mbar_init(o_full, 1);
-    mbar_init(p_ready, 128);
+    mbar_init(p_ready(0), 128);
+    mbar_init(p_ready(1), 128);
     mbar_init(q_ready, 128);
     abort_flag[0] = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -228,21 +266,23 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
         if (kt + 1 < nkt) {
           ok = mbar_wait(kv_full((kt + 1) & 1), ((kt + 1) >> 1) & 1, abort_flag, status);
           if (!ok) break;
+          if ((dbg & 4) && blockIdx.x == 0 && blockIdx.y == 0 && kt < 60) status[64 + kt * 4 + 2] = (uint32_t)global_ns();
           fence_after();
           issue_s(kt + 1);
         }
-        ok = mbar_wait(p_ready, kt & 1, abort_flag, status);
+        ok = mbar_wait(p_ready(kt & 1), (kt >> 1) & 1, abort_flag, status);
         if (!ok) break;
+        if ((dbg & 4) && blockIdx.x == 0 && blockIdx.y == 0 && kt < 60) status[64 + kt * 4 + 3] = (uint32_t)global_ns();
         fence_after();
         if (want_o) {
           const uint32_t sv = base + L::KV_OFF + (kt & 1) * L::KV_STAGE + (D / 64) * L::SUB;
 #pragma unroll
           for (int k = 0; k < ATC_BN / 16; ++k) {
-            const uint64_t da = desc_k_sw128(sp + (k / 4) * L::SUB + (k % 4) * 32);
+            const uint64_t da = desc_k_sw128(sp + (kt & 1) * L::P_BYTES + (k / 4) * L::SUB + (k % 4) * 32);
             const uint64_t db = desc_mn_sw128(sv + k * 16 * 128, L::SUB);
-            mma_f16(tmem_o, da, db, idesc_o, k != 0);
+            mma_f16(tmem_o, da, db, idesc_o, (kt | k) != 0);  // O accumulates over the key tiles in TMEM
           }
-          commit(o_full);
+          commit(p_free(kt & 1));  // P V of this tile is complete: its P buffer may be rewritten, O holds tiles 0..kt
         }
         commit(kv_empty(kt & 1));
       }
@@ -270,75 +310,94 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
       mbar_arrive(q_ready);
     }
 
-    float o_reg[D];
-#pragma unroll
-    for (int e = 0; e < D; ++e) o_reg[e] = 0.f;
-    float m_run = -INFINITY, l_run = 0.f, alpha_prev = 0.f;
+    // Exponent reference m_ref and row sum l_run relative to it.  The reference is the true maximum of the first
+    // tile and is raised later only when a logit exceeds it by more than 2^RESCALE_TH (rare once the first tiles
+    // are seen): then the output accumulated in TMEM and l_run are rescaled and the tile is redone.  Probabilities
+    // therefore stay below 2^RESCALE_TH, and the output needs no per-tile correction.
+    constexpr float RESCALE_TH = 8.f;
+    float m_ref = 0.f, l_run = 0.f;
     bool ok = true;
 
     for (int kt = 0; kt < nkt; ++kt) {
-      // the result of every wait is made warp-uniform: tcgen05.ld is a warp-wide instruction
+      // the result of every wait is made warp-uniform: tcgen05.ld/st are warp-wide instructions
       ok = __all_sync(0xffffffffu, mbar_wait(s_full(kt & 1), (kt >> 1) & 1, abort_flag, status));
       if (!ok) break;
       fence_after();
+      if ((dbg & 4) && blockIdx.x == 0 && blockIdx.y == 0 && row == 0 && kt < 60) status[64 + kt * 4 + 0] = (uint32_t)global_ns();
       const uint32_t ts = tmem_s0 + (kt & 1) * 128 + lane_addr;
       const int key0 = kt * ATC_BN;
       const bool need_mask = key0 + ATC_BN - 1 > minpos;
-      // pass 1: row maximum of the scaled, masked logits
-      float mx = -INFINITY;
+      if (kt == 0) {
+        float mx = -INFINITY;
 #pragma unroll 1
-      for (int c = 0; c < 4; ++c) {
-        float s[32];
-        ld32(ts + c * 32, s);
-        wait_ld();
-#pragma unroll
-        for (int e = 0; e < 32; ++e) {
-          float x = s[e] * scale_log2;
-          if (need_mask && key0 + c * 32 + e > lim) x = -INFINITY;
-          mx = fmaxf(mx, x);
-        }
-      }
-      const float m_new = fmaxf(m_run, mx);
-      const float mref = m_new == -INFINITY ? 0.f : m_new;
-      const float alpha = exp2f(m_run - mref);
-      m_run = m_new;
-      // previous tile's P V is needed before P may be overwritten; fold it into the running output
-      if (kt > 0 && want_o) {
-        ok = __all_sync(0xffffffffu, mbar_wait(o_full, (kt - 1) & 1, abort_flag, status));
-        if (!ok) break;
-        fence_after();
-#pragma unroll
-        for (int c = 0; c < D / 32; ++c) {
-          float t[32];
-          ld32(tmem_o + lane_addr + c * 32, t);
+        for (int c = 0; c < 4; ++c) {
+          float sv[32];
+          ld32(ts + c * 32, sv);
           wait_ld();
 #pragma unroll
-          for (int e = 0; e < 32; ++e) o_reg[c * 32 + e] = o_reg[c * 32 + e] * alpha_prev + t[e];
+          for (int e = 0; e < 32; ++e) {
+            float x = sv[e] * scale_log2;
+            if (need_mask && key0 + c * 32 + e > lim) x = -INFINITY;
+            mx = fmaxf(mx, x);
+          }
         }
+        m_ref = mx == -INFINITY ? 0.f : mx;
       }
-      alpha_prev = alpha;
-      // pass 2: probabilities, row sum, bf16 P into shared memory
-      float lsum = 0.f;
+      if (want_o && kt >= 2) {
+        // the P buffer of this tile was last read by the P V of tile kt-2
+        ok = __all_sync(0xffffffffu, mbar_wait(p_free(kt & 1), ((kt >> 1) & 1) ^ 1, abort_flag, status));
+        if (!ok) break;
+      }
 #pragma unroll 1
-      for (int c = 0; c < 4; ++c) {
-        float s[32];
-        ld32(ts + c * 32, s);
-        wait_ld();
+      for (int trip = 0; trip < 2; ++trip) {
+        // mx is tracked relative to the reference: the exponent argument itself, fmaf(s, scale, -m_ref)
+        float mx = -INFINITY, ls[4] = {0.f, 0.f, 0.f, 0.f};
+        const float neg_ref = -m_ref;
+        float buf[2][32];
+        ld32(ts, buf[0]);
 #pragma unroll
-        for (int e = 0; e < 32; ++e) {
-          float x = s[e] * scale_log2;
-          if (need_mask && key0 + c * 32 + e > lim) x = -INFINITY;
-          const float pe = exp2f(x - mref);
-          s[e] = pe;
-          lsum += pe;
+        for (int c = 0; c < 4; ++c) {
+          wait_ld();
+          if (c < 3) ld32(ts + (c + 1) * 32, buf[(c + 1) & 1]);
+          float* sv = buf[c & 1];
+          if (need_mask) softmax_chunk<true>(sv, key0 + c * 32, lim, scale_log2, neg_ref, mx, ls);
+          else softmax_chunk<false>(sv, key0 + c * 32, lim, scale_log2, neg_ref, mx, ls);
+          if (want_o) {
+#pragma unroll
+            for (int i = 0; i < 4; ++i)
+              *reinterpret_cast<uint4*>(base_ptr + L::P_OFF + (kt & 1) * L::P_BYTES + (c >> 1) * L::SUB + swz(row, (c & 1) * 4 + i)) = pack8(sv + 8 * i);
+          }
         }
-        if (want_o) {
+        const float lsum = (ls[0] + ls[1]) + (ls[2] + ls[3]);
+        if (!__any_sync(0xffffffffu, mx > RESCALE_TH)) {
+          l_run += lsum;
+          break;
+        }
+        if ((dbg & 2) && lane == 0) atomicAdd(status + 1, 1u);
+        const float raise = fmaxf(mx, 0.f);  // lanes below the threshold may move too: any value >= their maximum is valid
+        const float f = exp2f(-raise);
+        m_ref += raise;
+        l_run *= f;
+        if (want_o && kt > 0) {
+          // the output so far must be complete (P V of the previous tile) before it is rescaled in place
+          // (the threads follow every phase of p_free[b] in order - tile kt-1 waited for tile kt-3 on the same
+          // barrier - so a parity wait cannot mistake an older completion for this one)
+          ok = __all_sync(0xffffffffu, mbar_wait(p_free((kt - 1) & 1), ((kt - 1) >> 1) & 1, abort_flag, status));
+          if (!ok) break;
+          fence_after();
+#pragma unroll 1
+          for (int c = 0; c < D / 32; ++c) {
+            float t[32];
+            ld32(tmem_o + lane_addr + c * 32, t);
+            wait_ld();
 #pragma unroll
-          for (int i = 0; i < 4; ++i)
-            *reinterpret_cast<uint4*>(base_ptr + L::P_OFF + (c >> 1) * L::SUB + swz(row, (c & 1) * 4 + i)) = pack8(s + 8 * i);
+            for (int e = 0; e < 32; ++e) t[e] *= f;
+            st32(tmem_o + lane_addr + c * 32, t);
+          }
+          wait_st();
         }
       }
-      l_run = l_run * alpha + lsum;
+      if (!ok) break;
       if (want_o && kt == nkt - 1) {
         // slots beyond the CTA's last visible key may hold anything: they get probability zero, and zero times a
         // non-finite value would still poison the product, so clear those V rows of the last tile
@@ -352,38 +411,34 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
             for (int c = 0; c < 8; ++c) *reinterpret_cast<uint4*>(sv + j * L::SUB + row * 128 + c * 16) = make_uint4(0, 0, 0, 0);
         }
       }
+      if ((dbg & 2) && lane == 0) atomicAdd(status + 2, 1u);
+      if ((dbg & 4) && blockIdx.x == 0 && blockIdx.y == 0 && row == 0 && kt < 60) status[64 + kt * 4 + 1] = (uint32_t)global_ns();
       fence_async_smem();
       fence_before();
-      mbar_arrive(p_ready);
+      mbar_arrive(p_ready(kt & 1));
     }
+    const float inv = l_run > 0.f ? 1.f / l_run : 0.f;
     if (ok && want_o && nkt > 0) {
-      ok = __all_sync(0xffffffffu, mbar_wait(o_full, (nkt - 1) & 1, abort_flag, status));
+      ok = __all_sync(0xffffffffu, mbar_wait(p_free((nkt - 1) & 1), ((nkt - 1) >> 1) & 1, abort_flag, status));
       if (ok) {
         fence_after();
-#pragma unroll
+        bf16* dst = o + ((size_t)tok * Hq + hq) * D;
+#pragma unroll 1
         for (int c = 0; c < D / 32; ++c) {
           float t[32];
           ld32(tmem_o + lane_addr + c * 32, t);
           wait_ld();
+          if (row_ok) {
 #pragma unroll
-          for (int e = 0; e < 32; ++e) o_reg[c * 32 + e] = o_reg[c * 32 + e] * alpha_prev + t[e];
+            for (int e = 0; e < 32; ++e) t[e] *= inv;
+#pragma unroll
+            for (int i = 0; i < 4; ++i) reinterpret_cast<uint4*>(dst + c * 32)[i] = pack8(t + 8 * i);
+          }
+          __syncwarp();
         }
       }
     }
-    if (ok && row_ok) {
-      const float inv = l_run > 0.f ? 1.f / l_run : 0.f;
-      if (want_o) {
-        uint4* dst = reinterpret_cast<uint4*>(o + ((size_t)tok * Hq + hq) * D);
-#pragma unroll
-        for (int c = 0; c < D / 8; ++c) {
-          float t[8];
-#pragma unroll
-          for (int e = 0; e < 8; ++e) t[e] = o_reg[c * 8 + e] * inv;
-          dst[c] = pack8(t);
-        }
-      }
-      if (lse) lse[(size_t)tok * Hq + hq] = l_run > 0.f ? (m_run + log2f(l_run)) * ATC_LN2 : -INFINITY;
-    }
+    if (ok && row_ok && lse) lse[(size_t)tok * Hq + hq] = l_run > 0.f ? (m_ref + log2f(l_run)) * ATC_LN2 : -INFINITY;
   }
   atc::fence_before();
   __syncthreads();
@@ -418,6 +473,8 @@ static int make_cache_tmap(CUtensorMap* map, const void* ptr, long long rows, lo
   return A3_OK;
 }
 
+int g_attn_dbg = 0;
+
 int attention_rows_tc(const a3_handle* h, const bf16* q, const int32_t* pos, int M, const bf16* k, const bf16* v,
                       int kv_len, bf16* o, float* lse, cudaStream_t st) {
   if (M <= 0) return A3_OK;
@@ -436,11 +493,13 @@ int attention_rows_tc(const a3_handle* h, const bf16* q, const int32_t* pos, int
   }
   ProfScope prof(h, A3_K_ATTENTION, st);
   if (D == 128)
-    attention_tc_kernel<128><<<grid, ATC_THREADS, AtcLayout<128>::SMEM_BYTES, st>>>(tK, tV, q, pos, M, kv_len, o, lse, Hq, Hkv, scale_log2, h->dev_status);
+    attention_tc_kernel<128><<<grid, ATC_THREADS, AtcLayout<128>::SMEM_BYTES, st>>>(tK, tV, q, pos, M, kv_len, o, lse, Hq, Hkv, scale_log2, h->dev_status, g_attn_dbg);
   else
-    attention_tc_kernel<64><<<grid, ATC_THREADS, AtcLayout<64>::SMEM_BYTES, st>>>(tK, tV, q, pos, M, kv_len, o, lse, Hq, Hkv, scale_log2, h->dev_status);
+    attention_tc_kernel<64><<<grid, ATC_THREADS, AtcLayout<64>::SMEM_BYTES, st>>>(tK, tV, q, pos, M, kv_len, o, lse, Hq, Hkv, scale_log2, h->dev_status, g_attn_dbg);
   A3_LAUNCHED();
   return A3_OK;
 }
 
 }  // namespace a3
+
+extern "C" void a3_internal_set_attn_dbg(int v) { a3::g_attn_dbg = v; }
