@@ -12,9 +12,12 @@ int build_rope_table(float2* tab, int max_pos, int D, double base, cudaStream_t 
 struct LayerWs {
   bf16 *a, *q, *o, *hmid;
   float* lse;
+  void* attn_part;
+  size_t attn_part_bytes;
   size_t bytes;
 };
-static LayerWs carve_layer_ws(const a3_model_desc& m, int rows, void* base) {
+static LayerWs carve_layer_ws(const a3_handle* h, int rows, void* base) {
+  const a3_model_desc& m = h->m;
   LayerWs w;
   char* p = (char*)base;
   size_t off = 0;
@@ -29,6 +32,8 @@ static LayerWs carve_layer_ws(const a3_model_desc& m, int rows, void* base) {
   w.o = (bf16*)take(R * m.n_q_heads * m.head_dim * 2);
   w.hmid = (bf16*)take(R * m.d_ff * 2);
   w.lse = (float*)take(R * m.n_q_heads * 4);
+  w.attn_part_bytes = attention_part_bytes(h);
+  w.attn_part = take(w.attn_part_bytes);
   w.bytes = off;
   return w;
 }
@@ -40,7 +45,8 @@ struct RequestWs {
   void* layer;
   size_t bytes;
 };
-static RequestWs carve_request_ws(const a3_model_desc& m, int n, void* base) {
+static RequestWs carve_request_ws(const a3_handle* h, int n, void* base) {
+  const a3_model_desc& m = h->m;
   RequestWs w;
   char* p = (char*)base;
   size_t off = 0;
@@ -53,7 +59,7 @@ static RequestWs carve_request_ws(const a3_model_desc& m, int n, void* base) {
   w.x_all = (bf16*)take(N * m.d_model * 2);
   w.all_pos = (int32_t*)take(N * 4);
   w.lse_q = (float*)take(N * m.n_q_heads * 4);
-  w.layer = take(carve_layer_ws(m, n, nullptr).bytes);
+  w.layer = take(carve_layer_ws(h, n, nullptr).bytes);
   w.bytes = off;
   return w;
 }
@@ -203,12 +209,12 @@ extern "C" void a3_destroy(a3_handle* h) {
 
 extern "C" size_t a3_layer_workspace_bytes(const a3_handle* h, int max_rows) {
   if (!h || max_rows < 0) return 0;
-  return carve_layer_ws(h->m, max_rows, nullptr).bytes;
+  return carve_layer_ws(h, max_rows, nullptr).bytes;
 }
 
 extern "C" size_t a3_request_workspace_bytes(const a3_handle* h, int n) {
   if (!h || n < 0) return 0;
-  return carve_request_ws(h->m, n, nullptr).bytes;
+  return carve_request_ws(h, n, nullptr).bytes;
 }
 
 extern "C" int a3_device_status(const a3_handle* h, uint32_t* bits_out, a3_stream stream) {
@@ -272,7 +278,7 @@ static int recompute_layer_impl(const a3_handle* h, int layer, bf16* x, const in
   const int qd = m.n_q_heads * m.head_dim;
   A3_TRY(rmsnorm_rows(h, x, (const bf16*)lw.attn_norm, m.rms_eps, M, m.d_model, w.a, st));
   A3_TRY(qkv_project(h, layer, w.a, pos, M, 0, w.q, kc, vc, kv_len, st));
-  A3_TRY(attention_rows(h, w.q, pos, M, kc, vc, kv_len, w.o, lse_out, st));
+  A3_TRY(attention_rows(h, w.q, pos, M, kc, vc, kv_len, w.o, lse_out, w.attn_part, w.attn_part_bytes, st));
   GemmArgs g{};
   g.A = w.o;
   g.M = M;
@@ -313,7 +319,7 @@ extern "C" int a3_recompute_layer(const a3_handle* h, int layer, void* x_rows, c
   if (!x_rows || !pos || !k_layer || !v_layer || !ws) return A3_EINVAL;
   if (kv_len > h->m.max_positions || M > kv_len) return A3_EINVAL;
   if (((uintptr_t)x_rows | (uintptr_t)k_layer | (uintptr_t)v_layer | (uintptr_t)ws) & 15) return A3_EINVAL;
-  LayerWs w = carve_layer_ws(h->m, M, ws);
+  LayerWs w = carve_layer_ws(h, M, ws);
   if (w.bytes > ws_bytes) return A3_EWORKSPACE;
   cudaStream_t st = (cudaStream_t)stream;
   A3_TRY(check_rows(h, pos, M, kv_len, st));
@@ -334,7 +340,7 @@ extern "C" int a3_query_scores(const a3_handle* h, const void* q_rows, const int
     const size_t need = align_up((size_t)nq * h->m.n_q_heads * 4, 256);
     if (!ws || ws_bytes < need) return A3_EWORKSPACE;
     A3_TRY(attention_rows(h, (const bf16*)q_rows, q_pos, nq, (const bf16*)k_layer, (const bf16*)k_layer, kv_len, nullptr,
-                          (float*)ws, st));
+                          (float*)ws, nullptr, 0, st));
     lse = (const float*)ws;
   }
   return scores_pass(h, (const bf16*)q_rows, q_pos, nq, (const bf16*)k_layer, kv_len, cand_begin, cand_end, lse, scores, st);
@@ -356,11 +362,11 @@ extern "C" int a3_fuse_request(const a3_handle* h, const a3_request* r, void* ws
   const size_t layer_bytes = (size_t)n * m.n_kv_heads * m.head_dim * 2;
   if (r->layer_stride < layer_bytes || (r->layer_stride & 15)) return A3_EINVAL;
   if (((uintptr_t)r->x0 | (uintptr_t)r->k_fused | (uintptr_t)r->v_fused | (uintptr_t)r->x_out | (uintptr_t)ws) & 15) return A3_EINVAL;
-  RequestWs w = carve_request_ws(m, n, ws);
+  RequestWs w = carve_request_ws(h, n, ws);
   if (w.bytes > ws_bytes) return A3_EWORKSPACE;
   cudaStream_t st = (cudaStream_t)stream;
   const int p = r->n_recompute, nq = r->n_question, M = p + nq, ls = r->select_layer;
-  LayerWs lw = carve_layer_ws(m, n, w.layer);
+  LayerWs lw = carve_layer_ws(h, n, w.layer);
   auto kl = [&](int l) { return (bf16*)((char*)r->k_fused + (size_t)l * r->layer_stride); };
   auto vl = [&](int l) { return (bf16*)((char*)r->v_fused + (size_t)l * r->layer_stride); };
 
@@ -377,7 +383,7 @@ extern "C" int a3_fuse_request(const a3_handle* h, const a3_request* r, void* ws
   A3_TRY(qkv_project(h, ls, lw.a, w.all_pos, n, r->n_ctx, lw.q, kl(ls), vl(ls), n, st));
   A3_CUDA(cudaMemsetAsync(r->scores_out, 0, (size_t)n * 4, st));
   if (nq > 0) {
-    A3_TRY(attention_rows(h, lw.q, w.all_pos + r->n_ctx, nq, kl(ls), vl(ls), n, nullptr, w.lse_q, st));
+    A3_TRY(attention_rows(h, lw.q, w.all_pos + r->n_ctx, nq, kl(ls), vl(ls), n, nullptr, w.lse_q, nullptr, 0, st));
     A3_TRY(scores_pass(h, lw.q, w.all_pos + r->n_ctx, nq, kl(ls), n, r->n_system, r->n_ctx, w.lse_q, r->scores_out, st));
   }
   if (p > 0) {

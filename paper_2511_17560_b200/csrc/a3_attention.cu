@@ -223,14 +223,14 @@ attention_kernel(const bf16* __restrict__ q, const int32_t* __restrict__ pos, in
 }
 
 int attention_rows_tc(const a3_handle* h, const bf16* q, const int32_t* pos, int M, const bf16* k, const bf16* v,
-                      int kv_len, bf16* o, float* lse, cudaStream_t st);
+                      int kv_len, bf16* o, float* lse, void* part, size_t part_bytes, cudaStream_t st);
 // 0: tcgen05 kernel (a3_attention_tc.cu); 1: the warp-level mma.sync kernel in this file (cross-check for bring-up)
 int g_attn_impl = 0;
 
 int attention_rows(const a3_handle* h, const bf16* q, const int32_t* pos, int M, const bf16* k, const bf16* v,
-                   int kv_len, bf16* o, float* lse, cudaStream_t st) {
+                   int kv_len, bf16* o, float* lse, void* part, size_t part_bytes, cudaStream_t st) {
   if (M <= 0) return A3_OK;
-  if (g_attn_impl == 0) return attention_rows_tc(h, q, pos, M, k, v, kv_len, o, lse, st);
+  if (g_attn_impl == 0) return attention_rows_tc(h, q, pos, M, k, v, kv_len, o, lse, part, part_bytes, st);
   const int Hq = h->m.n_q_heads, Hkv = h->m.n_kv_heads, D = h->m.head_dim;
   const int G = Hq / Hkv;
   dim3 grid(cdiv((long long)M * G, AT_BM), Hkv);

@@ -164,11 +164,14 @@ struct AtcLayout {
   static constexpr int SMEM_BYTES = BAR_OFF + 256 + 1024;
 };
 
+#define ATC_PROBE(slot) do { if ((dbg & 16) && blockIdx.x == 0 && blockIdx.y == 0 && blockIdx.z == 0) status[64 + 3000 * 4 + (slot)] = (uint32_t)atc::global_ns(); } while (0)
+
 template <int D>
 __global__ void __launch_bounds__(ATC_THREADS, 1)
 attention_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV,
                     const bf16* __restrict__ q, const int32_t* __restrict__ pos, int M, int kv_len, bf16* __restrict__ o,
-                    float* __restrict__ lse, int Hq, int Hkv, float scale_log2, uint32_t* status, int dbg) {
+                    float* __restrict__ lse, int Hq, int Hkv, float scale_log2, uint32_t* status, int dbg,
+                    int tiles_per_split, float* __restrict__ part_o, float2* __restrict__ part_ml) {
   using L = AtcLayout<D>;
   using namespace atc;
   extern __shared__ unsigned char smem_raw[];
@@ -188,6 +191,7 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
   volatile int* abort_flag = reinterpret_cast<volatile int*>(base_ptr + L::BAR_OFF + 8 * 11 + 8);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const unsigned long long t_entry = (dbg & 8) ? atc::global_ns() : 0ull;
   const int G = Hq / Hkv;
   const int g = blockIdx.y;
   const int tile = gridDim.x - 1 - blockIdx.x;  // latest (longest) row tiles first
@@ -198,7 +202,15 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
   const int last_tok = min(M - 1, (r0 + ATC_BM - 1) / G);
   const int maxpos = min(pos[last_tok], kv_len - 1);
   const int minpos = pos[r0 / G];
-  const int nkt = maxpos < 0 ? 0 : maxpos / ATC_BN + 1;
+  const int nkt_all = maxpos < 0 ? 0 : maxpos / ATC_BN + 1;
+  // Split over the keys (blockIdx.z): when the grid has few row tiles, long tiles are cut into segments of
+  // tiles_per_split key tiles that run as separate CTAs and leave unnormalised partial results (output, exponent
+  // reference, row sum) for a combine kernel.  A row tile short enough for one segment writes its result directly.
+  const int n_active = (nkt_all + tiles_per_split - 1) / tiles_per_split;
+  if ((int)blockIdx.z >= max(n_active, 1)) return;  // uniform for the CTA: nothing has been set up yet
+  const int kt0 = blockIdx.z * tiles_per_split;
+  const int nkt = max(0, min(tiles_per_split, nkt_all - kt0));  // key tiles of this CTA; loops count locally
+  const bool partial = n_active > 1;
 
   if (threadIdx.x == 0) {
     for (int i = 0; i < 2; ++i) {
@@ -218,10 +230,12 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32((const void*)tmem_slot)), "r"(512) : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
   }
+  if (threadIdx.x == 64) { if ((dbg & 16) && blockIdx.x == 0 && blockIdx.y == 0 && blockIdx.z == 0) status[64 + 3000 * 4 + 0] = (uint32_t)t_entry; ATC_PROBE(1); }
   fence_before();
   __syncthreads();
   fence_after();
   const uint32_t tmem_base = *tmem_slot;
+  if (threadIdx.x == 64) ATC_PROBE(2);
   const uint32_t tmem_s0 = tmem_base, tmem_o = tmem_base + 256;
 
   if (warp == 0) {
@@ -236,8 +250,8 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
         mbar_expect_tx(kv_full(s), L::KV_STAGE);
 #pragma unroll
         for (int j = 0; j < D / 64; ++j) {
-          tma_load_2d(sk + j * L::SUB, &tmK, g * D + 64 * j, kt * ATC_BN, kv_full(s));
-          tma_load_2d(sv + j * L::SUB, &tmV, g * D + 64 * j, kt * ATC_BN, kv_full(s));
+          tma_load_2d(sk + j * L::SUB, &tmK, g * D + 64 * j, (kt0 + kt) * ATC_BN, kv_full(s));
+          tma_load_2d(sv + j * L::SUB, &tmV, g * D + 64 * j, (kt0 + kt) * ATC_BN, kv_full(s));
         }
       }
     }
@@ -257,7 +271,9 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
         commit(s_full(kt & 1));
       };
       bool ok = mbar_wait(q_ready, 0, abort_flag, status);
+      ATC_PROBE(3);
       ok = ok && mbar_wait(kv_full(0), 0, abort_flag, status);
+      ATC_PROBE(4);
       if (ok) {
         fence_after();
         issue_s(0);
@@ -266,13 +282,13 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
         if (kt + 1 < nkt) {
           ok = mbar_wait(kv_full((kt + 1) & 1), ((kt + 1) >> 1) & 1, abort_flag, status);
           if (!ok) break;
-          if ((dbg & 4) && blockIdx.x == 0 && blockIdx.y == 0 && kt < 60) status[64 + kt * 4 + 2] = (uint32_t)global_ns();
+
           fence_after();
           issue_s(kt + 1);
         }
         ok = mbar_wait(p_ready(kt & 1), (kt >> 1) & 1, abort_flag, status);
         if (!ok) break;
-        if ((dbg & 4) && blockIdx.x == 0 && blockIdx.y == 0 && kt < 60) status[64 + kt * 4 + 3] = (uint32_t)global_ns();
+
         fence_after();
         if (want_o) {
           const uint32_t sv = base + L::KV_OFF + (kt & 1) * L::KV_STAGE + (D / 64) * L::SUB;
@@ -308,6 +324,7 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
       }
       fence_async_smem();
       mbar_arrive(q_ready);
+      if (row == 0) ATC_PROBE(5);
     }
 
     // Exponent reference m_ref and row sum l_run relative to it.  The reference is the true maximum of the first
@@ -323,9 +340,9 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
       ok = __all_sync(0xffffffffu, mbar_wait(s_full(kt & 1), (kt >> 1) & 1, abort_flag, status));
       if (!ok) break;
       fence_after();
-      if ((dbg & 4) && blockIdx.x == 0 && blockIdx.y == 0 && row == 0 && kt < 60) status[64 + kt * 4 + 0] = (uint32_t)global_ns();
+      if (row == 0 && kt == 0) ATC_PROBE(6);
       const uint32_t ts = tmem_s0 + (kt & 1) * 128 + lane_addr;
-      const int key0 = kt * ATC_BN;
+      const int key0 = (kt0 + kt) * ATC_BN;
       const bool need_mask = key0 + ATC_BN - 1 > minpos;
       if (kt == 0) {
         float mx = -INFINITY;
@@ -398,7 +415,7 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
         }
       }
       if (!ok) break;
-      if (want_o && kt == nkt - 1) {
+      if (want_o && kt0 + kt == nkt_all - 1) {
         // slots beyond the CTA's last visible key may hold anything: they get probability zero, and zero times a
         // non-finite value would still poison the product, so clear those V rows of the last tile
         const int first_bad = maxpos - key0 + 1;
@@ -412,14 +429,17 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
         }
       }
       if ((dbg & 2) && lane == 0) atomicAdd(status + 2, 1u);
-      if ((dbg & 4) && blockIdx.x == 0 && blockIdx.y == 0 && row == 0 && kt < 60) status[64 + kt * 4 + 1] = (uint32_t)global_ns();
+      if (row == 0 && kt == 0) ATC_PROBE(7);
+      if (row == 0 && kt == nkt - 1) ATC_PROBE(8);
       fence_async_smem();
       fence_before();
       mbar_arrive(p_ready(kt & 1));
     }
     const float inv = l_run > 0.f ? 1.f / l_run : 0.f;
+    const size_t prow = ((size_t)blockIdx.z * Hkv + g) * ((size_t)gridDim.x * ATC_BM) + fr;  // partial-result row
     if (ok && want_o && nkt > 0) {
       ok = __all_sync(0xffffffffu, mbar_wait(p_free((nkt - 1) & 1), ((nkt - 1) >> 1) & 1, abort_flag, status));
+      if (row == 0) ATC_PROBE(10);
       if (ok) {
         fence_after();
         bf16* dst = o + ((size_t)tok * Hq + hq) * D;
@@ -428,7 +448,11 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
           float t[32];
           ld32(tmem_o + lane_addr + c * 32, t);
           wait_ld();
-          if (row_ok) {
+          if (row_ok && partial) {
+            float4* pd = reinterpret_cast<float4*>(part_o + prow * D + c * 32);
+#pragma unroll
+            for (int i = 0; i < 8; ++i) pd[i] = make_float4(t[4 * i], t[4 * i + 1], t[4 * i + 2], t[4 * i + 3]);
+          } else if (row_ok) {
 #pragma unroll
             for (int e = 0; e < 32; ++e) t[e] *= inv;
 #pragma unroll
@@ -438,11 +462,72 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
         }
       }
     }
-    if (ok && row_ok && lse) lse[(size_t)tok * Hq + hq] = l_run > 0.f ? (m_ref + log2f(l_run)) * ATC_LN2 : -INFINITY;
+    if (row == 0) ATC_PROBE(9);
+    if (ok && row_ok && partial) part_ml[prow] = make_float2(m_ref, l_run);
+    if (ok && row_ok && !partial && lse) lse[(size_t)tok * Hq + hq] = l_run > 0.f ? (m_ref + log2f(l_run)) * ATC_LN2 : -INFINITY;
+  }
+  if ((dbg & 8) && threadIdx.x == 64) {
+    // per-CTA record: entry, exit (ns, low 32 bits), key tiles, SM id
+    const int cta = (blockIdx.z * gridDim.y + blockIdx.y) * gridDim.x + blockIdx.x;
+    if (cta < 3000) {
+      uint32_t smid;
+      asm volatile("mov.u32 %0, %%smid;" : "=r"(smid));
+      status[64 + cta * 4 + 0] = (uint32_t)t_entry;
+      status[64 + cta * 4 + 1] = (uint32_t)atc::global_ns();
+      status[64 + cta * 4 + 2] = (uint32_t)nkt;
+      status[64 + cta * 4 + 3] = smid;
+    }
   }
   atc::fence_before();
   __syncthreads();
+  if (threadIdx.x == 64) ATC_PROBE(11);
   if (warp == 1) asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(512) : "memory");
+}
+
+// One warp per (flat row, KV head) of a row tile that was split over the keys: merges the segments' partial results
+// in segment order (fixed, so the result is reproducible): O = sum_z O_z 2^(m_z - m) / sum_z l_z 2^(m_z - m).
+template <int D>
+__global__ void __launch_bounds__(128)
+attention_combine_kernel(const int32_t* __restrict__ pos, int M, int kv_len, int Hq, int Hkv, int tiles_per_split, int rows_pad,
+                         const float* __restrict__ part_o, const float2* __restrict__ part_ml, bf16* __restrict__ o,
+                         float* __restrict__ lse) {
+  const int G = Hq / Hkv;
+  const int rows_total = M * G;
+  const int fr = blockIdx.x * 4 + (threadIdx.x >> 5);
+  const int g = blockIdx.y, lane = threadIdx.x & 31;
+  if (fr >= rows_total) return;
+  const int r0 = (fr / ATC_BM) * ATC_BM;
+  const int last_tok = min(M - 1, (r0 + ATC_BM - 1) / G);
+  const int maxpos = min(pos[last_tok], kv_len - 1);
+  const int nkt_all = maxpos < 0 ? 0 : maxpos / ATC_BN + 1;
+  const int n_active = (nkt_all + tiles_per_split - 1) / tiles_per_split;
+  if (n_active <= 1) return;  // written directly by the attention kernel
+  float m = -INFINITY;
+  for (int z = 0; z < n_active; ++z) {
+    const float2 ml = part_ml[((size_t)z * Hkv + g) * rows_pad + fr];
+    if (ml.y > 0.f) m = fmaxf(m, ml.x);
+  }
+  constexpr int PER = D / 32;
+  float acc[PER];
+#pragma unroll
+  for (int e = 0; e < PER; ++e) acc[e] = 0.f;
+  float l = 0.f;
+  for (int z = 0; z < n_active; ++z) {
+    const size_t prow = ((size_t)z * Hkv + g) * rows_pad + fr;
+    const float2 ml = part_ml[prow];
+    if (!(ml.y > 0.f)) continue;
+    const float w = exp2f(ml.x - m);
+    l += ml.y * w;
+    const float* src = part_o + prow * D + lane * PER;
+#pragma unroll
+    for (int e = 0; e < PER; ++e) acc[e] += src[e] * w;
+  }
+  const int tok = fr / G, hq = g * G + fr % G;
+  const float inv = l > 0.f ? 1.f / l : 0.f;
+  bf16* dst = o + ((size_t)tok * Hq + hq) * D + lane * PER;
+#pragma unroll
+  for (int e = 0; e < PER; e += 2) *reinterpret_cast<uint32_t*>(dst + e) = pack2(acc[e] * inv, acc[e + 1] * inv);
+  if (lse && lane == 0) lse[(size_t)tok * Hq + hq] = l > 0.f ? (m + log2f(l)) * ATC_LN2 : -INFINITY;
 }
 
 // ---------------------------------------------------------------- host side
@@ -474,9 +559,16 @@ static int make_cache_tmap(CUtensorMap* map, const void* ptr, long long rows, lo
 }
 
 int g_attn_dbg = 0;
+int g_attn_split = 0;  // 0: choose; otherwise the number of key segments (tuning)
+
+size_t attention_part_bytes(const a3_handle* h) {
+  // split only happens when the unsplit grid has fewer than two CTAs per SM; up to 4 segments
+  const size_t rows = (size_t)2 * (h->sm_count > 0 ? h->sm_count : 148) * ATC_BM;
+  return 4 * rows * ((size_t)h->m.head_dim + 2) * sizeof(float);
+}
 
 int attention_rows_tc(const a3_handle* h, const bf16* q, const int32_t* pos, int M, const bf16* k, const bf16* v,
-                      int kv_len, bf16* o, float* lse, cudaStream_t st) {
+                      int kv_len, bf16* o, float* lse, void* part, size_t part_bytes, cudaStream_t st) {
   if (M <= 0) return A3_OK;
   const int Hq = h->m.n_q_heads, Hkv = h->m.n_kv_heads, D = h->m.head_dim;
   const int G = Hq / Hkv;
@@ -485,6 +577,21 @@ int attention_rows_tc(const a3_handle* h, const bf16* q, const int32_t* pos, int
   A3_TRY(make_cache_tmap(&tV, v, kv_len, (long long)Hkv * D));
   dim3 grid(cdiv((long long)M * G, ATC_BM), Hkv);
   const float scale_log2 = ATC_LOG2E / sqrtf((float)D);
+  // split over the keys when the grid would leave SMs idle behind a few long row tiles
+  const int sms = h->sm_count > 0 ? h->sm_count : 148;
+  const int base_ctas = (int)grid.x * Hkv, all_tiles = cdiv(kv_len, ATC_BN);
+  int n_split = 1;
+  if (o && part && base_ctas < 2 * sms && all_tiles >= 8) {
+    n_split = g_attn_split > 0 ? g_attn_split : 2;  // measured: 2 segments beat 1, 3 and 4 at 208 base CTAs (7-8 us fixed cost per CTA)
+    const size_t need = (size_t)n_split * base_ctas * ATC_BM * ((size_t)D + 2) * sizeof(float);
+    if (need > part_bytes) n_split = 1;
+  }
+  const int tiles_per_split = cdiv(all_tiles, n_split);
+  n_split = cdiv(all_tiles, tiles_per_split);
+  grid.z = n_split;
+  const int rows_pad = (int)grid.x * ATC_BM;
+  float* part_o = (float*)part;
+  float2* part_ml = part ? (float2*)(part_o + (size_t)n_split * Hkv * rows_pad * D) : nullptr;
   static bool attr_set = false;
   if (!attr_set) {
     A3_CUDA(cudaFuncSetAttribute(attention_tc_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, AtcLayout<128>::SMEM_BYTES));
@@ -493,13 +600,20 @@ int attention_rows_tc(const a3_handle* h, const bf16* q, const int32_t* pos, int
   }
   ProfScope prof(h, A3_K_ATTENTION, st);
   if (D == 128)
-    attention_tc_kernel<128><<<grid, ATC_THREADS, AtcLayout<128>::SMEM_BYTES, st>>>(tK, tV, q, pos, M, kv_len, o, lse, Hq, Hkv, scale_log2, h->dev_status, g_attn_dbg);
+    attention_tc_kernel<128><<<grid, ATC_THREADS, AtcLayout<128>::SMEM_BYTES, st>>>(tK, tV, q, pos, M, kv_len, o, lse, Hq, Hkv, scale_log2, h->dev_status, g_attn_dbg, tiles_per_split, part_o, part_ml);
   else
-    attention_tc_kernel<64><<<grid, ATC_THREADS, AtcLayout<64>::SMEM_BYTES, st>>>(tK, tV, q, pos, M, kv_len, o, lse, Hq, Hkv, scale_log2, h->dev_status, g_attn_dbg);
+    attention_tc_kernel<64><<<grid, ATC_THREADS, AtcLayout<64>::SMEM_BYTES, st>>>(tK, tV, q, pos, M, kv_len, o, lse, Hq, Hkv, scale_log2, h->dev_status, g_attn_dbg, tiles_per_split, part_o, part_ml);
   A3_LAUNCHED();
+  if (n_split > 1) {
+    dim3 cgrid(cdiv((long long)M * G, 4), Hkv);
+    if (D == 128) attention_combine_kernel<128><<<cgrid, 128, 0, st>>>(pos, M, kv_len, Hq, Hkv, tiles_per_split, rows_pad, part_o, part_ml, o, lse);
+    else attention_combine_kernel<64><<<cgrid, 128, 0, st>>>(pos, M, kv_len, Hq, Hkv, tiles_per_split, rows_pad, part_o, part_ml, o, lse);
+    A3_LAUNCHED();
+  }
   return A3_OK;
 }
 
 }  // namespace a3
 
+extern "C" void a3_internal_set_attn_split(int v) { a3::g_attn_split = v; }
 extern "C" void a3_internal_set_attn_dbg(int v) { a3::g_attn_dbg = v; }

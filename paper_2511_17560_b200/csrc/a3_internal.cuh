@@ -118,8 +118,10 @@ int gemm_bf16(const a3_handle* h, GemmEpilogue epi, const GemmArgs& a, cudaStrea
 
 // Causal attention of M rows (at cache slots pos[m]) over a [kv_len][Hkv][D] cache.
 // q: [M][Hq][D]; o: [M][Hq][D] (may be null: statistics only); lse: [M][Hq] or null.
+// part / part_bytes: optional scratch for partial results when the keys are split across CTAs (attention_part_bytes).
 int attention_rows(const a3_handle* h, const bf16* q, const int32_t* pos, int M, const bf16* k, const bf16* v,
-                   int kv_len, bf16* o, float* lse, cudaStream_t st);
+                   int kv_len, bf16* o, float* lse, void* part, size_t part_bytes, cudaStream_t st);
+size_t attention_part_bytes(const a3_handle* h);
 
 int scores_pass(const a3_handle* h, const bf16* q, const int32_t* q_pos, int nq, const bf16* k, int kv_len,
                 int cand_begin, int cand_end, const float* lse, float* scores, cudaStream_t st);

@@ -60,6 +60,6 @@ extern "C" int a3_query_scores_static(const a3_handle* h, const void* q_rows, co
   A3_TRY(scratch_on_current_device(&lse));
   cudaStream_t st = (cudaStream_t)stream;
   if (nq > 0)
-    A3_TRY(attention_rows(h, (const bf16*)q_rows, q_pos, nq, (const bf16*)k_layer, (const bf16*)k_layer, kv_len, nullptr, lse, st));
+    A3_TRY(attention_rows(h, (const bf16*)q_rows, q_pos, nq, (const bf16*)k_layer, (const bf16*)k_layer, kv_len, nullptr, lse, nullptr, 0, st));
   return scores_pass(h, (const bf16*)q_rows, q_pos, nq, (const bf16*)k_layer, kv_len, cand_begin, cand_end, lse, scores, st);
 }
