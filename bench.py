@@ -63,7 +63,8 @@ def algorithmic_work(m, r, p, rows):
     vis_rows = float(np.sum(np.asarray(rows, dtype=np.float64) + 1.0))
     w["attention"] = 4.0 * D * Hq * (ls * vis_full + (L - ls) * vis_rows) + 2.0 * D * Hq * vis_q
     w["scores"] = 2.0 * D * Hq * vis_q
-    b = {"rerotate": 4.0 * r.n_ctx * kvd * 2 * L}
+    # position recovery is queued for the layers above the selection layer (the others are recomputed for every row)
+    b = {"rerotate": 4.0 * r.n_ctx * kvd * 2 * (L - ls - 1)}
     return w, b
 
 
@@ -365,7 +366,8 @@ def run_a3(args):
         torch.cuda.synchronize()
         wall = time.perf_counter() - t0
         sec_e = max_over_ranks(max(e0.elapsed_time(e1) / 1e3, wall), dev)
-        h2d = sum(k.numel() * 2 for k in hk) * 2 + hx.numel() * 2
+        copied_layers = m.n_layers - r.select_layer - 1  # caches of layers <= select_layer are recomputed, not copied
+        h2d = sum(k.numel() * 2 for k in hk) * 2 * copied_layers // m.n_layers + hx.numel() * 2
         d2h = rows_h.numel() * 4 + x_h.numel() * 2
         e2e = {"value": aggregate_value(r.n_ctx, args.steps, world, sec_e), "unit": UNIT, "ms_per_step": sec_e / args.steps * 1e3,
                "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h)}

@@ -191,6 +191,8 @@ int a3_gather_rows(const a3_handle* h, const void* src, int n_src, const int32_t
 /* The whole request (Method, "Attention-Aware Accurate Fusion"): position recovery of all layers,
  * the leading full blocks 0..select_layer-1 over all n rows, true K/V of all rows and question
  * queries at select_layer, scores, selection, then layers select_layer..L-1 on rows R only.
+ * (Position recovery is queued for layers above select_layer only: the layers below it and the
+ * selection layer itself get true K/V for every row, so recovered values there would never be read.)
  * Fills the fused cache in place, rows_out, scores_out, x_out. */
 int a3_fuse_request(const a3_handle* h, const a3_request* req, void* ws, size_t ws_bytes, a3_stream stream);
 
@@ -198,10 +200,12 @@ int a3_fuse_request(const a3_handle* h, const a3_request* req, void* ws, size_t 
 int a3_fuse_batch(const a3_handle* h, const a3_request* reqs, int n_requests, void* ws, size_t ws_bytes,
                   a3_stream stream);
 
-/* a3_fuse_request with the chunk caches and embeddings in HOST memory: copies them to `staging`
- * (dev, a3_host_staging_bytes), builds the chunk descriptors, fuses, copies rows_out and x_out
- * back to the host and waits for the stream.  req->chunks, req->x0 are ignored (taken from io);
- * the fused cache and scores stay on the device. */
+/* a3_fuse_request with the chunk caches and embeddings in HOST memory (pinned memory lets the copies
+ * overlap the compute): copies them to `staging` (dev, a3_host_staging_bytes) on a copy stream the
+ * handle creates on first use, layer by layer, while `stream` computes; builds the chunk descriptors,
+ * fuses, copies rows_out and x_out back to the host and waits for both streams.  Chunk caches of
+ * layers up to select_layer are not copied: those layers are recomputed for every row.
+ * req->chunks, req->x0 are ignored (taken from io); the fused cache and scores stay on the device. */
 int a3_fuse_request_host(const a3_handle* h, const a3_request* req, const a3_host_io* io, void* staging,
                          size_t staging_bytes, void* ws, size_t ws_bytes, a3_stream stream);
 

@@ -198,9 +198,12 @@ extern "C" int a3_internal_read_debug(const a3_handle* h, uint32_t* out, int n_w
   return A3_OK;
 }
 
+namespace a3 { static void host_pipe_destroy(a3_handle* h); }
+
 extern "C" void a3_destroy(a3_handle* h) {
   if (!h) return;
   a3_profile_enable(h, 0);
+  host_pipe_destroy(h);
   if (h->rope_tab) cudaFree(h->rope_tab);
   if (h->dev_status) cudaFree(h->dev_status);
   free(h->layers);
@@ -347,7 +350,19 @@ extern "C" int a3_query_scores(const a3_handle* h, const void* q_rows, const int
 }
 
 // ------------------------------------------------------------------ the whole request
+namespace a3 {
+// layer_ready (optional, [n_layers]): event after which layer l's chunk caches are in device memory; position
+// recovery of layer l is then queued behind it, just before the layer needs the cache (host-buffer entry).
+static int fuse_impl(const a3_handle* h, const a3_request* r, void* ws, size_t ws_bytes, a3_stream stream,
+                     const cudaEvent_t* layer_ready, cudaEvent_t x0_ready);
+}
+
 extern "C" int a3_fuse_request(const a3_handle* h, const a3_request* r, void* ws, size_t ws_bytes, a3_stream stream) {
+  return fuse_impl(h, r, ws, ws_bytes, stream, nullptr, nullptr);
+}
+
+static int a3::fuse_impl(const a3_handle* h, const a3_request* r, void* ws, size_t ws_bytes, a3_stream stream,
+                         const cudaEvent_t* layer_ready, cudaEvent_t x0_ready) {
   if (!h || !r || !ws) return A3_EINVAL;
   const a3_model_desc& m = h->m;
   if (r->n_ctx < 0 || r->n_question < 0 || r->n_system < 0 || r->n_system > r->n_ctx || r->n_chunks < 0) return A3_EINVAL;
@@ -370,10 +385,14 @@ extern "C" int a3_fuse_request(const a3_handle* h, const a3_request* r, void* ws
   auto kl = [&](int l) { return (bf16*)((char*)r->k_fused + (size_t)l * r->layer_stride); };
   auto vl = [&](int l) { return (bf16*)((char*)r->v_fused + (size_t)l * r->layer_stride); };
 
-  // position recovery of every layer in one launch (Eq. 2)
-  A3_TRY(a3_rope_rerotate(h, r->chunks, r->n_chunks, r->max_chunk_len, r->k_fused, r->v_fused, r->layer_stride, 0,
-                          m.n_layers, stream));
+  // Position recovery (Eq. 2) in one launch.  Layers up to the selection layer are skipped: every row of their
+  // caches is rewritten with true values below (full blocks; K/V of all rows at the selection layer), so the
+  // recovered values would never be read.
+  if (!layer_ready && ls + 1 < m.n_layers)
+    A3_TRY(a3_rope_rerotate(h, r->chunks, r->n_chunks, r->max_chunk_len, r->k_fused, r->v_fused, r->layer_stride, ls + 1,
+                            m.n_layers, stream));
   // leading full blocks: the whole input through layers 0..select_layer-1
+  if (x0_ready) A3_CUDA(cudaStreamWaitEvent(st, x0_ready, 0));
   A3_CUDA(cudaMemcpyAsync(w.x_all, r->x0, (size_t)n * m.d_model * 2, cudaMemcpyDeviceToDevice, st));
   A3_TRY(iota_rows(h, w.all_pos, 0, n, st));
   for (int l = 0; l < ls; ++l)
@@ -391,12 +410,24 @@ extern "C" int a3_fuse_request(const a3_handle* h, const a3_request* r, void* ws
     else A3_TRY(a3_topk_select(h, r->scores_out, r->n_system, r->n_ctx, p, r->rows_out, stream));
   }
   A3_TRY(iota_rows(h, r->rows_out + p, r->n_ctx, nq, st));
-  if (M == 0) return A3_OK;
+  if (M == 0) {
+    if (layer_ready)
+      for (int l = ls + 1; l < m.n_layers; ++l) {
+        A3_CUDA(cudaStreamWaitEvent(st, layer_ready[l], 0));
+        A3_TRY(a3_rope_rerotate(h, r->chunks, r->n_chunks, r->max_chunk_len, r->k_fused, r->v_fused, r->layer_stride, l, l + 1, stream));
+      }
+    return A3_OK;
+  }
   A3_TRY(check_rows(h, r->rows_out, M, n, st));
   A3_TRY(a3_gather_rows(h, w.x_all, n, r->rows_out, M, m.d_model, r->x_out, stream));
   // layers select_layer..L-1 on rows [Re, Q] only (Eq. 4, Eq. 5)
-  for (int l = ls; l < m.n_layers; ++l)
+  for (int l = ls; l < m.n_layers; ++l) {
+    if (layer_ready && l > ls) {
+      A3_CUDA(cudaStreamWaitEvent(st, layer_ready[l], 0));
+      A3_TRY(a3_rope_rerotate(h, r->chunks, r->n_chunks, r->max_chunk_len, r->k_fused, r->v_fused, r->layer_stride, l, l + 1, stream));
+    }
     A3_TRY(recompute_layer_impl(h, l, (bf16*)r->x_out, r->rows_out, M, kl(l), vl(l), n, nullptr, lw, st));
+  }
   return A3_OK;
 }
 
@@ -417,6 +448,48 @@ extern "C" size_t a3_host_staging_bytes(const a3_handle* h, int n_ctx, int n) {
          align_up((size_t)(n_ctx + 1) * sizeof(a3_chunk_ref), 256);
 }
 
+namespace a3 {
+// copy stream and events of the host-buffer entry, created on first use and kept by the handle
+struct HostPipe {
+  cudaStream_t copy_stream;
+  cudaEvent_t start, x0_ready;
+  cudaEvent_t* layer_ready;
+  int n_layers;
+};
+static int host_pipe(const a3_handle* h, HostPipe** out) {
+  a3_handle* hm = const_cast<a3_handle*>(h);
+  if (!hm->host_pipe) {
+    HostPipe* p = (HostPipe*)calloc(1, sizeof(HostPipe));
+    if (!p) return A3_EINVAL;
+    p->n_layers = h->m.n_layers;
+    p->layer_ready = (cudaEvent_t*)calloc(p->n_layers, sizeof(cudaEvent_t));
+    cudaError_t e = cudaStreamCreateWithFlags(&p->copy_stream, cudaStreamNonBlocking);
+    if (e == cudaSuccess) e = cudaEventCreateWithFlags(&p->start, cudaEventDisableTiming);
+    if (e == cudaSuccess) e = cudaEventCreateWithFlags(&p->x0_ready, cudaEventDisableTiming);
+    for (int l = 0; l < p->n_layers && e == cudaSuccess; ++l) e = cudaEventCreateWithFlags(&p->layer_ready[l], cudaEventDisableTiming);
+    if (e != cudaSuccess) return cuda_fail(e);
+    hm->host_pipe = p;
+  }
+  *out = (HostPipe*)hm->host_pipe;
+  return A3_OK;
+}
+static void host_pipe_destroy(a3_handle* h) {
+  HostPipe* p = (HostPipe*)h->host_pipe;
+  if (!p) return;
+  for (int l = 0; l < p->n_layers; ++l)
+    if (p->layer_ready[l]) cudaEventDestroy(p->layer_ready[l]);
+  if (p->start) cudaEventDestroy(p->start);
+  if (p->x0_ready) cudaEventDestroy(p->x0_ready);
+  if (p->copy_stream) cudaStreamDestroy(p->copy_stream);
+  free(p->layer_ready);
+  free(p);
+  h->host_pipe = nullptr;
+}
+}  // namespace a3
+
+// Copies run on the handle's own copy stream, layer by layer, while the compute stream works: the embeddings go
+// first (the full block needs only them), then each layer's chunk caches; position recovery of a layer is queued
+// behind that layer's copy.  Layers up to the selection layer are never copied: their caches are recomputed.
 extern "C" int a3_fuse_request_host(const a3_handle* h, const a3_request* req, const a3_host_io* io, void* staging,
                                     size_t staging_bytes, void* ws, size_t ws_bytes, a3_stream stream) {
   if (!h || !req || !io || !staging) return A3_EINVAL;
@@ -425,8 +498,11 @@ extern "C" int a3_fuse_request_host(const a3_handle* h, const a3_request* req, c
   const a3_model_desc& m = h->m;
   const int n = req->n_ctx + req->n_question;
   if (req->n_ctx < 0 || req->n_question < 0 || req->n_chunks < 0 || req->n_chunks > req->n_ctx + 1) return A3_EINVAL;
+  if (req->select_layer < 0 || req->select_layer >= m.n_layers) return A3_EINVAL;
   if (a3_host_staging_bytes(h, req->n_ctx, n) > staging_bytes) return A3_EWORKSPACE;
-  cudaStream_t st = (cudaStream_t)stream;
+  HostPipe* hp = nullptr;
+  A3_TRY(host_pipe(h, &hp));
+  cudaStream_t st = (cudaStream_t)stream, cs = hp->copy_stream;
   const size_t row = (size_t)m.n_kv_heads * m.head_dim * 2;
   char* base = (char*)staging;
   char* kv = base;
@@ -443,12 +519,6 @@ extern "C" int a3_fuse_request_host(const a3_handle* h, const a3_request* req, c
       return A3_EINVAL;
     }
     const size_t bytes = (size_t)m.n_layers * len * row;
-    cudaError_t e = cudaMemcpyAsync(kv + kvoff, io->chunk_k[c], bytes, cudaMemcpyHostToDevice, st);
-    if (e == cudaSuccess) e = cudaMemcpyAsync(kv + kvoff + bytes, io->chunk_v[c], bytes, cudaMemcpyHostToDevice, st);
-    if (e != cudaSuccess) {
-      free(href);
-      return cuda_fail(e);
-    }
     href[c].k_src = kv + kvoff;
     href[c].v_src = kv + kvoff + bytes;
     href[c].src_layer_stride = (uint64_t)len * row;
@@ -464,22 +534,36 @@ extern "C" int a3_fuse_request_host(const a3_handle* h, const a3_request* req, c
     free(href);
     return A3_EINVAL;
   }
-  cudaError_t e = cudaMemcpyAsync(x0, io->x0, (size_t)n * m.d_model * 2, cudaMemcpyHostToDevice, st);
+  // the copy stream starts after whatever the caller has already queued on `stream` (the staging area may be in use)
+  cudaError_t e = cudaEventRecord(hp->start, st);
+  if (e == cudaSuccess) e = cudaStreamWaitEvent(cs, hp->start, 0);
   // the descriptor array is pageable host memory: this copy returns only once it has been staged
   if (e == cudaSuccess && req->n_chunks > 0)
-    e = cudaMemcpyAsync(dref, href, sizeof(a3_chunk_ref) * req->n_chunks, cudaMemcpyHostToDevice, st);
+    e = cudaMemcpyAsync(dref, href, sizeof(a3_chunk_ref) * req->n_chunks, cudaMemcpyHostToDevice, cs);
+  if (e == cudaSuccess) e = cudaMemcpyAsync(x0, io->x0, (size_t)n * m.d_model * 2, cudaMemcpyHostToDevice, cs);
+  if (e == cudaSuccess) e = cudaEventRecord(hp->x0_ready, cs);
+  for (int l = req->select_layer + 1; l < m.n_layers && e == cudaSuccess; ++l) {
+    for (int c = 0; c < req->n_chunks && e == cudaSuccess; ++c) {
+      const size_t slice = (size_t)href[c].len * row;
+      e = cudaMemcpyAsync((char*)href[c].k_src + l * slice, (const char*)io->chunk_k[c] + l * slice, slice, cudaMemcpyHostToDevice, cs);
+      if (e == cudaSuccess)
+        e = cudaMemcpyAsync((char*)href[c].v_src + l * slice, (const char*)io->chunk_v[c] + l * slice, slice, cudaMemcpyHostToDevice, cs);
+    }
+    if (e == cudaSuccess) e = cudaEventRecord(hp->layer_ready[l], cs);
+  }
   free(href);
   if (e != cudaSuccess) return cuda_fail(e);
   a3_request r = *req;
   r.chunks = dref;
   r.max_chunk_len = maxlen;
   r.x0 = x0;
-  A3_TRY(a3_fuse_request(h, &r, ws, ws_bytes, stream));
+  A3_TRY(fuse_impl(h, &r, ws, ws_bytes, stream, hp->layer_ready, hp->x0_ready));
   const int M = r.n_recompute + r.n_question;
   if (M > 0) {
     A3_CUDA(cudaMemcpyAsync(io->rows_out, r.rows_out, (size_t)M * 4, cudaMemcpyDeviceToHost, st));
     A3_CUDA(cudaMemcpyAsync(io->x_out, r.x_out, (size_t)M * m.d_model * 2, cudaMemcpyDeviceToHost, st));
   }
   A3_CUDA(cudaStreamSynchronize(st));
+  A3_CUDA(cudaStreamSynchronize(cs));
   return A3_OK;
 }

@@ -191,7 +191,7 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
   volatile int* abort_flag = reinterpret_cast<volatile int*>(base_ptr + L::BAR_OFF + 8 * 11 + 8);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const unsigned long long t_entry = (dbg & 8) ? atc::global_ns() : 0ull;
+  const unsigned long long t_entry = (dbg & 24) ? atc::global_ns() : 0ull;
   const int G = Hq / Hkv;
   const int g = blockIdx.y;
   const int tile = gridDim.x - 1 - blockIdx.x;  // latest (longest) row tiles first
@@ -212,6 +212,7 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
   const int nkt = max(0, min(tiles_per_split, nkt_all - kt0));  // key tiles of this CTA; loops count locally
   const bool partial = n_active > 1;
 
+  if (threadIdx.x == 64) ATC_PROBE(12);  // after the position loads
   if (threadIdx.x == 0) {
     for (int i = 0; i < 2; ++i) {
       mbar_init(kv_full(i), 1);
@@ -229,6 +230,7 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
   if (warp == 1) {
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32((const void*)tmem_slot)), "r"(512) : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    if (lane == 0) ATC_PROBE(13);  // after the TMEM allocation
   }
   if (threadIdx.x == 64) { if ((dbg & 16) && blockIdx.x == 0 && blockIdx.y == 0 && blockIdx.z == 0) status[64 + 3000 * 4 + 0] = (uint32_t)t_entry; ATC_PROBE(1); }
   fence_before();

@@ -20,6 +20,7 @@ struct a3_handle {
   int sm_count;
   void* tmaps;               // host-side tensor-map cache (a3_gemm_tc.cu)
   a3::Profiler* prof;        // null unless a3_profile_enable is on
+  void* host_pipe;           // copy stream + events of a3_fuse_request_host, created on first use
 };
 
 namespace a3 {

@@ -235,15 +235,30 @@ int check_rows(const a3_handle* h, const int32_t* pos, int M, int kv_len, cudaSt
 }
 
 // ------------------------------------------------------------------ RMSNorm
-// One CTA per row; fp32 statistics; out = x * rsqrt(mean(x^2) + eps) * gain, rounded once to bf16.
-constexpr int RN_THREADS = 128;
+// One CTA per row; the row is read once into registers (16-byte vectors), fp32 sum of squares by shuffles and one
+// shared-memory exchange, out = x * rsqrt(mean(x^2) + eps) * gain rounded once to bf16.  Rows wider than
+// RN_THREADS * RN_VPT vectors fall back to a second read of the tail.
+constexpr int RN_THREADS = 128, RN_VPT = 4;
 __global__ void __launch_bounds__(RN_THREADS)
 rmsnorm_kernel(const uint4* __restrict__ x, const uint4* __restrict__ gain, float eps, int row_vecs, uint4* __restrict__ out) {
   const uint4* xr = x + (size_t)blockIdx.x * row_vecs;
+  uint4 v[RN_VPT];
   float ss = 0.f;
-  for (int v = threadIdx.x; v < row_vecs; v += RN_THREADS) {
+#pragma unroll
+  for (int i = 0; i < RN_VPT; ++i) {
+    const int idx = threadIdx.x + i * RN_THREADS;
+    v[i] = idx < row_vecs ? __ldg(xr + idx) : make_uint4(0, 0, 0, 0);
+  }
+#pragma unroll
+  for (int i = 0; i < RN_VPT; ++i) {
     float f[8];
-    unpack8(xr[v], f);
+    unpack8(v[i], f);
+#pragma unroll
+    for (int e = 0; e < 8; ++e) ss += f[e] * f[e];
+  }
+  for (int idx = threadIdx.x + RN_VPT * RN_THREADS; idx < row_vecs; idx += RN_THREADS) {
+    float f[8];
+    unpack8(__ldg(xr + idx), f);
 #pragma unroll
     for (int e = 0; e < 8; ++e) ss += f[e] * f[e];
   }
@@ -257,13 +272,25 @@ rmsnorm_kernel(const uint4* __restrict__ x, const uint4* __restrict__ gain, floa
   for (int w = 0; w < RN_THREADS / 32; ++w) tot += part[w];
   const float inv = rsqrtf(tot / (float)(row_vecs * 8) + eps);
   uint4* orow = out + (size_t)blockIdx.x * row_vecs;
-  for (int v = threadIdx.x; v < row_vecs; v += RN_THREADS) {
+#pragma unroll
+  for (int i = 0; i < RN_VPT; ++i) {
+    const int idx = threadIdx.x + i * RN_THREADS;
+    if (idx < row_vecs) {
+      float f[8], g[8], r[8];
+      unpack8(v[i], f);
+      unpack8(__ldg(gain + idx), g);
+#pragma unroll
+      for (int e = 0; e < 8; ++e) r[e] = f[e] * inv * g[e];
+      orow[idx] = pack8(r);
+    }
+  }
+  for (int idx = threadIdx.x + RN_VPT * RN_THREADS; idx < row_vecs; idx += RN_THREADS) {
     float f[8], g[8], r[8];
-    unpack8(xr[v], f);
-    unpack8(__ldg(gain + v), g);
+    unpack8(__ldg(xr + idx), f);
+    unpack8(__ldg(gain + idx), g);
 #pragma unroll
     for (int e = 0; e < 8; ++e) r[e] = f[e] * inv * g[e];
-    orow[v] = pack8(r);
+    orow[idx] = pack8(r);
   }
 }
 

@@ -66,5 +66,5 @@ def test_algorithmic_work_matches_hand_count():
     gemm = fl["gemm_qkv"] + fl["gemm_residual"] + fl["gemm_swiglu"]
     expect = per_row * (5152 + 31 * M) + 2 * 4096 * (5152 * 2048 + 32 * 4096)
     assert gemm == pytest.approx(expect)
-    assert by["rerotate"] == 4 * 5120 * 1024 * 2 * 32
+    assert by["rerotate"] == 4 * 5120 * 1024 * 2 * 30
     assert 14e12 < gemm + fl["attention"] + fl["scores"] < 15.5e12
