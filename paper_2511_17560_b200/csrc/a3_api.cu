@@ -123,8 +123,8 @@ extern "C" int a3_create(a3_handle** out, const a3_model_desc* m, const a3_layer
   cudaError_t e = cudaGetDevice(&h->device);
   if (e == cudaSuccess) e = cudaDeviceGetAttribute(&h->sm_count, cudaDevAttrMultiProcessorCount, h->device);
   if (e == cudaSuccess) e = cudaMalloc((void**)&h->rope_tab, (size_t)m->max_positions * (m->head_dim / 2) * sizeof(float2));
-  if (e == cudaSuccess) e = cudaMalloc((void**)&h->dev_status, 65536);
-  if (e == cudaSuccess) e = cudaMemset(h->dev_status, 0, 65536);
+  if (e == cudaSuccess) e = cudaMalloc((void**)&h->dev_status, 256);
+  if (e == cudaSuccess) e = cudaMemset(h->dev_status, 0, 256);
   if (e != cudaSuccess) {
     a3_destroy(h);
     return cuda_fail(e);
@@ -187,15 +187,6 @@ extern "C" const char* a3_kernel_class_name(int cls) {
   static const char* names[A3_K_CLASSES] = {"rerotate", "rmsnorm", "gemm_qkv", "attention", "gemm_residual",
                                             "gemm_swiglu", "scores", "topk", "rows"};
   return cls >= 0 && cls < A3_K_CLASSES ? names[cls] : "?";
-}
-
-// Debug words behind the status word (used by timing probes during tuning).
-extern "C" int a3_internal_read_debug(const a3_handle* h, uint32_t* out, int n_words) {
-  if (!h || !out || n_words < 0 || n_words > 16000) return A3_EINVAL;
-  A3_CUDA(cudaDeviceSynchronize());
-  A3_CUDA(cudaMemcpy(out, h->dev_status + 64, (size_t)n_words * 4, cudaMemcpyDeviceToHost));
-  A3_CUDA(cudaMemset(h->dev_status + 64, 0, (size_t)n_words * 4));
-  return A3_OK;
 }
 
 namespace a3 { static void host_pipe_destroy(a3_handle* h); }

@@ -1,353 +1,589 @@
-// Attention of the carried rows over the fused GQA cache (Eq. 4, Eq. 5) and the question->context relevance
-// scores (Eq. 3).  Row m sits at global position pos[m] and sees cache slots 0..pos[m].
+// Attention of the carried rows over the fused GQA cache (Eq. 4, Eq. 5) on the 5th-generation tensor cores.
 //
-// Both kernels pack the G = Hq/Hkv query heads that share one KV head into the row dimension of the tile
-// (flat row r -> token r / G, head r % G), so a K/V tile is read once per group rather than once per head.
-// Softmax statistics are fp32 in the exp2 domain; the score kernel never materialises the probability
-// matrix: it reduces exp(logit - lse) down the rows with warp shuffles and sums heads in a fixed order,
-// which makes the scores bit-reproducible from run to run.
+// Row m sits at global position pos[m] and sees cache slots 0..pos[m].  The G = Hq/Hkv query heads that share one
+// KV head are packed into the row dimension (flat row r -> token r / G, head r % G); one CTA owns 128 flat rows of
+// one KV head and walks the keys in tiles of 128 up to the largest position among its rows.
+//
+//   warp 0 (one lane)   TMA producer: K and V tiles of the cache ([slots][Hkv*D] seen as a 2-D tensor, 128-byte
+//                       swizzle, two stages).
+//   warp 1 (one lane)   tcgen05.mma issuer: S = Q K^T (128 x 128 x D) into one of two TMEM buffers, and, once the
+//                       probabilities of a tile are in shared memory, O~ = P V (128 x D x 128, V as an MN-major
+//                       operand) accumulated into a third TMEM buffer.  S of tile t+1 is issued before P V of tile t, so the
+//                       tensor core works while the softmax threads do.
+//   warps 2..5          one thread per row: one pass over the row of S in TMEM (exp2 against a lazily raised
+//                       reference maximum, row sum), P written as bf16 into shared memory in the swizzled K-major
+//                       layout the MMA reads; the output accumulates in TMEM across key tiles and is rescaled there
+//                       only when the reference has to be raised; final normalisation and stores.
+// Statistics are fp32 in the exp2 domain.  Every mbarrier wait is bounded (see a3_gemm.cu); there is no block-
+// wide or named barrier inside the loops, so a role that gives up cannot strand another.
+#include <cuda.h>
+
 #include "a3_internal.cuh"
 
 namespace a3 {
 
-constexpr int AT_THREADS = 128;  // 4 warps x 16 rows
-constexpr int AT_BM = 64, AT_BN = 64;
-constexpr float LOG2E = 1.4426950408889634f, LN2 = 0.6931471805599453f;
+constexpr int ATC_THREADS = 192;
+constexpr int ATC_BM = 128, ATC_BN = 128;
+constexpr unsigned long long ATC_WAIT_NS = 500000000ull;
+constexpr float ATC_LOG2E = 1.4426950408889634f, ATC_LN2 = 0.6931471805599453f;
 
-// byte offset of 16-byte chunk c of row r in a [rows][D] bf16 tile (row pitch D*2 bytes), XOR-swizzled
-template <int D>
-__device__ __forceinline__ uint32_t tswz(int r, int c) {
-  return (uint32_t)(r * (D * 2) + ((c ^ (r & 7)) << 4));
+namespace atc {
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
 }
-
-// copies a [64][D] tile; row i comes from base + row_index(i)*stride (elements); invalid rows are zero-filled
-template <int D, typename RowFn>
-__device__ __forceinline__ void load_tile(uint32_t sdst, const bf16* safe, RowFn row_ptr) {
-  constexpr int CPR = D / 8;
-#pragma unroll
-  for (int i = 0; i < (64 * CPR) / AT_THREADS; ++i) {
-    int idx = threadIdx.x + i * AT_THREADS;
-    int r = idx / CPR, c = idx % CPR;
-    const bf16* src = row_ptr(r);
-    cp_async16(sdst + tswz<D>(r, c), src ? src + c * 8 : safe, src != nullptr);
-  }
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
 }
-
-template <int D>
-__device__ __forceinline__ void load_q_frags(uint32_t sq, int warp, int lane, uint32_t (&qf)[D / 16][4]) {
-#pragma unroll
-  for (int ks = 0; ks < D / 16; ++ks) {
-    int r = warp * 16 + (lane & 7) + ((lane >> 3) & 1) * 8;
-    int c = ks * 2 + (lane >> 4);
-    ldmatrix_x4(sq + tswz<D>(r, c), qf[ks][0], qf[ks][1], qf[ks][2], qf[ks][3]);
-  }
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
 }
-
-// S(16 x 64) = Q(16 x D) K_tile(64 x D)^T for this warp
-template <int D>
-__device__ __forceinline__ void qk_tile(uint32_t sk, int lane, const uint32_t (&qf)[D / 16][4], float (&s)[8][4]) {
-#pragma unroll
-  for (int j = 0; j < 8; ++j)
-#pragma unroll
-    for (int e = 0; e < 4; ++e) s[j][e] = 0.f;
-#pragma unroll
-  for (int ks = 0; ks < D / 16; ++ks) {
-#pragma unroll
-    for (int jj = 0; jj < 4; ++jj) {
-      uint32_t b0, b1, b2, b3;
-      int r = jj * 16 + (lane & 7) + (lane >> 4) * 8;
-      int c = ks * 2 + ((lane >> 3) & 1);
-      ldmatrix_x4(sk + tswz<D>(r, c), b0, b1, b2, b3);
-      mma_bf16(s[2 * jj], qf[ks], b0, b1);
-      mma_bf16(s[2 * jj + 1], qf[ks], b2, b3);
+__device__ __forceinline__ uint32_t mbar_try_wait(uint32_t bar, uint32_t parity) {
+  uint32_t done;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.b32 %0, 1, 0, p;\n\t}"
+      : "=r"(done)
+      : "r"(bar), "r"(parity)
+      : "memory");
+  return done;
+}
+__device__ __forceinline__ unsigned long long global_ns() {
+  unsigned long long t;
+  asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
+  return t;
+}
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, uint32_t* status) {
+  if (mbar_try_wait(bar, parity)) return true;
+  const unsigned long long t0 = global_ns();
+  for (;;) {
+#pragma unroll 1
+    for (int i = 0; i < 32; ++i)
+      if (mbar_try_wait(bar, parity)) return true;
+    if (*abort_flag) return false;
+    if (global_ns() - t0 > ATC_WAIT_NS) {
+      *abort_flag = 1;
+      atomicOr(status, A3_DEV_WAIT_EXHAUSTED);
+      return false;
     }
   }
 }
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int x, int y, uint32_t bar) {
+  asm volatile("cp.async.bulk.tensor.2d.shared::cta.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+               ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(bar)
+               : "memory");
+}
+__device__ __forceinline__ void fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+__device__ __forceinline__ void commit(uint32_t bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void mma_f16(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+      ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+__device__ __forceinline__ void ld32(uint32_t taddr, float* v) {
+  uint32_t* r = reinterpret_cast<uint32_t*>(v);
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+        "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]),
+        "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]),
+        "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+      : "r"(taddr)
+      : "memory");
+}
+__device__ __forceinline__ void wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+__device__ __forceinline__ void st32(uint32_t taddr, const float* v) {
+  const uint32_t* r = reinterpret_cast<const uint32_t*>(v);
+  asm volatile(
+      "tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16, "
+      "%17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31, %32};"
+      ::"r"(taddr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]), "r"(r[8]),
+        "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15]), "r"(r[16]), "r"(r[17]),
+        "r"(r[18]), "r"(r[19]), "r"(r[20]), "r"(r[21]), "r"(r[22]), "r"(r[23]), "r"(r[24]), "r"(r[25]), "r"(r[26]),
+        "r"(r[27]), "r"(r[28]), "r"(r[29]), "r"(r[30]), "r"(r[31])
+      : "memory");
+}
+__device__ __forceinline__ void wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 
-// ------------------------------------------------------------------ attention
+// K-major [rows][64] bf16 sub-tile, 128-byte swizzle, 8-row groups 1024 bytes apart
+__device__ __forceinline__ uint64_t desc_k_sw128(uint32_t saddr) {
+  return (uint64_t)((saddr & 0x3FFFFu) >> 4) | ((uint64_t)(1024u >> 4) << 32) | (1ull << 46) | (2ull << 61);
+}
+// MN-major operand stored as [k rows][64 mn elements] sub-tiles (one 128-byte row per k), 128-byte swizzle:
+// 8-k-row groups are 1024 bytes apart (SBO), successive 64-element mn atoms `lbo` bytes apart (LBO)
+__device__ __forceinline__ uint64_t desc_mn_sw128(uint32_t saddr, uint32_t lbo) {
+  return (uint64_t)((saddr & 0x3FFFFu) >> 4) | ((uint64_t)((lbo >> 4) & 0x3FFFu) << 16) | ((uint64_t)(1024u >> 4) << 32) |
+         (1ull << 46) | (2ull << 61);
+}
+// bf16 x bf16 -> fp32, M = 128, A K-major; b_mn = 1 when B is MN-major
+__host__ __device__ constexpr uint32_t idesc(int n, int b_mn) {
+  return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)b_mn << 16) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(ATC_BM >> 4) << 24);
+}
+// byte offset of element chunk (16 bytes) j of row r inside a [rows][64] bf16 sub-tile with the 128-byte swizzle
+__device__ __forceinline__ uint32_t swz(int r, int j) { return (uint32_t)(r * 128 + ((j ^ (r & 7)) << 4)); }
+}  // namespace atc
+
+__device__ __forceinline__ float ex2_approx(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+// 32 logits of one row -> probabilities (in place), running relative maximum and four partial row sums.
+// t = s * scale - m_ref is one FMA; ex2.approx maps -inf to +0, so masked keys need no second select.
+template <bool MASK>
+__device__ __forceinline__ void softmax_chunk(float* sv, int key_base, int lim, float scale, float neg_ref, float& mx, float (&ls)[4]) {
+#pragma unroll
+  for (int e = 0; e < 32; ++e) {
+    float t = fmaf(sv[e], scale, neg_ref);
+    if (MASK && key_base + e > lim) t = -INFINITY;
+    mx = fmaxf(mx, t);
+    const float pe = ex2_approx(t);
+    sv[e] = pe;
+    ls[e & 3] += pe;
+  }
+}
+
 template <int D>
-__global__ void __launch_bounds__(AT_THREADS)
-attention_kernel(const bf16* __restrict__ q, const int32_t* __restrict__ pos, int M, const bf16* __restrict__ k,
-                 const bf16* __restrict__ v, int kv_len, bf16* __restrict__ o, float* __restrict__ lse, int Hq, int Hkv,
-                 float scale_log2) {
-  extern __shared__ __align__(128) unsigned char smem[];
-  constexpr int TILE = 64 * D * 2;
-  const uint32_t sq = smem_u32(smem);
-  const uint32_t skv = sq + TILE;  // [stage][K,V]
-  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+struct AtcLayout {
+  static constexpr int SUB = 128 * 64 * 2;           // one [128][64] bf16 sub-tile: 16 KiB
+  static constexpr int Q_BYTES = (D / 64) * SUB;
+  static constexpr int KV_STAGE = 2 * (D / 64) * SUB;  // K then V
+  static constexpr int P_BYTES = 2 * SUB;                // one P buffer; two of them alternate
+  static constexpr int Q_OFF = 0;
+  static constexpr int KV_OFF = Q_BYTES;
+  static constexpr int P_OFF = KV_OFF + 2 * KV_STAGE;
+  static constexpr int BAR_OFF = P_OFF + 2 * P_BYTES;
+  static constexpr int SMEM_BYTES = BAR_OFF + 256 + 1024;
+};
+
+template <int D>
+__global__ void __launch_bounds__(ATC_THREADS, 1)
+attention_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV,
+                    const bf16* __restrict__ q, const int32_t* __restrict__ pos, int M, int kv_len, bf16* __restrict__ o,
+                    float* __restrict__ lse, int Hq, int Hkv, float scale_log2, uint32_t* status,
+                    int tiles_per_split, float* __restrict__ part_o, float2* __restrict__ part_ml) {
+  using L = AtcLayout<D>;
+  using namespace atc;
+  extern __shared__ unsigned char smem_raw[];
+  const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+  unsigned char* base_ptr = smem_raw + (base - smem_u32(smem_raw));
+  // barriers: kv_full[2], kv_empty[2], s_full[2], p_ready[2], q_ready, p_free[2]
+  const uint32_t bars = base + L::BAR_OFF;
+  auto kv_full = [&](int s) { return bars + 8u * s; };
+  auto kv_empty = [&](int s) { return bars + 8u * (2 + s); };
+  auto s_full = [&](int b) { return bars + 8u * (4 + b); };
+  // p_ready alternates between two barriers: a fast warp may finish tile t+1 before a slow warp has arrived for
+  // tile t, and on a single barrier its second arrival would be counted towards tile t
+  auto p_ready = [&](int b) { return bars + 8u * (6 + b); };
+  const uint32_t q_ready = bars + 8u * 8;
+  auto p_free = [&](int b) { return bars + 8u * (9 + b); };
+  volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(base_ptr + L::BAR_OFF + 8 * 11);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(base_ptr + L::BAR_OFF + 8 * 11 + 8);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int G = Hq / Hkv;
   const int g = blockIdx.y;
-  const int tile = gridDim.x - 1 - blockIdx.x;  // heaviest (latest) row tiles first
-  const int r0 = tile * AT_BM;
+  const int tile = gridDim.x - 1 - blockIdx.x;  // latest (longest) row tiles first
+  const int r0 = tile * ATC_BM;
   const int rows_total = M * G;
-  const int kvrow = Hkv * D;
+  const bool want_o = o != nullptr;
 
-  auto q_row = [&](int r) -> const bf16* {
-    int fr = r0 + r;
-    if (fr >= rows_total) return nullptr;
-    int t = fr / G, hg = fr % G;
-    return q + ((size_t)t * Hq + g * G + hg) * D;
-  };
-  int last_tok = min(M - 1, (r0 + AT_BM - 1) / G);
-  int maxpos = min(pos[last_tok], kv_len - 1);
+  const int last_tok = min(M - 1, (r0 + ATC_BM - 1) / G);
+  const int maxpos = min(pos[last_tok], kv_len - 1);
   const int minpos = pos[r0 / G];
-  const int nkt = maxpos < 0 ? 0 : maxpos / AT_BN + 1;
+  const int nkt_all = maxpos < 0 ? 0 : maxpos / ATC_BN + 1;
+  // Split over the keys (blockIdx.z): when the grid has few row tiles, long tiles are cut into segments of
+  // tiles_per_split key tiles that run as separate CTAs and leave unnormalised partial results (output, exponent
+  // reference, row sum) for a combine kernel.  A row tile short enough for one segment writes its result directly.
+  const int n_active = (nkt_all + tiles_per_split - 1) / tiles_per_split;
+  if ((int)blockIdx.z >= max(n_active, 1)) return;  // uniform for the CTA: nothing has been set up yet
+  const int kt0 = blockIdx.z * tiles_per_split;
+  const int nkt = max(0, min(tiles_per_split, nkt_all - kt0));  // key tiles of this CTA; loops count locally
+  const bool partial = n_active > 1;
 
-  auto load_kv = [&](int stage, int kt) {
-    const int key0 = kt * AT_BN;
-    load_tile<D>(skv + stage * 2 * TILE, k, [&](int r) -> const bf16* {
-      int key = key0 + r;
-      return key <= maxpos ? k + (size_t)key * kvrow + g * D : nullptr;
-    });
-    load_tile<D>(skv + stage * 2 * TILE + TILE, v, [&](int r) -> const bf16* {
-      int key = key0 + r;
-      return key <= maxpos ? v + (size_t)key * kvrow + g * D : nullptr;
-    });
-  };
-
-  load_tile<D>(sq, q, q_row);
-  if (nkt > 0) load_kv(0, 0);
-  cp_async_commit();
-
-  // row limits of the two rows this thread owns in the accumulator layout
-  const int gq = lane >> 2, tq = lane & 3;
-  int lim[2];
-#pragma unroll
-  for (int hlf = 0; hlf < 2; ++hlf) {
-    int fr = r0 + warp * 16 + gq + hlf * 8;
-    lim[hlf] = fr < rows_total ? min(pos[fr / G], kv_len - 1) : -1;
+  if (threadIdx.x == 0) {
+    for (int i = 0; i < 2; ++i) {
+      mbar_init(kv_full(i), 1);
+      mbar_init(kv_empty(i), 1);
+      mbar_init(s_full(i), 1);
+      mbar_init(p_free(i), 1);
+    }
+    mbar_init(p_ready(0), 128);
+    mbar_init(p_ready(1), 128);
+    mbar_init(q_ready, 128);
+    abort_flag[0] = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    fence_async_smem();
   }
+  if (warp == 1) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32((const void*)tmem_slot)), "r"(512) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  fence_before();
+  __syncthreads();
+  fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+  const uint32_t tmem_s0 = tmem_base, tmem_o = tmem_base + 256;
 
-  uint32_t qf[D / 16][4];
-  float oacc[D / 8][4];
+  if (warp == 0) {
+    // ---------------- TMA producer
+    if (lane == 0) {
+      asm volatile("prefetch.tensormap [%0];" ::"l"(&tmK) : "memory");
+      asm volatile("prefetch.tensormap [%0];" ::"l"(&tmV) : "memory");
+      for (int kt = 0; kt < nkt; ++kt) {
+        const int s = kt & 1;
+        if (!mbar_wait(kv_empty(s), ((kt >> 1) & 1) ^ 1, abort_flag, status)) break;
+        const uint32_t sk = base + L::KV_OFF + s * L::KV_STAGE, sv = sk + (D / 64) * L::SUB;
+        mbar_expect_tx(kv_full(s), L::KV_STAGE);
 #pragma unroll
-  for (int j = 0; j < D / 8; ++j)
-#pragma unroll
-    for (int e = 0; e < 4; ++e) oacc[j][e] = 0.f;
-  float mx[2] = {-INFINITY, -INFINITY}, lsum[2] = {0.f, 0.f};
-
-  for (int kt = 0; kt < nkt; ++kt) {
-    if (kt + 1 < nkt) load_kv((kt + 1) & 1, kt + 1);
-    cp_async_commit();
-    cp_async_wait<1>();
-    __syncthreads();
-    if (kt == 0) load_q_frags<D>(sq, warp, lane, qf);
-    const uint32_t sk = skv + (kt & 1) * 2 * TILE, sv = sk + TILE;
-
-    float s[8][4];
-    qk_tile<D>(sk, lane, qf, s);
-
-    const int key0 = kt * AT_BN;
-    const bool need_mask = key0 + AT_BN - 1 > minpos;
-    float tmax[2] = {-INFINITY, -INFINITY};
-#pragma unroll
-    for (int j = 0; j < 8; ++j)
-#pragma unroll
-      for (int e = 0; e < 4; ++e) {
-        float x = s[j][e] * scale_log2;
-        if (need_mask) {
-          int key = key0 + j * 8 + 2 * tq + (e & 1);
-          if (key > lim[e >> 1]) x = -INFINITY;
+        for (int j = 0; j < D / 64; ++j) {
+          tma_load_2d(sk + j * L::SUB, &tmK, g * D + 64 * j, (kt0 + kt) * ATC_BN, kv_full(s));
+          tma_load_2d(sv + j * L::SUB, &tmV, g * D + 64 * j, (kt0 + kt) * ATC_BN, kv_full(s));
         }
-        s[j][e] = x;
-        tmax[e >> 1] = fmaxf(tmax[e >> 1], x);
-      }
-    float alpha[2], mref[2];
-#pragma unroll
-    for (int hlf = 0; hlf < 2; ++hlf) {
-      tmax[hlf] = fmaxf(tmax[hlf], __shfl_xor_sync(0xffffffffu, tmax[hlf], 1));
-      tmax[hlf] = fmaxf(tmax[hlf], __shfl_xor_sync(0xffffffffu, tmax[hlf], 2));
-      float mnew = fmaxf(mx[hlf], tmax[hlf]);
-      mref[hlf] = mnew == -INFINITY ? 0.f : mnew;
-      alpha[hlf] = exp2f(mx[hlf] - mref[hlf]);  // mx = -inf -> 0
-      mx[hlf] = mnew;
-      lsum[hlf] *= alpha[hlf];
-    }
-#pragma unroll
-    for (int j = 0; j < 8; ++j)
-#pragma unroll
-      for (int e = 0; e < 4; ++e) {
-        float pe = exp2f(s[j][e] - mref[e >> 1]);
-        s[j][e] = pe;
-        lsum[e >> 1] += pe;
-      }
-#pragma unroll
-    for (int j = 0; j < D / 8; ++j) {
-      oacc[j][0] *= alpha[0];
-      oacc[j][1] *= alpha[0];
-      oacc[j][2] *= alpha[1];
-      oacc[j][3] *= alpha[1];
-    }
-    // O += P V
-#pragma unroll
-    for (int kk = 0; kk < AT_BN / 16; ++kk) {
-      uint32_t pa[4];
-      pa[0] = pack2(s[2 * kk][0], s[2 * kk][1]);
-      pa[1] = pack2(s[2 * kk][2], s[2 * kk][3]);
-      pa[2] = pack2(s[2 * kk + 1][0], s[2 * kk + 1][1]);
-      pa[3] = pack2(s[2 * kk + 1][2], s[2 * kk + 1][3]);
-#pragma unroll
-      for (int jd = 0; jd < D / 16; ++jd) {
-        uint32_t b0, b1, b2, b3;
-        int mi = lane >> 3;
-        int r = kk * 16 + (lane & 7) + (mi & 1) * 8;
-        int c = jd * 2 + (mi >> 1);
-        ldmatrix_x4_trans(sv + tswz<D>(r, c), b0, b1, b2, b3);
-        mma_bf16(oacc[2 * jd], pa, b0, b1);
-        mma_bf16(oacc[2 * jd + 1], pa, b2, b3);
       }
     }
-    __syncthreads();  // everyone is done with this stage before it is refilled
-  }
-  cp_async_wait<0>();
+  } else if (warp == 1) {
+    // ---------------- MMA issuer
+    if (lane == 0 && nkt > 0) {
+      constexpr uint32_t idesc_s = idesc(ATC_BN, 0);
+      constexpr uint32_t idesc_o = idesc(D, 1);
+      const uint32_t sq = base + L::Q_OFF, sp = base + L::P_OFF;
+      auto issue_s = [&](int kt) {
+        const uint32_t sk = base + L::KV_OFF + (kt & 1) * L::KV_STAGE;
+#pragma unroll
+        for (int k = 0; k < D / 16; ++k) {
+          const uint32_t sub = (k / 4) * L::SUB + (k % 4) * 32;
+          mma_f16(tmem_s0 + (kt & 1) * 128, desc_k_sw128(sq + sub), desc_k_sw128(sk + sub), idesc_s, k != 0);
+        }
+        commit(s_full(kt & 1));
+      };
+      bool ok = mbar_wait(q_ready, 0, abort_flag, status);
+      ok = ok && mbar_wait(kv_full(0), 0, abort_flag, status);
+      if (ok) {
+        fence_after();
+        issue_s(0);
+      }
+      for (int kt = 0; kt < nkt && ok; ++kt) {
+        if (kt + 1 < nkt) {
+          ok = mbar_wait(kv_full((kt + 1) & 1), ((kt + 1) >> 1) & 1, abort_flag, status);
+          if (!ok) break;
 
+          fence_after();
+          issue_s(kt + 1);
+        }
+        ok = mbar_wait(p_ready(kt & 1), (kt >> 1) & 1, abort_flag, status);
+        if (!ok) break;
+
+        fence_after();
+        if (want_o) {
+          const uint32_t sv = base + L::KV_OFF + (kt & 1) * L::KV_STAGE + (D / 64) * L::SUB;
 #pragma unroll
-  for (int hlf = 0; hlf < 2; ++hlf) {
-    lsum[hlf] += __shfl_xor_sync(0xffffffffu, lsum[hlf], 1);
-    lsum[hlf] += __shfl_xor_sync(0xffffffffu, lsum[hlf], 2);
-  }
-#pragma unroll
-  for (int hlf = 0; hlf < 2; ++hlf) {
-    int fr = r0 + warp * 16 + gq + hlf * 8;
-    if (fr >= rows_total) continue;
-    int t = fr / G, hq = g * G + fr % G;
-    float inv = lsum[hlf] > 0.f ? 1.f / lsum[hlf] : 0.f;
-    if (o) {
-      bf16* orow = o + ((size_t)t * Hq + hq) * D;
-#pragma unroll
-      for (int j = 0; j < D / 8; ++j)
-        *reinterpret_cast<uint32_t*>(orow + j * 8 + 2 * tq) = pack2(oacc[j][2 * hlf] * inv, oacc[j][2 * hlf + 1] * inv);
+          for (int k = 0; k < ATC_BN / 16; ++k) {
+            const uint64_t da = desc_k_sw128(sp + (kt & 1) * L::P_BYTES + (k / 4) * L::SUB + (k % 4) * 32);
+            const uint64_t db = desc_mn_sw128(sv + k * 16 * 128, L::SUB);
+            mma_f16(tmem_o, da, db, idesc_o, (kt | k) != 0);  // O accumulates over the key tiles in TMEM
+          }
+          commit(p_free(kt & 1));  // P V of this tile is complete: its P buffer may be rewritten, O holds tiles 0..kt
+        }
+        commit(kv_empty(kt & 1));
+      }
     }
-    if (lse && tq == 0) lse[(size_t)t * Hq + hq] = lsum[hlf] > 0.f ? (mx[hlf] + log2f(lsum[hlf])) * LN2 : -INFINITY;
+  } else {
+    // ---------------- softmax / epilogue: thread = row
+    const int quarter = warp & 3;
+    const int row = quarter * 32 + lane;
+    const int fr = r0 + row;
+    const bool row_ok = fr < rows_total;
+    const int tok = row_ok ? fr / G : 0;
+    const int hq = g * G + (row_ok ? fr % G : 0);
+    const int lim = row_ok ? min(pos[tok], kv_len - 1) : -1;
+    const uint32_t lane_addr = (uint32_t)(quarter * 32) << 16;
+
+    // Q row -> shared memory, swizzled K-major sub-tiles
+    {
+      const uint4* src = reinterpret_cast<const uint4*>(q + ((size_t)tok * Hq + hq) * D);
+#pragma unroll
+      for (int c = 0; c < D / 8; ++c) {
+        uint4 v = row_ok ? __ldg(src + c) : make_uint4(0, 0, 0, 0);
+        *reinterpret_cast<uint4*>(base_ptr + L::Q_OFF + (c / 8) * L::SUB + swz(row, c % 8)) = v;
+      }
+      fence_async_smem();
+      mbar_arrive(q_ready);
+    }
+
+    // Exponent reference m_ref and row sum l_run relative to it.  The reference is the true maximum of the first
+    // tile and is raised later only when a logit exceeds it by more than 2^RESCALE_TH (rare once the first tiles
+    // are seen): then the output accumulated in TMEM and l_run are rescaled and the tile is redone.  Probabilities
+    // therefore stay below 2^RESCALE_TH, and the output needs no per-tile correction.
+    constexpr float RESCALE_TH = 8.f;
+    float m_ref = 0.f, l_run = 0.f;
+    bool ok = true;
+
+    for (int kt = 0; kt < nkt; ++kt) {
+      // the result of every wait is made warp-uniform: tcgen05.ld/st are warp-wide instructions
+      ok = __all_sync(0xffffffffu, mbar_wait(s_full(kt & 1), (kt >> 1) & 1, abort_flag, status));
+      if (!ok) break;
+      fence_after();
+      const uint32_t ts = tmem_s0 + (kt & 1) * 128 + lane_addr;
+      const int key0 = (kt0 + kt) * ATC_BN;
+      const bool need_mask = key0 + ATC_BN - 1 > minpos;
+      if (kt == 0) {
+        float mx = -INFINITY;
+#pragma unroll 1
+        for (int c = 0; c < 4; ++c) {
+          float sv[32];
+          ld32(ts + c * 32, sv);
+          wait_ld();
+#pragma unroll
+          for (int e = 0; e < 32; ++e) {
+            float x = sv[e] * scale_log2;
+            if (need_mask && key0 + c * 32 + e > lim) x = -INFINITY;
+            mx = fmaxf(mx, x);
+          }
+        }
+        m_ref = mx == -INFINITY ? 0.f : mx;
+      }
+      if (want_o && kt >= 2) {
+        // the P buffer of this tile was last read by the P V of tile kt-2
+        ok = __all_sync(0xffffffffu, mbar_wait(p_free(kt & 1), ((kt >> 1) & 1) ^ 1, abort_flag, status));
+        if (!ok) break;
+      }
+#pragma unroll 1
+      for (int trip = 0; trip < 2; ++trip) {
+        // mx is tracked relative to the reference: the exponent argument itself, fmaf(s, scale, -m_ref)
+        float mx = -INFINITY, ls[4] = {0.f, 0.f, 0.f, 0.f};
+        const float neg_ref = -m_ref;
+        float buf[2][32];
+        ld32(ts, buf[0]);
+#pragma unroll
+        for (int c = 0; c < 4; ++c) {
+          wait_ld();
+          if (c < 3) ld32(ts + (c + 1) * 32, buf[(c + 1) & 1]);
+          float* sv = buf[c & 1];
+          if (need_mask) softmax_chunk<true>(sv, key0 + c * 32, lim, scale_log2, neg_ref, mx, ls);
+          else softmax_chunk<false>(sv, key0 + c * 32, lim, scale_log2, neg_ref, mx, ls);
+          if (want_o) {
+#pragma unroll
+            for (int i = 0; i < 4; ++i)
+              *reinterpret_cast<uint4*>(base_ptr + L::P_OFF + (kt & 1) * L::P_BYTES + (c >> 1) * L::SUB + swz(row, (c & 1) * 4 + i)) = pack8(sv + 8 * i);
+          }
+        }
+        const float lsum = (ls[0] + ls[1]) + (ls[2] + ls[3]);
+        if (!__any_sync(0xffffffffu, mx > RESCALE_TH)) {
+          l_run += lsum;
+          break;
+        }
+        const float raise = fmaxf(mx, 0.f);  // lanes below the threshold may move too: any value >= their maximum is valid
+        const float f = exp2f(-raise);
+        m_ref += raise;
+        l_run *= f;
+        if (want_o && kt > 0) {
+          // the output so far must be complete (P V of the previous tile) before it is rescaled in place
+          // (the threads follow every phase of p_free[b] in order - tile kt-1 waited for tile kt-3 on the same
+          // barrier - so a parity wait cannot mistake an older completion for this one)
+          ok = __all_sync(0xffffffffu, mbar_wait(p_free((kt - 1) & 1), ((kt - 1) >> 1) & 1, abort_flag, status));
+          if (!ok) break;
+          fence_after();
+#pragma unroll 1
+          for (int c = 0; c < D / 32; ++c) {
+            float t[32];
+            ld32(tmem_o + lane_addr + c * 32, t);
+            wait_ld();
+#pragma unroll
+            for (int e = 0; e < 32; ++e) t[e] *= f;
+            st32(tmem_o + lane_addr + c * 32, t);
+          }
+          wait_st();
+        }
+      }
+      if (!ok) break;
+      if (want_o && kt0 + kt == nkt_all - 1) {
+        // slots beyond the CTA's last visible key may hold anything: they get probability zero, and zero times a
+        // non-finite value would still poison the product, so clear those V rows of the last tile
+        const int first_bad = maxpos - key0 + 1;
+        const bool landed = mbar_wait(kv_full(kt & 1), (kt >> 1) & 1, abort_flag, status);  // already complete: S of this tile was computed
+        if (landed && row >= first_bad) {
+          unsigned char* sv = base_ptr + L::KV_OFF + (kt & 1) * L::KV_STAGE + (D / 64) * L::SUB;
+#pragma unroll
+          for (int j = 0; j < D / 64; ++j)
+#pragma unroll
+            for (int c = 0; c < 8; ++c) *reinterpret_cast<uint4*>(sv + j * L::SUB + row * 128 + c * 16) = make_uint4(0, 0, 0, 0);
+        }
+      }
+      fence_async_smem();
+      fence_before();
+      mbar_arrive(p_ready(kt & 1));
+    }
+    const float inv = l_run > 0.f ? 1.f / l_run : 0.f;
+    const size_t prow = ((size_t)blockIdx.z * Hkv + g) * ((size_t)gridDim.x * ATC_BM) + fr;  // partial-result row
+    if (ok && want_o && nkt > 0) {
+      ok = __all_sync(0xffffffffu, mbar_wait(p_free((nkt - 1) & 1), ((nkt - 1) >> 1) & 1, abort_flag, status));
+      if (ok) {
+        fence_after();
+        bf16* dst = o + ((size_t)tok * Hq + hq) * D;
+#pragma unroll 1
+        for (int c = 0; c < D / 32; ++c) {
+          float t[32];
+          ld32(tmem_o + lane_addr + c * 32, t);
+          wait_ld();
+          if (row_ok && partial) {
+            float4* pd = reinterpret_cast<float4*>(part_o + prow * D + c * 32);
+#pragma unroll
+            for (int i = 0; i < 8; ++i) pd[i] = make_float4(t[4 * i], t[4 * i + 1], t[4 * i + 2], t[4 * i + 3]);
+          } else if (row_ok) {
+#pragma unroll
+            for (int e = 0; e < 32; ++e) t[e] *= inv;
+#pragma unroll
+            for (int i = 0; i < 4; ++i) reinterpret_cast<uint4*>(dst + c * 32)[i] = pack8(t + 8 * i);
+          }
+          __syncwarp();
+        }
+      }
+    }
+    if (ok && row_ok && partial) part_ml[prow] = make_float2(m_ref, l_run);
+    if (ok && row_ok && !partial && lse) lse[(size_t)tok * Hq + hq] = l_run > 0.f ? (m_ref + log2f(l_run)) * ATC_LN2 : -INFINITY;
   }
+  atc::fence_before();
+  __syncthreads();
+  if (warp == 1) asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(512) : "memory");
 }
 
-int attention_rows_tc(const a3_handle* h, const bf16* q, const int32_t* pos, int M, const bf16* k, const bf16* v,
-                      int kv_len, bf16* o, float* lse, void* part, size_t part_bytes, cudaStream_t st);
-// 0: tcgen05 kernel (a3_attention_tc.cu); 1: the warp-level mma.sync kernel in this file (cross-check for bring-up)
-int g_attn_impl = 0;
-
-int attention_rows(const a3_handle* h, const bf16* q, const int32_t* pos, int M, const bf16* k, const bf16* v,
-                   int kv_len, bf16* o, float* lse, void* part, size_t part_bytes, cudaStream_t st) {
-  if (M <= 0) return A3_OK;
-  if (g_attn_impl == 0) return attention_rows_tc(h, q, pos, M, k, v, kv_len, o, lse, part, part_bytes, st);
-  const int Hq = h->m.n_q_heads, Hkv = h->m.n_kv_heads, D = h->m.head_dim;
+// One warp per (flat row, KV head) of a row tile that was split over the keys: merges the segments' partial results
+// in segment order (fixed, so the result is reproducible): O = sum_z O_z 2^(m_z - m) / sum_z l_z 2^(m_z - m).
+template <int D>
+__global__ void __launch_bounds__(128)
+attention_combine_kernel(const int32_t* __restrict__ pos, int M, int kv_len, int Hq, int Hkv, int tiles_per_split, int rows_pad,
+                         const float* __restrict__ part_o, const float2* __restrict__ part_ml, bf16* __restrict__ o,
+                         float* __restrict__ lse) {
   const int G = Hq / Hkv;
-  dim3 grid(cdiv((long long)M * G, AT_BM), Hkv);
-  const float scale_log2 = LOG2E / sqrtf((float)D);
-  const int smem = 5 * 64 * D * 2;
-  static bool attr_set = false;
-  if (!attr_set) {
-    A3_CUDA(cudaFuncSetAttribute(attention_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, 5 * 64 * 128 * 2));
-    A3_CUDA(cudaFuncSetAttribute(attention_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, 5 * 64 * 64 * 2));
-    attr_set = true;
+  const int rows_total = M * G;
+  const int fr = blockIdx.x * 4 + (threadIdx.x >> 5);
+  const int g = blockIdx.y, lane = threadIdx.x & 31;
+  if (fr >= rows_total) return;
+  const int r0 = (fr / ATC_BM) * ATC_BM;
+  const int last_tok = min(M - 1, (r0 + ATC_BM - 1) / G);
+  const int maxpos = min(pos[last_tok], kv_len - 1);
+  const int nkt_all = maxpos < 0 ? 0 : maxpos / ATC_BN + 1;
+  const int n_active = (nkt_all + tiles_per_split - 1) / tiles_per_split;
+  if (n_active <= 1) return;  // written directly by the attention kernel
+  float m = -INFINITY;
+  for (int z = 0; z < n_active; ++z) {
+    const float2 ml = part_ml[((size_t)z * Hkv + g) * rows_pad + fr];
+    if (ml.y > 0.f) m = fmaxf(m, ml.x);
   }
-  ProfScope prof(h, A3_K_ATTENTION, st);
-  if (D == 128) attention_kernel<128><<<grid, AT_THREADS, smem, st>>>(q, pos, M, k, v, kv_len, o, lse, Hq, Hkv, scale_log2);
-  else attention_kernel<64><<<grid, AT_THREADS, smem, st>>>(q, pos, M, k, v, kv_len, o, lse, Hq, Hkv, scale_log2);
-  A3_LAUNCHED();
+  constexpr int PER = D / 32;
+  float acc[PER];
+#pragma unroll
+  for (int e = 0; e < PER; ++e) acc[e] = 0.f;
+  float l = 0.f;
+  for (int z = 0; z < n_active; ++z) {
+    const size_t prow = ((size_t)z * Hkv + g) * rows_pad + fr;
+    const float2 ml = part_ml[prow];
+    if (!(ml.y > 0.f)) continue;
+    const float w = exp2f(ml.x - m);
+    l += ml.y * w;
+    const float* src = part_o + prow * D + lane * PER;
+#pragma unroll
+    for (int e = 0; e < PER; ++e) acc[e] += src[e] * w;
+  }
+  const int tok = fr / G, hq = g * G + fr % G;
+  const float inv = l > 0.f ? 1.f / l : 0.f;
+  bf16* dst = o + ((size_t)tok * Hq + hq) * D + lane * PER;
+#pragma unroll
+  for (int e = 0; e < PER; e += 2) *reinterpret_cast<uint32_t*>(dst + e) = pack2(acc[e] * inv, acc[e + 1] * inv);
+  if (lse && lane == 0) lse[(size_t)tok * Hq + hq] = l > 0.f ? (m + log2f(l)) * ATC_LN2 : -INFINITY;
+}
+
+// ---------------------------------------------------------------- host side
+typedef CUresult (*EncodeTiledFn2)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                                   const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                   CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+static int make_cache_tmap(CUtensorMap* map, const void* ptr, long long rows, long long cols) {
+  static EncodeTiledFn2 fn = nullptr;
+  if (!fn) {
+    void* p = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &qres) != cudaSuccess || qres != cudaDriverEntryPointSuccess)
+      return A3_ECUDA;
+    fn = (EncodeTiledFn2)p;
+  }
+  cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
+  cuuint64_t strides[1] = {(cuuint64_t)cols * 2};
+  cuuint32_t box[2] = {64, (cuuint32_t)ATC_BN};
+  cuuint32_t estr[2] = {1, 1};
+  CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(ptr), dims, strides, box, estr,
+                  CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                  CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  if (r != CUDA_SUCCESS) {
+    g_last_cuda_error = (int)r;
+    return A3_ECUDA;
+  }
   return A3_OK;
 }
 
-// ------------------------------------------------------------------ relevance scores (Eq. 3)
-// One CTA per tile of 64 cache slots.  It loops over the KV heads and, per head, over blocks of 64 packed
-// question rows; column sums stay on chip and are added in a fixed order.
-template <int D>
-__global__ void __launch_bounds__(AT_THREADS)
-scores_kernel(const bf16* __restrict__ q, const int32_t* __restrict__ q_pos, int nq, const bf16* __restrict__ k,
-              int kv_len, int cand_begin, int cand_end, const float* __restrict__ lse, float* __restrict__ scores,
-              int Hq, int Hkv, float scale_log2) {
-  __shared__ __align__(128) unsigned char smem[2 * 64 * D * 2];
-  __shared__ float colpart[4][AT_BN];
-  const uint32_t sq = smem_u32(smem), sk = sq + 64 * D * 2;
-  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  const int gq = lane >> 2, tq = lane & 3;
-  const int G = Hq / Hkv;
-  const int key0 = blockIdx.x * AT_BN;
-  const int rows_total = nq * G;
-  const int nrb = (rows_total + AT_BM - 1) / AT_BM;
-  const int kvrow = Hkv * D;
-  float total = 0.f;  // thread c < 64 owns cache slot key0 + c
+int g_attn_split = 0;  // 0: choose; otherwise the number of key segments (tuning)
 
-  for (int g = 0; g < Hkv; ++g) {
-    __syncthreads();  // previous users of sk / sq are done
-    load_tile<D>(sk, k, [&](int r) -> const bf16* {
-      int key = key0 + r;
-      return key < kv_len ? k + (size_t)key * kvrow + g * D : nullptr;
-    });
-    for (int rb = 0; rb < nrb; ++rb) {
-      const int r0 = rb * AT_BM;
-      if (rb > 0) __syncthreads();
-      load_tile<D>(sq, q, [&](int r) -> const bf16* {
-        int fr = r0 + r;
-        if (fr >= rows_total) return nullptr;
-        return q + ((size_t)(fr / G) * Hq + g * G + fr % G) * D;
-      });
-      cp_async_commit();
-      cp_async_wait<0>();
-      __syncthreads();
-      uint32_t qf[D / 16][4];
-      load_q_frags<D>(sq, warp, lane, qf);
-      float s[8][4];
-      qk_tile<D>(sk, lane, qf, s);
-      int lim[2];
-      float l2[2];
-#pragma unroll
-      for (int hlf = 0; hlf < 2; ++hlf) {
-        int fr = r0 + warp * 16 + gq + hlf * 8;
-        if (fr < rows_total) {
-          int t = fr / G, hq = g * G + fr % G;
-          lim[hlf] = min(q_pos[t], kv_len - 1);
-          l2[hlf] = lse[(size_t)t * Hq + hq] * LOG2E;
-        } else {
-          lim[hlf] = -1;
-          l2[hlf] = 0.f;
-        }
-      }
-#pragma unroll
-      for (int j = 0; j < 8; ++j) {
-        float c0 = 0.f, c1 = 0.f;  // columns j*8 + 2*tq, +1: rows gq and gq+8
-#pragma unroll
-        for (int hlf = 0; hlf < 2; ++hlf) {
-          int key = key0 + j * 8 + 2 * tq;
-          float p0 = key <= lim[hlf] ? exp2f(s[j][2 * hlf] * scale_log2 - l2[hlf]) : 0.f;
-          float p1 = key + 1 <= lim[hlf] ? exp2f(s[j][2 * hlf + 1] * scale_log2 - l2[hlf]) : 0.f;
-          c0 += p0;
-          c1 += p1;
-        }
-#pragma unroll
-        for (int off = 4; off < 32; off <<= 1) {
-          c0 += __shfl_xor_sync(0xffffffffu, c0, off);
-          c1 += __shfl_xor_sync(0xffffffffu, c1, off);
-        }
-        if (gq == 0) {
-          colpart[warp][j * 8 + 2 * tq] = c0;
-          colpart[warp][j * 8 + 2 * tq + 1] = c1;
-        }
-      }
-      __syncthreads();
-      if (tid < AT_BN) total += (colpart[0][tid] + colpart[1][tid]) + (colpart[2][tid] + colpart[3][tid]);
-    }
-  }
-  if (tid < AT_BN) {
-    int key = key0 + tid;
-    if (key < kv_len) scores[key] = (key >= cand_begin && key < cand_end) ? total : 0.f;
-  }
+size_t attention_part_bytes(const a3_handle* h) {
+  // split only happens when the unsplit grid has fewer than two CTAs per SM; up to 4 segments
+  const size_t rows = (size_t)2 * (h->sm_count > 0 ? h->sm_count : 148) * ATC_BM;
+  return 4 * rows * ((size_t)h->m.head_dim + 2) * sizeof(float);
 }
 
-int scores_pass(const a3_handle* h, const bf16* q, const int32_t* q_pos, int nq, const bf16* k, int kv_len,
-                int cand_begin, int cand_end, const float* lse, float* scores, cudaStream_t st) {
-  if (kv_len <= 0) return A3_OK;
+int attention_rows(const a3_handle* h, const bf16* q, const int32_t* pos, int M, const bf16* k, const bf16* v,
+                      int kv_len, bf16* o, float* lse, void* part, size_t part_bytes, cudaStream_t st) {
+  if (M <= 0) return A3_OK;
   const int Hq = h->m.n_q_heads, Hkv = h->m.n_kv_heads, D = h->m.head_dim;
-  const float scale_log2 = LOG2E / sqrtf((float)D);
-  dim3 grid(cdiv(kv_len, AT_BN));
-  ProfScope prof(h, A3_K_SCORES, st);
-  if (D == 128) scores_kernel<128><<<grid, AT_THREADS, 0, st>>>(q, q_pos, nq, k, kv_len, cand_begin, cand_end, lse, scores, Hq, Hkv, scale_log2);
-  else scores_kernel<64><<<grid, AT_THREADS, 0, st>>>(q, q_pos, nq, k, kv_len, cand_begin, cand_end, lse, scores, Hq, Hkv, scale_log2);
+  const int G = Hq / Hkv;
+  CUtensorMap tK, tV;
+  A3_TRY(make_cache_tmap(&tK, k, kv_len, (long long)Hkv * D));
+  A3_TRY(make_cache_tmap(&tV, v, kv_len, (long long)Hkv * D));
+  dim3 grid(cdiv((long long)M * G, ATC_BM), Hkv);
+  const float scale_log2 = ATC_LOG2E / sqrtf((float)D);
+  // split over the keys when the grid would leave SMs idle behind a few long row tiles
+  const int sms = h->sm_count > 0 ? h->sm_count : 148;
+  const int base_ctas = (int)grid.x * Hkv, all_tiles = cdiv(kv_len, ATC_BN);
+  int n_split = 1;
+  if (o && part && base_ctas < 2 * sms && all_tiles >= 8) {
+    n_split = g_attn_split > 0 ? g_attn_split : 2;  // measured: 2 segments beat 1, 3 and 4 at 208 base CTAs (7-8 us fixed cost per CTA)
+    const size_t need = (size_t)n_split * base_ctas * ATC_BM * ((size_t)D + 2) * sizeof(float);
+    if (need > part_bytes) n_split = 1;
+  }
+  const int tiles_per_split = cdiv(all_tiles, n_split);
+  n_split = cdiv(all_tiles, tiles_per_split);
+  grid.z = n_split;
+  const int rows_pad = (int)grid.x * ATC_BM;
+  float* part_o = (float*)part;
+  float2* part_ml = part ? (float2*)(part_o + (size_t)n_split * Hkv * rows_pad * D) : nullptr;
+  static bool attr_set = false;
+  if (!attr_set) {
+    A3_CUDA(cudaFuncSetAttribute(attention_tc_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, AtcLayout<128>::SMEM_BYTES));
+    A3_CUDA(cudaFuncSetAttribute(attention_tc_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, AtcLayout<64>::SMEM_BYTES));
+    attr_set = true;
+  }
+  ProfScope prof(h, A3_K_ATTENTION, st);
+  if (D == 128)
+    attention_tc_kernel<128><<<grid, ATC_THREADS, AtcLayout<128>::SMEM_BYTES, st>>>(tK, tV, q, pos, M, kv_len, o, lse, Hq, Hkv, scale_log2, h->dev_status, tiles_per_split, part_o, part_ml);
+  else
+    attention_tc_kernel<64><<<grid, ATC_THREADS, AtcLayout<64>::SMEM_BYTES, st>>>(tK, tV, q, pos, M, kv_len, o, lse, Hq, Hkv, scale_log2, h->dev_status, tiles_per_split, part_o, part_ml);
   A3_LAUNCHED();
+  if (n_split > 1) {
+    dim3 cgrid(cdiv((long long)M * G, 4), Hkv);
+    if (D == 128) attention_combine_kernel<128><<<cgrid, 128, 0, st>>>(pos, M, kv_len, Hq, Hkv, tiles_per_split, rows_pad, part_o, part_ml, o, lse);
+    else attention_combine_kernel<64><<<cgrid, 128, 0, st>>>(pos, M, kv_len, Hq, Hkv, tiles_per_split, rows_pad, part_o, part_ml, o, lse);
+    A3_LAUNCHED();
+  }
   return A3_OK;
 }
 
 }  // namespace a3
 
-extern "C" void a3_internal_set_attn_impl(int impl) { a3::g_attn_impl = impl; }
+extern "C" void a3_internal_set_attn_split(int v) { a3::g_attn_split = v; }

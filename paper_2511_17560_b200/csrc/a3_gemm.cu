@@ -1,27 +1,31 @@
-// Projection / MLP GEMMs of the recompute path (Eq. 5: Q_l = X_l W^q, K <- X_l W^k, V <- X_l W^v; H(.)):
-//   C[M][N] = A[M][K] * B[N][K]^T, bf16 operands (both K-major), fp32 accumulation, fused epilogues:
+// Projection / MLP GEMMs of the recompute path (Eq. 5: Q_l = X_l W^q, K <- X_l W^k, V <- X_l W^v; H(.)) on the
+// 5th-generation tensor cores:  C[M][N] = A[M][K] * B[N][K]^T, bf16 operands (both K-major), fp32 accumulators in
+// tensor memory, fused epilogues:
 //   EPI_RESIDUAL  C <- C + A B^T                       (output projection and MLP down projection)
-//   EPI_SWIGLU    C <- silu(A Bg^T) * (A Bu^T)         (gate and up in one pass, 64 + 64 columns per tile)
+//   EPI_SWIGLU    C <- silu(A Bg^T) * (A Bu^T)         (gate and up rows interleaved per tile: BN/2 + BN/2 columns)
 //   EPI_QKV       +bias, RoPE of q/k at pos[m], q -> q_out, k/v -> cache rows pos[m] (the scatter of Eq. 5)
-// This translation unit is the mma.sync (warp-level tensor core) implementation: 128x128x64 tiles,
-// 3-stage cp.async pipeline, ldmatrix from 128-byte-swizzled shared memory.
+//
+// One CTA computes one 128 x BN tile.  Warp 0 (one lane) feeds a ring of shared-memory stages with TMA
+// (cp.async.bulk.tensor, 128-byte swizzle); warp 1 (one lane) issues tcgen05.mma (128 x BN x 16) on the stages and
+// commits them back to the producer through mbarriers; warps 2..5 read the accumulator with tcgen05.ld (each thread
+// owns one output row) and run the epilogue straight out of registers.  No cluster multicast is used.
+// Every barrier wait is bounded: after half a second a waiter raises the CTA's abort flag and the device status bit
+// A3_DEV_WAIT_EXHAUSTED, all roles leave their loops, in-flight copies are given time to land, tensor memory is
+// released and the CTA returns.
+#include <cuda.h>
+
 #include "a3_internal.cuh"
 
 namespace a3 {
 
-constexpr int BM = 128, BN = 128, BK = 64, STAGES = 3, GEMM_THREADS = 256;
-constexpr int STAGE_BYTES = (BM + BN) * BK * 2;        // 32 KiB
-constexpr int CT_LD = BN + 4;                          // fp32 staging tile leading dimension
-constexpr int GEMM_SMEM = STAGES * STAGE_BYTES;        // 96 KiB >= 128*132*4 = 66 KiB staging
+constexpr int TC_BM = 128, TC_BK = 64, TC_THREADS = 192;
+constexpr unsigned long long TC_WAIT_NS = 500000000ull;
 
-struct GemmDev {
-  const bf16* A;
-  int M, K;
-  const bf16* B[3];
-  const bf16* bias[3];
-  int seg_tiles_end[3];  // exclusive tile index where each segment ends (tiles of 128 columns)
+struct TcParams {
+  int M, K, N;
+  int seg_tiles_end[3];
   int kind[3];
-  const bf16* B2;
+  const bf16* bias[3];
   bf16* C;
   int ldc;
   bf16* q_out;
@@ -34,19 +38,133 @@ struct GemmDev {
   uint32_t* status;
 };
 
-// byte offset of 16-byte chunk `c` of row `r` in a [rows][64] bf16 tile with the 128-byte XOR swizzle
-__device__ __forceinline__ uint32_t swz(int r, int c) { return (uint32_t)(r * 128 + ((c ^ (r & 7)) << 4)); }
+// ---------------------------------------------------------------- PTX wrappers
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ uint32_t mbar_try_wait(uint32_t bar, uint32_t parity) {
+  uint32_t done;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.b32 %0, 1, 0, p;\n\t}"
+      : "=r"(done)
+      : "r"(bar), "r"(parity)
+      : "memory");
+  return done;
+}
+__device__ __forceinline__ unsigned long long global_ns() {
+  unsigned long long t;
+  asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
+  return t;
+}
+// Bounded wait.  Returns false when the wait was abandoned (own time-out or another role's abort).
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, uint32_t* status,
+                                          unsigned long long limit_ns = TC_WAIT_NS) {
+  if (mbar_try_wait(bar, parity)) return true;
+  const unsigned long long t0 = global_ns();
+  for (;;) {
+#pragma unroll 1
+    for (int i = 0; i < 32; ++i)
+      if (mbar_try_wait(bar, parity)) return true;
+    if (*abort_flag) return false;
+    if (global_ns() - t0 > limit_ns) {
+      *abort_flag = 1;
+      atomicOr(status, A3_DEV_WAIT_EXHAUSTED);
+      return false;
+    }
+  }
+}
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int x, int y, uint32_t bar) {
+  asm volatile("cp.async.bulk.tensor.2d.shared::cta.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+               ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(bar)
+               : "memory");
+}
+__device__ __forceinline__ void tmap_prefetch(const CUtensorMap* map) {
+  asm volatile("prefetch.tensormap [%0];" ::"l"(map) : "memory");
+}
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_commit(uint32_t bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void tc_mma_f16(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+      ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+// 32 lanes x 32 consecutive fp32 columns: thread i of the warp receives row (lane base + i)
+__device__ __forceinline__ void tc_ld32(uint32_t taddr, float* v) {
+  uint32_t* r = reinterpret_cast<uint32_t*>(v);
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+        "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]),
+        "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]),
+        "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+      : "r"(taddr)
+      : "memory");
+}
+__device__ __forceinline__ void tc_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 
-template <int EPI>
-__global__ void __launch_bounds__(GEMM_THREADS)
-gemm_mma_kernel(const GemmDev p) {
-  extern __shared__ __align__(128) unsigned char smem[];
-  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  const int wm = warp >> 2, wn = warp & 3;  // 2 x 4 warps, warp tile 64 x 32
-  const int m0 = blockIdx.x * BM;
+// Shared-memory matrix descriptor of a K-major [rows][64] bf16 tile written by TMA with the 128-byte swizzle:
+// rows are 128 bytes apart, groups of 8 rows (1024 bytes) follow one another, the tile base is 1024-byte aligned.
+__device__ __forceinline__ uint64_t smem_desc_sw128(uint32_t saddr) {
+  return (uint64_t)((saddr & 0x3FFFFu) >> 4) | ((uint64_t)(1024u >> 4) << 32) | (1ull << 46) | (2ull << 61);
+}
+// bf16 x bf16 -> fp32, both operands K-major, M = 128
+__host__ __device__ constexpr uint32_t idesc_bf16(int n) {
+  return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(TC_BM >> 4) << 24);
+}
+
+__device__ __forceinline__ void store32_bf16(bf16* dst, const float* f) {
+  uint4* d = reinterpret_cast<uint4*>(dst);
+#pragma unroll
+  for (int i = 0; i < 4; ++i) d[i] = pack8(f + 8 * i);
+}
+__device__ __forceinline__ void load32_bf16(const bf16* src, float* f) {
+  const uint4* s = reinterpret_cast<const uint4*>(src);
+#pragma unroll
+  for (int i = 0; i < 4; ++i) unpack8(s[i], f + 8 * i);
+}
+
+template <int BN, int STAGES>
+struct TcLayout {
+  static constexpr int A_BYTES = TC_BM * TC_BK * 2;
+  static constexpr int B_BYTES = BN * TC_BK * 2;
+  static constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
+  static constexpr int BAR_OFFSET = STAGES * STAGE_BYTES;
+  static constexpr int SMEM_BYTES = BAR_OFFSET + 256 + 1024;  // barriers + slack for the 1024-byte alignment
+};
+
+template <int EPI, int BN, int STAGES>
+__global__ void __launch_bounds__(TC_THREADS)
+gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB0,
+               const __grid_constant__ CUtensorMap tmB1, const __grid_constant__ CUtensorMap tmB2, const TcParams p) {
+  using L = TcLayout<BN, STAGES>;
+  constexpr int TMEM_COLS = BN <= 128 ? 128 : 256;  // allocations are powers of two
+  extern __shared__ unsigned char smem_raw[];
+  const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+  unsigned char* base_ptr = smem_raw + (base - smem_u32(smem_raw));
+  const uint32_t bars = base + L::BAR_OFFSET;  // full[S], empty[S], tmem_full: 8 bytes each
+  volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(base_ptr + L::BAR_OFFSET + 8 * (2 * STAGES + 1));
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(base_ptr + L::BAR_OFFSET + 8 * (2 * STAGES + 1) + 8);
+  auto full_bar = [&](int s) { return bars + 8u * s; };
+  auto empty_bar = [&](int s) { return bars + 8u * (STAGES + s); };
+  const uint32_t tmem_full_bar = bars + 8u * (2 * STAGES);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int m0 = blockIdx.x * TC_BM;
   const int nt = blockIdx.y;
+  const int KT = p.K / TC_BK;
 
-  // which B rows feed this tile
   int seg = 0, seg_tile0 = 0;
   if (EPI == EPI_QKV) {
     while (seg < 2 && nt >= p.seg_tiles_end[seg]) {
@@ -54,215 +172,312 @@ gemm_mma_kernel(const GemmDev p) {
       ++seg;
     }
   }
-  const bf16* Bbase = p.B[seg];
-  const int nb0 = (EPI == EPI_SWIGLU) ? nt * 64 : (nt - seg_tile0) * BN;  // first B row (column of the segment)
+  // first B row of this tile within its matrix (for SwiGLU: within gate and within up)
+  const int nb0 = (EPI == EPI_SWIGLU) ? nt * (BN / 2) : (nt - seg_tile0) * BN;
 
-  const uint32_t smem_base = smem_u32(smem);
-  const int KT = p.K / BK;
-
-  auto load_stage = [&](int stage, int kt) {
-    const uint32_t sa = smem_base + stage * STAGE_BYTES;
-    const uint32_t sb = sa + BM * BK * 2;
-    const int k0 = kt * BK;
-#pragma unroll
-    for (int i = 0; i < (BM * 8) / GEMM_THREADS; ++i) {
-      int idx = tid + i * GEMM_THREADS;
-      int r = idx >> 3, c = idx & 7;
-      int gr = m0 + r;
-      bool ok = gr < p.M;
-      const bf16* src = p.A + (size_t)(ok ? gr : 0) * p.K + k0 + c * 8;
-      cp_async16(sa + swz(r, c), src, ok);
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < STAGES; ++s) {
+      mbar_init(full_bar(s), 1);
+      mbar_init(empty_bar(s), 1);
     }
-#pragma unroll
-    for (int i = 0; i < (BN * 8) / GEMM_THREADS; ++i) {
-      int idx = tid + i * GEMM_THREADS;
-      int r = idx >> 3, c = idx & 7;
-      const bf16* src;
-      if (EPI == EPI_SWIGLU)
-        src = (r < 64 ? Bbase + (size_t)(nb0 + r) * p.K : p.B2 + (size_t)(nb0 + r - 64) * p.K) + k0 + c * 8;
-      else
-        src = Bbase + (size_t)(nb0 + r) * p.K + k0 + c * 8;
-      cp_async16(sb + swz(r, c), src, true);
-    }
-  };
-
-  float acc[4][4][4];
-#pragma unroll
-  for (int i = 0; i < 4; ++i)
-#pragma unroll
-    for (int j = 0; j < 4; ++j)
-#pragma unroll
-      for (int e = 0; e < 4; ++e) acc[i][j][e] = 0.f;
-
-  for (int s = 0; s < STAGES - 1; ++s) {
-    if (s < KT) load_stage(s, s);
-    cp_async_commit();
+    mbar_init(tmem_full_bar, 1);
+    abort_flag[0] = 0;
+    abort_flag[1] = 0;  // never raised: lets the drain below wait on its own clock only
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
   }
-
-  for (int kt = 0; kt < KT; ++kt) {
-    cp_async_wait<STAGES - 2>();
-    __syncthreads();
-    {
-      int nk = kt + STAGES - 1;
-      if (nk < KT) load_stage(nk % STAGES, nk);
-      cp_async_commit();
-    }
-    const uint32_t sa = smem_base + (kt % STAGES) * STAGE_BYTES;
-    const uint32_t sb = sa + BM * BK * 2;
-#pragma unroll
-    for (int ks = 0; ks < BK / 16; ++ks) {
-      uint32_t af[4][4], bfr[4][2];
-#pragma unroll
-      for (int i = 0; i < 4; ++i) {
-        int r = wm * 64 + i * 16 + (lane & 7) + ((lane >> 3) & 1) * 8;
-        int c = ks * 2 + (lane >> 4);
-        ldmatrix_x4(sa + swz(r, c), af[i][0], af[i][1], af[i][2], af[i][3]);
-      }
-#pragma unroll
-      for (int j = 0; j < 2; ++j) {
-        int r = wn * 32 + j * 16 + (lane & 7) + (lane >> 4) * 8;
-        int c = ks * 2 + ((lane >> 3) & 1);
-        ldmatrix_x4(sb + swz(r, c), bfr[2 * j][0], bfr[2 * j][1], bfr[2 * j + 1][0], bfr[2 * j + 1][1]);
-      }
-#pragma unroll
-      for (int i = 0; i < 4; ++i)
-#pragma unroll
-        for (int j = 0; j < 4; ++j) mma_bf16(acc[i][j], af[i], bfr[j][0], bfr[j][1]);
-    }
+  if (warp == 1) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32((const void*)tmem_slot)), "r"(TMEM_COLS) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
   }
-  cp_async_wait<0>();
+  tc_fence_before();
   __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
 
-  // ---- stage the fp32 tile in shared memory
-  float* ct = reinterpret_cast<float*>(smem);
-  {
-    const int g = lane >> 2, t = lane & 3;
-#pragma unroll
-    for (int i = 0; i < 4; ++i)
-#pragma unroll
-      for (int j = 0; j < 4; ++j) {
-        int r = wm * 64 + i * 16 + g, c = wn * 32 + j * 8 + 2 * t;
-        *reinterpret_cast<float2*>(&ct[r * CT_LD + c]) = make_float2(acc[i][j][0], acc[i][j][1]);
-        *reinterpret_cast<float2*>(&ct[(r + 8) * CT_LD + c]) = make_float2(acc[i][j][2], acc[i][j][3]);
+  if (warp == 0) {
+    // ---------------- TMA producer
+    if (lane == 0) {
+      const CUtensorMap* mapB = seg == 0 ? &tmB0 : (seg == 1 ? &tmB1 : &tmB2);
+      tmap_prefetch(&tmA);
+      tmap_prefetch(mapB);
+      if (EPI == EPI_SWIGLU) tmap_prefetch(&tmB1);
+      int issued = 0;
+      for (int kb = 0; kb < KT; ++kb) {
+        const int s = kb % STAGES;
+        const uint32_t ph = (kb / STAGES) & 1;
+        if (!mbar_wait(empty_bar(s), ph ^ 1, abort_flag, p.status)) break;
+        const uint32_t sa = base + s * L::STAGE_BYTES, sb = sa + L::A_BYTES;
+        mbar_expect_tx(full_bar(s), L::STAGE_BYTES);
+        tma_load_2d(sa, &tmA, kb * TC_BK, m0, full_bar(s));
+        if (EPI == EPI_SWIGLU) {
+          tma_load_2d(sb, &tmB0, kb * TC_BK, nb0, full_bar(s));
+          tma_load_2d(sb + L::B_BYTES / 2, &tmB1, kb * TC_BK, nb0, full_bar(s));
+        } else {
+          tma_load_2d(sb, mapB, kb * TC_BK, nb0, full_bar(s));
+        }
+        issued = kb + 1;
       }
-  }
-  __syncthreads();
-
-  if (EPI == EPI_RESIDUAL) {
-    const int n0 = nt * BN;
-    for (int idx = tid; idx < BM * 16; idx += GEMM_THREADS) {
-      int r = idx >> 4, v = idx & 15;
-      int gr = m0 + r;
-      if (gr >= p.M) continue;
-      uint4* cp = reinterpret_cast<uint4*>(p.C + (size_t)gr * p.ldc + n0 + v * 8);
-      float f[8];
-      unpack8(*cp, f);
-#pragma unroll
-      for (int e = 0; e < 8; ++e) f[e] += ct[r * CT_LD + v * 8 + e];
-      *cp = pack8(f);
+      if (*abort_flag) {
+        // let the copies already issued land before the CTA can exit (bounded)
+        for (int kb = max(0, issued - STAGES); kb < issued; ++kb)
+          mbar_wait(full_bar(kb % STAGES), (kb / STAGES) & 1, abort_flag + 1, p.status, 2000000ull);
+      }
     }
-  } else if (EPI == EPI_SWIGLU) {
-    const int n0 = nt * 64;
-    for (int idx = tid; idx < BM * 8; idx += GEMM_THREADS) {
-      int r = idx >> 3, v = idx & 7;
-      int gr = m0 + r;
-      if (gr >= p.M) continue;
-      float f[8];
+  } else if (warp == 1) {
+    // ---------------- MMA issuer
+    if (lane == 0) {
+      constexpr uint32_t idesc = idesc_bf16(BN);
+      bool ok = true;
+      for (int kb = 0; kb < KT && ok; ++kb) {
+        const int s = kb % STAGES;
+        const uint32_t ph = (kb / STAGES) & 1;
+        ok = mbar_wait(full_bar(s), ph, abort_flag, p.status);
+        if (!ok) break;
+        tc_fence_after();
+        const uint32_t sa = base + s * L::STAGE_BYTES, sb = sa + L::A_BYTES;
+        const uint64_t da = smem_desc_sw128(sa), db = smem_desc_sw128(sb);
 #pragma unroll
-      for (int e = 0; e < 8; ++e) {
-        float gte = ct[r * CT_LD + v * 8 + e], up = ct[r * CT_LD + 64 + v * 8 + e];
-        f[e] = gte / (1.f + __expf(-gte)) * up;
+        for (int k = 0; k < TC_BK / 16; ++k)  // +32 bytes per 16-element K step inside the 128-byte swizzle row
+          tc_mma_f16(tmem_base, da + (uint64_t)(2 * k), db + (uint64_t)(2 * k), idesc, (kb | k) != 0);
+        tc_commit(empty_bar(s));  // arrives once the MMAs above have finished reading this stage
       }
-      *reinterpret_cast<uint4*>(p.C + (size_t)gr * p.ldc + n0 + v * 8) = pack8(f);
+      if (ok) tc_commit(tmem_full_bar);
     }
   } else {
-    const int kind = p.kind[seg];
-    const int D = p.D, half = D / 2;
-    const bf16* bias = p.bias[seg];
-    for (int idx = tid; idx < BM * 8; idx += GEMM_THREADS) {
-      int r = idx >> 3, j = idx & 7;
-      int gr = m0 + r;
-      if (gr >= p.M) continue;
-      const int ps = p.pos[gr];
-      if (ps < 0 || ps >= p.kv_len || ps >= p.max_pos) {
-        if (j == 0) atomicOr(p.status, A3_DEV_BAD_POSITION);
-        continue;
-      }
-      const int upd = D / 16;                          // units per head
-      const int lo = (j / upd) * D + (j % upd) * 8;    // tile column of the low vector
-      const int hi = lo + half;
-      float a[8], b[8];
+    // ---------------- epilogue: warps 2..5, warp w may touch TMEM lanes 32*(w%4) .. +31
+    const int quarter = warp & 3;
+    const int row = quarter * 32 + lane;
+    const int gr = m0 + row;
+    const bool row_ok = gr < p.M;
+    const uint32_t trow = tmem_base + ((uint32_t)(quarter * 32) << 16);
+    const bool ready = mbar_wait(tmem_full_bar, 0, abort_flag, p.status);
+    tc_fence_after();
+    if (ready) {
+      if (EPI == EPI_RESIDUAL) {
+        const int n0 = nt * BN;
+#pragma unroll 1
+        for (int c = 0; c < BN / 32; ++c) {
+          __syncwarp();
+          float acc[32], old[32];
+          tc_ld32(trow + c * 32, acc);
+          const bool col_ok = row_ok && n0 + c * 32 < p.N;  // tiles need not divide N: TMA zero-fills, stores are cut
+          bf16* cp = p.C + (size_t)(row_ok ? gr : 0) * p.ldc + (col_ok ? n0 + c * 32 : 0);
+          if (col_ok) load32_bf16(cp, old);
+          tc_wait_ld();
+          if (col_ok) {
 #pragma unroll
-      for (int e = 0; e < 8; ++e) {
-        a[e] = ct[r * CT_LD + lo + e];
-        b[e] = ct[r * CT_LD + hi + e];
-      }
-      if (bias) {
-        float ba[8], bb[8];
-        unpack8(*reinterpret_cast<const uint4*>(bias + nb0 + lo), ba);
-        unpack8(*reinterpret_cast<const uint4*>(bias + nb0 + hi), bb);
-#pragma unroll
-        for (int e = 0; e < 8; ++e) {
-          a[e] += ba[e];
-          b[e] += bb[e];
-        }
-      }
-      if (kind != 2) {
-        const float2* trow = p.tab + (size_t)ps * half;
-        if (p.layout == 0) {
-          const int f0 = lo % D;  // frequency index of element e is f0 + e
-#pragma unroll
-          for (int e = 0; e < 8; ++e) {
-            float2 cs = __ldg(trow + f0 + e);
-            float x = a[e], y = b[e];
-            a[e] = x * cs.x - y * cs.y;
-            b[e] = x * cs.y + y * cs.x;
-          }
-        } else {
-          const int fa = (lo % D) / 2, fb = (hi % D) / 2;
-#pragma unroll
-          for (int e = 0; e < 4; ++e) {
-            float2 cs = __ldg(trow + fa + e);
-            float x = a[2 * e], y = a[2 * e + 1];
-            a[2 * e] = x * cs.x - y * cs.y;
-            a[2 * e + 1] = x * cs.y + y * cs.x;
-            cs = __ldg(trow + fb + e);
-            x = b[2 * e];
-            y = b[2 * e + 1];
-            b[2 * e] = x * cs.x - y * cs.y;
-            b[2 * e + 1] = x * cs.y + y * cs.x;
+            for (int e = 0; e < 32; ++e) acc[e] += old[e];
+            store32_bf16(cp, acc);
           }
         }
+      } else if (EPI == EPI_SWIGLU) {
+        const int n0 = nt * (BN / 2);
+#pragma unroll 1
+        for (int c = 0; c < BN / 64; ++c) {
+          __syncwarp();
+          float g[32], u[32];
+          tc_ld32(trow + c * 32, g);
+          tc_ld32(trow + BN / 2 + c * 32, u);
+          tc_wait_ld();
+          if (row_ok) {
+#pragma unroll
+            for (int e = 0; e < 32; ++e) g[e] = g[e] / (1.f + __expf(-g[e])) * u[e];
+            store32_bf16(p.C + (size_t)gr * p.ldc + n0 + c * 32, g);
+          }
+        }
+      } else {
+        const int kind = p.kind[seg];
+        const int D = p.D, half = D / 2;
+        const bf16* bias = p.bias[seg];
+        int ps = row_ok ? p.pos[gr] : 0;
+        bool ok = row_ok;
+        if (row_ok && (ps < 0 || ps >= p.kv_len || ps >= p.max_pos)) {
+          atomicOr(p.status, A3_DEV_BAD_POSITION);
+          ok = false;
+          ps = 0;
+        }
+        bf16* dst;
+        if (kind == 0) dst = p.q_out + (size_t)(row_ok ? gr : 0) * (p.Hq * D) + nb0;
+        else if (kind == 1) dst = p.k_cache + (size_t)ps * (p.Hkv * D) + nb0;
+        else dst = p.v_cache + (size_t)ps * (p.Hkv * D) + nb0;
+        const float2* trot = p.tab + (size_t)ps * half;
+        // pairs of 32-column chunks that hold the two halves of the rotation pairs (same chunk twice for the
+        // interleaved layout and for V, which is not rotated)
+        const int pair_stride = (p.layout == 0) ? half / 32 : 0;  // D=128: 2 chunks; D=64: 1 chunk
+#pragma unroll 1
+        for (int c = 0; c < BN / 32; ++c) {
+          const int in_head = (c * 32) % D;
+          if (p.layout == 0 && in_head >= half) continue;  // handled together with its low half
+          __syncwarp();
+          float a[32], b[32];
+          tc_ld32(trow + c * 32, a);
+          if (p.layout == 0) tc_ld32(trow + (c + pair_stride) * 32, b);
+          tc_wait_ld();
+          if (!ok) continue;
+          const int ca = c * 32, cb = (c + pair_stride) * 32;
+          if (bias) {
+            float t[32];
+            load32_bf16(bias + nb0 + ca, t);
+#pragma unroll
+            for (int e = 0; e < 32; ++e) a[e] += t[e];
+            if (p.layout == 0) {
+              load32_bf16(bias + nb0 + cb, t);
+#pragma unroll
+              for (int e = 0; e < 32; ++e) b[e] += t[e];
+            }
+          }
+          if (kind != 2) {
+            if (p.layout == 0) {
+#pragma unroll
+              for (int e = 0; e < 32; ++e) {
+                const float2 cs = __ldg(trot + in_head + e);
+                const float x = a[e], y = b[e];
+                a[e] = x * cs.x - y * cs.y;
+                b[e] = x * cs.y + y * cs.x;
+              }
+            } else {
+#pragma unroll
+              for (int e = 0; e < 16; ++e) {
+                const float2 cs = __ldg(trot + in_head / 2 + e);
+                const float x = a[2 * e], y = a[2 * e + 1];
+                a[2 * e] = x * cs.x - y * cs.y;
+                a[2 * e + 1] = x * cs.y + y * cs.x;
+              }
+            }
+          }
+          store32_bf16(dst + ca, a);
+          if (p.layout == 0) store32_bf16(dst + cb, b);
+        }
       }
-      bf16* dst;
-      if (kind == 0) dst = p.q_out + (size_t)gr * (p.Hq * D) + nb0;
-      else if (kind == 1) dst = p.k_cache + (size_t)ps * (p.Hkv * D) + nb0;
-      else dst = p.v_cache + (size_t)ps * (p.Hkv * D) + nb0;
-      *reinterpret_cast<uint4*>(dst + lo) = pack8(a);
-      *reinterpret_cast<uint4*>(dst + hi) = pack8(b);
     }
   }
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(TMEM_COLS) : "memory");
 }
 
-static int gemm_bf16_mma(const a3_handle* h, GemmEpilogue epi, const GemmArgs& a, cudaStream_t st) {
+// ---------------------------------------------------------------- host side
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                                  const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+static EncodeTiledFn encode_fn() {
+  static EncodeTiledFn fn = nullptr;
+  if (!fn) {
+    void* ptr = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ptr, cudaEnableDefault, &q) == cudaSuccess &&
+        q == cudaDriverEntryPointSuccess)
+      fn = (EncodeTiledFn)ptr;
+  }
+  return fn;
+}
+
+// [rows][cols] bf16 row-major matrix, box = box_rows x 64 columns, 128-byte swizzle, zero fill outside
+static int make_tmap(CUtensorMap* map, const void* ptr, long long rows, long long cols, int box_rows) {
+  EncodeTiledFn fn = encode_fn();
+  if (!fn) return A3_ECUDA;
+  cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
+  cuuint64_t strides[1] = {(cuuint64_t)cols * 2};
+  cuuint32_t box[2] = {(cuuint32_t)TC_BK, (cuuint32_t)box_rows};
+  cuuint32_t estr[2] = {1, 1};
+  CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(ptr), dims, strides, box, estr,
+                  CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                  CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  if (r != CUDA_SUCCESS) {
+    g_last_cuda_error = (int)r;
+    return A3_ECUDA;
+  }
+  return A3_OK;
+}
+
+template <int EPI, int BN, int STAGES>
+static int launch_tc(const a3_handle* h, const GemmArgs& a, const TcParams& p, int tiles, cudaStream_t st) {
+  using L = TcLayout<BN, STAGES>;
+  CUtensorMap tA, tB[3];
+  A3_TRY(make_tmap(&tA, a.A, a.M, a.K, TC_BM));
+  if (EPI == EPI_SWIGLU) {
+    A3_TRY(make_tmap(&tB[0], a.seg[0].B, a.seg[0].n, a.K, BN / 2));
+    A3_TRY(make_tmap(&tB[1], a.B2, a.seg[0].n, a.K, BN / 2));
+    tB[2] = tB[0];
+  } else {
+    for (int s = 0; s < 3; ++s) {
+      if (s < a.nseg) A3_TRY(make_tmap(&tB[s], a.seg[s].B, a.seg[s].n, a.K, BN));
+      else tB[s] = tB[0];
+    }
+  }
+  static bool attr_set = false;
+  if (!attr_set) {
+    A3_CUDA(cudaFuncSetAttribute(gemm_tc_kernel<EPI, BN, STAGES>, cudaFuncAttributeMaxDynamicSharedMemorySize, L::SMEM_BYTES));
+    attr_set = true;
+  }
+  dim3 grid(cdiv(a.M, TC_BM), tiles);
+  ProfScope prof(h, EPI == EPI_RESIDUAL ? A3_K_GEMM_RESIDUAL : EPI == EPI_SWIGLU ? A3_K_GEMM_SWIGLU : A3_K_GEMM_QKV, st);
+  gemm_tc_kernel<EPI, BN, STAGES><<<grid, TC_THREADS, L::SMEM_BYTES, st>>>(tA, tB[0], tB[1], tB[2], p);
+  A3_LAUNCHED();
+  return A3_OK;
+}
+
+// Tile width / pipeline depth per epilogue [EPI_RESIDUAL, EPI_SWIGLU, EPI_QKV] -> {BN, STAGES}; BN = 0 lets the
+// launcher choose (a3_internal_set_gemm_cfg pins a choice for tuning runs).  Measured on B200 at Llama-8B width:
+// two co-resident CTAs per SM (256/2, 128/3) overlap one tile's epilogue with the other's main loop and win when
+// the grid has several waves; a single wave prefers the widest tile that still gives every SM at most one CTA.
+int g_tc_cfg[3][2] = {{0, 0}, {256, 2}, {0, 0}};
+
+template <int EPI>
+static int dispatch_tc(const a3_handle* h, const GemmArgs& a, const TcParams& p, int tiles, int bn, int stages, cudaStream_t st) {
+  if (bn == 256 && stages == 4) return launch_tc<EPI, 256, 4>(h, a, p, tiles, st);
+  if (bn == 256 && stages == 3) return launch_tc<EPI, 256, 3>(h, a, p, tiles, st);
+  if (bn == 256 && stages == 2) return launch_tc<EPI, 256, 2>(h, a, p, tiles, st);
+  if (bn == 224 && stages == 4) return launch_tc<EPI, 224, 4>(h, a, p, tiles, st);
+  if (bn == 192 && stages == 4) return launch_tc<EPI, 192, 4>(h, a, p, tiles, st);
+  if (bn == 128 && stages == 3) return launch_tc<EPI, 128, 3>(h, a, p, tiles, st);
+  if (bn == 128 && stages == 6) return launch_tc<EPI, 128, 6>(h, a, p, tiles, st);
+  return launch_tc<EPI, 128, 4>(h, a, p, tiles, st);
+}
+
+int gemm_bf16(const a3_handle* h, GemmEpilogue epi, const GemmArgs& a, cudaStream_t st) {
   if (a.M <= 0) return A3_OK;
-  if (a.K % BK) return A3_EUNSUPPORTED;
-  GemmDev p{};
-  p.A = a.A;
+  if (a.K % TC_BK) return A3_EUNSUPPORTED;
+  int bn = g_tc_cfg[epi][0];
+  int stages = g_tc_cfg[epi][1];
+  if (bn == 0) {
+    const int m_tiles = cdiv(a.M, TC_BM), sms = h->sm_count > 0 ? h->sm_count : 148;
+    if (epi == EPI_RESIDUAL) {
+      // when a single wave of CTAs covers the output either way, the narrower 224-column tile shortens it
+      const int n = a.seg[0].n;
+      bn = (m_tiles * cdiv(n, 256) <= sms && m_tiles * cdiv(n, 224) <= sms) ? 224 : 256;
+      stages = 4;
+    } else {
+      bn = 256;
+      stages = 4;
+    }
+  }
+  // output columns per tile; QKV tiles must hold whole heads and divide every segment
+  int out_cols = epi == EPI_SWIGLU ? bn / 2 : bn;
+  if (epi == EPI_QKV) {
+    for (int s = 0; s < a.nseg; ++s)
+      if (a.seg[s].n % out_cols) {
+        bn = out_cols = 128;
+        stages = 3;
+      }
+  }
+  TcParams p{};
   p.M = a.M;
   p.K = a.K;
   int tiles = 0;
   for (int s = 0; s < 3; ++s) {
     if (s < a.nseg) {
-      if (a.seg[s].n % (epi == EPI_SWIGLU ? 64 : BN)) return A3_EUNSUPPORTED;
-      p.B[s] = a.seg[s].B;
+      if (epi != EPI_RESIDUAL && a.seg[s].n % out_cols) return A3_EUNSUPPORTED;
+      if (a.seg[s].n % 32) return A3_EUNSUPPORTED;
       p.bias[s] = a.seg[s].bias;
       p.kind[s] = a.seg[s].kind;
-      tiles += a.seg[s].n / (epi == EPI_SWIGLU ? 64 : BN);
+      tiles += cdiv(a.seg[s].n, out_cols);
     }
     p.seg_tiles_end[s] = tiles;
   }
-  p.B2 = a.B2;
+  p.N = a.seg[0].n;
   p.C = a.C;
   p.ldc = a.ldc;
   p.q_out = a.q_out;
@@ -277,31 +492,16 @@ static int gemm_bf16_mma(const a3_handle* h, GemmEpilogue epi, const GemmArgs& a
   p.max_pos = h->m.max_positions;
   p.tab = h->rope_tab;
   p.status = h->dev_status;
-  dim3 grid(cdiv(a.M, BM), tiles);
-  static bool attr_set = false;
-  if (!attr_set) {
-    A3_CUDA(cudaFuncSetAttribute(gemm_mma_kernel<EPI_RESIDUAL>, cudaFuncAttributeMaxDynamicSharedMemorySize, GEMM_SMEM));
-    A3_CUDA(cudaFuncSetAttribute(gemm_mma_kernel<EPI_SWIGLU>, cudaFuncAttributeMaxDynamicSharedMemorySize, GEMM_SMEM));
-    A3_CUDA(cudaFuncSetAttribute(gemm_mma_kernel<EPI_QKV>, cudaFuncAttributeMaxDynamicSharedMemorySize, GEMM_SMEM));
-    attr_set = true;
-  }
-  ProfScope prof(h, epi == EPI_RESIDUAL ? A3_K_GEMM_RESIDUAL : epi == EPI_SWIGLU ? A3_K_GEMM_SWIGLU : A3_K_GEMM_QKV, st);
-  if (epi == EPI_RESIDUAL) gemm_mma_kernel<EPI_RESIDUAL><<<grid, GEMM_THREADS, GEMM_SMEM, st>>>(p);
-  else if (epi == EPI_SWIGLU) gemm_mma_kernel<EPI_SWIGLU><<<grid, GEMM_THREADS, GEMM_SMEM, st>>>(p);
-  else gemm_mma_kernel<EPI_QKV><<<grid, GEMM_THREADS, GEMM_SMEM, st>>>(p);
-  A3_LAUNCHED();
-  return A3_OK;
-}
-
-int gemm_bf16_tc(const a3_handle* h, GemmEpilogue epi, const GemmArgs& a, cudaStream_t st);
-
-// 0: tcgen05 kernel (a3_gemm_tc.cu); 1: the warp-level mma.sync kernel above, kept as a cross-check for bring-up
-int g_gemm_impl = 0;
-
-int gemm_bf16(const a3_handle* h, GemmEpilogue epi, const GemmArgs& a, cudaStream_t st) {
-  return g_gemm_impl == 1 ? gemm_bf16_mma(h, epi, a, st) : gemm_bf16_tc(h, epi, a, st);
+  if (epi == EPI_RESIDUAL) return dispatch_tc<EPI_RESIDUAL>(h, a, p, tiles, bn, stages, st);
+  if (epi == EPI_SWIGLU) return dispatch_tc<EPI_SWIGLU>(h, a, p, tiles, bn, stages, st);
+  return dispatch_tc<EPI_QKV>(h, a, p, tiles, bn, stages, st);
 }
 
 }  // namespace a3
 
-extern "C" void a3_internal_set_gemm_impl(int impl) { a3::g_gemm_impl = impl; }
+extern "C" void a3_internal_set_gemm_cfg(int epi, int bn, int stages) {
+  if (epi >= 0 && epi < 3) {
+    a3::g_tc_cfg[epi][0] = bn;
+    a3::g_tc_cfg[epi][1] = stages;
+  }
+}

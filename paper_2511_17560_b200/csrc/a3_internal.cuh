@@ -18,7 +18,7 @@ struct a3_handle {
   uint32_t* dev_status;      // dev, 1 word (+ padding)
   int device;
   int sm_count;
-  void* tmaps;               // host-side tensor-map cache (a3_gemm_tc.cu)
+  void* tmaps;               // host-side tensor-map cache (a3_gemm.cu)
   a3::Profiler* prof;        // null unless a3_profile_enable is on
   void* host_pipe;           // copy stream + events of a3_fuse_request_host, created on first use
 };
