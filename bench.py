@@ -26,6 +26,10 @@ ROOT = os.path.dirname(os.path.abspath(__file__))
 if ROOT not in sys.path:
     sys.path.insert(0, ROOT)
 
+# DRAM bytes (read + write) per launch from the ncu capture summarised in profiles/gemm_tc_kernel_llama8b_2layer.txt:
+# the SwiGLU GEMM of a sparse layer (M = 804) and of the full block (M = 5152) at Llama-8B width.
+NCU_TRAFFIC = {("llama8b_10x512", "gemm_swiglu"): {"sparse": 255.72e6 + 19.23e6, "full": 390.77e6 + 136.75e6}}
+
 METRIC = "context_tokens_fused_per_s"
 UNIT = "tokens/s"
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
@@ -338,9 +342,14 @@ def run_a3(args):
         k["share"] = k["ms_per_step"] / tot_ms
     top = max(kernels, key=lambda nm: kernels[nm]["ms_per_step"])
     tk = kernels[top]
+    traffic = None
+    t = NCU_TRAFFIC.get((args.config, top))
+    if t and not args.layers:
+        n_full = r.select_layer
+        traffic = (t["full"] * n_full + t["sparse"] * (m.n_layers - n_full)) / m.n_layers  # average over the class's launches
     roofline = {"kernel": top, "bound": tk.get("bound"), "achieved": tk.get("achieved"),
                 "peak": peaks["bf16_tflops_sustained"] if tk.get("bound") == "tensor" else peaks["hbm_gbs"],
-                "unit": tk.get("unit"), "frac": tk.get("frac"), "traffic": None, "peak_source": peak_src + " (sustained)",
+                "unit": tk.get("unit"), "frac": tk.get("frac"), "traffic": traffic, "peak_source": peak_src + " (sustained)",
                 "avg_launch_ms": tk["ms_per_step"] / tk["launches_per_step"], "kernels": kernels}
     total_flops = sum(flops.values())
 
