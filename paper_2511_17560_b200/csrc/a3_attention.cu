@@ -140,15 +140,17 @@ __device__ __forceinline__ float ex2_approx(float x) {
 // t = s * scale - m_ref is one FMA; ex2.approx maps -inf to +0, so masked keys need no second select.
 template <bool MASK>
 __device__ __forceinline__ void softmax_chunk(float* sv, int key_base, int lim, float scale, float neg_ref, float& mx, float (&ls)[4]) {
+  float m4[4] = {mx, mx, mx, mx};  // four independent chains for the maximum, like the row sum
 #pragma unroll
   for (int e = 0; e < 32; ++e) {
     float t = fmaf(sv[e], scale, neg_ref);
     if (MASK && key_base + e > lim) t = -INFINITY;
-    mx = fmaxf(mx, t);
+    m4[e & 3] = fmaxf(m4[e & 3], t);
     const float pe = ex2_approx(t);
     sv[e] = pe;
     ls[e & 3] += pe;
   }
+  mx = fmaxf(fmaxf(m4[0], m4[1]), fmaxf(m4[2], m4[3]));
 }
 
 template <int D>
@@ -164,12 +166,49 @@ struct AtcLayout {
   static constexpr int SMEM_BYTES = BAR_OFF + 256 + 1024;
 };
 
+// One unit of work: a 128-row tile of one KV head and one segment of its key tiles.
+struct AtcItem {
+  int g, r0, maxpos, minpos;
+  int nkt_all;   // key tiles the row tile needs in total
+  int kt0, nkt;  // this segment: first key tile and count
+  int z;         // segment index
+  bool valid;    // the segment exists for this row tile
+  bool partial;  // the row tile has several segments: leave unnormalised partial results for the combine kernel
+};
+
+// Items are numbered longest row tile first (rows are sorted by position, so the last tile sees the most keys),
+// then segment, then KV head.
+__device__ __forceinline__ AtcItem atc_item(int i, const int32_t* __restrict__ pos, int M, int G, int Hkv, int kv_len,
+                                            int row_tiles, int n_split, int tiles_per_split) {
+  AtcItem it;
+  const int per_tile = n_split * Hkv;
+  const int tile = row_tiles - 1 - i / per_tile;
+  const int rem = i % per_tile;
+  it.z = rem / Hkv;
+  it.g = rem % Hkv;
+  it.r0 = tile * ATC_BM;
+  const int last_tok = min(M - 1, (it.r0 + ATC_BM - 1) / G);
+  it.maxpos = min(pos[last_tok], kv_len - 1);
+  it.minpos = pos[it.r0 / G];
+  it.nkt_all = it.maxpos < 0 ? 0 : it.maxpos / ATC_BN + 1;
+  const int n_active = (it.nkt_all + tiles_per_split - 1) / tiles_per_split;
+  it.valid = it.z < max(n_active, 1);
+  it.kt0 = it.z * tiles_per_split;
+  it.nkt = max(0, min(tiles_per_split, it.nkt_all - it.kt0));
+  it.partial = n_active > 1;
+  return it;
+}
+
+// Persistent kernel: one CTA per SM walks its share of the items.  Item i of round r goes to CTA (i mod C) on even
+// rounds and to CTA C-1-(i mod C) on odd ones, so every CTA gets a mix of long and short items without any atomic.
+// Barrier phases and buffer indices follow counters that run across items (`it`: key tiles, `qn`: items with work),
+// so the TMA producer keeps prefetching the next item's K/V while the current one drains.
 template <int D>
 __global__ void __launch_bounds__(ATC_THREADS, 1)
 attention_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV,
                     const bf16* __restrict__ q, const int32_t* __restrict__ pos, int M, int kv_len, bf16* __restrict__ o,
                     float* __restrict__ lse, int Hq, int Hkv, float scale_log2, uint32_t* status,
-                    int tiles_per_split, float* __restrict__ part_o, float2* __restrict__ part_ml) {
+                    int n_split, int tiles_per_split, float* __restrict__ part_o, float2* __restrict__ part_ml) {
   using L = AtcLayout<D>;
   using namespace atc;
   extern __shared__ unsigned char smem_raw[];
@@ -190,24 +229,18 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int G = Hq / Hkv;
-  const int g = blockIdx.y;
-  const int tile = gridDim.x - 1 - blockIdx.x;  // latest (longest) row tiles first
-  const int r0 = tile * ATC_BM;
   const int rows_total = M * G;
+  const int row_tiles = (rows_total + ATC_BM - 1) / ATC_BM;
+  const int rows_pad = row_tiles * ATC_BM;
+  const int n_items = row_tiles * n_split * Hkv;
+  const int C = gridDim.x, cta = blockIdx.x;
   const bool want_o = o != nullptr;
-
-  const int last_tok = min(M - 1, (r0 + ATC_BM - 1) / G);
-  const int maxpos = min(pos[last_tok], kv_len - 1);
-  const int minpos = pos[r0 / G];
-  const int nkt_all = maxpos < 0 ? 0 : maxpos / ATC_BN + 1;
-  // Split over the keys (blockIdx.z): when the grid has few row tiles, long tiles are cut into segments of
-  // tiles_per_split key tiles that run as separate CTAs and leave unnormalised partial results (output, exponent
-  // reference, row sum) for a combine kernel.  A row tile short enough for one segment writes its result directly.
-  const int n_active = (nkt_all + tiles_per_split - 1) / tiles_per_split;
-  if ((int)blockIdx.z >= max(n_active, 1)) return;  // uniform for the CTA: nothing has been set up yet
-  const int kt0 = blockIdx.z * tiles_per_split;
-  const int nkt = max(0, min(tiles_per_split, nkt_all - kt0));  // key tiles of this CTA; loops count locally
-  const bool partial = n_active > 1;
+  // item of round r for this CTA, or -1
+  auto item_index = [&](int r) {
+    const int i = r * C + ((r & 1) ? C - 1 - cta : cta);
+    return i < n_items ? i : -1;
+  };
+  const int rounds = (n_items + C - 1) / C;
 
   if (threadIdx.x == 0) {
     for (int i = 0; i < 2; ++i) {
@@ -238,195 +271,231 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
     if (lane == 0) {
       asm volatile("prefetch.tensormap [%0];" ::"l"(&tmK) : "memory");
       asm volatile("prefetch.tensormap [%0];" ::"l"(&tmV) : "memory");
-      for (int kt = 0; kt < nkt; ++kt) {
-        const int s = kt & 1;
-        if (!mbar_wait(kv_empty(s), ((kt >> 1) & 1) ^ 1, abort_flag, status)) break;
-        const uint32_t sk = base + L::KV_OFF + s * L::KV_STAGE, sv = sk + (D / 64) * L::SUB;
-        mbar_expect_tx(kv_full(s), L::KV_STAGE);
+      uint32_t it = 0;
+      bool ok = true;
+      for (int r = 0; r < rounds && ok; ++r) {
+        const int i = item_index(r);
+        if (i < 0) continue;
+        const AtcItem w = atc_item(i, pos, M, G, Hkv, kv_len, row_tiles, n_split, tiles_per_split);
+        if (!w.valid) continue;
+        for (int kt = 0; kt < w.nkt; ++kt, ++it) {
+          const int s = it & 1;
+          ok = mbar_wait(kv_empty(s), ((it >> 1) & 1) ^ 1, abort_flag, status);
+          if (!ok) break;
+          const uint32_t sk = base + L::KV_OFF + s * L::KV_STAGE, sv = sk + (D / 64) * L::SUB;
+          mbar_expect_tx(kv_full(s), L::KV_STAGE);
 #pragma unroll
-        for (int j = 0; j < D / 64; ++j) {
-          tma_load_2d(sk + j * L::SUB, &tmK, g * D + 64 * j, (kt0 + kt) * ATC_BN, kv_full(s));
-          tma_load_2d(sv + j * L::SUB, &tmV, g * D + 64 * j, (kt0 + kt) * ATC_BN, kv_full(s));
+          for (int j = 0; j < D / 64; ++j) {
+            tma_load_2d(sk + j * L::SUB, &tmK, w.g * D + 64 * j, (w.kt0 + kt) * ATC_BN, kv_full(s));
+            tma_load_2d(sv + j * L::SUB, &tmV, w.g * D + 64 * j, (w.kt0 + kt) * ATC_BN, kv_full(s));
+          }
         }
       }
     }
   } else if (warp == 1) {
     // ---------------- MMA issuer
-    if (lane == 0 && nkt > 0) {
+    if (lane == 0) {
       constexpr uint32_t idesc_s = idesc(ATC_BN, 0);
       constexpr uint32_t idesc_o = idesc(D, 1);
       const uint32_t sq = base + L::Q_OFF, sp = base + L::P_OFF;
-      auto issue_s = [&](int kt) {
-        const uint32_t sk = base + L::KV_OFF + (kt & 1) * L::KV_STAGE;
+      auto issue_s = [&](uint32_t t) {  // S of running key tile t into S buffer t & 1, from K stage t & 1
+        const uint32_t sk = base + L::KV_OFF + (t & 1) * L::KV_STAGE;
 #pragma unroll
         for (int k = 0; k < D / 16; ++k) {
           const uint32_t sub = (k / 4) * L::SUB + (k % 4) * 32;
-          mma_f16(tmem_s0 + (kt & 1) * 128, desc_k_sw128(sq + sub), desc_k_sw128(sk + sub), idesc_s, k != 0);
+          mma_f16(tmem_s0 + (t & 1) * 128, desc_k_sw128(sq + sub), desc_k_sw128(sk + sub), idesc_s, k != 0);
         }
-        commit(s_full(kt & 1));
+        commit(s_full(t & 1));
       };
-      bool ok = mbar_wait(q_ready, 0, abort_flag, status);
-      ok = ok && mbar_wait(kv_full(0), 0, abort_flag, status);
-      if (ok) {
-        fence_after();
-        issue_s(0);
-      }
-      for (int kt = 0; kt < nkt && ok; ++kt) {
-        if (kt + 1 < nkt) {
-          ok = mbar_wait(kv_full((kt + 1) & 1), ((kt + 1) >> 1) & 1, abort_flag, status);
-          if (!ok) break;
-
-          fence_after();
-          issue_s(kt + 1);
-        }
-        ok = mbar_wait(p_ready(kt & 1), (kt >> 1) & 1, abort_flag, status);
+      uint32_t it = 0, qn = 0;
+      bool ok = true;
+      for (int r = 0; r < rounds && ok; ++r) {
+        const int i = item_index(r);
+        if (i < 0) continue;
+        const AtcItem w = atc_item(i, pos, M, G, Hkv, kv_len, row_tiles, n_split, tiles_per_split);
+        if (!w.valid || w.nkt == 0) continue;
+        ok = mbar_wait(q_ready, qn & 1, abort_flag, status);
+        ++qn;
+        ok = ok && mbar_wait(kv_full(it & 1), (it >> 1) & 1, abort_flag, status);
         if (!ok) break;
-
         fence_after();
-        if (want_o) {
-          const uint32_t sv = base + L::KV_OFF + (kt & 1) * L::KV_STAGE + (D / 64) * L::SUB;
-#pragma unroll
-          for (int k = 0; k < ATC_BN / 16; ++k) {
-            const uint64_t da = desc_k_sw128(sp + (kt & 1) * L::P_BYTES + (k / 4) * L::SUB + (k % 4) * 32);
-            const uint64_t db = desc_mn_sw128(sv + k * 16 * 128, L::SUB);
-            mma_f16(tmem_o, da, db, idesc_o, (kt | k) != 0);  // O accumulates over the key tiles in TMEM
+        issue_s(it);
+        for (int kt = 0; kt < w.nkt; ++kt, ++it) {
+          if (kt + 1 < w.nkt) {
+            ok = mbar_wait(kv_full((it + 1) & 1), ((it + 1) >> 1) & 1, abort_flag, status);
+            if (!ok) break;
+            fence_after();
+            issue_s(it + 1);
           }
-          commit(p_free(kt & 1));  // P V of this tile is complete: its P buffer may be rewritten, O holds tiles 0..kt
+          ok = mbar_wait(p_ready(it & 1), (it >> 1) & 1, abort_flag, status);
+          if (!ok) break;
+          fence_after();
+          if (want_o) {
+            const uint32_t sv = base + L::KV_OFF + (it & 1) * L::KV_STAGE + (D / 64) * L::SUB;
+#pragma unroll
+            for (int k = 0; k < ATC_BN / 16; ++k) {
+              const uint64_t da = desc_k_sw128(sp + (it & 1) * L::P_BYTES + (k / 4) * L::SUB + (k % 4) * 32);
+              const uint64_t db = desc_mn_sw128(sv + k * 16 * 128, L::SUB);
+              mma_f16(tmem_o, da, db, idesc_o, (kt | k) != 0);  // O accumulates over the item's key tiles in TMEM
+            }
+            commit(p_free(it & 1));  // P V of this tile is complete: its P buffer may be rewritten, O holds tiles 0..kt
+          }
+          commit(kv_empty(it & 1));
         }
-        commit(kv_empty(kt & 1));
       }
     }
   } else {
     // ---------------- softmax / epilogue: thread = row
     const int quarter = warp & 3;
     const int row = quarter * 32 + lane;
-    const int fr = r0 + row;
-    const bool row_ok = fr < rows_total;
-    const int tok = row_ok ? fr / G : 0;
-    const int hq = g * G + (row_ok ? fr % G : 0);
-    const int lim = row_ok ? min(pos[tok], kv_len - 1) : -1;
     const uint32_t lane_addr = (uint32_t)(quarter * 32) << 16;
-
-    // Q row -> shared memory, swizzled K-major sub-tiles
-    {
-      const uint4* src = reinterpret_cast<const uint4*>(q + ((size_t)tok * Hq + hq) * D);
-#pragma unroll
-      for (int c = 0; c < D / 8; ++c) {
-        uint4 v = row_ok ? __ldg(src + c) : make_uint4(0, 0, 0, 0);
-        *reinterpret_cast<uint4*>(base_ptr + L::Q_OFF + (c / 8) * L::SUB + swz(row, c % 8)) = v;
-      }
-      fence_async_smem();
-      mbar_arrive(q_ready);
-    }
-
-    // Exponent reference m_ref and row sum l_run relative to it.  The reference is the true maximum of the first
-    // tile and is raised later only when a logit exceeds it by more than 2^RESCALE_TH (rare once the first tiles
-    // are seen): then the output accumulated in TMEM and l_run are rescaled and the tile is redone.  Probabilities
-    // therefore stay below 2^RESCALE_TH, and the output needs no per-tile correction.
     constexpr float RESCALE_TH = 8.f;
-    float m_ref = 0.f, l_run = 0.f;
+    uint32_t it = 0;
     bool ok = true;
 
-    for (int kt = 0; kt < nkt; ++kt) {
-      // the result of every wait is made warp-uniform: tcgen05.ld/st are warp-wide instructions
-      ok = __all_sync(0xffffffffu, mbar_wait(s_full(kt & 1), (kt >> 1) & 1, abort_flag, status));
-      if (!ok) break;
-      fence_after();
-      const uint32_t ts = tmem_s0 + (kt & 1) * 128 + lane_addr;
-      const int key0 = (kt0 + kt) * ATC_BN;
-      const bool need_mask = key0 + ATC_BN - 1 > minpos;
-      if (kt == 0) {
-        float mx = -INFINITY;
-#pragma unroll 1
-        for (int c = 0; c < 4; ++c) {
-          float sv[32];
-          ld32(ts + c * 32, sv);
-          wait_ld();
+    for (int r = 0; r < rounds && ok; ++r) {
+      const int i = item_index(r);
+      if (i < 0) continue;
+      const AtcItem w = atc_item(i, pos, M, G, Hkv, kv_len, row_tiles, n_split, tiles_per_split);
+      if (!w.valid) continue;
+      const int fr = w.r0 + row;
+      const bool row_ok = fr < rows_total;
+      const int tok = row_ok ? fr / G : 0;
+      const int hq = w.g * G + (row_ok ? fr % G : 0);
+      const int lim = row_ok ? min(pos[tok], kv_len - 1) : -1;
+      const size_t prow = ((size_t)w.z * Hkv + w.g) * (size_t)rows_pad + fr;  // partial-result row
+
+      if (w.nkt == 0) {
+        // no visible key at all (only with invalid positions): defined output, no pipeline work
+        if (row_ok && want_o && !w.partial) {
+          uint4* dst = reinterpret_cast<uint4*>(o + ((size_t)tok * Hq + hq) * D);
 #pragma unroll
-          for (int e = 0; e < 32; ++e) {
-            float x = sv[e] * scale_log2;
-            if (need_mask && key0 + c * 32 + e > lim) x = -INFINITY;
-            mx = fmaxf(mx, x);
-          }
+          for (int c = 0; c < D / 8; ++c) dst[c] = make_uint4(0, 0, 0, 0);
         }
-        m_ref = mx == -INFINITY ? 0.f : mx;
+        if (row_ok && w.partial) part_ml[prow] = make_float2(0.f, 0.f);
+        if (row_ok && !w.partial && lse) lse[(size_t)tok * Hq + hq] = -INFINITY;
+        continue;
       }
-      if (want_o && kt >= 2) {
-        // the P buffer of this tile was last read by the P V of tile kt-2
-        ok = __all_sync(0xffffffffu, mbar_wait(p_free(kt & 1), ((kt >> 1) & 1) ^ 1, abort_flag, status));
+
+      // Q row -> shared memory, swizzled K-major sub-tiles.  The previous item's S MMAs have all completed (their
+      // last s_full was waited for), so the Q buffer is free.
+      {
+        const uint4* src = reinterpret_cast<const uint4*>(q + ((size_t)tok * Hq + hq) * D);
+#pragma unroll
+        for (int c = 0; c < D / 8; ++c) {
+          uint4 v = row_ok ? __ldg(src + c) : make_uint4(0, 0, 0, 0);
+          *reinterpret_cast<uint4*>(base_ptr + L::Q_OFF + (c / 8) * L::SUB + swz(row, c % 8)) = v;
+        }
+        fence_async_smem();
+        mbar_arrive(q_ready);
+      }
+
+      // Exponent reference m_ref and row sum l_run relative to it.  The reference is the true maximum of the first
+      // tile and is raised later only when a logit exceeds it by more than 2^RESCALE_TH (rare once the first tiles
+      // are seen): then the output accumulated in TMEM and l_run are rescaled and the tile is redone.
+      float m_ref = 0.f, l_run = 0.f;
+      uint32_t it_last = it;
+      for (int kt = 0; kt < w.nkt; ++kt, ++it) {
+        it_last = it;
+        // the result of every wait is made warp-uniform: tcgen05.ld/st are warp-wide instructions
+        ok = __all_sync(0xffffffffu, mbar_wait(s_full(it & 1), (it >> 1) & 1, abort_flag, status));
         if (!ok) break;
-      }
+        fence_after();
+        const uint32_t ts = tmem_s0 + (it & 1) * 128 + lane_addr;
+        const int key0 = (w.kt0 + kt) * ATC_BN;
+        const bool need_mask = key0 + ATC_BN - 1 > w.minpos;
+        if (kt == 0) {
+          float mx = -INFINITY;
 #pragma unroll 1
-      for (int trip = 0; trip < 2; ++trip) {
-        // mx is tracked relative to the reference: the exponent argument itself, fmaf(s, scale, -m_ref)
-        float mx = -INFINITY, ls[4] = {0.f, 0.f, 0.f, 0.f};
-        const float neg_ref = -m_ref;
-        float buf[2][32];
-        ld32(ts, buf[0]);
-#pragma unroll
-        for (int c = 0; c < 4; ++c) {
-          wait_ld();
-          if (c < 3) ld32(ts + (c + 1) * 32, buf[(c + 1) & 1]);
-          float* sv = buf[c & 1];
-          if (need_mask) softmax_chunk<true>(sv, key0 + c * 32, lim, scale_log2, neg_ref, mx, ls);
-          else softmax_chunk<false>(sv, key0 + c * 32, lim, scale_log2, neg_ref, mx, ls);
-          if (want_o) {
-#pragma unroll
-            for (int i = 0; i < 4; ++i)
-              *reinterpret_cast<uint4*>(base_ptr + L::P_OFF + (kt & 1) * L::P_BYTES + (c >> 1) * L::SUB + swz(row, (c & 1) * 4 + i)) = pack8(sv + 8 * i);
-          }
-        }
-        const float lsum = (ls[0] + ls[1]) + (ls[2] + ls[3]);
-        if (!__any_sync(0xffffffffu, mx > RESCALE_TH)) {
-          l_run += lsum;
-          break;
-        }
-        const float raise = fmaxf(mx, 0.f);  // lanes below the threshold may move too: any value >= their maximum is valid
-        const float f = exp2f(-raise);
-        m_ref += raise;
-        l_run *= f;
-        if (want_o && kt > 0) {
-          // the output so far must be complete (P V of the previous tile) before it is rescaled in place
-          // (the threads follow every phase of p_free[b] in order - tile kt-1 waited for tile kt-3 on the same
-          // barrier - so a parity wait cannot mistake an older completion for this one)
-          ok = __all_sync(0xffffffffu, mbar_wait(p_free((kt - 1) & 1), ((kt - 1) >> 1) & 1, abort_flag, status));
-          if (!ok) break;
-          fence_after();
-#pragma unroll 1
-          for (int c = 0; c < D / 32; ++c) {
-            float t[32];
-            ld32(tmem_o + lane_addr + c * 32, t);
+          for (int c = 0; c < 4; ++c) {
+            float sv[32];
+            ld32(ts + c * 32, sv);
             wait_ld();
 #pragma unroll
-            for (int e = 0; e < 32; ++e) t[e] *= f;
-            st32(tmem_o + lane_addr + c * 32, t);
+            for (int e = 0; e < 32; ++e) {
+              float x = sv[e] * scale_log2;
+              if (need_mask && key0 + c * 32 + e > lim) x = -INFINITY;
+              mx = fmaxf(mx, x);
+            }
           }
-          wait_st();
+          m_ref = mx == -INFINITY ? 0.f : mx;
         }
+        if (want_o && it >= 2) {
+          // the P buffer of this tile was last read by the P V of running tile it-2
+          ok = __all_sync(0xffffffffu, mbar_wait(p_free(it & 1), ((it >> 1) & 1) ^ 1, abort_flag, status));
+          if (!ok) break;
+        }
+#pragma unroll 1
+        for (int trip = 0; trip < 2; ++trip) {
+          // mx is tracked relative to the reference: the exponent argument itself, fmaf(s, scale, -m_ref)
+          float mx = -INFINITY, ls[4] = {0.f, 0.f, 0.f, 0.f};
+          const float neg_ref = -m_ref;
+          float buf[2][32];
+          ld32(ts, buf[0]);
+#pragma unroll
+          for (int c = 0; c < 4; ++c) {
+            wait_ld();
+            if (c < 3) ld32(ts + (c + 1) * 32, buf[(c + 1) & 1]);
+            float* sv = buf[c & 1];
+            if (need_mask) softmax_chunk<true>(sv, key0 + c * 32, lim, scale_log2, neg_ref, mx, ls);
+            else softmax_chunk<false>(sv, key0 + c * 32, lim, scale_log2, neg_ref, mx, ls);
+            if (want_o) {
+#pragma unroll
+              for (int j = 0; j < 4; ++j)
+                *reinterpret_cast<uint4*>(base_ptr + L::P_OFF + (it & 1) * L::P_BYTES + (c >> 1) * L::SUB + swz(row, (c & 1) * 4 + j)) = pack8(sv + 8 * j);
+            }
+          }
+          const float lsum = (ls[0] + ls[1]) + (ls[2] + ls[3]);
+          if (!__any_sync(0xffffffffu, mx > RESCALE_TH)) {
+            l_run += lsum;
+            break;
+          }
+          const float raise = fmaxf(mx, 0.f);  // lanes below the threshold may move too: any value >= their maximum is valid
+          const float f = exp2f(-raise);
+          m_ref += raise;
+          l_run *= f;
+          if (want_o && kt > 0) {
+            // the output so far must be complete (P V of the previous tile) before it is rescaled in place
+            // (the threads follow every phase of p_free[b] in order - running tile it-1 waited for it-3 on the same
+            // barrier - so a parity wait cannot mistake an older completion for this one)
+            ok = __all_sync(0xffffffffu, mbar_wait(p_free((it - 1) & 1), ((it - 1) >> 1) & 1, abort_flag, status));
+            if (!ok) break;
+            fence_after();
+#pragma unroll 1
+            for (int c = 0; c < D / 32; ++c) {
+              float t[32];
+              ld32(tmem_o + lane_addr + c * 32, t);
+              wait_ld();
+#pragma unroll
+              for (int e = 0; e < 32; ++e) t[e] *= f;
+              st32(tmem_o + lane_addr + c * 32, t);
+            }
+            wait_st();
+          }
+        }
+        if (!ok) break;
+        if (want_o && w.kt0 + kt == w.nkt_all - 1) {
+          // slots beyond the row tile's last visible key may hold anything: they get probability zero, and zero
+          // times a non-finite value would still poison the product, so clear those V rows of the last tile
+          const int first_bad = w.maxpos - key0 + 1;
+          const bool landed = mbar_wait(kv_full(it & 1), (it >> 1) & 1, abort_flag, status);  // already complete: S of this tile was computed
+          if (landed && row >= first_bad) {
+            unsigned char* sv = base_ptr + L::KV_OFF + (it & 1) * L::KV_STAGE + (D / 64) * L::SUB;
+#pragma unroll
+            for (int j = 0; j < D / 64; ++j)
+#pragma unroll
+              for (int c = 0; c < 8; ++c) *reinterpret_cast<uint4*>(sv + j * L::SUB + row * 128 + c * 16) = make_uint4(0, 0, 0, 0);
+          }
+        }
+        fence_async_smem();
+        fence_before();
+        mbar_arrive(p_ready(it & 1));
       }
       if (!ok) break;
-      if (want_o && kt0 + kt == nkt_all - 1) {
-        // slots beyond the CTA's last visible key may hold anything: they get probability zero, and zero times a
-        // non-finite value would still poison the product, so clear those V rows of the last tile
-        const int first_bad = maxpos - key0 + 1;
-        const bool landed = mbar_wait(kv_full(kt & 1), (kt >> 1) & 1, abort_flag, status);  // already complete: S of this tile was computed
-        if (landed && row >= first_bad) {
-          unsigned char* sv = base_ptr + L::KV_OFF + (kt & 1) * L::KV_STAGE + (D / 64) * L::SUB;
-#pragma unroll
-          for (int j = 0; j < D / 64; ++j)
-#pragma unroll
-            for (int c = 0; c < 8; ++c) *reinterpret_cast<uint4*>(sv + j * L::SUB + row * 128 + c * 16) = make_uint4(0, 0, 0, 0);
-        }
-      }
-      fence_async_smem();
-      fence_before();
-      mbar_arrive(p_ready(kt & 1));
-    }
-    const float inv = l_run > 0.f ? 1.f / l_run : 0.f;
-    const size_t prow = ((size_t)blockIdx.z * Hkv + g) * ((size_t)gridDim.x * ATC_BM) + fr;  // partial-result row
-    if (ok && want_o && nkt > 0) {
-      ok = __all_sync(0xffffffffu, mbar_wait(p_free((nkt - 1) & 1), ((nkt - 1) >> 1) & 1, abort_flag, status));
-      if (ok) {
+      const float inv = l_run > 0.f ? 1.f / l_run : 0.f;
+      if (want_o) {
+        ok = __all_sync(0xffffffffu, mbar_wait(p_free(it_last & 1), (it_last >> 1) & 1, abort_flag, status));
+        if (!ok) break;
         fence_after();
         bf16* dst = o + ((size_t)tok * Hq + hq) * D;
 #pragma unroll 1
@@ -434,22 +503,25 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
           float t[32];
           ld32(tmem_o + lane_addr + c * 32, t);
           wait_ld();
-          if (row_ok && partial) {
+          if (row_ok && w.partial) {
             float4* pd = reinterpret_cast<float4*>(part_o + prow * D + c * 32);
 #pragma unroll
-            for (int i = 0; i < 8; ++i) pd[i] = make_float4(t[4 * i], t[4 * i + 1], t[4 * i + 2], t[4 * i + 3]);
+            for (int j = 0; j < 8; ++j) pd[j] = make_float4(t[4 * j], t[4 * j + 1], t[4 * j + 2], t[4 * j + 3]);
           } else if (row_ok) {
 #pragma unroll
             for (int e = 0; e < 32; ++e) t[e] *= inv;
 #pragma unroll
-            for (int i = 0; i < 4; ++i) reinterpret_cast<uint4*>(dst + c * 32)[i] = pack8(t + 8 * i);
+            for (int j = 0; j < 4; ++j) reinterpret_cast<uint4*>(dst + c * 32)[j] = pack8(t + 8 * j);
           }
           __syncwarp();
         }
+        // the next item's first P V overwrites O: it is issued only after this item's p_ready arrivals of all 128
+        // threads for that tile, which each thread makes after the loads above
+        fence_before();
       }
+      if (row_ok && w.partial) part_ml[prow] = make_float2(m_ref, l_run);
+      if (row_ok && !w.partial && lse) lse[(size_t)tok * Hq + hq] = l_run > 0.f ? (m_ref + log2f(l_run)) * ATC_LN2 : -INFINITY;
     }
-    if (ok && row_ok && partial) part_ml[prow] = make_float2(m_ref, l_run);
-    if (ok && row_ok && !partial && lse) lse[(size_t)tok * Hq + hq] = l_run > 0.f ? (m_ref + log2f(l_run)) * ATC_LN2 : -INFINITY;
   }
   atc::fence_before();
   __syncthreads();
@@ -553,14 +625,15 @@ int attention_rows(const a3_handle* h, const bf16* q, const int32_t* pos, int M,
   const int base_ctas = (int)grid.x * Hkv, all_tiles = cdiv(kv_len, ATC_BN);
   int n_split = 1;
   if (o && part && base_ctas < 2 * sms && all_tiles >= 8) {
-    n_split = g_attn_split > 0 ? g_attn_split : 2;  // measured: 2 segments beat 1, 3 and 4 at 208 base CTAs (7-8 us fixed cost per CTA)
+    n_split = g_attn_split > 0 ? g_attn_split : 1;  // measured: with the persistent schedule no split beats 2..4 segments (7 us per item)
     const size_t need = (size_t)n_split * base_ctas * ATC_BM * ((size_t)D + 2) * sizeof(float);
     if (need > part_bytes) n_split = 1;
   }
   const int tiles_per_split = cdiv(all_tiles, n_split);
   n_split = cdiv(all_tiles, tiles_per_split);
-  grid.z = n_split;
   const int rows_pad = (int)grid.x * ATC_BM;
+  const int n_items = (int)grid.x * Hkv * n_split;
+  const int n_ctas = n_items < sms ? n_items : sms;  // persistent: at most one CTA per SM
   float* part_o = (float*)part;
   float2* part_ml = part ? (float2*)(part_o + (size_t)n_split * Hkv * rows_pad * D) : nullptr;
   static bool attr_set = false;
@@ -571,9 +644,9 @@ int attention_rows(const a3_handle* h, const bf16* q, const int32_t* pos, int M,
   }
   ProfScope prof(h, A3_K_ATTENTION, st);
   if (D == 128)
-    attention_tc_kernel<128><<<grid, ATC_THREADS, AtcLayout<128>::SMEM_BYTES, st>>>(tK, tV, q, pos, M, kv_len, o, lse, Hq, Hkv, scale_log2, h->dev_status, tiles_per_split, part_o, part_ml);
+    attention_tc_kernel<128><<<n_ctas, ATC_THREADS, AtcLayout<128>::SMEM_BYTES, st>>>(tK, tV, q, pos, M, kv_len, o, lse, Hq, Hkv, scale_log2, h->dev_status, n_split, tiles_per_split, part_o, part_ml);
   else
-    attention_tc_kernel<64><<<grid, ATC_THREADS, AtcLayout<64>::SMEM_BYTES, st>>>(tK, tV, q, pos, M, kv_len, o, lse, Hq, Hkv, scale_log2, h->dev_status, tiles_per_split, part_o, part_ml);
+    attention_tc_kernel<64><<<n_ctas, ATC_THREADS, AtcLayout<64>::SMEM_BYTES, st>>>(tK, tV, q, pos, M, kv_len, o, lse, Hq, Hkv, scale_log2, h->dev_status, n_split, tiles_per_split, part_o, part_ml);
   A3_LAUNCHED();
   if (n_split > 1) {
     dim3 cgrid(cdiv((long long)M * G, 4), Hkv);
