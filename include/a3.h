@@ -196,6 +196,13 @@ int a3_gather_rows(const a3_handle* h, const void* src, int n_src, const int32_t
  * Fills the fused cache in place, rows_out, scores_out, x_out. */
 int a3_fuse_request(const a3_handle* h, const a3_request* req, void* ws, size_t ws_bytes, a3_stream stream);
 
+/* Precomputation (Eq. 1, K_i, V_i = LLM(i)): prefills one chunk alone at local positions 0..T-1, i.e. runs every
+ * layer over all T rows, and leaves the chunk's per-layer caches in k_chunk / v_chunk (dev [n_layers][T][Hkv][D],
+ * layer l at + l*layer_stride bytes).  x_chunk: dev [T][d_model], embeddings in, final hidden state out.
+ * Called on the whole input X it is the full prefill without reuse.  ws >= a3_request_workspace_bytes(T). */
+int a3_precompute_chunk(const a3_handle* h, void* x_chunk, int T, void* k_chunk, void* v_chunk, uint64_t layer_stride,
+                        void* ws, size_t ws_bytes, a3_stream stream);
+
 /* Several independent requests on one stream (batched serving). */
 int a3_fuse_batch(const a3_handle* h, const a3_request* reqs, int n_requests, void* ws, size_t ws_bytes,
                   a3_stream stream);

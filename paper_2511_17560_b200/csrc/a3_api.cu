@@ -422,6 +422,26 @@ static int a3::fuse_impl(const a3_handle* h, const a3_request* r, void* ws, size
   return A3_OK;
 }
 
+extern "C" int a3_precompute_chunk(const a3_handle* h, void* x_chunk, int T, void* k_chunk, void* v_chunk,
+                                   uint64_t layer_stride, void* ws, size_t ws_bytes, a3_stream stream) {
+  if (!h || T < 0) return A3_EINVAL;
+  if (T == 0) return A3_OK;
+  if (!x_chunk || !k_chunk || !v_chunk || !ws) return A3_EINVAL;
+  const a3_model_desc& m = h->m;
+  if (T > m.max_positions) return A3_EINVAL;
+  if (layer_stride < (uint64_t)T * m.n_kv_heads * m.head_dim * 2 || (layer_stride & 15)) return A3_EINVAL;
+  if (((uintptr_t)x_chunk | (uintptr_t)k_chunk | (uintptr_t)v_chunk | (uintptr_t)ws) & 15) return A3_EINVAL;
+  RequestWs w = carve_request_ws(h, T, ws);
+  if (w.bytes > ws_bytes) return A3_EWORKSPACE;
+  LayerWs lw = carve_layer_ws(h, T, w.layer);
+  cudaStream_t st = (cudaStream_t)stream;
+  A3_TRY(iota_rows(h, w.all_pos, 0, T, st));
+  for (int l = 0; l < m.n_layers; ++l)
+    A3_TRY(recompute_layer_impl(h, l, (bf16*)x_chunk, w.all_pos, T, (bf16*)((char*)k_chunk + (size_t)l * layer_stride),
+                                (bf16*)((char*)v_chunk + (size_t)l * layer_stride), T, nullptr, lw, st));
+  return A3_OK;
+}
+
 extern "C" int a3_fuse_batch(const a3_handle* h, const a3_request* reqs, int n_requests, void* ws, size_t ws_bytes,
                              a3_stream stream) {
   if (!h || n_requests < 0 || (n_requests > 0 && !reqs)) return A3_EINVAL;

@@ -212,3 +212,27 @@ def test_fuse_request_rejects_bad_arguments(a3mod):
     assert lib.a3_fuse_request(None, None, None, 0, None) == -1
     torch.cuda.synchronize()
     s.eng.close()
+
+
+def test_precompute_chunk_matches_oracle_and_layer_loop(a3mod):
+    """Eq. 1 as one call: equals the loop over a3_recompute_layer bit for bit, and the oracle's prefill within the gates."""
+    s = Setup(a3mod, "tiny_gqa", emb_std=0.02, w_std=0.02)
+    m, r = s.m, s.r
+    T = 150
+    x = s.dx0[:T].clone()
+    K = torch.zeros((m.n_layers, T, m.n_kv_heads, m.head_dim), dtype=torch.bfloat16, device=s.dev)
+    V = torch.zeros_like(K)
+    s.eng.precompute_chunk(x, K, V)
+    assert s.eng.device_status() == 0
+    x2 = s.dx0[:T].clone()
+    K2, V2 = torch.zeros_like(K), torch.zeros_like(V)
+    pos = torch.arange(T, dtype=torch.int32, device=s.dev)
+    for l in range(m.n_layers):
+        s.eng.recompute_layer(l, x2, pos, K2[l], V2[l])
+    assert torch.equal(K, K2) and torch.equal(V, V2) and torch.equal(x, x2)
+    Ko, Vo = O.precompute_chunk(s.x0[:T], s.weights, s.model, rnd=O.round_bf16)
+    check_drift(f64(K)[0], Ko[0], "chunk K layer 0", KV_MEAN)
+    check_drift(f64(V)[0], Vo[0], "chunk V layer 0", KV_MEAN)
+    for l in range(1, m.n_layers):
+        check_drift(f64(K)[l], Ko[l], f"chunk K layer {l}", 2 * KV_MEAN)
+    s.eng.close()
