@@ -214,18 +214,23 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
   extern __shared__ unsigned char smem_raw[];
   const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   unsigned char* base_ptr = smem_raw + (base - smem_u32(smem_raw));
-  // barriers: kv_full[2], kv_empty[2], s_full[2], p_ready[2], q_ready, p_free[2]
+  // barriers: k_full[2], k_empty[2], v_full[2], v_empty[2], s_full[2], p_ready[2], q_ready, p_free[2].
+  // K and V have separate rings: a K stage is free as soon as its S = Q K^T has run, so the next K tile is on its
+  // way long before the P V of the same tile releases the V stage; with one barrier for both, every tile would
+  // wait for a full copy latency.
   const uint32_t bars = base + L::BAR_OFF;
-  auto kv_full = [&](int s) { return bars + 8u * s; };
-  auto kv_empty = [&](int s) { return bars + 8u * (2 + s); };
+  auto k_full = [&](int s) { return bars + 8u * s; };
+  auto k_empty = [&](int s) { return bars + 8u * (2 + s); };
+  auto v_full = [&](int s) { return bars + 8u * (11 + s); };
+  auto v_empty = [&](int s) { return bars + 8u * (13 + s); };
   auto s_full = [&](int b) { return bars + 8u * (4 + b); };
   // p_ready alternates between two barriers: a fast warp may finish tile t+1 before a slow warp has arrived for
   // tile t, and on a single barrier its second arrival would be counted towards tile t
   auto p_ready = [&](int b) { return bars + 8u * (6 + b); };
   const uint32_t q_ready = bars + 8u * 8;
   auto p_free = [&](int b) { return bars + 8u * (9 + b); };
-  volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(base_ptr + L::BAR_OFF + 8 * 11);
-  volatile int* abort_flag = reinterpret_cast<volatile int*>(base_ptr + L::BAR_OFF + 8 * 11 + 8);
+  volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(base_ptr + L::BAR_OFF + 8 * 15);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(base_ptr + L::BAR_OFF + 8 * 15 + 8);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int G = Hq / Hkv;
@@ -244,8 +249,10 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
 
   if (threadIdx.x == 0) {
     for (int i = 0; i < 2; ++i) {
-      mbar_init(kv_full(i), 1);
-      mbar_init(kv_empty(i), 1);
+      mbar_init(k_full(i), 1);
+      mbar_init(k_empty(i), 1);
+      mbar_init(v_full(i), 1);
+      mbar_init(v_empty(i), 1);
       mbar_init(s_full(i), 1);
       mbar_init(p_free(i), 1);
     }
@@ -280,14 +287,18 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
         if (!w.valid) continue;
         for (int kt = 0; kt < w.nkt; ++kt, ++it) {
           const int s = it & 1;
-          ok = mbar_wait(kv_empty(s), ((it >> 1) & 1) ^ 1, abort_flag, status);
-          if (!ok) break;
           const uint32_t sk = base + L::KV_OFF + s * L::KV_STAGE, sv = sk + (D / 64) * L::SUB;
-          mbar_expect_tx(kv_full(s), L::KV_STAGE);
+          ok = mbar_wait(k_empty(s), ((it >> 1) & 1) ^ 1, abort_flag, status);
+          if (!ok) break;
+          mbar_expect_tx(k_full(s), L::KV_STAGE / 2);
 #pragma unroll
-          for (int j = 0; j < D / 64; ++j) {
-            tma_load_2d(sk + j * L::SUB, &tmK, w.g * D + 64 * j, (w.kt0 + kt) * ATC_BN, kv_full(s));
-            tma_load_2d(sv + j * L::SUB, &tmV, w.g * D + 64 * j, (w.kt0 + kt) * ATC_BN, kv_full(s));
+          for (int j = 0; j < D / 64; ++j) tma_load_2d(sk + j * L::SUB, &tmK, w.g * D + 64 * j, (w.kt0 + kt) * ATC_BN, k_full(s));
+          if (want_o) {  // the statistics-only pass never reads V
+            ok = mbar_wait(v_empty(s), ((it >> 1) & 1) ^ 1, abort_flag, status);
+            if (!ok) break;
+            mbar_expect_tx(v_full(s), L::KV_STAGE / 2);
+#pragma unroll
+            for (int j = 0; j < D / 64; ++j) tma_load_2d(sv + j * L::SUB, &tmV, w.g * D + 64 * j, (w.kt0 + kt) * ATC_BN, v_full(s));
           }
         }
       }
@@ -306,6 +317,7 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
           mma_f16(tmem_s0 + (t & 1) * 128, desc_k_sw128(sq + sub), desc_k_sw128(sk + sub), idesc_s, k != 0);
         }
         commit(s_full(t & 1));
+        commit(k_empty(t & 1));  // the K stage is free once these MMAs have read it
       };
       uint32_t it = 0, qn = 0;
       bool ok = true;
@@ -316,19 +328,23 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
         if (!w.valid || w.nkt == 0) continue;
         ok = mbar_wait(q_ready, qn & 1, abort_flag, status);
         ++qn;
-        ok = ok && mbar_wait(kv_full(it & 1), (it >> 1) & 1, abort_flag, status);
+        ok = ok && mbar_wait(k_full(it & 1), (it >> 1) & 1, abort_flag, status);
         if (!ok) break;
         fence_after();
         issue_s(it);
         for (int kt = 0; kt < w.nkt; ++kt, ++it) {
           if (kt + 1 < w.nkt) {
-            ok = mbar_wait(kv_full((it + 1) & 1), ((it + 1) >> 1) & 1, abort_flag, status);
+            ok = mbar_wait(k_full((it + 1) & 1), ((it + 1) >> 1) & 1, abort_flag, status);
             if (!ok) break;
             fence_after();
             issue_s(it + 1);
           }
           ok = mbar_wait(p_ready(it & 1), (it >> 1) & 1, abort_flag, status);
           if (!ok) break;
+          if (want_o) {
+            ok = mbar_wait(v_full(it & 1), (it >> 1) & 1, abort_flag, status);
+            if (!ok) break;
+          }
           fence_after();
           if (want_o) {
             const uint32_t sv = base + L::KV_OFF + (it & 1) * L::KV_STAGE + (D / 64) * L::SUB;
@@ -339,8 +355,8 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
               mma_f16(tmem_o, da, db, idesc_o, (kt | k) != 0);  // O accumulates over the item's key tiles in TMEM
             }
             commit(p_free(it & 1));  // P V of this tile is complete: its P buffer may be rewritten, O holds tiles 0..kt
+            commit(v_empty(it & 1));
           }
-          commit(kv_empty(it & 1));
         }
       }
     }
@@ -478,7 +494,7 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
           // slots beyond the row tile's last visible key may hold anything: they get probability zero, and zero
           // times a non-finite value would still poison the product, so clear those V rows of the last tile
           const int first_bad = w.maxpos - key0 + 1;
-          const bool landed = mbar_wait(kv_full(it & 1), (it >> 1) & 1, abort_flag, status);  // already complete: S of this tile was computed
+          const bool landed = mbar_wait(v_full(it & 1), (it >> 1) & 1, abort_flag, status);  // the V tile must have landed before rows of it are cleared
           if (landed && row >= first_bad) {
             unsigned char* sv = base_ptr + L::KV_OFF + (it & 1) * L::KV_STAGE + (D / 64) * L::SUB;
 #pragma unroll
@@ -602,6 +618,7 @@ static int make_cache_tmap(CUtensorMap* map, const void* ptr, long long rows, lo
   return A3_OK;
 }
 
+int g_attn_max_ctas = 0;  // tuning: cap on the persistent grid
 int g_attn_split = 0;  // 0: choose; otherwise the number of key segments (tuning)
 
 size_t attention_part_bytes(const a3_handle* h) {
@@ -633,7 +650,8 @@ int attention_rows(const a3_handle* h, const bf16* q, const int32_t* pos, int M,
   n_split = cdiv(all_tiles, tiles_per_split);
   const int rows_pad = (int)grid.x * ATC_BM;
   const int n_items = (int)grid.x * Hkv * n_split;
-  const int n_ctas = n_items < sms ? n_items : sms;  // persistent: at most one CTA per SM
+  int n_ctas = n_items < sms ? n_items : sms;  // persistent: at most one CTA per SM
+  if (g_attn_max_ctas > 0 && n_ctas > g_attn_max_ctas) n_ctas = g_attn_max_ctas;
   float* part_o = (float*)part;
   float2* part_ml = part ? (float2*)(part_o + (size_t)n_split * Hkv * rows_pad * D) : nullptr;
   static bool attr_set = false;
@@ -660,3 +678,4 @@ int attention_rows(const a3_handle* h, const bf16* q, const int32_t* pos, int M,
 }  // namespace a3
 
 extern "C" void a3_internal_set_attn_split(int v) { a3::g_attn_split = v; }
+extern "C" void a3_internal_set_attn_max_ctas(int v) { a3::g_attn_max_ctas = v; }
