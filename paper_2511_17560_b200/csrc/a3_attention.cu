@@ -10,10 +10,12 @@
 //                       probabilities of a tile are in shared memory, O~ = P V (128 x D x 128, V as an MN-major
 //                       operand) accumulated into a third TMEM buffer.  S of tile t+1 is issued before P V of tile t, so the
 //                       tensor core works while the softmax threads do.
-//   warps 2..5          one thread per row: one pass over the row of S in TMEM (exp2 against a lazily raised
-//                       reference maximum, row sum), P written as bf16 into shared memory in the swizzled K-major
-//                       layout the MMA reads; the output accumulates in TMEM across key tiles and is rescaled there
-//                       only when the reference has to be raised; final normalisation and stores.
+//   warps 2..9          two threads per row, each owning half of the tile's key columns: one pass over the row of
+//                       S in TMEM (exp2 against a lazily raised reference maximum, row sum), P written as bf16
+//                       into shared memory in the swizzled K-major layout the MMA reads; the output accumulates in
+//                       TMEM across key tiles and is rescaled there only when the reference has to be raised; final
+//                       normalisation and stores.  The softmax warps are the bottleneck of the kernel (measured by
+//                       ablation), hence two warps per scheduler.
 // Statistics are fp32 in the exp2 domain.  Every mbarrier wait is bounded (see a3_gemm.cu); there is no block-
 // wide or named barrier inside the loops, so a role that gives up cannot strand another.
 #include <cuda.h>
@@ -22,7 +24,7 @@
 
 namespace a3 {
 
-constexpr int ATC_THREADS = 192;
+constexpr int ATC_THREADS = 320;  // TMA warp, MMA warp, 8 softmax warps (two threads per row)
 constexpr int ATC_BM = 128, ATC_BN = 128;
 constexpr unsigned long long ATC_WAIT_NS = 500000000ull;
 constexpr float ATC_LOG2E = 1.4426950408889634f, ATC_LN2 = 0.6931471805599453f;
@@ -163,7 +165,8 @@ struct AtcLayout {
   static constexpr int KV_OFF = Q_BYTES;
   static constexpr int P_OFF = KV_OFF + 2 * KV_STAGE;
   static constexpr int BAR_OFF = P_OFF + 2 * P_BYTES;
-  static constexpr int SMEM_BYTES = BAR_OFF + 256 + 1024;
+  static constexpr int XCH_OFF = BAR_OFF + 256;          // float2 exchange[2 halves][128 rows]
+  static constexpr int SMEM_BYTES = XCH_OFF + 2048;      // the dynamic shared window must be 1024-byte aligned (checked)
 };
 
 // One unit of work: a 128-row tile of one KV head and one segment of its key tiles.
@@ -212,8 +215,12 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
   using L = AtcLayout<D>;
   using namespace atc;
   extern __shared__ unsigned char smem_raw[];
-  const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
-  unsigned char* base_ptr = smem_raw + (base - smem_u32(smem_raw));
+  const uint32_t base = smem_u32(smem_raw);
+  unsigned char* base_ptr = smem_raw;
+  if (base & 1023u) {  // the swizzled tiles need a 1024-byte aligned window; uniform for the CTA, nothing is set up yet
+    if (threadIdx.x == 0) atomicOr(status, A3_DEV_WAIT_EXHAUSTED);
+    return;
+  }
   // barriers: k_full[2], k_empty[2], v_full[2], v_empty[2], s_full[2], p_ready[2], q_ready, p_free[2].
   // K and V have separate rings: a K stage is free as soon as its S = Q K^T has run, so the next K tile is on its
   // way long before the P V of the same tile releases the V stage; with one barrier for both, every tile would
@@ -229,8 +236,11 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
   auto p_ready = [&](int b) { return bars + 8u * (6 + b); };
   const uint32_t q_ready = bars + 8u * 8;
   auto p_free = [&](int b) { return bars + 8u * (9 + b); };
-  volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(base_ptr + L::BAR_OFF + 8 * 15);
-  volatile int* abort_flag = reinterpret_cast<volatile int*>(base_ptr + L::BAR_OFF + 8 * 15 + 8);
+  // pair[q][parity]: the two warps that share TMEM lane quarter q (64 threads) meet here to exchange row statistics
+  auto pair_bar = [&](int qd, int par) { return bars + 8u * (15 + qd * 2 + par); };
+  volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(base_ptr + L::BAR_OFF + 8 * 23);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(base_ptr + L::BAR_OFF + 8 * 23 + 8);
+  float2* xch = reinterpret_cast<float2*>(base_ptr + L::XCH_OFF);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int G = Hq / Hkv;
@@ -256,9 +266,10 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
       mbar_init(s_full(i), 1);
       mbar_init(p_free(i), 1);
     }
-    mbar_init(p_ready(0), 128);
-    mbar_init(p_ready(1), 128);
-    mbar_init(q_ready, 128);
+    mbar_init(p_ready(0), 256);
+    mbar_init(p_ready(1), 256);
+    mbar_init(q_ready, 256);
+    for (int i = 0; i < 8; ++i) mbar_init(pair_bar(i >> 1, i & 1), 64);
     abort_flag[0] = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     fence_async_smem();
@@ -352,7 +363,8 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
             for (int k = 0; k < ATC_BN / 16; ++k) {
               const uint64_t da = desc_k_sw128(sp + (it & 1) * L::P_BYTES + (k / 4) * L::SUB + (k % 4) * 32);
               const uint64_t db = desc_mn_sw128(sv + k * 16 * 128, L::SUB);
-              mma_f16(tmem_o, da, db, idesc_o, (kt | k) != 0);  // O accumulates over the item's key tiles in TMEM
+              // each half of the tile's keys accumulates into an output of its own (see the softmax warps)
+              mma_f16(tmem_o + (k / 4) * D, da, db, idesc_o, (kt | (k % 4)) != 0);
             }
             commit(p_free(it & 1));  // P V of this tile is complete: its P buffer may be rewritten, O holds tiles 0..kt
             commit(v_empty(it & 1));
@@ -361,13 +373,32 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
       }
     }
   } else {
-    // ---------------- softmax / epilogue: thread = row
+    // ---------------- softmax / epilogue: two threads per row.  Thread `half` of a row owns keys 64*half .. +63 of
+    // every key tile, with an exponent reference, a row sum and an output accumulator in TMEM of its own, so the
+    // two never have to agree on anything while the keys stream; they meet once per item (warps w and w+4 share a
+    // TMEM lane quarter, a 64-thread mbarrier and an exchange slot in shared memory) to merge the two partial
+    // softmaxes, and each then normalises and stores half of the output columns.
+    const int half = (warp - 2) >> 2;
     const int quarter = warp & 3;
     const int row = quarter * 32 + lane;
     const uint32_t lane_addr = (uint32_t)(quarter * 32) << 16;
+    const uint32_t tmem_oh = tmem_o + half * D;  // this thread's accumulator
     constexpr float RESCALE_TH = 8.f;
-    uint32_t it = 0;
+    uint32_t it = 0, px = 0;  // running key tile; running count of pair exchanges (parity of the pair barrier)
     bool ok = true;
+    // publish `mine`, meet the partner, return the partner's value; false if the wait was abandoned
+    auto exchange = [&](float2 mine, float2& theirs) {
+      // One slot per thread is enough: a thread overwrites its slot at the end of the next item, after that item's
+      // first S tile, which the MMA warp issues only once all 256 threads have arrived at q_ready - and the
+      // partner arrives there after it has read this slot.
+      const int par = px & 1;
+      xch[half * 128 + row] = mine;
+      mbar_arrive(pair_bar(quarter, par));
+      const bool got = __all_sync(0xffffffffu, mbar_wait(pair_bar(quarter, par), (px >> 1) & 1, abort_flag, status));
+      theirs = xch[(half ^ 1) * 128 + row];
+      ++px;
+      return got;
+    };
 
     for (int r = 0; r < rounds && ok; ++r) {
       const int i = item_index(r);
@@ -384,21 +415,22 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
       if (w.nkt == 0) {
         // no visible key at all (only with invalid positions): defined output, no pipeline work
         if (row_ok && want_o && !w.partial) {
-          uint4* dst = reinterpret_cast<uint4*>(o + ((size_t)tok * Hq + hq) * D);
+          uint4* dst = reinterpret_cast<uint4*>(o + ((size_t)tok * Hq + hq) * D + half * (D / 2));
 #pragma unroll
-          for (int c = 0; c < D / 8; ++c) dst[c] = make_uint4(0, 0, 0, 0);
+          for (int c = 0; c < D / 16; ++c) dst[c] = make_uint4(0, 0, 0, 0);
         }
-        if (row_ok && w.partial) part_ml[prow] = make_float2(0.f, 0.f);
-        if (row_ok && !w.partial && lse) lse[(size_t)tok * Hq + hq] = -INFINITY;
+        if (row_ok && w.partial && half == 0) part_ml[prow] = make_float2(0.f, 0.f);
+        if (row_ok && !w.partial && lse && half == 0) lse[(size_t)tok * Hq + hq] = -INFINITY;
         continue;
       }
 
-      // Q row -> shared memory, swizzled K-major sub-tiles.  The previous item's S MMAs have all completed (their
-      // last s_full was waited for), so the Q buffer is free.
+      // Q row -> shared memory, swizzled K-major sub-tiles (each thread copies half of the row's 16-byte chunks).
+      // The previous item's S MMAs have all completed (their last s_full was waited for), so the Q buffer is free.
       {
         const uint4* src = reinterpret_cast<const uint4*>(q + ((size_t)tok * Hq + hq) * D);
 #pragma unroll
-        for (int c = 0; c < D / 8; ++c) {
+        for (int cc = 0; cc < D / 16; ++cc) {
+          const int c = half * (D / 16) + cc;
           uint4 v = row_ok ? __ldg(src + c) : make_uint4(0, 0, 0, 0);
           *reinterpret_cast<uint4*>(base_ptr + L::Q_OFF + (c / 8) * L::SUB + swz(row, c % 8)) = v;
         }
@@ -406,9 +438,9 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
         mbar_arrive(q_ready);
       }
 
-      // Exponent reference m_ref and row sum l_run relative to it.  The reference is the true maximum of the first
-      // tile and is raised later only when a logit exceeds it by more than 2^RESCALE_TH (rare once the first tiles
-      // are seen): then the output accumulated in TMEM and l_run are rescaled and the tile is redone.
+      // Exponent reference m_ref and row sum l_run of this thread's keys.
+      // The reference is the true maximum of the first tile and is raised later only when a logit exceeds it by
+      // more than RESCALE_TH (rare): then the output accumulated in TMEM and l_run are rescaled and the tile redone.
       float m_ref = 0.f, l_run = 0.f;
       uint32_t it_last = it;
       for (int kt = 0; kt < w.nkt; ++kt, ++it) {
@@ -417,13 +449,13 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
         ok = __all_sync(0xffffffffu, mbar_wait(s_full(it & 1), (it >> 1) & 1, abort_flag, status));
         if (!ok) break;
         fence_after();
-        const uint32_t ts = tmem_s0 + (it & 1) * 128 + lane_addr;
-        const int key0 = (w.kt0 + kt) * ATC_BN;
-        const bool need_mask = key0 + ATC_BN - 1 > w.minpos;
+        const uint32_t ts = tmem_s0 + (it & 1) * 128 + lane_addr + half * 64;
+        const int key0 = (w.kt0 + kt) * ATC_BN + half * 64;  // first key of this thread's columns
+        const bool need_mask = (w.kt0 + kt) * ATC_BN + ATC_BN - 1 > w.minpos;
         if (kt == 0) {
           float mx = -INFINITY;
 #pragma unroll 1
-          for (int c = 0; c < 4; ++c) {
+          for (int c = 0; c < 2; ++c) {
             float sv[32];
             ld32(ts + c * 32, sv);
             wait_ld();
@@ -449,16 +481,17 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
           float buf[2][32];
           ld32(ts, buf[0]);
 #pragma unroll
-          for (int c = 0; c < 4; ++c) {
+          for (int c = 0; c < 2; ++c) {
             wait_ld();
-            if (c < 3) ld32(ts + (c + 1) * 32, buf[(c + 1) & 1]);
+            if (c < 1) ld32(ts + (c + 1) * 32, buf[(c + 1) & 1]);
             float* sv = buf[c & 1];
             if (need_mask) softmax_chunk<true>(sv, key0 + c * 32, lim, scale_log2, neg_ref, mx, ls);
             else softmax_chunk<false>(sv, key0 + c * 32, lim, scale_log2, neg_ref, mx, ls);
             if (want_o) {
+              // this thread's 64 keys are sub-tile `half` of the P buffer
 #pragma unroll
               for (int j = 0; j < 4; ++j)
-                *reinterpret_cast<uint4*>(base_ptr + L::P_OFF + (it & 1) * L::P_BYTES + (c >> 1) * L::SUB + swz(row, (c & 1) * 4 + j)) = pack8(sv + 8 * j);
+                *reinterpret_cast<uint4*>(base_ptr + L::P_OFF + (it & 1) * L::P_BYTES + half * L::SUB + swz(row, c * 4 + j)) = pack8(sv + 8 * j);
             }
           }
           const float lsum = (ls[0] + ls[1]) + (ls[2] + ls[3]);
@@ -480,20 +513,22 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
 #pragma unroll 1
             for (int c = 0; c < D / 32; ++c) {
               float t[32];
-              ld32(tmem_o + lane_addr + c * 32, t);
+              const uint32_t to = tmem_oh + lane_addr + c * 32;
+              ld32(to, t);
               wait_ld();
 #pragma unroll
               for (int e = 0; e < 32; ++e) t[e] *= f;
-              st32(tmem_o + lane_addr + c * 32, t);
+              st32(to, t);
             }
             wait_st();
           }
         }
         if (!ok) break;
-        if (want_o && w.kt0 + kt == w.nkt_all - 1) {
+        if (want_o && w.kt0 + kt == w.nkt_all - 1 && half == 0) {
           // slots beyond the row tile's last visible key may hold anything: they get probability zero, and zero
           // times a non-finite value would still poison the product, so clear those V rows of the last tile
-          const int first_bad = w.maxpos - key0 + 1;
+          // (thread `row` of the first half clears key `row`)
+          const int first_bad = w.maxpos - (w.kt0 + kt) * ATC_BN + 1;
           const bool landed = mbar_wait(v_full(it & 1), (it >> 1) & 1, abort_flag, status);  // the V tile must have landed before rows of it are cleared
           if (landed && row >= first_bad) {
             unsigned char* sv = base_ptr + L::KV_OFF + (it & 1) * L::KV_STAGE + (D / 64) * L::SUB;
@@ -508,35 +543,54 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
         mbar_arrive(p_ready(it & 1));
       }
       if (!ok) break;
+      // merge the two partial softmaxes of the row: common reference m, weights f_mine / f_other for the two
+      // accumulators, row sum l (a half that saw no visible key has l == 0 and no say in the reference)
+      float f_mine, f_other;
+      {
+        float2 other;
+        ok = exchange(make_float2(m_ref, l_run), other);
+        if (!ok) break;
+        const float m_a = l_run > 0.f ? m_ref : -INFINITY, m_b = other.y > 0.f ? other.x : -INFINITY;
+        const float m = fmaxf(m_a, m_b);
+        f_mine = l_run > 0.f ? exp2f(m_a - m) : 0.f;
+        f_other = other.y > 0.f ? exp2f(m_b - m) : 0.f;
+        const float l0 = half == 0 ? l_run * f_mine : other.y * f_other, l1 = half == 0 ? other.y * f_other : l_run * f_mine;
+        l_run = l0 + l1;  // same order in both threads
+        m_ref = m == -INFINITY ? 0.f : m;
+      }
       const float inv = l_run > 0.f ? 1.f / l_run : 0.f;
       if (want_o) {
         ok = __all_sync(0xffffffffu, mbar_wait(p_free(it_last & 1), (it_last >> 1) & 1, abort_flag, status));
         if (!ok) break;
         fence_after();
-        bf16* dst = o + ((size_t)tok * Hq + hq) * D;
+        bf16* dst = o + ((size_t)tok * Hq + hq) * D + half * (D / 2);
+        const float fa = (half == 0 ? f_mine : f_other) * (w.partial ? 1.f : inv), fb = (half == 0 ? f_other : f_mine) * (w.partial ? 1.f : inv);
 #pragma unroll 1
-        for (int c = 0; c < D / 32; ++c) {
-          float t[32];
-          ld32(tmem_o + lane_addr + c * 32, t);
+        for (int c = 0; c < D / 64; ++c) {  // this thread's half of the output columns, from both accumulators
+          float t[32], u[32];
+          ld32(tmem_o + lane_addr + half * (D / 2) + c * 32, t);
+          ld32(tmem_o + D + lane_addr + half * (D / 2) + c * 32, u);
           wait_ld();
+#pragma unroll
+          for (int e = 0; e < 32; ++e) t[e] = fmaf(t[e], fa, u[e] * fb);
           if (row_ok && w.partial) {
-            float4* pd = reinterpret_cast<float4*>(part_o + prow * D + c * 32);
+            float4* pd = reinterpret_cast<float4*>(part_o + prow * D + half * (D / 2) + c * 32);
 #pragma unroll
             for (int j = 0; j < 8; ++j) pd[j] = make_float4(t[4 * j], t[4 * j + 1], t[4 * j + 2], t[4 * j + 3]);
           } else if (row_ok) {
-#pragma unroll
-            for (int e = 0; e < 32; ++e) t[e] *= inv;
 #pragma unroll
             for (int j = 0; j < 4; ++j) reinterpret_cast<uint4*>(dst + c * 32)[j] = pack8(t + 8 * j);
           }
           __syncwarp();
         }
-        // the next item's first P V overwrites O: it is issued only after this item's p_ready arrivals of all 128
+        // the next item's first P V overwrites O: it is issued only after this item's p_ready arrivals of all 256
         // threads for that tile, which each thread makes after the loads above
         fence_before();
       }
-      if (row_ok && w.partial) part_ml[prow] = make_float2(m_ref, l_run);
-      if (row_ok && !w.partial && lse) lse[(size_t)tok * Hq + hq] = l_run > 0.f ? (m_ref + log2f(l_run)) * ATC_LN2 : -INFINITY;
+      if (half == 0) {
+        if (row_ok && w.partial) part_ml[prow] = make_float2(m_ref, l_run);
+        if (row_ok && !w.partial && lse) lse[(size_t)tok * Hq + hq] = l_run > 0.f ? (m_ref + log2f(l_run)) * ATC_LN2 : -INFINITY;
+      }
     }
   }
   atc::fence_before();
