@@ -5,17 +5,19 @@
 // one KV head and walks the keys in tiles of 128 up to the largest position among its rows.
 //
 //   warp 0 (one lane)   TMA producer: K and V tiles of the cache ([slots][Hkv*D] seen as a 2-D tensor, 128-byte
-//                       swizzle, two stages).
+//                       swizzle), a ring of three stages each.
 //   warp 1 (one lane)   tcgen05.mma issuer: S = Q K^T (128 x 128 x D) into one of two TMEM buffers, and, once the
-//                       probabilities of a tile are in shared memory, O~ = P V (128 x D x 128, V as an MN-major
-//                       operand) accumulated into a third TMEM buffer.  S of tile t+1 is issued before P V of tile t, so the
-//                       tensor core works while the softmax threads do.
-//   warps 2..9          two threads per row, each owning half of the tile's key columns: one pass over the row of
-//                       S in TMEM (exp2 against a lazily raised reference maximum, row sum), P written as bf16
-//                       into shared memory in the swizzled K-major layout the MMA reads; the output accumulates in
-//                       TMEM across key tiles and is rescaled there only when the reference has to be raised; final
-//                       normalisation and stores.  The softmax warps are the bottleneck of the kernel (measured by
-//                       ablation), hence two warps per scheduler.
+//                       probabilities of a tile are back in tensor memory, O~ += P V (128 x D x 128; P is the A
+//                       operand read from TMEM, V an MN-major operand in shared memory) accumulated in TMEM.
+//                       S of tile t+1 is issued before P V of tile t, so the tensor core works while the
+//                       softmax threads do.
+//   warps 2..9          two threads per row, each owning half of the tile's key columns with an exponent
+//                       reference, a row sum and a TMEM output accumulator of its own: the row of S is read into
+//                       registers, its maximum checked against the lazily raised reference (the accumulator is
+//                       rescaled in TMEM only when the reference moves), P = exp2(s - ref) is written as bf16
+//                       pairs over the columns S came from; at the end of an item the two partial softmaxes of a
+//                       row are merged, normalised and stored.
+// TMEM (512 columns): S buffers at 0 and 128, the two output accumulators at 256 and 256 + D.
 // Statistics are fp32 in the exp2 domain.  Every mbarrier wait is bounded (see a3_gemm.cu); there is no block-
 // wide or named barrier inside the loops, so a role that gives up cannot strand another.
 #include <cuda.h>
@@ -89,6 +91,15 @@ __device__ __forceinline__ void mma_f16(uint32_t d_tmem, uint64_t a_desc, uint64
       ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
       : "memory");
 }
+// same, A operand read from tensor memory (128 lanes x k, two bf16 per 32-bit column)
+__device__ __forceinline__ void mma_f16_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}"
+      ::"r"(d_tmem), "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
 __device__ __forceinline__ void ld32(uint32_t taddr, float* v) {
   uint32_t* r = reinterpret_cast<uint32_t*>(v);
   asm volatile(
@@ -138,33 +149,15 @@ __device__ __forceinline__ float ex2_approx(float x) {
   asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
   return y;
 }
-// 32 logits of one row -> probabilities (in place), running relative maximum and four partial row sums.
-// t = s * scale - m_ref is one FMA; ex2.approx maps -inf to +0, so masked keys need no second select.
-template <bool MASK>
-__device__ __forceinline__ void softmax_chunk(float* sv, int key_base, int lim, float scale, float neg_ref, float& mx, float (&ls)[4]) {
-  float m4[4] = {mx, mx, mx, mx};  // four independent chains for the maximum, like the row sum
-#pragma unroll
-  for (int e = 0; e < 32; ++e) {
-    float t = fmaf(sv[e], scale, neg_ref);
-    if (MASK && key_base + e > lim) t = -INFINITY;
-    m4[e & 3] = fmaxf(m4[e & 3], t);
-    const float pe = ex2_approx(t);
-    sv[e] = pe;
-    ls[e & 3] += pe;
-  }
-  mx = fmaxf(fmaxf(m4[0], m4[1]), fmaxf(m4[2], m4[3]));
-}
-
 template <int D>
 struct AtcLayout {
   static constexpr int SUB = 128 * 64 * 2;           // one [128][64] bf16 sub-tile: 16 KiB
   static constexpr int Q_BYTES = (D / 64) * SUB;
   static constexpr int KV_STAGE = 2 * (D / 64) * SUB;  // K then V
-  static constexpr int P_BYTES = 2 * SUB;                // one P buffer; two of them alternate
+  static constexpr int KV_STAGES = 3;
   static constexpr int Q_OFF = 0;
   static constexpr int KV_OFF = Q_BYTES;
-  static constexpr int P_OFF = KV_OFF + 2 * KV_STAGE;
-  static constexpr int BAR_OFF = P_OFF + 2 * P_BYTES;
+  static constexpr int BAR_OFF = KV_OFF + KV_STAGES * KV_STAGE;
   static constexpr int XCH_OFF = BAR_OFF + 256;          // float2 exchange[2 halves][128 rows]
   static constexpr int SMEM_BYTES = XCH_OFF + 2048;      // the dynamic shared window must be 1024-byte aligned (checked)
 };
@@ -227,19 +220,19 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
   // wait for a full copy latency.
   const uint32_t bars = base + L::BAR_OFF;
   auto k_full = [&](int s) { return bars + 8u * s; };
-  auto k_empty = [&](int s) { return bars + 8u * (2 + s); };
-  auto v_full = [&](int s) { return bars + 8u * (11 + s); };
-  auto v_empty = [&](int s) { return bars + 8u * (13 + s); };
-  auto s_full = [&](int b) { return bars + 8u * (4 + b); };
+  auto k_empty = [&](int s) { return bars + 8u * (3 + s); };
+  auto v_full = [&](int s) { return bars + 8u * (6 + s); };
+  auto v_empty = [&](int s) { return bars + 8u * (9 + s); };
+  auto s_full = [&](int b) { return bars + 8u * (12 + b); };
   // p_ready alternates between two barriers: a fast warp may finish tile t+1 before a slow warp has arrived for
   // tile t, and on a single barrier its second arrival would be counted towards tile t
-  auto p_ready = [&](int b) { return bars + 8u * (6 + b); };
-  const uint32_t q_ready = bars + 8u * 8;
-  auto p_free = [&](int b) { return bars + 8u * (9 + b); };
+  auto p_ready = [&](int b) { return bars + 8u * (14 + b); };
+  const uint32_t q_ready = bars + 8u * 16;
+  auto p_free = [&](int b) { return bars + 8u * (17 + b); };
   // pair[q][parity]: the two warps that share TMEM lane quarter q (64 threads) meet here to exchange row statistics
-  auto pair_bar = [&](int qd, int par) { return bars + 8u * (15 + qd * 2 + par); };
-  volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(base_ptr + L::BAR_OFF + 8 * 23);
-  volatile int* abort_flag = reinterpret_cast<volatile int*>(base_ptr + L::BAR_OFF + 8 * 23 + 8);
+  auto pair_bar = [&](int qd, int par) { return bars + 8u * (19 + qd * 2 + par); };
+  volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(base_ptr + L::BAR_OFF + 8 * 27);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(base_ptr + L::BAR_OFF + 8 * 27 + 8);
   float2* xch = reinterpret_cast<float2*>(base_ptr + L::XCH_OFF);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -258,11 +251,13 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
   const int rounds = (n_items + C - 1) / C;
 
   if (threadIdx.x == 0) {
-    for (int i = 0; i < 2; ++i) {
+    for (int i = 0; i < L::KV_STAGES; ++i) {
       mbar_init(k_full(i), 1);
       mbar_init(k_empty(i), 1);
       mbar_init(v_full(i), 1);
       mbar_init(v_empty(i), 1);
+    }
+    for (int i = 0; i < 2; ++i) {
       mbar_init(s_full(i), 1);
       mbar_init(p_free(i), 1);
     }
@@ -297,15 +292,16 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
         const AtcItem w = atc_item(i, pos, M, G, Hkv, kv_len, row_tiles, n_split, tiles_per_split);
         if (!w.valid) continue;
         for (int kt = 0; kt < w.nkt; ++kt, ++it) {
-          const int s = it & 1;
+          const int s = it % L::KV_STAGES;
+          const uint32_t ph = (it / L::KV_STAGES) & 1;
           const uint32_t sk = base + L::KV_OFF + s * L::KV_STAGE, sv = sk + (D / 64) * L::SUB;
-          ok = mbar_wait(k_empty(s), ((it >> 1) & 1) ^ 1, abort_flag, status);
+          ok = mbar_wait(k_empty(s), ph ^ 1, abort_flag, status);
           if (!ok) break;
           mbar_expect_tx(k_full(s), L::KV_STAGE / 2);
 #pragma unroll
           for (int j = 0; j < D / 64; ++j) tma_load_2d(sk + j * L::SUB, &tmK, w.g * D + 64 * j, (w.kt0 + kt) * ATC_BN, k_full(s));
           if (want_o) {  // the statistics-only pass never reads V
-            ok = mbar_wait(v_empty(s), ((it >> 1) & 1) ^ 1, abort_flag, status);
+            ok = mbar_wait(v_empty(s), ph ^ 1, abort_flag, status);
             if (!ok) break;
             mbar_expect_tx(v_full(s), L::KV_STAGE / 2);
 #pragma unroll
@@ -319,16 +315,16 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
     if (lane == 0) {
       constexpr uint32_t idesc_s = idesc(ATC_BN, 0);
       constexpr uint32_t idesc_o = idesc(D, 1);
-      const uint32_t sq = base + L::Q_OFF, sp = base + L::P_OFF;
-      auto issue_s = [&](uint32_t t) {  // S of running key tile t into S buffer t & 1, from K stage t & 1
-        const uint32_t sk = base + L::KV_OFF + (t & 1) * L::KV_STAGE;
+      const uint32_t sq = base + L::Q_OFF;
+      auto issue_s = [&](uint32_t t) {  // S of running key tile t into S buffer t & 1, from K stage t mod 3
+        const uint32_t sk = base + L::KV_OFF + (t % L::KV_STAGES) * L::KV_STAGE;
 #pragma unroll
         for (int k = 0; k < D / 16; ++k) {
           const uint32_t sub = (k / 4) * L::SUB + (k % 4) * 32;
           mma_f16(tmem_s0 + (t & 1) * 128, desc_k_sw128(sq + sub), desc_k_sw128(sk + sub), idesc_s, k != 0);
         }
         commit(s_full(t & 1));
-        commit(k_empty(t & 1));  // the K stage is free once these MMAs have read it
+        commit(k_empty(t % L::KV_STAGES));  // the K stage is free once these MMAs have read it
       };
       uint32_t it = 0, qn = 0;
       bool ok = true;
@@ -339,13 +335,13 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
         if (!w.valid || w.nkt == 0) continue;
         ok = mbar_wait(q_ready, qn & 1, abort_flag, status);
         ++qn;
-        ok = ok && mbar_wait(k_full(it & 1), (it >> 1) & 1, abort_flag, status);
+        ok = ok && mbar_wait(k_full(it % L::KV_STAGES), (it / L::KV_STAGES) & 1, abort_flag, status);
         if (!ok) break;
         fence_after();
         issue_s(it);
         for (int kt = 0; kt < w.nkt; ++kt, ++it) {
           if (kt + 1 < w.nkt) {
-            ok = mbar_wait(k_full((it + 1) & 1), ((it + 1) >> 1) & 1, abort_flag, status);
+            ok = mbar_wait(k_full((it + 1) % L::KV_STAGES), ((it + 1) / L::KV_STAGES) & 1, abort_flag, status);
             if (!ok) break;
             fence_after();
             issue_s(it + 1);
@@ -353,21 +349,24 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
           ok = mbar_wait(p_ready(it & 1), (it >> 1) & 1, abort_flag, status);
           if (!ok) break;
           if (want_o) {
-            ok = mbar_wait(v_full(it & 1), (it >> 1) & 1, abort_flag, status);
+            ok = mbar_wait(v_full(it % L::KV_STAGES), (it / L::KV_STAGES) & 1, abort_flag, status);
             if (!ok) break;
           }
           fence_after();
           if (want_o) {
-            const uint32_t sv = base + L::KV_OFF + (it & 1) * L::KV_STAGE + (D / 64) * L::SUB;
+            const uint32_t sv = base + L::KV_OFF + (it % L::KV_STAGES) * L::KV_STAGE + (D / 64) * L::SUB;
+            // P of this tile lies over the first half of each thread's S columns (see the softmax warps): keys
+            // 64 h + 16 kk .. + 15 in the eight 32-bit columns at 64 h + 8 kk of S buffer it & 1.  The next S into
+            // that buffer is issued after these MMAs and the tensor pipe runs in order.
+            const uint32_t tp = tmem_s0 + (it & 1) * 128;
 #pragma unroll
             for (int k = 0; k < ATC_BN / 16; ++k) {
-              const uint64_t da = desc_k_sw128(sp + (it & 1) * L::P_BYTES + (k / 4) * L::SUB + (k % 4) * 32);
               const uint64_t db = desc_mn_sw128(sv + k * 16 * 128, L::SUB);
               // each half of the tile's keys accumulates into an output of its own (see the softmax warps)
-              mma_f16(tmem_o + (k / 4) * D, da, db, idesc_o, (kt | (k % 4)) != 0);
+              mma_f16_ts(tmem_o + (k / 4) * D, tp + (k / 4) * 64 + (k % 4) * 8, db, idesc_o, (kt | (k % 4)) != 0);
             }
-            commit(p_free(it & 1));  // P V of this tile is complete: its P buffer may be rewritten, O holds tiles 0..kt
-            commit(v_empty(it & 1));
+            commit(p_free(it & 1));  // P V of this tile is complete: the outputs hold tiles 0..kt
+            commit(v_empty(it % L::KV_STAGES));
           }
         }
       }
@@ -438,9 +437,9 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
         mbar_arrive(q_ready);
       }
 
-      // Exponent reference m_ref and row sum l_run of this thread's keys.
-      // The reference is the true maximum of the first tile and is raised later only when a logit exceeds it by
-      // more than RESCALE_TH (rare): then the output accumulated in TMEM and l_run are rescaled and the tile redone.
+      // Exponent reference m_ref and row sum l_run of this thread's keys.  The reference is the true maximum of the
+      // first tile and is raised later only when a logit exceeds it by more than RESCALE_TH (rare): then the output
+      // accumulated in TMEM and l_run are rescaled first.
       float m_ref = 0.f, l_run = 0.f;
       uint32_t it_last = it;
       for (int kt = 0; kt < w.nkt; ++kt, ++it) {
@@ -452,61 +451,44 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
         const uint32_t ts = tmem_s0 + (it & 1) * 128 + lane_addr + half * 64;
         const int key0 = (w.kt0 + kt) * ATC_BN + half * 64;  // first key of this thread's columns
         const bool need_mask = (w.kt0 + kt) * ATC_BN + ATC_BN - 1 > w.minpos;
-        if (kt == 0) {
-          float mx = -INFINITY;
-#pragma unroll 1
-          for (int c = 0; c < 2; ++c) {
-            float sv[32];
-            ld32(ts + c * 32, sv);
-            wait_ld();
+        // pass 1: scaled (and masked) logits into registers, their maximum
+        float x[64];
+        ld32(ts, x);
+        ld32(ts + 32, x + 32);
+        wait_ld();
+        float mx;
+        {
+          float m4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
+          if (need_mask) {
 #pragma unroll
-            for (int e = 0; e < 32; ++e) {
-              float x = sv[e] * scale_log2;
-              if (need_mask && key0 + c * 32 + e > lim) x = -INFINITY;
-              mx = fmaxf(mx, x);
+            for (int e = 0; e < 64; ++e) {
+              x[e] = key0 + e > lim ? -INFINITY : x[e] * scale_log2;
+              m4[e & 3] = fmaxf(m4[e & 3], x[e]);
+            }
+          } else {
+#pragma unroll
+            for (int e = 0; e < 64; ++e) {
+              x[e] *= scale_log2;
+              m4[e & 3] = fmaxf(m4[e & 3], x[e]);
             }
           }
-          m_ref = mx == -INFINITY ? 0.f : mx;
+          mx = fmaxf(fmaxf(m4[0], m4[1]), fmaxf(m4[2], m4[3]));
         }
         if (want_o && it >= 2) {
-          // the P buffer of this tile was last read by the P V of running tile it-2
+          // keeps every phase of p_free[b] observed in order, so that the parity waits below cannot mistake an older
+          // completion for the one they mean (P V of running tile it-2 finished long ago: this does not block)
           ok = __all_sync(0xffffffffu, mbar_wait(p_free(it & 1), ((it >> 1) & 1) ^ 1, abort_flag, status));
           if (!ok) break;
         }
-#pragma unroll 1
-        for (int trip = 0; trip < 2; ++trip) {
-          // mx is tracked relative to the reference: the exponent argument itself, fmaf(s, scale, -m_ref)
-          float mx = -INFINITY, ls[4] = {0.f, 0.f, 0.f, 0.f};
-          const float neg_ref = -m_ref;
-          float buf[2][32];
-          ld32(ts, buf[0]);
-#pragma unroll
-          for (int c = 0; c < 2; ++c) {
-            wait_ld();
-            if (c < 1) ld32(ts + (c + 1) * 32, buf[(c + 1) & 1]);
-            float* sv = buf[c & 1];
-            if (need_mask) softmax_chunk<true>(sv, key0 + c * 32, lim, scale_log2, neg_ref, mx, ls);
-            else softmax_chunk<false>(sv, key0 + c * 32, lim, scale_log2, neg_ref, mx, ls);
-            if (want_o) {
-              // this thread's 64 keys are sub-tile `half` of the P buffer
-#pragma unroll
-              for (int j = 0; j < 4; ++j)
-                *reinterpret_cast<uint4*>(base_ptr + L::P_OFF + (it & 1) * L::P_BYTES + half * L::SUB + swz(row, c * 4 + j)) = pack8(sv + 8 * j);
-            }
-          }
-          const float lsum = (ls[0] + ls[1]) + (ls[2] + ls[3]);
-          if (!__any_sync(0xffffffffu, mx > RESCALE_TH)) {
-            l_run += lsum;
-            break;
-          }
-          const float raise = fmaxf(mx, 0.f);  // lanes below the threshold may move too: any value >= their maximum is valid
+        if (kt == 0) {
+          m_ref = mx == -INFINITY ? 0.f : mx;
+        } else if (__any_sync(0xffffffffu, mx - m_ref > RESCALE_TH)) {
+          const float raise = fmaxf(mx - m_ref, 0.f);  // lanes below the threshold may move too: any value >= their maximum is valid
           const float f = exp2f(-raise);
           m_ref += raise;
           l_run *= f;
-          if (want_o && kt > 0) {
+          if (want_o) {
             // the output so far must be complete (P V of the previous tile) before it is rescaled in place
-            // (the threads follow every phase of p_free[b] in order - running tile it-1 waited for it-3 on the same
-            // barrier - so a parity wait cannot mistake an older completion for this one)
             ok = __all_sync(0xffffffffu, mbar_wait(p_free((it - 1) & 1), ((it - 1) >> 1) & 1, abort_flag, status));
             if (!ok) break;
             fence_after();
@@ -523,22 +505,44 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
             wait_st();
           }
         }
-        if (!ok) break;
-        if (want_o && w.kt0 + kt == w.nkt_all - 1 && half == 0) {
-          // slots beyond the row tile's last visible key may hold anything: they get probability zero, and zero
-          // times a non-finite value would still poison the product, so clear those V rows of the last tile
-          // (thread `row` of the first half clears key `row`)
-          const int first_bad = w.maxpos - (w.kt0 + kt) * ATC_BN + 1;
-          const bool landed = mbar_wait(v_full(it & 1), (it >> 1) & 1, abort_flag, status);  // the V tile must have landed before rows of it are cleared
-          if (landed && row >= first_bad) {
-            unsigned char* sv = base_ptr + L::KV_OFF + (it & 1) * L::KV_STAGE + (D / 64) * L::SUB;
+        // pass 2: probabilities (ex2.approx maps -inf to +0), row sum in four chains
+        {
+          float ls[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
-            for (int j = 0; j < D / 64; ++j)
+          for (int e = 0; e < 64; ++e) {
+            x[e] = ex2_approx(x[e] - m_ref);
+            ls[e & 3] += x[e];
+          }
+          l_run += (ls[0] + ls[1]) + (ls[2] + ls[3]);
+        }
+        if (want_o) {
+          // P as bf16 pairs over the first 32 of this thread's 64 S columns (all of them are in registers by now):
+          // the A operand of the P V MMA is read from tensor memory
+          uint32_t pk[32];
 #pragma unroll
-              for (int c = 0; c < 8; ++c) *reinterpret_cast<uint4*>(sv + j * L::SUB + row * 128 + c * 16) = make_uint4(0, 0, 0, 0);
+          for (int j = 0; j < 8; ++j) {
+            const uint4 v = pack8(x + 8 * j);
+            pk[4 * j] = v.x, pk[4 * j + 1] = v.y, pk[4 * j + 2] = v.z, pk[4 * j + 3] = v.w;
+          }
+          st32(ts, reinterpret_cast<const float*>(pk));
+          wait_st();
+          if (w.kt0 + kt == w.nkt_all - 1 && half == 0) {
+            // slots beyond the row tile's last visible key may hold anything: they get probability zero, and zero
+            // times a non-finite value would still poison the product, so clear those V rows of the last tile
+            // (thread `row` of the first half clears key `row`)
+            const int first_bad = w.maxpos - (w.kt0 + kt) * ATC_BN + 1;
+            const int vs = it % L::KV_STAGES;
+            const bool landed = mbar_wait(v_full(vs), (it / L::KV_STAGES) & 1, abort_flag, status);  // the V tile must have landed before rows of it are cleared
+            if (landed && row >= first_bad) {
+              unsigned char* sv = base_ptr + L::KV_OFF + vs * L::KV_STAGE + (D / 64) * L::SUB;
+#pragma unroll
+              for (int j = 0; j < D / 64; ++j)
+#pragma unroll
+                for (int c = 0; c < 8; ++c) *reinterpret_cast<uint4*>(sv + j * L::SUB + row * 128 + c * 16) = make_uint4(0, 0, 0, 0);
+            }
+            fence_async_smem();
           }
         }
-        fence_async_smem();
         fence_before();
         mbar_arrive(p_ready(it & 1));
       }
