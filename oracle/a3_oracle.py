@@ -152,13 +152,18 @@ def position_recovery(
     model: Model,
     dtype=np.float64,
     rnd: Callable = identity,
+    stored_unrotated: bool = False,
 ):
-    """Eq. 2 on caches stored at chunk-local positions.
+    """Eq. 2.
 
-    chunk_k[c], chunk_v[c]: [L][T_c][Hkv][D].  Token t of chunk c already carries
-    R(t); rotating it by the chunk's offset o_c gives R(o_c + t), its position in
-    the concatenated input.  V is copied unchanged.  Returns Kf, Vf of shape
-    [L][n_slots][Hkv][D]; slots not covered by a chunk (the question rows) are zero.
+    chunk_k[c], chunk_v[c]: [L][T_c][Hkv][D].  Two storage conventions of the
+    Position Recovery subsection:
+      * stored at chunk-local positions (default): token t of chunk c already
+        carries R(t); rotating it by the chunk's offset o_c gives R(o_c + t);
+      * stored without positional embedding (stored_unrotated): token t of chunk c
+        is rotated by its global position m = o_c + t, which is Eq. 2 as printed.
+    V is copied unchanged.  Returns Kf, Vf of shape [L][n_slots][Hkv][D]; slots not
+    covered by a chunk (the question rows) are zero.
     """
     L, Hkv, D = model.n_layers, model.n_kv_heads, model.head_dim
     Kf = np.zeros((L, n_slots, Hkv, D), dtype=dtype)
@@ -167,10 +172,21 @@ def position_recovery(
         T = kc.shape[1]
         o = int(offsets[c])
         delta = np.full(T, o, dtype=np.int64)
+        if stored_unrotated:
+            delta = delta + np.arange(T, dtype=np.int64)
         for l in range(L):
             Kf[l, o : o + T] = rnd(rope_rotate(kc[l].astype(dtype), delta, model.rope_theta, model.rope_layout))
             Vf[l, o : o + T] = vc[l].astype(dtype)
     return Kf, Vf
+
+
+def strip_positions(chunk_k: np.ndarray, model: Model, rnd: Callable = identity) -> np.ndarray:
+    """A chunk's keys [L][T][Hkv][D] stored at local positions -> the same keys "without
+    positional embedding" (Position Recovery subsection): token t is rotated by -t.
+    R(-t) R(t) = I, so this is the key before RoPE."""
+    T = chunk_k.shape[1]
+    back = -np.arange(T, dtype=np.int64)
+    return np.stack([rnd(rope_rotate(chunk_k[l], back, model.rope_theta, model.rope_layout)) for l in range(chunk_k.shape[0])])
 
 
 # --------------------------------------------------------------------------- block pieces

@@ -88,6 +88,35 @@ def test_position_recovery_offsets_and_value_copy():
     assert not Kf[:, 15:].any() and not Vf[:, 15:].any()
 
 
+@pytest.mark.parametrize("layout", [0, 1])
+def test_position_recovery_unrotated_storage_is_eq2_as_printed(layout):
+    """Keys stored without positional embedding and rotated by the global position m (Eq. 2) give the same
+    fused cache as keys stored at local positions rotated by the chunk offset; the angles are checked
+    against cos/sin written out for one pair, independently of rope_rotate."""
+    from dataclasses import replace
+    m = replace(W.TINY_GQA, rope_layout=layout)
+    model = oracle_model(m)
+    lens = (4, 7, 3)
+    offs = (0, 4, 11)
+    ks, vs = zip(*[W.make_cache_like(m, t, 0, c) for c, t in enumerate(lens)])
+    ks = [k.astype(np.float64) for k in ks]
+    raw = [O.strip_positions(k, model) for k in ks]
+    K_local, V_local = O.position_recovery(ks, vs, offs, 16, model)
+    K_raw, V_raw = O.position_recovery(raw, vs, offs, 16, model, stored_unrotated=True)
+    np.testing.assert_allclose(K_raw, K_local, atol=1e-9)
+    np.testing.assert_array_equal(V_raw, V_local)
+    # one pair by hand: chunk 1, layer 1, token 5, head 1, frequency index 2 -> global position 9
+    D = m.head_dim
+    i = 2
+    a, b = (i, i + D // 2) if layout == 0 else (2 * i, 2 * i + 1)
+    ang = 9 * m.rope_theta ** (-2.0 * i / D)
+    x, y = raw[1][1, 5, 1, a], raw[1][1, 5, 1, b]
+    assert K_raw[1, 9, 1, a] == pytest.approx(x * math.cos(ang) - y * math.sin(ang), abs=1e-12)
+    assert K_raw[1, 9, 1, b] == pytest.approx(x * math.sin(ang) + y * math.cos(ang), abs=1e-12)
+    # stripping is norm-preserving per pair and undoes the local rotation exactly (up to rounding)
+    np.testing.assert_allclose(np.linalg.norm(raw[2], axis=-1), np.linalg.norm(ks[2], axis=-1), rtol=1e-12)
+
+
 # ------------------------------------------------------------------ small building blocks against library routines
 
 
