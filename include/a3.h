@@ -70,15 +70,19 @@ typedef struct {
   const void *attn_norm, *wq, *wk, *wv, *bq, *bk, *bv, *wo, *mlp_norm, *w_gate, *w_up, *w_down;
 } a3_layer_weights;
 
-/* One precomputed chunk (Eq. 1): K_i, V_i of all layers, stored at local positions 0..len-1. */
+/* One precomputed chunk (Eq. 1): K_i, V_i of all layers.  Position recovery (Eq. 2) rotates the key of token t
+ * by delta + token_step * t positions:
+ *   stored at local positions 0..len-1 (the default):            delta = dst_offset, token_step = 0
+ *   stored without positional embedding (Eq. 2 as printed):      delta = dst_offset, token_step = 1
+ *   converting local-position storage to storage without one:    delta = 0,          token_step = -1 */
 typedef struct {
   const void* k_src;          /* dev, [n_layers][len][Hkv][D], layer l at k_src + l*src_layer_stride */
   const void* v_src;          /* dev, same layout */
   uint64_t src_layer_stride;  /* bytes between consecutive layers of this chunk */
   int32_t len;                /* tokens in the chunk */
   int32_t dst_offset;         /* first slot of the chunk in the fused cache (o_c) */
-  int32_t delta;              /* rotation to apply: global minus stored position (= dst_offset for local storage) */
-  int32_t reserved;
+  int32_t delta;              /* rotation of token 0: global minus stored position (= dst_offset for local storage) */
+  int32_t token_step;         /* additional rotation per token index: 0, +1 or -1 (see above) */
 } a3_chunk_ref;
 
 /* One fusion request.  Slots [0, n_ctx) are the chunks in input order, [n_ctx, n_ctx+n_question)
@@ -132,7 +136,7 @@ int a3_recompute_count(double ratio, int n, int n_candidates);
 /* ---- the steps --------------------------------------------------------------------- */
 
 /* Position recovery (Eq. 2): for layers [layer_begin, layer_end), every chunk c, token t:
- *   k_fused[l][dst_offset+t] = R(delta) k_src[l][t]   (rotation per head, fp32 arithmetic)
+ *   k_fused[l][dst_offset+t] = R(delta + token_step*t) k_src[l][t]   (rotation per head, fp32 arithmetic)
  *   v_fused[l][dst_offset+t] = v_src[l][t]
  * chunks: dev array; max_chunk_len >= every len (host copy of the largest length, sizes the grid).
  * Fused layer l lives at k_fused + l*layer_stride bytes. */

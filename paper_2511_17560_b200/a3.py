@@ -45,7 +45,7 @@ class LayerWeights(C.Structure):
 
 class ChunkRef(C.Structure):
     _fields_ = [("k_src", C.c_void_p), ("v_src", C.c_void_p), ("src_layer_stride", C.c_uint64), ("len", C.c_int32),
-                ("dst_offset", C.c_int32), ("delta", C.c_int32), ("reserved", C.c_int32)]
+                ("dst_offset", C.c_int32), ("delta", C.c_int32), ("token_step", C.c_int32)]
 
 
 class Request(C.Structure):
@@ -141,8 +141,10 @@ def launch_count(reset: bool = False) -> int:
 
 
 def chunk_table(chunk_k: Sequence[torch.Tensor], chunk_v: Sequence[torch.Tensor], offsets: Sequence[int],
-                deltas: Optional[Sequence[int]] = None, device=None) -> torch.Tensor:
-    """Device array of a3_chunk_ref for chunk caches shaped [L][T][Hkv][D] (bf16, contiguous)."""
+                deltas: Optional[Sequence[int]] = None, device=None, token_step: int = 0) -> torch.Tensor:
+    """Device array of a3_chunk_ref for chunk caches shaped [L][T][Hkv][D] (bf16, contiguous).
+    token_step: 0 for keys stored at local positions, 1 for keys stored without positional embedding,
+    -1 (with deltas of 0) to strip the local positions."""
     arr = (ChunkRef * max(1, len(chunk_k)))()
     for c, (k, v) in enumerate(zip(chunk_k, chunk_v)):
         assert k.dtype == torch.bfloat16 and k.is_contiguous() and v.is_contiguous() and k.shape == v.shape
@@ -151,6 +153,7 @@ def chunk_table(chunk_k: Sequence[torch.Tensor], chunk_v: Sequence[torch.Tensor]
         arr[c].len = k.shape[1]
         arr[c].dst_offset = int(offsets[c])
         arr[c].delta = int(offsets[c] if deltas is None else deltas[c])
+        arr[c].token_step = int(token_step)
     raw = np.frombuffer(bytes(arr), dtype=np.uint8).copy()
     dev = device if device is not None else (chunk_k[0].device if len(chunk_k) else "cuda")
     return torch.from_numpy(raw).to(dev)

@@ -536,7 +536,7 @@ extern "C" int a3_fuse_request_host(const a3_handle* h, const a3_request* req, c
     href[c].len = len;
     href[c].dst_offset = off;
     href[c].delta = off;
-    href[c].reserved = 0;
+    href[c].token_step = 0;  // the host entry takes chunks stored at local positions
     kvoff += 2 * bytes;
     off += len;
     if (len > maxlen) maxlen = len;

@@ -43,7 +43,9 @@ rerotate_kernel(const a3_chunk_ref* __restrict__ chunks, char* __restrict__ kf, 
   const int l = layer_begin + blockIdx.z;
   const int nt = min(tok_per_cta, ch.len - t0);
   int ad = ch.delta < 0 ? -ch.delta : ch.delta;
-  const bool bad = ad >= max_pos || ch.dst_offset < 0 || ((uintptr_t)ch.k_src & 15) || ((uintptr_t)ch.v_src & 15) ||
+  // with a per-token step the rotation of token t is delta + token_step * t: both ends must be in the table
+  const long long a_last = (long long)ch.delta + (long long)ch.token_step * (ch.len - 1);
+  const bool bad = ad >= max_pos || (a_last < 0 ? -a_last : a_last) >= max_pos || ch.dst_offset < 0 || ((uintptr_t)ch.k_src & 15) || ((uintptr_t)ch.v_src & 15) ||
                    (ch.src_layer_stride & 15);
   if (bad) {
     if (threadIdx.x == 0) atomicOr(status, A3_DEV_BAD_POSITION);
@@ -58,7 +60,58 @@ rerotate_kernel(const a3_chunk_ref* __restrict__ chunks, char* __restrict__ kf, 
   const int nvec = nt * (row_elems / 8);
   const float2* trow = tab + (size_t)ad * (D / 2);
 
-  if (LAYOUT == 0) {
+  if (ch.token_step != 0) {
+    // Keys stored without positional embedding (or being converted to that form): every token has an angle of
+    // its own, so cos/sin come from the table row of the token's rotation instead of living in registers.
+    const int vec_per_tok = row_elems / 8;
+    if (LAYOUT == 0) {
+      constexpr int UPH = D / 16;
+      const int nunit = nvec / 2;
+      for (int u = threadIdx.x; u < nunit; u += RR_THREADS) {
+        const int j = u % UPH;
+        const int lo = (u / UPH) * (D / 8) + j;
+        const int tok = lo / vec_per_tok;
+        const int a = ch.delta + ch.token_step * (t0 + tok);
+        const float sg = a < 0 ? -1.f : 1.f;
+        const float4* tr = reinterpret_cast<const float4*>(tab + (size_t)(a < 0 ? -a : a) * (D / 2) + 8 * j);
+        float fa[8], fb[8], ra[8], rb[8];
+        unpack8(__ldcs(ksrc + lo), fa);
+        unpack8(__ldcs(ksrc + lo + UPH), fb);
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+          const float4 t = __ldg(tr + e);  // (cos, sin) of frequencies 8j+2e and 8j+2e+1
+          const float c0 = t.x, s0 = sg * t.y, c1 = t.z, s1 = sg * t.w;
+          ra[2 * e] = fa[2 * e] * c0 - fb[2 * e] * s0;
+          rb[2 * e] = fa[2 * e] * s0 + fb[2 * e] * c0;
+          ra[2 * e + 1] = fa[2 * e + 1] * c1 - fb[2 * e + 1] * s1;
+          rb[2 * e + 1] = fa[2 * e + 1] * s1 + fb[2 * e + 1] * c1;
+        }
+        __stcs(kdst + lo, pack8(ra));
+        __stcs(kdst + lo + UPH, pack8(rb));
+      }
+    } else {
+      constexpr int VPH = D / 8;
+      for (int v = threadIdx.x; v < nvec; v += RR_THREADS) {
+        const int c = v % VPH;
+        const int tok = v / vec_per_tok;
+        const int a = ch.delta + ch.token_step * (t0 + tok);
+        const float sg = a < 0 ? -1.f : 1.f;
+        const float4* tr = reinterpret_cast<const float4*>(tab + (size_t)(a < 0 ? -a : a) * (D / 2) + 4 * c);
+        float f[8], r[8];
+        unpack8(__ldcs(ksrc + v), f);
+#pragma unroll
+        for (int e = 0; e < 2; ++e) {
+          const float4 t = __ldg(tr + e);
+          const float c0 = t.x, s0 = sg * t.y, c1 = t.z, s1 = sg * t.w;
+          r[4 * e] = f[4 * e] * c0 - f[4 * e + 1] * s0;
+          r[4 * e + 1] = f[4 * e] * s0 + f[4 * e + 1] * c0;
+          r[4 * e + 2] = f[4 * e + 2] * c1 - f[4 * e + 3] * s1;
+          r[4 * e + 3] = f[4 * e + 2] * s1 + f[4 * e + 3] * c1;
+        }
+        __stcs(kdst + v, pack8(r));
+      }
+    }
+  } else if (LAYOUT == 0) {
     // pairs (i, i + D/2): a unit is the two 16-byte vectors of one head that hold columns [8j,8j+8) and +D/2.
     constexpr int UPH = D / 16;  // units per head
     const int j = threadIdx.x % UPH;  // RR_THREADS is a multiple of UPH, so j is fixed per thread

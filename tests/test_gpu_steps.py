@@ -93,6 +93,59 @@ def test_rerotate_parity(a3mod, shape, layout):
     eng.close()
 
 
+@pytest.mark.parametrize("shape,layout", [(W.TINY3, 0), (W.TINY_GQA, 1), (W.TINY_G7, 0)])
+def test_rerotate_unrotated_storage(a3mod, shape, layout):
+    """Keys stored without positional embedding (token_step = 1: Eq. 2 as printed) and the conversion of
+    local-position storage into that form (token_step = -1)."""
+    from dataclasses import replace
+    m = replace(shape, rope_layout=layout)
+    eng, _, dev = make_engine(a3mod, m)
+    model = oracle_model(m)
+    lens = [1, 127, 300, 2047, 5]
+    base = 20000
+    offs, o = [], base
+    for t in lens:
+        offs.append(o)
+        o += t
+    n = o + 3
+    ck, cv = zip(*[W.make_cache_like(m, t, 2, c, std=1.28) for c, t in enumerate(lens)])  # bf16-representable values
+    dk = [to_dev(k, dev) for k in ck]
+    dv = [to_dev(v, dev) for v in cv]
+    canary = 7.0
+    # (i) the stored keys taken as un-rotated: token t of chunk c is rotated by o_c + t
+    Kf = torch.full((m.n_layers, n, m.n_kv_heads, m.head_dim), canary, dtype=torch.bfloat16, device=dev)
+    Vf = torch.full_like(Kf, canary)
+    eng.rope_rerotate(a3mod.chunk_table(dk, dv, offs, token_step=1), len(lens), max(lens), Kf, Vf)
+    assert eng.device_status() == 0
+    Ko, Vo = O.position_recovery(ck, cv, offs, n, model, stored_unrotated=True)
+    check_kv(f64(Kf)[:, base:o], Ko[:, base:o], "K from un-rotated storage")
+    np.testing.assert_array_equal(f64(Vf)[:, base:o], Vo[:, base:o])
+    assert (f64(Kf)[:, :base] == canary).all() and (f64(Kf)[:, o:] == canary).all()
+    # (ii) stripping local positions: token t rotated by -t, chunks written back to back from slot 0
+    offs0, o0 = [], 0
+    for t in lens:
+        offs0.append(o0)
+        o0 += t
+    Ks = torch.full((m.n_layers, o0 + 2, m.n_kv_heads, m.head_dim), canary, dtype=torch.bfloat16, device=dev)
+    Vs = torch.full_like(Ks, canary)
+    eng.rope_rerotate(a3mod.chunk_table(dk, dv, offs0, deltas=[0] * len(lens), token_step=-1), len(lens), max(lens), Ks, Vs)
+    assert eng.device_status() == 0
+    got = f64(Ks)
+    for c, (oo, t) in enumerate(zip(offs0, lens)):
+        want = O.strip_positions(ck[c].astype(np.float64), model)
+        check_kv(got[:, oo:oo + t], want, f"stripped K of chunk {c}")
+    assert (got[:, o0:] == canary).all()
+    # a rotation that would leave the table is refused on the device and flagged
+    eng2, _, _ = make_engine(a3mod, m, max_pos=1000)
+    K2 = torch.zeros((m.n_layers, 1200, m.n_kv_heads, m.head_dim), dtype=torch.bfloat16, device=dev)
+    V2 = torch.zeros_like(K2)
+    eng2.rope_rerotate(a3mod.chunk_table(dk[2:3], dv[2:3], [800], token_step=1), 1, 300, K2, V2)
+    assert eng2.device_status() & 1  # A3_DEV_BAD_POSITION
+    assert not K2.any()
+    eng2.close()
+    eng.close()
+
+
 def test_rerotate_bad_arguments(a3mod):
     eng, _, dev = make_engine(a3mod, W.TINY3, max_pos=1000)
     m = W.TINY3
