@@ -39,7 +39,7 @@ Pins (tests marked "not gpu"): RoPE composition / R(0)=I / norm / the D=4 matrix
 written out by hand; layer-0 and chunk-0 exactness of recovered caches against a
 full prefill; r=1 == full prefill; r=0 == position-recovered concatenation;
 softmax rows sum to one; uniform-key closed form; causality; brute-force top-k;
-nested selections.  Whole-request agreement of a deep bf16 stack with this oracle
+nested selections; first-token logits against a library matmul and planted rows.  Whole-request agreement of a deep bf16 stack with this oracle
 has no pin beyond the oracle itself ("parity unpinned" for that one statement).
 """
 from __future__ import annotations
@@ -357,6 +357,24 @@ def topk_select(s: np.ndarray, cand_begin: int, cand_end: int, k: int) -> np.nda
     k = max(0, min(int(k), cand.size))
     order = sorted(cand.tolist(), key=lambda i: (-float(s[i]), i))
     return np.array(sorted(order[:k]), dtype=np.int64)
+
+
+def first_token(x_last: np.ndarray, final_norm: np.ndarray, lm_head: np.ndarray, eps: float, rnd: Callable = identity):
+    """The first generated token after fusion (the quantity behind the paper's TTFT figures; Inference
+    paragraph of the Experiments): final RMSNorm of the last question row's hidden state, the
+    vocabulary projection, greedy choice.
+
+    x_last: [d]; final_norm: [d]; lm_head: [vocab][d].  Returns (logits [vocab], token) with ties
+    going to the lowest token id.
+    """
+    a = rnd(rmsnorm(x_last[None, :], final_norm, eps))[0]
+    logits = lm_head.astype(a.dtype) @ a
+    best = -np.inf
+    token = 0
+    for i, v in enumerate(logits.tolist()):
+        if v > best:
+            best, token = v, i
+    return logits, token
 
 
 def recompute_count(ratio: float, n: int, n_candidates: int) -> int:

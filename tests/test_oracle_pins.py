@@ -380,3 +380,32 @@ def test_bf16_mirrored_oracle_stays_close_to_exact(tiny3):
     c = O.fuse_request(ck, cv, x0, r.n_question, weights, model, ratio=0.15, select_layer=1, dtype=np.float32)
     assert c.Re.tolist() == a.Re.tolist()
     assert np.abs(a.K - c.K).max() < 1e-3
+
+
+# ------------------------------------------------------------------ first token
+
+
+def test_first_token_matches_library_and_planted_row():
+    rng = np.random.default_rng(5)
+    d, V = 64, 500
+    x = rng.standard_normal(d) * 3.0
+    g = 1.0 + 0.1 * rng.standard_normal(d)
+    Wm = rng.standard_normal((V, d)) * 0.05
+    eps = 1e-5
+    logits, tok = O.first_token(x, g, Wm, eps)
+    # library route: torch rms_norm + linear
+    xt = torch.from_numpy(x)[None]
+    a = torch.nn.functional.rms_norm(xt, (d,), torch.from_numpy(g), eps)
+    want = torch.nn.functional.linear(a, torch.from_numpy(Wm))[0].numpy()
+    np.testing.assert_allclose(logits, want, rtol=1e-12, atol=1e-12)
+    assert tok == int(np.argmax(want))
+    # a vocabulary row aligned with the normalised state wins, by the Cauchy-Schwarz bound
+    a_np = a[0].numpy()
+    W2 = Wm.copy()
+    W2[321] = a_np / np.linalg.norm(a_np) * (np.linalg.norm(Wm, axis=1).max() * 1.01)
+    assert O.first_token(x, g, W2, eps)[1] == 321
+    # ties go to the lowest id; scaling the hidden state does not change the logits (RMSNorm), up to eps
+    W3 = Wm.copy()
+    W3[7] = W3[400] = W2[321]
+    assert O.first_token(x, g, W3, eps)[1] == 7
+    np.testing.assert_allclose(O.first_token(4.0 * x, g, Wm, 0.0)[0], O.first_token(x, g, Wm, 0.0)[0], rtol=1e-12)
