@@ -222,6 +222,17 @@ int a3_fuse_request_host(const a3_handle* h, const a3_request* req, const a3_hos
 
 /* ---- diagnostics -------------------------------------------------------------------- */
 
+/* First token after fusion (what the paper's time-to-first-token figures end with; Inference paragraph of the
+ * Experiments): a = RMSNorm(x_row) * final_norm (rounded to bf16), logits = lm_head a, token = argmax (lowest id
+ * on ties).  x_row: dev [d_model] bf16, normally the last row of a3_fuse_request's x_out; final_norm: dev
+ * [d_model] bf16; lm_head: dev [vocab][d_model] bf16, 16-byte aligned; logits_out: dev [vocab] fp32 or NULL;
+ * token_out: dev int32.  ws: dev, 256-byte aligned, a3_first_token_workspace_bytes(h) bytes, borrowed for the
+ * call.  One kernel launch (plus a 4-byte memset), no allocation, no synchronisation.  Non-finite logits set
+ * A3_DEV_NONFINITE_SCORE and never win. */
+size_t a3_first_token_workspace_bytes(const a3_handle* h);
+int a3_first_token(const a3_handle* h, const void* x_row, const void* final_norm, const void* lm_head, int vocab,
+                   float* logits_out, int32_t* token_out, void* ws, size_t ws_bytes, a3_stream stream);
+
 /* Waits for `stream`, reads and clears the device status word (A3_DEV_* bits). */
 int a3_device_status(const a3_handle* h, uint32_t* bits_out, a3_stream stream);
 const char* a3_status_string(int status);
@@ -236,7 +247,7 @@ uint64_t a3_launch_count(int reset);
  * a3_profile_read waits for `stream`, adds up the elapsed time per class and clears the records. */
 typedef enum {
   A3_K_REROTATE = 0, A3_K_RMSNORM, A3_K_GEMM_QKV, A3_K_ATTENTION, A3_K_GEMM_RESIDUAL, A3_K_GEMM_SWIGLU,
-  A3_K_SCORES, A3_K_TOPK, A3_K_ROWS /* gather, scatter, index kernels */, A3_K_CLASSES
+  A3_K_SCORES, A3_K_TOPK, A3_K_ROWS /* gather, scatter, index kernels */, A3_K_FIRST_TOKEN, A3_K_CLASSES
 } a3_kernel_class;
 typedef struct { uint64_t launches; double ms; } a3_profile_entry;
 int a3_profile_enable(a3_handle* h, int max_records);

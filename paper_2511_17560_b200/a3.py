@@ -63,10 +63,10 @@ class HostIO(C.Structure):
 
 EXPORTS = ("a3_create", "a3_destroy", "a3_layer_workspace_bytes", "a3_request_workspace_bytes", "a3_host_staging_bytes",
            "a3_recompute_count", "a3_rope_rerotate", "a3_query_scores", "a3_query_scores_static", "a3_topk_select", "a3_recompute_layer",
-           "a3_scatter_kv", "a3_gather_rows", "a3_precompute_chunk", "a3_fuse_request", "a3_fuse_batch", "a3_fuse_request_host",
+           "a3_scatter_kv", "a3_gather_rows", "a3_precompute_chunk", "a3_first_token_workspace_bytes", "a3_first_token", "a3_fuse_request", "a3_fuse_batch", "a3_fuse_request_host",
            "a3_device_status", "a3_status_string", "a3_last_cuda_error", "a3_launch_count", "a3_profile_enable",
            "a3_profile_read", "a3_kernel_class_name")
-K_CLASSES = 9
+K_CLASSES = 10
 
 
 class ProfileEntry(C.Structure):
@@ -99,6 +99,9 @@ def _load():
     lib.a3_scatter_kv.argtypes = [vp, vp, vp, vp, i32, vp, vp, i32, vp]
     lib.a3_gather_rows.argtypes = [vp, vp, i32, vp, i32, i32, vp, vp]
     lib.a3_precompute_chunk.argtypes = [vp, vp, i32, vp, vp, u64, vp, sz, vp]
+    lib.a3_first_token_workspace_bytes.argtypes = [vp]
+    lib.a3_first_token_workspace_bytes.restype = sz
+    lib.a3_first_token.argtypes = [vp, vp, vp, vp, i32, vp, vp, vp, sz, vp]
     lib.a3_fuse_request.argtypes = [vp, C.POINTER(Request), vp, sz, vp]
     lib.a3_fuse_batch.argtypes = [vp, C.POINTER(Request), i32, vp, sz, vp]
     lib.a3_fuse_request_host.argtypes = [vp, C.POINTER(Request), C.POINTER(HostIO), vp, sz, vp, sz, vp]
@@ -272,6 +275,17 @@ class A3:
         _check(_load().a3_precompute_chunk(self._h, _ptr(x_chunk), T, _ptr(k_chunk), _ptr(v_chunk), k_chunk.stride(0) * 2,
                                            _ptr(ws), ws.numel(), _stream()), "a3_precompute_chunk")
         return x_chunk
+
+    def first_token(self, x_row, final_norm, lm_head, want_logits=True):
+        """Final norm + vocabulary projection + greedy choice for one hidden row [d]; returns (logits or None, token)."""
+        vocab = lm_head.shape[0]
+        dev = lm_head.device
+        logits = torch.empty(vocab, dtype=torch.float32, device=dev) if want_logits else None
+        token = torch.empty(1, dtype=torch.int32, device=dev)
+        ws = self.workspace(int(_load().a3_first_token_workspace_bytes(self._h)))
+        _check(_load().a3_first_token(self._h, _ptr(x_row), _ptr(final_norm), _ptr(lm_head), vocab, _ptr(logits), _ptr(token),
+                                      _ptr(ws), ws.numel(), _stream()), "a3_first_token")
+        return logits, token
 
     def make_request(self, chunks, n_chunks, max_chunk_len, n_ctx, n_question, x0, k_fused, v_fused, ratio=0.15,
                      select_layer=1, n_system=0, forced_re=None, n_recompute=None):

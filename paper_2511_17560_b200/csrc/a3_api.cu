@@ -185,7 +185,7 @@ extern "C" int a3_profile_read(a3_handle* h, a3_profile_entry* out, a3_stream st
 
 extern "C" const char* a3_kernel_class_name(int cls) {
   static const char* names[A3_K_CLASSES] = {"rerotate", "rmsnorm", "gemm_qkv", "attention", "gemm_residual",
-                                            "gemm_swiglu", "scores", "topk", "rows"};
+                                            "gemm_swiglu", "scores", "topk", "rows", "first_token"};
   return cls >= 0 && cls < A3_K_CLASSES ? names[cls] : "?";
 }
 

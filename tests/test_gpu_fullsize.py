@@ -231,3 +231,30 @@ def test_batched_serving_matches_single_requests():
         n_ctx = rb.n_ctx
         assert ob["rows"].cpu().numpy()[:p].tolist() == O.topk_select(s, 0, n_ctx, p).tolist()
     eng.close()
+
+
+def test_first_token_llama_vocabulary():
+    """Final norm + 128 256 x 4 096 vocabulary projection + greedy choice at Llama-3-8B size: logits of sampled
+    vocabulary rows (and of the chosen one) against the oracle, the choice against the kernel's own logits."""
+    from paper_2511_17560_b200 import a3
+    from tests.test_gpu_steps import FT_TOL
+    m = replace(W.LLAMA8B, n_layers=1)
+    eng = a3.A3(m, W.make_weights_device(m, DEV, 0), 64)
+    vocab, d = 128256, m.d_model
+    g = torch.Generator(device=DEV)
+    g.manual_seed(21)
+    lm = (torch.randn((vocab, d), device=DEV, generator=g) * 0.02).to(torch.bfloat16)
+    x = (torch.randn(d, device=DEV, generator=g) * 3.0).to(torch.bfloat16)
+    gain = (1.0 + 0.1 * torch.randn(d, device=DEV, generator=g)).to(torch.bfloat16)
+    logits, token = eng.first_token(x, gain, lm)
+    assert eng.device_status() == 0
+    got = logits.cpu().numpy().astype(np.float64)
+    tok = int(token.item())
+    assert tok == int(np.flatnonzero(got == got.max())[0])
+    rows = np.unique(np.concatenate([np.random.default_rng(3).integers(0, vocab, 4096), [0, 1, vocab - 2, vocab - 1, tok]]))
+    want, _ = O.first_token(f64(x), f64(gain), f64(lm[torch.from_numpy(rows).to(DEV)]), m.rms_eps, rnd=O.round_bf16)
+    scale = np.sqrt(np.mean(want ** 2))
+    assert np.abs(got[rows] - want).max() <= FT_TOL * scale
+    # the chosen logit is the largest of the sample in the oracle's arithmetic too (up to the tolerance)
+    assert want[np.searchsorted(rows, tok)] >= want.max() - 2 * FT_TOL * scale
+    eng.close()

@@ -363,3 +363,64 @@ def test_attention_key_split_matches_unsplit(a3mod):
     err = (a[0].float() - b[0].float()).abs()
     assert err.max().item() <= 0.07 and err.mean().item() <= 4e-3  # bf16 rounding of the attention output, propagated
     eng.close()
+
+
+# ------------------------------------------------------------------ first token (final norm, vocabulary projection, greedy choice)
+
+# fp32 dot products of bf16 factors over d terms of size ~|a||w|: the summation error is ~1e-6 relative; a
+# normalised activation that lands on a bf16 rounding tie may differ by one ulp (2^-8 relative) between the fp32
+# and the fp64 statistics, which moves a logit by at most 2^-8 * max|a_i w_i|.  5e-4 * (rms logit) covers both.
+FT_TOL = 5e-4
+
+
+@pytest.mark.parametrize("shape,vocab", [(W.TINY3, 1001), (W.TINY_GQA, 32003), (W.TINY3, 2)])
+def test_first_token_parity(a3mod, shape, vocab):
+    m = shape
+    eng, _, dev = make_engine(a3mod, m)
+    rng = np.random.default_rng(11)
+    d = m.d_model
+    x = W.bf16_round(rng.standard_normal(d).astype(np.float32) * 2.5)
+    g = W.bf16_round((1.0 + 0.1 * rng.standard_normal(d)).astype(np.float32))
+    Wm = W.bf16_round((rng.standard_normal((vocab, d)) * 0.02).astype(np.float32))
+    logits, token = eng.first_token(to_dev(x, dev), to_dev(g, dev), to_dev(Wm, dev))
+    assert eng.device_status() == 0
+    want, want_tok = O.first_token(x.astype(np.float64), g.astype(np.float64), Wm.astype(np.float64), m.rms_eps, rnd=O.round_bf16)
+    got = logits.cpu().numpy().astype(np.float64)
+    scale = max(np.sqrt(np.mean(want ** 2)), 1e-6)
+    assert np.abs(got - want).max() <= FT_TOL * scale
+    tok = int(token.item())
+    # index work: the token is the first maximum of the logits the kernel itself wrote (bit-exact) ...
+    assert tok == int(np.flatnonzero(got == got.max())[0])
+    # ... and, in the oracle's logits, within the tolerance of the oracle's own choice
+    assert want[tok] >= want[want_tok] - 2 * FT_TOL * scale
+    # without the logits output the choice is the same; a second call reuses the workspace (ticket left at zero)
+    _, token2 = eng.first_token(to_dev(x, dev), to_dev(g, dev), to_dev(Wm, dev), want_logits=False)
+    assert int(token2.item()) == tok
+    eng.close()
+
+
+def test_first_token_ties_and_nonfinite(a3mod):
+    m = W.TINY3
+    eng, _, dev = make_engine(a3mod, m)
+    rng = np.random.default_rng(12)
+    d, vocab = m.d_model, 4099
+    x = W.bf16_round(rng.standard_normal(d).astype(np.float32))
+    g = np.ones(d, dtype=np.float32)
+    Wm = W.bf16_round((rng.standard_normal((vocab, d)) * 0.02).astype(np.float32))
+    # plant the same winning row three times: the lowest id wins
+    a = O.round_bf16(O.rmsnorm(x[None].astype(np.float64), g.astype(np.float64), m.rms_eps))[0]
+    win = W.bf16_round((a / np.linalg.norm(a) * 0.5).astype(np.float32))
+    for i in (4000, 17, 2049):
+        Wm[i] = win
+    logits, token = eng.first_token(to_dev(x, dev), to_dev(g, dev), to_dev(Wm, dev))
+    assert int(token.item()) == 17 == O.first_token(x.astype(np.float64), g.astype(np.float64), Wm.astype(np.float64), m.rms_eps, rnd=O.round_bf16)[1]
+    assert eng.device_status() == 0
+    # a non-finite vocabulary row is flagged and never chosen
+    Wm[5] = np.inf
+    _, token = eng.first_token(to_dev(x, dev), to_dev(g, dev), to_dev(Wm, dev))
+    assert int(token.item()) == 17
+    assert eng.device_status() & 2  # A3_DEV_NONFINITE_SCORE
+    # bad arguments
+    with pytest.raises(a3mod.A3Error):
+        eng.first_token(to_dev(x, dev), to_dev(g, dev), to_dev(Wm, dev)[:0])
+    eng.close()
