@@ -392,6 +392,25 @@ def run_a3(args):
     full_prefill_ms = e0.elapsed_time(e1) / len(xs)
     del Kp, Vp, xs
 
+    # ... and the first token itself (final norm, vocabulary projection, greedy choice) on the last question row:
+    # HBM-bound, vocab*d*2 bytes read once; synthetic final-norm gains and vocabulary matrix
+    g = torch.Generator(device=dev)
+    g.manual_seed(7)
+    lm_head = (torch.randn((m.vocab, m.d_model), device=dev, generator=g) * 0.02).to(torch.bfloat16)
+    fnorm = torch.ones(m.d_model, dtype=torch.bfloat16, device=dev)
+    x_last = out["x"][-1]
+    for _ in range(3):
+        eng.first_token(x_last, fnorm, lm_head, want_logits=False)
+    torch.cuda.synchronize()
+    e0.record(stream)
+    for _ in range(10):
+        eng.first_token(x_last, fnorm, lm_head, want_logits=False)
+    e1.record(stream)
+    torch.cuda.synchronize()
+    first_token_ms = e0.elapsed_time(e1) / 10
+    first_token_gbs = m.vocab * m.d_model * 2 / (first_token_ms * 1e-3) / 1e9
+    del lm_head
+
     cpu = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         S = oracle_sample(args.config)
@@ -410,6 +429,10 @@ def run_a3(args):
                                                     f"({sum(t.numel() for w in eng._weights for t in w.values()) * 2 / 2**30:.1f} GiB) and the fused cache"},
                 "request_ms": seconds / args.steps * 1e3,
                 "full_prefill_ms": full_prefill_ms, "speedup_vs_full_prefill": full_prefill_ms / (seconds / args.steps * 1e3),
+                "first_token": {"ms": first_token_ms, "achieved_gbs": first_token_gbs, "frac_of_hbm_peak": first_token_gbs / peaks["hbm_gbs"],
+                                "ttft_fused_ms": seconds / args.steps * 1e3 + first_token_ms,
+                                "ttft_full_prefill_ms": full_prefill_ms + first_token_ms,
+                                "ttft_ratio": (full_prefill_ms + first_token_ms) / (seconds / args.steps * 1e3 + first_token_ms)},
                 "algorithmic_tflop_per_request": total_flops / 1e12,
                 "request_tflops": total_flops / (seconds / args.steps) / 1e12,
                 "request_frac_of_sustained_peak": total_flops / (seconds / args.steps) / 1e12 / peaks["bf16_tflops_sustained"],
