@@ -410,6 +410,7 @@ def fuse_request(
     rnd: Callable = identity,
     forced_Re: Optional[np.ndarray] = None,
     keep_trace: bool = False,
+    scores_from_cached_keys: bool = False,
 ) -> FuseResult:
     """Attention-aware fusion of independently prefilled chunk caches (Method section).
 
@@ -418,6 +419,14 @@ def fuse_request(
     x0: [n][d] embeddings of the whole input X = (S, D, Q); the last n_question rows
     are the question.  `forced_Re` replaces the selection (used by tests that pin
     both sides to one index set).
+
+    scores_from_cached_keys: the cheaper reading of the Attention Recovery subsection.
+    The text obtains Q_true, K_true at layer 1 by passing the whole input through
+    block 0; here only the question rows are passed through the leading blocks (over
+    the position-recovered cache), their queries are scored against the recovered
+    cached keys K' of the selection layer, and rows [Re, Q] are then recomputed
+    through every layer from the embeddings (Eq. 5 from l = 0), since no true hidden
+    state of Re exists at the selection layer.
     """
     L = model.n_layers
     n = x0.shape[0]
@@ -432,6 +441,30 @@ def fuse_request(
     # position recovery (Eq. 2)
     K, V = position_recovery(chunk_k, chunk_v, offsets, n, model, dtype, rnd)
     stamps.append(("position_recovery", time.perf_counter()))
+
+    if scores_from_cached_keys:
+        q_rows = np.arange(n_ctx, n)
+        Xq = x0[q_rows].astype(dtype)
+        for l in range(select_layer):
+            Xq = recompute_layer(Xq, q_rows, weights[l], model, K[l], V[l], rnd)
+        w = weights[select_layer]
+        a = rnd(rmsnorm(Xq, w.attn_norm, model.rms_eps))
+        q_q, k_q, v_q = project_qkv(a, w, model, q_rows, rnd)
+        K[select_layer][q_rows] = k_q
+        V[select_layer][q_rows] = v_q
+        s = query_scores(q_q, q_rows, K[select_layer], model, cand_begin, cand_end)
+        p = recompute_count(ratio, n, cand_end - cand_begin)
+        Re = topk_select(s, cand_begin, cand_end, p) if forced_Re is None else np.asarray(forced_Re, dtype=np.int64)
+        R = np.concatenate([Re, q_rows]).astype(np.int64)
+        stamps.append(("selection", time.perf_counter()))
+        X = x0[R].astype(dtype)
+        for l in range(L):
+            if keep_trace:
+                trace[f"x_in_{l}"] = X.copy()
+            X = recompute_layer(X, R, weights[l], model, K[l], V[l], rnd)
+            stamps.append((f"recompute_{l}", time.perf_counter()))
+        trace["seconds"] = {name: t - stamps[i][1] for i, (name, t) in enumerate(stamps[1:])}
+        return FuseResult(K=K, V=V, Re=Re, R=R, scores=s, X=X, trace=trace)
 
     # embedding + leading decoder blocks over the whole input -> true states at the selection layer
     X = x0.astype(dtype)

@@ -409,3 +409,45 @@ def test_first_token_matches_library_and_planted_row():
     W3[7] = W3[400] = W2[321]
     assert O.first_token(x, g, W3, eps)[1] == 7
     np.testing.assert_allclose(O.first_token(4.0 * x, g, Wm, 0.0)[0], O.first_token(x, g, Wm, 0.0)[0], rtol=1e-12)
+
+
+# ------------------------------------------------------------------ scores from the cached keys (cheaper reading)
+
+
+@pytest.mark.parametrize("select_layer", [0, 1, 2])
+def test_cached_key_scores_ratio_one_is_full_prefill(tiny3, select_layer):
+    m, r, model, weights, x0, ck, cv, Kv, Vv, Xv = tiny3
+    res = O.fuse_request(ck, cv, x0, r.n_question, weights, model, ratio=1.0, select_layer=select_layer, scores_from_cached_keys=True)
+    assert res.Re.tolist() == list(range(r.n_ctx))
+    np.testing.assert_allclose(res.K, Kv, atol=1e-9)
+    np.testing.assert_allclose(res.V, Vv, atol=1e-9)
+    np.testing.assert_allclose(res.X, Xv, atol=1e-8)
+
+
+def test_cached_key_scores_single_chunk_equals_literal_reading():
+    """With one chunk at offset 0 its cache is exact at every layer, so the cached keys are the true keys: both
+    readings give the same scores, the same selection and the same fused cache (= the full prefill)."""
+    m = W.TINY3
+    r = W.RequestShape((40,), 6, 0.25, 1)
+    model, weights, x0, ck, cv = make_request(m, r, seed=3, emb_std=1.0, w_std=0.05)
+    lit = O.fuse_request(ck, cv, x0, r.n_question, weights, model, ratio=r.ratio, select_layer=1)
+    che = O.fuse_request(ck, cv, x0, r.n_question, weights, model, ratio=r.ratio, select_layer=1, scores_from_cached_keys=True)
+    np.testing.assert_allclose(che.scores, lit.scores, atol=1e-10)
+    assert che.Re.tolist() == lit.Re.tolist()
+    Kv, Vv, _ = O.full_prefill(x0, weights, model)
+    np.testing.assert_allclose(che.K, Kv, atol=1e-9)
+    np.testing.assert_allclose(che.V, Vv, atol=1e-9)
+
+
+def test_cached_key_scores_differ_from_literal_with_several_chunks(tiny3):
+    """Several chunks: the cached keys of later chunks lack the cross-chunk attention, so the scores move - but the
+    rows outside R still hold the position-recovered values and the score mass stays bounded by |Q| * Hq."""
+    m, r, model, weights, x0, ck, cv, Kv, Vv, Xv = tiny3
+    che = O.fuse_request(ck, cv, x0, r.n_question, weights, model, ratio=r.ratio, select_layer=1, scores_from_cached_keys=True)
+    lit = O.fuse_request(ck, cv, x0, r.n_question, weights, model, ratio=r.ratio, select_layer=1)
+    assert np.abs(che.scores - lit.scores).max() > 1e-6
+    assert 0 < che.scores.sum() <= r.n_question * m.n_q_heads + 1e-9
+    Kf, Vf = O.position_recovery(ck, cv, r.offsets, r.n, model)
+    keep = np.setdiff1d(np.arange(r.n), che.R)
+    np.testing.assert_array_equal(che.K[:, keep], Kf[:, keep])
+    np.testing.assert_array_equal(che.V[:, keep], Vf[:, keep])
