@@ -85,6 +85,16 @@ typedef struct {
   int32_t token_step;         /* additional rotation per token index: 0, +1 or -1 (see above) */
 } a3_chunk_ref;
 
+/* Which keys the relevance scores (Eq. 3) are taken against.
+ * A3_SCORES_TRUE_KEYS: the Attention Recovery subsection as written - the whole input passes through the blocks
+ *   below select_layer, K_true of every row is formed at select_layer, rows [Re, Q] are recomputed from there on.
+ * A3_SCORES_CACHED_KEYS: only the question rows pass through the leading blocks (over the position-recovered
+ *   cache); their queries are scored against the recovered cached keys of select_layer; rows [Re, Q] are then
+ *   recomputed through every layer from the embeddings.  Skips the full blocks (about 15 % of the work at
+ *   10 x 512 tokens, r = 0.15); not supported by a3_fuse_request_host. */
+#define A3_SCORES_TRUE_KEYS 0
+#define A3_SCORES_CACHED_KEYS 1
+
 /* One fusion request.  Slots [0, n_ctx) are the chunks in input order, [n_ctx, n_ctx+n_question)
  * the question.  Slots [0, n_system) (a system prompt) are attendable but never candidates. */
 typedef struct {
@@ -93,7 +103,7 @@ typedef struct {
   int32_t n_ctx, n_question, n_system;
   int32_t select_layer;       /* layer whose true Q/K give the scores (paper: 1) */
   int32_t n_recompute;        /* p = |Re| (a3_recompute_count) */
-  int32_t reserved;
+  int32_t score_source;       /* A3_SCORES_TRUE_KEYS (0, the paper's text) or A3_SCORES_CACHED_KEYS */
   const void* x0;             /* dev [n][d_model]: embeddings of the whole input */
   void* k_fused;              /* dev [n_layers][n][Hkv][D], layer l at + l*layer_stride */
   void* v_fused;

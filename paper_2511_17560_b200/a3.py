@@ -51,7 +51,7 @@ class ChunkRef(C.Structure):
 class Request(C.Structure):
     _fields_ = [("chunks", C.c_void_p), ("n_chunks", C.c_int32), ("max_chunk_len", C.c_int32), ("n_ctx", C.c_int32),
                 ("n_question", C.c_int32), ("n_system", C.c_int32), ("select_layer", C.c_int32),
-                ("n_recompute", C.c_int32), ("reserved", C.c_int32), ("x0", C.c_void_p), ("k_fused", C.c_void_p),
+                ("n_recompute", C.c_int32), ("score_source", C.c_int32), ("x0", C.c_void_p), ("k_fused", C.c_void_p),
                 ("v_fused", C.c_void_p), ("layer_stride", C.c_uint64), ("forced_re", C.c_void_p),
                 ("rows_out", C.c_void_p), ("scores_out", C.c_void_p), ("x_out", C.c_void_p)]
 
@@ -288,7 +288,7 @@ class A3:
         return logits, token
 
     def make_request(self, chunks, n_chunks, max_chunk_len, n_ctx, n_question, x0, k_fused, v_fused, ratio=0.15,
-                     select_layer=1, n_system=0, forced_re=None, n_recompute=None):
+                     select_layer=1, n_system=0, forced_re=None, n_recompute=None, score_source=0):
         """Allocates the outputs and fills an a3_request; returns (Request, dict of output tensors)."""
         n = n_ctx + n_question
         p = recompute_count(ratio, n, n_ctx - n_system) if n_recompute is None else n_recompute
@@ -302,7 +302,7 @@ class A3:
         r = Request()
         r.chunks, r.n_chunks, r.max_chunk_len = _ptr(chunks), n_chunks, max_chunk_len
         r.n_ctx, r.n_question, r.n_system = n_ctx, n_question, n_system
-        r.select_layer, r.n_recompute = select_layer, p
+        r.select_layer, r.n_recompute, r.score_source = select_layer, p, int(score_source)
         r.x0, r.k_fused, r.v_fused = _ptr(x0), _ptr(k_fused), _ptr(v_fused)
         r.layer_stride = k_fused.stride(0) * 2
         r.forced_re = _ptr(forced_re)

@@ -361,6 +361,8 @@ static int a3::fuse_impl(const a3_handle* h, const a3_request* r, void* ws, size
   if (n == 0) return A3_OK;
   if (n > m.max_positions) return A3_EINVAL;
   if (r->select_layer < 0 || r->select_layer >= m.n_layers) return A3_EINVAL;
+  if (r->score_source != A3_SCORES_TRUE_KEYS && r->score_source != A3_SCORES_CACHED_KEYS) return A3_EINVAL;
+  if (r->score_source == A3_SCORES_CACHED_KEYS && layer_ready) return A3_EUNSUPPORTED;
   const int n_cand = r->n_ctx - r->n_system;
   if (r->n_recompute < 0 || r->n_recompute > n_cand) return A3_EINVAL;
   if (!r->x0 || !r->k_fused || !r->v_fused || !r->rows_out || !r->scores_out || !r->x_out) return A3_EINVAL;
@@ -375,6 +377,35 @@ static int a3::fuse_impl(const a3_handle* h, const a3_request* r, void* ws, size
   LayerWs lw = carve_layer_ws(h, n, w.layer);
   auto kl = [&](int l) { return (bf16*)((char*)r->k_fused + (size_t)l * r->layer_stride); };
   auto vl = [&](int l) { return (bf16*)((char*)r->v_fused + (size_t)l * r->layer_stride); };
+
+  if (r->score_source == A3_SCORES_CACHED_KEYS) {
+    // Scores against the recovered cached keys: every layer is position-recovered; only the question rows pass
+    // through the leading blocks; rows [Re, Q] are recomputed through every layer from the embeddings.
+    A3_TRY(a3_rope_rerotate(h, r->chunks, r->n_chunks, r->max_chunk_len, r->k_fused, r->v_fused, r->layer_stride, 0, m.n_layers, stream));
+    A3_TRY(iota_rows(h, w.all_pos, 0, n, st));
+    const int32_t* q_pos = w.all_pos + r->n_ctx;
+    A3_CUDA(cudaMemsetAsync(r->scores_out, 0, (size_t)n * 4, st));
+    if (nq > 0) {
+      bf16* xq = w.x_all;  // [nq][d] scratch for the question rows
+      A3_CUDA(cudaMemcpyAsync(xq, (const bf16*)r->x0 + (size_t)r->n_ctx * m.d_model, (size_t)nq * m.d_model * 2, cudaMemcpyDeviceToDevice, st));
+      for (int l = 0; l < ls; ++l) A3_TRY(recompute_layer_impl(h, l, xq, q_pos, nq, kl(l), vl(l), n, nullptr, lw, st));
+      A3_TRY(rmsnorm_rows(h, xq, (const bf16*)h->layers[ls].attn_norm, m.rms_eps, nq, m.d_model, lw.a, st));
+      A3_TRY(qkv_project(h, ls, lw.a, q_pos, nq, 0, lw.q, kl(ls), vl(ls), n, st));
+      A3_TRY(attention_rows(h, lw.q, q_pos, nq, kl(ls), vl(ls), n, nullptr, w.lse_q, nullptr, 0, st));
+      A3_TRY(scores_pass(h, lw.q, q_pos, nq, kl(ls), n, r->n_system, r->n_ctx, w.lse_q, r->scores_out, st));
+    }
+    if (p > 0) {
+      if (r->forced_re) A3_CUDA(cudaMemcpyAsync(r->rows_out, r->forced_re, (size_t)p * 4, cudaMemcpyDeviceToDevice, st));
+      else A3_TRY(a3_topk_select(h, r->scores_out, r->n_system, r->n_ctx, p, r->rows_out, stream));
+    }
+    A3_TRY(iota_rows(h, r->rows_out + p, r->n_ctx, nq, st));
+    if (M == 0) return A3_OK;
+    A3_TRY(check_rows(h, r->rows_out, M, n, st));
+    A3_TRY(a3_gather_rows(h, r->x0, n, r->rows_out, M, m.d_model, r->x_out, stream));
+    for (int l = 0; l < m.n_layers; ++l)
+      A3_TRY(recompute_layer_impl(h, l, (bf16*)r->x_out, r->rows_out, M, kl(l), vl(l), n, nullptr, lw, st));
+    return A3_OK;
+  }
 
   // Position recovery (Eq. 2) in one launch.  Layers up to the selection layer are skipped: every row of their
   // caches is rewritten with true values below (full blocks; K/V of all rows at the selection layer), so the

@@ -56,22 +56,23 @@ class Setup:
         K = torch.zeros((m.n_layers, r.n, m.n_kv_heads, m.head_dim), dtype=torch.bfloat16, device=self.dev)
         return K, torch.zeros_like(K)
 
-    def run_gpu(self, ratio, select_layer=None, forced=None):
+    def run_gpu(self, ratio, select_layer=None, forced=None, score_source=0):
         r = self.r
         K, V = self.fused_buffers()
         sl = r.select_layer if select_layer is None else select_layer
         fr = None if forced is None else torch.from_numpy(np.asarray(forced, dtype=np.int32)).to(self.dev)
         req, out = self.eng.make_request(self.tab, len(self.dk), max(r.chunk_lens), r.n_ctx, r.n_question, self.dx0, K, V,
-                                         ratio=ratio, select_layer=sl, n_system=self.n_system, forced_re=fr)
+                                         ratio=ratio, select_layer=sl, n_system=self.n_system, forced_re=fr,
+                                         score_source=score_source)
         self.eng.fuse_request(req)
         assert self.eng.device_status() == 0
         return K, V, out
 
-    def run_oracle(self, ratio, select_layer=None, forced=None):
+    def run_oracle(self, ratio, select_layer=None, forced=None, cached_keys=False):
         r = self.r
         sl = r.select_layer if select_layer is None else select_layer
         return O.fuse_request(self.ck, self.cv, self.x0, r.n_question, self.weights, self.model, ratio, select_layer=sl,
-                              n_system=self.n_system, rnd=O.round_bf16, forced_Re=forced)
+                              n_system=self.n_system, rnd=O.round_bf16, forced_Re=forced, scores_from_cached_keys=cached_keys)
 
 
 # "spec": the configurations' own distributions, weights and embeddings N(0, 0.02^2).  "wide": weights N(0, 0.05^2) and
@@ -235,4 +236,50 @@ def test_precompute_chunk_matches_oracle_and_layer_loop(a3mod):
     check_drift(f64(V)[0], Vo[0], "chunk V layer 0", KV_MEAN)
     for l in range(1, m.n_layers):
         check_drift(f64(K)[l], Ko[l], f"chunk K layer {l}", 2 * KV_MEAN)
+    s.eng.close()
+
+
+@pytest.mark.parametrize("config,n_system,select_layer", [("tiny3", 0, 1), ("tiny_gqa", 100, 2), ("tiny_g7", 0, 0)])
+def test_fuse_request_scores_from_cached_keys(a3mod, config, n_system, select_layer):
+    """A3_SCORES_CACHED_KEYS: question rows alone through the leading blocks, scores against the recovered cached
+    keys, rows [Re, Q] recomputed through every layer from the embeddings."""
+    s = Setup(a3mod, config, n_system=n_system, emb_std=0.02, w_std=0.02)
+    m, r = s.m, s.r
+    K, V, out = s.run_gpu(r.ratio, select_layer=select_layer, score_source=1)
+    p = out["p"]
+    rows = out["rows"].cpu().numpy()
+    gs = out["scores"].cpu().numpy().astype(np.float64)
+    Re_gpu = rows[:p]
+    assert rows[p:].tolist() == list(range(r.n_ctx, r.n))
+    assert Re_gpu.tolist() == O.topk_select(gs, n_system, r.n_ctx, p).tolist()
+    ref = s.run_oracle(r.ratio, select_layer=select_layer, cached_keys=True)
+    cand = slice(n_system, r.n_ctx)
+    rel = np.abs(gs[cand] - ref.scores[cand]) / ref.scores[cand]
+    assert rel.max() <= 3e-2, rel.max()
+    assert not gs[:n_system].any() and not gs[r.n_ctx:].any()
+    tau = np.sort(ref.scores[cand])[-p]
+    for i in set(Re_gpu.tolist()) ^ set(ref.Re.tolist()):
+        assert abs(ref.scores[i] - tau) <= 3e-2 * tau
+    ref = s.run_oracle(r.ratio, select_layer=select_layer, forced=Re_gpu, cached_keys=True)
+    gK, gV, gX = f64(K), f64(V), f64(out["x"])
+    for l in range(m.n_layers):
+        gate = KV_MEAN if l == 0 else 2 * KV_MEAN
+        check_drift(gK[l], ref.K[l], f"fused K layer {l}", gate)
+        check_drift(gV[l], ref.V[l], f"fused V layer {l}", gate)
+    # rows outside R hold the re-rotated chunk rows at EVERY layer in this mode, bit for bit
+    Kr, Vr = s.fused_buffers()
+    s.eng.rope_rerotate(s.tab, len(s.dk), max(r.chunk_lens), Kr, Vr)
+    mask = torch.ones(r.n, dtype=torch.bool, device=s.dev)
+    mask[out["rows"].long()] = False
+    assert torch.equal(K[:, mask], Kr[:, mask]) and torch.equal(V[:, mask], Vr[:, mask])
+    check_drift(gX, ref.X, "final hidden rows", 6e-3 * float(np.abs(ref.X).std()) * 2 ** (m.n_layers - 1))
+    # ratio 1 in this mode is the full prefill too: same kernels, same rows, same order as the literal mode
+    # (with a system prompt its rows are never recomputed here, so they keep the stored values instead)
+    if n_system == 0:
+        K1, V1, out1 = s.run_gpu(1.0, select_layer=select_layer, score_source=1)
+        K2, V2, out2 = s.run_gpu(1.0, select_layer=select_layer, score_source=0)
+        assert torch.equal(K1, K2) and torch.equal(V1, V2) and torch.equal(out1["x"], out2["x"])
+    # an unknown source is refused
+    with pytest.raises(a3mod.A3Error):
+        s.run_gpu(r.ratio, score_source=7)
     s.eng.close()
