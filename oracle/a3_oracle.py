@@ -39,7 +39,8 @@ Pins (tests marked "not gpu"): RoPE composition / R(0)=I / norm / the D=4 matrix
 written out by hand; layer-0 and chunk-0 exactness of recovered caches against a
 full prefill; r=1 == full prefill; r=0 == position-recovered concatenation;
 softmax rows sum to one; uniform-key closed form; causality; brute-force top-k;
-nested selections; first-token logits against a library matmul and planted rows.  Whole-request agreement of a deep bf16 stack with this oracle
+nested selections; first-token logits against a library matmul and planted rows;
+eviction votes summing to Eq. 3's scores, brute-force kept sets, capacity >= n keeps all.  Whole-request agreement of a deep bf16 stack with this oracle
 has no pin beyond the oracle itself ("parity unpinned" for that one statement).
 """
 from __future__ import annotations
@@ -357,6 +358,64 @@ def topk_select(s: np.ndarray, cand_begin: int, cand_end: int, k: int) -> np.nda
     k = max(0, min(int(k), cand.size))
     order = sorted(cand.tolist(), key=lambda i: (-float(s[i]), i))
     return np.array(sorted(order[:k]), dtype=np.int64)
+
+
+def eviction_scores(q: np.ndarray, q_pos: np.ndarray, K: np.ndarray, model: Model, cand_begin: int, cand_end: int) -> np.ndarray:
+    """Extension subsection: the attention the question window pays to every cached token, per KV head.
+
+    e[g][i] = sum over question rows j and the query heads h of group g of
+    Softmax_row(q_{j,h} K^T / sqrt(D))[i]; zero outside [cand_begin, cand_end).
+    Summed over g this is s(d_i) of Eq. 3.  (SnapKV votes with the observation window's
+    attention per head; with grouped-query attention the cache has one entry per KV head,
+    so the votes of the heads that share it are added.)
+    """
+    n = K.shape[0]
+    G = model.n_q_heads // model.n_kv_heads
+    e = np.zeros((model.n_kv_heads, n), dtype=q.dtype)
+    for h in range(model.n_q_heads):
+        P = attention_probs(q, q_pos, K, model, h)
+        e[h // G] += P.sum(axis=0)
+    e[:, :cand_begin] = 0
+    e[:, cand_end:] = 0
+    return e
+
+
+def pool_scores(e: np.ndarray, cand_begin: int, cand_end: int, width: int) -> np.ndarray:
+    """SnapKV's clustering step: every candidate takes the maximum of the scores in the window of `width`
+    (odd) candidates centred on it; the window is cut at the candidate range.  width 1 leaves e unchanged."""
+    assert width % 2 == 1
+    hw = width // 2
+    out = np.zeros_like(e)
+    for i in range(cand_begin, cand_end):
+        lo, hi = max(cand_begin, i - hw), min(cand_end, i + hw + 1)
+        out[:, i] = e[:, lo:hi].max(axis=1)
+    return out
+
+
+def evict_layer(q: np.ndarray, q_pos: np.ndarray, K: np.ndarray, V: np.ndarray, model: Model, n_system: int, n_ctx: int,
+                capacity: int, pool: int = 1):
+    """Extension subsection (`ex`): keep the system prompt S and the question Q whole and, per KV head, the
+    top C - |S| - |Q| document tokens by question-window attention (SnapKV's strategy), for one layer.
+
+    q: [|Q|][Hq][D] rotated question queries of this layer at positions q_pos; K, V: [n][Hkv][D].
+    Returns (K_c, V_c, kept): K_c, V_c [C'][Hkv][D] with C' = |S| + k + |Q|, k = clamp(C - |S| - |Q|,
+    0, number of document tokens); kept [Hkv][C'] the source slot of every kept entry, ascending.
+    """
+    n = K.shape[0]
+    nq = n - n_ctx
+    k = max(0, min(n_ctx - n_system, capacity - n_system - nq))
+    e = pool_scores(eviction_scores(q, q_pos, K, model, n_system, n_ctx), n_system, n_ctx, pool)
+    Hkv = model.n_kv_heads
+    C = n_system + k + nq
+    kept = np.zeros((Hkv, C), dtype=np.int64)
+    Kc = np.zeros((C, Hkv, K.shape[2]), dtype=K.dtype)
+    Vc = np.zeros_like(Kc)
+    for g in range(Hkv):
+        sel = topk_select(e[g], n_system, n_ctx, k)
+        kept[g] = np.concatenate([np.arange(n_system), sel, np.arange(n_ctx, n)])
+        Kc[:, g] = K[kept[g], g]
+        Vc[:, g] = V[kept[g], g]
+    return Kc, Vc, kept
 
 
 def first_token(x_last: np.ndarray, final_norm: np.ndarray, lm_head: np.ndarray, eps: float, rnd: Callable = identity):

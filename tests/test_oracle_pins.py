@@ -451,3 +451,75 @@ def test_cached_key_scores_differ_from_literal_with_several_chunks(tiny3):
     keep = np.setdiff1d(np.arange(r.n), che.R)
     np.testing.assert_array_equal(che.K[:, keep], Kf[:, keep])
     np.testing.assert_array_equal(che.V[:, keep], Vf[:, keep])
+
+
+# ------------------------------------------------------------------ `ex`: eviction after fusion (Extension subsection)
+
+
+def _evict_case(seed=9, Hq=8, Hkv=2, D=16, n_system=5, n_ctx=61, nq=7):
+    rng = np.random.default_rng(seed)
+    model = O.Model(1, Hq * D, Hq, Hkv, D, 64)
+    n = n_ctx + nq
+    K = rng.standard_normal((n, Hkv, D))
+    V = rng.standard_normal((n, Hkv, D))
+    q = rng.standard_normal((nq, Hq, D)) * 2.0
+    return model, K, V, q, np.arange(n_ctx, n), n_system, n_ctx, nq
+
+
+def test_eviction_votes_sum_to_eq3_scores_and_heads_are_independent():
+    model, K, V, q, q_pos, ns, nc, nq = _evict_case()
+    e = O.eviction_scores(q, q_pos, K, model, ns, nc)
+    np.testing.assert_allclose(e.sum(axis=0), O.query_scores(q, q_pos, K, model, ns, nc), atol=1e-12)
+    # KV head 1's votes do not depend on KV head 0's keys
+    K2 = K.copy()
+    K2[:, 0] += 1.0
+    np.testing.assert_array_equal(O.eviction_scores(q, q_pos, K2, model, ns, nc)[1], e[1])
+    assert not e[:, :ns].any() and not e[:, nc:].any()
+
+
+def test_eviction_kept_sets_bruteforce_and_edges():
+    model, K, V, q, q_pos, ns, nc, nq = _evict_case()
+    n = nc + nq
+    C = ns + nq + 11
+    Kc, Vc, kept = O.evict_layer(q, q_pos, K, V, model, ns, nc, C)
+    assert Kc.shape == (C, 2, 16) and kept.shape == (2, C)
+    G = model.n_q_heads // model.n_kv_heads
+    scale = 1.0 / math.sqrt(16)
+    for g in range(2):
+        # brute force: softmax rows written out with python loops
+        votes = np.zeros(n)
+        for j in range(nq):
+            for h in range(g * G, (g + 1) * G):
+                logits = np.array([float(q[j, h] @ K[i, g]) * scale for i in range(q_pos[j] + 1)])
+                pr = np.exp(logits - logits.max())
+                pr /= pr.sum()
+                votes[:len(pr)] += pr
+        docs = sorted(range(ns, nc), key=lambda i: (-votes[i], i))[:11]
+        want = list(range(ns)) + sorted(docs) + list(range(nc, n))
+        assert kept[g].tolist() == want
+        np.testing.assert_array_equal(Kc[:, g], K[want, g])
+        np.testing.assert_array_equal(Vc[:, g], V[want, g])
+    assert kept[0].tolist() != kept[1].tolist()  # the heads really choose differently
+    # capacity >= n keeps everything in order; capacity below |S| + |Q| keeps S and Q only
+    Kall, Vall, kall = O.evict_layer(q, q_pos, K, V, model, ns, nc, n + 50)
+    assert kall.tolist() == [list(range(n))] * 2
+    np.testing.assert_array_equal(Kall, K)
+    _, _, kmin = O.evict_layer(q, q_pos, K, V, model, ns, nc, 3)
+    assert kmin.tolist() == [list(range(ns)) + list(range(nc, n))] * 2
+
+
+def test_eviction_pooling_is_a_running_maximum():
+    e = np.zeros((1, 12))
+    e[0, 2:10] = [1, 5, 2, 2, 0, 0, 3, 1]
+    got = O.pool_scores(e, 2, 10, 3)
+    assert got[0].tolist() == [0, 0, 5, 5, 5, 2, 2, 3, 3, 3, 0, 0]
+    np.testing.assert_array_equal(O.pool_scores(e, 2, 10, 1), e)
+    # with pooling the neighbours of a peak are kept with it
+    model, K, V, q, q_pos, ns, nc, nq = _evict_case(seed=4)
+    _, _, kept = O.evict_layer(q, q_pos, K, V, model, ns, nc, ns + nq + 9, pool=3)
+    ev = O.eviction_scores(q, q_pos, K, model, ns, nc)
+    for g in range(2):
+        peak = ns + int(np.argmax(ev[g, ns:nc]))
+        for i in (peak - 1, peak, peak + 1):
+            if ns <= i < nc:
+                assert i in kept[g]
