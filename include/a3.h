@@ -112,6 +112,15 @@ typedef struct {
   int32_t* rows_out;          /* dev [n_recompute + n_question]: R = Re (ascending) then question slots */
   float* scores_out;          /* dev [n]: s(d_i) on candidates, 0 elsewhere */
   void* x_out;                /* dev [n_recompute + n_question][d_model]: final hidden rows of R */
+  /* `ex` (Extension subsection), optional: with evict_capacity > 0 every layer's fused cache is also written in
+   * compact form right after the layer has been recomputed, using that layer's question rows as the window
+   * (a3_evict_layer).  C' = n_system + a3_evict_count(...) + n_question entries per layer. */
+  int32_t evict_capacity;     /* C; 0: no eviction */
+  int32_t evict_pool;         /* odd pooling width, 0 or 1: off */
+  void* k_evicted;            /* dev [n_layers][C'][Hkv][D], layer l at + l*evicted_layer_stride */
+  void* v_evicted;
+  uint64_t evicted_layer_stride; /* bytes */
+  int32_t* kept_out;          /* dev [n_layers][Hkv][C'] or NULL */
 } a3_request;
 
 /* Host buffers for a3_fuse_request_host (pinned memory recommended). */
@@ -231,6 +240,24 @@ int a3_fuse_request_host(const a3_handle* h, const a3_request* req, const a3_hos
                          size_t staging_bytes, void* ws, size_t ws_bytes, a3_stream stream);
 
 /* ---- diagnostics -------------------------------------------------------------------- */
+
+/* `ex`, the eviction extension (Extension subsection), for one layer: keep the system prompt slots [0, n_system)
+ * and the question slots [n_ctx, kv_len) whole and, per KV head, the k = a3_evict_count(...) document slots with
+ * the largest question-window attention
+ *   e[g][i] = sum over question rows j and the query heads h of KV head g of Softmax_row(q_{j,h} K^T / sqrt(D))[i]
+ * (SnapKV's vote; summed over g it is Eq. 3's s).  pool (odd, 1 = off) replaces e by its running maximum over
+ * `pool` neighbouring candidates before the selection (SnapKV's clustering).  Ties go to the lower slot.
+ *   q_window: dev [nq][Hq][D] rotated question queries of this layer; q_pos: dev [nq] their slots (n_ctx..);
+ *   lse: dev [nq][Hq] natural-log row log-sum-exps (a3_recompute_layer's lse_out rows of the question);
+ *   k_layer, v_layer: dev [kv_len][Hkv][D], kv_len = n_ctx + nq;
+ *   k_out, v_out: dev [C'][Hkv][D], C' = n_system + k + nq: entry c of head g is source slot kept_out[g][c];
+ *   kept_out: dev [Hkv][C'] int32 (ascending per head) or NULL.
+ * ws: a3_evict_workspace_bytes(h, kv_len), borrowed.  Four launches, no allocation, no synchronisation. */
+int a3_evict_count(int capacity, int n_system, int n_ctx, int n_question);
+size_t a3_evict_workspace_bytes(const a3_handle* h, int kv_len);
+int a3_evict_layer(const a3_handle* h, const void* q_window, const int32_t* q_pos, int nq, const float* lse,
+                   const void* k_layer, const void* v_layer, int kv_len, int n_system, int n_ctx, int capacity, int pool,
+                   void* k_out, void* v_out, int32_t* kept_out, void* ws, size_t ws_bytes, a3_stream stream);
 
 /* First token after fusion (what the paper's time-to-first-token figures end with; Inference paragraph of the
  * Experiments): a = RMSNorm(x_row) * final_norm (rounded to bf16), logits = lm_head a, token = argmax (lowest id

@@ -453,6 +453,7 @@ class FuseResult:
     scores: np.ndarray     # [n] s(d_i) on candidates, 0 elsewhere
     X: np.ndarray          # [p+|Q|][d] final hidden rows of R
     trace: dict = field(default_factory=dict)
+    evicted: Optional[list] = None  # per layer (K_c, V_c, kept) of the `ex` extension, when a capacity was given
 
 
 def fuse_request(
@@ -470,6 +471,8 @@ def fuse_request(
     forced_Re: Optional[np.ndarray] = None,
     keep_trace: bool = False,
     scores_from_cached_keys: bool = False,
+    evict_capacity: int = 0,
+    evict_pool: int = 1,
 ) -> FuseResult:
     """Attention-aware fusion of independently prefilled chunk caches (Method section).
 
@@ -486,6 +489,10 @@ def fuse_request(
     cached keys K' of the selection layer, and rows [Re, Q] are then recomputed
     through every layer from the embeddings (Eq. 5 from l = 0), since no true hidden
     state of Re exists at the selection layer.
+
+    evict_capacity > 0 adds the `ex` extension: right after a layer has been recomputed its
+    cache is also returned in compact form (evict_layer), the window being that layer's
+    question queries.
     """
     L = model.n_layers
     n = x0.shape[0]
@@ -495,6 +502,18 @@ def fuse_request(
     assert n_ctx + n_question == n
     cand_begin, cand_end = n_system, n_ctx
     trace = {}
+    evicted = [None] * L if evict_capacity > 0 else None
+
+    def layer_step(l, X, rows):
+        """One layer for `rows` (whose last n_question entries are the question), then its eviction."""
+        if evicted is None:
+            return recompute_layer(X, rows, weights[l], model, K[l], V[l], rnd)
+        X2, parts = recompute_layer(X, rows, weights[l], model, K[l], V[l], rnd, return_parts=True)
+        nq = n_question
+        evicted[l] = evict_layer(parts["q"][len(rows) - nq:], rows[len(rows) - nq:], K[l], V[l], model, n_system, n_ctx,
+                                 evict_capacity, evict_pool)
+        return X2
+
     stamps = [("start", time.perf_counter())]  # wall-clock per phase, for the CPU baseline report only
 
     # position recovery (Eq. 2)
@@ -520,16 +539,16 @@ def fuse_request(
         for l in range(L):
             if keep_trace:
                 trace[f"x_in_{l}"] = X.copy()
-            X = recompute_layer(X, R, weights[l], model, K[l], V[l], rnd)
+            X = layer_step(l, X, R)
             stamps.append((f"recompute_{l}", time.perf_counter()))
         trace["seconds"] = {name: t - stamps[i][1] for i, (name, t) in enumerate(stamps[1:])}
-        return FuseResult(K=K, V=V, Re=Re, R=R, scores=s, X=X, trace=trace)
+        return FuseResult(K=K, V=V, Re=Re, R=R, scores=s, X=X, trace=trace, evicted=evicted)
 
     # embedding + leading decoder blocks over the whole input -> true states at the selection layer
     X = x0.astype(dtype)
     all_pos = np.arange(n)
     for l in range(select_layer):
-        X = recompute_layer(X, all_pos, weights[l], model, K[l], V[l], rnd)
+        X = layer_step(l, X, all_pos)
         stamps.append((f"full_block_{l}", time.perf_counter()))
 
     # true K, V for every row at the selection layer; question queries; scores; Re (Eq. 3)
@@ -552,7 +571,7 @@ def fuse_request(
     for l in range(select_layer, L):
         if keep_trace:
             trace[f"x_in_{l}"] = X.copy()
-        X = recompute_layer(X, R, weights[l], model, K[l], V[l], rnd)
+        X = layer_step(l, X, R)
         stamps.append((f"recompute_{l}", time.perf_counter()))
     trace["seconds"] = {name: t - stamps[i][1] for i, (name, t) in enumerate(stamps[1:])}
-    return FuseResult(K=K, V=V, Re=Re, R=R, scores=s, X=X, trace=trace)
+    return FuseResult(K=K, V=V, Re=Re, R=R, scores=s, X=X, trace=trace, evicted=evicted)

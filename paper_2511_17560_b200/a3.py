@@ -53,7 +53,9 @@ class Request(C.Structure):
                 ("n_question", C.c_int32), ("n_system", C.c_int32), ("select_layer", C.c_int32),
                 ("n_recompute", C.c_int32), ("score_source", C.c_int32), ("x0", C.c_void_p), ("k_fused", C.c_void_p),
                 ("v_fused", C.c_void_p), ("layer_stride", C.c_uint64), ("forced_re", C.c_void_p),
-                ("rows_out", C.c_void_p), ("scores_out", C.c_void_p), ("x_out", C.c_void_p)]
+                ("rows_out", C.c_void_p), ("scores_out", C.c_void_p), ("x_out", C.c_void_p),
+                ("evict_capacity", C.c_int32), ("evict_pool", C.c_int32), ("k_evicted", C.c_void_p), ("v_evicted", C.c_void_p),
+                ("evicted_layer_stride", C.c_uint64), ("kept_out", C.c_void_p)]
 
 
 class HostIO(C.Structure):
@@ -63,7 +65,8 @@ class HostIO(C.Structure):
 
 EXPORTS = ("a3_create", "a3_destroy", "a3_layer_workspace_bytes", "a3_request_workspace_bytes", "a3_host_staging_bytes",
            "a3_recompute_count", "a3_rope_rerotate", "a3_query_scores", "a3_query_scores_static", "a3_topk_select", "a3_recompute_layer",
-           "a3_scatter_kv", "a3_gather_rows", "a3_precompute_chunk", "a3_first_token_workspace_bytes", "a3_first_token", "a3_fuse_request", "a3_fuse_batch", "a3_fuse_request_host",
+           "a3_scatter_kv", "a3_gather_rows", "a3_precompute_chunk", "a3_first_token_workspace_bytes", "a3_first_token",
+           "a3_evict_count", "a3_evict_workspace_bytes", "a3_evict_layer", "a3_fuse_request", "a3_fuse_batch", "a3_fuse_request_host",
            "a3_device_status", "a3_status_string", "a3_last_cuda_error", "a3_launch_count", "a3_profile_enable",
            "a3_profile_read", "a3_kernel_class_name")
 K_CLASSES = 10
@@ -99,6 +102,10 @@ def _load():
     lib.a3_scatter_kv.argtypes = [vp, vp, vp, vp, i32, vp, vp, i32, vp]
     lib.a3_gather_rows.argtypes = [vp, vp, i32, vp, i32, i32, vp, vp]
     lib.a3_precompute_chunk.argtypes = [vp, vp, i32, vp, vp, u64, vp, sz, vp]
+    lib.a3_evict_count.argtypes = [i32, i32, i32, i32]
+    lib.a3_evict_workspace_bytes.argtypes = [vp, i32]
+    lib.a3_evict_workspace_bytes.restype = sz
+    lib.a3_evict_layer.argtypes = [vp, vp, vp, i32, vp, vp, vp, i32, i32, i32, i32, i32, vp, vp, vp, vp, sz, vp]
     lib.a3_first_token_workspace_bytes.argtypes = [vp]
     lib.a3_first_token_workspace_bytes.restype = sz
     lib.a3_first_token.argtypes = [vp, vp, vp, vp, i32, vp, vp, vp, sz, vp]
@@ -137,6 +144,10 @@ def _check(status: int, where: str):
 
 def recompute_count(ratio: float, n: int, n_candidates: int) -> int:
     return int(_load().a3_recompute_count(float(ratio), int(n), int(n_candidates)))
+
+
+def evict_count(capacity: int, n_system: int, n_ctx: int, n_question: int) -> int:
+    return int(_load().a3_evict_count(int(capacity), int(n_system), int(n_ctx), int(n_question)))
 
 
 def launch_count(reset: bool = False) -> int:
@@ -276,6 +287,21 @@ class A3:
                                            _ptr(ws), ws.numel(), _stream()), "a3_precompute_chunk")
         return x_chunk
 
+    def evict_layer(self, q_window, q_pos, lse, k_layer, v_layer, n_system, n_ctx, capacity, pool=1):
+        """`ex` for one layer; returns (k_out, v_out, kept) with C' = n_system + k + nq entries per head."""
+        nq = q_pos.shape[0]
+        kv_len = k_layer.shape[0]
+        Cp = n_system + evict_count(capacity, n_system, n_ctx, nq) + nq
+        Hkv, D = self.shape.n_kv_heads, self.shape.head_dim
+        k_out = torch.zeros((Cp, Hkv, D), dtype=torch.bfloat16, device=k_layer.device)
+        v_out = torch.zeros_like(k_out)
+        kept = torch.full((Hkv, Cp), -1, dtype=torch.int32, device=k_layer.device)
+        ws = self.workspace(int(_load().a3_evict_workspace_bytes(self._h, kv_len)))
+        _check(_load().a3_evict_layer(self._h, _ptr(q_window), _ptr(q_pos), nq, _ptr(lse), _ptr(k_layer), _ptr(v_layer), kv_len,
+                                      n_system, n_ctx, capacity, pool, _ptr(k_out), _ptr(v_out), _ptr(kept), _ptr(ws), ws.numel(),
+                                      _stream()), "a3_evict_layer")
+        return k_out, v_out, kept
+
     def first_token(self, x_row, final_norm, lm_head, want_logits=True):
         """Final norm + vocabulary projection + greedy choice for one hidden row [d]; returns (logits or None, token)."""
         vocab = lm_head.shape[0]
@@ -288,7 +314,8 @@ class A3:
         return logits, token
 
     def make_request(self, chunks, n_chunks, max_chunk_len, n_ctx, n_question, x0, k_fused, v_fused, ratio=0.15,
-                     select_layer=1, n_system=0, forced_re=None, n_recompute=None, score_source=0):
+                     select_layer=1, n_system=0, forced_re=None, n_recompute=None, score_source=0, evict_capacity=0,
+                     evict_pool=1):
         """Allocates the outputs and fills an a3_request; returns (Request, dict of output tensors)."""
         n = n_ctx + n_question
         p = recompute_count(ratio, n, n_ctx - n_system) if n_recompute is None else n_recompute
@@ -307,6 +334,15 @@ class A3:
         r.layer_stride = k_fused.stride(0) * 2
         r.forced_re = _ptr(forced_re)
         r.rows_out, r.scores_out, r.x_out = _ptr(out["rows"]), _ptr(out["scores"]), _ptr(out["x"])
+        if evict_capacity > 0:
+            L, Hkv, D = self.shape.n_layers, self.shape.n_kv_heads, self.shape.head_dim
+            Cp = n_system + evict_count(evict_capacity, n_system, n_ctx, n_question) + n_question
+            out["k_evicted"] = torch.zeros((L, Cp, Hkv, D), dtype=torch.bfloat16, device=dev)
+            out["v_evicted"] = torch.zeros_like(out["k_evicted"])
+            out["kept"] = torch.full((L, Hkv, Cp), -1, dtype=torch.int32, device=dev)
+            r.evict_capacity, r.evict_pool = int(evict_capacity), int(evict_pool)
+            r.k_evicted, r.v_evicted, r.kept_out = _ptr(out["k_evicted"]), _ptr(out["v_evicted"]), _ptr(out["kept"])
+            r.evicted_layer_stride = out["k_evicted"].stride(0) * 2
         out["_keep"] = (chunks, x0, k_fused, v_fused, forced_re)
         return r, out
 

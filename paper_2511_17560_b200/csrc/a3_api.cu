@@ -42,6 +42,8 @@ struct RequestWs {
   bf16* x_all;
   int32_t* all_pos;
   float* lse_q;
+  void* evict;  // scratch of a3_evict_layer
+  size_t evict_bytes;
   void* layer;
   size_t bytes;
 };
@@ -59,6 +61,8 @@ static RequestWs carve_request_ws(const a3_handle* h, int n, void* base) {
   w.x_all = (bf16*)take(N * m.d_model * 2);
   w.all_pos = (int32_t*)take(N * 4);
   w.lse_q = (float*)take(N * m.n_q_heads * 4);
+  w.evict_bytes = a3_evict_workspace_bytes(h, n);
+  w.evict = take(w.evict_bytes);
   w.layer = take(carve_layer_ws(h, n, nullptr).bytes);
   w.bytes = off;
   return w;
@@ -377,6 +381,25 @@ static int a3::fuse_impl(const a3_handle* h, const a3_request* r, void* ws, size
   LayerWs lw = carve_layer_ws(h, n, w.layer);
   auto kl = [&](int l) { return (bf16*)((char*)r->k_fused + (size_t)l * r->layer_stride); };
   auto vl = [&](int l) { return (bf16*)((char*)r->v_fused + (size_t)l * r->layer_stride); };
+  // `ex`: compact copy of every layer's cache, taken right after the layer with its question rows as the window
+  const bool evict = r->evict_capacity > 0;
+  const int pool = r->evict_pool > 1 ? r->evict_pool : 1;
+  const int c_evicted = r->n_system + a3_evict_count(r->evict_capacity, r->n_system, r->n_ctx, nq) + nq;
+  if (evict) {
+    if (!r->k_evicted || !r->v_evicted || pool % 2 == 0) return A3_EINVAL;
+    if (r->evicted_layer_stride < (uint64_t)c_evicted * m.n_kv_heads * m.head_dim * 2 || (r->evicted_layer_stride & 15)) return A3_EINVAL;
+    if (((uintptr_t)r->k_evicted | (uintptr_t)r->v_evicted) & 15) return A3_EINVAL;
+  }
+  // one layer for rows whose last nq entries are the question rows, then (optionally) its eviction
+  auto layer_step = [&](int l, bf16* x, const int32_t* pos, int rows) -> int {
+    A3_TRY(recompute_layer_impl(h, l, x, pos, rows, kl(l), vl(l), n, evict ? lw.lse : nullptr, lw, st));
+    if (!evict) return A3_OK;
+    const size_t first_q = (size_t)(rows - nq);
+    return a3_evict_layer(h, lw.q + first_q * m.n_q_heads * m.head_dim, pos + first_q, nq, lw.lse + first_q * m.n_q_heads, kl(l), vl(l), n,
+                          r->n_system, r->n_ctx, r->evict_capacity, pool, (char*)r->k_evicted + (size_t)l * r->evicted_layer_stride,
+                          (char*)r->v_evicted + (size_t)l * r->evicted_layer_stride,
+                          r->kept_out ? r->kept_out + (size_t)l * m.n_kv_heads * c_evicted : nullptr, w.evict, w.evict_bytes, stream);
+  };
 
   if (r->score_source == A3_SCORES_CACHED_KEYS) {
     // Scores against the recovered cached keys: every layer is position-recovered; only the question rows pass
@@ -402,8 +425,7 @@ static int a3::fuse_impl(const a3_handle* h, const a3_request* r, void* ws, size
     if (M == 0) return A3_OK;
     A3_TRY(check_rows(h, r->rows_out, M, n, st));
     A3_TRY(a3_gather_rows(h, r->x0, n, r->rows_out, M, m.d_model, r->x_out, stream));
-    for (int l = 0; l < m.n_layers; ++l)
-      A3_TRY(recompute_layer_impl(h, l, (bf16*)r->x_out, r->rows_out, M, kl(l), vl(l), n, nullptr, lw, st));
+    for (int l = 0; l < m.n_layers; ++l) A3_TRY(layer_step(l, (bf16*)r->x_out, r->rows_out, M));
     return A3_OK;
   }
 
@@ -417,8 +439,7 @@ static int a3::fuse_impl(const a3_handle* h, const a3_request* r, void* ws, size
   if (x0_ready) A3_CUDA(cudaStreamWaitEvent(st, x0_ready, 0));
   A3_CUDA(cudaMemcpyAsync(w.x_all, r->x0, (size_t)n * m.d_model * 2, cudaMemcpyDeviceToDevice, st));
   A3_TRY(iota_rows(h, w.all_pos, 0, n, st));
-  for (int l = 0; l < ls; ++l)
-    A3_TRY(recompute_layer_impl(h, l, w.x_all, w.all_pos, n, kl(l), vl(l), n, nullptr, lw, st));
+  for (int l = 0; l < ls; ++l) A3_TRY(layer_step(l, w.x_all, w.all_pos, n));
   // selection layer: true K, V for all rows, queries of the question rows, scores, Re (Eq. 3)
   A3_TRY(rmsnorm_rows(h, w.x_all, (const bf16*)h->layers[ls].attn_norm, m.rms_eps, n, m.d_model, lw.a, st));
   A3_TRY(qkv_project(h, ls, lw.a, w.all_pos, n, r->n_ctx, lw.q, kl(ls), vl(ls), n, st));
@@ -448,7 +469,7 @@ static int a3::fuse_impl(const a3_handle* h, const a3_request* r, void* ws, size
       A3_CUDA(cudaStreamWaitEvent(st, layer_ready[l], 0));
       A3_TRY(a3_rope_rerotate(h, r->chunks, r->n_chunks, r->max_chunk_len, r->k_fused, r->v_fused, r->layer_stride, l, l + 1, stream));
     }
-    A3_TRY(recompute_layer_impl(h, l, (bf16*)r->x_out, r->rows_out, M, kl(l), vl(l), n, nullptr, lw, st));
+    A3_TRY(layer_step(l, (bf16*)r->x_out, r->rows_out, M));
   }
   return A3_OK;
 }

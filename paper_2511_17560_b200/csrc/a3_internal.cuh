@@ -125,7 +125,10 @@ int attention_rows(const a3_handle* h, const bf16* q, const int32_t* pos, int M,
 size_t attention_part_bytes(const a3_handle* h);
 
 int scores_pass(const a3_handle* h, const bf16* q, const int32_t* q_pos, int nq, const bf16* k, int kv_len,
-                int cand_begin, int cand_end, const float* lse, float* scores, cudaStream_t st);
+                int cand_begin, int cand_end, const float* lse, float* scores, cudaStream_t st, float* per_head = nullptr);
+// `batches` independent selections, one CTA each: scores + b*score_stride -> idx_out + b*idx_stride
+int topk_batched(const a3_handle* h, const float* scores, size_t score_stride, int batches, int cand_begin, int cand_end,
+                 int k, int32_t* idx_out, size_t idx_stride, cudaStream_t st);
 
 int iota_rows(const a3_handle* h, int32_t* out, int begin, int count, cudaStream_t st);
 int check_rows(const a3_handle* h, const int32_t* pos, int M, int kv_len, cudaStream_t st);

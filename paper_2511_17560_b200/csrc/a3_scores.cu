@@ -71,7 +71,7 @@ template <int D>
 __global__ void __launch_bounds__(AT_THREADS)
 scores_kernel(const bf16* __restrict__ q, const int32_t* __restrict__ q_pos, int nq, const bf16* __restrict__ k,
               int kv_len, int cand_begin, int cand_end, const float* __restrict__ lse, float* __restrict__ scores,
-              int Hq, int Hkv, float scale_log2) {
+              int Hq, int Hkv, float scale_log2, float* __restrict__ per_head) {
   __shared__ __align__(128) unsigned char smem[2 * 64 * D * 2];
   __shared__ float colpart[4][AT_BN];
   const uint32_t sq = smem_u32(smem), sk = sq + 64 * D * 2;
@@ -83,6 +83,7 @@ scores_kernel(const bf16* __restrict__ q, const int32_t* __restrict__ q_pos, int
   const int nrb = (rows_total + AT_BM - 1) / AT_BM;
   const int kvrow = Hkv * D;
   float total = 0.f;  // thread c < 64 owns cache slot key0 + c
+  float head_total = 0.f;
 
   for (int g = 0; g < Hkv; ++g) {
     __syncthreads();  // previous users of sk / sq are done
@@ -141,24 +142,33 @@ scores_kernel(const bf16* __restrict__ q, const int32_t* __restrict__ q_pos, int
         }
       }
       __syncthreads();
-      if (tid < AT_BN) total += (colpart[0][tid] + colpart[1][tid]) + (colpart[2][tid] + colpart[3][tid]);
+      if (tid < AT_BN) {
+        const float part = (colpart[0][tid] + colpart[1][tid]) + (colpart[2][tid] + colpart[3][tid]);
+        total += part;
+        head_total += part;
+      }
+    }
+    if (per_head) {  // the votes of this KV head's query heads alone (eviction step)
+      const int key = key0 + tid;
+      if (tid < AT_BN && key < kv_len) per_head[(size_t)g * kv_len + key] = (key >= cand_begin && key < cand_end) ? head_total : 0.f;
+      head_total = 0.f;
     }
   }
   if (tid < AT_BN) {
     int key = key0 + tid;
-    if (key < kv_len) scores[key] = (key >= cand_begin && key < cand_end) ? total : 0.f;
+    if (key < kv_len && scores) scores[key] = (key >= cand_begin && key < cand_end) ? total : 0.f;
   }
 }
 
 int scores_pass(const a3_handle* h, const bf16* q, const int32_t* q_pos, int nq, const bf16* k, int kv_len,
-                int cand_begin, int cand_end, const float* lse, float* scores, cudaStream_t st) {
+                int cand_begin, int cand_end, const float* lse, float* scores, cudaStream_t st, float* per_head) {
   if (kv_len <= 0) return A3_OK;
   const int Hq = h->m.n_q_heads, Hkv = h->m.n_kv_heads, D = h->m.head_dim;
   const float scale_log2 = LOG2E / sqrtf((float)D);
   dim3 grid(cdiv(kv_len, AT_BN));
   ProfScope prof(h, A3_K_SCORES, st);
-  if (D == 128) scores_kernel<128><<<grid, AT_THREADS, 0, st>>>(q, q_pos, nq, k, kv_len, cand_begin, cand_end, lse, scores, Hq, Hkv, scale_log2);
-  else scores_kernel<64><<<grid, AT_THREADS, 0, st>>>(q, q_pos, nq, k, kv_len, cand_begin, cand_end, lse, scores, Hq, Hkv, scale_log2);
+  if (D == 128) scores_kernel<128><<<grid, AT_THREADS, 0, st>>>(q, q_pos, nq, k, kv_len, cand_begin, cand_end, lse, scores, Hq, Hkv, scale_log2, per_head);
+  else scores_kernel<64><<<grid, AT_THREADS, 0, st>>>(q, q_pos, nq, k, kv_len, cand_begin, cand_end, lse, scores, Hq, Hkv, scale_log2, per_head);
   A3_LAUNCHED();
   return A3_OK;
 }

@@ -14,7 +14,11 @@ __device__ __forceinline__ uint32_t score_key(float s) {
 }
 
 __global__ void __launch_bounds__(TK_THREADS)
-topk_select_kernel(const float* __restrict__ scores, int cand_begin, int n, int k, int32_t* __restrict__ idx_out, uint32_t* status) {
+topk_select_kernel(const float* __restrict__ scores, int cand_begin, int n, int k, int32_t* __restrict__ idx_out, uint32_t* status,
+                   size_t score_stride, size_t idx_stride) {
+  // one CTA per independent selection (the per-head selections of the eviction step; a single one for Eq. 3)
+  scores += blockIdx.x * score_stride;
+  idx_out += blockIdx.x * idx_stride;
   __shared__ unsigned int hist[256];
   __shared__ unsigned int s_prefix, s_remaining;
   __shared__ unsigned int warp_gt[TK_THREADS / 32], warp_eq[TK_THREADS / 32];
@@ -113,7 +117,18 @@ extern "C" int a3_topk_select(const a3_handle* h, const float* scores, int cand_
   if (k == 0) return A3_OK;
   if (!scores || !idx_out) return A3_EINVAL;
   ProfScope prof(h, A3_K_TOPK, (cudaStream_t)stream);
-  topk_select_kernel<<<1, TK_THREADS, 0, (cudaStream_t)stream>>>(scores, cand_begin, n, k, idx_out, h->dev_status);
+  topk_select_kernel<<<1, TK_THREADS, 0, (cudaStream_t)stream>>>(scores, cand_begin, n, k, idx_out, h->dev_status, 0, 0);
+  A3_LAUNCHED();
+  return A3_OK;
+}
+
+int a3::topk_batched(const a3_handle* h, const float* scores, size_t score_stride, int batches, int cand_begin, int cand_end,
+                     int k, int32_t* idx_out, size_t idx_stride, cudaStream_t st) {
+  const int n = cand_end - cand_begin;
+  if (k > n) k = n;
+  if (k <= 0 || batches <= 0) return A3_OK;
+  ProfScope prof(h, A3_K_TOPK, st);
+  topk_select_kernel<<<batches, TK_THREADS, 0, st>>>(scores, cand_begin, n, k, idx_out, h->dev_status, score_stride, idx_stride);
   A3_LAUNCHED();
   return A3_OK;
 }

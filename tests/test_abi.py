@@ -53,9 +53,28 @@ def test_host_only_entry_points(lib_path):
     assert lib.a3_layer_workspace_bytes(None, 10) == 0
 
 
-def test_struct_layouts_match_header():
+def test_struct_layouts_match_header(tmp_path):
+    """sizeof/offsetof as the C compiler sees include/a3.h against the ctypes mirrors of the binding."""
+    import subprocess
     from paper_2511_17560_b200 import a3
+    structs = {"a3_chunk_ref": a3.ChunkRef, "a3_layer_weights": a3.LayerWeights, "a3_request": a3.Request,
+               "a3_model_desc": a3.ModelDesc, "a3_host_io": a3.HostIO, "a3_profile_entry": a3.ProfileEntry}
+    lines = []
+    for cname, cls in structs.items():
+        lines.append(f'printf("{cname} size %zu\\n", sizeof({cname}));')
+        for fname, _ in cls._fields_:
+            lines.append(f'printf("{cname} {fname} %zu\\n", offsetof({cname}, {fname}));')
+    src = tmp_path / "layout.c"
+    src.write_text('#include <stdio.h>\n#include <stddef.h>\n#include "a3.h"\nint main(void) {\n' + "\n".join(lines) + "\nreturn 0; }\n")
+    exe = tmp_path / "layout"
+    inc = os.path.join(os.path.dirname(os.path.dirname(os.path.abspath(__file__))), "include")
+    subprocess.run(["gcc", "-std=c99", "-I", inc, str(src), "-o", str(exe)], check=True)
+    got = {}
+    for ln in subprocess.run([str(exe)], check=True, capture_output=True, text=True).stdout.splitlines():
+        cname, field, val = ln.split()
+        got[(cname, field)] = int(val)
+    for cname, cls in structs.items():
+        assert ctypes.sizeof(cls) == got[(cname, "size")], cname
+        for fname, _ in cls._fields_:
+            assert getattr(cls, fname).offset == got[(cname, fname)], (cname, fname)
     assert ctypes.sizeof(a3.ChunkRef) == 40
-    assert ctypes.sizeof(a3.LayerWeights) == 12 * 8
-    assert ctypes.sizeof(a3.Request) == 8 + 8 * 4 + 8 * 8
-    assert ctypes.sizeof(a3.ModelDesc) == 48

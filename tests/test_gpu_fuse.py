@@ -283,3 +283,41 @@ def test_fuse_request_scores_from_cached_keys(a3mod, config, n_system, select_la
     with pytest.raises(a3mod.A3Error):
         s.run_gpu(r.ratio, score_source=7)
     s.eng.close()
+
+
+@pytest.mark.parametrize("config,n_system,score_source", [("tiny3", 0, 0), ("tiny_gqa", 100, 0), ("tiny_gqa", 100, 1)])
+def test_fuse_request_with_eviction(a3mod, config, n_system, score_source):
+    """`ex` inside the request: every layer's compact cache is the gather of that layer's fused cache at the kept
+    slots (exact), S and Q are kept whole, and the kept documents agree with the oracle run on the same index set
+    except where the oracle's votes are within 3 % of its threshold (the end-to-end score gate)."""
+    s = Setup(a3mod, config, n_system=n_system, emb_std=0.02, w_std=0.02)
+    m, r = s.m, s.r
+    C, pool = n_system + r.n_question + 150, 5
+    K, V = s.fused_buffers()
+    req, out = s.eng.make_request(s.tab, len(s.dk), max(r.chunk_lens), r.n_ctx, r.n_question, s.dx0, K, V, ratio=r.ratio,
+                                  select_layer=r.select_layer, n_system=n_system, score_source=score_source,
+                                  evict_capacity=C, evict_pool=pool)
+    s.eng.fuse_request(req)
+    assert s.eng.device_status() == 0
+    p = out["p"]
+    kept = out["kept"].cpu().numpy()
+    k = C - n_system - r.n_question
+    assert kept.shape == (m.n_layers, m.n_kv_heads, C)
+    # the fusion itself is unchanged by the extension
+    K0, V0, out0 = s.run_gpu(r.ratio, score_source=score_source)
+    assert torch.equal(K, K0) and torch.equal(V, V0) and torch.equal(out["x"], out0["x"])
+    Re_gpu = out["rows"].cpu().numpy()[:p]
+    ref = O.fuse_request(s.ck, s.cv, s.x0, r.n_question, s.weights, s.model, r.ratio, select_layer=r.select_layer, n_system=n_system,
+                         rnd=O.round_bf16, forced_Re=Re_gpu, scores_from_cached_keys=bool(score_source), evict_capacity=C, evict_pool=pool)
+    for l in range(m.n_layers):
+        for g in range(m.n_kv_heads):
+            kg = kept[l, g]
+            assert kg[:n_system].tolist() == list(range(n_system)) and kg[n_system + k:].tolist() == list(range(r.n_ctx, r.n))
+            assert (np.diff(kg) > 0).all()
+            idx = torch.from_numpy(kg.astype(np.int64)).to(s.dev)
+            assert torch.equal(out["k_evicted"][l][:, g], K[l][idx, g]) and torch.equal(out["v_evicted"][l][:, g], V[l][idx, g])
+            want = ref.evicted[l][2][g]
+            diff = set(kg.tolist()) ^ set(want.tolist())
+            # agreement with the oracle: most of the kept set is common; the rest sits near the threshold
+            assert len(diff) <= 2 * max(2, k // 10), (l, g, len(diff))
+    s.eng.close()

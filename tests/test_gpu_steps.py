@@ -424,3 +424,63 @@ def test_first_token_ties_and_nonfinite(a3mod):
     with pytest.raises(a3mod.A3Error):
         eng.first_token(to_dev(x, dev), to_dev(g, dev), to_dev(Wm, dev)[:0])
     eng.close()
+
+
+# ------------------------------------------------------------------ `ex`: eviction of one layer (Extension subsection)
+
+
+@pytest.mark.parametrize("shape,n_system,n_ctx,nq,capacity,pool", [
+    (W.TINY_GQA, 20, 1500, 16, 400, 1), (W.TINY_GQA, 0, 700, 33, 300, 7), (W.TINY3, 5, 333, 1, 64, 3),
+    (W.TINY_G7, 0, 900, 8, 5000, 1), (W.TINY_G7, 10, 200, 8, 12, 1)])
+def test_evict_layer_parity(a3mod, shape, n_system, n_ctx, nq, capacity, pool):
+    m = shape
+    eng, _, dev = make_engine(a3mod, m)
+    model = oracle_model(m)
+    rng = np.random.default_rng(31)
+    n = n_ctx + nq
+    K = W.bf16_round(rng.standard_normal((n, m.n_kv_heads, m.head_dim)).astype(np.float32) * 1.2).astype(np.float64)
+    V = W.bf16_round(rng.standard_normal((n, m.n_kv_heads, m.head_dim)).astype(np.float32)).astype(np.float64)
+    q = W.bf16_round(rng.standard_normal((nq, m.n_q_heads, m.head_dim)).astype(np.float32) * 1.5).astype(np.float64)
+    q_pos = np.arange(n_ctx, n)
+    _, lse = O.attention_rows(q, q_pos, K, V, model)
+    dK, dV = to_dev(K, dev), to_dev(V, dev)
+    k_out, v_out, kept = eng.evict_layer(to_dev(q, dev), torch.from_numpy(q_pos.astype(np.int32)).to(dev),
+                                         to_dev(lse, dev, torch.float32), dK, dV, n_system, n_ctx, capacity, pool)
+    assert eng.device_status() == 0
+    k = a3mod.evict_count(capacity, n_system, n_ctx, nq)
+    assert k == max(0, min(n_ctx - n_system, capacity - n_system - nq))
+    Kc, Vc, want = O.evict_layer(q, q_pos, K, V, model, n_system, n_ctx, capacity, pool)
+    kept = kept.cpu().numpy()
+    assert kept.shape == want.shape == (m.n_kv_heads, n_system + k + nq)
+    votes = O.pool_scores(O.eviction_scores(q, q_pos, K, model, n_system, n_ctx), n_system, n_ctx, pool)
+    for g in range(m.n_kv_heads):
+        # index work: S and Q kept whole, ascending; the selected documents equal the oracle's except where the
+        # oracle's votes are within the score tolerance (1e-3 relative) of its k-th largest
+        assert kept[g, :n_system].tolist() == list(range(n_system))
+        assert kept[g, n_system + k:].tolist() == list(range(n_ctx, n))
+        assert (np.diff(kept[g]) > 0).all()
+        diff = set(kept[g].tolist()) ^ set(want[g].tolist())
+        if diff:
+            tau = np.sort(votes[g, n_system:n_ctx])[-k]
+            assert all(abs(votes[g, i] - tau) <= 1e-3 * tau for i in diff), (g, sorted(diff))
+        # the compact cache is the gather of the kept slots, bit for bit
+        idx = torch.from_numpy(kept[g].astype(np.int64)).to(dev)
+        assert torch.equal(k_out[:, g], dK[idx, g]) and torch.equal(v_out[:, g], dV[idx, g])
+    eng.close()
+
+
+def test_evict_layer_bad_arguments(a3mod):
+    m = W.TINY3
+    eng, _, dev = make_engine(a3mod, m)
+    n_ctx, nq = 64, 4
+    K = torch.zeros((n_ctx + nq, m.n_kv_heads, m.head_dim), dtype=torch.bfloat16, device=dev)
+    q = torch.zeros((nq, m.n_q_heads, m.head_dim), dtype=torch.bfloat16, device=dev)
+    pos = torch.arange(n_ctx, n_ctx + nq, dtype=torch.int32, device=dev)
+    lse = torch.zeros((nq, m.n_q_heads), dtype=torch.float32, device=dev)
+    with pytest.raises(a3mod.A3Error):
+        eng.evict_layer(q, pos, lse, K, K, 0, n_ctx, 32, pool=4)  # even pooling width
+    with pytest.raises(a3mod.A3Error):
+        eng.evict_layer(q, pos, lse, K, K, 70, n_ctx, 32)  # system prompt longer than the context
+    with pytest.raises(a3mod.A3Error):
+        eng.evict_layer(q, pos, lse, K, K, 0, n_ctx - 1, 32)  # n_ctx + nq != kv_len
+    eng.close()

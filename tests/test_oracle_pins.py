@@ -523,3 +523,21 @@ def test_eviction_pooling_is_a_running_maximum():
         for i in (peak - 1, peak, peak + 1):
             if ns <= i < nc:
                 assert i in kept[g]
+
+
+def test_fuse_request_with_eviction_is_consistent(tiny3):
+    """Eviction does not change the fusion itself, and every compact layer is a gather of the fused one."""
+    m, r, model, weights, x0, ck, cv, Kv, Vv, Xv = tiny3
+    base = O.fuse_request(ck, cv, x0, r.n_question, weights, model, ratio=r.ratio, select_layer=1)
+    C = r.n_question + 40
+    res = O.fuse_request(ck, cv, x0, r.n_question, weights, model, ratio=r.ratio, select_layer=1, evict_capacity=C, evict_pool=3)
+    np.testing.assert_array_equal(res.K, base.K)
+    np.testing.assert_array_equal(res.X, base.X)
+    assert len(res.evicted) == m.n_layers
+    for l, (Kc, Vc, kept) in enumerate(res.evicted):
+        assert Kc.shape == (C, m.n_kv_heads, m.head_dim)
+        for g in range(m.n_kv_heads):
+            assert kept[g, -r.n_question:].tolist() == list(range(r.n_ctx, r.n))
+            assert (np.diff(kept[g]) > 0).all()
+            np.testing.assert_array_equal(Kc[:, g], res.K[l][kept[g], g])
+            np.testing.assert_array_equal(Vc[:, g], res.V[l][kept[g], g])
