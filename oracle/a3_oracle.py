@@ -349,6 +349,30 @@ def query_scores(q: np.ndarray, q_pos: np.ndarray, K: np.ndarray, model: Model, 
     return s
 
 
+def value_deviation_scores(V_true: np.ndarray, V_cached: np.ndarray, cand_begin: int, cand_end: int) -> np.ndarray:
+    """The selector the paper compares against (Baselines, CacheBlend): a token's score is the squared
+    distance between its concatenated (cached) value and its ground-truth value at the selection layer,
+    summed over KV heads and channels.  V_true, V_cached: [n][Hkv][D]; zero outside the candidates."""
+    dvi = V_true - V_cached
+    s = (dvi * dvi).sum(axis=(1, 2))
+    s[:cand_begin] = 0
+    s[cand_end:] = 0
+    return s
+
+
+def chunk_edge_rows(chunk_lens: Sequence[int], m: int, n_system: int = 0) -> np.ndarray:
+    """The other selector of the comparison (Baselines, LegoLink; Details: the first and last 20 tokens of
+    each chunk): slots of the first m and last m tokens of every chunk, ascending, system prompt slots left out."""
+    rows = []
+    o = 0
+    for t in chunk_lens:
+        for i in range(t):
+            if (i < m or i >= t - m) and o + i >= n_system:
+                rows.append(o + i)
+        o += t
+    return np.array(rows, dtype=np.int64)
+
+
 def topk_select(s: np.ndarray, cand_begin: int, cand_end: int, k: int) -> np.ndarray:
     """Re = top_p(s): the k candidate slots with the largest score (Eq. 3).
 
@@ -473,6 +497,7 @@ def fuse_request(
     scores_from_cached_keys: bool = False,
     evict_capacity: int = 0,
     evict_pool: int = 1,
+    selector: str = "attention",
 ) -> FuseResult:
     """Attention-aware fusion of independently prefilled chunk caches (Method section).
 
@@ -489,6 +514,11 @@ def fuse_request(
     cached keys K' of the selection layer, and rows [Re, Q] are then recomputed
     through every layer from the embeddings (Eq. 5 from l = 0), since no true hidden
     state of Re exists at the selection layer.
+
+    selector: "attention" is Eq. 3; "value_deviation" ranks the candidates by the distance between
+    cached and true values at the selection layer instead (the comparison method of the Baselines
+    paragraph), everything else unchanged.  Index-only selectors (chunk edges, random) go through
+    forced_Re.
 
     evict_capacity > 0 adds the `ex` extension: right after a layer has been recomputed its
     cache is also returned in compact form (evict_layer), the window being that layer's
@@ -521,6 +551,7 @@ def fuse_request(
     stamps.append(("position_recovery", time.perf_counter()))
 
     if scores_from_cached_keys:
+        assert selector == "attention"  # no true values exist in this mode
         q_rows = np.arange(n_ctx, n)
         Xq = x0[q_rows].astype(dtype)
         for l in range(select_layer):
@@ -555,10 +586,15 @@ def fuse_request(
     w = weights[select_layer]
     a = rnd(rmsnorm(X, w.attn_norm, model.rms_eps))
     q_all, k_all, v_all = project_qkv(a, w, model, all_pos, rnd)
+    V_cached = V[select_layer].copy()
     K[select_layer][:] = k_all
     V[select_layer][:] = v_all
     q_rows = np.arange(n_ctx, n)
-    s = query_scores(q_all[q_rows], q_rows, K[select_layer], model, cand_begin, cand_end)
+    if selector == "value_deviation":
+        s = value_deviation_scores(V[select_layer], V_cached, cand_begin, cand_end)
+    else:
+        assert selector == "attention"
+        s = query_scores(q_all[q_rows], q_rows, K[select_layer], model, cand_begin, cand_end)
     p = recompute_count(ratio, n, cand_end - cand_begin)
     Re = topk_select(s, cand_begin, cand_end, p) if forced_Re is None else np.asarray(forced_Re, dtype=np.int64)
     R = np.concatenate([Re, q_rows]).astype(np.int64)

@@ -541,3 +541,34 @@ def test_fuse_request_with_eviction_is_consistent(tiny3):
             assert (np.diff(kept[g]) > 0).all()
             np.testing.assert_array_equal(Kc[:, g], res.K[l][kept[g], g])
             np.testing.assert_array_equal(Vc[:, g], res.V[l][kept[g], g])
+
+
+# ------------------------------------------------------------------ the comparison selectors (Baselines paragraph)
+
+
+def test_value_deviation_selector(tiny3):
+    m, r, model, weights, x0, ck, cv, Kv, Vv, Xv = tiny3
+    res = O.fuse_request(ck, cv, x0, r.n_question, weights, model, ratio=r.ratio, select_layer=1, selector="value_deviation")
+    # the score is the squared distance between the cached and the full-prefill value at layer 1 ...
+    _, Vf = O.position_recovery(ck, cv, r.offsets, r.n, model)
+    want = ((Vv[1] - Vf[1]) ** 2).sum(axis=(1, 2))
+    want[r.n_ctx:] = 0
+    np.testing.assert_allclose(res.scores, want, atol=1e-12)
+    # ... which vanishes on the first chunk (its cache is exact) and not on the later ones
+    first = r.chunk_lens[0]
+    assert res.scores[:first].max() < 1e-18 and res.scores[first:r.n_ctx].min() > 1e-12
+    assert not set(res.Re.tolist()) & set(range(first))
+    # the selection is the brute-force top-p of it, and the rest of the path is unchanged: forcing the same rows
+    # through the attention path gives the same cache
+    p = O.recompute_count(r.ratio, r.n, r.n_ctx)
+    assert res.Re.tolist() == sorted(sorted(range(r.n_ctx), key=lambda i: (-want[i], i))[:p])
+    same = O.fuse_request(ck, cv, x0, r.n_question, weights, model, ratio=r.ratio, select_layer=1, forced_Re=res.Re)
+    np.testing.assert_array_equal(same.K, res.K)
+    np.testing.assert_array_equal(same.V, res.V)
+
+
+def test_chunk_edge_rows():
+    assert O.chunk_edge_rows((5, 3, 10), 2).tolist() == [0, 1, 3, 4, 5, 6, 7, 8, 9, 16, 17]
+    assert O.chunk_edge_rows((5, 3, 10), 2, n_system=5).tolist() == [5, 6, 7, 8, 9, 16, 17]
+    assert O.chunk_edge_rows((512,) * 10, 20).size == 400
+    assert O.chunk_edge_rows((4,), 20).tolist() == [0, 1, 2, 3]
