@@ -95,6 +95,14 @@ typedef struct {
 #define A3_SCORES_TRUE_KEYS 0
 #define A3_SCORES_CACHED_KEYS 1
 
+/* What ranks the candidates.  A3_SELECT_ATTENTION is Eq. 3.  A3_SELECT_VALUE_DEVIATION is the comparison method
+ * of the Baselines paragraph (CacheBlend): score = squared distance between a token's cached value and its true
+ * value at select_layer, over all KV heads and channels (needs A3_SCORES_TRUE_KEYS, which forms the true values);
+ * scores_out then holds these distances.  Index-only selections (chunk edges - a3_chunk_edge_rows -, random) are
+ * passed through forced_re. */
+#define A3_SELECT_ATTENTION 0
+#define A3_SELECT_VALUE_DEVIATION 1
+
 /* One fusion request.  Slots [0, n_ctx) are the chunks in input order, [n_ctx, n_ctx+n_question)
  * the question.  Slots [0, n_system) (a system prompt) are attendable but never candidates. */
 typedef struct {
@@ -104,6 +112,8 @@ typedef struct {
   int32_t select_layer;       /* layer whose true Q/K give the scores (paper: 1) */
   int32_t n_recompute;        /* p = |Re| (a3_recompute_count) */
   int32_t score_source;       /* A3_SCORES_TRUE_KEYS (0, the paper's text) or A3_SCORES_CACHED_KEYS */
+  int32_t selector;           /* A3_SELECT_ATTENTION (0, Eq. 3) or A3_SELECT_VALUE_DEVIATION */
+  int32_t reserved;
   const void* x0;             /* dev [n][d_model]: embeddings of the whole input */
   void* k_fused;              /* dev [n_layers][n][Hkv][D], layer l at + l*layer_stride */
   void* v_fused;
@@ -148,6 +158,11 @@ size_t a3_layer_workspace_bytes(const a3_handle* h, int max_rows);
 size_t a3_request_workspace_bytes(const a3_handle* h, int n);
 /* Additional device staging bytes a3_fuse_request_host needs. */
 size_t a3_host_staging_bytes(const a3_handle* h, int n_ctx, int n);
+
+/* Slots of the first m and last m tokens of every chunk, ascending, without slots below n_system (the comparison
+ * method of the Baselines paragraph, LegoLink: m = 20).  chunk_len: host [n_chunks].  Writes at most `capacity`
+ * slots to rows_out (host; may be NULL) and returns the full count.  Host only. */
+int a3_chunk_edge_rows(const int32_t* chunk_len, int n_chunks, int m, int n_system, int32_t* rows_out, int capacity);
 
 /* p = min(n_candidates, floor(ratio * n + 1e-9)): the size of Re (Eq. 3, p = r n). Host only. */
 int a3_recompute_count(double ratio, int n, int n_candidates);

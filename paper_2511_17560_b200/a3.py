@@ -51,7 +51,7 @@ class ChunkRef(C.Structure):
 class Request(C.Structure):
     _fields_ = [("chunks", C.c_void_p), ("n_chunks", C.c_int32), ("max_chunk_len", C.c_int32), ("n_ctx", C.c_int32),
                 ("n_question", C.c_int32), ("n_system", C.c_int32), ("select_layer", C.c_int32),
-                ("n_recompute", C.c_int32), ("score_source", C.c_int32), ("x0", C.c_void_p), ("k_fused", C.c_void_p),
+                ("n_recompute", C.c_int32), ("score_source", C.c_int32), ("selector", C.c_int32), ("reserved", C.c_int32), ("x0", C.c_void_p), ("k_fused", C.c_void_p),
                 ("v_fused", C.c_void_p), ("layer_stride", C.c_uint64), ("forced_re", C.c_void_p),
                 ("rows_out", C.c_void_p), ("scores_out", C.c_void_p), ("x_out", C.c_void_p),
                 ("evict_capacity", C.c_int32), ("evict_pool", C.c_int32), ("k_evicted", C.c_void_p), ("v_evicted", C.c_void_p),
@@ -66,7 +66,7 @@ class HostIO(C.Structure):
 EXPORTS = ("a3_create", "a3_destroy", "a3_layer_workspace_bytes", "a3_request_workspace_bytes", "a3_host_staging_bytes",
            "a3_recompute_count", "a3_rope_rerotate", "a3_query_scores", "a3_query_scores_static", "a3_topk_select", "a3_recompute_layer",
            "a3_scatter_kv", "a3_gather_rows", "a3_precompute_chunk", "a3_first_token_workspace_bytes", "a3_first_token",
-           "a3_evict_count", "a3_evict_workspace_bytes", "a3_evict_layer", "a3_fuse_request", "a3_fuse_batch", "a3_fuse_request_host",
+           "a3_evict_count", "a3_evict_workspace_bytes", "a3_evict_layer", "a3_chunk_edge_rows", "a3_fuse_request", "a3_fuse_batch", "a3_fuse_request_host",
            "a3_device_status", "a3_status_string", "a3_last_cuda_error", "a3_launch_count", "a3_profile_enable",
            "a3_profile_read", "a3_kernel_class_name")
 K_CLASSES = 10
@@ -102,6 +102,7 @@ def _load():
     lib.a3_scatter_kv.argtypes = [vp, vp, vp, vp, i32, vp, vp, i32, vp]
     lib.a3_gather_rows.argtypes = [vp, vp, i32, vp, i32, i32, vp, vp]
     lib.a3_precompute_chunk.argtypes = [vp, vp, i32, vp, vp, u64, vp, sz, vp]
+    lib.a3_chunk_edge_rows.argtypes = [C.POINTER(C.c_int32), i32, i32, i32, C.POINTER(C.c_int32), i32]
     lib.a3_evict_count.argtypes = [i32, i32, i32, i32]
     lib.a3_evict_workspace_bytes.argtypes = [vp, i32]
     lib.a3_evict_workspace_bytes.restype = sz
@@ -144,6 +145,15 @@ def _check(status: int, where: str):
 
 def recompute_count(ratio: float, n: int, n_candidates: int) -> int:
     return int(_load().a3_recompute_count(float(ratio), int(n), int(n_candidates)))
+
+
+def chunk_edge_rows(chunk_lens: Sequence[int], m: int, n_system: int = 0) -> np.ndarray:
+    """Slots of the first/last m tokens of every chunk (ascending), for use as forced_re."""
+    lens = (C.c_int32 * max(1, len(chunk_lens)))(*[int(t) for t in chunk_lens])
+    count = int(_load().a3_chunk_edge_rows(lens, len(chunk_lens), int(m), int(n_system), None, 0))
+    out = (C.c_int32 * max(1, count))()
+    _load().a3_chunk_edge_rows(lens, len(chunk_lens), int(m), int(n_system), out, count)
+    return np.frombuffer(out, dtype=np.int32, count=count).copy()
 
 
 def evict_count(capacity: int, n_system: int, n_ctx: int, n_question: int) -> int:
@@ -315,7 +325,7 @@ class A3:
 
     def make_request(self, chunks, n_chunks, max_chunk_len, n_ctx, n_question, x0, k_fused, v_fused, ratio=0.15,
                      select_layer=1, n_system=0, forced_re=None, n_recompute=None, score_source=0, evict_capacity=0,
-                     evict_pool=1):
+                     evict_pool=1, selector=0):
         """Allocates the outputs and fills an a3_request; returns (Request, dict of output tensors)."""
         n = n_ctx + n_question
         p = recompute_count(ratio, n, n_ctx - n_system) if n_recompute is None else n_recompute
@@ -330,6 +340,7 @@ class A3:
         r.chunks, r.n_chunks, r.max_chunk_len = _ptr(chunks), n_chunks, max_chunk_len
         r.n_ctx, r.n_question, r.n_system = n_ctx, n_question, n_system
         r.select_layer, r.n_recompute, r.score_source = select_layer, p, int(score_source)
+        r.selector = int(selector)
         r.x0, r.k_fused, r.v_fused = _ptr(x0), _ptr(k_fused), _ptr(v_fused)
         r.layer_stride = k_fused.stride(0) * 2
         r.forced_re = _ptr(forced_re)

@@ -92,6 +92,23 @@ extern "C" uint64_t a3_launch_count(int reset) {
   return v;
 }
 
+extern "C" int a3_chunk_edge_rows(const int32_t* chunk_len, int n_chunks, int m, int n_system, int32_t* rows_out, int capacity) {
+  if (!chunk_len || n_chunks <= 0 || m <= 0) return 0;
+  int count = 0, o = 0;
+  for (int c = 0; c < n_chunks; ++c) {
+    const int t = chunk_len[c] > 0 ? chunk_len[c] : 0;
+    for (int i = 0; i < t; ++i) {
+      if ((i < m || i >= t - m) && o + i >= n_system) {
+        if (rows_out && count < capacity) rows_out[count] = o + i;
+        ++count;
+      }
+      if (i == m - 1 && t - m > m) i = t - m - 1;  // jump over the middle of a long chunk
+    }
+    o += t;
+  }
+  return count;
+}
+
 extern "C" int a3_recompute_count(double ratio, int n, int n_candidates) {
   if (n_candidates <= 0 || n <= 0 || !(ratio > 0.0)) return 0;
   double p = floor(ratio * (double)n + 1e-9);
@@ -367,6 +384,9 @@ static int a3::fuse_impl(const a3_handle* h, const a3_request* r, void* ws, size
   if (r->select_layer < 0 || r->select_layer >= m.n_layers) return A3_EINVAL;
   if (r->score_source != A3_SCORES_TRUE_KEYS && r->score_source != A3_SCORES_CACHED_KEYS) return A3_EINVAL;
   if (r->score_source == A3_SCORES_CACHED_KEYS && layer_ready) return A3_EUNSUPPORTED;
+  if (r->selector != A3_SELECT_ATTENTION && r->selector != A3_SELECT_VALUE_DEVIATION) return A3_EINVAL;
+  // the value-deviation selector compares true with cached values: it needs the true ones and device-resident chunks
+  if (r->selector == A3_SELECT_VALUE_DEVIATION && (r->score_source != A3_SCORES_TRUE_KEYS || layer_ready)) return A3_EUNSUPPORTED;
   const int n_cand = r->n_ctx - r->n_system;
   if (r->n_recompute < 0 || r->n_recompute > n_cand) return A3_EINVAL;
   if (!r->x0 || !r->k_fused || !r->v_fused || !r->rows_out || !r->scores_out || !r->x_out) return A3_EINVAL;
@@ -444,7 +464,9 @@ static int a3::fuse_impl(const a3_handle* h, const a3_request* r, void* ws, size
   A3_TRY(rmsnorm_rows(h, w.x_all, (const bf16*)h->layers[ls].attn_norm, m.rms_eps, n, m.d_model, lw.a, st));
   A3_TRY(qkv_project(h, ls, lw.a, w.all_pos, n, r->n_ctx, lw.q, kl(ls), vl(ls), n, st));
   A3_CUDA(cudaMemsetAsync(r->scores_out, 0, (size_t)n * 4, st));
-  if (nq > 0) {
+  if (r->selector == A3_SELECT_VALUE_DEVIATION) {
+    A3_TRY(value_deviation(h, r->chunks, r->n_chunks, r->max_chunk_len, ls, vl(ls), r->n_system, r->n_ctx, r->scores_out, st));
+  } else if (nq > 0) {
     A3_TRY(attention_rows(h, lw.q, w.all_pos + r->n_ctx, nq, kl(ls), vl(ls), n, nullptr, w.lse_q, nullptr, 0, st));
     A3_TRY(scores_pass(h, lw.q, w.all_pos + r->n_ctx, nq, kl(ls), n, r->n_system, r->n_ctx, w.lse_q, r->scores_out, st));
   }

@@ -130,6 +130,9 @@ int scores_pass(const a3_handle* h, const bf16* q, const int32_t* q_pos, int nq,
 int topk_batched(const a3_handle* h, const float* scores, size_t score_stride, int batches, int cand_begin, int cand_end,
                  int k, int32_t* idx_out, size_t idx_stride, cudaStream_t st);
 
+// scores[slot] = |v_true[slot] - cached value of that slot|^2 for candidate slots covered by a chunk (others untouched)
+int value_deviation(const a3_handle* h, const a3_chunk_ref* chunks, int n_chunks, int max_chunk_len, int layer, const bf16* v_true,
+                    int cand_begin, int cand_end, float* scores, cudaStream_t st);
 int iota_rows(const a3_handle* h, int32_t* out, int begin, int count, cudaStream_t st);
 int check_rows(const a3_handle* h, const int32_t* pos, int M, int kv_len, cudaStream_t st);
 

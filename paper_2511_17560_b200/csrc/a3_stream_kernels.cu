@@ -222,6 +222,52 @@ extern "C" int a3_rope_rerotate(const a3_handle* h, const a3_chunk_ref* chunks, 
   return A3_OK;
 }
 
+// ------------------------------------------------------------------ value deviation (comparison selector)
+namespace a3 {
+
+// scores[o_c + t] = sum over KV heads and channels of (v_true[o_c + t] - v_cached_c[t])^2 for candidate slots.
+// grid: (token tiles of the longest chunk, chunk); one warp per token, 16-byte loads, fp32 accumulation in a
+// fixed order (lane-strided partial sums, then a shuffle tree): deterministic.
+__global__ void __launch_bounds__(256)
+value_deviation_kernel(const a3_chunk_ref* __restrict__ chunks, int layer, const uint4* __restrict__ v_true, int row_vecs, int cand_begin,
+                       int cand_end, float* __restrict__ scores) {
+  const a3_chunk_ref ch = chunks[blockIdx.y];
+  const int t = blockIdx.x * 8 + (threadIdx.x >> 5);
+  if (t >= ch.len) return;
+  const int slot = ch.dst_offset + t;
+  if (slot < cand_begin || slot >= cand_end) return;
+  const int lane = threadIdx.x & 31;
+  const uint4* a = v_true + (size_t)slot * row_vecs;
+  const uint4* b = reinterpret_cast<const uint4*>((const char*)ch.v_src + (size_t)layer * ch.src_layer_stride) + (size_t)t * row_vecs;
+  float acc = 0.f;
+  for (int v = lane; v < row_vecs; v += 32) {
+    float fa[8], fb[8];
+    unpack8(__ldg(a + v), fa);
+    unpack8(__ldcs(b + v), fb);
+#pragma unroll
+    for (int e = 0; e < 8; ++e) {
+      const float d = fa[e] - fb[e];
+      acc = fmaf(d, d, acc);
+    }
+  }
+#pragma unroll
+  for (int o = 16; o; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
+  if (lane == 0) scores[slot] = acc;
+}
+
+int value_deviation(const a3_handle* h, const a3_chunk_ref* chunks, int n_chunks, int max_chunk_len, int layer, const bf16* v_true,
+                    int cand_begin, int cand_end, float* scores, cudaStream_t st) {
+  if (n_chunks <= 0 || max_chunk_len <= 0) return A3_OK;
+  if (n_chunks > 65535) return A3_EUNSUPPORTED;
+  ProfScope prof(h, A3_K_SCORES, st);
+  value_deviation_kernel<<<dim3(cdiv(max_chunk_len, 8), n_chunks), 256, 0, st>>>(chunks, layer, (const uint4*)v_true,
+                                                                                 h->m.n_kv_heads * h->m.head_dim / 8, cand_begin, cand_end, scores);
+  A3_LAUNCHED();
+  return A3_OK;
+}
+
+}  // namespace a3
+
 // ------------------------------------------------------------------ scatter / gather
 namespace a3 {
 

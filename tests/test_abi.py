@@ -78,3 +78,20 @@ def test_struct_layouts_match_header(tmp_path):
         for fname, _ in cls._fields_:
             assert getattr(cls, fname).offset == got[(cname, fname)], (cname, fname)
     assert ctypes.sizeof(a3.ChunkRef) == 40
+
+
+def test_host_only_helpers_match_oracle():
+    """a3_chunk_edge_rows, a3_recompute_count and a3_evict_count are host arithmetic: no GPU needed."""
+    import numpy as np
+    from oracle import a3_oracle as O
+    from paper_2511_17560_b200 import a3
+    rng = np.random.default_rng(0)
+    for _ in range(50):
+        lens = rng.integers(0, 90, size=rng.integers(1, 9)).tolist()
+        m = int(rng.integers(1, 30))
+        ns = int(rng.integers(0, max(1, lens[0] + 1)))
+        assert a3.chunk_edge_rows(lens, m, ns).tolist() == O.chunk_edge_rows(lens, m, ns).tolist()
+    assert a3.chunk_edge_rows((512,) * 10, 20).size == 400
+    for ratio, n, nc in ((0.15, 5152, 5120), (1.0, 100, 90), (0.0, 10, 10), (0.3, 10, 2), (0.15, 20, 20)):
+        assert a3.recompute_count(ratio, n, nc) == O.recompute_count(ratio, n, nc)
+    assert a3.evict_count(1024, 40, 5120, 32) == 952 and a3.evict_count(10, 40, 5120, 32) == 0 and a3.evict_count(10**6, 0, 100, 5) == 100

@@ -321,3 +321,44 @@ def test_fuse_request_with_eviction(a3mod, config, n_system, score_source):
             # agreement with the oracle: most of the kept set is common; the rest sits near the threshold
             assert len(diff) <= 2 * max(2, k // 10), (l, g, len(diff))
     s.eng.close()
+
+
+@pytest.mark.parametrize("config,n_system", [("tiny3", 0), ("tiny_gqa", 100)])
+def test_fuse_request_value_deviation_selector(a3mod, config, n_system):
+    """A3_SELECT_VALUE_DEVIATION: candidates ranked by |v_true - v_cached|^2 at the selection layer; the rest of
+    the path is the same (forcing the chosen rows through the attention selector gives the same cache)."""
+    s = Setup(a3mod, config, n_system=n_system, emb_std=0.02, w_std=0.02)
+    m, r = s.m, s.r
+    K, V = s.fused_buffers()
+    req, out = s.eng.make_request(s.tab, len(s.dk), max(r.chunk_lens), r.n_ctx, r.n_question, s.dx0, K, V, ratio=r.ratio,
+                                  select_layer=r.select_layer, n_system=n_system, selector=1)
+    s.eng.fuse_request(req)
+    assert s.eng.device_status() == 0
+    p = out["p"]
+    gs = out["scores"].cpu().numpy().astype(np.float64)
+    Re_gpu = out["rows"].cpu().numpy()[:p]
+    assert Re_gpu.tolist() == O.topk_select(gs, n_system, r.n_ctx, p).tolist()  # exactly the top-p of the GPU's own scores
+    ref = O.fuse_request(s.ck, s.cv, s.x0, r.n_question, s.weights, s.model, r.ratio, select_layer=r.select_layer,
+                         n_system=n_system, rnd=O.round_bf16, selector="value_deviation")
+    cand = slice(n_system, r.n_ctx)
+    # both sides difference two bf16 tensors; the true values come through two bf16 pipelines, so single elements may
+    # differ by an ulp: compare the distances with a tolerance relative to their typical size
+    typical = np.median(ref.scores[cand][ref.scores[cand] > 0])
+    assert np.abs(gs[cand] - ref.scores[cand]).max() <= 0.05 * typical + 0.03 * ref.scores[cand].max()
+    assert not gs[:n_system].any() and not gs[r.n_ctx:].any()
+    first = r.chunk_lens[0]
+    assert not set(Re_gpu.tolist()) & set(range(n_system, first)) or gs[n_system:first].max() > 0  # first chunk: (near) zero deviation
+    # same rows through the default selector: identical result
+    K2, V2, out2 = s.run_gpu(r.ratio, forced=Re_gpu)
+    assert torch.equal(K, K2) and torch.equal(V, V2) and torch.equal(out["x"], out2["x"])
+    # chunk-edge rows as a forced selection (the other comparison method)
+    edges = a3mod.chunk_edge_rows(r.chunk_lens, 20, n_system)
+    assert edges.tolist() == O.chunk_edge_rows(r.chunk_lens, 20, n_system).tolist()
+    K3, V3, out3 = s.run_gpu(r.ratio, forced=edges)
+    assert out3["rows"].cpu().numpy()[:edges.size].tolist() == edges.tolist()
+    # unsupported combination: value deviation needs the true values
+    with pytest.raises(a3mod.A3Error):
+        rq, _ = s.eng.make_request(s.tab, len(s.dk), max(r.chunk_lens), r.n_ctx, r.n_question, s.dx0, K, V, ratio=r.ratio,
+                                   select_layer=r.select_layer, n_system=n_system, selector=1, score_source=1)
+        s.eng.fuse_request(rq)
+    s.eng.close()
