@@ -144,6 +144,123 @@ struct TcLayout {
   static constexpr int SMEM_BYTES = BAR_OFFSET + 256 + 1024;  // barriers + slack for the 1024-byte alignment
 };
 
+// Epilogue of one accumulator row (thread = row `gr` of the output, `trow` its tensor-memory address), straight out
+// of registers.  For EPI_RESIDUAL the row's old values arrive in `pre` (see tc_prefetch_residual).
+template <int EPI, int BN>
+__device__ __forceinline__ void tc_epilogue_row(const TcParams& p, uint32_t trow, int gr, bool row_ok, int nt, int seg, int nb0,
+                                                const uint4* pre) {
+    if (EPI == EPI_RESIDUAL) {
+      // the old values of C were fetched while the main loop ran (`pre`): only tensor memory is waited for here
+      const int n0 = nt * BN;
+#pragma unroll
+      for (int c = 0; c < BN / 32; ++c) {
+        float acc[32];
+        tc_ld32(trow + c * 32, acc);
+        tc_wait_ld();
+        if (row_ok && n0 + c * 32 < p.N) {  // tiles need not divide N: TMA zero-fills, stores are cut
+          float old[32];
+#pragma unroll
+          for (int i = 0; i < 4; ++i) unpack8(pre[c * 4 + i], old + 8 * i);
+#pragma unroll
+          for (int e = 0; e < 32; ++e) acc[e] += old[e];
+          store32_bf16(p.C + (size_t)gr * p.ldc + n0 + c * 32, acc);
+        }
+      }
+    } else if (EPI == EPI_SWIGLU) {
+      const int n0 = nt * (BN / 2);
+#pragma unroll 1
+      for (int c = 0; c < BN / 64; ++c) {
+        __syncwarp();
+        float g[32], u[32];
+        tc_ld32(trow + c * 32, g);
+        tc_ld32(trow + BN / 2 + c * 32, u);
+        tc_wait_ld();
+        if (row_ok) {
+#pragma unroll
+          for (int e = 0; e < 32; ++e) g[e] = g[e] / (1.f + __expf(-g[e])) * u[e];
+          store32_bf16(p.C + (size_t)gr * p.ldc + n0 + c * 32, g);
+        }
+      }
+    } else {
+      const int kind = p.kind[seg];
+      const int D = p.D, half = D / 2;
+      const bf16* bias = p.bias[seg];
+      int ps = row_ok ? p.pos[gr] : 0;
+      bool ok = row_ok;
+      if (row_ok && (ps < 0 || ps >= p.kv_len || ps >= p.max_pos)) {
+        atomicOr(p.status, A3_DEV_BAD_POSITION);
+        ok = false;
+        ps = 0;
+      }
+      bf16* dst;
+      if (kind == 0) dst = p.q_out + (size_t)(row_ok ? gr : 0) * (p.Hq * D) + nb0;
+      else if (kind == 1) dst = p.k_cache + (size_t)ps * (p.Hkv * D) + nb0;
+      else dst = p.v_cache + (size_t)ps * (p.Hkv * D) + nb0;
+      const float2* trot = p.tab + (size_t)ps * half;
+      // pairs of 32-column chunks that hold the two halves of the rotation pairs (same chunk twice for the
+      // interleaved layout and for V, which is not rotated)
+      const int pair_stride = (p.layout == 0) ? half / 32 : 0;  // D=128: 2 chunks; D=64: 1 chunk
+#pragma unroll 1
+      for (int c = 0; c < BN / 32; ++c) {
+        const int in_head = (c * 32) % D;
+        if (p.layout == 0 && in_head >= half) continue;  // handled together with its low half
+        __syncwarp();
+        float a[32], b[32];
+        tc_ld32(trow + c * 32, a);
+        if (p.layout == 0) tc_ld32(trow + (c + pair_stride) * 32, b);
+        tc_wait_ld();
+        if (!ok) continue;
+        const int ca = c * 32, cb = (c + pair_stride) * 32;
+        if (bias) {
+          float t[32];
+          load32_bf16(bias + nb0 + ca, t);
+#pragma unroll
+          for (int e = 0; e < 32; ++e) a[e] += t[e];
+          if (p.layout == 0) {
+            load32_bf16(bias + nb0 + cb, t);
+#pragma unroll
+            for (int e = 0; e < 32; ++e) b[e] += t[e];
+          }
+        }
+        if (kind != 2) {
+          if (p.layout == 0) {
+#pragma unroll
+            for (int e = 0; e < 32; ++e) {
+              const float2 cs = __ldg(trot + in_head + e);
+              const float x = a[e], y = b[e];
+              a[e] = x * cs.x - y * cs.y;
+              b[e] = x * cs.y + y * cs.x;
+            }
+          } else {
+#pragma unroll
+            for (int e = 0; e < 16; ++e) {
+              const float2 cs = __ldg(trot + in_head / 2 + e);
+              const float x = a[2 * e], y = a[2 * e + 1];
+              a[2 * e] = x * cs.x - y * cs.y;
+              a[2 * e + 1] = x * cs.y + y * cs.x;
+            }
+          }
+        }
+        store32_bf16(dst + ca, a);
+        if (p.layout == 0) store32_bf16(dst + cb, b);
+      }
+    }
+}
+
+// Old values of this thread's row of C for the residual epilogue: issued before the accumulator is waited for, so
+// the global-memory latency (a row per lane: uncoalesced, L2-resident) hides behind the main loop.
+template <int BN>
+__device__ __forceinline__ void tc_prefetch_residual(const TcParams& p, int gr, bool row_ok, int nt, uint4 (&pre)[BN / 8]) {
+  const int n0 = nt * BN;
+#pragma unroll
+  for (int c = 0; c < BN / 32; ++c) {
+    const bool col_ok = row_ok && n0 + c * 32 < p.N;
+    const uint4* src = reinterpret_cast<const uint4*>(p.C + (size_t)(col_ok ? gr : 0) * p.ldc + (col_ok ? n0 + c * 32 : 0));
+#pragma unroll
+    for (int i = 0; i < 4; ++i) pre[c * 4 + i] = col_ok ? __ldg(src + i) : make_uint4(0, 0, 0, 0);
+  }
+}
+
 template <int EPI, int BN, int STAGES>
 __global__ void __launch_bounds__(TC_THREADS)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB0,
@@ -251,106 +368,11 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     const int gr = m0 + row;
     const bool row_ok = gr < p.M;
     const uint32_t trow = tmem_base + ((uint32_t)(quarter * 32) << 16);
+    uint4 pre[EPI == EPI_RESIDUAL ? BN / 8 : 1];
+    if (EPI == EPI_RESIDUAL) tc_prefetch_residual<BN>(p, gr, row_ok, nt, *reinterpret_cast<uint4(*)[BN / 8]>(pre));
     const bool ready = mbar_wait(tmem_full_bar, 0, abort_flag, p.status);
     tc_fence_after();
-    if (ready) {
-      if (EPI == EPI_RESIDUAL) {
-        const int n0 = nt * BN;
-#pragma unroll 1
-        for (int c = 0; c < BN / 32; ++c) {
-          __syncwarp();
-          float acc[32], old[32];
-          tc_ld32(trow + c * 32, acc);
-          const bool col_ok = row_ok && n0 + c * 32 < p.N;  // tiles need not divide N: TMA zero-fills, stores are cut
-          bf16* cp = p.C + (size_t)(row_ok ? gr : 0) * p.ldc + (col_ok ? n0 + c * 32 : 0);
-          if (col_ok) load32_bf16(cp, old);
-          tc_wait_ld();
-          if (col_ok) {
-#pragma unroll
-            for (int e = 0; e < 32; ++e) acc[e] += old[e];
-            store32_bf16(cp, acc);
-          }
-        }
-      } else if (EPI == EPI_SWIGLU) {
-        const int n0 = nt * (BN / 2);
-#pragma unroll 1
-        for (int c = 0; c < BN / 64; ++c) {
-          __syncwarp();
-          float g[32], u[32];
-          tc_ld32(trow + c * 32, g);
-          tc_ld32(trow + BN / 2 + c * 32, u);
-          tc_wait_ld();
-          if (row_ok) {
-#pragma unroll
-            for (int e = 0; e < 32; ++e) g[e] = g[e] / (1.f + __expf(-g[e])) * u[e];
-            store32_bf16(p.C + (size_t)gr * p.ldc + n0 + c * 32, g);
-          }
-        }
-      } else {
-        const int kind = p.kind[seg];
-        const int D = p.D, half = D / 2;
-        const bf16* bias = p.bias[seg];
-        int ps = row_ok ? p.pos[gr] : 0;
-        bool ok = row_ok;
-        if (row_ok && (ps < 0 || ps >= p.kv_len || ps >= p.max_pos)) {
-          atomicOr(p.status, A3_DEV_BAD_POSITION);
-          ok = false;
-          ps = 0;
-        }
-        bf16* dst;
-        if (kind == 0) dst = p.q_out + (size_t)(row_ok ? gr : 0) * (p.Hq * D) + nb0;
-        else if (kind == 1) dst = p.k_cache + (size_t)ps * (p.Hkv * D) + nb0;
-        else dst = p.v_cache + (size_t)ps * (p.Hkv * D) + nb0;
-        const float2* trot = p.tab + (size_t)ps * half;
-        // pairs of 32-column chunks that hold the two halves of the rotation pairs (same chunk twice for the
-        // interleaved layout and for V, which is not rotated)
-        const int pair_stride = (p.layout == 0) ? half / 32 : 0;  // D=128: 2 chunks; D=64: 1 chunk
-#pragma unroll 1
-        for (int c = 0; c < BN / 32; ++c) {
-          const int in_head = (c * 32) % D;
-          if (p.layout == 0 && in_head >= half) continue;  // handled together with its low half
-          __syncwarp();
-          float a[32], b[32];
-          tc_ld32(trow + c * 32, a);
-          if (p.layout == 0) tc_ld32(trow + (c + pair_stride) * 32, b);
-          tc_wait_ld();
-          if (!ok) continue;
-          const int ca = c * 32, cb = (c + pair_stride) * 32;
-          if (bias) {
-            float t[32];
-            load32_bf16(bias + nb0 + ca, t);
-#pragma unroll
-            for (int e = 0; e < 32; ++e) a[e] += t[e];
-            if (p.layout == 0) {
-              load32_bf16(bias + nb0 + cb, t);
-#pragma unroll
-              for (int e = 0; e < 32; ++e) b[e] += t[e];
-            }
-          }
-          if (kind != 2) {
-            if (p.layout == 0) {
-#pragma unroll
-              for (int e = 0; e < 32; ++e) {
-                const float2 cs = __ldg(trot + in_head + e);
-                const float x = a[e], y = b[e];
-                a[e] = x * cs.x - y * cs.y;
-                b[e] = x * cs.y + y * cs.x;
-              }
-            } else {
-#pragma unroll
-              for (int e = 0; e < 16; ++e) {
-                const float2 cs = __ldg(trot + in_head / 2 + e);
-                const float x = a[2 * e], y = a[2 * e + 1];
-                a[2 * e] = x * cs.x - y * cs.y;
-                a[2 * e + 1] = x * cs.y + y * cs.x;
-              }
-            }
-          }
-          store32_bf16(dst + ca, a);
-          if (p.layout == 0) store32_bf16(dst + cb, b);
-        }
-      }
-    }
+    if (ready) tc_epilogue_row<EPI, BN>(p, trow, gr, row_ok, nt, seg, nb0, pre);
   }
   tc_fence_before();
   __syncthreads();
