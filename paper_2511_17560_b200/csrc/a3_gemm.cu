@@ -8,7 +8,8 @@
 // One CTA computes one 128 x BN tile.  Warp 0 (one lane) feeds a ring of shared-memory stages with TMA
 // (cp.async.bulk.tensor, 128-byte swizzle); warp 1 (one lane) issues tcgen05.mma (128 x BN x 16) on the stages and
 // commits them back to the producer through mbarriers; warps 2..5 read the accumulator with tcgen05.ld (each thread
-// owns one output row) and run the epilogue straight out of registers.  No cluster multicast is used.
+// owns one output row) and run the epilogue straight out of registers.  A second kernel shares a 256 x 256 tile
+// between the two CTAs of a cluster (tcgen05 cta_group::2, see below).  No load uses cluster multicast.
 // Every barrier wait is bounded: after half a second a waiter raises the CTA's abort flag and the device status bit
 // A3_DEV_WAIT_EXHAUSTED, all roles leave their loops, in-flight copies are given time to land, tensor memory is
 // released and the CTA returns.
@@ -379,6 +380,190 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
   if (warp == 1) asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(TMEM_COLS) : "memory");
 }
 
+// ---------------------------------------------------------------- CTA-pair kernel (tcgen05 cta_group::2)
+// With one CTA per tile every SM pulls A (128 x 64) and B (256 x 64) of each k-block through its own 64-byte-per-
+// clock L2 port: 48 KiB per 512 clocks of MMA, i.e. the port, not the tensor core, sets the pace.  Here two CTAs of
+// a cluster (two SMs) share one 256 x 256 output tile: each loads its own 128 rows of A and HALF of the B tile
+// (32 KiB per k-block per SM), the leader CTA issues tcgen05.mma.cta_group::2 (M = 256, N = 256), which reads both
+// halves of B from the two SMs' shared memory and leaves rows 0..127 of the accumulator in the leader's tensor
+// memory and rows 128..255 in its peer's.  Both CTAs then run the same epilogues as the single-CTA kernel.
+// Loads are plain per-CTA TMA copies (no multicast); the peer's copies complete on the leader's "full" barrier;
+// tcgen05.commit with a CTA mask releases a stage (and, at the end, publishes the accumulator) in both CTAs.
+constexpr int PAIR_BN = 256;
+template <int STAGES>
+struct PairLayout {
+  static constexpr int A_BYTES = TC_BM * TC_BK * 2;
+  static constexpr int B_BYTES = (PAIR_BN / 2) * TC_BK * 2;  // this CTA's half of the B tile
+  static constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
+  static constexpr int BAR_OFFSET = STAGES * STAGE_BYTES;
+  static constexpr int SMEM_BYTES = BAR_OFFSET + 256 + 1024;
+};
+constexpr uint32_t PAIR_LEADER_MASK = 0xFEFFFFFFu;  // clears the CTA-rank bit of a shared::cluster address: same offset in CTA 0
+
+__device__ __forceinline__ uint32_t cluster_ctarank() {
+  uint32_t r;
+  asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+  return r;
+}
+__device__ __forceinline__ void cluster_sync_all() {
+  asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+  asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+// this CTA's own copy into its own shared memory; the bytes are counted on the barrier at `bar` (a shared::cluster
+// address, here always the leader's)
+__device__ __forceinline__ void tma_load_2d_pair(uint32_t dst, const CUtensorMap* map, int x, int y, uint32_t bar) {
+  asm volatile("cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+               ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(bar)
+               : "memory");
+}
+__device__ __forceinline__ void tc_commit_pair(uint32_t bar, uint16_t cta_mask) {
+  asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;" ::"r"(bar), "h"(cta_mask) : "memory");
+}
+__device__ __forceinline__ void tc_mma_pair_f16(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
+  const uint32_t z = 0;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, {%5, %5, %5, %5, %5, %5, %5, %5}, p;\n\t}"
+      ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate), "r"(z)
+      : "memory");
+}
+// bf16 x bf16 -> fp32, both operands K-major, M = 256 over the CTA pair
+__host__ __device__ constexpr uint32_t idesc_bf16_pair(int n) {
+  return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(256 >> 4) << 24);
+}
+
+template <int EPI, int STAGES>
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(TC_THREADS)
+gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB0,
+                 const __grid_constant__ CUtensorMap tmB1, const __grid_constant__ CUtensorMap tmB2, const TcParams p) {
+  using L = PairLayout<STAGES>;
+  constexpr int BN = PAIR_BN;
+  extern __shared__ unsigned char smem_raw[];
+  const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;  // same offset in both CTAs of the pair
+  unsigned char* base_ptr = smem_raw + (base - smem_u32(smem_raw));
+  const uint32_t bars = base + L::BAR_OFFSET;  // full[S] (used in the leader), empty[S], tmem_full: 8 bytes each
+  volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(base_ptr + L::BAR_OFFSET + 8 * (2 * STAGES + 1));
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(base_ptr + L::BAR_OFFSET + 8 * (2 * STAGES + 1) + 8);
+  auto full_bar = [&](int s) { return bars + 8u * s; };
+  auto empty_bar = [&](int s) { return bars + 8u * (STAGES + s); };
+  const uint32_t tmem_full_bar = bars + 8u * (2 * STAGES);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const uint32_t rank = cluster_ctarank();
+  const bool leader = rank == 0;
+  const int m0 = blockIdx.x * TC_BM;  // CTAs 2i and 2i+1 of a row of the grid form a pair: consecutive row tiles
+  const int nt = blockIdx.y;
+  const int KT = p.K / TC_BK;
+
+  int seg = 0, seg_tile0 = 0;
+  if (EPI == EPI_QKV) {
+    while (seg < 2 && nt >= p.seg_tiles_end[seg]) {
+      seg_tile0 = p.seg_tiles_end[seg];
+      ++seg;
+    }
+  }
+  // first output column of this tile within its matrix (for SwiGLU: within gate and within up)
+  const int nb0 = (EPI == EPI_SWIGLU) ? nt * (BN / 2) : (nt - seg_tile0) * BN;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < STAGES; ++s) {
+      mbar_init(full_bar(s), 1);
+      mbar_init(empty_bar(s), 1);
+    }
+    mbar_init(tmem_full_bar, 1);
+    abort_flag[0] = 0;
+    abort_flag[1] = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+  }
+  if (warp == 1) {  // the same warp of both CTAs
+    asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32((const void*)tmem_slot)), "r"(256) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
+  cluster_sync_all();  // the peer's barriers exist before anything is signalled on them
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+
+  if (warp == 0) {
+    // ---------------- TMA producer (both CTAs): own rows of A, own half of B
+    if (lane == 0) {
+      const CUtensorMap* mapB;
+      int brow0;
+      if (EPI == EPI_SWIGLU) {
+        mapB = leader ? &tmB0 : &tmB1;  // accumulator columns 0..127 = gate (leader's half), 128..255 = up (peer's half)
+        brow0 = nb0;
+      } else {
+        mapB = seg == 0 ? &tmB0 : (seg == 1 ? &tmB1 : &tmB2);
+        brow0 = nb0 + (int)rank * (BN / 2);
+      }
+      tmap_prefetch(&tmA);
+      tmap_prefetch(mapB);
+      int issued = 0;
+      for (int kb = 0; kb < KT; ++kb) {
+        const int s = kb % STAGES;
+        const uint32_t ph = (kb / STAGES) & 1;
+        if (!mbar_wait(empty_bar(s), ph ^ 1, abort_flag, p.status)) break;
+        const uint32_t sa = base + s * L::STAGE_BYTES, sb = sa + L::A_BYTES;
+        const uint32_t full_leader = full_bar(s) & PAIR_LEADER_MASK;
+        // The leader announces the bytes of both CTAs.  A copy of the peer may complete before that: the phase
+        // cannot end early, because the leader's own arrival is still pending until its expect_tx.
+        if (leader) mbar_expect_tx(full_bar(s), 2 * L::STAGE_BYTES);
+        tma_load_2d_pair(sa, &tmA, kb * TC_BK, m0, full_leader);
+        tma_load_2d_pair(sb, mapB, kb * TC_BK, brow0, full_leader);
+        issued = kb + 1;
+      }
+      if (*abort_flag) {
+        // let the copies already issued land before the CTA can exit (bounded)
+        if (leader) {
+          for (int kb = max(0, issued - STAGES); kb < issued; ++kb)
+            mbar_wait(full_bar(kb % STAGES), (kb / STAGES) & 1, abort_flag + 1, p.status, 2000000ull);
+        } else {
+          const unsigned long long t0 = global_ns();
+          while (global_ns() - t0 < 200000ull) {
+          }
+        }
+      }
+    }
+  } else if (warp == 1) {
+    // ---------------- MMA issuer: the leader alone, for both CTAs
+    if (lane == 0 && leader) {
+      constexpr uint32_t idesc = idesc_bf16_pair(BN);
+      bool ok = true;
+      for (int kb = 0; kb < KT && ok; ++kb) {
+        const int s = kb % STAGES;
+        const uint32_t ph = (kb / STAGES) & 1;
+        ok = mbar_wait(full_bar(s), ph, abort_flag, p.status);
+        if (!ok) break;
+        tc_fence_after();
+        const uint32_t sa = base + s * L::STAGE_BYTES, sb = sa + L::A_BYTES;
+        const uint64_t da = smem_desc_sw128(sa), db = smem_desc_sw128(sb);
+#pragma unroll
+        for (int k = 0; k < TC_BK / 16; ++k)
+          tc_mma_pair_f16(tmem_base, da + (uint64_t)(2 * k), db + (uint64_t)(2 * k), idesc, (kb | k) != 0);
+        tc_commit_pair(empty_bar(s), 3);  // frees this stage in both CTAs once the MMAs above have read it
+      }
+      if (ok) tc_commit_pair(tmem_full_bar, 3);
+    }
+  } else {
+    // ---------------- epilogue: warps 2..5 of both CTAs, each CTA its own 128 rows
+    const int quarter = warp & 3;
+    const int row = quarter * 32 + lane;
+    const int gr = m0 + row;
+    const bool row_ok = gr < p.M;
+    const uint32_t trow = tmem_base + ((uint32_t)(quarter * 32) << 16);
+    uint4 pre[EPI == EPI_RESIDUAL ? BN / 8 : 1];
+    if (EPI == EPI_RESIDUAL) tc_prefetch_residual<BN>(p, gr, row_ok, nt, *reinterpret_cast<uint4(*)[BN / 8]>(pre));
+    const bool ready = mbar_wait(tmem_full_bar, 0, abort_flag, p.status);
+    tc_fence_after();
+    if (ready) tc_epilogue_row<EPI, BN>(p, trow, gr, row_ok, nt, seg, nb0, pre);
+  }
+  tc_fence_before();
+  cluster_sync_all();  // neither CTA releases tensor or shared memory while the other may still use it
+  if (warp == 1) asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(256) : "memory");
+}
+
 // ---------------------------------------------------------------- host side
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
                                   const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
@@ -441,14 +626,45 @@ static int launch_tc(const a3_handle* h, const GemmArgs& a, const TcParams& p, i
   return A3_OK;
 }
 
+template <int EPI, int STAGES>
+static int launch_pair(const a3_handle* h, const GemmArgs& a, const TcParams& p, int tiles, cudaStream_t st) {
+  using L = PairLayout<STAGES>;
+  CUtensorMap tA, tB[3];
+  A3_TRY(make_tmap(&tA, a.A, a.M, a.K, TC_BM));
+  if (EPI == EPI_SWIGLU) {
+    A3_TRY(make_tmap(&tB[0], a.seg[0].B, a.seg[0].n, a.K, PAIR_BN / 2));
+    A3_TRY(make_tmap(&tB[1], a.B2, a.seg[0].n, a.K, PAIR_BN / 2));
+    tB[2] = tB[0];
+  } else {
+    for (int s = 0; s < 3; ++s) {
+      if (s < a.nseg) A3_TRY(make_tmap(&tB[s], a.seg[s].B, a.seg[s].n, a.K, PAIR_BN / 2));
+      else tB[s] = tB[0];
+    }
+  }
+  static bool attr_set = false;
+  if (!attr_set) {
+    A3_CUDA(cudaFuncSetAttribute(gemm_pair_kernel<EPI, STAGES>, cudaFuncAttributeMaxDynamicSharedMemorySize, L::SMEM_BYTES));
+    attr_set = true;
+  }
+  dim3 grid(2 * cdiv(cdiv(a.M, TC_BM), 2), tiles);  // whole pairs: a last odd row tile gets an all-padding partner
+  ProfScope prof(h, EPI == EPI_RESIDUAL ? A3_K_GEMM_RESIDUAL : EPI == EPI_SWIGLU ? A3_K_GEMM_SWIGLU : A3_K_GEMM_QKV, st);
+  gemm_pair_kernel<EPI, STAGES><<<grid, TC_THREADS, L::SMEM_BYTES, st>>>(tA, tB[0], tB[1], tB[2], p);
+  A3_LAUNCHED();
+  return A3_OK;
+}
+
 // Tile width / pipeline depth per epilogue [EPI_RESIDUAL, EPI_SWIGLU, EPI_QKV] -> {BN, STAGES}; BN = 0 lets the
 // launcher choose (a3_internal_set_gemm_cfg pins a choice for tuning runs).  Measured on B200 at Llama-8B width:
 // two co-resident CTAs per SM (256/2, 128/3) overlap one tile's epilogue with the other's main loop and win when
-// the grid has several waves; a single wave prefers the widest tile that still gives every SM at most one CTA.
+// the grid has several waves.  The CTA-pair kernel wins for the residual GEMMs (N = d_model: few tiles, one CTA per
+// SM); for SwiGLU and QKV its extra all-padding row tile at 804 rows (7 -> 8) costs more than the halved B traffic
+// saves: under the power cap the tensor work, not the L2 port, sets the pace.
 int g_tc_cfg[3][2] = {{0, 0}, {256, 2}, {0, 0}};
 
 template <int EPI>
 static int dispatch_tc(const a3_handle* h, const GemmArgs& a, const TcParams& p, int tiles, int bn, int stages, cudaStream_t st) {
+  if (bn == 512 && stages == 3) return launch_pair<EPI, 3>(h, a, p, tiles, st);
+  if (bn == 512) return launch_pair<EPI, 6>(h, a, p, tiles, st);
   if (bn == 256 && stages == 4) return launch_tc<EPI, 256, 4>(h, a, p, tiles, st);
   if (bn == 256 && stages == 3) return launch_tc<EPI, 256, 3>(h, a, p, tiles, st);
   if (bn == 256 && stages == 2) return launch_tc<EPI, 256, 2>(h, a, p, tiles, st);
@@ -467,16 +683,26 @@ int gemm_bf16(const a3_handle* h, GemmEpilogue epi, const GemmArgs& a, cudaStrea
   if (bn == 0) {
     const int m_tiles = cdiv(a.M, TC_BM), sms = h->sm_count > 0 ? h->sm_count : 148;
     if (epi == EPI_RESIDUAL) {
-      // when a single wave of CTAs covers the output either way, the narrower 224-column tile shortens it
-      const int n = a.seg[0].n;
-      bn = (m_tiles * cdiv(n, 256) <= sms && m_tiles * cdiv(n, 224) <= sms) ? 224 : 256;
-      stages = 4;
+      // the CTA-pair kernel (bn 512 selects it): measured 5-7 % faster than one CTA per 128 x 224/256 tile at
+      // Llama-8B width for 804 and 5 152 rows
+      (void)m_tiles;
+      (void)sms;
+      bn = 512;
+      stages = 6;
     } else {
       bn = 256;
       stages = 4;
     }
   }
   // output columns per tile; QKV tiles must hold whole heads and divide every segment
+  bool pair = bn == 512;  // the CTA-pair kernel: 256 accumulator columns over two CTAs
+  if (pair) {
+    bn = PAIR_BN;
+    if (epi != EPI_RESIDUAL)
+      for (int s = 0; s < a.nseg; ++s)
+        if (a.seg[s].n % (epi == EPI_SWIGLU ? PAIR_BN / 2 : PAIR_BN)) pair = false;  // falls back to one CTA per tile
+    if (!pair) stages = 4;
+  }
   int out_cols = epi == EPI_SWIGLU ? bn / 2 : bn;
   if (epi == EPI_QKV) {
     for (int s = 0; s < a.nseg; ++s)
@@ -514,6 +740,7 @@ int gemm_bf16(const a3_handle* h, GemmEpilogue epi, const GemmArgs& a, cudaStrea
   p.max_pos = h->m.max_positions;
   p.tab = h->rope_tab;
   p.status = h->dev_status;
+  if (pair) bn = 512;
   if (epi == EPI_RESIDUAL) return dispatch_tc<EPI_RESIDUAL>(h, a, p, tiles, bn, stages, st);
   if (epi == EPI_SWIGLU) return dispatch_tc<EPI_SWIGLU>(h, a, p, tiles, bn, stages, st);
   return dispatch_tc<EPI_QKV>(h, a, p, tiles, bn, stages, st);
