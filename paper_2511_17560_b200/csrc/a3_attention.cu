@@ -277,6 +277,8 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
   __syncthreads();
   fence_after();
   const uint32_t tmem_base = *tmem_slot;
+  pdl_wait();  // the set-up above overlapped the previous kernel's tail; positions, Q and the cache are read below
+  pdl_launch_dependents();
   const uint32_t tmem_s0 = tmem_base, tmem_o = tmem_base + 256;
 
   if (warp == 0) {
@@ -720,9 +722,11 @@ int attention_rows(const a3_handle* h, const bf16* q, const int32_t* pos, int M,
   }
   ProfScope prof(h, A3_K_ATTENTION, st);
   if (D == 128)
-    attention_tc_kernel<128><<<n_ctas, ATC_THREADS, AtcLayout<128>::SMEM_BYTES, st>>>(tK, tV, q, pos, M, kv_len, o, lse, Hq, Hkv, scale_log2, h->dev_status, n_split, tiles_per_split, part_o, part_ml);
+    A3_CUDA(launch_pdl(attention_tc_kernel<128>, dim3(n_ctas), dim3(ATC_THREADS), (size_t)AtcLayout<128>::SMEM_BYTES, st, tK, tV, q, pos, M, kv_len, o,
+                       lse, Hq, Hkv, scale_log2, h->dev_status, n_split, tiles_per_split, part_o, part_ml));
   else
-    attention_tc_kernel<64><<<n_ctas, ATC_THREADS, AtcLayout<64>::SMEM_BYTES, st>>>(tK, tV, q, pos, M, kv_len, o, lse, Hq, Hkv, scale_log2, h->dev_status, n_split, tiles_per_split, part_o, part_ml);
+    A3_CUDA(launch_pdl(attention_tc_kernel<64>, dim3(n_ctas), dim3(ATC_THREADS), (size_t)AtcLayout<64>::SMEM_BYTES, st, tK, tV, q, pos, M, kv_len, o,
+                       lse, Hq, Hkv, scale_log2, h->dev_status, n_split, tiles_per_split, part_o, part_ml));
   A3_LAUNCHED();
   if (n_split > 1) {
     dim3 cgrid(cdiv((long long)M * G, 4), Hkv);

@@ -312,6 +312,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
+  pdl_wait();  // everything above overlapped the previous kernel's tail; from here on its results are read
+  pdl_launch_dependents();
 
   if (warp == 0) {
     // ---------------- TMA producer
@@ -485,6 +487,8 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
   cluster_sync_all();  // the peer's barriers exist before anything is signalled on them
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
+  pdl_wait();
+  pdl_launch_dependents();
 
   if (warp == 0) {
     // ---------------- TMA producer (both CTAs): own rows of A, own half of B
@@ -621,7 +625,7 @@ static int launch_tc(const a3_handle* h, const GemmArgs& a, const TcParams& p, i
   }
   dim3 grid(cdiv(a.M, TC_BM), tiles);
   ProfScope prof(h, EPI == EPI_RESIDUAL ? A3_K_GEMM_RESIDUAL : EPI == EPI_SWIGLU ? A3_K_GEMM_SWIGLU : A3_K_GEMM_QKV, st);
-  gemm_tc_kernel<EPI, BN, STAGES><<<grid, TC_THREADS, L::SMEM_BYTES, st>>>(tA, tB[0], tB[1], tB[2], p);
+  A3_CUDA(launch_pdl(gemm_tc_kernel<EPI, BN, STAGES>, grid, dim3(TC_THREADS), (size_t)L::SMEM_BYTES, st, tA, tB[0], tB[1], tB[2], p));
   A3_LAUNCHED();
   return A3_OK;
 }
@@ -648,7 +652,7 @@ static int launch_pair(const a3_handle* h, const GemmArgs& a, const TcParams& p,
   }
   dim3 grid(2 * cdiv(cdiv(a.M, TC_BM), 2), tiles);  // whole pairs: a last odd row tile gets an all-padding partner
   ProfScope prof(h, EPI == EPI_RESIDUAL ? A3_K_GEMM_RESIDUAL : EPI == EPI_SWIGLU ? A3_K_GEMM_SWIGLU : A3_K_GEMM_QKV, st);
-  gemm_pair_kernel<EPI, STAGES><<<grid, TC_THREADS, L::SMEM_BYTES, st>>>(tA, tB[0], tB[1], tB[2], p);
+  A3_CUDA(launch_pdl(gemm_pair_kernel<EPI, STAGES>, grid, dim3(TC_THREADS), (size_t)L::SMEM_BYTES, st, tA, tB[0], tB[1], tB[2], p));
   A3_LAUNCHED();
   return A3_OK;
 }

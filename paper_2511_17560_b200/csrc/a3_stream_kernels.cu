@@ -340,6 +340,8 @@ int check_rows(const a3_handle* h, const int32_t* pos, int M, int kv_len, cudaSt
 constexpr int RN_THREADS = 128, RN_VPT = 4;
 __global__ void __launch_bounds__(RN_THREADS)
 rmsnorm_kernel(const uint4* __restrict__ x, const uint4* __restrict__ gain, float eps, int row_vecs, uint4* __restrict__ out) {
+  pdl_wait();
+  pdl_launch_dependents();
   const uint4* xr = x + (size_t)blockIdx.x * row_vecs;
   uint4 v[RN_VPT];
   float ss = 0.f;
@@ -396,7 +398,7 @@ rmsnorm_kernel(const uint4* __restrict__ x, const uint4* __restrict__ gain, floa
 int rmsnorm_rows(const a3_handle* h, const bf16* x, const bf16* gain, float eps, int M, int d, bf16* out, cudaStream_t st) {
   if (M <= 0) return A3_OK;
   ProfScope prof(h, A3_K_RMSNORM, st);
-  rmsnorm_kernel<<<M, RN_THREADS, 0, st>>>((const uint4*)x, (const uint4*)gain, eps, d / 8, (uint4*)out);
+  A3_CUDA(launch_pdl(rmsnorm_kernel, dim3(M), dim3(RN_THREADS), 0, st, (const uint4*)x, (const uint4*)gain, eps, d / 8, (uint4*)out));
   A3_LAUNCHED();
   return A3_OK;
 }
