@@ -413,65 +413,76 @@ def run_a3(args):
                "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h)}
         assert torch.equal(rows_h, out["rows"].cpu()), "host entry selected different rows"
 
-    # context for the paper's TTFT comparison: a full prefill of the concatenated input on the same kernels
-    Kp, Vp = torch.zeros_like(K), torch.zeros_like(V)
-    eng.precompute_chunk(x0.clone(), Kp, Vp)
-    torch.cuda.synchronize()
-    xs = [x0.clone() for _ in range(3)]
-    e0.record(stream)
-    for xx in xs:
-        eng.precompute_chunk(xx, Kp, Vp)
-    e1.record(stream)
-    torch.cuda.synchronize()
-    full_prefill_ms = e0.elapsed_time(e1) / len(xs)
-    del Kp, Vp, xs
+    context = {}
+    if not args.no_context:
+        # context for the paper's TTFT comparison: a full prefill of the concatenated input on the same kernels
+        Kp, Vp = torch.zeros_like(K), torch.zeros_like(V)
+        eng.precompute_chunk(x0.clone(), Kp, Vp)
+        torch.cuda.synchronize()
+        xs = [x0.clone() for _ in range(3)]
+        e0.record(stream)
+        for xx in xs:
+            eng.precompute_chunk(xx, Kp, Vp)
+        e1.record(stream)
+        torch.cuda.synchronize()
+        full_prefill_ms = e0.elapsed_time(e1) / len(xs)
+        del Kp, Vp, xs
 
-    # the cheaper reading of the selection (scores against the recovered cached keys, no full block), same request
-    req_c, out_c = eng.make_request(tab, len(ck), max(r.chunk_lens), r.n_ctx, r.n_question, x0, K, V, ratio=r.ratio,
-                                    select_layer=r.select_layer, score_source=1)
-    for _ in range(2):
-        eng.fuse_request(req_c)
-    torch.cuda.synchronize()
-    e0.record(stream)
-    for _ in range(3):
-        eng.fuse_request(req_c)
-    e1.record(stream)
-    torch.cuda.synchronize()
-    cached_ms = e0.elapsed_time(e1) / 3
-    overlap = len(set(out_c["rows"][:p].tolist()) & set(out["rows"][:p].tolist())) / max(p, 1)
+        # the cheaper reading of the selection (scores against the recovered cached keys, no full block), same request
+        req_c, out_c = eng.make_request(tab, len(ck), max(r.chunk_lens), r.n_ctx, r.n_question, x0, K, V, ratio=r.ratio,
+                                        select_layer=r.select_layer, score_source=1)
+        for _ in range(2):
+            eng.fuse_request(req_c)
+        torch.cuda.synchronize()
+        e0.record(stream)
+        for _ in range(3):
+            eng.fuse_request(req_c)
+        e1.record(stream)
+        torch.cuda.synchronize()
+        cached_ms = e0.elapsed_time(e1) / 3
+        overlap = len(set(out_c["rows"][:p].tolist()) & set(out["rows"][:p].tolist())) / max(p, 1)
 
-    # the `ex` extension on top of the request: compact caches of capacity C = 1024 (the paper's setting) per layer
-    req_e, out_e = eng.make_request(tab, len(ck), max(r.chunk_lens), r.n_ctx, r.n_question, x0, K, V, ratio=r.ratio,
-                                    select_layer=r.select_layer, evict_capacity=1024, evict_pool=7)
-    for _ in range(2):
-        eng.fuse_request(req_e)
-    torch.cuda.synchronize()
-    e0.record(stream)
-    for _ in range(3):
-        eng.fuse_request(req_e)
-    e1.record(stream)
-    torch.cuda.synchronize()
-    evict_ms = e0.elapsed_time(e1) / 3
-    del out_e
+        # the `ex` extension on top of the request: compact caches of capacity C = 1024 (the paper's setting) per layer
+        req_e, out_e = eng.make_request(tab, len(ck), max(r.chunk_lens), r.n_ctx, r.n_question, x0, K, V, ratio=r.ratio,
+                                        select_layer=r.select_layer, evict_capacity=1024, evict_pool=7)
+        for _ in range(2):
+            eng.fuse_request(req_e)
+        torch.cuda.synchronize()
+        e0.record(stream)
+        for _ in range(3):
+            eng.fuse_request(req_e)
+        e1.record(stream)
+        torch.cuda.synchronize()
+        evict_ms = e0.elapsed_time(e1) / 3
+        del out_e
 
-    # ... and the first token itself (final norm, vocabulary projection, greedy choice) on the last question row:
-    # HBM-bound, vocab*d*2 bytes read once; synthetic final-norm gains and vocabulary matrix
-    g = torch.Generator(device=dev)
-    g.manual_seed(7)
-    lm_head = (torch.randn((m.vocab, m.d_model), device=dev, generator=g) * 0.02).to(torch.bfloat16)
-    fnorm = torch.ones(m.d_model, dtype=torch.bfloat16, device=dev)
-    x_last = out["x"][-1]
-    for _ in range(3):
-        eng.first_token(x_last, fnorm, lm_head, want_logits=False)
-    torch.cuda.synchronize()
-    e0.record(stream)
-    for _ in range(10):
-        eng.first_token(x_last, fnorm, lm_head, want_logits=False)
-    e1.record(stream)
-    torch.cuda.synchronize()
-    first_token_ms = e0.elapsed_time(e1) / 10
-    first_token_gbs = m.vocab * m.d_model * 2 / (first_token_ms * 1e-3) / 1e9
-    del lm_head
+        # ... and the first token itself (final norm, vocabulary projection, greedy choice) on the last question row:
+        # HBM-bound, vocab*d*2 bytes read once; synthetic final-norm gains and vocabulary matrix
+        g = torch.Generator(device=dev)
+        g.manual_seed(7)
+        lm_head = (torch.randn((m.vocab, m.d_model), device=dev, generator=g) * 0.02).to(torch.bfloat16)
+        fnorm = torch.ones(m.d_model, dtype=torch.bfloat16, device=dev)
+        x_last = out["x"][-1]
+        for _ in range(3):
+            eng.first_token(x_last, fnorm, lm_head, want_logits=False)
+        torch.cuda.synchronize()
+        e0.record(stream)
+        for _ in range(10):
+            eng.first_token(x_last, fnorm, lm_head, want_logits=False)
+        e1.record(stream)
+        torch.cuda.synchronize()
+        first_token_ms = e0.elapsed_time(e1) / 10
+        first_token_gbs = m.vocab * m.d_model * 2 / (first_token_ms * 1e-3) / 1e9
+        del lm_head
+        req_ms = seconds / args.steps * 1e3
+        context = {
+            "full_prefill_ms": full_prefill_ms, "speedup_vs_full_prefill": full_prefill_ms / req_ms,
+            "scores_from_cached_keys": {"request_ms": cached_ms, "tokens_per_s": r.n_ctx / (cached_ms * 1e-3),
+                                        "selection_overlap_with_true_keys": overlap},
+            "ex_eviction": {"capacity": 1024, "pool": 7, "request_ms": evict_ms, "overhead_ms": evict_ms - req_ms},
+            "first_token": {"ms": first_token_ms, "achieved_gbs": first_token_gbs, "frac_of_hbm_peak": first_token_gbs / peaks["hbm_gbs"],
+                            "ttft_fused_ms": req_ms + first_token_ms, "ttft_full_prefill_ms": full_prefill_ms + first_token_ms,
+                            "ttft_ratio": (full_prefill_ms + first_token_ms) / (req_ms + first_token_ms)}}
 
     cpu = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
@@ -492,14 +503,7 @@ def run_a3(args):
                 "request_ms": seconds / args.steps * 1e3,
                 "request_ms_with_profiling_events": profiled_ms,
                 "cuda_graph_replay": None if graph_ms is None else {"ms_per_step": graph_ms, "value": r.n_ctx / (graph_ms * 1e-3)},
-                "full_prefill_ms": full_prefill_ms, "speedup_vs_full_prefill": full_prefill_ms / (seconds / args.steps * 1e3),
-                "scores_from_cached_keys": {"request_ms": cached_ms, "tokens_per_s": r.n_ctx / (cached_ms * 1e-3),
-                                            "selection_overlap_with_true_keys": overlap},
-                "ex_eviction": {"capacity": 1024, "pool": 7, "request_ms": evict_ms, "overhead_ms": evict_ms - seconds / args.steps * 1e3},
-                "first_token": {"ms": first_token_ms, "achieved_gbs": first_token_gbs, "frac_of_hbm_peak": first_token_gbs / peaks["hbm_gbs"],
-                                "ttft_fused_ms": seconds / args.steps * 1e3 + first_token_ms,
-                                "ttft_full_prefill_ms": full_prefill_ms + first_token_ms,
-                                "ttft_ratio": (full_prefill_ms + first_token_ms) / (seconds / args.steps * 1e3 + first_token_ms)},
+                **context,
                 "algorithmic_tflop_per_request": total_flops / 1e12,
                 "request_tflops": total_flops / (seconds / args.steps) / 1e12,
                 "request_frac_of_sustained_peak": total_flops / (seconds / args.steps) / 1e12 / peaks["bf16_tflops_sustained"],
@@ -518,6 +522,7 @@ def main():
     ap.add_argument("--layers", type=int, default=0, help="truncate the stack (ncu captures of a small case only)")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-graph", action="store_true")
+    ap.add_argument("--no-context", action="store_true", help="skip the context measurements (full prefill, variants, first token)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
     if args.impl == "reference":
