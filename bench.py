@@ -26,9 +26,9 @@ ROOT = os.path.dirname(os.path.abspath(__file__))
 if ROOT not in sys.path:
     sys.path.insert(0, ROOT)
 
-# DRAM bytes (read + write) per launch from the ncu capture summarised in profiles/gemm_tc_kernel_llama8b_2layer.txt:
+# DRAM bytes (read + write) per launch from the ncu capture summarised in profiles/gemm_kernels_llama8b_2layer.txt:
 # the SwiGLU GEMM of a sparse layer (M = 804) and of the full block (M = 5152) at Llama-8B width.
-NCU_TRAFFIC = {("llama8b_10x512", "gemm_swiglu"): {"sparse": 255.72e6 + 19.23e6, "full": 390.77e6 + 136.75e6}}
+NCU_TRAFFIC = {("llama8b_10x512", "gemm_swiglu"): {"sparse": 255.70e6 + 19.30e6, "full": 453.80e6 + 137.45e6}}
 
 METRIC = "context_tokens_fused_per_s"
 UNIT = "tokens/s"
