@@ -145,11 +145,75 @@ struct TcLayout {
   static constexpr int SMEM_BYTES = BAR_OFFSET + 256 + 1024;  // barriers + slack for the 1024-byte alignment
 };
 
+// QKV epilogue of one row: bias, RoPE with the prefetched (cos, sin) row, q -> buffer, k/v -> cache row pos[m].
+template <int BN, int D>
+__device__ __forceinline__ void tc_epilogue_qkv_row(const TcParams& p, uint32_t trow, int gr, bool row_ok, int seg, int nb0,
+                                                    const uint4* pre, int qkv_pos) {
+  const int kind = p.kind[seg];
+  constexpr int half = D / 2;
+  const bf16* bias = p.bias[seg];
+  // the row's position was read and checked, and its cos/sin row fetched into `pre`, while the main loop ran
+  const bool ok = row_ok && qkv_pos >= 0;
+  const int ps = ok ? qkv_pos : 0;
+  const float2* cs_row = reinterpret_cast<const float2*>(pre);
+  bf16* dst;
+  if (kind == 0) dst = p.q_out + (size_t)(row_ok ? gr : 0) * (p.Hq * D) + nb0;
+  else if (kind == 1) dst = p.k_cache + (size_t)ps * (p.Hkv * D) + nb0;
+  else dst = p.v_cache + (size_t)ps * (p.Hkv * D) + nb0;
+  // pairs of 32-column chunks that hold the two halves of the rotation pairs (same chunk twice for the
+  // interleaved layout and for V, which is not rotated)
+  const int pair_stride = (p.layout == 0) ? half / 32 : 0;  // D=128: 2 chunks; D=64: 1 chunk
+#pragma unroll
+  for (int c = 0; c < BN / 32; ++c) {
+    const int in_head = (c * 32) % D;  // static after unrolling: `pre` stays in registers
+    if (p.layout == 0 && in_head >= half) continue;  // handled together with its low half
+    __syncwarp();
+    float a[32], b[32];
+    tc_ld32(trow + c * 32, a);
+    if (p.layout == 0) tc_ld32(trow + (c + pair_stride) * 32, b);
+    tc_wait_ld();
+    if (!ok) continue;
+    const int ca = c * 32, cb = (c + pair_stride) * 32;
+    if (bias) {
+      float t[32];
+      load32_bf16(bias + nb0 + ca, t);
+#pragma unroll
+      for (int e = 0; e < 32; ++e) a[e] += t[e];
+      if (p.layout == 0) {
+        load32_bf16(bias + nb0 + cb, t);
+#pragma unroll
+        for (int e = 0; e < 32; ++e) b[e] += t[e];
+      }
+    }
+    if (kind != 2) {
+      if (p.layout == 0) {
+#pragma unroll
+        for (int e = 0; e < 32; ++e) {
+          const float2 cs = cs_row[in_head + e];
+          const float x = a[e], y = b[e];
+          a[e] = x * cs.x - y * cs.y;
+          b[e] = x * cs.y + y * cs.x;
+        }
+      } else {
+#pragma unroll
+        for (int e = 0; e < 16; ++e) {
+          const float2 cs = cs_row[in_head / 2 + e];
+          const float x = a[2 * e], y = a[2 * e + 1];
+          a[2 * e] = x * cs.x - y * cs.y;
+          a[2 * e + 1] = x * cs.y + y * cs.x;
+        }
+      }
+    }
+    store32_bf16(dst + ca, a);
+    if (p.layout == 0) store32_bf16(dst + cb, b);
+  }
+}
+
 // Epilogue of one accumulator row (thread = row `gr` of the output, `trow` its tensor-memory address), straight out
 // of registers.  For EPI_RESIDUAL the row's old values arrive in `pre` (see tc_prefetch_residual).
 template <int EPI, int BN>
 __device__ __forceinline__ void tc_epilogue_row(const TcParams& p, uint32_t trow, int gr, bool row_ok, int nt, int seg, int nb0,
-                                                const uint4* pre) {
+                                                const uint4* pre, int qkv_pos) {
     if (EPI == EPI_RESIDUAL) {
       // the old values of C were fetched while the main loop ran (`pre`): only tensor memory is waited for here
       const int n0 = nt * BN;
@@ -183,73 +247,32 @@ __device__ __forceinline__ void tc_epilogue_row(const TcParams& p, uint32_t trow
         }
       }
     } else {
-      const int kind = p.kind[seg];
-      const int D = p.D, half = D / 2;
-      const bf16* bias = p.bias[seg];
-      int ps = row_ok ? p.pos[gr] : 0;
-      bool ok = row_ok;
-      if (row_ok && (ps < 0 || ps >= p.kv_len || ps >= p.max_pos)) {
-        atomicOr(p.status, A3_DEV_BAD_POSITION);
-        ok = false;
-        ps = 0;
-      }
-      bf16* dst;
-      if (kind == 0) dst = p.q_out + (size_t)(row_ok ? gr : 0) * (p.Hq * D) + nb0;
-      else if (kind == 1) dst = p.k_cache + (size_t)ps * (p.Hkv * D) + nb0;
-      else dst = p.v_cache + (size_t)ps * (p.Hkv * D) + nb0;
-      const float2* trot = p.tab + (size_t)ps * half;
-      // pairs of 32-column chunks that hold the two halves of the rotation pairs (same chunk twice for the
-      // interleaved layout and for V, which is not rotated)
-      const int pair_stride = (p.layout == 0) ? half / 32 : 0;  // D=128: 2 chunks; D=64: 1 chunk
-#pragma unroll 1
-      for (int c = 0; c < BN / 32; ++c) {
-        const int in_head = (c * 32) % D;
-        if (p.layout == 0 && in_head >= half) continue;  // handled together with its low half
-        __syncwarp();
-        float a[32], b[32];
-        tc_ld32(trow + c * 32, a);
-        if (p.layout == 0) tc_ld32(trow + (c + pair_stride) * 32, b);
-        tc_wait_ld();
-        if (!ok) continue;
-        const int ca = c * 32, cb = (c + pair_stride) * 32;
-        if (bias) {
-          float t[32];
-          load32_bf16(bias + nb0 + ca, t);
-#pragma unroll
-          for (int e = 0; e < 32; ++e) a[e] += t[e];
-          if (p.layout == 0) {
-            load32_bf16(bias + nb0 + cb, t);
-#pragma unroll
-            for (int e = 0; e < 32; ++e) b[e] += t[e];
-          }
-        }
-        if (kind != 2) {
-          if (p.layout == 0) {
-#pragma unroll
-            for (int e = 0; e < 32; ++e) {
-              const float2 cs = __ldg(trot + in_head + e);
-              const float x = a[e], y = b[e];
-              a[e] = x * cs.x - y * cs.y;
-              b[e] = x * cs.y + y * cs.x;
-            }
-          } else {
-#pragma unroll
-            for (int e = 0; e < 16; ++e) {
-              const float2 cs = __ldg(trot + in_head / 2 + e);
-              const float x = a[2 * e], y = a[2 * e + 1];
-              a[2 * e] = x * cs.x - y * cs.y;
-              a[2 * e + 1] = x * cs.y + y * cs.x;
-            }
-          }
-        }
-        store32_bf16(dst + ca, a);
-        if (p.layout == 0) store32_bf16(dst + cb, b);
-      }
+      if (p.D == 128) tc_epilogue_qkv_row<BN, 128>(p, trow, gr, row_ok, seg, nb0, pre, qkv_pos);
+      else tc_epilogue_qkv_row<BN, 64>(p, trow, gr, row_ok, seg, nb0, pre, qkv_pos);
     }
 }
 
 // Old values of this thread's row of C for the residual epilogue: issued before the accumulator is waited for, so
 // the global-memory latency (a row per lane: uncoalesced, L2-resident) hides behind the main loop.
+// Position of this thread's row (checked; -1 if unusable) and, for q and k tiles, the row's D/2 (cos, sin) pairs into
+// `pre`: issued before the accumulator is waited for, like the residual rows below.
+__device__ __forceinline__ int tc_prefetch_rope(const TcParams& p, int gr, bool row_ok, int seg, uint4 (&pre)[32]) {
+  if (!row_ok) return -1;
+  const int ps = p.pos[gr];
+  if (ps < 0 || ps >= p.kv_len || ps >= p.max_pos) {
+    atomicOr(p.status, A3_DEV_BAD_POSITION);
+    return -1;
+  }
+  if (p.kind[seg] != 2) {
+    const uint4* src = reinterpret_cast<const uint4*>(p.tab + (size_t)ps * (p.D / 2));
+    const int nvec = p.D / 4;  // D/2 float2 = D/4 16-byte vectors (at most 32)
+#pragma unroll
+    for (int i = 0; i < 32; ++i)
+      if (i < nvec) pre[i] = __ldg(src + i);
+  }
+  return ps;
+}
+
 template <int BN>
 __device__ __forceinline__ void tc_prefetch_residual(const TcParams& p, int gr, bool row_ok, int nt, uint4 (&pre)[BN / 8]) {
   const int n0 = nt * BN;
@@ -371,11 +394,13 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     const int gr = m0 + row;
     const bool row_ok = gr < p.M;
     const uint32_t trow = tmem_base + ((uint32_t)(quarter * 32) << 16);
-    uint4 pre[EPI == EPI_RESIDUAL ? BN / 8 : 1];
+    uint4 pre[EPI == EPI_RESIDUAL ? BN / 8 : (EPI == EPI_QKV ? 32 : 1)];
+    int qkv_pos = -1;
     if (EPI == EPI_RESIDUAL) tc_prefetch_residual<BN>(p, gr, row_ok, nt, *reinterpret_cast<uint4(*)[BN / 8]>(pre));
+    if (EPI == EPI_QKV) qkv_pos = tc_prefetch_rope(p, gr, row_ok, seg, *reinterpret_cast<uint4(*)[32]>(pre));
     const bool ready = mbar_wait(tmem_full_bar, 0, abort_flag, p.status);
     tc_fence_after();
-    if (ready) tc_epilogue_row<EPI, BN>(p, trow, gr, row_ok, nt, seg, nb0, pre);
+    if (ready) tc_epilogue_row<EPI, BN>(p, trow, gr, row_ok, nt, seg, nb0, pre, qkv_pos);
   }
   tc_fence_before();
   __syncthreads();
@@ -557,11 +582,13 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
     const int gr = m0 + row;
     const bool row_ok = gr < p.M;
     const uint32_t trow = tmem_base + ((uint32_t)(quarter * 32) << 16);
-    uint4 pre[EPI == EPI_RESIDUAL ? BN / 8 : 1];
+    uint4 pre[EPI == EPI_RESIDUAL ? BN / 8 : (EPI == EPI_QKV ? 32 : 1)];
+    int qkv_pos = -1;
     if (EPI == EPI_RESIDUAL) tc_prefetch_residual<BN>(p, gr, row_ok, nt, *reinterpret_cast<uint4(*)[BN / 8]>(pre));
+    if (EPI == EPI_QKV) qkv_pos = tc_prefetch_rope(p, gr, row_ok, seg, *reinterpret_cast<uint4(*)[32]>(pre));
     const bool ready = mbar_wait(tmem_full_bar, 0, abort_flag, p.status);
     tc_fence_after();
-    if (ready) tc_epilogue_row<EPI, BN>(p, trow, gr, row_ok, nt, seg, nb0, pre);
+    if (ready) tc_epilogue_row<EPI, BN>(p, trow, gr, row_ok, nt, seg, nb0, pre, qkv_pos);
   }
   tc_fence_before();
   cluster_sync_all();  // neither CTA releases tensor or shared memory while the other may still use it
