@@ -85,7 +85,10 @@ scores_kernel(const bf16* __restrict__ q, const int32_t* __restrict__ q_pos, int
   float total = 0.f;  // thread c < 64 owns cache slot key0 + c
   float head_total = 0.f;
 
-  for (int g = 0; g < Hkv; ++g) {
+  // gridDim.y == 1: this CTA walks all KV heads (their sum is Eq. 3's score); gridDim.y == Hkv: one KV head per CTA
+  // (the per-head votes of the eviction step, where no sum over heads is wanted)
+  const int g_begin = gridDim.y == 1 ? 0 : blockIdx.y, g_end = gridDim.y == 1 ? Hkv : blockIdx.y + 1;
+  for (int g = g_begin; g < g_end; ++g) {
     __syncthreads();  // previous users of sk / sq are done
     load_tile<D>(sk, k, [&](int r) -> const bf16* {
       int key = key0 + r;
@@ -165,7 +168,7 @@ int scores_pass(const a3_handle* h, const bf16* q, const int32_t* q_pos, int nq,
   if (kv_len <= 0) return A3_OK;
   const int Hq = h->m.n_q_heads, Hkv = h->m.n_kv_heads, D = h->m.head_dim;
   const float scale_log2 = LOG2E / sqrtf((float)D);
-  dim3 grid(cdiv(kv_len, AT_BN));
+  dim3 grid(cdiv(kv_len, AT_BN), (per_head && !scores) ? Hkv : 1);
   ProfScope prof(h, A3_K_SCORES, st);
   if (D == 128) scores_kernel<128><<<grid, AT_THREADS, 0, st>>>(q, q_pos, nq, k, kv_len, cand_begin, cand_end, lse, scores, Hq, Hkv, scale_log2, per_head);
   else scores_kernel<64><<<grid, AT_THREADS, 0, st>>>(q, q_pos, nq, k, kv_len, cand_begin, cand_end, lse, scores, Hq, Hkv, scale_log2, per_head);
