@@ -151,6 +151,68 @@ def test_llama8b_10x512_three_layers():
     c.eng.close()
 
 
+def test_llama8b_10x512_extensions_three_layers():
+    """The rows built after the hot path, at the benchmark configuration's width and length: scores from the cached
+    keys, `ex` eviction inside the request, the value-deviation selector."""
+    c = Case("llama8b_10x512")
+    m, r = c.m, c.r
+    p = O.recompute_count(r.ratio, r.n, r.n_ctx)
+    Kr, Vr = c.buffers()
+    c.eng.rope_rerotate(c.tab, len(c.ck), max(r.chunk_lens), Kr, Vr)
+    # (i) cached-key scores: exact selection on the GPU's own scores, rows outside R untouched at EVERY layer
+    K, V = c.buffers()
+    req, out = c.eng.make_request(c.tab, len(c.ck), max(r.chunk_lens), r.n_ctx, r.n_question, c.x0, K, V, ratio=r.ratio,
+                                  select_layer=r.select_layer, score_source=1)
+    c.eng.fuse_request(req)
+    assert c.eng.device_status() == 0
+    rows = out["rows"].cpu().numpy()
+    s = out["scores"].cpu().numpy().astype(np.float64)
+    assert rows[:p].tolist() == O.topk_select(s, 0, r.n_ctx, p).tolist() and rows[p:].tolist() == list(range(r.n_ctx, r.n))
+    assert 0.5 * r.n_question * m.n_q_heads < s.sum() <= r.n_question * m.n_q_heads * (1 + 1e-5)
+    keep = torch.ones(r.n, dtype=torch.bool, device=DEV)
+    keep[out["rows"].long()] = False
+    assert torch.equal(K[:, keep], Kr[:, keep]) and torch.equal(V[:, keep], Vr[:, keep])
+    # (the score kernel itself is checked against the oracle at this size in test_query_scores_parity)
+    # (ii) eviction at C = 1024 with pooling: kept sets well-formed, compaction exact, fusion unchanged
+    K2, V2 = c.buffers()
+    req2, out2 = c.eng.make_request(c.tab, len(c.ck), max(r.chunk_lens), r.n_ctx, r.n_question, c.x0, K2, V2, ratio=r.ratio,
+                                    select_layer=r.select_layer, evict_capacity=1024, evict_pool=7)
+    c.eng.fuse_request(req2)
+    assert c.eng.device_status() == 0
+    K0, V0, out0 = c.fuse()
+    assert torch.equal(K2, K0) and torch.equal(V2, V0) and torch.equal(out2["x"], out0["x"])
+    kept = out2["kept"].cpu().numpy()
+    k = 1024 - r.n_question
+    assert kept.shape == (m.n_layers, m.n_kv_heads, 1024)
+    for l in range(m.n_layers):
+        for g in range(m.n_kv_heads):
+            kg = kept[l, g]
+            assert (np.diff(kg) > 0).all() and kg[k:].tolist() == list(range(r.n_ctx, r.n)) and kg[0] >= 0
+            idx = torch.from_numpy(kg.astype(np.int64)).to(DEV)
+            assert torch.equal(out2["k_evicted"][l][:, g], K2[l][idx, g]) and torch.equal(out2["v_evicted"][l][:, g], V2[l][idx, g])
+    assert len({tuple(kept[1, g].tolist()) for g in range(m.n_kv_heads)}) > 1  # heads keep different tokens
+    # (iii) value deviation: scores are the squared distances between cached and true values at the selection layer
+    K3, V3 = c.buffers()
+    req3, out3 = c.eng.make_request(c.tab, len(c.ck), max(r.chunk_lens), r.n_ctx, r.n_question, c.x0, K3, V3, ratio=r.ratio,
+                                    select_layer=r.select_layer, selector=1)
+    c.eng.fuse_request(req3)
+    assert c.eng.device_status() == 0
+    s3 = out3["scores"].cpu().numpy().astype(np.float64)
+    rows3 = out3["rows"].cpu().numpy()
+    assert rows3[:p].tolist() == O.topk_select(s3, 0, r.n_ctx, p).tolist()
+    ls = r.select_layer
+    keep3 = torch.ones(r.n, dtype=torch.bool, device=DEV)
+    keep3[out3["rows"].long()] = False
+    # rows that were NOT recomputed still hold the true values at the selection layer: recompute the distances there
+    rng = np.random.default_rng(5)
+    cand = np.flatnonzero(keep3[: r.n_ctx].cpu().numpy())
+    for i in rng.choice(cand, size=32, replace=False):
+        want = float(((f64(V3[ls, i]) - f64(Vr[ls, i])) ** 2).sum())
+        assert abs(s3[i] - want) <= 1e-4 * max(want, 1e-6) + 1e-7
+    assert s3[: r.chunk_lens[0]].max() <= 1e-3 * max(s3.max(), 1e-9) + 1e-6  # first chunk: cached values are (nearly) the true ones
+    c.eng.close()
+
+
 def test_llama8b_10x512_full_depth_runs_clean():
     c = Case("llama8b_10x512", layers=32)
     K, V, out = c.fuse()

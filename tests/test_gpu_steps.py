@@ -277,7 +277,10 @@ def test_query_scores_parity(a3mod, shape, n_ctx, nq, n_sys):
 
 
 @pytest.mark.parametrize("shape,kv_len,M,seed", [(W.TINY3, 528, 95, 0), (W.TINY_GQA, 700, 131, 1), (W.TINY_G7, 300, 77, 2),
-                                                 (W.TINY_GQA, 257, 257, 3), (W.TINY3, 40, 1, 4)])
+                                                 (W.TINY_GQA, 257, 257, 3), (W.TINY3, 40, 1, 4),
+                                                 # row counts around the 128-row tile and the 256-row CTA-pair boundaries
+                                                 (W.TINY3, 600, 128, 5), (W.TINY_GQA, 600, 129, 6), (W.TINY3, 700, 384, 7),
+                                                 (W.TINY_G7, 520, 511, 8)])
 def test_recompute_layer_parity(a3mod, shape, kv_len, M, seed):
     m = shape
     # weights N(0, 0.05), hidden rows N(0,1): K/V come out with a spread of about one, as at full width
