@@ -13,10 +13,12 @@
 //                       softmax threads do.
 //   warps 2..9          two threads per row, each owning half of the tile's key columns with an exponent
 //                       reference, a row sum and a TMEM output accumulator of its own: the row of S is read into
-//                       registers, its maximum checked against the lazily raised reference (the accumulator is
-//                       rescaled in TMEM only when the reference moves), P = exp2(s - ref) is written as bf16
-//                       pairs over the columns S came from; at the end of an item the two partial softmaxes of a
-//                       row are merged, normalised and stored.
+//                       registers, P = exp2(s * scale - ref) (one FMA and one ex2.approx per element) is written
+//                       as bf16 pairs over the columns S came from.  The reference is the first tile's maximum; no
+//                       maximum is tracked afterwards - a logit far above the reference shows as a row sum beyond
+//                       2^16, and only then is the tile's maximum taken, the reference raised, the accumulator
+//                       rescaled in TMEM and the tile redone.  At the end of an item the two partial softmaxes of
+//                       a row are merged, normalised and stored.
 // TMEM (512 columns): S buffers at 0 and 128, the two output accumulators at 256 and 256 + D.
 // Statistics are fp32 in the exp2 domain.  Every mbarrier wait is bounded (see a3_gemm.cu); there is no block-
 // wide or named barrier inside the loops, so a role that gives up cannot strand another.
@@ -384,7 +386,7 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
     const int row = quarter * 32 + lane;
     const uint32_t lane_addr = (uint32_t)(quarter * 32) << 16;
     const uint32_t tmem_oh = tmem_o + half * D;  // this thread's accumulator
-    constexpr float RESCALE_TH = 8.f;
+    constexpr float OVERFLOW_GUARD = 65536.f;
     uint32_t it = 0, px = 0;  // running key tile; running count of pair exchanges (parity of the pair barrier)
     bool ok = true;
     // publish `mine`, meet the partner, return the partner's value; false if the wait was abandoned
@@ -439,9 +441,7 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
         mbar_arrive(q_ready);
       }
 
-      // Exponent reference m_ref and row sum l_run of this thread's keys.  The reference is the true maximum of the
-      // first tile and is raised later only when a logit exceeds it by more than RESCALE_TH (rare): then the output
-      // accumulated in TMEM and l_run are rescaled first.
+      // Exponent reference m_ref and row sum l_run of this thread's keys (see the file header for the protocol).
       float m_ref = 0.f, l_run = 0.f;
       uint32_t it_last = it;
       for (int kt = 0; kt < w.nkt; ++kt, ++it) {
@@ -453,39 +453,63 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
         const uint32_t ts = tmem_s0 + (it & 1) * 128 + lane_addr + half * 64;
         const int key0 = (w.kt0 + kt) * ATC_BN + half * 64;  // first key of this thread's columns
         const bool need_mask = (w.kt0 + kt) * ATC_BN + ATC_BN - 1 > w.minpos;
-        // pass 1: scaled (and masked) logits into registers, their maximum
+        // The row's 64 logits of this thread, raw, into registers
         float x[64];
         ld32(ts, x);
         ld32(ts + 32, x + 32);
         wait_ld();
-        float mx;
-        {
-          float m4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
-          if (need_mask) {
-#pragma unroll
-            for (int e = 0; e < 64; ++e) {
-              x[e] = key0 + e > lim ? -INFINITY : x[e] * scale_log2;
-              m4[e & 3] = fmaxf(m4[e & 3], x[e]);
-            }
-          } else {
-#pragma unroll
-            for (int e = 0; e < 64; ++e) {
-              x[e] *= scale_log2;
-              m4[e & 3] = fmaxf(m4[e & 3], x[e]);
-            }
-          }
-          mx = fmaxf(fmaxf(m4[0], m4[1]), fmaxf(m4[2], m4[3]));
-        }
         if (want_o && it >= 2) {
           // keeps every phase of p_free[b] observed in order, so that the parity waits below cannot mistake an older
           // completion for the one they mean (P V of running tile it-2 finished long ago: this does not block)
           ok = __all_sync(0xffffffffu, mbar_wait(p_free(it & 1), ((it >> 1) & 1) ^ 1, abort_flag, status));
           if (!ok) break;
         }
+        // maximum of the scaled, masked logits (first tile and the rare re-reference only)
+        auto row_max = [&]() {
+          float m4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
+#pragma unroll
+          for (int e = 0; e < 64; ++e) {
+            const float t = (need_mask && key0 + e > lim) ? -INFINITY : x[e] * scale_log2;
+            m4[e & 3] = fmaxf(m4[e & 3], t);
+          }
+          return fmaxf(fmaxf(m4[0], m4[1]), fmaxf(m4[2], m4[3]));
+        };
+        // x <- exp2(x * scale - m_ref) (one FMA and one ex2.approx per element; ex2 maps -inf to +0); returns the sum
+        auto to_probabilities = [&]() {
+          float ls[4] = {0.f, 0.f, 0.f, 0.f};
+          const float neg_ref = -m_ref;
+          if (need_mask) {
+#pragma unroll
+            for (int e = 0; e < 64; ++e) {
+              float t = fmaf(x[e], scale_log2, neg_ref);
+              if (key0 + e > lim) t = -INFINITY;
+              x[e] = ex2_approx(t);
+              ls[e & 3] += x[e];
+            }
+          } else {
+#pragma unroll
+            for (int e = 0; e < 64; ++e) {
+              x[e] = ex2_approx(fmaf(x[e], scale_log2, neg_ref));
+              ls[e & 3] += x[e];
+            }
+          }
+          return (ls[0] + ls[1]) + (ls[2] + ls[3]);
+        };
         if (kt == 0) {
+          const float mx = row_max();
           m_ref = mx == -INFINITY ? 0.f : mx;
-        } else if (__any_sync(0xffffffffu, mx - m_ref > RESCALE_TH)) {
-          const float raise = fmaxf(mx - m_ref, 0.f);  // lanes below the threshold may move too: any value >= their maximum is valid
+        }
+        float lsum = to_probabilities();
+        // No maximum is tracked on the way: a logit far above the reference shows in the sum (each of the 64 terms
+        // is at most the largest one), and anything below 2^16 is harmless for bf16 P and the fp32 accumulators.
+        // Above it - rare - the reference is raised to the tile's true maximum, the output and the sum so far are
+        // rescaled, and the tile is redone from the logits still in tensor memory.
+        if (kt > 0 && __any_sync(0xffffffffu, !(lsum <= OVERFLOW_GUARD))) {
+          ld32(ts, x);
+          ld32(ts + 32, x + 32);
+          wait_ld();
+          const float mx = row_max();
+          const float raise = fmaxf(mx - m_ref, 0.f);  // lanes that triggered nothing keep their reference (raise 0)
           const float f = exp2f(-raise);
           m_ref += raise;
           l_run *= f;
@@ -506,17 +530,9 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
             }
             wait_st();
           }
+          lsum = to_probabilities();
         }
-        // pass 2: probabilities (ex2.approx maps -inf to +0), row sum in four chains
-        {
-          float ls[4] = {0.f, 0.f, 0.f, 0.f};
-#pragma unroll
-          for (int e = 0; e < 64; ++e) {
-            x[e] = ex2_approx(x[e] - m_ref);
-            ls[e & 3] += x[e];
-          }
-          l_run += (ls[0] + ls[1]) + (ls[2] + ls[3]);
-        }
+        l_run += lsum;
         if (want_o) {
           // P as bf16 pairs over the first 32 of this thread's 64 S columns (all of them are in registers by now):
           // the A operand of the P V MMA is read from tensor memory

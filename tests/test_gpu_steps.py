@@ -317,6 +317,58 @@ def test_recompute_layer_parity(a3mod, shape, kv_len, M, seed):
     eng.close()
 
 
+@pytest.mark.parametrize("shape,kv_len,M,beta", [(W.TINY_GQA, 1200, 131, 6.0), (W.TINY3, 900, 77, 9.0)])
+def test_recompute_layer_growing_logits(a3mod, shape, kv_len, M, beta):
+    """Keys whose projection on a fixed direction grows with the position: for the query heads that point along it
+    the logits climb by tens of nats from key tile to key tile, so the attention kernel's exponent reference (taken
+    from the first tile) must be raised again and again and the accumulated output rescaled; heads that point the
+    other way see falling logits.  Against the exact softmax of the oracle."""
+    m = shape
+    eng, layers, dev = make_engine(a3mod, m, seed=11, w_std=0.05)
+    model, weights = oracle_model(m), oracle_weights(layers)
+    rng = np.random.default_rng(311)
+    pos = np.sort(rng.choice(kv_len, size=M, replace=False))
+    pos[-1] = kv_len - 1
+    X = W.bf16_round(rng.standard_normal((M, m.d_model), dtype=np.float32))
+    layer = m.n_layers - 1
+    v_dir = rng.standard_normal((m.n_kv_heads, m.head_dim)).astype(np.float32)
+    # the queries do not depend on the cache: take them from a preliminary oracle pass and scale the ramp so that the
+    # steepest head of the last row climbs by `beta` * 10 in the exp2 domain over the whole cache
+    zero = np.zeros((kv_len, m.n_kv_heads, m.head_dim))
+    q0 = O.recompute_layer(X.astype(np.float64), pos, weights[layer], model, zero.copy(), zero.copy(), rnd=O.round_bf16, return_parts=True)[1]["q"]
+    G0 = m.n_q_heads // m.n_kv_heads
+    slope = max(abs(float(q0[M - 1, h] @ v_dir[h // G0])) for h in range(m.n_q_heads)) / np.sqrt(m.head_dim) * np.log2(np.e)
+    ramp = (np.arange(kv_len, dtype=np.float32) / kv_len * (beta * 10.0 / slope))[:, None, None]
+    Kc = W.bf16_round(ramp * v_dir[None] + 0.05 * rng.standard_normal((kv_len, m.n_kv_heads, m.head_dim)).astype(np.float32))
+    Vc = W.bf16_round(rng.standard_normal((kv_len, m.n_kv_heads, m.head_dim)).astype(np.float32))
+    dX, dpos = to_dev(X, dev), torch.from_numpy(pos.astype(np.int32)).to(dev)
+    dK, dV = to_dev(Kc, dev), to_dev(Vc, dev)
+    lse = torch.empty((M, m.n_q_heads), dtype=torch.float32, device=dev)
+    eng.recompute_layer(layer, dX, dpos, dK, dV, lse_out=lse)
+    assert eng.device_status() == 0
+    Ko, Vo = Kc.astype(np.float64), Vc.astype(np.float64)
+    Xo, parts = O.recompute_layer(X.astype(np.float64), pos, weights[layer], model, Ko, Vo, rnd=O.round_bf16, return_parts=True)
+    # the case really is the one described: within single rows the logits span far more than the 2^16 guard
+    q, Kf = parts["q"], Ko
+    G = m.n_q_heads // m.n_kv_heads
+    row = M - 1
+    spans = []
+    for h in range(m.n_q_heads):
+        logit = Kf[: pos[row] + 1, h // G] @ q[row, h] / np.sqrt(m.head_dim) * np.log2(np.e)
+        spans.append(logit[-128:].max() - logit[:128].max())
+    assert max(spans) > 30, spans  # at least one head climbs by more than 2^30 from the first to the last key tile
+    gX = f64(dX)
+    assert np.isfinite(gX).all()
+    check_kv(f64(dK)[pos], parts["k_exact"], "recomputed K rows")
+    check_kv(gX, parts["x_exact"], "hidden rows", scale=2.0 * float(parts["x_exact"].std()))
+    # The two pipelines round q to bf16 from slightly different fp32 values; an element that lands on the other side
+    # of a rounding boundary moves a logit by 2^-9 |q_e| |k_e| / sqrt(D), and the keys are large here: allow two such
+    # flips per row on the log-sum-exp (the usual 5e-3 gate assumes keys of unit size).
+    lse_tol = 2 * 2.0 ** -9 * float(np.abs(q).max()) * float(np.abs(Kc).max()) / np.sqrt(m.head_dim)
+    np.testing.assert_allclose(lse.cpu().numpy(), parts["lse"], atol=max(5e-3, lse_tol), rtol=1e-5)
+    eng.close()
+
+
 def test_recompute_layer_rejects_bad_arguments(a3mod):
     m = W.TINY3
     eng, _, dev = make_engine(a3mod, m, max_pos=600)
