@@ -487,11 +487,17 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
               ls[e & 3] += x[e];
             }
           } else {
+            // packed fp32 pairs (fma.rn.f32x2 / add.rn.f32x2): half the issue slots for the FMA and the sum
+            const float2 sc2 = make_float2(scale_log2, scale_log2), nr2 = make_float2(neg_ref, neg_ref);
+            float2 s2[2] = {make_float2(0.f, 0.f), make_float2(0.f, 0.f)};
 #pragma unroll
-            for (int e = 0; e < 64; ++e) {
-              x[e] = ex2_approx(fmaf(x[e], scale_log2, neg_ref));
-              ls[e & 3] += x[e];
+            for (int e = 0; e < 64; e += 2) {
+              const float2 t = __ffma2_rn(make_float2(x[e], x[e + 1]), sc2, nr2);
+              x[e] = ex2_approx(t.x);
+              x[e + 1] = ex2_approx(t.y);
+              s2[(e >> 1) & 1] = __fadd2_rn(s2[(e >> 1) & 1], make_float2(x[e], x[e + 1]));
             }
+            ls[0] = s2[0].x, ls[1] = s2[0].y, ls[2] = s2[1].x, ls[3] = s2[1].y;
           }
           return (ls[0] + ls[1]) + (ls[2] + ls[3]);
         };
