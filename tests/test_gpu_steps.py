@@ -539,3 +539,54 @@ def test_evict_layer_bad_arguments(a3mod):
     with pytest.raises(a3mod.A3Error):
         eng.evict_layer(q, pos, lse, K, K, 0, n_ctx - 1, 32)  # n_ctx + nq != kv_len
     eng.close()
+
+
+@pytest.mark.parametrize("shape,kv_len,M,grow", [(W.TINY_GQA, 1500, 700, False), (W.TINY_G7, 900, 333, False), (W.TINY_GQA, 1200, 300, True),
+                                                  (W.TINY_GQA, 300, 31, False)])
+def test_attention_two_row_tiles_per_cta(a3mod, shape, kv_len, M, grow):
+    """The attention kernel that gives a CTA two row tiles (chosen by itself only for launches with many row tiles) on
+    small cases, forced: against the oracle like the one-tile kernel, including logits that outgrow the exponent
+    reference (grow), an odd number of row tiles and a single, ragged one."""
+    import ctypes
+    m = shape
+    eng, layers, dev = make_engine(a3mod, m, seed=21, w_std=0.05)
+    lib = a3mod._load()
+    lib.a3_internal_set_attn_pair.argtypes = [ctypes.c_int]
+    model, weights = oracle_model(m), oracle_weights(layers)
+    rng = np.random.default_rng(77)
+    pos = np.sort(rng.choice(kv_len, size=M, replace=False))
+    pos[-1] = kv_len - 1
+    X = W.bf16_round(rng.standard_normal((M, m.d_model), dtype=np.float32))
+    layer = m.n_layers - 1
+    if grow:
+        v_dir = rng.standard_normal((m.n_kv_heads, m.head_dim)).astype(np.float32)
+        zero = np.zeros((kv_len, m.n_kv_heads, m.head_dim))
+        q0 = O.recompute_layer(X.astype(np.float64), pos, weights[layer], model, zero.copy(), zero.copy(), rnd=O.round_bf16, return_parts=True)[1]["q"]
+        G0 = m.n_q_heads // m.n_kv_heads
+        slope = max(abs(float(q0[M - 1, h] @ v_dir[h // G0])) for h in range(m.n_q_heads)) / np.sqrt(m.head_dim) * np.log2(np.e)
+        ramp = (np.arange(kv_len, dtype=np.float32) / kv_len * (60.0 / slope))[:, None, None]
+        Kc = W.bf16_round(ramp * v_dir[None] + 0.05 * rng.standard_normal((kv_len, m.n_kv_heads, m.head_dim)).astype(np.float32))
+    else:
+        Kc = W.bf16_round(rng.standard_normal((kv_len, m.n_kv_heads, m.head_dim)).astype(np.float32))
+    Vc = W.bf16_round(rng.standard_normal((kv_len, m.n_kv_heads, m.head_dim)).astype(np.float32))
+    Ko, Vo = Kc.astype(np.float64), Vc.astype(np.float64)
+    Xo, parts = O.recompute_layer(X.astype(np.float64), pos, weights[layer], model, Ko, Vo, rnd=O.round_bf16, return_parts=True)
+    dpos = torch.from_numpy(pos.astype(np.int32)).to(dev)
+    outs = []
+    try:
+        for rep in range(2):
+            lib.a3_internal_set_attn_pair(1)
+            dX, dK, dV = to_dev(X, dev), to_dev(Kc, dev), to_dev(Vc, dev)
+            lse = torch.empty((M, m.n_q_heads), dtype=torch.float32, device=dev)
+            eng.recompute_layer(layer, dX, dpos, dK, dV, lse_out=lse)
+            assert eng.device_status() == 0
+            outs.append((dX, lse))
+    finally:
+        lib.a3_internal_set_attn_pair(-1)
+    assert torch.equal(outs[0][0], outs[1][0]) and torch.equal(outs[0][1], outs[1][1])  # reproducible
+    gX = f64(outs[0][0])
+    assert np.isfinite(gX).all()
+    check_kv(gX, parts["x_exact"], "hidden rows", scale=2.0 * float(parts["x_exact"].std()))
+    lse_tol = 2 * 2.0 ** -9 * float(np.abs(parts["q"]).max()) * float(np.abs(Kc).max()) / np.sqrt(m.head_dim)
+    np.testing.assert_allclose(outs[0][1].cpu().numpy(), parts["lse"], atol=max(5e-3, lse_tol), rtol=1e-5)
+    eng.close()
