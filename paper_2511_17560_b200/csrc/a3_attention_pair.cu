@@ -8,7 +8,8 @@
 //   warp 0 (one lane)   TMA producer: K and V tiles, two stages each
 //   warp 1 (one lane)   tcgen05.mma: S_A = Q_A K^T, S_B = Q_B K^T, O_A += P_A V, O_B += P_B V.  P_X is read from
 //                       tensor memory, where it lies over the first half of S_X, so S_X of the next key tile is
-//                       issued after P_X V of the current one
+//                       issued after P_X V of the current one.  P V goes in two halves of 64 keys: the first is
+//                       issued as soon as its P is stored, under the softmax of the second
 //   warps 2..5          softmax of row tile A, one thread per row (exponent reference, row sum, rescale as in
 //                       a3_attention.cu; the 128 logits of a row are taken in two halves of 64)
 //   warps 6..9          the same for row tile B
@@ -88,8 +89,10 @@ attention_pair_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_cons
   auto p_ready = [&](int x) { return bars + 8u * (10 + x); };
   auto pv_done = [&](int x) { return bars + 8u * (12 + x); };
   const uint32_t q_ready = bars + 8u * 14;
-  volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(base_ptr + L::BAR_OFF + 8 * 15);
-  volatile int* abort_flag = reinterpret_cast<volatile int*>(base_ptr + L::BAR_OFF + 8 * 15 + 8);
+  auto p0_ready = [&](int x) { return bars + 8u * (15 + x); };  // P of the first 64 keys is in tensor memory
+  auto pv0_done = [&](int x) { return bars + 8u * (17 + x); };  // ... and its P V has completed
+  volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(base_ptr + L::BAR_OFF + 8 * 19);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(base_ptr + L::BAR_OFF + 8 * 19 + 8);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int G = Hq / Hkv;
@@ -113,6 +116,8 @@ attention_pair_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_cons
       mbar_init(s_full(i), 1);
       mbar_init(p_ready(i), 128);
       mbar_init(pv_done(i), 1);
+      mbar_init(p0_ready(i), 128);
+      mbar_init(pv0_done(i), 1);
     }
     mbar_init(q_ready, 256);
     abort_flag[0] = 0;
@@ -172,14 +177,15 @@ attention_pair_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_cons
         }
         commit(s_full(x));
       };
-      auto issue_pv = [&](int x, uint32_t vstage, bool first) {
+      // P V in two halves of 64 keys: the first is issued as soon as its P is there, under the softmax of the second
+      auto issue_pv_half = [&](int x, int hh, uint32_t vstage, bool first) {
         const uint32_t sv = base + L::V_OFF + vstage * L::TILE;
 #pragma unroll
-        for (int k = 0; k < ATC_BN / 16; ++k) {
+        for (int k = 4 * hh; k < 4 * hh + 4; ++k) {
           const uint64_t db = desc_mn_sw128(sv + k * 16 * 128, L::SUB);
           mma_f16_ts(tmem_base + 256 + x * 128, tmem_base + x * 128 + k * 8, db, idesc_o, !(first && k == 0));
         }
-        commit(pv_done(x));
+        commit(hh == 0 ? pv0_done(x) : pv_done(x));
       };
       bool ok = true;
       for (int r = 0; r < rounds && ok; ++r) {
@@ -201,11 +207,15 @@ attention_pair_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_cons
           const uint32_t vs = it & 1, vph = (it >> 1) & 1;
           bool v_here = false;
           if (t < w.nkt[0]) {
-            ok = mbar_wait(p_ready(0), cx[0] & 1, abort_flag, status) && mbar_wait(v_full(vs), vph, abort_flag, status);
+            ok = mbar_wait(p0_ready(0), cx[0] & 1, abort_flag, status) && mbar_wait(v_full(vs), vph, abort_flag, status);
             if (!ok) break;
             v_here = true;
             fence_after();
-            issue_pv(0, vs, t == 0);
+            issue_pv_half(0, 0, vs, t == 0);
+            ok = mbar_wait(p_ready(0), cx[0] & 1, abort_flag, status);
+            if (!ok) break;
+            fence_after();
+            issue_pv_half(0, 1, vs, t == 0);
             ++cx[0];
           }
           if (more) {
@@ -215,11 +225,15 @@ attention_pair_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_cons
             if (t + 1 < w.nkt[0]) issue_s(0, (it + 1) & 1);  // follows P_A V of this tile: P_A lies over S_A
           }
           if (t < w.nkt[1]) {
-            ok = mbar_wait(p_ready(1), cx[1] & 1, abort_flag, status);
+            ok = mbar_wait(p0_ready(1), cx[1] & 1, abort_flag, status);
             if (ok && !v_here) ok = mbar_wait(v_full(vs), vph, abort_flag, status);
             if (!ok) break;
             fence_after();
-            issue_pv(1, vs, t == 0);
+            issue_pv_half(1, 0, vs, t == 0);
+            ok = mbar_wait(p_ready(1), cx[1] & 1, abort_flag, status);
+            if (!ok) break;
+            fence_after();
+            issue_pv_half(1, 1, vs, t == 0);
             ++cx[1];
           }
           commit(v_empty(vs));
@@ -346,52 +360,6 @@ attention_pair_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_cons
           mx = fmaxf(mx, row_max64(key0 + 64));
           m_ref = mx == -INFINITY ? 0.f : mx;
         }
-        float l_tile = 0.f;
-#pragma unroll 1
-        for (int h = 0; h < 2; ++h) {
-          load64(h);
-          float lsum = to_probabilities(key0 + 64 * h);
-          // A logit far above the reference shows in the sum; anything below 2^16 is harmless.  Above it - rare -
-          // the reference goes up to this half's maximum, and what was accumulated under the old one is rescaled:
-          // the output, the row sum, and the first half of this tile's P if it is already in tensor memory.
-          if (t > 0 && __any_sync(0xffffffffu, !(lsum <= OVERFLOW_GUARD))) {
-            load64(h);
-            const float mx = row_max64(key0 + 64 * h);
-            const float raise = fmaxf(mx - m_ref, 0.f);
-            const float f = exp2f(-raise);
-            m_ref += raise;
-            l_run *= f;
-            l_tile *= f;
-            rescale_output(f);
-            if (h == 1) {
-              float pv[32];
-              ld32(ts, pv);  // 64 probabilities of the first half as bf16 pairs
-              wait_ld();
-#pragma unroll
-              for (int e = 0; e < 32; ++e) {
-                const uint32_t u = __float_as_uint(pv[e]);
-                const float lo = __uint_as_float(u << 16) * f, hi = __uint_as_float(u & 0xffff0000u) * f;
-                float two[8] = {lo, hi, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
-                pv[e] = __uint_as_float(pack8(two).x);
-              }
-              st32(ts, pv);
-              wait_st();
-            }
-            load64(h);
-            lsum = to_probabilities(key0 + 64 * h);
-          }
-          l_tile += lsum;
-          // P of this half as bf16 pairs: 32 columns at 32 h of S_X (columns whose logits are in registers or done)
-          uint32_t pk[32];
-#pragma unroll
-          for (int j = 0; j < 8; ++j) {
-            const uint4 v = pack8(xv + 8 * j);
-            pk[4 * j] = v.x, pk[4 * j + 1] = v.y, pk[4 * j + 2] = v.z, pk[4 * j + 3] = v.w;
-          }
-          st32(ts + 32 * h, reinterpret_cast<const float*>(pk));
-        }
-        wait_st();
-        l_run += l_tile;
         // Slots beyond the last visible key of the pair may hold anything (probability zero times a non-finite
         // value would still poison the product): clear those V rows of the last key tile before the first P V that
         // reads it - row tile A does it when it walks to the last tile (its P V is issued first), else B.
@@ -408,6 +376,51 @@ attention_pair_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_cons
           }
           fence_async_smem();
         }
+        float l_tile = 0.f;
+#pragma unroll 1
+        for (int h = 0; h < 2; ++h) {
+          load64(h);
+          float lsum = to_probabilities(key0 + 64 * h);
+          // A logit far above the reference shows in the sum; anything below 2^16 is harmless.  Above it - rare -
+          // the reference goes up to this half's maximum, and what was accumulated under the old one is rescaled:
+          // the row sums and the output (which, in the second half, includes the first half's P V: see below).
+          if (t > 0 && __any_sync(0xffffffffu, !(lsum <= OVERFLOW_GUARD))) {
+            load64(h);
+            const float mx = row_max64(key0 + 64 * h);
+            const float raise = fmaxf(mx - m_ref, 0.f);
+            const float f = exp2f(-raise);
+            m_ref += raise;
+            l_run *= f;
+            l_tile *= f;
+            if (h == 1) {
+              // the first half's P V was released under the old reference: once it has completed, the output holds
+              // its contribution too and the factor applies to all of it
+              ok = __all_sync(0xffffffffu, mbar_wait(pv0_done(x), cxx & 1, abort_flag, status));
+              if (!ok) break;
+              fence_after();
+            }
+            rescale_output(f);
+            load64(h);
+            lsum = to_probabilities(key0 + 64 * h);
+          }
+          l_tile += lsum;
+          // P of this half as bf16 pairs: 32 columns at 32 h of S_X (columns whose logits are in registers or done)
+          uint32_t pk[32];
+#pragma unroll
+          for (int j = 0; j < 8; ++j) {
+            const uint4 v = pack8(xv + 8 * j);
+            pk[4 * j] = v.x, pk[4 * j + 1] = v.y, pk[4 * j + 2] = v.z, pk[4 * j + 3] = v.w;
+          }
+          st32(ts + 32 * h, reinterpret_cast<const float*>(pk));
+          if (h == 0) {
+            wait_st();
+            fence_before();
+            mbar_arrive(p0_ready(x));
+          }
+        }
+        if (!ok) break;
+        wait_st();
+        l_run += l_tile;
         fence_before();
         mbar_arrive(p_ready(x));
       }
