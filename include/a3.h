@@ -18,7 +18,10 @@
  *  - Hot calls allocate nothing, do not synchronise and copy nothing between host and
  *    device (a3_fuse_request_host excepted); all work is queued on `stream`
  *    (a cudaStream_t passed as void*).  Calls on different streams may overlap only if
- *    they use different workspaces.
+ *    they use different workspaces.  A handle may be used from several host threads as
+ *    long as the calls on it do not run at the same time (the launch counter, the
+ *    profiling records and the lazily created copy stream are not locked); device
+ *    memory and kernels are per call and need no such care.
  *  - Return value: A3_OK or a negative a3_status.  Host-detectable problems are
  *    rejected before any launch.  Problems only the device can see (a position outside
  *    the cache, a non-finite score, an exhausted bounded wait) set the handle's device
