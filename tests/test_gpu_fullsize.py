@@ -4,7 +4,8 @@ The oracle cannot run these sizes whole in test time, so each request is checked
 hold at any size (the selection is the top-p of the scores the GPU computed; rows outside R keep the re-rotated
 chunk values bit for bit; scores vanish outside the candidates and their mass is bounded), (b) position recovery on
 sampled rows against the oracle, and (c) one recompute layer at full width and length, teacher-forced, on sampled
-rows the oracle computes one by one.  Stacks are truncated to three layers (selection at layer 1) except for one
+rows the oracle computes one by one.  (b) and (c) run on seeded synthetic inputs of the configuration's shapes: no
+value the library computed is ever an input of the oracle.  Stacks are truncated to three layers (selection at layer 1) except for one
 full-depth run; widths, lengths, chunk structure and ratios are the configurations' own.
 """
 from dataclasses import replace
@@ -96,33 +97,48 @@ def check_request_properties(c: Case, K, V, out, ratio=None):
     return rows, s, Kr, Vr
 
 
-def check_position_recovery_samples(c: Case, Kr, Vr, n_samples=64, seed=0):
-    """Eq. 2 on sampled (layer, chunk, token) rows against the oracle, incl. the last chunk (largest offset)."""
+def check_position_recovery_samples(c: Case, n_samples=64, seed=0):
+    """Eq. 2 at the configuration's chunk structure on seeded synthetic chunk caches (nothing the library computed
+    goes into the oracle): sampled (layer, chunk, token) rows against the oracle, incl. the last chunk (largest
+    offset); V copied bit for bit."""
     m, r = c.m, c.r
+    ck, cv = zip(*[W.make_cache_device(m, t, DEV, 7 + seed, i, std=1.2) for i, t in enumerate(r.chunk_lens)])
+    tab = c.a3.chunk_table(ck, cv, r.offsets)
+    Kr, Vr = c.buffers()
+    c.eng.rope_rerotate(tab, len(ck), max(r.chunk_lens), Kr, Vr)
+    assert c.eng.device_status() == 0
     rng = np.random.default_rng(seed)
     errs = []
     for i in range(n_samples):
         l = int(rng.integers(0, m.n_layers))
         ch = len(r.chunk_lens) - 1 if i % 4 == 0 else int(rng.integers(0, len(r.chunk_lens)))
         t = int(rng.integers(0, r.chunk_lens[ch]))
-        src = c.ck[ch][l, t].float().cpu().numpy().astype(np.float64)[None]
+        src = ck[ch][l, t].float().cpu().numpy().astype(np.float64)[None]
         want = O.rope_rotate(src, np.array([r.offsets[ch]]), m.rope_theta, m.rope_layout)[0]
         got = f64(Kr[l, r.offsets[ch] + t])
         errs.append(np.abs(got - want))
-        assert torch.equal(Vr[l, r.offsets[ch] + t], c.cv[ch][l, t])
+        assert torch.equal(Vr[l, r.offsets[ch] + t], cv[ch][l, t])
     errs = np.stack(errs)
     assert errs.max() <= KV_MAX and errs.mean() <= KV_MEAN, (errs.max(), errs.mean())
 
 
-def check_layer_samples(c: Case, layer, rows, K_layer, V_layer, n_samples=10, seed=0):
-    """One recompute layer at full width/length, teacher-forced: the GPU runs all carried rows; the oracle recomputes
-    sampled rows one by one from the same inputs (cache taken from the GPU after its scatter)."""
+def check_layer_samples(c: Case, layer, rows, n_samples=10, seed=0):
+    """One recompute layer at full width/length, teacher-forced on seeded synthetic inputs (hidden rows and a cache
+    of unit spread drawn with torch's generator; nothing the library computed goes into the oracle).  The GPU runs
+    all carried rows; the oracle projects K and V of all carried rows itself (the cache every row attends over)
+    and then recomputes sampled rows one by one."""
     m, r = c.m, c.r
+    if rows is None:
+        # a seeded selection of the request's size: p random document slots (ascending), then the question slots
+        p = O.recompute_count(r.ratio, r.n, r.n_ctx)
+        rows = np.concatenate([np.sort(np.random.default_rng(900 + seed).choice(r.n_ctx, size=p, replace=False)), np.arange(r.n_ctx, r.n)])
     M = rows.shape[0]
     g = torch.Generator(device=DEV)
     g.manual_seed(1234 + seed)
     X = torch.randn((M, m.d_model), generator=g, device=DEV, dtype=torch.float32).to(torch.bfloat16)
-    Kc, Vc = K_layer.clone(), V_layer.clone()
+    K0 = torch.randn((r.n, m.n_kv_heads, m.head_dim), generator=g, device=DEV, dtype=torch.float32).to(torch.bfloat16)
+    V0 = torch.randn((r.n, m.n_kv_heads, m.head_dim), generator=g, device=DEV, dtype=torch.float32).to(torch.bfloat16)
+    Kc, Vc = K0.clone(), V0.clone()
     pos = torch.from_numpy(rows.astype(np.int32)).to(DEV)
     Xg = X.clone()
     lse = torch.empty((M, m.n_q_heads), dtype=torch.float32, device=DEV)
@@ -131,12 +147,23 @@ def check_layer_samples(c: Case, layer, rows, K_layer, V_layer, n_samples=10, se
     rng = np.random.default_rng(seed)
     sel = np.unique(np.concatenate([[0, M - 1], rng.choice(M, size=n_samples, replace=False)]))
     w, model = c.oracle_layer(layer), oracle_model(m)
-    Ko, Vo = f64(Kc), f64(Vc)
-    Xo, parts = O.recompute_layer(f64(X[sel]), rows[sel], w, model, Ko, Vo, rnd=O.round_bf16, return_parts=True)
+    # the oracle's own cache: the synthetic one with K, V of ALL carried rows projected by the oracle (Eq. 5 writes
+    # them before the attention); float32 products of bf16 values in float64 accumulation are exact enough here
+    Ko, Vo = f64(K0), f64(V0)
+    Xall = f64(X)
+    a_all = O.round_bf16(O.rmsnorm(Xall, w.attn_norm, model.rms_eps))
+    _, k_all, v_all = O.project_qkv(a_all, w, model, rows, O.round_bf16)
+    Ko[rows] = k_all
+    Vo[rows] = v_all
+    Xo, parts = O.recompute_layer(Xall[sel], rows[sel], w, model, Ko, Vo, rnd=O.round_bf16, return_parts=True)
     check_kv(f64(Kc[pos[sel].long()]), parts["k_exact"], "K rows at full width")
     check_kv(f64(Vc[pos[sel].long()]), parts["v_exact"], "V rows at full width")
     check_kv(f64(Xg[sel]), parts["x_exact"], "hidden rows at full width", scale=2.0 * float(parts["x_exact"].std()))
     np.testing.assert_allclose(lse[sel].cpu().numpy(), parts["lse"], atol=5e-3)
+    # rows outside the carried ones are untouched
+    keep = torch.ones(r.n, dtype=torch.bool, device=DEV)
+    keep[pos.long()] = False
+    assert torch.equal(Kc[keep], K0[keep]) and torch.equal(Vc[keep], V0[keep])
 
 
 def test_llama8b_10x512_three_layers():
@@ -144,10 +171,10 @@ def test_llama8b_10x512_three_layers():
     K, V, out = c.fuse()
     rows, s, Kr, Vr = check_request_properties(c, K, V, out)
     assert out["p"] == 772
-    check_position_recovery_samples(c, Kr, Vr)
-    check_layer_samples(c, 2, rows, K[2], V[2])
+    check_position_recovery_samples(c)
+    check_layer_samples(c, 2, None)
     # the full block: all 5152 rows at positions 0..n-1 (launch shape of the leading block), sampled rows
-    check_layer_samples(c, 0, np.arange(c.r.n), Kr[0], Vr[0], n_samples=6, seed=1)
+    check_layer_samples(c, 0, np.arange(c.r.n), n_samples=6, seed=1)
     c.eng.close()
 
 
@@ -231,8 +258,8 @@ def test_llama8b_32k_planted_relevance():
     Re = rows[: out["p"]]
     share = np.mean([(r // 512) in planted for r in Re])
     assert share >= 3 * len(planted) / 64, share  # the selection concentrates on the planted chunks
-    check_position_recovery_samples(c, Kr, Vr, seed=2)
-    check_layer_samples(c, 2, rows, K[2], V[2], n_samples=6, seed=2)
+    check_position_recovery_samples(c, seed=2)
+    check_layer_samples(c, 2, None, n_samples=6, seed=2)
     c.eng.close()
 
 
@@ -248,8 +275,8 @@ def test_qwen7b_ragged_ratio_sweep():
             assert prev <= cur  # nested selections on the same request
         prev = cur
         if ratio == 0.15:
-            check_position_recovery_samples(c, Kr, Vr, seed=3)
-            check_layer_samples(c, 2, rows, K[2], V[2], n_samples=6, seed=3)  # G = 7 packing, q/k/v bias
+            check_position_recovery_samples(c, seed=3)
+            check_layer_samples(c, 2, None, n_samples=6, seed=3)  # G = 7 packing, q/k/v bias
     c.eng.close()
 
 
