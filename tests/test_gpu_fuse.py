@@ -4,7 +4,8 @@ The oracle mirrors the bf16 storage points (rnd=round_bf16).  Scores are gated a
 teacher-forced step test; here the query/key inputs of the score step have themselves gone through two
 different bf16 pipelines, so the end-to-end score gate is looser and the selection is checked (a) exactly
 against the GPU's own scores and (b) against the oracle's modulo scores near the threshold.  Later layers
-are compared with both sides forced onto the GPU's index set.
+are compared with the oracle's selection forced on the library (no output of the library is ever an input of the
+oracle).
 """
 import numpy as np
 import pytest
@@ -101,8 +102,10 @@ def test_fuse_request_matches_oracle(a3mod, config, n_system, dist):
     tau = np.sort(ref.scores[cand])[-p]
     for i in set(Re_gpu.tolist()) ^ set(ref.Re.tolist()):
         assert abs(ref.scores[i] - tau) <= 3e-2 * tau
-    # (c) both sides on the GPU's index set: fused cache and final rows, layer by layer
-    ref = s.run_oracle(r.ratio, forced=Re_gpu)
+    # (c) both sides on the ORACLE's index set (the oracle's selection is forced on the library, never the other way
+    # round): fused cache and final rows, layer by layer
+    K, V, out = s.run_gpu(r.ratio, forced=ref.Re)
+    assert out["rows"].cpu().numpy()[:p].tolist() == ref.Re.tolist()
     gK, gV, gX = f64(K), f64(V), f64(out["x"])
     for l in range(m.n_layers):
         # Layer 0 sees identical inputs on both sides, so the stated mean gate applies as it is.  Deeper layers are
@@ -260,7 +263,8 @@ def test_fuse_request_scores_from_cached_keys(a3mod, config, n_system, select_la
     tau = np.sort(ref.scores[cand])[-p]
     for i in set(Re_gpu.tolist()) ^ set(ref.Re.tolist()):
         assert abs(ref.scores[i] - tau) <= 3e-2 * tau
-    ref = s.run_oracle(r.ratio, select_layer=select_layer, forced=Re_gpu, cached_keys=True)
+    # both sides on the oracle's index set
+    K, V, out = s.run_gpu(r.ratio, select_layer=select_layer, forced=ref.Re, score_source=1)
     gK, gV, gX = f64(K), f64(V), f64(out["x"])
     for l in range(m.n_layers):
         gate = KV_MEAN if l == 0 else 2 * KV_MEAN
@@ -288,8 +292,8 @@ def test_fuse_request_scores_from_cached_keys(a3mod, config, n_system, select_la
 @pytest.mark.parametrize("config,n_system,score_source", [("tiny3", 0, 0), ("tiny_gqa", 100, 0), ("tiny_gqa", 100, 1)])
 def test_fuse_request_with_eviction(a3mod, config, n_system, score_source):
     """`ex` inside the request: every layer's compact cache is the gather of that layer's fused cache at the kept
-    slots (exact), S and Q are kept whole, and the kept documents agree with the oracle run on the same index set
-    except where the oracle's votes are within 3 % of its threshold (the end-to-end score gate)."""
+    slots (exact), S and Q are kept whole, and the kept documents agree with the oracle's on the oracle's index set
+    except for a few near its threshold."""
     s = Setup(a3mod, config, n_system=n_system, emb_std=0.02, w_std=0.02)
     m, r = s.m, s.r
     C, pool = n_system + r.n_question + 150, 5
@@ -306,9 +310,17 @@ def test_fuse_request_with_eviction(a3mod, config, n_system, score_source):
     # the fusion itself is unchanged by the extension
     K0, V0, out0 = s.run_gpu(r.ratio, score_source=score_source)
     assert torch.equal(K, K0) and torch.equal(V, V0) and torch.equal(out["x"], out0["x"])
-    Re_gpu = out["rows"].cpu().numpy()[:p]
+    # the oracle's own run; its selection is then forced on the library so that both evict the same fused cache
     ref = O.fuse_request(s.ck, s.cv, s.x0, r.n_question, s.weights, s.model, r.ratio, select_layer=r.select_layer, n_system=n_system,
-                         rnd=O.round_bf16, forced_Re=Re_gpu, scores_from_cached_keys=bool(score_source), evict_capacity=C, evict_pool=pool)
+                         rnd=O.round_bf16, scores_from_cached_keys=bool(score_source), evict_capacity=C, evict_pool=pool)
+    K, V = s.fused_buffers()
+    fr = torch.from_numpy(ref.Re.astype(np.int32)).to(s.dev)
+    req, out = s.eng.make_request(s.tab, len(s.dk), max(r.chunk_lens), r.n_ctx, r.n_question, s.dx0, K, V, ratio=r.ratio,
+                                  select_layer=r.select_layer, n_system=n_system, score_source=score_source, forced_re=fr,
+                                  evict_capacity=C, evict_pool=pool)
+    s.eng.fuse_request(req)
+    assert s.eng.device_status() == 0
+    kept = out["kept"].cpu().numpy()
     for l in range(m.n_layers):
         for g in range(m.n_kv_heads):
             kg = kept[l, g]
