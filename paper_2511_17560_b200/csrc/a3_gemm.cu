@@ -169,12 +169,22 @@ __device__ __forceinline__ void tc_prefetch_residual(const TcParams& p, int gr, 
   }
 }
 
+// QKV tiles made of whole heads of 128 columns (BN = 384: three heads), which may straddle the q/k/v matrices:
+// head g of the concatenated [q | k | v] output -> its matrix (segment) and its first row there.
+__device__ __forceinline__ void qkv_head_of(const TcParams& p, int g, int& seg, int& row0) {
+  seg = (g >= p.seg_heads_end[0]) + (g >= p.seg_heads_end[1]);
+  row0 = (g - (seg == 0 ? 0 : p.seg_heads_end[seg - 1])) * 128;
+}
+
 template <int EPI, int BN, int STAGES>
 __global__ void __launch_bounds__(TC_THREADS)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB0,
                const __grid_constant__ CUtensorMap tmB1, const __grid_constant__ CUtensorMap tmB2, const TcParams p) {
   using L = TcLayout<BN, STAGES>;
-  constexpr int TMEM_COLS = BN <= 128 ? 128 : 256;  // allocations are powers of two
+  constexpr int TMEM_COLS = BN <= 128 ? 128 : (BN <= 256 ? 256 : 512);  // allocations are powers of two
+  // head tiles: the tile is BN/128 whole heads, each loaded from its own matrix (QKV at head dimension 128 only)
+  constexpr bool HEAD_TILES = (EPI == EPI_QKV && BN > 256);
+  constexpr int HEADS = BN / 128;
   extern __shared__ unsigned char smem_raw[];
   const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   unsigned char* base_ptr = smem_raw + (base - smem_u32(smem_raw));
@@ -191,7 +201,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
   const int KT = p.K / TC_BK;
 
   int seg = 0, seg_tile0 = 0;
-  if (EPI == EPI_QKV) {
+  if (EPI == EPI_QKV && !HEAD_TILES) {
     while (seg < 2 && nt >= p.seg_tiles_end[seg]) {
       seg_tile0 = p.seg_tiles_end[seg];
       ++seg;
@@ -199,6 +209,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
   }
   // first B row of this tile within its matrix (for SwiGLU: within gate and within up)
   const int nb0 = (EPI == EPI_SWIGLU) ? nt * (BN / 2) : (nt - seg_tile0) * BN;
+  // head tiles: heads nt*HEADS .. of [q | k | v]; the last tile may hold fewer
+  const int heads_here = HEAD_TILES ? min(HEADS, p.seg_heads_end[2] - nt * HEADS) : 0;
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < STAGES; ++s) {
@@ -226,6 +238,20 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     // ---------------- TMA producer
     if (lane == 0) {
       const CUtensorMap* mapB = seg == 0 ? &tmB0 : (seg == 1 ? &tmB1 : &tmB2);
+      const CUtensorMap* head_map[HEADS];
+      int head_row0[HEADS];
+      if (HEAD_TILES) {
+#pragma unroll
+        for (int j = 0; j < HEADS; ++j) {
+          int sj = 0;
+          head_row0[j] = 0;
+          if (j < heads_here) qkv_head_of(p, nt * HEADS + j, sj, head_row0[j]);
+          head_map[j] = sj == 0 ? &tmB0 : (sj == 1 ? &tmB1 : &tmB2);
+        }
+        tmap_prefetch(&tmB0);
+        tmap_prefetch(&tmB1);
+        tmap_prefetch(&tmB2);
+      }
       tmap_prefetch(&tmA);
       tmap_prefetch(mapB);
       if (EPI == EPI_SWIGLU) tmap_prefetch(&tmB1);
@@ -235,9 +261,13 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         const uint32_t ph = (kb / STAGES) & 1;
         if (!mbar_wait(empty_bar(s), ph ^ 1, abort_flag, p.status)) break;
         const uint32_t sa = base + s * L::STAGE_BYTES, sb = sa + L::A_BYTES;
-        mbar_expect_tx(full_bar(s), L::STAGE_BYTES);
+        mbar_expect_tx(full_bar(s), HEAD_TILES ? L::A_BYTES + heads_here * (L::B_BYTES / HEADS) : L::STAGE_BYTES);
         tma_load_2d(sa, &tmA, kb * TC_BK, m0, full_bar(s));
-        if (EPI == EPI_SWIGLU) {
+        if (HEAD_TILES) {
+#pragma unroll
+          for (int j = 0; j < HEADS; ++j)
+            if (j < heads_here) tma_load_2d(sb + j * (L::B_BYTES / HEADS), head_map[j], kb * TC_BK, head_row0[j], full_bar(s));
+        } else if (EPI == EPI_SWIGLU) {
           tma_load_2d(sb, &tmB0, kb * TC_BK, nb0, full_bar(s));
           tma_load_2d(sb + L::B_BYTES / 2, &tmB1, kb * TC_BK, nb0, full_bar(s));
         } else {
@@ -254,7 +284,10 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
   } else if (warp == 1) {
     // ---------------- MMA issuer
     if (lane == 0) {
-      constexpr uint32_t idesc = idesc_bf16(BN);
+      constexpr uint32_t idesc = idesc_bf16(BN > 256 ? 256 : BN);
+      // head tiles: an instruction spans at most 256 columns, so heads 0-1 and head 2 are separate instructions
+      const uint32_t idesc_lo = heads_here >= 2 ? idesc_bf16(256) : idesc_bf16(128);
+      constexpr uint32_t idesc_hi = idesc_bf16(128);
       bool ok = true;
       for (int kb = 0; kb < KT && ok; ++kb) {
         const int s = kb % STAGES;
@@ -264,9 +297,18 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         tc_fence_after();
         const uint32_t sa = base + s * L::STAGE_BYTES, sb = sa + L::A_BYTES;
         const uint64_t da = smem_desc_sw128(sa), db = smem_desc_sw128(sb);
+        if (HEAD_TILES) {
+          const uint64_t db_hi = smem_desc_sw128(sb + 2 * (L::B_BYTES / HEADS));
 #pragma unroll
-        for (int k = 0; k < TC_BK / 16; ++k)  // +32 bytes per 16-element K step inside the 128-byte swizzle row
-          tc_mma_f16(tmem_base, da + (uint64_t)(2 * k), db + (uint64_t)(2 * k), idesc, (kb | k) != 0);
+          for (int k = 0; k < TC_BK / 16; ++k) {
+            tc_mma_f16(tmem_base, da + (uint64_t)(2 * k), db + (uint64_t)(2 * k), idesc_lo, (kb | k) != 0);
+            if (heads_here > 2) tc_mma_f16(tmem_base + 256, da + (uint64_t)(2 * k), db_hi + (uint64_t)(2 * k), idesc_hi, (kb | k) != 0);
+          }
+        } else {
+#pragma unroll
+          for (int k = 0; k < TC_BK / 16; ++k)  // +32 bytes per 16-element K step inside the 128-byte swizzle row
+            tc_mma_f16(tmem_base, da + (uint64_t)(2 * k), db + (uint64_t)(2 * k), idesc, (kb | k) != 0);
+        }
         tc_commit(empty_bar(s));  // arrives once the MMAs above have finished reading this stage
       }
       if (ok) tc_commit(tmem_full_bar);
@@ -281,10 +323,28 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     uint4 pre[EPI == EPI_RESIDUAL ? BN / 8 : (EPI == EPI_QKV ? 32 : 1)];
     int qkv_pos = -1;
     if (EPI == EPI_RESIDUAL) tc_prefetch_residual<BN>(p, gr, row_ok, nt, *reinterpret_cast<uint4(*)[BN / 8]>(pre));
-    if (EPI == EPI_QKV) qkv_pos = tc_prefetch_rope(p, gr, row_ok, seg, *reinterpret_cast<uint4(*)[32]>(pre));
+    if (EPI == EPI_QKV) {
+      int seg_first = seg;  // head tiles: q/k heads come first in a tile, so the first head tells whether RoPE is needed
+      if (HEAD_TILES) {
+        int r0;
+        qkv_head_of(p, nt * HEADS, seg_first, r0);
+      }
+      qkv_pos = tc_prefetch_rope(p, gr, row_ok, seg_first, *reinterpret_cast<uint4(*)[32]>(pre));
+    }
     const bool ready = mbar_wait(tmem_full_bar, 0, abort_flag, p.status);
     tc_fence_after();
-    if (ready) tc_epilogue_row<EPI, BN>(p, trow, gr, row_ok, nt, seg, nb0, pre, qkv_pos);
+    if (ready) {
+      if (HEAD_TILES) {
+#pragma unroll 1
+        for (int j = 0; j < heads_here; ++j) {
+          int sj, r0;
+          qkv_head_of(p, nt * HEADS + j, sj, r0);
+          tc_epilogue_qkv_row<128, 128>(p, trow + j * 128, gr, row_ok, sj, r0, pre, qkv_pos);
+        }
+      } else {
+        tc_epilogue_row<EPI, BN>(p, trow, gr, row_ok, nt, seg, nb0, pre, qkv_pos);
+      }
+    }
   }
   tc_fence_before();
   __syncthreads();
@@ -456,7 +516,8 @@ static int launch_tc(const a3_handle* h, const GemmArgs& a, const TcParams& p, i
     tB[2] = tB[0];
   } else {
     for (int s = 0; s < 3; ++s) {
-      if (s < a.nseg) A3_TRY(make_tmap(&tB[s], a.seg[s].B, a.seg[s].n, a.K, BN));
+      // head tiles (QKV, BN > 256) load one 128-row head per copy
+      if (s < a.nseg) A3_TRY(make_tmap(&tB[s], a.seg[s].B, a.seg[s].n, a.K, (EPI == EPI_QKV && BN > 256) ? 128 : BN));
       else tB[s] = tB[0];
     }
   }
@@ -511,6 +572,9 @@ template <int EPI>
 static int dispatch_tc(const a3_handle* h, const GemmArgs& a, const TcParams& p, int tiles, int bn, int stages, cudaStream_t st) {
   if (bn == 512 && stages == 3) return launch_pair<EPI, 3>(h, a, p, tiles, st);
   if (bn == 512) return launch_pair<EPI, 6>(h, a, p, tiles, st);
+  if constexpr (EPI == EPI_QKV) {
+    if (bn == 384) return launch_tc<EPI, 384, 3>(h, a, p, tiles, st);
+  }
   if (bn == 256 && stages == 4) return launch_tc<EPI, 256, 4>(h, a, p, tiles, st);
   if (bn == 256 && stages == 3) return launch_tc<EPI, 256, 3>(h, a, p, tiles, st);
   if (bn == 256 && stages == 2) return launch_tc<EPI, 256, 2>(h, a, p, tiles, st);
@@ -539,6 +603,21 @@ int gemm_bf16(const a3_handle* h, GemmEpilogue epi, const GemmArgs& a, cudaStrea
     } else {
       bn = 256;
       stages = 4;
+      // QKV at head dimension 128: tiles of two or three whole heads, whichever needs less tensor time per SM
+      // (rounds of the grid x heads per tile).  804 rows of Llama-8B: 7 x 24 two-head tiles are two rounds on 148
+      // SMs (4 head-times), 7 x 16 three-head tiles are one (3 head-times).
+      if (epi == EPI_QKV && h->m.head_dim == 128 && a.nseg == 3) {
+        bool whole = true;
+        int heads = 0;
+        for (int s = 0; s < 3; ++s) {
+          whole = whole && a.seg[s].n % 128 == 0;
+          heads += a.seg[s].n / 128;
+        }
+        if (whole && cdiv(m_tiles * cdiv(heads, 3), sms) * 3 < cdiv(m_tiles * cdiv(heads, 2), sms) * 2) {
+          bn = 384;
+          stages = 3;
+        }
+      }
     }
   }
   // output columns per tile; QKV tiles must hold whole heads and divide every segment
@@ -551,7 +630,12 @@ int gemm_bf16(const a3_handle* h, GemmEpilogue epi, const GemmArgs& a, cudaStrea
     if (!pair) stages = 4;
   }
   int out_cols = epi == EPI_SWIGLU ? bn / 2 : bn;
-  if (epi == EPI_QKV) {
+  const bool head_tiles = epi == EPI_QKV && bn == 384;
+  if (head_tiles) {
+    if (h->m.head_dim != 128 || a.nseg != 3) return A3_EUNSUPPORTED;
+    for (int s = 0; s < 3; ++s)
+      if (a.seg[s].n % 128) return A3_EUNSUPPORTED;
+  } else if (epi == EPI_QKV) {
     for (int s = 0; s < a.nseg; ++s)
       if (a.seg[s].n % out_cols) {
         bn = out_cols = 128;
@@ -561,10 +645,14 @@ int gemm_bf16(const a3_handle* h, GemmEpilogue epi, const GemmArgs& a, cudaStrea
   TcParams p{};
   p.M = a.M;
   p.K = a.K;
-  int tiles = 0;
+  int tiles = 0, heads = 0;
+  for (int s = 0; s < 3; ++s) {
+    if (s < a.nseg) heads += a.seg[s].n / 128;
+    p.seg_heads_end[s] = heads;
+  }
   for (int s = 0; s < 3; ++s) {
     if (s < a.nseg) {
-      if (epi != EPI_RESIDUAL && a.seg[s].n % out_cols) return A3_EUNSUPPORTED;
+      if (epi != EPI_RESIDUAL && !head_tiles && a.seg[s].n % out_cols) return A3_EUNSUPPORTED;
       if (a.seg[s].n % 32) return A3_EUNSUPPORTED;
       p.bias[s] = a.seg[s].bias;
       p.kind[s] = a.seg[s].kind;
@@ -572,6 +660,7 @@ int gemm_bf16(const a3_handle* h, GemmEpilogue epi, const GemmArgs& a, cudaStrea
     }
     p.seg_tiles_end[s] = tiles;
   }
+  if (head_tiles) tiles = cdiv(heads, 3);
   p.N = a.seg[0].n;
   p.C = a.C;
   p.ldc = a.ldc;

@@ -13,6 +13,7 @@ constexpr unsigned long long TC_WAIT_NS = 500000000ull;
 struct TcParams {
   int M, K, N;
   int seg_tiles_end[3];
+  int seg_heads_end[3];  // head tiles (QKV): cumulative 128-column heads of q, q+k, q+k+v
   int kind[3];
   const bf16* bias[3];
   bf16* C;

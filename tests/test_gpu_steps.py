@@ -590,3 +590,47 @@ def test_attention_two_row_tiles_per_cta(a3mod, shape, kv_len, M, grow):
     lse_tol = 2 * 2.0 ** -9 * float(np.abs(parts["q"]).max()) * float(np.abs(Kc).max()) / np.sqrt(m.head_dim)
     np.testing.assert_allclose(outs[0][1].cpu().numpy(), parts["lse"], atol=max(5e-3, lse_tol), rtol=1e-5)
     eng.close()
+
+
+@pytest.mark.parametrize("shape,kv_len,M", [(W.TINY_GQA, 900, 300), (W.TINY_G7, 700, 131)])
+def test_qkv_three_head_tiles(a3mod, shape, kv_len, M):
+    """The QKV projection with tiles of three whole heads (chosen by itself when that saves a round of the grid, as at
+    804 rows of the Llama-shaped model), forced on small models whose tiles mix q, k and v heads and whose last tile
+    holds fewer than three: K/V rows against the oracle, and everything bit for bit against the two-head tiling (the
+    sum over the model dimension runs in the same order in both)."""
+    import ctypes
+    m = shape
+    eng, layers, dev = make_engine(a3mod, m, seed=33, w_std=0.05)
+    lib = a3mod._load()
+    lib.a3_internal_set_gemm_cfg.argtypes = [ctypes.c_int, ctypes.c_int, ctypes.c_int]
+    model, weights = oracle_model(m), oracle_weights(layers)
+    rng = np.random.default_rng(91)
+    pos = np.sort(rng.choice(kv_len, size=M, replace=False))
+    pos[-1] = kv_len - 1
+    X = W.bf16_round(rng.standard_normal((M, m.d_model), dtype=np.float32))
+    Kc, Vc = W.make_cache_like(m, kv_len, 33, 9, std=1.0)
+    layer = m.n_layers - 1
+    dpos = torch.from_numpy(pos.astype(np.int32)).to(dev)
+    outs = {}
+    try:
+        for bn, stages in ((384, 3), (0, 0)):
+            lib.a3_internal_set_gemm_cfg(2, bn, stages)
+            dX, dK, dV = to_dev(X, dev), to_dev(Kc[layer], dev), to_dev(Vc[layer], dev)
+            eng.recompute_layer(layer, dX, dpos, dK, dV)
+            assert eng.device_status() == 0
+            outs[bn] = (dX, dK, dV)
+    finally:
+        lib.a3_internal_set_gemm_cfg(2, 0, 0)
+    for a, b in zip(outs[384], outs[0]):
+        assert torch.equal(a, b)
+    Ko, Vo = Kc[layer].astype(np.float64), Vc[layer].astype(np.float64)
+    Xo, parts = O.recompute_layer(X.astype(np.float64), pos, weights[layer], model, Ko, Vo, rnd=O.round_bf16, return_parts=True)
+    gK, gV = f64(outs[384][1]), f64(outs[384][2])
+    check_kv(gK[pos], parts["k_exact"], "recomputed K rows")
+    check_kv(gV[pos], parts["v_exact"], "recomputed V rows")
+    mask = np.ones(kv_len, bool)
+    mask[pos] = False
+    np.testing.assert_array_equal(gK[mask], Kc[layer][mask])
+    np.testing.assert_array_equal(gV[mask], Vc[layer][mask])
+    check_kv(f64(outs[384][0]), parts["x_exact"], "hidden rows", scale=2.0 * float(parts["x_exact"].std()))
+    eng.close()
