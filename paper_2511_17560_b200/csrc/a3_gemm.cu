@@ -97,7 +97,7 @@ __device__ __forceinline__ void tc_epilogue_qkv_row(const TcParams& p, uint32_t 
 // of registers.  For EPI_RESIDUAL the row's old values arrive in `pre` (see tc_prefetch_residual).
 template <int EPI, int BN>
 __device__ __forceinline__ void tc_epilogue_row(const TcParams& p, uint32_t trow, int gr, bool row_ok, int nt, int seg, int nb0,
-                                                const uint4* pre, int qkv_pos) {
+                                                const uint4* pre, int qkv_pos, int g_cols = BN / 2) {
     if (EPI == EPI_RESIDUAL) {
       // the old values of C were fetched while the main loop ran (`pre`): only tensor memory is waited for here
       const int n0 = nt * BN;
@@ -116,18 +116,38 @@ __device__ __forceinline__ void tc_epilogue_row(const TcParams& p, uint32_t trow
         }
       }
     } else if (EPI == EPI_SWIGLU) {
-      const int n0 = nt * (BN / 2);
+      // gate columns 0..g_cols-1, up columns g_cols..2 g_cols-1 of the accumulator; the tile's first feature is nb0
+      const int n0 = nb0;
+      // 32 columns at a time; a narrow tile's remainder, and a last tile that reaches the end of the matrix (its
+      // loads beyond it were zero-filled), 8 at a time.  The branch depends on the tile only: uniform for the warp.
+      const int n8 = g_cols / 8;
+      int c8 = 0;
 #pragma unroll 1
-      for (int c = 0; c < BN / 64; ++c) {
+      while (c8 < n8) {
         __syncwarp();
-        float g[32], u[32];
-        tc_ld32(trow + c * 32, g);
-        tc_ld32(trow + BN / 2 + c * 32, u);
-        tc_wait_ld();
-        if (row_ok) {
+        const int col = n0 + c8 * 8;
+        if (c8 + 4 <= n8 && col + 32 <= p.N) {
+          float g[32], u[32];
+          tc_ld32(trow + c8 * 8, g);
+          tc_ld32(trow + g_cols + c8 * 8, u);
+          tc_wait_ld();
+          if (row_ok) {
 #pragma unroll
-          for (int e = 0; e < 32; ++e) g[e] = g[e] / (1.f + __expf(-g[e])) * u[e];
-          store32_bf16(p.C + (size_t)gr * p.ldc + n0 + c * 32, g);
+            for (int e = 0; e < 32; ++e) g[e] = g[e] / (1.f + __expf(-g[e])) * u[e];
+            store32_bf16(p.C + (size_t)gr * p.ldc + col, g);
+          }
+          c8 += 4;
+        } else {
+          float g[8], u[8];
+          tc_ld8(trow + c8 * 8, g);
+          tc_ld8(trow + g_cols + c8 * 8, u);
+          tc_wait_ld();
+          if (row_ok && col + 8 <= p.N) {
+#pragma unroll
+            for (int e = 0; e < 8; ++e) g[e] = g[e] / (1.f + __expf(-g[e])) * u[e];
+            *reinterpret_cast<uint4*>(p.C + (size_t)gr * p.ldc + col) = pack8(g);
+          }
+          c8 += 1;
         }
       }
     } else {
@@ -179,7 +199,8 @@ __device__ __forceinline__ void qkv_head_of(const TcParams& p, int g, int& seg, 
 template <int EPI, int BN, int STAGES>
 __global__ void __launch_bounds__(TC_THREADS)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB0,
-               const __grid_constant__ CUtensorMap tmB1, const __grid_constant__ CUtensorMap tmB2, const TcParams p) {
+               const __grid_constant__ CUtensorMap tmB1, const __grid_constant__ CUtensorMap tmB2,
+               const __grid_constant__ CUtensorMap tmN0, const __grid_constant__ CUtensorMap tmN1, const TcParams p) {
   using L = TcLayout<BN, STAGES>;
   constexpr int TMEM_COLS = BN <= 128 ? 128 : (BN <= 256 ? 256 : 512);  // allocations are powers of two
   // head tiles: the tile is BN/128 whole heads, each loaded from its own matrix (QKV at head dimension 128 only)
@@ -208,7 +229,14 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     }
   }
   // first B row of this tile within its matrix (for SwiGLU: within gate and within up)
-  const int nb0 = (EPI == EPI_SWIGLU) ? nt * (BN / 2) : (nt - seg_tile0) * BN;
+  int nb0 = (EPI == EPI_SWIGLU) ? nt * (BN / 2) : (nt - seg_tile0) * BN;
+  // SwiGLU: features per tile; the column tiles from y_wide on are narrower (maps tmN0/tmN1, box g_narrow rows)
+  int g_cols = BN / 2;
+  const bool narrow = EPI == EPI_SWIGLU && p.g_narrow > 0 && nt >= p.y_wide;
+  if (narrow) {
+    g_cols = p.g_narrow;
+    nb0 = p.y_wide * (BN / 2) + (nt - p.y_wide) * g_cols;
+  }
   // head tiles: heads nt*HEADS .. of [q | k | v]; the last tile may hold fewer
   const int heads_here = HEAD_TILES ? min(HEADS, p.seg_heads_end[2] - nt * HEADS) : 0;
 
@@ -255,21 +283,27 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
       tmap_prefetch(&tmA);
       tmap_prefetch(mapB);
       if (EPI == EPI_SWIGLU) tmap_prefetch(&tmB1);
+      if (narrow) {
+        tmap_prefetch(&tmN0);
+        tmap_prefetch(&tmN1);
+      }
       int issued = 0;
       for (int kb = 0; kb < KT; ++kb) {
         const int s = kb % STAGES;
         const uint32_t ph = (kb / STAGES) & 1;
         if (!mbar_wait(empty_bar(s), ph ^ 1, abort_flag, p.status)) break;
         const uint32_t sa = base + s * L::STAGE_BYTES, sb = sa + L::A_BYTES;
-        mbar_expect_tx(full_bar(s), HEAD_TILES ? L::A_BYTES + heads_here * (L::B_BYTES / HEADS) : L::STAGE_BYTES);
+        mbar_expect_tx(full_bar(s), HEAD_TILES ? L::A_BYTES + heads_here * (L::B_BYTES / HEADS)
+                                    : (EPI == EPI_SWIGLU ? L::A_BYTES + 2 * g_cols * TC_BK * 2 : L::STAGE_BYTES));
         tma_load_2d(sa, &tmA, kb * TC_BK, m0, full_bar(s));
         if (HEAD_TILES) {
 #pragma unroll
           for (int j = 0; j < HEADS; ++j)
             if (j < heads_here) tma_load_2d(sb + j * (L::B_BYTES / HEADS), head_map[j], kb * TC_BK, head_row0[j], full_bar(s));
         } else if (EPI == EPI_SWIGLU) {
-          tma_load_2d(sb, &tmB0, kb * TC_BK, nb0, full_bar(s));
-          tma_load_2d(sb + L::B_BYTES / 2, &tmB1, kb * TC_BK, nb0, full_bar(s));
+          // gate rows, then up rows (g_cols is a multiple of 8, so the up block starts on a 1024-byte boundary)
+          tma_load_2d(sb, narrow ? &tmN0 : &tmB0, kb * TC_BK, nb0, full_bar(s));
+          tma_load_2d(sb + g_cols * TC_BK * 2, narrow ? &tmN1 : &tmB1, kb * TC_BK, nb0, full_bar(s));
         } else {
           tma_load_2d(sb, mapB, kb * TC_BK, nb0, full_bar(s));
         }
@@ -284,7 +318,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
   } else if (warp == 1) {
     // ---------------- MMA issuer
     if (lane == 0) {
-      constexpr uint32_t idesc = idesc_bf16(BN > 256 ? 256 : BN);
+      const uint32_t idesc = EPI == EPI_SWIGLU ? idesc_bf16(2 * g_cols) : idesc_bf16(BN > 256 ? 256 : BN);
       // head tiles: an instruction spans at most 256 columns, so heads 0-1 and head 2 are separate instructions
       const uint32_t idesc_lo = heads_here >= 2 ? idesc_bf16(256) : idesc_bf16(128);
       constexpr uint32_t idesc_hi = idesc_bf16(128);
@@ -342,7 +376,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
           tc_epilogue_qkv_row<128, 128>(p, trow + j * 128, gr, row_ok, sj, r0, pre, qkv_pos);
         }
       } else {
-        tc_epilogue_row<EPI, BN>(p, trow, gr, row_ok, nt, seg, nb0, pre, qkv_pos);
+        tc_epilogue_row<EPI, BN>(p, trow, gr, row_ok, nt, seg, nb0, pre, qkv_pos, g_cols);
       }
     }
   }
@@ -508,12 +542,16 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
 template <int EPI, int BN, int STAGES>
 static int launch_tc(const a3_handle* h, const GemmArgs& a, const TcParams& p, int tiles, cudaStream_t st) {
   using L = TcLayout<BN, STAGES>;
-  CUtensorMap tA, tB[3];
+  CUtensorMap tA, tB[3], tN[2];
   A3_TRY(make_tmap(&tA, a.A, a.M, a.K, TC_BM));
   if (EPI == EPI_SWIGLU) {
     A3_TRY(make_tmap(&tB[0], a.seg[0].B, a.seg[0].n, a.K, BN / 2));
     A3_TRY(make_tmap(&tB[1], a.B2, a.seg[0].n, a.K, BN / 2));
     tB[2] = tB[0];
+    if (p.g_narrow > 0) {
+      A3_TRY(make_tmap(&tN[0], a.seg[0].B, a.seg[0].n, a.K, p.g_narrow));
+      A3_TRY(make_tmap(&tN[1], a.B2, a.seg[0].n, a.K, p.g_narrow));
+    }
   } else {
     for (int s = 0; s < 3; ++s) {
       // head tiles (QKV, BN > 256) load one 128-row head per copy
@@ -528,7 +566,8 @@ static int launch_tc(const a3_handle* h, const GemmArgs& a, const TcParams& p, i
   }
   dim3 grid(cdiv(a.M, TC_BM), tiles);
   ProfScope prof(h, EPI == EPI_RESIDUAL ? A3_K_GEMM_RESIDUAL : EPI == EPI_SWIGLU ? A3_K_GEMM_SWIGLU : A3_K_GEMM_QKV, st);
-  A3_CUDA(launch_pdl(gemm_tc_kernel<EPI, BN, STAGES>, grid, dim3(TC_THREADS), (size_t)L::SMEM_BYTES, st, tA, tB[0], tB[1], tB[2], p));
+  if (!(EPI == EPI_SWIGLU && p.g_narrow > 0)) tN[0] = tN[1] = tB[0];
+  A3_CUDA(launch_pdl(gemm_tc_kernel<EPI, BN, STAGES>, grid, dim3(TC_THREADS), (size_t)L::SMEM_BYTES, st, tA, tB[0], tB[1], tB[2], tN[0], tN[1], p));
   A3_LAUNCHED();
   return A3_OK;
 }
@@ -566,6 +605,7 @@ static int launch_pair(const a3_handle* h, const GemmArgs& a, const TcParams& p,
 // the grid has several waves.  The CTA-pair kernel wins for the residual GEMMs (N = d_model: few tiles, one CTA per
 // SM); for SwiGLU and QKV its extra all-padding row tile at 804 rows (7 -> 8) costs more than the halved B traffic
 // saves: under the power cap the tensor work, not the L2 port, sets the pace.
+int g_tc_narrow = 1;  // 0: no narrower last wave in the SwiGLU grid; 1: choose; 16..120: that width on half the tiles (tests)
 int g_tc_cfg[3][2] = {{0, 0}, {256, 2}, {0, 0}};
 
 template <int EPI>
@@ -661,6 +701,30 @@ int gemm_bf16(const a3_handle* h, GemmEpilogue epi, const GemmArgs& a, cudaStrea
     p.seg_tiles_end[s] = tiles;
   }
   if (head_tiles) tiles = cdiv(heads, 3);
+  // SwiGLU with two CTAs per SM: the grid runs in waves of 2 x SMs tiles and a partly filled last wave costs a whole
+  // one (measured: 58 us per wave at Llama-8B width whatever its fill).  The column tiles of the last wave are
+  // therefore made narrower, so that they all fit into it: a wave's time follows the bytes its tiles pull through
+  // the SM's L2 port (A: 128 rows, B: 2 g rows per k-block), i.e. (128 + 2 g) / 384 of a full one.
+  if (epi == EPI_SWIGLU && bn == 256 && stages == 2 && g_tc_narrow && a.seg[0].n % 128 == 0) {
+    const int m_tiles = cdiv(a.M, TC_BM), slots = 2 * (h->sm_count > 0 ? h->sm_count : 148), ct = a.seg[0].n / 128;
+    const int total = m_tiles * ct, waves_full = total / slots;
+    if (g_tc_narrow >= 16 && g_tc_narrow < 128 && g_tc_narrow % 8 == 0 && ct >= 2) {  // forced (tests): half the tiles narrow
+      p.y_wide = ct / 2;
+      p.g_narrow = g_tc_narrow;
+      tiles = p.y_wide + cdiv(a.seg[0].n - p.y_wide * 128, p.g_narrow);
+    } else if (waves_full >= 1 && total % slots) {
+      const int y_wide = waves_full * slots / m_tiles;
+      const int rest = a.seg[0].n - y_wide * 128;
+      const int per_row = (slots + waves_full * slots - y_wide * m_tiles) / m_tiles;
+      const int rnd = 16;  // measured at 804..2 000 rows: widths that are multiples of 16 features never lose
+      const int g = per_row > 0 ? cdiv(cdiv(rest, per_row), rnd) * rnd : 128;
+      if (g >= 16 && g < 128) {
+        p.y_wide = y_wide;
+        p.g_narrow = g;
+        tiles = y_wide + cdiv(rest, g);
+      }
+    }
+  }
   p.N = a.seg[0].n;
   p.C = a.C;
   p.ldc = a.ldc;
@@ -684,6 +748,7 @@ int gemm_bf16(const a3_handle* h, GemmEpilogue epi, const GemmArgs& a, cudaStrea
 
 }  // namespace a3
 
+extern "C" void a3_internal_set_gemm_narrow(int on) { a3::g_tc_narrow = on; }
 extern "C" void a3_internal_set_gemm_cfg(int epi, int bn, int stages) {
   if (epi >= 0 && epi < 3) {
     a3::g_tc_cfg[epi][0] = bn;

@@ -26,6 +26,8 @@ struct TcParams {
   int Hq, Hkv, D, layout, max_pos;
   const float2* tab;
   uint32_t* status;
+  // SwiGLU with a narrower last wave: column tiles 0..y_wide-1 hold BN/2 features, the rest g_narrow (0: all wide)
+  int y_wide, g_narrow;
 };
 
 // ---------------------------------------------------------------- PTX wrappers
@@ -101,6 +103,14 @@ __device__ __forceinline__ void tc_ld32(uint32_t taddr, float* v) {
         "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
       : "r"(taddr)
       : "memory");
+}
+// 32 lanes x 8 consecutive fp32 columns
+__device__ __forceinline__ void tc_ld8(uint32_t taddr, float* v) {
+  uint32_t* r = reinterpret_cast<uint32_t*>(v);
+  asm volatile("tcgen05.ld.sync.aligned.32x32b.x8.b32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];"
+               : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7])
+               : "r"(taddr)
+               : "memory");
 }
 __device__ __forceinline__ void tc_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 

@@ -634,3 +634,39 @@ def test_qkv_three_head_tiles(a3mod, shape, kv_len, M):
     np.testing.assert_array_equal(gV[mask], Vc[layer][mask])
     check_kv(f64(outs[384][0]), parts["x_exact"], "hidden rows", scale=2.0 * float(parts["x_exact"].std()))
     eng.close()
+
+
+@pytest.mark.parametrize("shape,M,g", [(W.TINY_GQA, 300, 88), (W.TINY_G7, 131, 40), (W.TINY, 95, 104)])
+def test_swiglu_narrow_column_tiles(a3mod, shape, M, g):
+    """The SwiGLU GEMM gives the column tiles of a partly filled last wave fewer features each (by itself only for
+    grids of several waves); forced here on half the column tiles, with widths that leave a remainder of 8-column
+    pieces and a last tile reaching past the matrix: bit for bit against the uniform tiling, and against the oracle."""
+    import ctypes
+    m = shape
+    eng, layers, dev = make_engine(a3mod, m, seed=41, w_std=0.05)
+    lib = a3mod._load()
+    lib.a3_internal_set_gemm_narrow.argtypes = [ctypes.c_int]
+    model, weights = oracle_model(m), oracle_weights(layers)
+    rng = np.random.default_rng(17)
+    kv_len = 3 * M
+    pos = np.sort(rng.choice(kv_len, size=M, replace=False))
+    pos[-1] = kv_len - 1
+    X = W.bf16_round(rng.standard_normal((M, m.d_model), dtype=np.float32))
+    Kc, Vc = W.make_cache_like(m, kv_len, 41, 9, std=1.0)
+    layer = m.n_layers - 1
+    dpos = torch.from_numpy(pos.astype(np.int32)).to(dev)
+    outs = {}
+    try:
+        for mode in (g, 0):
+            lib.a3_internal_set_gemm_narrow(mode)
+            dX, dK, dV = to_dev(X, dev), to_dev(Kc[layer], dev), to_dev(Vc[layer], dev)
+            eng.recompute_layer(layer, dX, dpos, dK, dV)
+            assert eng.device_status() == 0
+            outs[mode] = dX
+    finally:
+        lib.a3_internal_set_gemm_narrow(1)
+    assert torch.equal(outs[g], outs[0])
+    Ko, Vo = Kc[layer].astype(np.float64), Vc[layer].astype(np.float64)
+    Xo, parts = O.recompute_layer(X.astype(np.float64), pos, weights[layer], model, Ko, Vo, rnd=O.round_bf16, return_parts=True)
+    check_kv(f64(outs[g]), parts["x_exact"], "hidden rows", scale=2.0 * float(parts["x_exact"].std()))
+    eng.close()
