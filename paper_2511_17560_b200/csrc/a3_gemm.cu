@@ -133,7 +133,7 @@ __device__ __forceinline__ void tc_epilogue_row(const TcParams& p, uint32_t trow
           tc_wait_ld();
           if (row_ok) {
 #pragma unroll
-            for (int e = 0; e < 32; ++e) g[e] = g[e] / (1.f + __expf(-g[e])) * u[e];
+            for (int e = 0; e < 32; ++e) g[e] = __fdividef(g[e], 1.f + __expf(-g[e])) * u[e];
             store32_bf16(p.C + (size_t)gr * p.ldc + col, g);
           }
           c8 += 4;
@@ -144,7 +144,7 @@ __device__ __forceinline__ void tc_epilogue_row(const TcParams& p, uint32_t trow
           tc_wait_ld();
           if (row_ok && col + 8 <= p.N) {
 #pragma unroll
-            for (int e = 0; e < 8; ++e) g[e] = g[e] / (1.f + __expf(-g[e])) * u[e];
+            for (int e = 0; e < 8; ++e) g[e] = __fdividef(g[e], 1.f + __expf(-g[e])) * u[e];
             *reinterpret_cast<uint4*>(p.C + (size_t)gr * p.ldc + col) = pack8(g);
           }
           c8 += 1;
@@ -628,6 +628,7 @@ static int dispatch_tc(const a3_handle* h, const GemmArgs& a, const TcParams& p,
 int gemm_bf16(const a3_handle* h, GemmEpilogue epi, const GemmArgs& a, cudaStream_t st) {
   if (a.M <= 0) return A3_OK;
   if (a.K % TC_BK) return A3_EUNSUPPORTED;
+  if (epi == EPI_SWIGLU && swiglu_pair_usable(h, a)) return gemm_swiglu_pair(h, a, st);
   int bn = g_tc_cfg[epi][0];
   int stages = g_tc_cfg[epi][1];
 

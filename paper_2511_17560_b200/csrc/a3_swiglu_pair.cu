@@ -1,0 +1,367 @@
+// SwiGLU GEMM of the recompute path (the feed-forward part of H(.) in Eq. 5) with the operand roles swapped and a
+// persistent schedule:   out[t][f] = silu(x[t] . Wg[f]) * (x[t] . Wu[f]).
+//
+// Why another kernel.  With one CTA per 128-token x 256-column tile, an SM pulls 48 KiB per k-block through its L2
+// port and that port, not the tensor pipe, sets the pace (measured: a wave's time follows the bytes, 107 GB/s per
+// SM); at 804 tokens the 128-row tiles also pad the rows to 896 and the grid to three waves.  Here
+//   * the WEIGHTS are the M-side operand of tcgen05.mma.cta_group::2 (M = 256 over a CTA pair): each CTA holds 64
+//     gate rows and 64 up rows of the same 64 features (its 128 accumulator lanes), so gate and up of a feature
+//     meet inside one CTA;
+//   * the TOKENS are the N-side operand, in tiles of N <= 256 tokens chosen to divide the row count evenly
+//     (804 rows -> 4 x 208: 3 % padding instead of 11 %); each CTA loads half of the token tile, the instruction
+//     reads both halves.  Per k-block an SM pulls 16 KiB of weights + N/2 token rows (13 KiB at N = 208) for
+//     64 x N outputs: 0.6 of the bytes per output of the one-CTA kernel;
+//   * the kernel is persistent: CTA pair p walks units p, p + pairs, ... (unit = 128 features x one token tile),
+//     accumulators are double-buffered in tensor memory (2 x N <= 512 columns), so the epilogue of a unit runs under
+//     the main loop of the next one.
+// Epilogue: the warps that own the "up" lanes park their values in shared memory, the warps that own the "gate"
+// lanes combine and store out[t][f] (a warp writes 32 consecutive features of one token: 64 bytes).
+// No load uses cluster multicast.  Every wait is bounded (see a3_tc.cuh): a waiter that gives up raises the CTA's
+// abort flag and the device status bit, all roles leave their loops, tensor memory is released and the CTA returns.
+#include <cuda.h>
+
+#include "a3_internal.cuh"
+#include "a3_tc.cuh"
+
+namespace a3 {
+
+constexpr int SP_THREADS = 320;  // warp 0: TMA, warp 1: MMA (leader CTA), warps 2..9: epilogue (two sets of four)
+constexpr int SP_MAX_STAGES = 8;
+constexpr int SP_SUB = 2;  // k-blocks of 64 per ring stage: one barrier hand-shake and one commit per 8 MMAs
+constexpr int SP_FEAT = 64;                              // features per CTA (64 gate lanes + 64 up lanes)
+constexpr int SP_A_BYTES = 2 * SP_FEAT * TC_BK * 2;      // 16 KiB: gate rows, then up rows
+constexpr int SP_XCH_BYTES = 2 * 2 * 32 * SP_FEAT * 4;   // per warp set: two buffers of float [32 tokens][64 features]
+constexpr int SP_SMEM_LIMIT = 227 * 1024;
+
+struct SpParams {
+  int M, K, F;
+  int tok_tiles, tok_n;  // token tiles and tokens per tile (multiple of 16, at most 256)
+  int n_units, n_pairs;
+  int stages, stage_bytes, sub_bytes;  // ring depth; bytes per stage = SP_SUB x sub_bytes (A + this CTA's half of the token tile for one k-block, 1024-byte multiple)
+  bf16* C;
+  int ldc;
+  uint32_t* status;
+};
+
+__device__ __forceinline__ void named_bar_sync(int id, int threads) {
+  asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(threads) : "memory");
+}
+__device__ __forceinline__ void named_bar_arrive(int id, int threads) {
+  asm volatile("bar.arrive %0, %1;" ::"r"(id), "r"(threads) : "memory");
+}
+// arrives on the barrier at the same shared-memory offset in CTA `cta` of the cluster
+__device__ __forceinline__ void mbar_arrive_in_cta(uint32_t bar, uint32_t cta) {
+  uint32_t remote;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(remote) : "r"(bar), "r"(cta));
+  asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(remote) : "memory");
+}
+// w (8, 16, 24 or 32; uniform for the warp) consecutive accumulator columns of this thread's lane
+__device__ __forceinline__ void sp_ld_chunk(uint32_t taddr, int w, float* v) {
+  if (w == 32) {
+    tc_ld32(taddr, v);
+  } else {  // static register indices: the array must not go to local memory
+    if (w >= 8) tc_ld8(taddr, v);
+    if (w >= 16) tc_ld8(taddr + 8, v + 8);
+    if (w >= 24) tc_ld8(taddr + 16, v + 16);
+  }
+  tc_wait_ld();
+}
+
+// D += A B over the CTA pair (accumulating form: no predicate to set up)
+__device__ __forceinline__ void tc_mma_pair_acc(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.eq.u32 p, 0, 0;\n\t"
+      "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+      ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc)
+      : "memory");
+}
+
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(SP_THREADS, 1)
+swiglu_pair_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUtensorMap tmG,
+                   const __grid_constant__ CUtensorMap tmU, const SpParams p) {
+  extern __shared__ unsigned char smem_raw[];
+  const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;  // same offset in both CTAs of the pair
+  unsigned char* base_ptr = smem_raw + (base - smem_u32(smem_raw));
+  const int S = p.stages;
+  const int xch_off = S * p.stage_bytes, bar_off = xch_off + SP_XCH_BYTES;
+  // barriers (8 bytes each): full[8] (used in the leader), empty[8], tmem_full[2], tmem_empty[2] (used in the leader)
+  const uint32_t bars = base + bar_off;
+  auto full_bar = [&](int s) { return bars + 8u * s; };
+  auto empty_bar = [&](int s) { return bars + 8u * (SP_MAX_STAGES + s); };
+  auto tmem_full = [&](int b) { return bars + 8u * (2 * SP_MAX_STAGES + b); };
+  auto tmem_empty = [&](int b) { return bars + 8u * (2 * SP_MAX_STAGES + 2 + b); };
+  volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(base_ptr + bar_off + 8 * (2 * SP_MAX_STAGES + 4));
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(base_ptr + bar_off + 8 * (2 * SP_MAX_STAGES + 4) + 8);
+  volatile int* ep_ok = abort_flag + 2;  // the epilogue's one waiter tells the other 127 threads how its wait ended
+  float* xch = reinterpret_cast<float*>(base_ptr + xch_off);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const uint32_t rank = cluster_ctarank();
+  const bool leader = rank == 0;
+  const int pair = blockIdx.x >> 1;
+  const int KT = p.K / TC_BK;  // a multiple of SP_SUB (checked by the launcher)
+  const int half_n = p.tok_n >> 1;  // token rows this CTA loads per k-block (multiple of 8)
+  const uint32_t b_bytes = (uint32_t)half_n * TC_BK * 2;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < S; ++s) {
+      mbar_init(full_bar(s), 1);
+      mbar_init(empty_bar(s), 1);
+    }
+    for (int b = 0; b < 2; ++b) {
+      mbar_init(tmem_full(b), 1);
+      mbar_init(tmem_empty(b), 8);  // the gate warps and the up warps of both warp sets of each CTA of the pair
+    }
+    abort_flag[0] = 0;
+    abort_flag[1] = 0;
+    ep_ok[0] = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+  }
+  if (warp == 1) {  // the same warp of both CTAs
+    asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32((const void*)tmem_slot)), "r"(512) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
+  cluster_sync_all();  // the peer's barriers exist before anything is signalled on them
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+  pdl_wait();
+  pdl_launch_dependents();
+
+  if (warp == 0) {
+    // ---------------- TMA producer (both CTAs): own gate/up rows, own half of the token tile
+    if (lane == 0) {
+      tmap_prefetch(&tmX);
+      tmap_prefetch(&tmG);
+      tmap_prefetch(&tmU);
+      int kbg = 0, issued = 0;
+      int s = 0;        // ring position and phase, kept by counting: S is a run-time value and a division per
+      uint32_t ph = 0;  // k-block is a long dependent chain in a one-thread role
+      bool ok = true;
+      for (int u = pair; u < p.n_units && ok; u += p.n_pairs) {
+        const int f0 = (u / p.tok_tiles) * (2 * SP_FEAT) + (int)rank * SP_FEAT;
+        const int t0 = (u % p.tok_tiles) * p.tok_n + (int)rank * half_n;
+        for (int kb = 0; kb < KT; kb += SP_SUB, ++kbg) {
+          if (!mbar_wait(empty_bar(s), ph ^ 1, abort_flag, p.status)) {
+            ok = false;
+            break;
+          }
+          const uint32_t full_leader = full_bar(s) & PAIR_LEADER_MASK;
+          // the leader announces the bytes of both CTAs; a copy of the peer that completes earlier cannot end the
+          // phase, because the leader's own arrival is still pending until its expect_tx
+          if (leader) mbar_expect_tx(full_bar(s), 2 * SP_SUB * (SP_A_BYTES + b_bytes));
+#pragma unroll
+          for (int j = 0; j < SP_SUB; ++j) {
+            const uint32_t sa = base + s * p.stage_bytes + j * p.sub_bytes, sb = sa + SP_A_BYTES;
+            tma_load_2d_pair(sa, &tmG, (kb + j) * TC_BK, f0, full_leader);
+            tma_load_2d_pair(sa + SP_A_BYTES / 2, &tmU, (kb + j) * TC_BK, f0, full_leader);
+            tma_load_2d_pair(sb, &tmX, (kb + j) * TC_BK, t0, full_leader);
+          }
+          issued = kbg + 1;
+          if (++s == S) {
+            s = 0;
+            ph ^= 1;
+          }
+        }
+      }
+      if (*abort_flag) {
+        // let the copies already issued land before the CTA can exit (bounded)
+        if (leader) {
+          for (int k = max(0, issued - S); k < issued; ++k)
+            mbar_wait(full_bar(k % S), (k / S) & 1, abort_flag + 1, p.status, 2000000ull);
+        } else {
+          const unsigned long long t0 = global_ns();
+          while (global_ns() - t0 < 200000ull) {
+          }
+        }
+      }
+    }
+  } else if (warp == 1) {
+    // ---------------- MMA issuer: the leader alone, for both CTAs
+    if (lane == 0 && leader) {
+      const uint32_t idesc = idesc_bf16_pair(p.tok_n);
+      int kbg = 0, it = 0;
+      int s = 0;
+      uint32_t ph = 0;
+      bool ok = true;
+      const uint64_t da0 = smem_desc_sw128(base), db0 = smem_desc_sw128(base + SP_A_BYTES);
+      const uint32_t stage16 = (uint32_t)p.stage_bytes >> 4, sub16 = (uint32_t)p.sub_bytes >> 4;
+      uint32_t stage_off = 0;
+      for (int u = pair; u < p.n_units && ok; u += p.n_pairs, ++it) {
+        const int b = it & 1;
+        // the epilogues of both CTAs have drained this accumulator (first use: passes at once)
+        ok = mbar_wait(tmem_empty(b), ((it >> 1) & 1) ^ 1, abort_flag, p.status);
+        if (!ok) break;
+        tc_fence_after();
+        const uint32_t d = tmem_base + (uint32_t)b * 256u;
+        for (int kb = 0; kb < KT; kb += SP_SUB, ++kbg) {
+          ok = mbar_wait(full_bar(s), ph, abort_flag, p.status);
+          if (!ok) break;
+          tc_fence_after();
+          // descriptors of this stage: the address field counts 16-byte units, so stage and k-step offsets are added
+          // to the descriptors of the ring's first stage (all of shared memory fits the field)
+          const uint64_t da_s = da0 + stage_off, db_s = db0 + stage_off;
+#pragma unroll
+          for (int j = 0; j < SP_SUB; ++j) {
+#pragma unroll
+            for (int k = 0; k < TC_BK / 16; ++k) {
+              const uint64_t koff = (uint64_t)(j * sub16 + 2 * k);
+              if (j == 0 && k == 0) tc_mma_pair_f16(d, da_s, db_s, idesc, kb != 0);
+              else tc_mma_pair_acc(d, da_s + koff, db_s + koff, idesc);
+            }
+          }
+          tc_commit_pair(empty_bar(s), 3);  // frees this stage in both CTAs once the MMAs above have read it
+          stage_off += stage16;
+          if (++s == S) {
+            s = 0;
+            ph ^= 1;
+            stage_off = 0;
+          }
+        }
+        if (ok) tc_commit_pair(tmem_full(b), 3);  // publishes the accumulator in both CTAs
+      }
+    }
+  } else {
+    // ---------------- epilogue: warps 2..9 of both CTAs; warp w may touch TMEM lanes 32*(w%4) .. +31.
+    // Lanes 0..63 hold the gate rows of this CTA's 64 features, lanes 64..127 their up rows.  Warp set 0 (warps
+    // 2..5) takes the first half of the token columns, set 1 (warps 6..9) the second.  Inside a set the two halves of
+    // silu(g) * u meet through shared memory, 32 tokens at a time, in two buffers: on even chunks the up warps write
+    // buffer 0 and the gate warps combine and store, on odd chunks the gate warps write buffer 1 and the up warps
+    // combine and store.  Named barriers of a set: "buffer written" (writers arrive, readers wait) and "buffer read"
+    // (readers arrive, writers wait before writing it again) per buffer; each is used by the same 64 + 64 threads in
+    // strict alternation, so no phase can be overtaken.
+    const int quarter = warp & 3;
+    const int set = (warp - 2) >> 2;
+    const bool up_warp = quarter >= 2;
+    const int feat = (quarter & 1) * 32 + lane;  // feature within this CTA's 64
+    const int ep_tid = (warp - 2) * 32 + lane;
+    const int set_n = p.tok_n >> 1;              // token columns of a set (multiple of 8)
+    const int n_chunks = (set_n + 31) >> 5;
+    const int my_units = pair < p.n_units ? (p.n_units - pair + p.n_pairs - 1) / p.n_pairs : 0;
+    const int total_chunks = my_units * n_chunks;
+    const int bar_written = 2 + set * 4, bar_read = 4 + set * 4, bar_group = 10 + set * 2 + (up_warp ? 0 : 1);
+    float* xset = xch + set * (2 * 32 * SP_FEAT);
+    int it = 0, cc = 0;
+    for (int u = pair; u < p.n_units; u += p.n_pairs, ++it) {
+      const int b = it & 1;
+      if (ep_tid == 0) ep_ok[0] = mbar_wait(tmem_full(b), (it >> 1) & 1, abort_flag, p.status) ? 1 : 0;
+      named_bar_sync(1, 256);
+      if (!ep_ok[0]) break;  // uniform for the 256 threads
+      tc_fence_after();
+      const uint32_t trow = tmem_base + (uint32_t)b * 256u + (uint32_t)(set * set_n) + ((uint32_t)(quarter * 32) << 16);
+      const int f = (u / p.tok_tiles) * (2 * SP_FEAT) + (int)rank * SP_FEAT + feat;
+      const int t0 = (u % p.tok_tiles) * p.tok_n + set * set_n;
+      bf16* out = p.C + f;
+#pragma unroll 1
+      for (int c = 0; c < n_chunks; ++c, ++cc) {
+        const int buf = cc & 1;
+        const int w = min(32, set_n - c * 32);
+        float* xb = xset + buf * (32 * SP_FEAT);
+        float v[32];
+        __syncwarp();
+        sp_ld_chunk(trow + c * 32, w, v);
+        const bool writer = up_warp == (buf == 0);
+        if (writer) {
+          if (cc >= 2) named_bar_sync(bar_read + buf, 128);  // the readers are done with what this buffer held
+          if (w == 32) {
+#pragma unroll
+            for (int e = 0; e < 32; ++e) xb[e * SP_FEAT + feat] = v[e];
+          } else {
+#pragma unroll
+            for (int e = 0; e < 32; ++e)
+              if (e < w) xb[e * SP_FEAT + feat] = v[e];
+          }
+          named_bar_arrive(bar_written + buf, 128);
+        } else {
+          named_bar_sync(bar_written + buf, 128);
+          bf16* orow = out + (size_t)(t0 + c * 32) * p.ldc;
+          const int valid = min(w, p.M - (t0 + c * 32));  // tokens of this chunk that exist
+#pragma unroll
+          for (int e = 0; e < 32; ++e) {
+            const float o = xb[e * SP_FEAT + feat];
+            const float g = up_warp ? o : v[e], uv = up_warp ? v[e] : o;
+            // silu(g) * u with the fast exponential and reciprocal (relative error 2^-21, far below the bf16 rounding)
+            const float r = __fdividef(g, 1.f + __expf(-g)) * uv;
+            if (e < valid) orow[(size_t)e * p.ldc] = __float2bfloat16_rn(r);
+          }
+          if (cc + 2 < total_chunks) named_bar_arrive(bar_read + buf, 128);  // nobody waits for the last two
+        }
+      }
+      // this half of the set has read its part of the accumulator (wait::ld in sp_ld_chunk): one arrival per half,
+      // set and CTA on the leader's barrier hands it back to the MMA issuer
+      tc_fence_before();
+      named_bar_sync(bar_group, 64);
+      if (lane == 0 && (quarter == 0 || quarter == 2)) mbar_arrive_in_cta(tmem_empty(b), 0);
+    }
+  }
+  tc_fence_before();
+  cluster_sync_all();  // neither CTA releases tensor or shared memory while the other may still use it
+  if (warp == 1) asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(512) : "memory");
+}
+
+// 0: never; 1: whenever the shape allows (default); tuning/tests switch it off to compare with the one-CTA kernel
+int g_swiglu_pair = 1;
+
+bool swiglu_pair_usable(const a3_handle* h, const GemmArgs& a) {
+  (void)h;
+  return g_swiglu_pair != 0 && a.M > 0 && a.K % (SP_SUB * TC_BK) == 0 && a.seg[0].n % (2 * SP_FEAT) == 0 && a.seg[0].bias == nullptr;
+}
+
+int gemm_swiglu_pair(const a3_handle* h, const GemmArgs& a, cudaStream_t st) {
+  SpParams p{};
+  p.M = a.M;
+  p.K = a.K;
+  p.F = a.seg[0].n;
+  p.tok_tiles = cdiv(a.M, 256);
+  p.tok_n = cdiv(cdiv(a.M, p.tok_tiles), 16) * 16;  // even split, multiple of 16: 804 rows -> 4 x 208
+  p.n_units = (p.F / (2 * SP_FEAT)) * p.tok_tiles;
+  const int sms = h->sm_count > 0 ? h->sm_count : 148;
+  p.n_pairs = p.n_units < sms / 2 ? p.n_units : sms / 2;
+  p.C = a.C;
+  p.ldc = a.ldc;
+  p.status = h->dev_status;
+  // as many ring stages as fit beside the exchange buffers
+  p.sub_bytes = SP_A_BYTES + (int)align_up((size_t)(p.tok_n / 2) * TC_BK * 2, 1024);
+  p.stage_bytes = SP_SUB * p.sub_bytes;
+  p.stages = (SP_SMEM_LIMIT - SP_XCH_BYTES - 256 - 1024) / p.stage_bytes;
+  if (p.stages > SP_MAX_STAGES) p.stages = SP_MAX_STAGES;
+  const int smem_bytes = p.stages * p.stage_bytes + SP_XCH_BYTES + 256 + 1024;
+  CUtensorMap tX, tG, tU;
+  A3_TRY(make_tmap(&tX, a.A, a.M, a.K, p.tok_n / 2));
+  A3_TRY(make_tmap(&tG, a.seg[0].B, p.F, a.K, SP_FEAT));
+  A3_TRY(make_tmap(&tU, a.B2, p.F, a.K, SP_FEAT));
+  static bool attr_set = false;
+  if (!attr_set) {
+    A3_CUDA(cudaFuncSetAttribute(swiglu_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SP_SMEM_LIMIT));
+    attr_set = true;
+  }
+  ProfScope prof(h, A3_K_GEMM_SWIGLU, st);
+  if (g_swiglu_pair == 2) {
+    swiglu_pair_kernel<<<dim3(2 * p.n_pairs), dim3(SP_THREADS), (size_t)smem_bytes, st>>>(tX, tG, tU, p);
+  } else {
+    A3_CUDA(launch_pdl(swiglu_pair_kernel, dim3(2 * p.n_pairs), dim3(SP_THREADS), (size_t)smem_bytes, st, tX, tG, tU, p));
+  }
+  A3_LAUNCHED();
+  return A3_OK;
+}
+
+}  // namespace a3
+
+extern "C" void a3_internal_set_swiglu_pair(int v) { a3::g_swiglu_pair = v; }
+
+
+// Tuning hook: the SwiGLU GEMM of one layer alone, out[M][d_ff] = silu(x Wg^T) * (x Wu^T), x [M][d_model].
+extern "C" int a3_internal_swiglu(const a3_handle* h, int layer, const void* x, void* out, int M, void* stream) {
+  a3::GemmArgs u{};
+  u.A = (const bf16*)x;
+  u.M = M;
+  u.K = h->m.d_model;
+  u.nseg = 1;
+  u.seg[0] = {(const bf16*)h->layers[layer].w_gate, nullptr, h->m.d_ff, 0};
+  u.B2 = (const bf16*)h->layers[layer].w_up;
+  u.C = (bf16*)out;
+  u.ldc = h->m.d_ff;
+  return a3::gemm_bf16(h, a3::EPI_SWIGLU, u, (cudaStream_t)stream);
+}

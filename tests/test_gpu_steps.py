@@ -646,6 +646,7 @@ def test_swiglu_narrow_column_tiles(a3mod, shape, M, g):
     eng, layers, dev = make_engine(a3mod, m, seed=41, w_std=0.05)
     lib = a3mod._load()
     lib.a3_internal_set_gemm_narrow.argtypes = [ctypes.c_int]
+    lib.a3_internal_set_swiglu_pair.argtypes = [ctypes.c_int]
     model, weights = oracle_model(m), oracle_weights(layers)
     rng = np.random.default_rng(17)
     kv_len = 3 * M
@@ -657,6 +658,7 @@ def test_swiglu_narrow_column_tiles(a3mod, shape, M, g):
     dpos = torch.from_numpy(pos.astype(np.int32)).to(dev)
     outs = {}
     try:
+        lib.a3_internal_set_swiglu_pair(0)  # the one-CTA-per-tile kernel (the CTA-pair kernel is the default)
         for mode in (g, 0):
             lib.a3_internal_set_gemm_narrow(mode)
             dX, dK, dV = to_dev(X, dev), to_dev(Kc[layer], dev), to_dev(Vc[layer], dev)
@@ -665,8 +667,47 @@ def test_swiglu_narrow_column_tiles(a3mod, shape, M, g):
             outs[mode] = dX
     finally:
         lib.a3_internal_set_gemm_narrow(1)
+        lib.a3_internal_set_swiglu_pair(1)
     assert torch.equal(outs[g], outs[0])
     Ko, Vo = Kc[layer].astype(np.float64), Vc[layer].astype(np.float64)
     Xo, parts = O.recompute_layer(X.astype(np.float64), pos, weights[layer], model, Ko, Vo, rnd=O.round_bf16, return_parts=True)
     check_kv(f64(outs[g]), parts["x_exact"], "hidden rows", scale=2.0 * float(parts["x_exact"].std()))
+    eng.close()
+
+
+@pytest.mark.parametrize("shape,M", [(W.TINY, 1), (W.TINY, 95), (W.TINY_GQA, 257), (W.TINY_GQA, 700), (W.TINY_G7, 131), (W.TINY_G7, 513)])
+def test_swiglu_pair_kernel_matches_one_cta_kernel(a3mod, shape, M):
+    """The SwiGLU GEMM in use (weights as the M-side operand of a CTA pair, token tiles that divide the row count
+    evenly, persistent schedule with double-buffered accumulators) against the one-CTA-per-tile kernel it replaced:
+    two independent kernels, one formula, the same sum order over the model dimension - bit for bit; row counts of one
+    row, of one ragged token tile, of several tiles and of several units per CTA pair; and against the oracle."""
+    import ctypes
+    m = shape
+    eng, layers, dev = make_engine(a3mod, m, seed=51, w_std=0.05)
+    lib = a3mod._load()
+    lib.a3_internal_set_swiglu_pair.argtypes = [ctypes.c_int]
+    model, weights = oracle_model(m), oracle_weights(layers)
+    rng = np.random.default_rng(23)
+    kv_len = 2 * M + 40
+    pos = np.sort(rng.choice(kv_len, size=M, replace=False))
+    pos[-1] = kv_len - 1
+    X = W.bf16_round(rng.standard_normal((M, m.d_model), dtype=np.float32))
+    Kc, Vc = W.make_cache_like(m, kv_len, 51, 9, std=1.0)
+    layer = m.n_layers - 1
+    dpos = torch.from_numpy(pos.astype(np.int32)).to(dev)
+    outs = {}
+    try:
+        for mode in (1, 0, 1):
+            lib.a3_internal_set_swiglu_pair(mode)
+            dX, dK, dV = to_dev(X, dev), to_dev(Kc[layer], dev), to_dev(Vc[layer], dev)
+            eng.recompute_layer(layer, dX, dpos, dK, dV)
+            assert eng.device_status() == 0
+            outs.setdefault(mode, []).append(dX)
+    finally:
+        lib.a3_internal_set_swiglu_pair(1)
+    assert torch.equal(outs[1][0], outs[1][1])  # reproducible
+    assert torch.equal(outs[1][0], outs[0][0])
+    Ko, Vo = Kc[layer].astype(np.float64), Vc[layer].astype(np.float64)
+    Xo, parts = O.recompute_layer(X.astype(np.float64), pos, weights[layer], model, Ko, Vo, rnd=O.round_bf16, return_parts=True)
+    check_kv(f64(outs[1][0]), parts["x_exact"], "hidden rows", scale=2.0 * float(parts["x_exact"].std()))
     eng.close()
