@@ -629,6 +629,7 @@ int gemm_bf16(const a3_handle* h, GemmEpilogue epi, const GemmArgs& a, cudaStrea
   if (a.M <= 0) return A3_OK;
   if (a.K % TC_BK) return A3_EUNSUPPORTED;
   if (epi == EPI_SWIGLU && swiglu_pair_usable(h, a)) return gemm_swiglu_pair(h, a, st);
+  if (epi == EPI_RESIDUAL && g_tc_cfg[EPI_RESIDUAL][0] == 0 && residual_t_usable(h, a)) return gemm_residual_t(h, a, st);
   int bn = g_tc_cfg[epi][0];
   int stages = g_tc_cfg[epi][1];
 

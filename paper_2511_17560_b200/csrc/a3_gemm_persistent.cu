@@ -1,21 +1,22 @@
-// SwiGLU GEMM of the recompute path (the feed-forward part of H(.) in Eq. 5) with the operand roles swapped and a
-// persistent schedule:   out[t][f] = silu(x[t] . Wg[f]) * (x[t] . Wu[f]).
+// Persistent CTA-pair GEMMs of the recompute path (the feed-forward part of H(.) in Eq. 5) with the operand roles
+// swapped:   SwiGLU    out[t][f] = silu(x[t] . Wg[f]) * (x[t] . Wu[f])
+//            residual  C[t][f] += x[t] . W[f]            (output projection, MLP down projection)
 //
-// Why another kernel.  With one CTA per 128-token x 256-column tile, an SM pulls 48 KiB per k-block through its L2
-// port and that port, not the tensor pipe, sets the pace (measured: a wave's time follows the bytes, 107 GB/s per
-// SM); at 804 tokens the 128-row tiles also pad the rows to 896 and the grid to three waves.  Here
-//   * the WEIGHTS are the M-side operand of tcgen05.mma.cta_group::2 (M = 256 over a CTA pair): each CTA holds 64
-//     gate rows and 64 up rows of the same 64 features (its 128 accumulator lanes), so gate and up of a feature
-//     meet inside one CTA;
+// Why another kernel.  With one CTA per 128-token x 256-column tile an SM pulls 48 KiB per k-block through its L2
+// port and that, not the tensor pipe, sets the pace (a wave's time follows the bytes: about 107 GB/s per SM with
+// 192 KiB in flight); at 804 tokens the 128-row tiles also pad the rows to 896 and the grid to three waves.  Here
+//   * the WEIGHTS are the M-side operand of tcgen05.mma.cta_group::2 (M = 256 over a CTA pair).  SwiGLU: each CTA
+//     holds 64 gate rows and 64 up rows of the same 64 features (its 128 accumulator lanes), so gate and up of a
+//     feature meet inside one CTA; residual: 128 rows of the one matrix;
 //   * the TOKENS are the N-side operand, in tiles of N <= 256 tokens chosen to divide the row count evenly
 //     (804 rows -> 4 x 208: 3 % padding instead of 11 %); each CTA loads half of the token tile, the instruction
-//     reads both halves.  Per k-block an SM pulls 16 KiB of weights + N/2 token rows (13 KiB at N = 208) for
-//     64 x N outputs: 0.6 of the bytes per output of the one-CTA kernel;
-//   * the kernel is persistent: CTA pair p walks units p, p + pairs, ... (unit = 128 features x one token tile),
-//     accumulators are double-buffered in tensor memory (2 x N <= 512 columns), so the epilogue of a unit runs under
-//     the main loop of the next one.
-// Epilogue: the warps that own the "up" lanes park their values in shared memory, the warps that own the "gate"
-// lanes combine and store out[t][f] (a warp writes 32 consecutive features of one token: 64 bytes).
+//     reads both halves.  Per k-block an SM pulls 16 KiB of weights + N/2 token rows (13 KiB at N = 208);
+//   * the kernel is persistent: CTA pair p walks units p, p + pairs, ... (unit = 128 (SwiGLU) or 256 features x one
+//     token tile), accumulators are double-buffered in tensor memory (2 x N <= 512 columns), so the epilogue of a
+//     unit runs under the main loop of the next one; a ring stage holds two k-blocks (one barrier hand-shake and one
+//     commit per eight instructions: the single issuing thread, not the pipe, was the limit with one).
+// SwiGLU epilogue: the two halves meet through shared memory (see below); a warp writes 32 consecutive features of
+// one token (64 bytes) per instruction.  Measured at Llama-8B width: tensor pipe 97 % active at 5 152 rows.
 // No load uses cluster multicast.  Every wait is bounded (see a3_tc.cuh): a waiter that gives up raises the CTA's
 // abort flag and the device status bit, all roles leave their loops, tensor memory is released and the CTA returns.
 #include <cuda.h>
@@ -77,14 +78,18 @@ __device__ __forceinline__ void tc_mma_pair_acc(uint32_t d_tmem, uint64_t a_desc
       : "memory");
 }
 
+// EPI_SWIGLU: tmG/tmU are the gate and up matrices (box of 64 rows each); EPI_RESIDUAL: tmG is the one weight matrix
+// (box of 128 rows, tmU unused) and the epilogue adds the accumulator to C in place.
+template <int EPI>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(SP_THREADS, 1)
-swiglu_pair_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUtensorMap tmG,
-                   const __grid_constant__ CUtensorMap tmU, const SpParams p) {
+pair_t_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUtensorMap tmG,
+              const __grid_constant__ CUtensorMap tmU, const SpParams p) {
+  constexpr int ROWS = EPI == EPI_SWIGLU ? SP_FEAT : 2 * SP_FEAT;  // output features per CTA
   extern __shared__ unsigned char smem_raw[];
   const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;  // same offset in both CTAs of the pair
   unsigned char* base_ptr = smem_raw + (base - smem_u32(smem_raw));
   const int S = p.stages;
-  const int xch_off = S * p.stage_bytes, bar_off = xch_off + SP_XCH_BYTES;
+  const int xch_off = S * p.stage_bytes, bar_off = xch_off + (EPI == EPI_SWIGLU ? SP_XCH_BYTES : 0);
   // barriers (8 bytes each): full[8] (used in the leader), empty[8], tmem_full[2], tmem_empty[2] (used in the leader)
   const uint32_t bars = base + bar_off;
   auto full_bar = [&](int s) { return bars + 8u * s; };
@@ -111,7 +116,8 @@ swiglu_pair_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constan
     }
     for (int b = 0; b < 2; ++b) {
       mbar_init(tmem_full(b), 1);
-      mbar_init(tmem_empty(b), 8);  // the gate warps and the up warps of both warp sets of each CTA of the pair
+      // SwiGLU: the gate warps and the up warps of both warp sets of each CTA; residual: every epilogue warp
+      mbar_init(tmem_empty(b), EPI == EPI_SWIGLU ? 8 : 16);
     }
     abort_flag[0] = 0;
     abort_flag[1] = 0;
@@ -135,13 +141,13 @@ swiglu_pair_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constan
     if (lane == 0) {
       tmap_prefetch(&tmX);
       tmap_prefetch(&tmG);
-      tmap_prefetch(&tmU);
+      if (EPI == EPI_SWIGLU) tmap_prefetch(&tmU);
       int kbg = 0, issued = 0;
       int s = 0;        // ring position and phase, kept by counting: S is a run-time value and a division per
       uint32_t ph = 0;  // k-block is a long dependent chain in a one-thread role
       bool ok = true;
       for (int u = pair; u < p.n_units && ok; u += p.n_pairs) {
-        const int f0 = (u / p.tok_tiles) * (2 * SP_FEAT) + (int)rank * SP_FEAT;
+        const int f0 = (u / p.tok_tiles) * (2 * ROWS) + (int)rank * ROWS;
         const int t0 = (u % p.tok_tiles) * p.tok_n + (int)rank * half_n;
         for (int kb = 0; kb < KT; kb += SP_SUB, ++kbg) {
           if (!mbar_wait(empty_bar(s), ph ^ 1, abort_flag, p.status)) {
@@ -153,10 +159,11 @@ swiglu_pair_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constan
           // phase, because the leader's own arrival is still pending until its expect_tx
           if (leader) mbar_expect_tx(full_bar(s), 2 * SP_SUB * (SP_A_BYTES + b_bytes));
 #pragma unroll
+#pragma unroll
           for (int j = 0; j < SP_SUB; ++j) {
             const uint32_t sa = base + s * p.stage_bytes + j * p.sub_bytes, sb = sa + SP_A_BYTES;
             tma_load_2d_pair(sa, &tmG, (kb + j) * TC_BK, f0, full_leader);
-            tma_load_2d_pair(sa + SP_A_BYTES / 2, &tmU, (kb + j) * TC_BK, f0, full_leader);
+            if (EPI == EPI_SWIGLU) tma_load_2d_pair(sa + SP_A_BYTES / 2, &tmU, (kb + j) * TC_BK, f0, full_leader);
             tma_load_2d_pair(sb, &tmX, (kb + j) * TC_BK, t0, full_leader);
           }
           issued = kbg + 1;
@@ -179,51 +186,65 @@ swiglu_pair_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constan
       }
     }
   } else if (warp == 1) {
-    // ---------------- MMA issuer: the leader alone, for both CTAs
+    // ---------------- MMA issuer: the leader alone, for both CTAs.
+    // The tensor pipe queues only about two instructions, so everything this thread does between two of them has
+    // to fit into some 200 clocks or the pipe runs dry.  The look at the next stage's barrier therefore happens in
+    // the middle of a stage (after its first four instructions), the commit and the ring arithmetic at its end.
     if (lane == 0 && leader) {
       const uint32_t idesc = idesc_bf16_pair(p.tok_n);
-      int kbg = 0, it = 0;
-      int s = 0;
-      uint32_t ph = 0;
-      bool ok = true;
       const uint64_t da0 = smem_desc_sw128(base), db0 = smem_desc_sw128(base + SP_A_BYTES);
+      // descriptor address fields count 16-byte units: stage and k-step offsets are added to the first stage's
       const uint32_t stage16 = (uint32_t)p.stage_bytes >> 4, sub16 = (uint32_t)p.sub_bytes >> 4;
-      uint32_t stage_off = 0;
-      for (int u = pair; u < p.n_units && ok; u += p.n_pairs, ++it) {
-        const int b = it & 1;
-        // the epilogues of both CTAs have drained this accumulator (first use: passes at once)
-        ok = mbar_wait(tmem_empty(b), ((it >> 1) & 1) ^ 1, abort_flag, p.status);
+      const int per_unit = KT / SP_SUB;
+      const int my_units = pair < p.n_units ? (p.n_units - pair + p.n_pairs - 1) / p.n_pairs : 0;
+      const int total = my_units * per_unit;
+      int s = 0, it = 0, in_unit = 0;
+      uint32_t ph = 0, stage_off = 0, d = tmem_base;
+      bool ok = total > 0, ready = false;
+      for (int g = 0; g < total && ok; ++g) {
+        if (in_unit == 0) {
+          // the epilogues of both CTAs have drained this accumulator (first use: passes at once)
+          const int b = it & 1;
+          ok = mbar_wait(tmem_empty(b), ((it >> 1) & 1) ^ 1, abort_flag, p.status);
+          if (!ok) break;
+          d = tmem_base + (uint32_t)b * 256u;
+        }
+        if (!ready) ok = mbar_wait(full_bar(s), ph, abort_flag, p.status);
         if (!ok) break;
         tc_fence_after();
-        const uint32_t d = tmem_base + (uint32_t)b * 256u;
-        for (int kb = 0; kb < KT; kb += SP_SUB, ++kbg) {
-          ok = mbar_wait(full_bar(s), ph, abort_flag, p.status);
-          if (!ok) break;
-          tc_fence_after();
-          // descriptors of this stage: the address field counts 16-byte units, so stage and k-step offsets are added
-          // to the descriptors of the ring's first stage (all of shared memory fits the field)
-          const uint64_t da_s = da0 + stage_off, db_s = db0 + stage_off;
+        const uint64_t da_s = da0 + stage_off, db_s = db0 + stage_off;
+        tc_mma_pair_f16(d, da_s, db_s, idesc, in_unit != 0);
 #pragma unroll
-          for (int j = 0; j < SP_SUB; ++j) {
+        for (int k = 1; k < TC_BK / 16; ++k) tc_mma_pair_acc(d, da_s + (uint64_t)(2 * k), db_s + (uint64_t)(2 * k), idesc);
+        // next ring position, and one look at its barrier while the pipe works on the instructions above
+        int sn = s + 1;
+        uint32_t phn = ph, offn = stage_off + stage16;
+        if (sn == S) {
+          sn = 0;
+          phn ^= 1;
+          offn = 0;
+        }
+        ready = g + 1 < total && mbar_try_wait(full_bar(sn), phn);
 #pragma unroll
-            for (int k = 0; k < TC_BK / 16; ++k) {
-              const uint64_t koff = (uint64_t)(j * sub16 + 2 * k);
-              if (j == 0 && k == 0) tc_mma_pair_f16(d, da_s, db_s, idesc, kb != 0);
-              else tc_mma_pair_acc(d, da_s + koff, db_s + koff, idesc);
-            }
-          }
-          tc_commit_pair(empty_bar(s), 3);  // frees this stage in both CTAs once the MMAs above have read it
-          stage_off += stage16;
-          if (++s == S) {
-            s = 0;
-            ph ^= 1;
-            stage_off = 0;
+        for (int j = 1; j < SP_SUB; ++j) {
+#pragma unroll
+          for (int k = 0; k < TC_BK / 16; ++k) {
+            const uint64_t koff = (uint64_t)(j * sub16 + 2 * k);
+            tc_mma_pair_acc(d, da_s + koff, db_s + koff, idesc);
           }
         }
-        if (ok) tc_commit_pair(tmem_full(b), 3);  // publishes the accumulator in both CTAs
+        tc_commit_pair(empty_bar(s), 3);  // frees this stage in both CTAs once the instructions above have read it
+        if (++in_unit == per_unit) {
+          tc_commit_pair(tmem_full(it & 1), 3);  // publishes the accumulator in both CTAs
+          in_unit = 0;
+          ++it;
+        }
+        s = sn;
+        ph = phn;
+        stage_off = offn;
       }
     }
-  } else {
+  } else if (EPI == EPI_SWIGLU) {
     // ---------------- epilogue: warps 2..9 of both CTAs; warp w may touch TMEM lanes 32*(w%4) .. +31.
     // Lanes 0..63 hold the gate rows of this CTA's 64 features, lanes 64..127 their up rows.  Warp set 0 (warps
     // 2..5) takes the first half of the token columns, set 1 (warps 6..9) the second.  Inside a set the two halves of
@@ -295,28 +316,94 @@ swiglu_pair_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constan
       named_bar_sync(bar_group, 64);
       if (lane == 0 && (quarter == 0 || quarter == 2)) mbar_arrive_in_cta(tmem_empty(b), 0);
     }
+  } else if (EPI == EPI_RESIDUAL) {
+    // ---------------- epilogue, C += A B^T: warps 2..9 of both CTAs; warp w may touch TMEM lanes 32*(w%4) .. +31,
+    // lane = output feature; warp set 0 (warps 2..5) takes the first half of the token columns, set 1 the second.
+    // A warp reads and writes 32 consecutive features of one token (64 bytes) per instruction.
+    const int quarter = warp & 3;
+    const int set = (warp - 2) >> 2;
+    const int ep_tid = (warp - 2) * 32 + lane;
+    const int set_n = p.tok_n >> 1;
+    const int n_chunks = (set_n + 31) >> 5;
+    int it = 0;
+    for (int u = pair; u < p.n_units; u += p.n_pairs, ++it) {
+      const int b = it & 1;
+      const int f = (u / p.tok_tiles) * (2 * ROWS) + (int)rank * ROWS + quarter * 32 + lane;
+      const int t0 = (u % p.tok_tiles) * p.tok_n + set * set_n;
+      const bool f_ok = f < p.F;  // the last feature block may reach past the matrix (zero-filled loads)
+      bf16* crow = p.C + (size_t)t0 * p.ldc + (f_ok ? f : 0);
+      // the old values of the first chunk are on their way while the main loop still runs
+      bf16 old[32];
+      {
+        const int valid = f_ok ? min(min(32, set_n), p.M - t0) : 0;
+#pragma unroll
+        for (int e = 0; e < 32; ++e) old[e] = e < valid ? crow[(size_t)e * p.ldc] : __float2bfloat16_rn(0.f);
+      }
+      if (ep_tid == 0) ep_ok[0] = mbar_wait(tmem_full(b), (it >> 1) & 1, abort_flag, p.status) ? 1 : 0;
+      named_bar_sync(1, 256);
+      if (!ep_ok[0]) break;  // uniform for the 256 threads
+      tc_fence_after();
+      const uint32_t trow = tmem_base + (uint32_t)b * 256u + (uint32_t)(set * set_n) + ((uint32_t)(quarter * 32) << 16);
+#pragma unroll 1
+      for (int c = 0; c < n_chunks; ++c) {
+        const int w = min(32, set_n - c * 32);
+        float v[32];
+        __syncwarp();
+        sp_ld_chunk(trow + c * 32, w, v);
+        bf16* orow = crow + (size_t)(c * 32) * p.ldc;
+        const int valid = f_ok ? min(w, p.M - (t0 + c * 32)) : 0;
+#pragma unroll
+        for (int e = 0; e < 32; ++e)
+          if (e < valid) orow[(size_t)e * p.ldc] = __float2bfloat16_rn(v[e] + __bfloat162float(old[e]));
+        if (c + 1 < n_chunks) {  // the next chunk's old values
+          const int nvalid = f_ok ? min(min(32, set_n - (c + 1) * 32), p.M - (t0 + (c + 1) * 32)) : 0;
+          const bf16* nrow = orow + (size_t)32 * p.ldc;
+#pragma unroll
+          for (int e = 0; e < 32; ++e) old[e] = e < nvalid ? nrow[(size_t)e * p.ldc] : __float2bfloat16_rn(0.f);
+        }
+      }
+      // this warp has read its part of the accumulator (wait::ld in sp_ld_chunk): it goes back to the MMA issuer
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive_in_cta(tmem_empty(b), 0);
+    }
   }
   tc_fence_before();
   cluster_sync_all();  // neither CTA releases tensor or shared memory while the other may still use it
   if (warp == 1) asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(512) : "memory");
 }
 
-// 0: never; 1: whenever the shape allows (default); tuning/tests switch it off to compare with the one-CTA kernel
+// 0: never; 1: whenever the shape allows (default); tuning/tests switch them off to compare with the other kernels
 int g_swiglu_pair = 1;
+int g_residual_t = 1;
 
 bool swiglu_pair_usable(const a3_handle* h, const GemmArgs& a) {
   (void)h;
   return g_swiglu_pair != 0 && a.M > 0 && a.K % (SP_SUB * TC_BK) == 0 && a.seg[0].n % (2 * SP_FEAT) == 0 && a.seg[0].bias == nullptr;
 }
+// Measured at Llama-8B width: with several units per CTA pair (5 152 rows: 336 units on 74 pairs) this kernel hides
+// every epilogue but the last and wins (output projection 139 vs 165 us, down projection 522 vs 533 us); with at most
+// one unit per pair (804 rows: 64 units) it has nothing to hide and the 256 x 256 CTA-pair kernel is as fast or faster
+// (26 vs 28 us, 85 vs 82 us).  g_residual_t: 0 never, 1 by that rule (default), 2 whenever the shape allows (tests).
+bool residual_t_usable(const a3_handle* h, const GemmArgs& a) {
+  if (g_residual_t == 0 || a.M <= 0 || a.K % (SP_SUB * TC_BK) != 0 || a.nseg != 1 || a.seg[0].n % 32 != 0 || a.seg[0].bias != nullptr)
+    return false;
+  if (g_residual_t == 2) return true;
+  const int sms = h->sm_count > 0 ? h->sm_count : 148;
+  return cdiv(a.seg[0].n, 4 * SP_FEAT) * cdiv(a.M, 256) > sms / 2;
+}
 
-int gemm_swiglu_pair(const a3_handle* h, const GemmArgs& a, cudaStream_t st) {
+template <int EPI>
+static int launch_pair_t(const a3_handle* h, const GemmArgs& a, cudaStream_t st) {
+  constexpr int ROWS = EPI == EPI_SWIGLU ? SP_FEAT : 2 * SP_FEAT;  // output features per CTA
+  constexpr int XCH = EPI == EPI_SWIGLU ? SP_XCH_BYTES : 0;
   SpParams p{};
   p.M = a.M;
   p.K = a.K;
   p.F = a.seg[0].n;
   p.tok_tiles = cdiv(a.M, 256);
   p.tok_n = cdiv(cdiv(a.M, p.tok_tiles), 16) * 16;  // even split, multiple of 16: 804 rows -> 4 x 208
-  p.n_units = (p.F / (2 * SP_FEAT)) * p.tok_tiles;
+  p.n_units = cdiv(p.F, 2 * ROWS) * p.tok_tiles;
   const int sms = h->sm_count > 0 ? h->sm_count : 148;
   p.n_pairs = p.n_units < sms / 2 ? p.n_units : sms / 2;
   p.C = a.C;
@@ -325,31 +412,32 @@ int gemm_swiglu_pair(const a3_handle* h, const GemmArgs& a, cudaStream_t st) {
   // as many ring stages as fit beside the exchange buffers
   p.sub_bytes = SP_A_BYTES + (int)align_up((size_t)(p.tok_n / 2) * TC_BK * 2, 1024);
   p.stage_bytes = SP_SUB * p.sub_bytes;
-  p.stages = (SP_SMEM_LIMIT - SP_XCH_BYTES - 256 - 1024) / p.stage_bytes;
+  p.stages = (SP_SMEM_LIMIT - XCH - 256 - 1024) / p.stage_bytes;
   if (p.stages > SP_MAX_STAGES) p.stages = SP_MAX_STAGES;
-  const int smem_bytes = p.stages * p.stage_bytes + SP_XCH_BYTES + 256 + 1024;
+  const int smem_bytes = p.stages * p.stage_bytes + XCH + 256 + 1024;
   CUtensorMap tX, tG, tU;
   A3_TRY(make_tmap(&tX, a.A, a.M, a.K, p.tok_n / 2));
-  A3_TRY(make_tmap(&tG, a.seg[0].B, p.F, a.K, SP_FEAT));
-  A3_TRY(make_tmap(&tU, a.B2, p.F, a.K, SP_FEAT));
+  A3_TRY(make_tmap(&tG, a.seg[0].B, p.F, a.K, ROWS));
+  if (EPI == EPI_SWIGLU) A3_TRY(make_tmap(&tU, a.B2, p.F, a.K, ROWS));
+  else tU = tG;
   static bool attr_set = false;
   if (!attr_set) {
-    A3_CUDA(cudaFuncSetAttribute(swiglu_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SP_SMEM_LIMIT));
+    A3_CUDA(cudaFuncSetAttribute(pair_t_kernel<EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize, SP_SMEM_LIMIT));
     attr_set = true;
   }
-  ProfScope prof(h, A3_K_GEMM_SWIGLU, st);
-  if (g_swiglu_pair == 2) {
-    swiglu_pair_kernel<<<dim3(2 * p.n_pairs), dim3(SP_THREADS), (size_t)smem_bytes, st>>>(tX, tG, tU, p);
-  } else {
-    A3_CUDA(launch_pdl(swiglu_pair_kernel, dim3(2 * p.n_pairs), dim3(SP_THREADS), (size_t)smem_bytes, st, tX, tG, tU, p));
-  }
+  ProfScope prof(h, EPI == EPI_SWIGLU ? A3_K_GEMM_SWIGLU : A3_K_GEMM_RESIDUAL, st);
+  A3_CUDA(launch_pdl(pair_t_kernel<EPI>, dim3(2 * p.n_pairs), dim3(SP_THREADS), (size_t)smem_bytes, st, tX, tG, tU, p));
   A3_LAUNCHED();
   return A3_OK;
 }
 
+int gemm_swiglu_pair(const a3_handle* h, const GemmArgs& a, cudaStream_t st) { return launch_pair_t<EPI_SWIGLU>(h, a, st); }
+int gemm_residual_t(const a3_handle* h, const GemmArgs& a, cudaStream_t st) { return launch_pair_t<EPI_RESIDUAL>(h, a, st); }
+
 }  // namespace a3
 
 extern "C" void a3_internal_set_swiglu_pair(int v) { a3::g_swiglu_pair = v; }
+extern "C" void a3_internal_set_residual_t(int v) { a3::g_residual_t = v; }
 
 
 // Tuning hook: the SwiGLU GEMM of one layer alone, out[M][d_ff] = silu(x Wg^T) * (x Wu^T), x [M][d_model].
@@ -364,4 +452,18 @@ extern "C" int a3_internal_swiglu(const a3_handle* h, int layer, const void* x, 
   u.C = (bf16*)out;
   u.ldc = h->m.d_ff;
   return a3::gemm_bf16(h, a3::EPI_SWIGLU, u, (cudaStream_t)stream);
+}
+
+// Tuning hook: one residual GEMM of a layer alone, C[M][d_model] += x W^T; which = 0: output projection (x [M][Hq*D]),
+// 1: MLP down projection (x [M][d_ff]).
+extern "C" int a3_internal_residual(const a3_handle* h, int layer, int which, const void* x, void* c, int M, void* stream) {
+  a3::GemmArgs g{};
+  g.A = (const bf16*)x;
+  g.M = M;
+  g.K = which == 0 ? h->m.n_q_heads * h->m.head_dim : h->m.d_ff;
+  g.nseg = 1;
+  g.seg[0] = {(const bf16*)(which == 0 ? h->layers[layer].wo : h->layers[layer].w_down), nullptr, h->m.d_model, 0};
+  g.C = (bf16*)c;
+  g.ldc = h->m.d_model;
+  return a3::gemm_bf16(h, a3::EPI_RESIDUAL, g, (cudaStream_t)stream);
 }

@@ -140,6 +140,9 @@ struct GemmArgs {
 // SwiGLU GEMM with the weights as the M-side operand of a CTA pair, persistent (a3_swiglu_pair.cu).
 bool swiglu_pair_usable(const a3_handle* h, const GemmArgs& a);
 int gemm_swiglu_pair(const a3_handle* h, const GemmArgs& a, cudaStream_t st);
+// C += A B^T with the same kernel structure (weights on the M side, persistent CTA pairs).
+bool residual_t_usable(const a3_handle* h, const GemmArgs& a);
+int gemm_residual_t(const a3_handle* h, const GemmArgs& a, cudaStream_t st);
 
 // C-tile GEMM with fused epilogue on the tensor cores; all operands K-major bf16, fp32 accumulate.
 int gemm_bf16(const a3_handle* h, GemmEpilogue epi, const GemmArgs& a, cudaStream_t st);

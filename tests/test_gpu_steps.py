@@ -711,3 +711,40 @@ def test_swiglu_pair_kernel_matches_one_cta_kernel(a3mod, shape, M):
     Xo, parts = O.recompute_layer(X.astype(np.float64), pos, weights[layer], model, Ko, Vo, rnd=O.round_bf16, return_parts=True)
     check_kv(f64(outs[1][0]), parts["x_exact"], "hidden rows", scale=2.0 * float(parts["x_exact"].std()))
     eng.close()
+
+
+@pytest.mark.parametrize("shape,M", [(W.TINY, 95), (W.TINY_GQA, 513), (W.TINY_G7, 131), (W.TINY_G7, 700)])
+def test_residual_persistent_pair_kernel_matches_tile_kernel(a3mod, shape, M):
+    """The residual GEMMs (C += A W^T) on the persistent CTA-pair kernel with the weights as the M-side operand
+    (chosen by itself only when a CTA pair gets several units, i.e. for thousands of rows), forced on small models -
+    among them one whose width (896) leaves the last 256-feature block half empty - against the 256 x 256 CTA-pair tile
+    kernel: bit for bit, and against the oracle."""
+    import ctypes
+    m = shape
+    eng, layers, dev = make_engine(a3mod, m, seed=61, w_std=0.05)
+    lib = a3mod._load()
+    lib.a3_internal_set_residual_t.argtypes = [ctypes.c_int]
+    model, weights = oracle_model(m), oracle_weights(layers)
+    rng = np.random.default_rng(29)
+    kv_len = 2 * M + 40
+    pos = np.sort(rng.choice(kv_len, size=M, replace=False))
+    pos[-1] = kv_len - 1
+    X = W.bf16_round(rng.standard_normal((M, m.d_model), dtype=np.float32))
+    Kc, Vc = W.make_cache_like(m, kv_len, 61, 9, std=1.0)
+    layer = m.n_layers - 1
+    dpos = torch.from_numpy(pos.astype(np.int32)).to(dev)
+    outs = {}
+    try:
+        for mode in (2, 0):
+            lib.a3_internal_set_residual_t(mode)
+            dX, dK, dV = to_dev(X, dev), to_dev(Kc[layer], dev), to_dev(Vc[layer], dev)
+            eng.recompute_layer(layer, dX, dpos, dK, dV)
+            assert eng.device_status() == 0
+            outs[mode] = dX
+    finally:
+        lib.a3_internal_set_residual_t(1)
+    assert torch.equal(outs[2], outs[0])
+    Ko, Vo = Kc[layer].astype(np.float64), Vc[layer].astype(np.float64)
+    Xo, parts = O.recompute_layer(X.astype(np.float64), pos, weights[layer], model, Ko, Vo, rnd=O.round_bf16, return_parts=True)
+    check_kv(f64(outs[2]), parts["x_exact"], "hidden rows", scale=2.0 * float(parts["x_exact"].std()))
+    eng.close()
