@@ -28,7 +28,7 @@ if ROOT not in sys.path:
 
 # DRAM bytes (read + write) per launch from the ncu capture summarised in profiles/gemm_kernels_llama8b_2layer.txt:
 # the SwiGLU GEMM of a sparse layer (M = 804) and of the full block (M = 5152) at Llama-8B width.
-NCU_TRAFFIC = {("llama8b_10x512", "gemm_swiglu"): {"sparse": 243.42e6 + 18.49e6, "full": 417.43e6 + 139.85e6}}
+NCU_TRAFFIC = {("llama8b_10x512", "gemm_swiglu"): {"sparse": 243.44e6 + 18.51e6, "full": 418.15e6 + 140.63e6}}
 
 METRIC = "context_tokens_fused_per_s"
 UNIT = "tokens/s"
