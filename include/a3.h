@@ -237,6 +237,22 @@ int a3_gather_rows(const a3_handle* h, const void* src, int n_src, const int32_t
  * Fills the fused cache in place, rows_out, scores_out, x_out. */
 int a3_fuse_request(const a3_handle* h, const a3_request* req, void* ws, size_t ws_bytes, a3_stream stream);
 
+/* The same request as a CUDA graph (the request allocates nothing and never synchronises, so it can be captured).
+ * a3_graph_capture runs the request once on `stream` (first launches set kernel attributes, which a capture must not
+ * see), then records it a second time into a graph and instantiates it; `stream` must not be the legacy default
+ * stream and must have nothing else captured on it; profiling (a3_profile_enable) must be off.  The graph holds the
+ * pointers of req, ws and the handle's weights: they must stay valid and unchanged in place until a3_graph_destroy;
+ * their CONTENTS (chunk caches, x0) may change between launches.  a3_graph_launch replays every kernel of the request
+ * on `stream` (asynchronous, no allocation); results land where a3_fuse_request would have put them.
+ * Errors: A3_EINVAL (null argument, default stream, profiling on), the request's own status, A3_ECUDA. */
+typedef struct a3_graph a3_graph;
+int a3_graph_capture(const a3_handle* h, const a3_request* req, void* ws, size_t ws_bytes, a3_stream stream,
+                     a3_graph** out);
+int a3_graph_launch(const a3_graph* g, a3_stream stream);
+/* Kernel launches one replay stands for (what a3_launch_count advances by per a3_graph_launch). */
+int a3_graph_kernel_count(const a3_graph* g);
+void a3_graph_destroy(a3_graph* g);
+
 /* Precomputation (Eq. 1, K_i, V_i = LLM(i)): prefills one chunk alone at local positions 0..T-1, i.e. runs every
  * layer over all T rows, and leaves the chunk's per-layer caches in k_chunk / v_chunk (dev [n_layers][T][Hkv][D],
  * layer l at + l*layer_stride bytes).  x_chunk: dev [T][d_model], embeddings in, final hidden state out.

@@ -67,6 +67,7 @@ EXPORTS = ("a3_create", "a3_destroy", "a3_layer_workspace_bytes", "a3_request_wo
            "a3_recompute_count", "a3_rope_rerotate", "a3_query_scores", "a3_query_scores_static", "a3_topk_select", "a3_recompute_layer",
            "a3_scatter_kv", "a3_gather_rows", "a3_precompute_chunk", "a3_first_token_workspace_bytes", "a3_first_token",
            "a3_evict_count", "a3_evict_workspace_bytes", "a3_evict_layer", "a3_chunk_edge_rows", "a3_fuse_request", "a3_fuse_batch", "a3_fuse_request_host",
+           "a3_graph_capture", "a3_graph_launch", "a3_graph_kernel_count", "a3_graph_destroy",
            "a3_device_status", "a3_status_string", "a3_last_cuda_error", "a3_launch_count", "a3_profile_enable",
            "a3_profile_read", "a3_kernel_class_name")
 K_CLASSES = 10
@@ -113,6 +114,11 @@ def _load():
     lib.a3_fuse_request.argtypes = [vp, C.POINTER(Request), vp, sz, vp]
     lib.a3_fuse_batch.argtypes = [vp, C.POINTER(Request), i32, vp, sz, vp]
     lib.a3_fuse_request_host.argtypes = [vp, C.POINTER(Request), C.POINTER(HostIO), vp, sz, vp, sz, vp]
+    lib.a3_graph_capture.argtypes = [vp, C.POINTER(Request), vp, sz, vp, C.POINTER(vp)]
+    lib.a3_graph_launch.argtypes = [vp, vp]
+    lib.a3_graph_kernel_count.argtypes = [vp]
+    lib.a3_graph_destroy.argtypes = [vp]
+    lib.a3_graph_destroy.restype = None
     lib.a3_device_status.argtypes = [vp, C.POINTER(C.c_uint32), vp]
     lib.a3_status_string.argtypes = [i32]
     lib.a3_status_string.restype = C.c_char_p
@@ -158,6 +164,31 @@ def chunk_edge_rows(chunk_lens: Sequence[int], m: int, n_system: int = 0) -> np.
 
 def evict_count(capacity: int, n_system: int, n_ctx: int, n_question: int) -> int:
     return int(_load().a3_evict_count(int(capacity), int(n_system), int(n_ctx), int(n_question)))
+
+
+class RequestGraph:
+    """A request captured by a3_graph_capture: launch() replays it on the current stream."""
+
+    def __init__(self, handle, req, ws):
+        self._g, self._req, self._ws = handle, req, ws
+
+    def launch(self):
+        _check(_load().a3_graph_launch(self._g, _stream()), "a3_graph_launch")
+
+    @property
+    def kernels(self) -> int:
+        return int(_load().a3_graph_kernel_count(self._g))
+
+    def close(self):
+        if self._g:
+            _load().a3_graph_destroy(self._g)
+            self._g = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
 
 
 def launch_count(reset: bool = False) -> int:
@@ -361,6 +392,15 @@ class A3:
         n = req.n_ctx + req.n_question
         ws = self.workspace(self.request_workspace_bytes(n))
         _check(_load().a3_fuse_request(self._h, C.byref(req), _ptr(ws), ws.numel(), _stream()), "a3_fuse_request")
+
+    def graph_capture(self, req: Request) -> "RequestGraph":
+        """a3_graph_capture on the current stream (not the default stream); the graph keeps `req` and a workspace of
+        its own alive."""
+        n = req.n_ctx + req.n_question
+        ws = torch.empty(int(self.request_workspace_bytes(n)) + 256, dtype=torch.uint8, device=self.device)
+        g = C.c_void_p()
+        _check(_load().a3_graph_capture(self._h, C.byref(req), _ptr(ws), ws.numel(), _stream(), C.byref(g)), "a3_graph_capture")
+        return RequestGraph(g, req, ws)
 
     def fuse_batch(self, reqs: Sequence[Request]):
         arr = (Request * len(reqs))(*reqs)

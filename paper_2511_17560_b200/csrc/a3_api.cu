@@ -373,6 +373,67 @@ extern "C" int a3_fuse_request(const a3_handle* h, const a3_request* r, void* ws
   return fuse_impl(h, r, ws, ws_bytes, stream, nullptr, nullptr);
 }
 
+// ---------------------------------------------------------------- the request as a CUDA graph
+struct a3_graph {
+  cudaGraph_t graph;
+  cudaGraphExec_t exec;
+  int kernels;
+};
+
+extern "C" int a3_graph_capture(const a3_handle* h, const a3_request* req, void* ws, size_t ws_bytes, a3_stream stream,
+                                a3_graph** out) {
+  if (!h || !req || !ws || !out || !stream || h->prof) return A3_EINVAL;
+  *out = nullptr;
+  cudaStream_t st = (cudaStream_t)stream;
+  // once for real: every kernel's one-time attribute set-up happens here, outside the capture
+  A3_TRY(a3_fuse_request(h, req, ws, ws_bytes, stream));
+  const unsigned long long before = g_launches;
+  A3_CUDA(cudaStreamBeginCapture(st, cudaStreamCaptureModeThreadLocal));
+  const int status = a3_fuse_request(h, req, ws, ws_bytes, stream);
+  cudaGraph_t graph = nullptr;
+  const cudaError_t e = cudaStreamEndCapture(st, &graph);  // always ends the capture, also after a failed request
+  const int kernels = (int)(g_launches - before);
+  g_launches = before;  // nothing ran during the capture
+  if (status != A3_OK || e != cudaSuccess || !graph) {
+    if (graph) cudaGraphDestroy(graph);
+    if (status != A3_OK) return status;
+    return cuda_fail(e != cudaSuccess ? e : cudaErrorUnknown);
+  }
+  cudaGraphExec_t exec = nullptr;
+  const cudaError_t ei = cudaGraphInstantiate(&exec, graph, 0);
+  if (ei != cudaSuccess) {
+    cudaGraphDestroy(graph);
+    return cuda_fail(ei);
+  }
+  a3_graph* g = (a3_graph*)calloc(1, sizeof(a3_graph));
+  if (!g) {
+    cudaGraphExecDestroy(exec);
+    cudaGraphDestroy(graph);
+    return A3_EINVAL;
+  }
+  g->graph = graph;
+  g->exec = exec;
+  g->kernels = kernels;
+  *out = g;
+  return A3_OK;
+}
+
+extern "C" int a3_graph_launch(const a3_graph* g, a3_stream stream) {
+  if (!g || !g->exec) return A3_EINVAL;
+  A3_CUDA(cudaGraphLaunch(g->exec, (cudaStream_t)stream));
+  g_launches += (unsigned long long)g->kernels;
+  return A3_OK;
+}
+
+extern "C" int a3_graph_kernel_count(const a3_graph* g) { return g ? g->kernels : 0; }
+
+extern "C" void a3_graph_destroy(a3_graph* g) {
+  if (!g) return;
+  if (g->exec) cudaGraphExecDestroy(g->exec);
+  if (g->graph) cudaGraphDestroy(g->graph);
+  free(g);
+}
+
 static int a3::fuse_impl(const a3_handle* h, const a3_request* r, void* ws, size_t ws_bytes, a3_stream stream,
                          const cudaEvent_t* layer_ready, cudaEvent_t x0_ready) {
   if (!h || !r || !ws) return A3_EINVAL;

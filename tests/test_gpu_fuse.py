@@ -374,3 +374,43 @@ def test_fuse_request_value_deviation_selector(a3mod, config, n_system):
                                    select_layer=r.select_layer, n_system=n_system, selector=1, score_source=1)
         s.eng.fuse_request(rq)
     s.eng.close()
+
+
+def test_request_graph_replays_the_request(a3mod):
+    """a3_graph_capture / a3_graph_launch: a replay leaves exactly what a3_fuse_request leaves (fused cache, rows,
+    scores, hidden rows), follows changed input CONTENTS (the graph holds pointers, not data), counts its kernels, and
+    the entry point rejects the default stream."""
+    s = Setup(a3mod, "tiny_gqa")
+    m, r = s.m, s.r
+    K, V, out = s.run_gpu(r.ratio)
+    Kg, Vg = s.fused_buffers()
+    rq, og = s.eng.make_request(s.tab, len(s.dk), max(r.chunk_lens), r.n_ctx, r.n_question, s.dx0, Kg, Vg,
+                                ratio=r.ratio, select_layer=r.select_layer)
+    with pytest.raises(a3mod.A3Error):
+        s.eng.graph_capture(rq)  # current stream is the default stream
+    side = torch.cuda.Stream()
+    with torch.cuda.stream(side):
+        g = s.eng.graph_capture(rq)
+        assert g.kernels > 0
+        for t in (Kg, Vg, og["x"], og["rows"], og["scores"]):
+            t.zero_()
+        before = a3mod.launch_count()
+        g.launch()
+        side.synchronize()
+        assert a3mod.launch_count() - before == g.kernels
+        assert torch.equal(Kg, K) and torch.equal(Vg, V) and torch.equal(og["x"], out["x"]) and torch.equal(og["rows"], out["rows"])
+        assert torch.equal(og["scores"], out["scores"])
+        # other embeddings in the same buffer: the replay must follow them like a fresh call does
+        x_saved = s.dx0.clone()
+        s.dx0.copy_((s.dx0.float() * -0.5).to(torch.bfloat16))
+        g.launch()
+        side.synchronize()
+        xg, rg = og["x"].clone(), og["rows"].clone()
+        s.eng.fuse_request(rq)
+        side.synchronize()
+        assert torch.equal(og["x"], xg) and torch.equal(og["rows"], rg)
+        assert not torch.equal(xg, out["x"])
+        s.dx0.copy_(x_saved)
+        g.close()
+    assert s.eng.device_status() == 0
+    s.eng.close()
