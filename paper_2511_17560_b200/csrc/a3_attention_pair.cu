@@ -6,14 +6,18 @@
 // under the other's MMAs:
 //
 //   warp 0 (one lane)   TMA producer: K and V tiles, two stages each
-//   warp 1 (one lane)   tcgen05.mma: S_A = Q_A K^T, S_B = Q_B K^T, O_A += P_A V, O_B += P_B V.  P_X is read from
-//                       tensor memory, where it lies over the first half of S_X, so S_X of the next key tile is
-//                       issued after P_X V of the current one.  P V goes in two halves of 64 keys: the first is
-//                       issued as soon as its P is stored, under the softmax of the second
+//   warps 1 and 10      (one lane each; warp 1 row tile A, warp 10 row tile B: one thread cannot issue the 24
+//                       instructions per key tile and row tile fast enough for both) tcgen05.mma: S_A = Q_A K^T, S_B = Q_B K^T, O_A += P_A V, O_B += P_B V, everything in halves
+//                       of 64 keys.  P of a half is read from tensor memory, where it lies over the first 32 columns
+//                       of that half's own logits; a half's P V is issued as soon as its P is stored, and right
+//                       behind it the same half of S_X for the NEXT key tile (those columns are free from then on),
+//                       so the softmax warps find their next logits waiting: the first half of tile t+1 is computed
+//                       under the softmax of the second half of tile t, the second half under that of the first
 //   warps 2..5          softmax of row tile A, one thread per row (exponent reference, row sum, rescale as in
 //                       a3_attention.cu; the 128 logits of a row are taken in two halves of 64)
 //   warps 6..9          the same for row tile B
-// Tensor memory (512 columns): S_A at 0, S_B at 128, O_A at 256, O_B at 384.  Head dimension 128 only; rows sorted
+// Tensor memory (512 columns): S_A at 0 (keys 0..63 in columns 0..63, keys 64..127 in 64..127), S_B at 128, O_A at 256,
+// O_B at 384.  Head dimension 128 only; rows sorted
 // by position, so B (the later rows) sees at least as many key tiles as A.  Every wait is bounded.
 #include <cuda.h>
 
@@ -22,8 +26,9 @@
 
 namespace a3 {
 
-constexpr int AT2_THREADS = 320;
+constexpr int AT2_THREADS = 352;  // warp 0 TMA, warp 1 MMA of row tile A, warps 2..9 softmax, warp 10 MMA of row tile B
 constexpr int AT2_D = 128;
+constexpr int POLY_EVERY = 4;  // every POLY_EVERY-th pair of exponentials goes to the FMA pipe (0: none)
 
 struct At2Layout {
   static constexpr int SUB = 128 * 64 * 2;  // one [128][64] bf16 sub-tile: 16 KiB
@@ -85,14 +90,14 @@ attention_pair_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_cons
   auto k_empty = [&](int s) { return bars + 8u * (2 + s); };
   auto v_full = [&](int s) { return bars + 8u * (4 + s); };
   auto v_empty = [&](int s) { return bars + 8u * (6 + s); };
-  auto s_full = [&](int x) { return bars + 8u * (8 + x); };
+  auto s_full = [&](int x, int hh) { return bars + 8u * (hh == 0 ? 8 + x : 19 + x); };  // logits of half hh of S_X are in tensor memory
   auto p_ready = [&](int x) { return bars + 8u * (10 + x); };
   auto pv_done = [&](int x) { return bars + 8u * (12 + x); };
   const uint32_t q_ready = bars + 8u * 14;
   auto p0_ready = [&](int x) { return bars + 8u * (15 + x); };  // P of the first 64 keys is in tensor memory
   auto pv0_done = [&](int x) { return bars + 8u * (17 + x); };  // ... and its P V has completed
-  volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(base_ptr + L::BAR_OFF + 8 * 19);
-  volatile int* abort_flag = reinterpret_cast<volatile int*>(base_ptr + L::BAR_OFF + 8 * 19 + 8);
+  volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(base_ptr + L::BAR_OFF + 8 * 21);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(base_ptr + L::BAR_OFF + 8 * 21 + 8);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int G = Hq / Hkv;
@@ -110,10 +115,11 @@ attention_pair_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_cons
   if (threadIdx.x == 0) {
     for (int i = 0; i < 2; ++i) {
       mbar_init(k_full(i), 1);
-      mbar_init(k_empty(i), 1);
+      mbar_init(k_empty(i), 2);  // one arrival per MMA thread
       mbar_init(v_full(i), 1);
-      mbar_init(v_empty(i), 1);
-      mbar_init(s_full(i), 1);
+      mbar_init(v_empty(i), 2);
+      mbar_init(s_full(i, 0), 1);
+      mbar_init(s_full(i, 1), 1);
       mbar_init(p_ready(i), 128);
       mbar_init(pv_done(i), 1);
       mbar_init(p0_ready(i), 128);
@@ -162,28 +168,30 @@ attention_pair_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_cons
         }
       }
     }
-  } else if (warp == 1) {
-    // ---------------- MMA issuer
+  } else if (warp == 1 || warp == 10) {
+    // ---------------- MMA issuers: this thread owns row tile x; K and V stages are released by both threads
     if (lane == 0) {
-      constexpr uint32_t idesc_s = idesc(ATC_BN, 0);
+      const int x = warp == 1 ? 0 : 1;
+      constexpr uint32_t idesc_s = idesc(ATC_BN / 2, 0);
       constexpr uint32_t idesc_o = idesc(D, 1);
-      uint32_t it = 0, qn = 0, cx[2] = {0, 0};  // running key tile; items; tiles done per row tile (barrier phases)
-      auto issue_s = [&](int x, uint32_t kstage) {
-        const uint32_t sq = base + L::Q_OFF + x * L::TILE, sk = base + L::K_OFF + kstage * L::TILE;
+      uint32_t it = 0, qn = 0, cx = 0;  // running key tile; items; tiles this row tile has done (barrier phases)
+      // logits of 64 keys (half hh of the key tile in K stage `kstage`)
+      auto issue_s = [&](int hh, uint32_t kstage) {
+        const uint32_t sq = base + L::Q_OFF + x * L::TILE, sk = base + L::K_OFF + kstage * L::TILE + hh * (64 * 128);
 #pragma unroll
         for (int k = 0; k < D / 16; ++k) {
           const uint32_t sub = (k / 4) * L::SUB + (k % 4) * 32;
-          mma_f16(tmem_base + x * 128, desc_k_sw128(sq + sub), desc_k_sw128(sk + sub), idesc_s, k != 0);
+          mma_f16(tmem_base + x * 128 + hh * 64, desc_k_sw128(sq + sub), desc_k_sw128(sk + sub), idesc_s, k != 0);
         }
-        commit(s_full(x));
+        commit(s_full(x, hh));
       };
-      // P V in two halves of 64 keys: the first is issued as soon as its P is there, under the softmax of the second
-      auto issue_pv_half = [&](int x, int hh, uint32_t vstage, bool first) {
+      // P V of 64 keys: P of half hh lies over the first 32 columns of that half of S_X
+      auto issue_pv_half = [&](int hh, uint32_t vstage, bool first) {
         const uint32_t sv = base + L::V_OFF + vstage * L::TILE;
 #pragma unroll
         for (int k = 4 * hh; k < 4 * hh + 4; ++k) {
           const uint64_t db = desc_mn_sw128(sv + k * 16 * 128, L::SUB);
-          mma_f16_ts(tmem_base + 256 + x * 128, tmem_base + x * 128 + k * 8, db, idesc_o, !(first && k == 0));
+          mma_f16_ts(tmem_base + 256 + x * 128, tmem_base + x * 128 + hh * 64 + (k - 4 * hh) * 8, db, idesc_o, !(first && k == 0));
         }
         commit(hh == 0 ? pv0_done(x) : pv_done(x));
       };
@@ -192,6 +200,7 @@ attention_pair_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_cons
         const int i = item_index(r);
         if (i < 0) continue;
         const At2Item w = at2_item(i, pos, M, G, Hkv, kv_len, row_tiles, n_pairs);
+        const int nkt = w.nkt[x];
         ok = mbar_wait(q_ready, qn & 1, abort_flag, status);
         ++qn;
         if (!ok) break;
@@ -199,47 +208,58 @@ attention_pair_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_cons
         ok = mbar_wait(k_full(it & 1), (it >> 1) & 1, abort_flag, status);
         if (!ok) break;
         fence_after();
-        if (w.nkt[0] > 0) issue_s(0, it & 1);
-        if (w.nkt[1] > 0) issue_s(1, it & 1);
-        commit(k_empty(it & 1));
+        if (nkt > 0) {
+          issue_s(0, it & 1);
+          issue_s(1, it & 1);
+          commit(k_empty(it & 1));
+        } else {
+          mbar_arrive(k_empty(it & 1));
+        }
         for (int t = 0; t < w.T && ok; ++t, ++it) {
           const bool more = t + 1 < w.T;
-          const uint32_t vs = it & 1, vph = (it >> 1) & 1;
-          bool v_here = false;
-          if (t < w.nkt[0]) {
-            ok = mbar_wait(p0_ready(0), cx[0] & 1, abort_flag, status) && mbar_wait(v_full(vs), vph, abort_flag, status);
-            if (!ok) break;
-            v_here = true;
-            fence_after();
-            issue_pv_half(0, 0, vs, t == 0);
-            ok = mbar_wait(p_ready(0), cx[0] & 1, abort_flag, status);
+          const uint32_t vs = it & 1, vph = (it >> 1) & 1, kn = (it + 1) & 1, kph = ((it + 1) >> 1) & 1;
+          if (t < nkt) {
+            const bool next = t + 1 < nkt;
+            // halves in key order.  Each P V is followed by the same half of the next key tile's logits: P V has read
+            // the columns they go to, and the pipe runs this thread's instructions in order.
+            ok = mbar_wait(p0_ready(x), cx & 1, abort_flag, status) && mbar_wait(v_full(vs), vph, abort_flag, status);
             if (!ok) break;
             fence_after();
-            issue_pv_half(0, 1, vs, t == 0);
-            ++cx[0];
-          }
-          if (more) {
-            ok = mbar_wait(k_full((it + 1) & 1), ((it + 1) >> 1) & 1, abort_flag, status);
+            issue_pv_half(0, vs, t == 0);
+            if (next) {
+              ok = mbar_wait(k_full(kn), kph, abort_flag, status);
+              if (!ok) break;
+              fence_after();
+              issue_s(0, kn);
+            }
+            ok = mbar_wait(p_ready(x), cx & 1, abort_flag, status);
             if (!ok) break;
             fence_after();
-            if (t + 1 < w.nkt[0]) issue_s(0, (it + 1) & 1);  // follows P_A V of this tile: P_A lies over S_A
-          }
-          if (t < w.nkt[1]) {
-            ok = mbar_wait(p0_ready(1), cx[1] & 1, abort_flag, status);
-            if (ok && !v_here) ok = mbar_wait(v_full(vs), vph, abort_flag, status);
+            issue_pv_half(1, vs, t == 0);
+            if (next) issue_s(1, kn);
+            ++cx;
+            commit(v_empty(vs));
+            if (more) {
+              if (next) {
+                commit(k_empty(kn));
+              } else {
+                // this row tile is done, the other walks on: its stages still need this thread's arrival, and an
+                // arrival must not run ahead of the stage's use (it would be counted in the wrong phase): wait
+                // until the tile has landed
+                ok = mbar_wait(k_full(kn), kph, abort_flag, status);
+                if (!ok) break;
+                mbar_arrive(k_empty(kn));
+              }
+            }
+          } else {
+            ok = mbar_wait(v_full(vs), vph, abort_flag, status);
             if (!ok) break;
-            fence_after();
-            issue_pv_half(1, 0, vs, t == 0);
-            ok = mbar_wait(p_ready(1), cx[1] & 1, abort_flag, status);
-            if (!ok) break;
-            fence_after();
-            issue_pv_half(1, 1, vs, t == 0);
-            ++cx[1];
-          }
-          commit(v_empty(vs));
-          if (more) {
-            if (t + 1 < w.nkt[1]) issue_s(1, (it + 1) & 1);
-            commit(k_empty((it + 1) & 1));
+            mbar_arrive(v_empty(vs));
+            if (more) {
+              ok = mbar_wait(k_full(kn), kph, abort_flag, status);
+              if (!ok) break;
+              mbar_arrive(k_empty(kn));
+            }
           }
         }
       }
@@ -294,9 +314,9 @@ attention_pair_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_cons
       float m_ref = 0.f, l_run = 0.f;
       for (int t = 0; t < nkt; ++t, ++cxx) {
         // the result of every wait is made warp-uniform: tcgen05.ld/st are warp-wide instructions
-        ok = __all_sync(0xffffffffu, mbar_wait(s_full(x), cxx & 1, abort_flag, status));
+        ok = __all_sync(0xffffffffu, mbar_wait(s_full(x, 0), cxx & 1, abort_flag, status));
         if (!ok) break;
-        fence_after();  // also: every earlier MMA of this row tile, P V of the previous key tile included, is complete
+        fence_after();  // the first half of the logits is there (and the first-half P V of the previous key tile is complete)
         const int key0 = t * ATC_BN;
         const bool need_mask = key0 + ATC_BN - 1 > w.minpos[x];
         float xv[64];
@@ -326,8 +346,24 @@ attention_pair_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_cons
 #pragma unroll
             for (int e = 0; e < 64; e += 2) {
               const float2 v = __ffma2_rn(make_float2(xv[e], xv[e + 1]), sc2, nr2);
-              xv[e] = ex2_approx(v.x);
-              xv[e + 1] = ex2_approx(v.y);
+              if (POLY_EVERY > 0 && ((e >> 1) % POLY_EVERY) == POLY_EVERY - 1) {
+                // 2^v on the FMA pipe (the exponential unit, 16 results per clock and SM, is what bounds two row
+                // tiles per CTA): v = n + f, n integer, |f| <= 1/2; 2^f by a cubic (2e-4 relative, a tenth of the
+                // bf16 step of P), 2^n by an add into the exponent field
+                const float2 vc = make_float2(fmaxf(v.x, -125.f), fmaxf(v.y, -125.f));
+                const float2 magic = make_float2(12582912.f, 12582912.f), nmagic = make_float2(-12582912.f, -12582912.f);
+                const float2 tt = __fadd2_rn(vc, magic);
+                const float2 rr = __fadd2_rn(tt, nmagic);
+                const float2 ff = __fadd2_rn(vc, make_float2(-rr.x, -rr.y));
+                float2 pp = __ffma2_rn(make_float2(0.054848004f, 0.054848004f), ff, make_float2(0.24180661f, 0.24180661f));
+                pp = __ffma2_rn(pp, ff, make_float2(0.69324821f, 0.69324821f));
+                pp = __ffma2_rn(pp, ff, make_float2(0.99998868f, 0.99998868f));
+                xv[e] = __int_as_float(__float_as_int(pp.x) + (__float_as_int(tt.x) << 23));
+                xv[e + 1] = __int_as_float(__float_as_int(pp.y) + (__float_as_int(tt.y) << 23));
+              } else {
+                xv[e] = ex2_approx(v.x);
+                xv[e + 1] = ex2_approx(v.y);
+              }
               s2[(e >> 1) & 1] = __fadd2_rn(s2[(e >> 1) & 1], make_float2(xv[e], xv[e + 1]));
             }
             ls[0] = s2[0].x, ls[1] = s2[0].y, ls[2] = s2[1].x, ls[3] = s2[1].y;
@@ -339,7 +375,7 @@ attention_pair_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_cons
           ld32(ts + h * 64 + 32, xv + 32);
           wait_ld();
         };
-        // multiplies this row of O_X by f (all earlier P V are complete, see the fence above)
+        // multiplies this row of O_X by f (the caller has waited for every P V issued so far)
         auto rescale_output = [&](float f) {
 #pragma unroll 1
           for (int c = 0; c < D / 32; ++c) {
@@ -354,6 +390,9 @@ attention_pair_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_cons
         };
         if (t == 0) {
           // the reference is the true maximum of the first tile
+          ok = __all_sync(0xffffffffu, mbar_wait(s_full(x, 1), cxx & 1, abort_flag, status));
+          if (!ok) break;
+          fence_after();
           load64(0);
           float mx = row_max64(key0);
           load64(1);
@@ -379,6 +418,12 @@ attention_pair_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_cons
         float l_tile = 0.f;
 #pragma unroll 1
         for (int h = 0; h < 2; ++h) {
+          if (h == 1) {
+            // the second half of the logits (issued behind the second-half P V of the previous key tile)
+            ok = __all_sync(0xffffffffu, mbar_wait(s_full(x, 1), cxx & 1, abort_flag, status));
+            if (!ok) break;
+            fence_after();
+          }
           load64(h);
           float lsum = to_probabilities(key0 + 64 * h);
           // A logit far above the reference shows in the sum; anything below 2^16 is harmless.  Above it - rare -
@@ -392,26 +437,27 @@ attention_pair_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_cons
             m_ref += raise;
             l_run *= f;
             l_tile *= f;
-            if (h == 1) {
-              // the first half's P V was released under the old reference: once it has completed, the output holds
-              // its contribution too and the factor applies to all of it
-              ok = __all_sync(0xffffffffu, mbar_wait(pv0_done(x), cxx & 1, abort_flag, status));
-              if (!ok) break;
-              fence_after();
-            }
+            // Every P V issued so far must have landed in the output before it is rescaled.  In the first half the
+            // last one is the second-half P V of the previous key tile; in the second half it is this tile's
+            // first-half P V, released under the old reference: once it has completed, the output holds its
+            // contribution too and the factor applies to all of it.  (Older ones are complete: the pipe runs in order.)
+            ok = __all_sync(0xffffffffu, h == 1 ? mbar_wait(pv0_done(x), cxx & 1, abort_flag, status)
+                                                : mbar_wait(pv_done(x), (cxx - 1) & 1, abort_flag, status));
+            if (!ok) break;
+            fence_after();
             rescale_output(f);
             load64(h);
             lsum = to_probabilities(key0 + 64 * h);
           }
           l_tile += lsum;
-          // P of this half as bf16 pairs: 32 columns at 32 h of S_X (columns whose logits are in registers or done)
+          // P of this half as bf16 pairs: the first 32 columns of this half of S_X (its logits are in registers)
           uint32_t pk[32];
 #pragma unroll
           for (int j = 0; j < 8; ++j) {
             const uint4 v = pack8(xv + 8 * j);
             pk[4 * j] = v.x, pk[4 * j + 1] = v.y, pk[4 * j + 2] = v.z, pk[4 * j + 3] = v.w;
           }
-          st32(ts + 32 * h, reinterpret_cast<const float*>(pk));
+          st32(ts + 64 * h, reinterpret_cast<const float*>(pk));
           if (h == 0) {
             wait_st();
             fence_before();
