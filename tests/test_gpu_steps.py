@@ -748,3 +748,39 @@ def test_residual_persistent_pair_kernel_matches_tile_kernel(a3mod, shape, M):
     Xo, parts = O.recompute_layer(X.astype(np.float64), pos, weights[layer], model, Ko, Vo, rnd=O.round_bf16, return_parts=True)
     check_kv(f64(outs[2]), parts["x_exact"], "hidden rows", scale=2.0 * float(parts["x_exact"].std()))
     eng.close()
+
+
+@pytest.mark.parametrize("shape", [W.TINY_G7, W.TINY_GQA])
+def test_persistent_gemms_row_count_sweep(a3mod, shape):
+    """Row counts around every boundary of the persistent CTA-pair GEMMs (one row, token tiles of 16, one full tile of
+    256, one row more, several tiles, several units per pair): SwiGLU and both residual GEMMs forced onto them, against
+    the tile kernels, bit for bit; no device status bit, no non-finite value."""
+    import ctypes
+    m = shape
+    eng, layers, dev = make_engine(a3mod, m, seed=71, w_std=0.05, max_pos=3000)
+    lib = a3mod._load()
+    lib.a3_internal_set_swiglu_pair.argtypes = [ctypes.c_int]
+    lib.a3_internal_set_residual_t.argtypes = [ctypes.c_int]
+    kv_len = 2600
+    layer = m.n_layers - 1
+    g = torch.Generator(device=dev)
+    try:
+        for M in (1, 2, 15, 16, 17, 33, 127, 128, 129, 255, 256, 257, 511, 513, 767, 1025, 1300):
+            g.manual_seed(M)
+            pos = torch.sort(torch.randperm(kv_len, device=dev, generator=g)[:M]).values.to(torch.int32)
+            X0 = torch.randn((M, m.d_model), device=dev, generator=g).to(torch.bfloat16)
+            K = torch.randn((kv_len, m.n_kv_heads, m.head_dim), device=dev, generator=g).to(torch.bfloat16)
+            outs = []
+            for sw, rs in ((1, 2), (0, 0)):
+                lib.a3_internal_set_swiglu_pair(sw)
+                lib.a3_internal_set_residual_t(rs)
+                X, Kc, Vc = X0.clone(), K.clone(), K.clone()
+                eng.recompute_layer(layer, X, pos, Kc, Vc)
+                assert eng.device_status() == 0, M
+                outs.append(X)
+            assert torch.isfinite(outs[0].float()).all(), M
+            assert torch.equal(outs[0], outs[1]), M
+    finally:
+        lib.a3_internal_set_swiglu_pair(1)
+        lib.a3_internal_set_residual_t(1)
+    eng.close()
