@@ -9,7 +9,7 @@ and the recompute layers) on synthetic inputs of the configured shape.  One JSON
 N > 1 runs N independent replicas (one process per GPU, launched with torch.distributed.run); the path has no
 exchange step, so there is no data-path collective: only the barrier and the max-over-ranks of the time.
 `--impl reference` times the CPU oracle (as it stands, fp32) on the host cores on a bounded sample of the same
-workload.
+workload.  `--config llama8b_batch16` times the batched-serving workload (16 requests, `a3_fuse_batch`) instead.
 """
 from __future__ import annotations
 
@@ -263,6 +263,100 @@ def precompute_chunks(eng, m, r, x0, dev):
         ck.append(K)
         cv.append(V)
     return ck, cv
+
+
+def run_a3_batch(args):
+    """Batched serving (16 requests over a pool of 200 precomputed chunks, Llama-shaped): `a3_fuse_batch` timed as one
+    step; aggregate context tokens per second and the spread of the single-request latencies.  Context, not the
+    headline: one JSON line of the same shape, `config.workload` = llama8b_batch16."""
+    import torch
+    from paper_2511_17560_b200 import a3
+    from paper_2511_17560_b200 import workloads as W
+
+    rank, world, local = dist_setup(args.gpus)
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    peaks, _ = load_peaks()
+    m = W.LLAMA8B
+    if args.layers:
+        from dataclasses import replace
+        m = replace(m, n_layers=args.layers)
+    pool_lens, reqs = W.batched_requests(seed=0)
+    n_max = max(sum(pool_lens[i] for i in ids) + nq for ids, nq in reqs)
+    eng = a3.A3(m, W.make_weights_device(m, dev, seed=0), n_max + 8)
+    torch.cuda.synchronize()
+    stream = torch.cuda.Stream()
+    torch.cuda.set_stream(stream)
+    pool = {}
+    for i in sorted({i for ids, _ in reqs for i in ids}):  # only the pool chunks some request uses are prefilled
+        t = pool_lens[i]
+        x = W.make_embeddings_device(m, t, dev, 0, stream=1000 + i)
+        K = torch.zeros((m.n_layers, t, m.n_kv_heads, m.head_dim), dtype=torch.bfloat16, device=dev)
+        V = torch.zeros_like(K)
+        eng.precompute_chunk(x.clone(), K, V)
+        pool[i] = (K, V, x)
+    batch, keep, n_ctx_total, rows_total, flops_total = [], [], 0, 0, 0.0
+    for j, (ids, nq) in enumerate(reqs):
+        lens = tuple(pool_lens[i] for i in ids)
+        r = W.RequestShape(lens, nq, 0.15, 1)
+        xq = W.make_embeddings_device(m, nq, dev, 0, stream=5000 + j)
+        x0 = torch.cat([pool[i][2] for i in ids] + [xq]).contiguous()
+        tab = a3.chunk_table([pool[i][0] for i in ids], [pool[i][1] for i in ids], r.offsets)
+        K = torch.zeros((m.n_layers, r.n, m.n_kv_heads, m.head_dim), dtype=torch.bfloat16, device=dev)
+        V = torch.zeros_like(K)
+        req, out = eng.make_request(tab, len(ids), max(lens), r.n_ctx, nq, x0, K, V, ratio=0.15, select_layer=1)
+        batch.append((req, out, r))
+        keep.append((x0, tab, K, V))
+        n_ctx_total += r.n_ctx
+        rows_total += out["p"] + nq
+    reqs_c = [b[0] for b in batch]
+    for _ in range(max(args.warmup, 3)):
+        eng.fuse_batch(reqs_c)
+    torch.cuda.synchronize()
+    assert eng.device_status() == 0, "device status word set during warm-up"
+    for req, out, r in batch:
+        flops, _ = algorithmic_work(m, r, out["p"], out["rows"].cpu().numpy())
+        flops_total += sum(flops.values())
+    a3.launch_count(reset=True)
+    sampler = ClockSampler(local) if rank == 0 else None
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    torch.cuda.synchronize()
+    e0.record(stream)
+    for _ in range(args.steps):
+        eng.fuse_batch(reqs_c)
+    e1.record(stream)
+    torch.cuda.synchronize()
+    barrier()
+    seconds = max_over_ranks(e0.elapsed_time(e1) / 1e3, dev)
+    gpu_launches = a3.launch_count(reset=True)
+    clocks = sampler.stop() if sampler else None
+    assert eng.device_status() == 0, "device status word set during the timed region"
+    lat = []
+    for req, out, r in batch:  # each request alone, for the latency spread
+        eng.fuse_request(req)
+        torch.cuda.synchronize()
+        e0.record(stream)
+        eng.fuse_request(req)
+        e1.record(stream)
+        torch.cuda.synchronize()
+        lat.append(e0.elapsed_time(e1))
+    if rank == 0:
+        lat_s = sorted(lat)
+        line = {"metric": METRIC, "value": aggregate_value(n_ctx_total, args.steps, world, seconds), "unit": UNIT, "n_gpus": world,
+                "steps": args.steps, "warmup": max(args.warmup, 3), "ms_per_step": seconds / args.steps * 1e3, "higher_is_better": True,
+                "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+                "config": {"workload": "llama8b_batch16", "model": m.name, "requests": len(batch), "pool_chunks": len(pool_lens),
+                           "pool_chunks_used": len(pool), "n_ctx_total": n_ctx_total, "rows_recomputed_total": rows_total,
+                           "recompute_ratio": 0.15, "select_layer": 1, "replicas": world, "layers": m.n_layers,
+                           "timed_call": "a3_fuse_batch (16 requests, one step)",
+                           "l2": "inputs larger than L2: every request streams the stack's weights and its fused cache"},
+                "request_latency_ms": {"min": lat_s[0], "median": lat_s[len(lat_s) // 2], "max": lat_s[-1]},
+                "algorithmic_tflop_per_step": flops_total / 1e12,
+                "step_frac_of_sustained_peak": flops_total / (seconds / args.steps) / 1e12 / peaks["bf16_tflops_sustained"],
+                "gpu_launches": int(gpu_launches), "clocks": clocks}
+        print(json.dumps(line), flush=True)
+    eng.close()
 
 
 def run_a3(args):
@@ -535,7 +629,10 @@ def main():
     if args.impl == "reference":
         run_reference(args)
     else:
-        run_a3(args)
+        if args.config == "llama8b_batch16":
+            run_a3_batch(args)
+        else:
+            run_a3(args)
 
 
 if __name__ == "__main__":
