@@ -28,7 +28,6 @@ namespace a3 {
 
 constexpr int AT2_THREADS = 352;  // warp 0 TMA, warp 1 MMA of row tile A, warps 2..9 softmax, warp 10 MMA of row tile B
 constexpr int AT2_D = 128;
-constexpr int POLY_EVERY = 4;  // every POLY_EVERY-th pair of exponentials goes to the FMA pipe (0: none)
 
 struct At2Layout {
   static constexpr int SUB = 128 * 64 * 2;  // one [128][64] bf16 sub-tile: 16 KiB
@@ -346,20 +345,12 @@ attention_pair_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_cons
 #pragma unroll
             for (int e = 0; e < 64; e += 2) {
               const float2 v = __ffma2_rn(make_float2(xv[e], xv[e + 1]), sc2, nr2);
-              if (POLY_EVERY > 0 && ((e >> 1) % POLY_EVERY) == POLY_EVERY - 1) {
-                // 2^v on the FMA pipe (the exponential unit, 16 results per clock and SM, is what bounds two row
-                // tiles per CTA): v = n + f, n integer, |f| <= 1/2; 2^f by a cubic (2e-4 relative, a tenth of the
-                // bf16 step of P), 2^n by an add into the exponent field
-                const float2 vc = make_float2(fmaxf(v.x, -125.f), fmaxf(v.y, -125.f));
-                const float2 magic = make_float2(12582912.f, 12582912.f), nmagic = make_float2(-12582912.f, -12582912.f);
-                const float2 tt = __fadd2_rn(vc, magic);
-                const float2 rr = __fadd2_rn(tt, nmagic);
-                const float2 ff = __fadd2_rn(vc, make_float2(-rr.x, -rr.y));
-                float2 pp = __ffma2_rn(make_float2(0.054848004f, 0.054848004f), ff, make_float2(0.24180661f, 0.24180661f));
-                pp = __ffma2_rn(pp, ff, make_float2(0.69324821f, 0.69324821f));
-                pp = __ffma2_rn(pp, ff, make_float2(0.99998868f, 0.99998868f));
-                xv[e] = __int_as_float(__float_as_int(pp.x) + (__float_as_int(tt.x) << 23));
-                xv[e + 1] = __int_as_float(__float_as_int(pp.y) + (__float_as_int(tt.y) << 23));
+              if (ATC_POLY_EVERY > 0 && ((e >> 1) % ATC_POLY_EVERY) == ATC_POLY_EVERY - 1) {
+                // on the FMA pipe: with both row tiles' softmax running all the time the exponential unit (16 results
+                // per clock and SM = 2 048 clocks per key tile) is the bound
+                const float2 p2 = exp2_poly2(v);
+                xv[e] = p2.x;
+                xv[e + 1] = p2.y;
               } else {
                 xv[e] = ex2_approx(v.x);
                 xv[e + 1] = ex2_approx(v.y);

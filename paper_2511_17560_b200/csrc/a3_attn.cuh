@@ -124,6 +124,23 @@ __host__ __device__ constexpr uint32_t idesc(int n, int b_mn) {
 __device__ __forceinline__ uint32_t swz(int r, int j) { return (uint32_t)(r * 128 + ((j ^ (r & 7)) << 4)); }
 }  // namespace atc
 
+// 2^v for a pair on the FMA pipe: v = n + f with n integer and |f| <= 1/2 (magic-number rounding), 2^f by a cubic
+// (2e-4 relative, a tenth of the bf16 step of P), 2^n by an add into the exponent field.  Inputs below -125 are
+// clamped (the result is then 2^-125, i.e. nothing); -inf must not be passed (masked logits take ex2.approx).
+// Every ATC_POLY_EVERY-th pair of exponentials of an unmasked tile goes this way: the exponential unit delivers 16
+// results per clock and SM and paces the softmax warps (measured: 1 300 of their 2 100 clocks per key tile).
+constexpr int ATC_POLY_EVERY = 4;
+__device__ __forceinline__ float2 exp2_poly2(float2 v) {
+  const float2 vc = make_float2(fmaxf(v.x, -125.f), fmaxf(v.y, -125.f));
+  const float2 tt = __fadd2_rn(vc, make_float2(12582912.f, 12582912.f));
+  const float2 rr = __fadd2_rn(tt, make_float2(-12582912.f, -12582912.f));
+  const float2 ff = __fadd2_rn(vc, make_float2(-rr.x, -rr.y));
+  float2 pp = __ffma2_rn(make_float2(0.054848004f, 0.054848004f), ff, make_float2(0.24180661f, 0.24180661f));
+  pp = __ffma2_rn(pp, ff, make_float2(0.69324821f, 0.69324821f));
+  pp = __ffma2_rn(pp, ff, make_float2(0.99998868f, 0.99998868f));
+  return make_float2(__int_as_float(__float_as_int(pp.x) + (__float_as_int(tt.x) << 23)),
+                     __int_as_float(__float_as_int(pp.y) + (__float_as_int(tt.y) << 23)));
+}
 __device__ __forceinline__ float ex2_approx(float x) {
   float y;
   asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
