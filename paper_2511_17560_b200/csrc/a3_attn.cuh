@@ -125,13 +125,15 @@ __device__ __forceinline__ uint32_t swz(int r, int j) { return (uint32_t)(r * 12
 }  // namespace atc
 
 // 2^v for a pair on the FMA pipe: v = n + f with n integer and |f| <= 1/2 (magic-number rounding), 2^f by a cubic
-// (2e-4 relative, a tenth of the bf16 step of P), 2^n by an add into the exponent field.  Inputs below -125 are
-// clamped (the result is then 2^-125, i.e. nothing); -inf must not be passed (masked logits take ex2.approx).
+// (2e-4 relative, a tenth of the bf16 step of P), 2^n by an add into the exponent field.  Inputs are clamped to
+// [-125, 126]: below, the result is 2^-125, i.e. nothing; above, it is 2^126, which the row sum's overflow guard
+// catches like the +inf of ex2.approx (an unclamped exponent would wrap around and could go unnoticed); -inf must
+// not be passed (masked logits take ex2.approx).
 // Every ATC_POLY_EVERY-th pair of exponentials of an unmasked tile goes this way: the exponential unit delivers 16
 // results per clock and SM and paces the softmax warps (measured: 1 300 of their 2 100 clocks per key tile).
 constexpr int ATC_POLY_EVERY = 4;
 __device__ __forceinline__ float2 exp2_poly2(float2 v) {
-  const float2 vc = make_float2(fmaxf(v.x, -125.f), fmaxf(v.y, -125.f));
+  const float2 vc = make_float2(fminf(fmaxf(v.x, -125.f), 126.f), fminf(fmaxf(v.y, -125.f), 126.f));
   const float2 tt = __fadd2_rn(vc, make_float2(12582912.f, 12582912.f));
   const float2 rr = __fadd2_rn(tt, make_float2(-12582912.f, -12582912.f));
   const float2 ff = __fadd2_rn(vc, make_float2(-rr.x, -rr.y));

@@ -784,3 +784,57 @@ def test_persistent_gemms_row_count_sweep(a3mod, shape):
         lib.a3_internal_set_swiglu_pair(1)
         lib.a3_internal_set_residual_t(1)
     eng.close()
+
+
+@pytest.mark.parametrize("pair", [False, True])
+def test_attention_logit_spikes(a3mod, pair):
+    """Single keys whose logits tower over everything before them by 300, 600, ... in the exp2 domain (170, 340, ... for the other query head of the group), each in a key tile
+    of its own that no row masks, all at offsets 6 and 7 modulo 8 - the register pairs whose exponential runs on the
+    FMA pipe, where the exponent arithmetic would wrap around for such inputs (and the key, the last one above all,
+    would silently get weight zero) if they were not clamped into the range the overflow guard catches.  Both
+    attention kernels, against the exact softmax of the oracle."""
+    import ctypes
+    m = W.TINY_GQA
+    eng, layers, dev = make_engine(a3mod, m, seed=13, w_std=0.05)
+    lib = a3mod._load()
+    lib.a3_internal_set_attn_pair.argtypes = [ctypes.c_int]
+    model, weights = oracle_model(m), oracle_weights(layers)
+    rng = np.random.default_rng(313)
+    kv_len, M = 1500, 131
+    spikes = [262, 391, 526, 655, 774, 903, 1038]  # one per key tile, all below the first row (no tile of theirs is masked); residues 6, 7, 6, 7, ... modulo 8
+    assert all(p % 8 in (6, 7) for p in spikes)
+    pos = np.sort(rng.choice(np.arange(1200, kv_len), size=M, replace=False))
+    pos[-1] = kv_len - 1
+    assert not set(spikes) & set(pos.tolist())
+    X = W.bf16_round(rng.standard_normal((M, m.d_model), dtype=np.float32))
+    layer = m.n_layers - 1
+    v_dir = rng.standard_normal((m.n_kv_heads, m.head_dim)).astype(np.float32)
+    zero = np.zeros((kv_len, m.n_kv_heads, m.head_dim))
+    q0 = O.recompute_layer(X.astype(np.float64), pos, weights[layer], model, zero.copy(), zero.copy(), rnd=O.round_bf16, return_parts=True)[1]["q"]
+    G0 = m.n_q_heads // m.n_kv_heads
+    slope = max(abs(float(q0[M - 1, h] @ v_dir[h // G0])) for h in range(m.n_q_heads)) / np.sqrt(m.head_dim) * np.log2(np.e)
+    Kc = 0.05 * rng.standard_normal((kv_len, m.n_kv_heads, m.head_dim)).astype(np.float32)
+    for j, p in enumerate(spikes):
+        Kc[p] = (300.0 * (j + 1) / slope) * v_dir
+    Kc = W.bf16_round(Kc)
+    Vc = W.bf16_round(rng.standard_normal((kv_len, m.n_kv_heads, m.head_dim)).astype(np.float32))
+    Ko, Vo = Kc.astype(np.float64), Vc.astype(np.float64)
+    Xo, parts = O.recompute_layer(X.astype(np.float64), pos, weights[layer], model, Ko, Vo, rnd=O.round_bf16, return_parts=True)
+    q = parts["q"]
+    top = max(float(Ko[spikes[-1], h // G0] @ q[M - 1, h]) / np.sqrt(m.head_dim) * np.log2(np.e) for h in range(m.n_q_heads))
+    assert top > 2000  # the last spike of the steepest head really is that far out
+    dX, dpos = to_dev(X, dev), torch.from_numpy(pos.astype(np.int32)).to(dev)
+    dK, dV = to_dev(Kc, dev), to_dev(Vc, dev)
+    lse = torch.empty((M, m.n_q_heads), dtype=torch.float32, device=dev)
+    try:
+        lib.a3_internal_set_attn_pair(1 if pair else 0)
+        eng.recompute_layer(layer, dX, dpos, dK, dV, lse_out=lse)
+    finally:
+        lib.a3_internal_set_attn_pair(-1)
+    assert eng.device_status() == 0
+    gX = f64(dX)
+    assert np.isfinite(gX).all()
+    check_kv(gX, parts["x_exact"], "hidden rows", scale=2.0 * float(parts["x_exact"].std()))
+    lse_tol = 2 * 2.0 ** -9 * float(np.abs(q).max()) * float(np.abs(Kc).max()) / np.sqrt(m.head_dim)
+    np.testing.assert_allclose(lse.cpu().numpy(), parts["lse"], atol=max(5e-3, lse_tol), rtol=1e-5)
+    eng.close()
