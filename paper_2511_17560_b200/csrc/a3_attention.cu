@@ -372,14 +372,8 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
 #pragma unroll
             for (int e = 0; e < 64; e += 2) {
               const float2 t = __ffma2_rn(make_float2(x[e], x[e + 1]), sc2, nr2);
-              if (ATC_POLY_EVERY > 0 && ((e >> 1) % ATC_POLY_EVERY) == ATC_POLY_EVERY - 1) {
-                const float2 p2 = exp2_poly2(t);  // on the FMA pipe: the exponential unit paces this loop
-                x[e] = p2.x;
-                x[e + 1] = p2.y;
-              } else {
-                x[e] = ex2_approx(t.x);
-                x[e + 1] = ex2_approx(t.y);
-              }
+              x[e] = ex2_approx(t.x);
+              x[e + 1] = ex2_approx(t.y);
               s2[(e >> 1) & 1] = __fadd2_rn(s2[(e >> 1) & 1], make_float2(x[e], x[e + 1]));
             }
             ls[0] = s2[0].x, ls[1] = s2[0].y, ls[2] = s2[1].x, ls[3] = s2[1].y;

@@ -129,8 +129,9 @@ __device__ __forceinline__ uint32_t swz(int r, int j) { return (uint32_t)(r * 12
 // [-125, 126]: below, the result is 2^-125, i.e. nothing; above, it is 2^126, which the row sum's overflow guard
 // catches like the +inf of ex2.approx (an unclamped exponent would wrap around and could go unnoticed); -inf must
 // not be passed (masked logits take ex2.approx).
-// Every ATC_POLY_EVERY-th pair of exponentials of an unmasked tile goes this way: the exponential unit delivers 16
-// results per clock and SM and paces the softmax warps (measured: 1 300 of their 2 100 clocks per key tile).
+// The two-row-tile kernel sends every ATC_POLY_EVERY-th pair of exponentials of an unmasked tile this way: with both
+// row tiles' softmax running all the time the exponential unit (16 results per clock and SM) paces it (+3 %).  In
+// the one-tile kernel the gain was inside the noise of the measurement and the path is not used.
 constexpr int ATC_POLY_EVERY = 4;
 __device__ __forceinline__ float2 exp2_poly2(float2 v) {
   const float2 vc = make_float2(fminf(fmaxf(v.x, -125.f), 126.f), fminf(fmaxf(v.y, -125.f), 126.f));
