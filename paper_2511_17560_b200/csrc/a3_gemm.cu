@@ -133,7 +133,7 @@ __device__ __forceinline__ void tc_epilogue_row(const TcParams& p, uint32_t trow
           tc_wait_ld();
           if (row_ok) {
 #pragma unroll
-            for (int e = 0; e < 32; ++e) g[e] = __fdividef(g[e], 1.f + __expf(-g[e])) * u[e];
+            for (int e = 0; e < 32; ++e) g[e] = silu_mul(g[e], u[e]);
             store32_bf16(p.C + (size_t)gr * p.ldc + col, g);
           }
           c8 += 4;
@@ -144,7 +144,7 @@ __device__ __forceinline__ void tc_epilogue_row(const TcParams& p, uint32_t trow
           tc_wait_ld();
           if (row_ok && col + 8 <= p.N) {
 #pragma unroll
-            for (int e = 0; e < 8; ++e) g[e] = __fdividef(g[e], 1.f + __expf(-g[e])) * u[e];
+            for (int e = 0; e < 8; ++e) g[e] = silu_mul(g[e], u[e]);
             *reinterpret_cast<uint4*>(p.C + (size_t)gr * p.ldc + col) = pack8(g);
           }
           c8 += 1;

@@ -303,8 +303,7 @@ pair_t_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ C
           for (int e = 0; e < 32; ++e) {
             const float o = xb[e * SP_FEAT + feat];
             const float g = up_warp ? o : v[e], uv = up_warp ? v[e] : o;
-            // silu(g) * u with the fast exponential and reciprocal (relative error 2^-21, far below the bf16 rounding)
-            const float r = __fdividef(g, 1.f + __expf(-g)) * uv;
+            const float r = silu_mul(g, uv);
             if (e < valid) orow[(size_t)e * p.ldc] = __float2bfloat16_rn(r);
           }
           if (cc + 2 < total_chunks) named_bar_arrive(bar_read + buf, 128);  // nobody waits for the last two

@@ -128,6 +128,16 @@ __host__ __device__ constexpr uint32_t idesc_bf16(int n) {
   return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(TC_BM >> 4) << 24);
 }
 
+// silu(g) * u with the fast exponential and the approximate reciprocal (relative error about 2^-21, far below the
+// bf16 rounding of the result).  Written as g * rcp(1 + e^-g): for g below about -88.7 the exponential overflows to
+// +inf and rcp.approx(+inf) is +0, so the product is the correct -0 (an IEEE division would give the same; the
+// explicit form keeps that case in view).
+__device__ __forceinline__ float silu_mul(float g, float u) {
+  float r;
+  asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(r) : "f"(1.f + __expf(-g)));
+  return g * r * u;
+}
+
 __device__ __forceinline__ void store32_bf16(bf16* dst, const float* f) {
   uint4* d = reinterpret_cast<uint4*>(dst);
 #pragma unroll

@@ -838,3 +838,43 @@ def test_attention_logit_spikes(a3mod, pair):
     lse_tol = 2 * 2.0 ** -9 * float(np.abs(q).max()) * float(np.abs(Kc).max()) / np.sqrt(m.head_dim)
     np.testing.assert_allclose(lse.cpu().numpy(), parts["lse"], atol=max(5e-3, lse_tol), rtol=1e-5)
     eng.close()
+
+
+def test_swiglu_far_negative_gate(a3mod):
+    """Gate pre-activations far below -88.7 (where e^-g overflows fp32): silu(g) u must come out as a signed zero (the
+    kernels use a fast exponential and an approximate reciprocal: inf and NaN must not leak out of that corner); and
+    far above, as g u.  One layer's SwiGLU GEMM alone (tuning hook), both kernels, against the oracle's silu on the
+    same products."""
+    import ctypes
+    m = W.TINY
+    eng, layers, dev = make_engine(a3mod, m, seed=81, w_std=0.05)
+    lib = a3mod._load()
+    lib.a3_internal_set_swiglu_pair.argtypes = [ctypes.c_int]
+    lib.a3_internal_swiglu.argtypes = [ctypes.c_void_p, ctypes.c_int, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int, ctypes.c_void_p]
+    wg, wu = layers[0]["w_gate"].astype(np.float64), layers[0]["w_up"].astype(np.float64)
+    rng = np.random.default_rng(37)
+    M = 70
+    X = rng.standard_normal((M, m.d_model))
+    # rows 0..9 point against gate rows 0..9 (pre-activation about -400), rows 10..19 along rows 10..19 (+400)
+    for i in range(20):
+        X[i] = (-1.0 if i < 10 else 1.0) * 400.0 * wg[i] / float(wg[i] @ wg[i])
+    X = W.bf16_round(X.astype(np.float32))
+    g, u = X.astype(np.float64) @ wg.T, X.astype(np.float64) @ wu.T
+    assert g[np.arange(10), np.arange(10)].max() < -300 and g[np.arange(10, 20), np.arange(10, 20)].min() > 300
+    with np.errstate(over="ignore"):
+        want = O.silu(g) * u
+    dX = to_dev(X, dev)
+    try:
+        for mode in (1, 0):
+            lib.a3_internal_set_swiglu_pair(mode)
+            out = torch.full((M, m.d_ff), float("nan"), dtype=torch.bfloat16, device=dev)
+            st = torch.cuda.current_stream().cuda_stream
+            assert lib.a3_internal_swiglu(eng._h, 0, dX.data_ptr(), out.data_ptr(), M, st) == 0
+            got = f64(out)
+            assert eng.device_status() == 0
+            assert np.isfinite(got).all(), mode
+            np.testing.assert_allclose(got, want, rtol=2.0 ** -7, atol=2e-3)
+            assert np.all(got[np.arange(10), np.arange(10)] == 0.0)
+    finally:
+        lib.a3_internal_set_swiglu_pair(1)
+    eng.close()
