@@ -439,7 +439,7 @@ extern "C" void a3_internal_set_swiglu_pair(int v) { a3::g_swiglu_pair = v; }
 extern "C" void a3_internal_set_residual_t(int v) { a3::g_residual_t = v; }
 
 
-// Tuning hook: the SwiGLU GEMM of one layer alone, out[M][d_ff] = silu(x Wg^T) * (x Wu^T), x [M][d_model].
+// Test hook: the SwiGLU GEMM of one layer alone, out[M][d_ff] = silu(x Wg^T) * (x Wu^T), x [M][d_model].
 extern "C" int a3_internal_swiglu(const a3_handle* h, int layer, const void* x, void* out, int M, void* stream) {
   a3::GemmArgs u{};
   u.A = (const bf16*)x;
@@ -453,16 +453,3 @@ extern "C" int a3_internal_swiglu(const a3_handle* h, int layer, const void* x, 
   return a3::gemm_bf16(h, a3::EPI_SWIGLU, u, (cudaStream_t)stream);
 }
 
-// Tuning hook: one residual GEMM of a layer alone, C[M][d_model] += x W^T; which = 0: output projection (x [M][Hq*D]),
-// 1: MLP down projection (x [M][d_ff]).
-extern "C" int a3_internal_residual(const a3_handle* h, int layer, int which, const void* x, void* c, int M, void* stream) {
-  a3::GemmArgs g{};
-  g.A = (const bf16*)x;
-  g.M = M;
-  g.K = which == 0 ? h->m.n_q_heads * h->m.head_dim : h->m.d_ff;
-  g.nseg = 1;
-  g.seg[0] = {(const bf16*)(which == 0 ? h->layers[layer].wo : h->layers[layer].w_down), nullptr, h->m.d_model, 0};
-  g.C = (bf16*)c;
-  g.ldc = h->m.d_model;
-  return a3::gemm_bf16(h, a3::EPI_RESIDUAL, g, (cudaStream_t)stream);
-}
