@@ -36,7 +36,10 @@ Readings adopted where the paper is silent (stated once here, used throughout):
     the global position (Eq. 2).
 
 Pins (tests marked "not gpu"): RoPE composition / R(0)=I / norm / the D=4 matrix
-written out by hand; layer-0 and chunk-0 exactness of recovered caches against a
+written out by hand; the decoder block (recompute_layer, project_qkv) against a
+2-token d=4 block multiplied out with `math` only and against the Llama and
+Qwen2 decoder layers of the `transformers` package in float64 (keys, values,
+block output, a two-layer stack); layer-0 and chunk-0 exactness of recovered caches against a
 full prefill; r=1 == full prefill; r=0 == position-recovered concatenation;
 softmax rows sum to one; uniform-key closed form; causality; brute-force top-k;
 nested selections; first-token logits against a library matmul and planted rows;
