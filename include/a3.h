@@ -146,6 +146,27 @@ typedef struct {
   void* x_out;                /* host [n_recompute + n_question][d_model] */
 } a3_host_io;
 
+/* Kernel-variant choices of a handle (a3_set_option).  Several steps exist in more than one kernel variant; by
+ * default the launcher picks one from the shape.  These options pin a variant on ONE handle, for cross-checks
+ * (every variant must meet the same tolerances; some pairs are bit-identical) and for measurements.  They are plain
+ * fields of the handle: set them while no call on the handle is in flight. */
+typedef enum {
+  A3_OPT_ATTN_SPLIT = 0,        /* attention, one row tile per CTA: key segments per row tile; 0 = choose (default) */
+  A3_OPT_ATTN_PAIR,             /* two-row-tile attention kernel: -1 choose (default), 0 never, 1 whenever supported */
+  A3_OPT_ATTN_MAX_CTAS,         /* cap on the persistent attention grid; 0 = one CTA per SM (default) */
+  A3_OPT_SWIGLU_NARROW,         /* one-CTA gate/up GEMM: 0 uniform tiles, 1 narrower last wave (default), 16..120 forced width */
+  A3_OPT_SWIGLU_PAIR,           /* persistent CTA-pair gate/up GEMM: 0 never, 1 whenever the shape allows (default) */
+  A3_OPT_RESIDUAL_T,            /* persistent CTA-pair C += A B^T: 0 never, 1 by shape (default), 2 whenever the shape allows */
+  A3_OPT_GEMM_BN_RESIDUAL,      /* tile width of the tile GEMMs per epilogue; 0 = choose; 512 = the 256 x 256 CTA-pair tile */
+  A3_OPT_GEMM_BN_SWIGLU,
+  A3_OPT_GEMM_BN_QKV,
+  A3_OPT_GEMM_STAGES_RESIDUAL,  /* pipeline depth that goes with the width above */
+  A3_OPT_GEMM_STAGES_SWIGLU,
+  A3_OPT_GEMM_STAGES_QKV,
+  A3_OPT_SCORES_KERNEL,         /* relevance scores: 0 choose (default), 1 the tcgen05 kernel, 2 the warp-level MMA kernel */
+  A3_OPT_COUNT
+} a3_option;
+
 /* ---- lifetime ---------------------------------------------------------------------- */
 
 /* Creates a handle on the current device: checks the shape, borrows `layers` (host array
@@ -153,6 +174,10 @@ typedef struct {
  * from float64 angles.  Allocates; not a hot call. */
 int a3_create(a3_handle** out, const a3_model_desc* model, const a3_layer_weights* layers);
 void a3_destroy(a3_handle* h);
+
+/* Sets one a3_option of the handle.  A3_EINVAL for an unknown option; values outside an option's range fall back
+ * to the default behaviour at the launch that reads them.  Host only; no device work. */
+int a3_set_option(a3_handle* h, int option, int value);
 
 /* Bytes of workspace a3_recompute_layer needs for max_rows rows (also enough for
  * a3_query_scores / a3_topk_select on caches up to max_rows slots). */
@@ -176,17 +201,22 @@ int a3_recompute_count(double ratio, int n, int n_candidates);
  *   k_fused[l][dst_offset+t] = R(delta + token_step*t) k_src[l][t]   (rotation per head, fp32 arithmetic)
  *   v_fused[l][dst_offset+t] = v_src[l][t]
  * chunks: dev array; max_chunk_len >= every len (host copy of the largest length, sizes the grid).
- * Fused layer l lives at k_fused + l*layer_stride bytes. */
+ * Fused layer l lives at k_fused + l*layer_stride bytes and has kv_len slots (kv_len rows must fit in
+ * layer_stride).  A chunk whose slots [dst_offset, dst_offset + len) do not lie inside [0, kv_len), whose len
+ * exceeds max_chunk_len, or whose rotation leaves the RoPE table is skipped as a whole - nothing of it is written -
+ * and A3_DEV_BAD_POSITION is set. */
 int a3_rope_rerotate(const a3_handle* h, const a3_chunk_ref* chunks, int n_chunks, int max_chunk_len,
-                     void* k_fused, void* v_fused, uint64_t layer_stride, int layer_begin, int layer_end,
+                     void* k_fused, void* v_fused, uint64_t layer_stride, int kv_len, int layer_begin, int layer_end,
                      a3_stream stream);
 
 /* Relevance scores (Eq. 3): scores[i] = sum over question rows j and query heads h of
  * Softmax_row(q_{j,h} K^T / sqrt(D))[i] for i in [cand_begin, cand_end), 0 for other i < kv_len.
  * Each softmax row runs over slots 0..q_pos[j].  q_rows: dev [nq][Hq][D], already rotated;
- * k_layer: dev [kv_len][Hkv][D].  lse: dev [nq][Hq] natural-log row log-sum-exps of the scaled
- * logits (as a3_recompute_layer emits) or NULL, in which case a statistics pass runs first.
- * The result is deterministic (fixed summation order). */
+ * q_pos: dev [nq], strictly ascending, each in [0, kv_len) (checked on the device: A3_DEV_UNSORTED_ROWS /
+ * A3_DEV_BAD_POSITION).  k_layer: dev [kv_len][Hkv][D].  lse: dev [nq][Hq] natural-log row log-sum-exps of the
+ * scaled logits (as a3_recompute_layer emits) or NULL, in which case a statistics pass runs first (ws then needs
+ * a3_scores_workspace_bytes(h, nq) bytes).  The result is deterministic (fixed summation order). */
+size_t a3_scores_workspace_bytes(const a3_handle* h, int nq);
 int a3_query_scores(const a3_handle* h, const void* q_rows, const int32_t* q_pos, int nq, const void* k_layer,
                     int kv_len, int cand_begin, int cand_end, const float* lse, float* scores, void* ws,
                     size_t ws_bytes, a3_stream stream);
@@ -194,15 +224,18 @@ int a3_query_scores(const a3_handle* h, const void* q_rows, const int32_t* q_pos
 /* a3_query_scores without a workspace, for callers that cannot allocate device memory where they need the
  * scores (for example a serving engine that gave all free HBM to its KV-cache pool at start-up, or plug-in code
  * inside a framework that owns the allocator).  The paper has no counterpart: this is a packaging variant of the
- * call above, with the same arguments minus lse/ws and the same result.  The row log-sum-exps go to a fixed
- * array inside the library image: A3_STATIC_LSE_MAX floats (256 KiB) that every GPU which loads the library
- * holds until the process exits.  nq * n_q_heads above that limit returns A3_ETOOLARGE and launches nothing.
+ * call above, with the same arguments minus lse/ws and the same result, bit for bit.  The row log-sum-exps and
+ * the partial statistics of the pass that computes them go to a fixed array inside the library image:
+ * A3_STATIC_SCRATCH_BYTES (1 MiB: room for A3_STATIC_LSE_MAX log-sum-exps plus 768 KiB of partial statistics) that
+ * every GPU which loads the library holds until the process exits.  nq * n_q_heads above A3_STATIC_LSE_MAX
+ * returns A3_ETOOLARGE and launches nothing.
  * The call makes no allocation of any kind.  Its first call on a device looks up the array's device address
  * (once per device; that device must be current and must be the handle's) and should therefore be made before
  * any stream capture begins.  All calls share the array; it keeps the previous call's contents, and nothing in
  * it needs clearing because each call overwrites the entries it later reads.  Calls whose kernels may overlap
  * on the GPU race on it: order them. */
 #define A3_STATIC_LSE_MAX 65536
+#define A3_STATIC_SCRATCH_BYTES (A3_STATIC_LSE_MAX * 4 + 768 * 1024)
 int a3_query_scores_static(const a3_handle* h, const void* q_rows, const int32_t* q_pos, int nq, const void* k_layer,
                            int kv_len, int cand_begin, int cand_end, float* scores, a3_stream stream);
 
@@ -224,6 +257,11 @@ int a3_recompute_layer(const a3_handle* h, int layer, void* x_rows, const int32_
  * k_rows/v_rows: dev [M][Hkv][D]; slots: dev [M], each in [0, kv_len). */
 int a3_scatter_kv(const a3_handle* h, const void* k_rows, const void* v_rows, const int32_t* slots, int M,
                   void* k_layer, void* v_layer, int kv_len, a3_stream stream);
+
+/* The gate/up half of the feed-forward network (the MLP inside H(.) of Eq. 5) of one layer alone:
+ * out[M][d_ff] = silu(x Wg^T) * (x Wu^T) rounded to bf16, x: dev [M][d_model].  One launch; used to compare the
+ * kernel variants of this GEMM with one another (a3_set_option) and with the oracle. */
+int a3_swiglu_rows(const a3_handle* h, int layer, const void* x, void* out, int M, a3_stream stream);
 
 /* Row gather X[R] (Eq. 4, Q_true[Re, Q]): dst[m] = src[rows[m]], rows of `width` bf16 elements. */
 int a3_gather_rows(const a3_handle* h, const void* src, int n_src, const int32_t* rows, int M, int width,
@@ -267,9 +305,12 @@ int a3_fuse_batch(const a3_handle* h, const a3_request* reqs, int n_requests, vo
 /* a3_fuse_request with the chunk caches and embeddings in HOST memory (pinned memory lets the copies
  * overlap the compute): copies them to `staging` (dev, a3_host_staging_bytes) on a copy stream the
  * handle creates on first use, layer by layer, while `stream` computes; builds the chunk descriptors,
- * fuses, copies rows_out and x_out back to the host and waits for both streams.  Chunk caches of
- * layers up to select_layer are not copied: those layers are recomputed for every row.
- * req->chunks, req->x0 are ignored (taken from io); the fused cache and scores stay on the device. */
+ * fuses, copies rows_out and x_out back to the host and waits for both streams - also when it returns an
+ * error after the first copy was queued, so the host buffers and the staging area are free on return whatever
+ * the status.  Chunk caches of layers up to select_layer are not copied: those layers are recomputed for every
+ * row.  req->chunks, req->x0 are ignored (taken from io); the fused cache and scores stay on the device.
+ * The handle keeps a host copy of the chunk descriptors, grown (realloc) only when a call has more chunks than
+ * any before it. */
 int a3_fuse_request_host(const a3_handle* h, const a3_request* req, const a3_host_io* io, void* staging,
                          size_t staging_bytes, void* ws, size_t ws_bytes, a3_stream stream);
 

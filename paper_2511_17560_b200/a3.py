@@ -63,7 +63,12 @@ class HostIO(C.Structure):
                 ("x0", C.c_void_p), ("rows_out", C.c_void_p), ("x_out", C.c_void_p)]
 
 
-EXPORTS = ("a3_create", "a3_destroy", "a3_layer_workspace_bytes", "a3_request_workspace_bytes", "a3_host_staging_bytes",
+# a3_option (include/a3.h)
+(OPT_ATTN_SPLIT, OPT_ATTN_PAIR, OPT_ATTN_MAX_CTAS, OPT_SWIGLU_NARROW, OPT_SWIGLU_PAIR, OPT_RESIDUAL_T, OPT_GEMM_BN_RESIDUAL,
+ OPT_GEMM_BN_SWIGLU, OPT_GEMM_BN_QKV, OPT_GEMM_STAGES_RESIDUAL, OPT_GEMM_STAGES_SWIGLU, OPT_GEMM_STAGES_QKV,
+ OPT_SCORES_KERNEL, OPT_COUNT) = range(14)
+
+EXPORTS = ("a3_create", "a3_destroy", "a3_set_option", "a3_scores_workspace_bytes", "a3_swiglu_rows", "a3_layer_workspace_bytes", "a3_request_workspace_bytes", "a3_host_staging_bytes",
            "a3_recompute_count", "a3_rope_rerotate", "a3_query_scores", "a3_query_scores_static", "a3_topk_select", "a3_recompute_layer",
            "a3_scatter_kv", "a3_gather_rows", "a3_precompute_chunk", "a3_first_token_workspace_bytes", "a3_first_token",
            "a3_evict_count", "a3_evict_workspace_bytes", "a3_evict_layer", "a3_chunk_edge_rows", "a3_fuse_request", "a3_fuse_batch", "a3_fuse_request_host",
@@ -89,13 +94,15 @@ def _load():
     lib.a3_create.argtypes = [C.POINTER(vp), C.POINTER(ModelDesc), C.POINTER(LayerWeights)]
     lib.a3_destroy.argtypes = [vp]
     lib.a3_destroy.restype = None
-    for name in ("a3_layer_workspace_bytes", "a3_request_workspace_bytes"):
+    lib.a3_set_option.argtypes = [vp, i32, i32]
+    lib.a3_swiglu_rows.argtypes = [vp, i32, vp, vp, i32, vp]
+    for name in ("a3_layer_workspace_bytes", "a3_request_workspace_bytes", "a3_scores_workspace_bytes"):
         getattr(lib, name).argtypes = [vp, i32]
         getattr(lib, name).restype = sz
     lib.a3_host_staging_bytes.argtypes = [vp, i32, i32]
     lib.a3_host_staging_bytes.restype = sz
     lib.a3_recompute_count.argtypes = [C.c_double, i32, i32]
-    lib.a3_rope_rerotate.argtypes = [vp, vp, i32, i32, vp, vp, u64, i32, i32, vp]
+    lib.a3_rope_rerotate.argtypes = [vp, vp, i32, i32, vp, vp, u64, i32, i32, i32, vp]
     lib.a3_query_scores.argtypes = [vp, vp, vp, i32, vp, i32, i32, i32, vp, vp, vp, sz, vp]
     lib.a3_query_scores_static.argtypes = [vp, vp, vp, i32, vp, i32, i32, i32, vp, vp]
     lib.a3_topk_select.argtypes = [vp, vp, i32, i32, i32, vp, vp]
@@ -263,18 +270,30 @@ class A3:
         return self._ws
 
     # ---- the steps (names as in the C ABI)
+    def set_option(self, option: int, value: int):
+        """a3_set_option: pins a kernel variant on this handle (cross-checks and measurements)."""
+        _check(_load().a3_set_option(self._h, int(option), int(value)), "a3_set_option")
+
     def rope_rerotate(self, chunks: torch.Tensor, n_chunks: int, max_chunk_len: int, k_fused: torch.Tensor,
-                      v_fused: torch.Tensor, layer_begin: int = 0, layer_end: Optional[int] = None):
+                      v_fused: torch.Tensor, layer_begin: int = 0, layer_end: Optional[int] = None, kv_len: Optional[int] = None):
+        """kv_len: slots of a fused layer (default: the tensor's second dimension)."""
         layer_end = self.shape.n_layers if layer_end is None else layer_end
         stride = k_fused.stride(0) * 2
+        kv_len = k_fused.shape[1] if kv_len is None else kv_len
         _check(_load().a3_rope_rerotate(self._h, _ptr(chunks), n_chunks, max_chunk_len, _ptr(k_fused), _ptr(v_fused),
-                                        stride, layer_begin, layer_end, _stream()), "a3_rope_rerotate")
+                                        stride, kv_len, layer_begin, layer_end, _stream()), "a3_rope_rerotate")
+
+    def swiglu_rows(self, layer: int, x: torch.Tensor, out: Optional[torch.Tensor] = None) -> torch.Tensor:
+        if out is None:
+            out = torch.empty((x.shape[0], self.shape.d_ff), dtype=torch.bfloat16, device=x.device)
+        _check(_load().a3_swiglu_rows(self._h, layer, _ptr(x), _ptr(out), x.shape[0], _stream()), "a3_swiglu_rows")
+        return out
 
     def query_scores(self, q_rows, q_pos, k_layer, cand_begin, cand_end, lse=None, scores=None):
         nq, kv_len = q_rows.shape[0], k_layer.shape[0]
         if scores is None:
             scores = torch.empty(kv_len, dtype=torch.float32, device=k_layer.device)
-        ws = self.workspace(self.layer_workspace_bytes(max(nq, 1)))
+        ws = self.workspace(int(_load().a3_scores_workspace_bytes(self._h, nq)))
         _check(_load().a3_query_scores(self._h, _ptr(q_rows), _ptr(q_pos), nq, _ptr(k_layer), kv_len, cand_begin,
                                        cand_end, _ptr(lse), _ptr(scores), _ptr(ws), ws.numel(), _stream()),
                "a3_query_scores")

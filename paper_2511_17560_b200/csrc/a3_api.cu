@@ -139,6 +139,12 @@ extern "C" int a3_create(a3_handle** out, const a3_model_desc* m, const a3_layer
   a3_handle* h = (a3_handle*)calloc(1, sizeof(a3_handle));
   if (!h) return A3_EINVAL;
   h->m = *m;
+  h->opt[A3_OPT_ATTN_PAIR] = -1;
+  h->opt[A3_OPT_SWIGLU_NARROW] = 1;
+  h->opt[A3_OPT_SWIGLU_PAIR] = 1;
+  h->opt[A3_OPT_RESIDUAL_T] = 1;
+  h->opt[A3_OPT_GEMM_BN_SWIGLU] = 256;  // the one-CTA gate/up kernel runs two CTAs per SM: 256 columns, 2 stages
+  h->opt[A3_OPT_GEMM_STAGES_SWIGLU] = 2;
   h->layers = (a3_layer_weights*)malloc(sizeof(a3_layer_weights) * m->n_layers);
   memcpy(h->layers, layers, sizeof(a3_layer_weights) * m->n_layers);
   cudaError_t e = cudaGetDevice(&h->device);
@@ -160,6 +166,12 @@ extern "C" int a3_create(a3_handle** out, const a3_model_desc* m, const a3_layer
     return s;
   }
   *out = h;
+  return A3_OK;
+}
+
+extern "C" int a3_set_option(a3_handle* h, int option, int value) {
+  if (!h || option < 0 || option >= A3_OPT_COUNT) return A3_EINVAL;
+  h->opt[option] = value;
   return A3_OK;
 }
 
@@ -342,6 +354,21 @@ extern "C" int a3_recompute_layer(const a3_handle* h, int layer, void* x_rows, c
 }
 
 // ------------------------------------------------------------------ scores (Eq. 3)
+extern "C" size_t a3_scores_workspace_bytes(const a3_handle* h, int nq) {
+  if (!h || nq < 0) return 0;
+  return align_up((size_t)(nq > 0 ? nq : 1) * h->m.n_q_heads * 4, 256) + stats_part_bytes(h, nq);
+}
+
+namespace a3 {
+// Row log-sum-exps of the question rows (statistics pass of the attention kernel, keys split over the SMs), then the
+// score pass.  `part` may be null (no split: one CTA per row tile and KV head).
+int scores_with_stats(const a3_handle* h, const bf16* q, const int32_t* q_pos, int nq, const bf16* k, int kv_len, int cand_begin,
+                      int cand_end, float* lse, void* part, size_t part_bytes, float* scores, cudaStream_t st) {
+  if (nq > 0) A3_TRY(attention_rows(h, q, q_pos, nq, k, k, kv_len, nullptr, lse, part, part_bytes, st));
+  return scores_pass(h, q, q_pos, nq, k, kv_len, cand_begin, cand_end, lse, scores, st);
+}
+}  // namespace a3
+
 extern "C" int a3_query_scores(const a3_handle* h, const void* q_rows, const int32_t* q_pos, int nq, const void* k_layer,
                                int kv_len, int cand_begin, int cand_end, const float* lse, float* scores, void* ws,
                                size_t ws_bytes, a3_stream stream) {
@@ -350,13 +377,14 @@ extern "C" int a3_query_scores(const a3_handle* h, const void* q_rows, const int
   if (!scores || !k_layer) return A3_EINVAL;
   if (nq > 0 && (!q_rows || !q_pos)) return A3_EINVAL;
   if (((uintptr_t)q_rows | (uintptr_t)k_layer) & 15) return A3_EINVAL;
+  if (kv_len > h->m.max_positions) return A3_EINVAL;
   cudaStream_t st = (cudaStream_t)stream;
+  A3_TRY(check_rows(h, q_pos, nq, kv_len, st));  // the key range of a row tile is taken from its first and last row
   if (!lse && nq > 0) {
-    const size_t need = align_up((size_t)nq * h->m.n_q_heads * 4, 256);
-    if (!ws || ws_bytes < need) return A3_EWORKSPACE;
-    A3_TRY(attention_rows(h, (const bf16*)q_rows, q_pos, nq, (const bf16*)k_layer, (const bf16*)k_layer, kv_len, nullptr,
-                          (float*)ws, nullptr, 0, st));
-    lse = (const float*)ws;
+    const size_t lse_bytes = align_up((size_t)nq * h->m.n_q_heads * 4, 256);
+    if (!ws || ((uintptr_t)ws & 15) || ws_bytes < lse_bytes + stats_part_bytes(h, nq)) return A3_EWORKSPACE;
+    return scores_with_stats(h, (const bf16*)q_rows, q_pos, nq, (const bf16*)k_layer, kv_len, cand_begin, cand_end, (float*)ws,
+                             (char*)ws + lse_bytes, stats_part_bytes(h, nq), scores, st);
   }
   return scores_pass(h, (const bf16*)q_rows, q_pos, nq, (const bf16*)k_layer, kv_len, cand_begin, cand_end, lse, scores, st);
 }
@@ -485,7 +513,7 @@ static int a3::fuse_impl(const a3_handle* h, const a3_request* r, void* ws, size
   if (r->score_source == A3_SCORES_CACHED_KEYS) {
     // Scores against the recovered cached keys: every layer is position-recovered; only the question rows pass
     // through the leading blocks; rows [Re, Q] are recomputed through every layer from the embeddings.
-    A3_TRY(a3_rope_rerotate(h, r->chunks, r->n_chunks, r->max_chunk_len, r->k_fused, r->v_fused, r->layer_stride, 0, m.n_layers, stream));
+    A3_TRY(a3_rope_rerotate(h, r->chunks, r->n_chunks, r->max_chunk_len, r->k_fused, r->v_fused, r->layer_stride, r->n_ctx, 0, m.n_layers, stream));
     A3_TRY(iota_rows(h, w.all_pos, 0, n, st));
     const int32_t* q_pos = w.all_pos + r->n_ctx;
     A3_CUDA(cudaMemsetAsync(r->scores_out, 0, (size_t)n * 4, st));
@@ -495,8 +523,8 @@ static int a3::fuse_impl(const a3_handle* h, const a3_request* r, void* ws, size
       for (int l = 0; l < ls; ++l) A3_TRY(recompute_layer_impl(h, l, xq, q_pos, nq, kl(l), vl(l), n, nullptr, lw, st));
       A3_TRY(rmsnorm_rows(h, xq, (const bf16*)h->layers[ls].attn_norm, m.rms_eps, nq, m.d_model, lw.a, st));
       A3_TRY(qkv_project(h, ls, lw.a, q_pos, nq, 0, lw.q, kl(ls), vl(ls), n, st));
-      A3_TRY(attention_rows(h, lw.q, q_pos, nq, kl(ls), vl(ls), n, nullptr, w.lse_q, nullptr, 0, st));
-      A3_TRY(scores_pass(h, lw.q, q_pos, nq, kl(ls), n, r->n_system, r->n_ctx, w.lse_q, r->scores_out, st));
+      A3_TRY(scores_with_stats(h, lw.q, q_pos, nq, kl(ls), n, r->n_system, r->n_ctx, w.lse_q, lw.attn_part, lw.attn_part_bytes,
+                               r->scores_out, st));
     }
     if (p > 0) {
       if (r->forced_re) A3_CUDA(cudaMemcpyAsync(r->rows_out, r->forced_re, (size_t)p * 4, cudaMemcpyDeviceToDevice, st));
@@ -514,7 +542,7 @@ static int a3::fuse_impl(const a3_handle* h, const a3_request* r, void* ws, size
   // caches is rewritten with true values below (full blocks; K/V of all rows at the selection layer), so the
   // recovered values would never be read.
   if (!layer_ready && ls + 1 < m.n_layers)
-    A3_TRY(a3_rope_rerotate(h, r->chunks, r->n_chunks, r->max_chunk_len, r->k_fused, r->v_fused, r->layer_stride, ls + 1,
+    A3_TRY(a3_rope_rerotate(h, r->chunks, r->n_chunks, r->max_chunk_len, r->k_fused, r->v_fused, r->layer_stride, r->n_ctx, ls + 1,
                             m.n_layers, stream));
   // leading full blocks: the whole input through layers 0..select_layer-1
   if (x0_ready) A3_CUDA(cudaStreamWaitEvent(st, x0_ready, 0));
@@ -528,8 +556,8 @@ static int a3::fuse_impl(const a3_handle* h, const a3_request* r, void* ws, size
   if (r->selector == A3_SELECT_VALUE_DEVIATION) {
     A3_TRY(value_deviation(h, r->chunks, r->n_chunks, r->max_chunk_len, ls, vl(ls), r->n_system, r->n_ctx, r->scores_out, st));
   } else if (nq > 0) {
-    A3_TRY(attention_rows(h, lw.q, w.all_pos + r->n_ctx, nq, kl(ls), vl(ls), n, nullptr, w.lse_q, nullptr, 0, st));
-    A3_TRY(scores_pass(h, lw.q, w.all_pos + r->n_ctx, nq, kl(ls), n, r->n_system, r->n_ctx, w.lse_q, r->scores_out, st));
+    A3_TRY(scores_with_stats(h, lw.q, w.all_pos + r->n_ctx, nq, kl(ls), n, r->n_system, r->n_ctx, w.lse_q, lw.attn_part,
+                             lw.attn_part_bytes, r->scores_out, st));
   }
   if (p > 0) {
     if (r->forced_re) A3_CUDA(cudaMemcpyAsync(r->rows_out, r->forced_re, (size_t)p * 4, cudaMemcpyDeviceToDevice, st));
@@ -540,7 +568,7 @@ static int a3::fuse_impl(const a3_handle* h, const a3_request* r, void* ws, size
     if (layer_ready)
       for (int l = ls + 1; l < m.n_layers; ++l) {
         A3_CUDA(cudaStreamWaitEvent(st, layer_ready[l], 0));
-        A3_TRY(a3_rope_rerotate(h, r->chunks, r->n_chunks, r->max_chunk_len, r->k_fused, r->v_fused, r->layer_stride, l, l + 1, stream));
+        A3_TRY(a3_rope_rerotate(h, r->chunks, r->n_chunks, r->max_chunk_len, r->k_fused, r->v_fused, r->layer_stride, r->n_ctx, l, l + 1, stream));
       }
     return A3_OK;
   }
@@ -550,7 +578,7 @@ static int a3::fuse_impl(const a3_handle* h, const a3_request* r, void* ws, size
   for (int l = ls; l < m.n_layers; ++l) {
     if (layer_ready && l > ls) {
       A3_CUDA(cudaStreamWaitEvent(st, layer_ready[l], 0));
-      A3_TRY(a3_rope_rerotate(h, r->chunks, r->n_chunks, r->max_chunk_len, r->k_fused, r->v_fused, r->layer_stride, l, l + 1, stream));
+      A3_TRY(a3_rope_rerotate(h, r->chunks, r->n_chunks, r->max_chunk_len, r->k_fused, r->v_fused, r->layer_stride, r->n_ctx, l, l + 1, stream));
     }
     A3_TRY(layer_step(l, (bf16*)r->x_out, r->rows_out, M));
   }
@@ -601,6 +629,8 @@ struct HostPipe {
   cudaEvent_t start, x0_ready;
   cudaEvent_t* layer_ready;
   int n_layers;
+  a3_chunk_ref* href;  // host copy of the chunk descriptors of the last call
+  int href_cap;
 };
 static int host_pipe(const a3_handle* h, HostPipe** out) {
   a3_handle* hm = const_cast<a3_handle*>(h);
@@ -628,6 +658,7 @@ static void host_pipe_destroy(a3_handle* h) {
   if (p->x0_ready) cudaEventDestroy(p->x0_ready);
   if (p->copy_stream) cudaStreamDestroy(p->copy_stream);
   free(p->layer_ready);
+  free(p->href);
   free(p);
   h->host_pipe = nullptr;
 }
@@ -654,16 +685,19 @@ extern "C" int a3_fuse_request_host(const a3_handle* h, const a3_request* req, c
   char* kv = base;
   char* x0 = base + align_up(2 * (size_t)m.n_layers * req->n_ctx * row, 256);
   a3_chunk_ref* dref = (a3_chunk_ref*)(x0 + align_up((size_t)n * m.d_model * 2, 256));
-  a3_chunk_ref* href = (a3_chunk_ref*)malloc(sizeof(a3_chunk_ref) * (req->n_chunks > 0 ? req->n_chunks : 1));
-  if (!href) return A3_EINVAL;
+  // host copy of the descriptors: kept by the handle and grown on demand, so that a steady stream of calls allocates nothing
+  if (hp->href_cap < req->n_chunks) {
+    a3_chunk_ref* grown = (a3_chunk_ref*)realloc(hp->href, sizeof(a3_chunk_ref) * (size_t)req->n_chunks);
+    if (!grown) return A3_EINVAL;
+    hp->href = grown;
+    hp->href_cap = req->n_chunks;
+  }
+  a3_chunk_ref* href = hp->href;
   int off = 0, maxlen = 0;
   size_t kvoff = 0;
   for (int c = 0; c < req->n_chunks; ++c) {
     const int len = io->chunk_len[c];
-    if (len < 0 || off + len > req->n_ctx) {
-      free(href);
-      return A3_EINVAL;
-    }
+    if (len < 0 || off + len > req->n_ctx) return A3_EINVAL;
     const size_t bytes = (size_t)m.n_layers * len * row;
     href[c].k_src = kv + kvoff;
     href[c].v_src = kv + kvoff + bytes;
@@ -676,40 +710,42 @@ extern "C" int a3_fuse_request_host(const a3_handle* h, const a3_request* req, c
     off += len;
     if (len > maxlen) maxlen = len;
   }
-  if (off != req->n_ctx) {
-    free(href);
-    return A3_EINVAL;
-  }
+  if (off != req->n_ctx) return A3_EINVAL;
+  // From here on copies are in flight: every exit waits for both streams first, so that the caller may reuse or free
+  // its host buffers and the staging area whatever the status.
+  int status = A3_OK;
+  auto note = [&](cudaError_t e) {
+    if (e != cudaSuccess && status == A3_OK) status = cuda_fail(e);
+    return status == A3_OK;
+  };
   // the copy stream starts after whatever the caller has already queued on `stream` (the staging area may be in use)
-  cudaError_t e = cudaEventRecord(hp->start, st);
-  if (e == cudaSuccess) e = cudaStreamWaitEvent(cs, hp->start, 0);
+  note(cudaEventRecord(hp->start, st));
+  if (status == A3_OK) note(cudaStreamWaitEvent(cs, hp->start, 0));
   // the descriptor array is pageable host memory: this copy returns only once it has been staged
-  if (e == cudaSuccess && req->n_chunks > 0)
-    e = cudaMemcpyAsync(dref, href, sizeof(a3_chunk_ref) * req->n_chunks, cudaMemcpyHostToDevice, cs);
-  if (e == cudaSuccess) e = cudaMemcpyAsync(x0, io->x0, (size_t)n * m.d_model * 2, cudaMemcpyHostToDevice, cs);
-  if (e == cudaSuccess) e = cudaEventRecord(hp->x0_ready, cs);
-  for (int l = req->select_layer + 1; l < m.n_layers && e == cudaSuccess; ++l) {
-    for (int c = 0; c < req->n_chunks && e == cudaSuccess; ++c) {
+  if (status == A3_OK && req->n_chunks > 0)
+    note(cudaMemcpyAsync(dref, href, sizeof(a3_chunk_ref) * req->n_chunks, cudaMemcpyHostToDevice, cs));
+  if (status == A3_OK) note(cudaMemcpyAsync(x0, io->x0, (size_t)n * m.d_model * 2, cudaMemcpyHostToDevice, cs));
+  if (status == A3_OK) note(cudaEventRecord(hp->x0_ready, cs));
+  for (int l = req->select_layer + 1; l < m.n_layers && status == A3_OK; ++l) {
+    for (int c = 0; c < req->n_chunks && status == A3_OK; ++c) {
       const size_t slice = (size_t)href[c].len * row;
-      e = cudaMemcpyAsync((char*)href[c].k_src + l * slice, (const char*)io->chunk_k[c] + l * slice, slice, cudaMemcpyHostToDevice, cs);
-      if (e == cudaSuccess)
-        e = cudaMemcpyAsync((char*)href[c].v_src + l * slice, (const char*)io->chunk_v[c] + l * slice, slice, cudaMemcpyHostToDevice, cs);
+      if (note(cudaMemcpyAsync((char*)href[c].k_src + l * slice, (const char*)io->chunk_k[c] + l * slice, slice, cudaMemcpyHostToDevice, cs)))
+        note(cudaMemcpyAsync((char*)href[c].v_src + l * slice, (const char*)io->chunk_v[c] + l * slice, slice, cudaMemcpyHostToDevice, cs));
     }
-    if (e == cudaSuccess) e = cudaEventRecord(hp->layer_ready[l], cs);
+    if (status == A3_OK) note(cudaEventRecord(hp->layer_ready[l], cs));
   }
-  free(href);
-  if (e != cudaSuccess) return cuda_fail(e);
   a3_request r = *req;
   r.chunks = dref;
   r.max_chunk_len = maxlen;
   r.x0 = x0;
-  A3_TRY(fuse_impl(h, &r, ws, ws_bytes, stream, hp->layer_ready, hp->x0_ready));
+  if (status == A3_OK) status = fuse_impl(h, &r, ws, ws_bytes, stream, hp->layer_ready, hp->x0_ready);
   const int M = r.n_recompute + r.n_question;
-  if (M > 0) {
-    A3_CUDA(cudaMemcpyAsync(io->rows_out, r.rows_out, (size_t)M * 4, cudaMemcpyDeviceToHost, st));
-    A3_CUDA(cudaMemcpyAsync(io->x_out, r.x_out, (size_t)M * m.d_model * 2, cudaMemcpyDeviceToHost, st));
+  if (status == A3_OK && M > 0) {
+    if (note(cudaMemcpyAsync(io->rows_out, r.rows_out, (size_t)M * 4, cudaMemcpyDeviceToHost, st)))
+      note(cudaMemcpyAsync(io->x_out, r.x_out, (size_t)M * m.d_model * 2, cudaMemcpyDeviceToHost, st));
   }
-  A3_CUDA(cudaStreamSynchronize(st));
-  A3_CUDA(cudaStreamSynchronize(cs));
-  return A3_OK;
+  note(cudaStreamSynchronize(cs));  // the copy stream first: the compute stream may be waiting on its events
+  const cudaError_t es = cudaStreamSynchronize(st);
+  if (es != cudaSuccess && status == A3_OK) status = cuda_fail(es);
+  return status;
 }

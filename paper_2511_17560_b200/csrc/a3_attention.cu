@@ -539,15 +539,19 @@ attention_combine_kernel(const int32_t* __restrict__ pos, int M, int kv_len, int
     if (!(ml.y > 0.f)) continue;
     const float w = exp2f(ml.x - m);
     l += ml.y * w;
-    const float* src = part_o + prow * D + lane * PER;
+    if (o) {
+      const float* src = part_o + prow * D + lane * PER;
 #pragma unroll
-    for (int e = 0; e < PER; ++e) acc[e] += src[e] * w;
+      for (int e = 0; e < PER; ++e) acc[e] += src[e] * w;
+    }
   }
   const int tok = fr / G, hq = g * G + fr % G;
   const float inv = l > 0.f ? 1.f / l : 0.f;
-  bf16* dst = o + ((size_t)tok * Hq + hq) * D + lane * PER;
+  if (o) {
+    bf16* dst = o + ((size_t)tok * Hq + hq) * D + lane * PER;
 #pragma unroll
-  for (int e = 0; e < PER; e += 2) *reinterpret_cast<uint32_t*>(dst + e) = pack2(acc[e] * inv, acc[e + 1] * inv);
+    for (int e = 0; e < PER; e += 2) *reinterpret_cast<uint32_t*>(dst + e) = pack2(acc[e] * inv, acc[e + 1] * inv);
+  }
   if (lse && lane == 0) lse[(size_t)tok * Hq + hq] = l > 0.f ? (m + log2f(l)) * ATC_LN2 : -INFINITY;
 }
 
@@ -579,9 +583,22 @@ static int make_cache_tmap(CUtensorMap* map, const void* ptr, long long rows, lo
   return A3_OK;
 }
 
-int g_attn_max_ctas = 0;  // tuning: cap on the persistent grid
-int g_attn_pair = -1;  // -1: choose; 0: never; 1: whenever supported (tuning)
-int g_attn_split = 0;  // 0: choose; otherwise the number of key segments (tuning)
+// Key segments of a statistics-only call on nq rows: as many as leave every SM at most one item, within the cap.
+static int stats_max_splits(const a3_handle* h, int nq) {
+  const int Hkv = h->m.n_kv_heads, G = h->m.n_q_heads / Hkv;
+  const int sms = h->sm_count > 0 ? h->sm_count : 148;
+  const long long row_tiles = cdiv((long long)(nq > 0 ? nq : 1) * G, ATC_BM);
+  const long long per_split = row_tiles * ATC_BM * Hkv * (long long)sizeof(float2);
+  long long s = sms / (row_tiles * Hkv);
+  if (s > (long long)(STATS_PART_CAP / per_split)) s = (long long)(STATS_PART_CAP / per_split);
+  return s < 2 ? 1 : (int)s;
+}
+size_t stats_part_bytes(const a3_handle* h, int nq) {
+  const int Hkv = h->m.n_kv_heads, G = h->m.n_q_heads / Hkv;
+  const int s = stats_max_splits(h, nq);
+  if (s < 2) return 0;
+  return (size_t)s * cdiv((long long)(nq > 0 ? nq : 1) * G, ATC_BM) * ATC_BM * Hkv * sizeof(float2);
+}
 
 size_t attention_part_bytes(const a3_handle* h) {
   // split only happens when the unsplit grid has fewer than two CTAs per SM; up to 4 segments
@@ -603,7 +620,7 @@ int attention_rows(const a3_handle* h, const bf16* q, const int32_t* pos, int M,
     // many row tiles: two per CTA (a3_attention_pair.cu); few: one per CTA, where the longest item sets the time
     const int sms_ = h->sm_count > 0 ? h->sm_count : 148;
     const int pair_items = (((int)grid.x + 1) / 2) * Hkv;
-    const bool use_pair = g_attn_pair < 0 ? pair_items >= 2 * sms_ : g_attn_pair > 0;
+    const bool use_pair = h->opt[A3_OPT_ATTN_PAIR] < 0 ? pair_items >= 2 * sms_ : h->opt[A3_OPT_ATTN_PAIR] > 0;
     if (use_pair && o && D == 128) {
       const int s = attention_rows_pair(h, tK, tV, q, pos, M, kv_len, o, lse, st);
       if (s != A3_EUNSUPPORTED) return s;
@@ -614,24 +631,28 @@ int attention_rows(const a3_handle* h, const bf16* q, const int32_t* pos, int M,
   const int base_ctas = (int)grid.x * Hkv, all_tiles = cdiv(kv_len, ATC_BN);
   int n_split = 1;
   if (o && part && base_ctas < 2 * sms && all_tiles >= 8) {
-    n_split = g_attn_split > 0 ? g_attn_split : 1;  // measured: with the persistent schedule no split beats 2..4 segments (7 us per item)
+    n_split = h->opt[A3_OPT_ATTN_SPLIT] > 0 ? h->opt[A3_OPT_ATTN_SPLIT] : 1;  // measured: with the persistent schedule no split beats 2..4 segments (7 us per item)
     const size_t need = (size_t)n_split * base_ctas * ATC_BM * ((size_t)D + 2) * sizeof(float);
     if (need > part_bytes) n_split = 1;
+  }
+  if (!o && part && all_tiles >= 2) {
+    // statistics only (the question rows' log-sum-exps before the score pass): a handful of row tiles, so the keys are
+    // split over the SMs; partial (reference, sum) pairs only, merged in segment order by the combine kernel
+    n_split = stats_max_splits(h, M);
+    if (n_split > all_tiles) n_split = all_tiles;
+    if ((size_t)n_split * base_ctas * ATC_BM * sizeof(float2) > part_bytes) n_split = 1;
   }
   const int tiles_per_split = cdiv(all_tiles, n_split);
   n_split = cdiv(all_tiles, tiles_per_split);
   const int rows_pad = (int)grid.x * ATC_BM;
   const int n_items = (int)grid.x * Hkv * n_split;
   int n_ctas = n_items < sms ? n_items : sms;  // persistent: at most one CTA per SM
-  if (g_attn_max_ctas > 0 && n_ctas > g_attn_max_ctas) n_ctas = g_attn_max_ctas;
+  if (h->opt[A3_OPT_ATTN_MAX_CTAS] > 0 && n_ctas > h->opt[A3_OPT_ATTN_MAX_CTAS]) n_ctas = h->opt[A3_OPT_ATTN_MAX_CTAS];
   float* part_o = (float*)part;
-  float2* part_ml = part ? (float2*)(part_o + (size_t)n_split * Hkv * rows_pad * D) : nullptr;
-  static bool attr_set = false;
-  if (!attr_set) {
-    A3_CUDA(cudaFuncSetAttribute(attention_tc_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, AtcLayout<128>::SMEM_BYTES));
-    A3_CUDA(cudaFuncSetAttribute(attention_tc_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, AtcLayout<64>::SMEM_BYTES));
-    attr_set = true;
-  }
+  float2* part_ml = !part ? nullptr : !o ? (float2*)part : (float2*)(part_o + (size_t)n_split * Hkv * rows_pad * D);
+  static SmemAttrOnce attr128, attr64;
+  if (D == 128) A3_TRY(smem_attr_once(attr128, h->device, attention_tc_kernel<128>, AtcLayout<128>::SMEM_BYTES));
+  else A3_TRY(smem_attr_once(attr64, h->device, attention_tc_kernel<64>, AtcLayout<64>::SMEM_BYTES));
   ProfScope prof(h, A3_K_ATTENTION, st);
   if (D == 128)
     A3_CUDA(launch_pdl(attention_tc_kernel<128>, dim3(n_ctas), dim3(ATC_THREADS), (size_t)AtcLayout<128>::SMEM_BYTES, st, tK, tV, q, pos, M, kv_len, o,
@@ -651,6 +672,3 @@ int attention_rows(const a3_handle* h, const bf16* q, const int32_t* pos, int M,
 
 }  // namespace a3
 
-extern "C" void a3_internal_set_attn_split(int v) { a3::g_attn_split = v; }
-extern "C" void a3_internal_set_attn_pair(int v) { a3::g_attn_pair = v; }
-extern "C" void a3_internal_set_attn_max_ctas(int v) { a3::g_attn_max_ctas = v; }

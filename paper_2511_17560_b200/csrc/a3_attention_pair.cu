@@ -501,11 +501,8 @@ int attention_rows_pair(const a3_handle* h, const CUtensorMap& tK, const CUtenso
   const int sms = h->sm_count > 0 ? h->sm_count : 148;
   const int n_ctas = n_items < sms ? n_items : sms;
   const float scale_log2 = ATC_LOG2E / sqrtf((float)D);
-  static bool attr_set = false;
-  if (!attr_set) {
-    A3_CUDA(cudaFuncSetAttribute(attention_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, At2Layout::SMEM_BYTES));
-    attr_set = true;
-  }
+  static SmemAttrOnce attr;
+  A3_TRY(smem_attr_once(attr, h->device, attention_pair_kernel, At2Layout::SMEM_BYTES));
   ProfScope prof(h, A3_K_ATTENTION, st);
   A3_CUDA(launch_pdl(attention_pair_kernel, dim3(n_ctas), dim3(AT2_THREADS), (size_t)At2Layout::SMEM_BYTES, st, tK, tV, q, pos, M, kv_len, o, lse,
                      Hq, Hkv, scale_log2, h->dev_status));

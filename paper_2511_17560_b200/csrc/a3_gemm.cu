@@ -559,11 +559,8 @@ static int launch_tc(const a3_handle* h, const GemmArgs& a, const TcParams& p, i
       else tB[s] = tB[0];
     }
   }
-  static bool attr_set = false;
-  if (!attr_set) {
-    A3_CUDA(cudaFuncSetAttribute(gemm_tc_kernel<EPI, BN, STAGES>, cudaFuncAttributeMaxDynamicSharedMemorySize, L::SMEM_BYTES));
-    attr_set = true;
-  }
+  static SmemAttrOnce attr;
+  A3_TRY(smem_attr_once(attr, h->device, gemm_tc_kernel<EPI, BN, STAGES>, L::SMEM_BYTES));
   dim3 grid(cdiv(a.M, TC_BM), tiles);
   ProfScope prof(h, EPI == EPI_RESIDUAL ? A3_K_GEMM_RESIDUAL : EPI == EPI_SWIGLU ? A3_K_GEMM_SWIGLU : A3_K_GEMM_QKV, st);
   if (!(EPI == EPI_SWIGLU && p.g_narrow > 0)) tN[0] = tN[1] = tB[0];
@@ -587,11 +584,8 @@ static int launch_pair(const a3_handle* h, const GemmArgs& a, const TcParams& p,
       else tB[s] = tB[0];
     }
   }
-  static bool attr_set = false;
-  if (!attr_set) {
-    A3_CUDA(cudaFuncSetAttribute(gemm_pair_kernel<EPI, STAGES>, cudaFuncAttributeMaxDynamicSharedMemorySize, L::SMEM_BYTES));
-    attr_set = true;
-  }
+  static SmemAttrOnce attr;
+  A3_TRY(smem_attr_once(attr, h->device, gemm_pair_kernel<EPI, STAGES>, L::SMEM_BYTES));
   dim3 grid(2 * cdiv(cdiv(a.M, TC_BM), 2), tiles);  // whole pairs: a last odd row tile gets an all-padding partner
   ProfScope prof(h, EPI == EPI_RESIDUAL ? A3_K_GEMM_RESIDUAL : EPI == EPI_SWIGLU ? A3_K_GEMM_SWIGLU : A3_K_GEMM_QKV, st);
   A3_CUDA(launch_pdl(gemm_pair_kernel<EPI, STAGES>, grid, dim3(TC_THREADS), (size_t)L::SMEM_BYTES, st, tA, tB[0], tB[1], tB[2], p));
@@ -600,13 +594,12 @@ static int launch_pair(const a3_handle* h, const GemmArgs& a, const TcParams& p,
 }
 
 // Tile width / pipeline depth per epilogue [EPI_RESIDUAL, EPI_SWIGLU, EPI_QKV] -> {BN, STAGES}; BN = 0 lets the
-// launcher choose (a3_internal_set_gemm_cfg pins a choice for tuning runs).  Measured on B200 at Llama-8B width:
+// launcher choose (a3_set_option pins a choice on a handle for cross-checks).  Measured on B200 at Llama-8B width:
 // two co-resident CTAs per SM (256/2, 128/3) overlap one tile's epilogue with the other's main loop and win when
 // the grid has several waves.  The CTA-pair kernel wins for the residual GEMMs (N = d_model: few tiles, one CTA per
 // SM); for SwiGLU and QKV its extra all-padding row tile at 804 rows (7 -> 8) costs more than the halved B traffic
 // saves: under the power cap the tensor work, not the L2 port, sets the pace.
-int g_tc_narrow = 1;  // 0: no narrower last wave in the SwiGLU grid; 1: choose; 16..120: that width on half the tiles (tests)
-int g_tc_cfg[3][2] = {{0, 0}, {256, 2}, {0, 0}};
+// A3_OPT_SWIGLU_NARROW: 0: no narrower last wave in the SwiGLU grid; 1: choose; 16..120: that width on half the tiles.
 
 template <int EPI>
 static int dispatch_tc(const a3_handle* h, const GemmArgs& a, const TcParams& p, int tiles, int bn, int stages, cudaStream_t st) {
@@ -629,9 +622,10 @@ int gemm_bf16(const a3_handle* h, GemmEpilogue epi, const GemmArgs& a, cudaStrea
   if (a.M <= 0) return A3_OK;
   if (a.K % TC_BK) return A3_EUNSUPPORTED;
   if (epi == EPI_SWIGLU && swiglu_pair_usable(h, a)) return gemm_swiglu_pair(h, a, st);
-  if (epi == EPI_RESIDUAL && g_tc_cfg[EPI_RESIDUAL][0] == 0 && residual_t_usable(h, a)) return gemm_residual_t(h, a, st);
-  int bn = g_tc_cfg[epi][0];
-  int stages = g_tc_cfg[epi][1];
+  const int g_tc_narrow = h->opt[A3_OPT_SWIGLU_NARROW];
+  int bn = h->opt[A3_OPT_GEMM_BN_RESIDUAL + (int)epi];
+  int stages = h->opt[A3_OPT_GEMM_STAGES_RESIDUAL + (int)epi];
+  if (epi == EPI_RESIDUAL && bn == 0 && residual_t_usable(h, a)) return gemm_residual_t(h, a, st);
 
   if (bn == 0) {
     const int m_tiles = cdiv(a.M, TC_BM), sms = h->sm_count > 0 ? h->sm_count : 148;
@@ -750,10 +744,3 @@ int gemm_bf16(const a3_handle* h, GemmEpilogue epi, const GemmArgs& a, cudaStrea
 
 }  // namespace a3
 
-extern "C" void a3_internal_set_gemm_narrow(int on) { a3::g_tc_narrow = on; }
-extern "C" void a3_internal_set_gemm_cfg(int epi, int bn, int stages) {
-  if (epi >= 0 && epi < 3) {
-    a3::g_tc_cfg[epi][0] = bn;
-    a3::g_tc_cfg[epi][1] = stages;
-  }
-}

@@ -372,19 +372,17 @@ pair_t_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ C
   if (warp == 1) asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(512) : "memory");
 }
 
-// 0: never; 1: whenever the shape allows (default); tuning/tests switch them off to compare with the other kernels
-int g_swiglu_pair = 1;
-int g_residual_t = 1;
-
+// A3_OPT_SWIGLU_PAIR / A3_OPT_RESIDUAL_T: 0 never; 1 whenever the shape allows (default); cross-checks switch them off
+// to compare with the other kernels
 bool swiglu_pair_usable(const a3_handle* h, const GemmArgs& a) {
-  (void)h;
-  return g_swiglu_pair != 0 && a.M > 0 && a.K % (SP_SUB * TC_BK) == 0 && a.seg[0].n % (2 * SP_FEAT) == 0 && a.seg[0].bias == nullptr;
+  return h->opt[A3_OPT_SWIGLU_PAIR] != 0 && a.M > 0 && a.K % (SP_SUB * TC_BK) == 0 && a.seg[0].n % (2 * SP_FEAT) == 0 && a.seg[0].bias == nullptr;
 }
 // Measured at Llama-8B width: with several units per CTA pair (5 152 rows: 336 units on 74 pairs) this kernel hides
 // every epilogue but the last and wins (output projection 139 vs 165 us, down projection 522 vs 533 us); with at most
 // one unit per pair (804 rows: 64 units) it has nothing to hide and the 256 x 256 CTA-pair kernel is as fast or faster
-// (26 vs 28 us, 85 vs 82 us).  g_residual_t: 0 never, 1 by that rule (default), 2 whenever the shape allows (tests).
+// (26 vs 28 us, 85 vs 82 us).  A3_OPT_RESIDUAL_T: 0 never, 1 by that rule (default), 2 whenever the shape allows.
 bool residual_t_usable(const a3_handle* h, const GemmArgs& a) {
+  const int g_residual_t = h->opt[A3_OPT_RESIDUAL_T];
   if (g_residual_t == 0 || a.M <= 0 || a.K % (SP_SUB * TC_BK) != 0 || a.nseg != 1 || a.seg[0].n % 32 != 0 || a.seg[0].bias != nullptr)
     return false;
   if (g_residual_t == 2) return true;
@@ -419,11 +417,8 @@ static int launch_pair_t(const a3_handle* h, const GemmArgs& a, cudaStream_t st)
   A3_TRY(make_tmap(&tG, a.seg[0].B, p.F, a.K, ROWS));
   if (EPI == EPI_SWIGLU) A3_TRY(make_tmap(&tU, a.B2, p.F, a.K, ROWS));
   else tU = tG;
-  static bool attr_set = false;
-  if (!attr_set) {
-    A3_CUDA(cudaFuncSetAttribute(pair_t_kernel<EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize, SP_SMEM_LIMIT));
-    attr_set = true;
-  }
+  static SmemAttrOnce attr;
+  A3_TRY(smem_attr_once(attr, h->device, pair_t_kernel<EPI>, SP_SMEM_LIMIT));
   ProfScope prof(h, EPI == EPI_SWIGLU ? A3_K_GEMM_SWIGLU : A3_K_GEMM_RESIDUAL, st);
   A3_CUDA(launch_pdl(pair_t_kernel<EPI>, dim3(2 * p.n_pairs), dim3(SP_THREADS), (size_t)smem_bytes, st, tX, tG, tU, p));
   A3_LAUNCHED();
@@ -435,12 +430,11 @@ int gemm_residual_t(const a3_handle* h, const GemmArgs& a, cudaStream_t st) { re
 
 }  // namespace a3
 
-extern "C" void a3_internal_set_swiglu_pair(int v) { a3::g_swiglu_pair = v; }
-extern "C" void a3_internal_set_residual_t(int v) { a3::g_residual_t = v; }
-
-
-// Test hook: the SwiGLU GEMM of one layer alone, out[M][d_ff] = silu(x Wg^T) * (x Wu^T), x [M][d_model].
-extern "C" int a3_internal_swiglu(const a3_handle* h, int layer, const void* x, void* out, int M, void* stream) {
+// The gate/up GEMM of one layer alone (a3_swiglu_rows): out[M][d_ff] = silu(x Wg^T) * (x Wu^T), x [M][d_model].
+extern "C" int a3_swiglu_rows(const a3_handle* h, int layer, const void* x, void* out, int M, a3_stream stream) {
+  if (!h || layer < 0 || layer >= h->m.n_layers || M < 0) return A3_EINVAL;
+  if (M == 0) return A3_OK;
+  if (!x || !out || (((uintptr_t)x | (uintptr_t)out) & 15)) return A3_EINVAL;
   a3::GemmArgs u{};
   u.A = (const bf16*)x;
   u.M = M;
@@ -452,4 +446,3 @@ extern "C" int a3_internal_swiglu(const a3_handle* h, int layer, const void* x, 
   u.ldc = h->m.d_ff;
   return a3::gemm_bf16(h, a3::EPI_SWIGLU, u, (cudaStream_t)stream);
 }
-

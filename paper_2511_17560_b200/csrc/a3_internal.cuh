@@ -5,6 +5,8 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include <atomic>
+
 #include "a3.h"
 
 typedef __nv_bfloat16 bf16;
@@ -21,6 +23,7 @@ struct a3_handle {
   void* tmaps;               // host-side tensor-map cache (a3_gemm.cu)
   a3::Profiler* prof;        // null unless a3_profile_enable is on
   void* host_pipe;           // copy stream + events of a3_fuse_request_host, created on first use
+  int opt[A3_OPT_COUNT];     // kernel-variant choices (a3_set_option); defaults set by a3_create
 };
 
 namespace a3 {
@@ -104,6 +107,20 @@ inline cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, s
 }
 #endif
 
+// The opt-in to more than 48 KiB of dynamic shared memory is a per-device attribute of a kernel: it is set once per
+// device (the handle's, which is current during its calls), not once per process.
+struct SmemAttrOnce {
+  std::atomic<unsigned long long> devices{0};
+};
+template <typename F>
+inline int smem_attr_once(SmemAttrOnce& once, int device, F func, int bytes) {
+  const unsigned long long bit = 1ull << (device & 63);
+  if (once.devices.load(std::memory_order_acquire) & bit) return A3_OK;
+  A3_CUDA(cudaFuncSetAttribute(func, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes));
+  once.devices.fetch_or(bit, std::memory_order_release);
+  return A3_OK;
+}
+
 inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 inline int cdiv(long long a, long long b) { return (int)((a + b - 1) / b); }
 
@@ -153,6 +170,13 @@ int gemm_bf16(const a3_handle* h, GemmEpilogue epi, const GemmArgs& a, cudaStrea
 int attention_rows(const a3_handle* h, const bf16* q, const int32_t* pos, int M, const bf16* k, const bf16* v,
                    int kv_len, bf16* o, float* lse, void* part, size_t part_bytes, cudaStream_t st);
 size_t attention_part_bytes(const a3_handle* h);
+// Statistics-only calls (o == null) split the keys of the few question row tiles over the SMs; the partial row
+// statistics of nq rows need at most this much of `part` (a fixed cap, so that every caller - whatever scratch it
+// has - arrives at the same split and therefore at bit-identical log-sum-exps).
+constexpr size_t STATS_PART_CAP = 768 * 1024;
+size_t stats_part_bytes(const a3_handle* h, int nq);
+int scores_with_stats(const a3_handle* h, const bf16* q, const int32_t* q_pos, int nq, const bf16* k, int kv_len, int cand_begin,
+                      int cand_end, float* lse, void* part, size_t part_bytes, float* scores, cudaStream_t st);
 
 int scores_pass(const a3_handle* h, const bf16* q, const int32_t* q_pos, int nq, const bf16* k, int kv_len,
                 int cand_begin, int cand_end, const float* lse, float* scores, cudaStream_t st, float* per_head = nullptr);

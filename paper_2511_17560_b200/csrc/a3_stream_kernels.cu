@@ -35,18 +35,22 @@ constexpr int RR_THREADS = 256;
 template <int D, int LAYOUT>
 __global__ void __launch_bounds__(RR_THREADS)
 rerotate_kernel(const a3_chunk_ref* __restrict__ chunks, char* __restrict__ kf, char* __restrict__ vf,
-                unsigned long long layer_stride, int layer_begin, int row_elems, int tok_per_cta,
+                unsigned long long layer_stride, int kv_len, int max_chunk_len, int layer_begin, int row_elems, int tok_per_cta,
                 const float2* __restrict__ tab, int max_pos, uint32_t* status) {
   const a3_chunk_ref ch = chunks[blockIdx.y];
   const int t0 = blockIdx.x * tok_per_cta;
+  if (ch.len < 0 && blockIdx.x == 0 && threadIdx.x == 0) atomicOr(status, A3_DEV_BAD_POSITION);
   if (t0 >= ch.len) return;
   const int l = layer_begin + blockIdx.z;
   const int nt = min(tok_per_cta, ch.len - t0);
   int ad = ch.delta < 0 ? -ch.delta : ch.delta;
   // with a per-token step the rotation of token t is delta + token_step * t: both ends must be in the table
   const long long a_last = (long long)ch.delta + (long long)ch.token_step * (ch.len - 1);
-  const bool bad = ad >= max_pos || (a_last < 0 ? -a_last : a_last) >= max_pos || ch.dst_offset < 0 || ((uintptr_t)ch.k_src & 15) || ((uintptr_t)ch.v_src & 15) ||
-                   (ch.src_layer_stride & 15);
+  // the chunk's slots must lie inside the fused cache and its length inside what the grid was sized for: a chunk that
+  // fails either check is skipped as a whole (every CTA of it takes this exit, so nothing of it is written)
+  const bool bad = ad >= max_pos || (a_last < 0 ? -a_last : a_last) >= max_pos || ch.dst_offset < 0 ||
+                   (long long)ch.dst_offset + ch.len > (long long)kv_len || ch.len > max_chunk_len ||
+                   ((uintptr_t)ch.k_src & 15) || ((uintptr_t)ch.v_src & 15) || (ch.src_layer_stride & 15);
   if (bad) {
     if (threadIdx.x == 0) atomicOr(status, A3_DEV_BAD_POSITION);
     return;
@@ -195,11 +199,12 @@ rerotate_kernel(const a3_chunk_ref* __restrict__ chunks, char* __restrict__ kf, 
 using namespace a3;
 
 extern "C" int a3_rope_rerotate(const a3_handle* h, const a3_chunk_ref* chunks, int n_chunks, int max_chunk_len,
-                                void* k_fused, void* v_fused, uint64_t layer_stride, int layer_begin, int layer_end,
+                                void* k_fused, void* v_fused, uint64_t layer_stride, int kv_len, int layer_begin, int layer_end,
                                 a3_stream stream) {
   if (!h || !chunks || !k_fused || !v_fused) return A3_EINVAL;
-  if (n_chunks < 0 || max_chunk_len < 0 || layer_begin < 0 || layer_end > h->m.n_layers || layer_begin > layer_end) return A3_EINVAL;
+  if (n_chunks < 0 || max_chunk_len < 0 || kv_len < 0 || layer_begin < 0 || layer_end > h->m.n_layers || layer_begin > layer_end) return A3_EINVAL;
   if (((uintptr_t)k_fused & 15) || ((uintptr_t)v_fused & 15) || (layer_stride & 15)) return A3_EINVAL;
+  if ((uint64_t)kv_len * h->m.n_kv_heads * h->m.head_dim * 2 > layer_stride) return A3_EINVAL;  // kv_len rows must fit in a layer
   if (n_chunks == 0 || max_chunk_len == 0 || layer_begin == layer_end) return A3_OK;
   if (n_chunks > 65535 || layer_end - layer_begin > 65535) return A3_EUNSUPPORTED;
   const int row_elems = h->m.n_kv_heads * h->m.head_dim;
@@ -209,9 +214,9 @@ extern "C" int a3_rope_rerotate(const a3_handle* h, const a3_chunk_ref* chunks, 
   dim3 grid(cdiv(max_chunk_len, tok), n_chunks, layer_end - layer_begin);
   cudaStream_t st = (cudaStream_t)stream;
 #define RR_LAUNCH(DD, LL)                                                                                             \
-  rerotate_kernel<DD, LL><<<grid, RR_THREADS, 0, st>>>(chunks, (char*)k_fused, (char*)v_fused, layer_stride,          \
-                                                       layer_begin, row_elems, tok, h->rope_tab, h->m.max_positions, \
-                                                       h->dev_status)
+  rerotate_kernel<DD, LL><<<grid, RR_THREADS, 0, st>>>(chunks, (char*)k_fused, (char*)v_fused, layer_stride, kv_len,  \
+                                                       max_chunk_len, layer_begin, row_elems, tok, h->rope_tab,      \
+                                                       h->m.max_positions, h->dev_status)
   ProfScope prof(h, A3_K_REROTATE, st);
   if (h->m.head_dim == 128 && h->m.rope_layout == 0) RR_LAUNCH(128, 0);
   else if (h->m.head_dim == 128) RR_LAUNCH(128, 1);

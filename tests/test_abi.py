@@ -35,6 +35,14 @@ def test_binding_lists_the_same_symbols(lib_path):
     a3._load()
 
 
+def test_no_undeclared_a3_symbols_are_exported(lib_path):
+    """Everything the library exports under the a3_ prefix is declared (and documented) in include/a3.h."""
+    import subprocess
+    out = subprocess.run(["nm", "-D", "--defined-only", lib_path], check=True, capture_output=True, text=True).stdout
+    exported = sorted({ln.split()[-1] for ln in out.splitlines() if ln.split() and ln.split()[-1].startswith("a3_")})
+    assert exported == declared_symbols()
+
+
 def test_host_only_entry_points(lib_path):
     from paper_2511_17560_b200 import a3
     lib = a3._load()
@@ -48,7 +56,10 @@ def test_host_only_entry_points(lib_path):
     # argument validation happens before any CUDA call
     assert lib.a3_create(None, None, None) == -1
     assert lib.a3_fuse_request(None, None, None, 0, None) == -1
-    assert lib.a3_rope_rerotate(None, None, 0, 0, None, None, 0, 0, 0, None) == -1
+    assert lib.a3_rope_rerotate(None, None, 0, 0, None, None, 0, 0, 0, 0, None) == -1
+    assert lib.a3_set_option(None, 0, 0) == -1
+    assert lib.a3_scores_workspace_bytes(None, 10) == 0
+    assert lib.a3_swiglu_rows(None, 0, None, None, 0, None) == -1
     assert lib.a3_topk_select(None, None, 0, 0, 0, None, None) == -1
     assert lib.a3_layer_workspace_bytes(None, 10) == 0
 

@@ -194,10 +194,51 @@ def test_scatter_and_gather_exact(a3mod):
     eng.close()
 
 
+def test_rerotate_destination_bounds(a3mod):
+    """A chunk whose slots leave the fused cache, or whose length exceeds the stated maximum, is skipped as a whole and
+    flagged; the others are written.  The buffer is larger than kv_len and filled with a canary, so that even an
+    unchecked write would stay inside the allocation."""
+    m = W.TINY_GQA
+    eng, _, dev = make_engine(a3mod, m)
+    lens = [40, 33, 50]
+    ck, cv = zip(*[W.make_cache_like(m, t, 3, c, std=1.0) for c, t in enumerate(lens)])
+    dk, dv = [to_dev(k, dev) for k in ck], [to_dev(v, dev) for v in cv]
+    kv_len, alloc = 100, 260
+    canary = 5.0
+
+    def run(offs, max_len, kv=kv_len):
+        Kf = torch.full((m.n_layers, alloc, m.n_kv_heads, m.head_dim), canary, dtype=torch.bfloat16, device=dev)
+        Vf = torch.full_like(Kf, canary)
+        eng.rope_rerotate(a3mod.chunk_table(dk, dv, offs), len(lens), max_len, Kf, Vf, kv_len=kv)
+        return f64(Kf), f64(Vf), eng.device_status()
+
+    # all inside: no flag, last chunk ends exactly at kv_len
+    K, V, st = run([0, 40, 50], 50)
+    assert st == 0 and (K[:, kv_len:] == canary).all() and (K[:, :33] != canary).any()
+    # the last chunk would end at slot 101: skipped whole, the others written, nothing beyond kv_len touched
+    K, V, st = run([0, 40, 51], 50)
+    assert st & a3mod.DEV_BAD_POSITION
+    assert (K[:, 73:] == canary).all() and (V[:, 73:] == canary).all()
+    np.testing.assert_array_equal(V[:, 0:40], cv[0])
+    np.testing.assert_array_equal(V[:, 40:73], cv[1])
+    # a chunk that starts beyond the cache altogether
+    K, V, st = run([0, 40, 150], 50)
+    assert st & a3mod.DEV_BAD_POSITION and (K[:, 73:] == canary).all()
+    # a chunk longer than the stated maximum: not silently truncated, skipped and flagged
+    K, V, st = run([0, 40, 50], 40)
+    assert st & a3mod.DEV_BAD_POSITION and (K[:, 73:] == canary).all() and (V[:, 73:] == canary).all()
+    np.testing.assert_array_equal(V[:, 0:40], cv[0])
+    # kv_len larger than a layer holds is rejected on the host
+    with pytest.raises(a3mod.A3Error):
+        run([0, 40, 50], 50, kv=alloc + 1)
+    eng.close()
+
+
 # ------------------------------------------------------------------ a5: top-p
 
 
-@pytest.mark.parametrize("n,k", [(1, 1), (7, 3), (512, 79), (5120, 772), (32768, 4920), (32768, 32768), (5000, 0), (1025, 1024)])
+@pytest.mark.parametrize("n,k", [(1, 1), (7, 3), (512, 79), (5120, 772), (32768, 4920), (32768, 32768), (5000, 0), (1025, 1024),
+                                 (33, 32), (1056, 17), (51200, 7680), (51201, 7680), (70001, 10500)])
 def test_topk_bit_exact(a3mod, n, k):
     eng, _, dev = make_engine(a3mod, W.TINY)
     rng = np.random.default_rng(n * 31 + k)
@@ -270,6 +311,71 @@ def test_query_scores_parity(a3mod, shape, n_ctx, nq, n_sys):
     for i in set(idx.tolist()) ^ set(ref.tolist()):
         assert abs(want[i] - tau) <= 1e-4 * tau
     assert eng.device_status() == 0
+    eng.close()
+
+
+@pytest.mark.parametrize("shape,n_ctx,nq", [(W.TINY, 300, 5), (W.TINY_GQA, 1000, 13), (W.TINY_G7, 700, 40), (W.LLAMA8B, 2500, 32),
+                                            (W.QWEN7B, 1500, 64), (W.TINY_GQA, 130, 1), (W.TINY_GQA, 40, 100)])
+def test_query_scores_kernel_variants(a3mod, shape, n_ctx, nq):
+    """The tensor-memory score kernel (one cache slot per thread, transposed product) and the warp-level MMA kernel it
+    replaced: each against the oracle within the stated 1e-3, each reproducible bit for bit, on shapes with one and
+    with several chunks of packed question rows per KV head, ragged key tiles, a question longer than the context,
+    and question rows whose causal limit cuts through several key tiles."""
+    from dataclasses import replace
+    m = replace(shape, n_layers=1, d_ff=256, vocab=8)
+    eng, _, dev = make_engine(a3mod, m)
+    rng = np.random.default_rng(19)
+    n = n_ctx + nq
+    q = W.bf16_round(rng.standard_normal((nq, m.n_q_heads, m.head_dim), dtype=np.float32) * 1.3)
+    K = W.bf16_round(rng.standard_normal((n, m.n_kv_heads, m.head_dim), dtype=np.float32) * 1.3)
+    qpos = np.arange(n_ctx, n)
+    model = oracle_model(m)
+    want = O.query_scores(q.astype(np.float64), qpos, K.astype(np.float64), model, 0, n)  # question slots scored too: masked tiles
+    _, lse = O.attention_rows(q.astype(np.float64), qpos, K.astype(np.float64), K.astype(np.float64), model)
+    dq, dK, dpos = to_dev(q, dev), to_dev(K, dev), torch.from_numpy(qpos.astype(np.int32)).to(dev)
+    try:
+        for variant in (1, 2):
+            eng.set_option(a3mod.OPT_SCORES_KERNEL, variant)
+            got = eng.query_scores(dq, dpos, dK, 0, n).cpu().numpy().astype(np.float64)
+            again = eng.query_scores(dq, dpos, dK, 0, n).cpu().numpy().astype(np.float64)
+            np.testing.assert_array_equal(got, again)
+            live = want > 1e-30
+            rel = np.abs(got[live] - want[live]) / want[live]
+            assert rel.max() <= 1e-3, (variant, rel.max())
+            assert np.abs(got[~live]).max(initial=0.0) <= 1e-30
+            got2 = eng.query_scores(dq, dpos, dK, 0, n, lse=to_dev(lse, dev, torch.float32)).cpu().numpy().astype(np.float64)
+            rel2 = np.abs(got2[live] - want[live]) / want[live]
+            assert rel2.max() <= 1e-3, (variant, rel2.max())
+    finally:
+        eng.set_option(a3mod.OPT_SCORES_KERNEL, 0)
+    assert eng.device_status() == 0
+    eng.close()
+
+
+def test_query_scores_statistics_pass_split(a3mod):
+    """The row log-sum-exps behind the scores come from a statistics pass whose keys are split over the SMs: the
+    scores of a3_query_scores without supplied log-sum-exps equal those with the oracle's log-sum-exps within the
+    stated tolerance on a cache of many key tiles, and unsorted question positions are flagged, not mis-scored."""
+    from dataclasses import replace
+    m = replace(W.LLAMA8B, n_layers=1, d_ff=256, vocab=8)
+    eng, _, dev = make_engine(a3mod, m)
+    rng = np.random.default_rng(23)
+    n_ctx, nq = 9000, 32
+    n = n_ctx + nq
+    q = W.bf16_round(rng.standard_normal((nq, m.n_q_heads, m.head_dim), dtype=np.float32) * 1.3)
+    K = W.bf16_round(rng.standard_normal((n, m.n_kv_heads, m.head_dim), dtype=np.float32) * 1.3)
+    qpos = np.arange(n_ctx, n)
+    model = oracle_model(m)
+    want = O.query_scores(q.astype(np.float64), qpos, K.astype(np.float64), model, 0, n_ctx)
+    dq, dK, dpos = to_dev(q, dev), to_dev(K, dev), torch.from_numpy(qpos.astype(np.int32)).to(dev)
+    got = eng.query_scores(dq, dpos, dK, 0, n_ctx).cpu().numpy().astype(np.float64)
+    rel = np.abs(got[:n_ctx] - want[:n_ctx]) / want[:n_ctx]
+    assert rel.max() <= 1e-3, rel.max()
+    assert eng.device_status() == 0
+    swapped = qpos.copy()
+    swapped[[3, 4]] = swapped[[4, 3]]
+    eng.query_scores(dq, torch.from_numpy(swapped.astype(np.int32)).to(dev), dK, 0, n_ctx)
+    assert eng.device_status() & a3mod.DEV_UNSORTED_ROWS
     eng.close()
 
 
@@ -389,11 +495,8 @@ def test_recompute_layer_rejects_bad_arguments(a3mod):
 
 def test_attention_key_split_matches_unsplit(a3mod):
     """The split over the keys (segments + combine kernel) gives the unsplit result up to rounding, reproducibly."""
-    import ctypes
     m = W.TINY_GQA
     eng, layers, dev = make_engine(a3mod, m, seed=5, w_std=0.05)
-    lib = a3mod._load()
-    lib.a3_internal_set_attn_split.argtypes = [ctypes.c_int]
     rng = np.random.default_rng(55)
     kv_len, M = 2100, 300  # 17 key tiles, 10 row tiles x 2 KV heads
     pos = np.sort(rng.choice(kv_len, size=M, replace=False))
@@ -403,7 +506,7 @@ def test_attention_key_split_matches_unsplit(a3mod):
     outs = {}
     try:
         for split in (1, 3, 3):
-            lib.a3_internal_set_attn_split(split)
+            eng.set_option(a3mod.OPT_ATTN_SPLIT, split)
             dX, dpos = to_dev(X, dev), torch.from_numpy(pos.astype(np.int32)).to(dev)
             dK, dV = to_dev(Kc[0], dev), to_dev(Vc[0], dev)
             lse = torch.empty((M, m.n_q_heads), dtype=torch.float32, device=dev)
@@ -411,7 +514,7 @@ def test_attention_key_split_matches_unsplit(a3mod):
             assert eng.device_status() == 0
             outs.setdefault(split, []).append((dX.clone(), lse.clone()))
     finally:
-        lib.a3_internal_set_attn_split(0)
+        eng.set_option(a3mod.OPT_ATTN_SPLIT, 0)
     a, b, c = outs[1][0], outs[3][0], outs[3][1]
     assert torch.equal(b[0], c[0]) and torch.equal(b[1], c[1])  # reproducible
     np.testing.assert_allclose(b[1].cpu().numpy(), a[1].cpu().numpy(), atol=1e-4)
@@ -547,11 +650,8 @@ def test_attention_two_row_tiles_per_cta(a3mod, shape, kv_len, M, grow):
     """The attention kernel that gives a CTA two row tiles (chosen by itself only for launches with many row tiles) on
     small cases, forced: against the oracle like the one-tile kernel, including logits that outgrow the exponent
     reference (grow), an odd number of row tiles and a single, ragged one."""
-    import ctypes
     m = shape
     eng, layers, dev = make_engine(a3mod, m, seed=21, w_std=0.05)
-    lib = a3mod._load()
-    lib.a3_internal_set_attn_pair.argtypes = [ctypes.c_int]
     model, weights = oracle_model(m), oracle_weights(layers)
     rng = np.random.default_rng(77)
     pos = np.sort(rng.choice(kv_len, size=M, replace=False))
@@ -575,14 +675,14 @@ def test_attention_two_row_tiles_per_cta(a3mod, shape, kv_len, M, grow):
     outs = []
     try:
         for rep in range(2):
-            lib.a3_internal_set_attn_pair(1)
+            eng.set_option(a3mod.OPT_ATTN_PAIR, 1)
             dX, dK, dV = to_dev(X, dev), to_dev(Kc, dev), to_dev(Vc, dev)
             lse = torch.empty((M, m.n_q_heads), dtype=torch.float32, device=dev)
             eng.recompute_layer(layer, dX, dpos, dK, dV, lse_out=lse)
             assert eng.device_status() == 0
             outs.append((dX, lse))
     finally:
-        lib.a3_internal_set_attn_pair(-1)
+        eng.set_option(a3mod.OPT_ATTN_PAIR, -1)
     assert torch.equal(outs[0][0], outs[1][0]) and torch.equal(outs[0][1], outs[1][1])  # reproducible
     gX = f64(outs[0][0])
     assert np.isfinite(gX).all()
@@ -598,11 +698,8 @@ def test_qkv_three_head_tiles(a3mod, shape, kv_len, M):
     804 rows of the Llama-shaped model), forced on small models whose tiles mix q, k and v heads and whose last tile
     holds fewer than three: K/V rows against the oracle, and everything bit for bit against the two-head tiling (the
     sum over the model dimension runs in the same order in both)."""
-    import ctypes
     m = shape
     eng, layers, dev = make_engine(a3mod, m, seed=33, w_std=0.05)
-    lib = a3mod._load()
-    lib.a3_internal_set_gemm_cfg.argtypes = [ctypes.c_int, ctypes.c_int, ctypes.c_int]
     model, weights = oracle_model(m), oracle_weights(layers)
     rng = np.random.default_rng(91)
     pos = np.sort(rng.choice(kv_len, size=M, replace=False))
@@ -614,13 +711,15 @@ def test_qkv_three_head_tiles(a3mod, shape, kv_len, M):
     outs = {}
     try:
         for bn, stages in ((384, 3), (0, 0)):
-            lib.a3_internal_set_gemm_cfg(2, bn, stages)
+            eng.set_option(a3mod.OPT_GEMM_BN_QKV, bn)
+            eng.set_option(a3mod.OPT_GEMM_STAGES_QKV, stages)
             dX, dK, dV = to_dev(X, dev), to_dev(Kc[layer], dev), to_dev(Vc[layer], dev)
             eng.recompute_layer(layer, dX, dpos, dK, dV)
             assert eng.device_status() == 0
             outs[bn] = (dX, dK, dV)
     finally:
-        lib.a3_internal_set_gemm_cfg(2, 0, 0)
+        eng.set_option(a3mod.OPT_GEMM_BN_QKV, 0)
+        eng.set_option(a3mod.OPT_GEMM_STAGES_QKV, 0)
     for a, b in zip(outs[384], outs[0]):
         assert torch.equal(a, b)
     Ko, Vo = Kc[layer].astype(np.float64), Vc[layer].astype(np.float64)
@@ -641,12 +740,8 @@ def test_swiglu_narrow_column_tiles(a3mod, shape, M, g):
     """The SwiGLU GEMM gives the column tiles of a partly filled last wave fewer features each (by itself only for
     grids of several waves); forced here on half the column tiles, with widths that leave a remainder of 8-column
     pieces and a last tile reaching past the matrix: bit for bit against the uniform tiling, and against the oracle."""
-    import ctypes
     m = shape
     eng, layers, dev = make_engine(a3mod, m, seed=41, w_std=0.05)
-    lib = a3mod._load()
-    lib.a3_internal_set_gemm_narrow.argtypes = [ctypes.c_int]
-    lib.a3_internal_set_swiglu_pair.argtypes = [ctypes.c_int]
     model, weights = oracle_model(m), oracle_weights(layers)
     rng = np.random.default_rng(17)
     kv_len = 3 * M
@@ -658,16 +753,16 @@ def test_swiglu_narrow_column_tiles(a3mod, shape, M, g):
     dpos = torch.from_numpy(pos.astype(np.int32)).to(dev)
     outs = {}
     try:
-        lib.a3_internal_set_swiglu_pair(0)  # the one-CTA-per-tile kernel (the CTA-pair kernel is the default)
+        eng.set_option(a3mod.OPT_SWIGLU_PAIR, 0)  # the one-CTA-per-tile kernel (the CTA-pair kernel is the default)
         for mode in (g, 0):
-            lib.a3_internal_set_gemm_narrow(mode)
+            eng.set_option(a3mod.OPT_SWIGLU_NARROW, mode)
             dX, dK, dV = to_dev(X, dev), to_dev(Kc[layer], dev), to_dev(Vc[layer], dev)
             eng.recompute_layer(layer, dX, dpos, dK, dV)
             assert eng.device_status() == 0
             outs[mode] = dX
     finally:
-        lib.a3_internal_set_gemm_narrow(1)
-        lib.a3_internal_set_swiglu_pair(1)
+        eng.set_option(a3mod.OPT_SWIGLU_NARROW, 1)
+        eng.set_option(a3mod.OPT_SWIGLU_PAIR, 1)
     assert torch.equal(outs[g], outs[0])
     Ko, Vo = Kc[layer].astype(np.float64), Vc[layer].astype(np.float64)
     Xo, parts = O.recompute_layer(X.astype(np.float64), pos, weights[layer], model, Ko, Vo, rnd=O.round_bf16, return_parts=True)
@@ -681,11 +776,8 @@ def test_swiglu_pair_kernel_matches_one_cta_kernel(a3mod, shape, M):
     evenly, persistent schedule with double-buffered accumulators) against the one-CTA-per-tile kernel it replaced:
     two independent kernels, one formula, the same sum order over the model dimension - bit for bit; row counts of one
     row, of one ragged token tile, of several tiles and of several units per CTA pair; and against the oracle."""
-    import ctypes
     m = shape
     eng, layers, dev = make_engine(a3mod, m, seed=51, w_std=0.05)
-    lib = a3mod._load()
-    lib.a3_internal_set_swiglu_pair.argtypes = [ctypes.c_int]
     model, weights = oracle_model(m), oracle_weights(layers)
     rng = np.random.default_rng(23)
     kv_len = 2 * M + 40
@@ -698,13 +790,13 @@ def test_swiglu_pair_kernel_matches_one_cta_kernel(a3mod, shape, M):
     outs = {}
     try:
         for mode in (1, 0, 1):
-            lib.a3_internal_set_swiglu_pair(mode)
+            eng.set_option(a3mod.OPT_SWIGLU_PAIR, mode)
             dX, dK, dV = to_dev(X, dev), to_dev(Kc[layer], dev), to_dev(Vc[layer], dev)
             eng.recompute_layer(layer, dX, dpos, dK, dV)
             assert eng.device_status() == 0
             outs.setdefault(mode, []).append(dX)
     finally:
-        lib.a3_internal_set_swiglu_pair(1)
+        eng.set_option(a3mod.OPT_SWIGLU_PAIR, 1)
     assert torch.equal(outs[1][0], outs[1][1])  # reproducible
     assert torch.equal(outs[1][0], outs[0][0])
     Ko, Vo = Kc[layer].astype(np.float64), Vc[layer].astype(np.float64)
@@ -719,11 +811,8 @@ def test_residual_persistent_pair_kernel_matches_tile_kernel(a3mod, shape, M):
     (chosen by itself only when a CTA pair gets several units, i.e. for thousands of rows), forced on small models -
     among them one whose width (896) leaves the last 256-feature block half empty - against the 256 x 256 CTA-pair tile
     kernel: bit for bit, and against the oracle."""
-    import ctypes
     m = shape
     eng, layers, dev = make_engine(a3mod, m, seed=61, w_std=0.05)
-    lib = a3mod._load()
-    lib.a3_internal_set_residual_t.argtypes = [ctypes.c_int]
     model, weights = oracle_model(m), oracle_weights(layers)
     rng = np.random.default_rng(29)
     kv_len = 2 * M + 40
@@ -736,13 +825,13 @@ def test_residual_persistent_pair_kernel_matches_tile_kernel(a3mod, shape, M):
     outs = {}
     try:
         for mode in (2, 0):
-            lib.a3_internal_set_residual_t(mode)
+            eng.set_option(a3mod.OPT_RESIDUAL_T, mode)
             dX, dK, dV = to_dev(X, dev), to_dev(Kc[layer], dev), to_dev(Vc[layer], dev)
             eng.recompute_layer(layer, dX, dpos, dK, dV)
             assert eng.device_status() == 0
             outs[mode] = dX
     finally:
-        lib.a3_internal_set_residual_t(1)
+        eng.set_option(a3mod.OPT_RESIDUAL_T, 1)
     assert torch.equal(outs[2], outs[0])
     Ko, Vo = Kc[layer].astype(np.float64), Vc[layer].astype(np.float64)
     Xo, parts = O.recompute_layer(X.astype(np.float64), pos, weights[layer], model, Ko, Vo, rnd=O.round_bf16, return_parts=True)
@@ -755,12 +844,8 @@ def test_persistent_gemms_row_count_sweep(a3mod, shape):
     """Row counts around every boundary of the persistent CTA-pair GEMMs (one row, token tiles of 16, one full tile of
     256, one row more, several tiles, several units per pair): SwiGLU and both residual GEMMs forced onto them, against
     the tile kernels, bit for bit; no device status bit, no non-finite value."""
-    import ctypes
     m = shape
     eng, layers, dev = make_engine(a3mod, m, seed=71, w_std=0.05, max_pos=3000)
-    lib = a3mod._load()
-    lib.a3_internal_set_swiglu_pair.argtypes = [ctypes.c_int]
-    lib.a3_internal_set_residual_t.argtypes = [ctypes.c_int]
     kv_len = 2600
     layer = m.n_layers - 1
     g = torch.Generator(device=dev)
@@ -772,8 +857,8 @@ def test_persistent_gemms_row_count_sweep(a3mod, shape):
             K = torch.randn((kv_len, m.n_kv_heads, m.head_dim), device=dev, generator=g).to(torch.bfloat16)
             outs = []
             for sw, rs in ((1, 2), (0, 0)):
-                lib.a3_internal_set_swiglu_pair(sw)
-                lib.a3_internal_set_residual_t(rs)
+                eng.set_option(a3mod.OPT_SWIGLU_PAIR, sw)
+                eng.set_option(a3mod.OPT_RESIDUAL_T, rs)
                 X, Kc, Vc = X0.clone(), K.clone(), K.clone()
                 eng.recompute_layer(layer, X, pos, Kc, Vc)
                 assert eng.device_status() == 0, M
@@ -781,8 +866,8 @@ def test_persistent_gemms_row_count_sweep(a3mod, shape):
             assert torch.isfinite(outs[0].float()).all(), M
             assert torch.equal(outs[0], outs[1]), M
     finally:
-        lib.a3_internal_set_swiglu_pair(1)
-        lib.a3_internal_set_residual_t(1)
+        eng.set_option(a3mod.OPT_SWIGLU_PAIR, 1)
+        eng.set_option(a3mod.OPT_RESIDUAL_T, 1)
     eng.close()
 
 
@@ -793,11 +878,8 @@ def test_attention_logit_spikes(a3mod, pair):
     FMA pipe, where the exponent arithmetic would wrap around for such inputs (and the key, the last one above all,
     would silently get weight zero) if they were not clamped into the range the overflow guard catches.  Both
     attention kernels, against the exact softmax of the oracle."""
-    import ctypes
     m = W.TINY_GQA
     eng, layers, dev = make_engine(a3mod, m, seed=13, w_std=0.05)
-    lib = a3mod._load()
-    lib.a3_internal_set_attn_pair.argtypes = [ctypes.c_int]
     model, weights = oracle_model(m), oracle_weights(layers)
     rng = np.random.default_rng(313)
     kv_len, M = 1500, 131
@@ -827,10 +909,10 @@ def test_attention_logit_spikes(a3mod, pair):
     dK, dV = to_dev(Kc, dev), to_dev(Vc, dev)
     lse = torch.empty((M, m.n_q_heads), dtype=torch.float32, device=dev)
     try:
-        lib.a3_internal_set_attn_pair(1 if pair else 0)
+        eng.set_option(a3mod.OPT_ATTN_PAIR, 1 if pair else 0)
         eng.recompute_layer(layer, dX, dpos, dK, dV, lse_out=lse)
     finally:
-        lib.a3_internal_set_attn_pair(-1)
+        eng.set_option(a3mod.OPT_ATTN_PAIR, -1)
     assert eng.device_status() == 0
     gX = f64(dX)
     assert np.isfinite(gX).all()
@@ -843,14 +925,10 @@ def test_attention_logit_spikes(a3mod, pair):
 def test_swiglu_far_negative_gate(a3mod):
     """Gate pre-activations far below -88.7 (where e^-g overflows fp32): silu(g) u must come out as a signed zero (the
     kernels use a fast exponential and an approximate reciprocal: inf and NaN must not leak out of that corner); and
-    far above, as g u.  One layer's SwiGLU GEMM alone (tuning hook), both kernels, against the oracle's silu on the
+    far above, as g u.  One layer's SwiGLU GEMM alone (a3_swiglu_rows), both kernels, against the oracle's silu on the
     same products."""
-    import ctypes
     m = W.TINY
     eng, layers, dev = make_engine(a3mod, m, seed=81, w_std=0.05)
-    lib = a3mod._load()
-    lib.a3_internal_set_swiglu_pair.argtypes = [ctypes.c_int]
-    lib.a3_internal_swiglu.argtypes = [ctypes.c_void_p, ctypes.c_int, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int, ctypes.c_void_p]
     wg, wu = layers[0]["w_gate"].astype(np.float64), layers[0]["w_up"].astype(np.float64)
     rng = np.random.default_rng(37)
     M = 70
@@ -866,15 +944,14 @@ def test_swiglu_far_negative_gate(a3mod):
     dX = to_dev(X, dev)
     try:
         for mode in (1, 0):
-            lib.a3_internal_set_swiglu_pair(mode)
+            eng.set_option(a3mod.OPT_SWIGLU_PAIR, mode)
             out = torch.full((M, m.d_ff), float("nan"), dtype=torch.bfloat16, device=dev)
-            st = torch.cuda.current_stream().cuda_stream
-            assert lib.a3_internal_swiglu(eng._h, 0, dX.data_ptr(), out.data_ptr(), M, st) == 0
+            eng.swiglu_rows(0, dX, out)
             got = f64(out)
             assert eng.device_status() == 0
             assert np.isfinite(got).all(), mode
             np.testing.assert_allclose(got, want, rtol=2.0 ** -7, atol=2e-3)
             assert np.all(got[np.arange(10), np.arange(10)] == 0.0)
     finally:
-        lib.a3_internal_set_swiglu_pair(1)
+        eng.set_option(a3mod.OPT_SWIGLU_PAIR, 1)
     eng.close()
