@@ -349,7 +349,8 @@ scores_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
           ld32(tmem_base + b * 256 + lane_addr + cc * 32, x);
           wait_ld();
           const int rb = r0 + cc * 32;
-          if (rb + 32 <= r0 + n_valid && !need_mask && vec_ok) {
+          const bool whole = rb + 32 <= r0 + n_valid && vec_ok;  // 32 live packed rows, tables readable as vectors
+          if (whole && !need_mask) {
 #pragma unroll
             for (int e = 0; e < 32; e += 4) {
               const float4 l4 = *reinterpret_cast<const float4*>(l2g + rb + e);
@@ -357,6 +358,19 @@ scores_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
               acc[1] += ex2_approx(fmaf(x[e + 1], p.scale_log2, -l4.y));
               acc[2] += ex2_approx(fmaf(x[e + 2], p.scale_log2, -l4.z));
               acc[3] += ex2_approx(fmaf(x[e + 3], p.scale_log2, -l4.w));
+            }
+          } else if (whole) {
+            // the key tiles around the question: a slot counts for a row only up to the row's own position
+#pragma unroll
+            for (int e = 0; e < 32; e += 4) {
+              const float4 l4 = *reinterpret_cast<const float4*>(l2g + rb + e);
+              const int4 m4 = *reinterpret_cast<const int4*>(postab + rb + e);
+              const float p0 = ex2_approx(fmaf(x[e], p.scale_log2, -l4.x)), p1 = ex2_approx(fmaf(x[e + 1], p.scale_log2, -l4.y));
+              const float p2 = ex2_approx(fmaf(x[e + 2], p.scale_log2, -l4.z)), p3 = ex2_approx(fmaf(x[e + 3], p.scale_log2, -l4.w));
+              acc[0] += key <= m4.x ? p0 : 0.f;
+              acc[1] += key <= m4.y ? p1 : 0.f;
+              acc[2] += key <= m4.z ? p2 : 0.f;
+              acc[3] += key <= m4.w ? p3 : 0.f;
             }
           } else {
 #pragma unroll

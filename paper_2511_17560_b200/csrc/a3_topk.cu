@@ -1,9 +1,10 @@
 // Selection Re = top_p(s) (Eq. 3): block-radix select on the order-preserving integer image of the fp32 scores.
 // One CTA per score array.  The scores are read from global memory once, as integer keys into shared memory (up to
 // TK_SMEM_KEYS of them; longer arrays are re-read from global memory in every pass).  Four 8-bit histogram passes
-// find the key of the k-th largest score: a warp adds up equal digits among its lanes before it touches the
-// histogram (scores of one request share their leading bits, so a plain atomic per element would serialise on one
-// bin), and the bin of the k-th element is found by a parallel suffix sum over the 256 bins.  The emission is
+// find the key of the k-th largest score: the warps count into TK_HISTS private histograms (a warp whose lanes all
+// hold the same digit - the rule in the first pass, since the scores of one request share their leading bits - adds
+// 32 with one instruction instead of serialising 32 atomics on one bin), the histograms are summed, and the bin of
+// the k-th element is found by a parallel suffix sum over the 256 bins.  The emission is
 // ordered: every warp owns a contiguous span of the slots, counts what it will emit, and after one exchange of the
 // 32 warp totals writes every slot above the threshold key plus, in slot order, as many slots equal to it as are
 // still needed.  The result is exact: ties go to the lower slot and the output is ascending.
@@ -13,7 +14,8 @@ namespace a3 {
 
 constexpr int TK_THREADS = 1024;
 constexpr int TK_WARPS = TK_THREADS / 32;
-constexpr int TK_SMEM_KEYS = 50 * 1024;  // 200 KiB of keys
+constexpr int TK_HISTS = 16;              // private histograms (warp w counts into number w % TK_HISTS)
+constexpr int TK_SMEM_KEYS = 48 * 1024;  // 192 KiB of keys
 
 __device__ __forceinline__ uint32_t score_key(float s) {
   uint32_t u = __float_as_uint(s);
@@ -24,6 +26,7 @@ template <bool IN_SMEM>
 __device__ __forceinline__ void topk_body(const float* __restrict__ s, uint32_t* __restrict__ keys, int cand_begin, int n, int k,
                                           int32_t* __restrict__ idx_out, uint32_t* status) {
   __shared__ unsigned int hist[256];
+  __shared__ unsigned int whist[TK_HISTS][256];
   __shared__ unsigned int warp_tot[8];
   __shared__ unsigned int s_prefix, s_remaining;
   __shared__ unsigned int warp_gt[TK_WARPS], warp_eq[TK_WARPS];
@@ -32,6 +35,7 @@ __device__ __forceinline__ void topk_body(const float* __restrict__ s, uint32_t*
 
   // ---- load: scores -> keys (shared memory), non-finite scores flagged
   bool nonfinite = false;
+#pragma unroll 4
   for (int i = tid; i < n; i += TK_THREADS) {
     const float v = s[i];
     if (!(fabsf(v) <= 3.0e38f)) nonfinite = true;
@@ -44,16 +48,28 @@ __device__ __forceinline__ void topk_body(const float* __restrict__ s, uint32_t*
   unsigned int remaining = (unsigned int)k;  // rank (1-based, from the top) inside the current bucket
   const int n_round = (n + 31) & ~31;        // whole warps walk the array, so that the lanes can vote together
   for (int shift = 24; shift >= 0; shift -= 8) {
-    if (tid < 256) hist[tid] = 0;
+    for (int i = tid; i < TK_HISTS * 256; i += TK_THREADS) (&whist[0][0])[i] = 0;
     __syncthreads();
+    unsigned int* mine = whist[warp % TK_HISTS];
     for (int i = tid; i < n_round; i += TK_THREADS) {
       uint32_t digit = 0xFFFFFFFFu;  // lanes with nothing to count
       if (i < n) {
         const uint32_t key = key_at(i);
         if ((key & mask) == prefix) digit = (key >> shift) & 255u;
       }
-      const unsigned int same = __match_any_sync(0xffffffffu, digit);
-      if (digit != 0xFFFFFFFFu && (same & ((1u << lane) - 1u)) == 0) atomicAdd(&hist[digit], (unsigned int)__popc(same));
+      const uint32_t first = __shfl_sync(0xffffffffu, digit, 0);
+      if (__all_sync(0xffffffffu, digit == first)) {
+        if (lane == 0 && digit != 0xFFFFFFFFu) atomicAdd(&mine[digit], 32u);
+      } else if (digit != 0xFFFFFFFFu) {
+        atomicAdd(&mine[digit], 1u);
+      }
+    }
+    __syncthreads();
+    if (tid < 256) {
+      unsigned int v = 0;
+#pragma unroll
+      for (int w = 0; w < TK_HISTS; ++w) v += whist[w][tid];
+      hist[tid] = v;
     }
     __syncthreads();
     // suffix sums over the bins: S[d] = count of elements with digit >= d; the k-th element's digit is the largest d

@@ -238,7 +238,7 @@ def test_rerotate_destination_bounds(a3mod):
 
 
 @pytest.mark.parametrize("n,k", [(1, 1), (7, 3), (512, 79), (5120, 772), (32768, 4920), (32768, 32768), (5000, 0), (1025, 1024),
-                                 (33, 32), (1056, 17), (51200, 7680), (51201, 7680), (70001, 10500)])
+                                 (33, 32), (1056, 17), (49152, 7000), (49153, 7000), (70001, 10500)])
 def test_topk_bit_exact(a3mod, n, k):
     eng, _, dev = make_engine(a3mod, W.TINY)
     rng = np.random.default_rng(n * 31 + k)
