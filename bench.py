@@ -1,15 +1,19 @@
 #!/usr/bin/env python
 """Benchmark of the A^3 fusion hot path: context tokens fused per second on B200.
 
-A step is one whole fusion request (position recovery of all layers, the leading full block, selection,
-and the recompute layers) on synthetic inputs of the configured shape.  One JSON line is printed by rank 0.
+A step is one whole fusion request (position recovery of all layers, the leading full block, selection, and the
+recompute layers) on synthetic inputs of the configured shape.  One JSON line is printed by rank 0.
 
-  python bench.py [--gpus N] [--steps K] [--warmup W] [--impl a3|reference] [--config NAME]
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--impl a3|reference] [--config NAME] [--ratio R]
 
-N > 1 runs N independent replicas (one process per GPU, launched with torch.distributed.run); the path has no
-exchange step, so there is no data-path collective: only the barrier and the max-over-ranks of the time.
-`--impl reference` times the CPU oracle (as it stands, fp32) on the host cores on a bounded sample of the same
-workload.  `--config llama8b_batch16` times the batched-serving workload (16 requests, `a3_fuse_batch`) instead.
+Without --config the headline workload is the largest single-GPU request, `llama8b_64x512` (Llama-3-8B-shaped,
+64 chunks x 512 tokens = 32 768 context tokens, relevance planted in two chunks), and the other configurations are
+measured in the same run and reported under `configs` in the same line: `llama8b_10x512`, the recompute-ratio sweep
+of `qwen7b_16xU` (5, 10, 15, 30 %) and the batched-serving workload `llama8b_batch16`.  With --config only that
+workload is measured.  N > 1 runs N independent replicas (one process per GPU, launched with
+torch.distributed.run); the path has no exchange step, so there is no data-path collective: only the barrier and
+the max-over-ranks of the time.  `--impl reference` times the CPU oracle (as it stands, fp32) on the host cores on
+a bounded sample of the same workload.
 """
 from __future__ import annotations
 
@@ -26,22 +30,29 @@ ROOT = os.path.dirname(os.path.abspath(__file__))
 if ROOT not in sys.path:
     sys.path.insert(0, ROOT)
 
-# DRAM bytes (read + write) per launch from the ncu capture summarised in profiles/gemm_kernels_llama8b_2layer.txt:
-# the SwiGLU GEMM of a sparse layer (M = 804) and of the full block (M = 5152) at Llama-8B width.
+# DRAM bytes (read + write) per launch of the dominant kernel classes from the ncu captures summarised under profiles/
+# (gemm_kernels_llama8b_2layer.txt: SwiGLU GEMM of a sparse layer, M = 804, and of the full block, M = 5152;
+# attention_kernels_*: see that file).  Used for `roofline.traffic` of the workloads they were captured on.
 NCU_TRAFFIC = {("llama8b_10x512", "gemm_swiglu"): {"sparse": 243.44e6 + 18.51e6, "full": 418.15e6 + 140.63e6}}
 
 METRIC = "context_tokens_fused_per_s"
 UNIT = "tokens/s"
-FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+HEADLINE = "llama8b_64x512"
+PLANTED_CHUNKS = (20, 45)  # the two chunks whose embeddings share a direction with the question's (cosine 0.5)
+SWEEP_RATIOS = (0.05, 0.10, 0.15, 0.30)
+FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "sustained_mhz": 1300.0}
 
 
 def load_peaks():
+    """Measured peaks of this machine (generated file) and the SM clock the sustained matmul figure was taken at."""
     path = os.path.join(ROOT, "MEASURED_PEAKS.json")
     if os.path.exists(path):
         try:
             with open(path) as f:
                 p = json.load(f)
-            return {k: float(p[k]) for k in FALLBACK_PEAKS}, "measured"
+            out = {k: float(p[k]) for k in ("hbm_gbs", "bf16_tflops", "bf16_tflops_sustained")}
+            out["sustained_mhz"] = float(p.get("clocks_under_load", {}).get("sm_mhz_median") or FALLBACK_PEAKS["sustained_mhz"])
+            return out, "measured"
         except Exception:
             pass
     return dict(FALLBACK_PEAKS), "fallback"
@@ -79,10 +90,10 @@ class ClockSampler:
     Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
          "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
 
-    def __init__(self, gpu_index: int):
+    def __init__(self, gpu_index: int, period_ms: int = 100):
         self.proc = None
         try:
-            self.proc = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits", "-lms", "100",
+            self.proc = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits", "-lms", str(period_ms),
                                           "-i", str(gpu_index)], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
         except Exception:
             self.proc = None
@@ -154,11 +165,23 @@ def aggregate_value(units_per_rank_per_step: float, steps: int, world: int, max_
     return units_per_rank_per_step * steps * world / max_seconds
 
 
+def workload_config(name, m, r, p, world, ratio=None, extra=None):
+    """The `config` object of a JSON line: the same keys in the CUDA arm and in the reference arm."""
+    cfg = {"workload": name, "model": m.name, "chunks": len(r.chunk_lens), "n_ctx": r.n_ctx, "n_question": r.n_question,
+           "recompute_ratio": r.ratio if ratio is None else ratio, "n_recompute": p, "select_layer": r.select_layer,
+           "replicas": world, "layers": m.n_layers,
+           "planted_chunks": list(PLANTED_CHUNKS) if name == HEADLINE else None,
+           "l2": "inputs larger than L2: every step streams the stack's weights and the fused cache"}
+    if extra:
+        cfg.update(extra)
+    return cfg
+
+
 # ------------------------------------------------------------------ the CPU oracle arm
 
 
 def oracle_sample(config: str, seed: int = 0):
-    """Builds the inputs of the bounded oracle sample: 3 layers of the stack at full width, random caches."""
+    """Inputs of the bounded oracle sample: 3 layers of the stack at full width, random caches of the workload's shape."""
     from dataclasses import replace
     from oracle import a3_oracle as O
     from paper_2511_17560_b200 import workloads as W
@@ -171,34 +194,42 @@ def oracle_sample(config: str, seed: int = 0):
     return dict(O=O, m_full=m_full, m=m, r=r, model=model, weights=weights, x0=x0, ck=ck, cv=cv)
 
 
-def oracle_step(S, stride: int = 4):
-    """One bounded sample of the request on the oracle (fp32), extrapolated to the whole request.
+def oracle_strides(n: int, M: int, budget_rows: int):
+    """Row strides of the bounded sample: about `budget_rows` rows through the full block and through the recompute layer."""
+    return max(1, -(-n // budget_rows)), max(1, -(-M // budget_rows))
+
+
+def oracle_step(S, stride_full: int = 4, stride_rows: int = 1):
+    """One bounded sample of the request on the oracle (fp32), with the factors that scale it to the whole request.
 
     Timed pieces, each the oracle's own function: position recovery of one layer (x L); one full block on every
-    `stride`-th row (x stride x select_layer); the selection layer's norm + QKV on every `stride`-th row (x stride),
-    scores and top-p at full size; one recompute layer on the p + |Q| carried rows (x (L - select_layer)).
+    `stride_full`-th row (x stride_full x select_layer); the selection layer's norm + QKV on every `stride_full`-th row
+    (x stride_full), scores and top-p at full size; one recompute layer on every `stride_rows`-th of the p + |Q| carried
+    rows (x stride_rows x (L - select_layer)).  Returns (measured seconds, extrapolated seconds, parts).
     """
     O, m, mf, r, model, weights = S["O"], S["m"], S["m_full"], S["r"], S["model"], S["weights"]
     dt = np.float32
     L, ls = mf.n_layers, min(r.select_layer, m.n_layers - 1)
     n, nq = r.n, r.n_question
     one = O.Model(1, m.d_model, m.n_q_heads, m.n_kv_heads, m.head_dim, m.d_ff, m.rope_theta, m.rms_eps, m.rope_layout)
-    t = {}
+    meas, t = {}, {}
     c0 = time.perf_counter()
     K, V = O.position_recovery(S["ck"], S["cv"], r.offsets, n, one, dtype=dt)
-    t["position_recovery"] = (time.perf_counter() - c0) * L
+    meas["position_recovery"] = time.perf_counter() - c0
+    t["position_recovery"] = meas["position_recovery"] * L
     K, V = K[0], V[0]
     X = S["x0"].astype(dt)
-    sub = np.arange(0, n, stride)
+    sub = np.arange(0, n, stride_full)
     c0 = time.perf_counter()
     if ls > 0:
         O.recompute_layer(X[sub], sub, weights[0], model, K, V)
-    t["full_blocks"] = (time.perf_counter() - c0) * stride * ls
+    meas["full_blocks"] = time.perf_counter() - c0
+    t["full_blocks"] = meas["full_blocks"] * stride_full * ls
     c0 = time.perf_counter()
     w = weights[ls]
     a = O.rmsnorm(X[sub], w.attn_norm, model.rms_eps)
     O.project_qkv(a, w, model, sub)
-    t_kv = (time.perf_counter() - c0) * stride
+    t_kv = time.perf_counter() - c0
     c0 = time.perf_counter()
     q_rows = np.arange(r.n_ctx, n)
     aq = O.rmsnorm(X[q_rows], w.attn_norm, model.rms_eps)
@@ -206,12 +237,34 @@ def oracle_step(S, stride: int = 4):
     s = O.query_scores(q, q_rows, K, model, 0, r.n_ctx)
     p = O.recompute_count(r.ratio, n, r.n_ctx)
     Re = O.topk_select(s, 0, r.n_ctx, p)
-    t["selection"] = t_kv + (time.perf_counter() - c0)
-    R = np.concatenate([Re, q_rows])
+    t_sel = time.perf_counter() - c0
+    meas["selection"] = t_kv + t_sel
+    t["selection"] = t_kv * stride_full + t_sel
+    R = np.concatenate([Re, q_rows])[::stride_rows]
     c0 = time.perf_counter()
     O.recompute_layer(X[R], R, weights[min(ls + 1, m.n_layers - 1)], model, K, V)
-    t["recompute_layers"] = (time.perf_counter() - c0) * (L - ls)
-    return sum(t.values()), t
+    meas["recompute_layers"] = time.perf_counter() - c0
+    t["recompute_layers"] = meas["recompute_layers"] * stride_rows * (L - ls)
+    return sum(meas.values()), sum(t.values()), t
+
+
+def oracle_full_request(config: str, seed: int = 0):
+    """The oracle's fuse_request on the WHOLE request (every layer, every row; fp32), not extrapolated.  The stack
+    cycles through three distinct layers' weights and the chunk caches are random values of the workload's shape:
+    the arithmetic, the shapes and the layer count are the request's own, the values do not matter for a timing."""
+    from dataclasses import replace
+    from oracle import a3_oracle as O
+    from paper_2511_17560_b200 import workloads as W
+    m, r = W.request_for(config)
+    model = O.Model(m.n_layers, m.d_model, m.n_q_heads, m.n_kv_heads, m.head_dim, m.d_ff, m.rope_theta, m.rms_eps, m.rope_layout)
+    three = [O.LayerWeights(**w) for w in W.make_weights(replace(m, n_layers=min(3, m.n_layers)), seed)]
+    weights = [three[l % len(three)] for l in range(m.n_layers)]
+    x0 = W.make_embeddings_device(m, r.n, "cpu", seed).float().numpy()
+    ck, cv = zip(*[W.make_cache_like(m, t, seed, c, std=1.28) for c, t in enumerate(r.chunk_lens)])
+    t0 = time.perf_counter()
+    res = O.fuse_request(ck, cv, x0, r.n_question, weights, model, r.ratio, select_layer=r.select_layer, dtype=np.float32)
+    seconds = time.perf_counter() - t0
+    return seconds, r, res.trace.get("seconds", {})
 
 
 def oracle_threads() -> int:
@@ -223,28 +276,36 @@ def oracle_threads() -> int:
 
 
 def run_reference(args):
+    """The reference arm: the oracle on the host cores.  A step is one bounded sample of the workload (sized so that
+    the run ends within minutes); `ms_per_step` is the measured time of that sample, `value` the metric it
+    extrapolates to for the whole request (`extrapolated`: true)."""
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
         return
-    S = oracle_sample(args.config)
-    r = S["r"]
+    from paper_2511_17560_b200 import workloads as W
+    config = args.config or HEADLINE
+    S = oracle_sample(config)
+    m, r = S["m_full"], S["r"]
+    p = S["O"].recompute_count(r.ratio, r.n, r.n_ctx)
+    sf, sr = oracle_strides(r.n, p + r.n_question, args.oracle_rows)
     for _ in range(args.warmup):
-        oracle_step(S)
-    secs, parts = [], None
+        oracle_step(S, sf, sr)
+    meas, extr, parts = [], [], None
     for _ in range(args.steps):
-        s, parts = oracle_step(S)
-        secs.append(s)
-    t = float(np.mean(secs))
-    value = r.n_ctx / t
-    sample = ("per step: position recovery of 1 layer, one full block and the selection-layer QKV on every 4th row, "
-              "scores + top-p at full size, one recompute layer on the p+|Q| rows; scaled to all layers/rows "
+        a, b, parts = oracle_step(S, sf, sr)
+        meas.append(a)
+        extr.append(b)
+    t_meas, t_extr = float(np.mean(meas)), float(np.mean(extr))
+    value = r.n_ctx / t_extr
+    sample = (f"per step: position recovery of 1 layer, one full block and the selection-layer QKV on every {sf}-th row, scores + "
+              f"top-p at full size, one recompute layer on every {sr}-th of the p+|Q| rows; scaled to all layers/rows "
               "(extrapolated); oracle in fp32 with random caches of the workload's shape")
     line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
-            "warmup": args.warmup, "ms_per_step": t * 1e3, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
-            "dtype": "f32", "data": "synthetic",
-            "config": {"workload": args.config, "recompute_ratio": r.ratio, "n_ctx": r.n_ctx, "n_question": r.n_question},
+            "warmup": args.warmup, "ms_per_step": t_meas * 1e3, "extrapolated": True, "extrapolated_request_ms": t_extr * 1e3,
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+            "config": workload_config(config, m, r, p, args.gpus),
             "cpu_baseline": {"value": value, "unit": UNIT, "cores": oracle_threads(), "kind": "oracle", "sample": sample,
-                             "seconds_by_phase": parts},
+                             "seconds_by_phase_extrapolated": parts},
             "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
     print(json.dumps(line), flush=True)
 
@@ -252,11 +313,11 @@ def run_reference(args):
 # ------------------------------------------------------------------ the CUDA arm
 
 
-def precompute_chunks(eng, m, r, x0, dev):
+def precompute_chunks(eng, m, lens, offsets, x0, dev):
     """Eq. 1 on the GPU: each chunk alone at local positions 0..T-1 through every layer (same kernels, all rows)."""
     import torch
     ck, cv = [], []
-    for o, t in zip(r.offsets, r.chunk_lens):
+    for o, t in zip(offsets, lens):
         K = torch.zeros((m.n_layers, t, m.n_kv_heads, m.head_dim), dtype=torch.bfloat16, device=dev)
         V = torch.zeros_like(K)
         eng.precompute_chunk(x0[o:o + t].clone(), K, V)
@@ -265,28 +326,177 @@ def precompute_chunks(eng, m, r, x0, dev):
     return ck, cv
 
 
-def run_a3_batch(args):
-    """Batched serving (16 requests over a pool of 200 precomputed chunks, Llama-shaped): `a3_fuse_batch` timed as one
-    step; aggregate context tokens per second and the spread of the single-request latencies.  Context, not the
-    headline: one JSON line of the same shape, `config.workload` = llama8b_batch16."""
-    import torch
-    from paper_2511_17560_b200 import a3
-    from paper_2511_17560_b200 import workloads as W
+class Timer:
+    """CUDA-event timing of `steps` calls on the launching stream, bracketed by a barrier and a synchronize on both
+    sides; the maximum over ranks is returned."""
 
-    rank, world, local = dist_setup(args.gpus)
-    torch.cuda.set_device(local)
-    dev = torch.device("cuda", local)
-    peaks, _ = load_peaks()
-    m = W.LLAMA8B
-    if args.layers:
-        from dataclasses import replace
-        m = replace(m, n_layers=args.layers)
+    def __init__(self, stream, dev):
+        import torch
+        self.torch, self.stream, self.dev = torch, stream, dev
+        self.e0, self.e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+
+    def run(self, call, steps, sync_ranks=True):
+        torch = self.torch
+        if sync_ranks:
+            barrier()
+        torch.cuda.synchronize()
+        self.e0.record(self.stream)
+        for _ in range(steps):
+            call()
+        self.e1.record(self.stream)
+        torch.cuda.synchronize()
+        if sync_ranks:
+            barrier()
+        sec = self.e0.elapsed_time(self.e1) / 1e3
+        return max_over_ranks(sec, self.dev) if sync_ranks else sec
+
+
+def kernel_table(prof, steps, flops, bts, peaks, run_mhz):
+    """Per kernel class: time per step and achieved rate against the measured peaks.  `frac` is against the sustained
+    matmul peak (the kernels run inside a long step), `frac_burst` against the burst figure, and
+    `frac_clock_normalised` puts the class time on the SM clock at which the sustained peak was measured
+    (time x this pass's median SM MHz / that MHz), so that a pass running at a higher clock is not flattered."""
+    kernels = {}
+    for name, e in prof.items():
+        if not e["launches"]:
+            continue
+        per_step_ms = e["ms"] / steps
+        k = {"launches_per_step": e["launches"] / steps, "ms_per_step": per_step_ms}
+        if name in flops:
+            ach = flops[name] / (per_step_ms * 1e-3) / 1e12
+            k.update(bound="tensor", achieved=ach, unit="TFLOP/s", frac=ach / peaks["bf16_tflops_sustained"],
+                     frac_burst=ach / peaks["bf16_tflops"])
+            if run_mhz:
+                k["frac_clock_normalised"] = k["frac"] * peaks["sustained_mhz"] / run_mhz
+        elif name in bts:
+            ach = bts[name] / (per_step_ms * 1e-3) / 1e9
+            k.update(bound="hbm", achieved=ach, unit="GB/s", frac=ach / peaks["hbm_gbs"])
+        kernels[name] = k
+    tot_ms = sum(k["ms_per_step"] for k in kernels.values())
+    for k in kernels.values():
+        k["share"] = k["ms_per_step"] / tot_ms if tot_ms else 0.0
+    return kernels
+
+
+class RequestWorkload:
+    """One fusion request of a named configuration on an engine: inputs, chunk caches (Eq. 1 on the same kernels),
+    fused-cache buffers and the request descriptor."""
+
+    def __init__(self, a3, eng, name, m, r, dev, seed=0, ratio=None, planted=False, shared=None):
+        import torch
+        from paper_2511_17560_b200 import workloads as W
+        self.name, self.m, self.r, self.eng = name, m, r, eng
+        self.ratio = r.ratio if ratio is None else ratio
+        if shared is not None:  # the same request at another ratio: inputs and chunk caches are reused
+            self.x0, self.ck, self.cv, self.tab = shared.x0, shared.ck, shared.cv, shared.tab
+        else:
+            self.x0 = W.make_embeddings_device(m, r.n, dev, seed=seed, std=1.0 if planted else 0.02)
+            if planted:
+                self.x0 = W.plant_embeddings(self.x0, r, PLANTED_CHUNKS, 0.5, seed)
+            self.ck, self.cv = precompute_chunks(eng, m, r.chunk_lens, r.offsets, self.x0, dev)
+            self.tab = a3.chunk_table(self.ck, self.cv, r.offsets)
+        self.K = torch.zeros((m.n_layers, r.n, m.n_kv_heads, m.head_dim), dtype=torch.bfloat16, device=dev)
+        self.V = torch.zeros_like(self.K)
+        self.req, self.out = eng.make_request(self.tab, len(self.ck), max(r.chunk_lens), r.n_ctx, r.n_question, self.x0, self.K, self.V,
+                                              ratio=self.ratio, select_layer=r.select_layer)
+        self.p = self.out["p"]
+
+    def measure(self, a3, timer, peaks, steps, warmup, local, rank, use_graph=True, want_plain=False):
+        """Warm-up, the timed region (K requests through the public call, nothing else on the stream), then the same
+        K requests again with the library's per-launch CUDA events on, for the per-class times."""
+        import torch
+        eng, req, r, m = self.eng, self.req, self.r, self.m
+        eng.workspace(eng.request_workspace_bytes(r.n))
+        for _ in range(max(warmup, 3)):
+            eng.fuse_request(req)
+        torch.cuda.synchronize()
+        assert eng.device_status() == 0, "device status word set during warm-up"
+        a3.launch_count(reset=True)
+        eng.fuse_request(req)
+        torch.cuda.synchronize()
+        launches_per_step = a3.launch_count(reset=True)
+        sampler = ClockSampler(local) if rank == 0 else None
+        graph = eng.graph_capture(req) if use_graph else None
+        torch.cuda.synchronize()
+        a3.launch_count(reset=True)
+        if graph is not None:
+            graph.launch()  # one untimed replay after the capture
+            torch.cuda.synchronize()
+            a3.launch_count(reset=True)
+            seconds = timer.run(graph.launch, steps)
+        else:
+            seconds = timer.run(lambda: eng.fuse_request(req), steps)
+        gpu_launches = a3.launch_count(reset=True)
+        clocks = sampler.stop() if sampler else None
+        other = timer.run(lambda: eng.fuse_request(req), steps) if (graph is not None and want_plain) else None
+        a3.launch_count(reset=True)
+        assert eng.device_status() == 0, "device status word set during the timed region"
+        # second pass: per-launch CUDA events (about 1 ms per request of their own, which is why `value` is not taken here)
+        sampler = ClockSampler(local) if rank == 0 else None
+        eng.profile_enable(launches_per_step * steps + 16)
+        prof_seconds = timer.run(lambda: eng.fuse_request(req), steps, sync_ranks=False)
+        prof = eng.profile_read()
+        eng.profile_enable(0)
+        prof_clocks = sampler.stop() if sampler else None
+        a3.launch_count(reset=True)
+        if graph is not None:
+            graph.close()
+        rows = self.out["rows"].cpu().numpy()
+        flops, bts = algorithmic_work(m, r, self.p, rows)
+        kernels = kernel_table(prof, steps, flops, bts, peaks, (prof_clocks or {}).get("sm_mhz"))
+        total = sum(flops.values())
+        ms = seconds / steps * 1e3
+        tfs = total / (seconds / steps) / 1e12
+        res = {"ms_per_step": ms, "tokens_per_s_per_replica": r.n_ctx / (seconds / steps), "seconds": seconds, "gpu_launches": int(gpu_launches),
+               "launches_per_step": int(launches_per_step), "clocks": clocks, "profiled_pass": {"request_ms": prof_seconds / steps * 1e3, "clocks": prof_clocks},
+               "plain_seconds": other, "kernels": kernels, "algorithmic_tflop_per_request": total / 1e12, "request_tflops": tfs,
+               "request_frac_of_sustained_peak": tfs / peaks["bf16_tflops_sustained"], "request_frac_of_burst_peak": tfs / peaks["bf16_tflops"],
+               "timed_call": "a3_fuse_request" if graph is None else
+                             "a3_graph_launch (the request recorded once by a3_graph_capture; every kernel runs at every replay)"}
+        if clocks and clocks.get("sm_mhz"):
+            res["request_frac_clock_normalised"] = res["request_frac_of_sustained_peak"] * peaks["sustained_mhz"] / clocks["sm_mhz"]
+        if self.name == HEADLINE or (self.r.n_ctx == 32768):
+            planted = set(PLANTED_CHUNKS)
+            re = rows[: self.p]
+            res["planted_share_of_Re"] = float(np.mean([(int(x) // 512) in planted for x in re])) if len(re) else None
+        return res
+
+    def roofline(self, res, peaks, peak_src):
+        kernels = res["kernels"]
+        top = max(kernels, key=lambda nm: kernels[nm]["ms_per_step"])
+        tk = kernels[top]
+        traffic = None
+        t = NCU_TRAFFIC.get((self.name, top))
+        if t:
+            nf = self.r.select_layer
+            traffic = (t["full"] * nf + t["sparse"] * (self.m.n_layers - nf)) / self.m.n_layers  # average over the class's launches
+        return {"kernel": top, "bound": tk.get("bound"), "achieved": tk.get("achieved"),
+                "peak": peaks["bf16_tflops_sustained"] if tk.get("bound") == "tensor" else peaks["hbm_gbs"],
+                "unit": tk.get("unit"), "frac": tk.get("frac"), "frac_burst": tk.get("frac_burst"),
+                "frac_clock_normalised": tk.get("frac_clock_normalised"), "traffic": traffic,
+                "peak_source": peak_src + " (sustained: the kernel is timed inside a long step); frac_burst is against the burst figure, "
+                               "frac_clock_normalised rescales the time to the SM clock the sustained peak was measured at",
+                "timing": "CUDA events the library records around every launch, in a second pass of the same K requests",
+                "avg_launch_ms": tk["ms_per_step"] / tk["launches_per_step"], "kernels": kernels}
+
+
+def sub_result(res, world, steps, n_ctx):
+    """What a `configs` entry keeps of a measurement."""
+    keep = {"ms_per_step": res["ms_per_step"], "value": aggregate_value(n_ctx, steps, world, res["seconds"]), "unit": UNIT, "steps": steps,
+            "request_frac_of_sustained_peak": res["request_frac_of_sustained_peak"], "request_frac_of_burst_peak": res["request_frac_of_burst_peak"],
+            "request_frac_clock_normalised": res.get("request_frac_clock_normalised"), "algorithmic_tflop_per_request": res["algorithmic_tflop_per_request"],
+            "gpu_launches": res["gpu_launches"], "clocks": res["clocks"],
+            "kernels": {k: {f: v[f] for f in ("ms_per_step", "achieved", "unit", "frac", "frac_burst", "frac_clock_normalised", "share") if f in v}
+                        for k, v in res["kernels"].items()}}
+    return keep
+
+
+def measure_batch(a3, eng, m, dev, timer, peaks, steps, warmup, local, rank, world):
+    """Batched serving (16 requests over a pool of 200 precomputed chunks, Llama-shaped): `a3_fuse_batch` timed as one
+    step; aggregate context tokens per second and the spread of the single-request latencies."""
+    import torch
+    from paper_2511_17560_b200 import workloads as W
     pool_lens, reqs = W.batched_requests(seed=0)
-    n_max = max(sum(pool_lens[i] for i in ids) + nq for ids, nq in reqs)
-    eng = a3.A3(m, W.make_weights_device(m, dev, seed=0), n_max + 8)
-    torch.cuda.synchronize()
-    stream = torch.cuda.Stream()
-    torch.cuda.set_stream(stream)
     pool = {}
     for i in sorted({i for ids, _ in reqs for i in ids}):  # only the pool chunks some request uses are prefilled
         t = pool_lens[i]
@@ -310,7 +520,7 @@ def run_a3_batch(args):
         n_ctx_total += r.n_ctx
         rows_total += out["p"] + nq
     reqs_c = [b[0] for b in batch]
-    for _ in range(max(args.warmup, 3)):
+    for _ in range(max(warmup, 3)):
         eng.fuse_batch(reqs_c)
     torch.cuda.synchronize()
     assert eng.device_status() == 0, "device status word set during warm-up"
@@ -319,261 +529,95 @@ def run_a3_batch(args):
         flops_total += sum(flops.values())
     a3.launch_count(reset=True)
     sampler = ClockSampler(local) if rank == 0 else None
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    barrier()
-    torch.cuda.synchronize()
-    e0.record(stream)
-    for _ in range(args.steps):
-        eng.fuse_batch(reqs_c)
-    e1.record(stream)
-    torch.cuda.synchronize()
-    barrier()
-    seconds = max_over_ranks(e0.elapsed_time(e1) / 1e3, dev)
+    seconds = timer.run(lambda: eng.fuse_batch(reqs_c), steps)
     gpu_launches = a3.launch_count(reset=True)
     clocks = sampler.stop() if sampler else None
     assert eng.device_status() == 0, "device status word set during the timed region"
     lat = []
     for req, out, r in batch:  # each request alone, for the latency spread
         eng.fuse_request(req)
-        torch.cuda.synchronize()
-        e0.record(stream)
-        eng.fuse_request(req)
-        e1.record(stream)
-        torch.cuda.synchronize()
-        lat.append(e0.elapsed_time(e1))
-    if rank == 0:
-        lat_s = sorted(lat)
-        line = {"metric": METRIC, "value": aggregate_value(n_ctx_total, args.steps, world, seconds), "unit": UNIT, "n_gpus": world,
-                "steps": args.steps, "warmup": max(args.warmup, 3), "ms_per_step": seconds / args.steps * 1e3, "higher_is_better": True,
-                "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
-                "config": {"workload": "llama8b_batch16", "model": m.name, "requests": len(batch), "pool_chunks": len(pool_lens),
-                           "pool_chunks_used": len(pool), "n_ctx_total": n_ctx_total, "rows_recomputed_total": rows_total,
-                           "recompute_ratio": 0.15, "select_layer": 1, "replicas": world, "layers": m.n_layers,
-                           "timed_call": "a3_fuse_batch (16 requests, one step)",
-                           "l2": "inputs larger than L2: every request streams the stack's weights and its fused cache"},
-                "request_latency_ms": {"min": lat_s[0], "median": lat_s[len(lat_s) // 2], "max": lat_s[-1]},
-                "algorithmic_tflop_per_step": flops_total / 1e12,
-                "step_frac_of_sustained_peak": flops_total / (seconds / args.steps) / 1e12 / peaks["bf16_tflops_sustained"],
-                "gpu_launches": int(gpu_launches), "clocks": clocks}
-        print(json.dumps(line), flush=True)
-    eng.close()
+        lat.append(timer.run(lambda: eng.fuse_request(req), 1, sync_ranks=False) * 1e3)
+    lat_s = sorted(lat)
+    tfs = flops_total / (seconds / steps) / 1e12
+    res = {"ms_per_step": seconds / steps * 1e3, "value": aggregate_value(n_ctx_total, steps, world, seconds), "unit": UNIT, "steps": steps,
+           "config": {"workload": "llama8b_batch16", "model": m.name, "requests": len(batch), "pool_chunks": len(pool_lens),
+                      "pool_chunks_used": len(pool), "n_ctx_total": n_ctx_total, "rows_recomputed_total": rows_total, "recompute_ratio": 0.15,
+                      "select_layer": 1, "replicas": world, "layers": m.n_layers, "timed_call": "a3_fuse_batch (16 requests, one step)"},
+           "request_latency_ms": {"min": lat_s[0], "median": lat_s[len(lat_s) // 2], "max": lat_s[-1]},
+           "algorithmic_tflop_per_step": flops_total / 1e12, "request_frac_of_sustained_peak": tfs / peaks["bf16_tflops_sustained"],
+           "request_frac_of_burst_peak": tfs / peaks["bf16_tflops"], "gpu_launches": int(gpu_launches), "clocks": clocks, "seconds": seconds}
+    if clocks and clocks.get("sm_mhz"):
+        res["request_frac_clock_normalised"] = res["request_frac_of_sustained_peak"] * peaks["sustained_mhz"] / clocks["sm_mhz"]
+    del keep
+    return res
 
 
-def run_a3(args):
+def measure_e2e(eng, wl, timer, steps, world, dev):
+    """The same request through the host-buffer entry: pinned chunk caches + embeddings in, rows + hidden rows out,
+    every step; the fused cache itself stays on the device (it is what the decode that follows reads)."""
     import torch
-    from paper_2511_17560_b200 import a3
-    from paper_2511_17560_b200 import workloads as W
-
-    rank, world, local = dist_setup(args.gpus)
-    torch.cuda.set_device(local)
-    dev = torch.device("cuda", local)
-    peaks, peak_src = load_peaks()
-    m, r = W.request_for(args.config)
-    if args.layers:
-        from dataclasses import replace
-        m = replace(m, n_layers=args.layers)  # profiling captures only: a truncated stack is not a bench result
-    eng = a3.A3(m, W.make_weights_device(m, dev, seed=0), r.n + 8)
-    x0 = W.make_embeddings_device(m, r.n, dev, seed=0)
-    ck, cv = precompute_chunks(eng, m, r, x0, dev)
-    tab = a3.chunk_table(ck, cv, r.offsets)
-    K = torch.zeros((m.n_layers, r.n, m.n_kv_heads, m.head_dim), dtype=torch.bfloat16, device=dev)
-    V = torch.zeros_like(K)
-    req, out = eng.make_request(tab, len(ck), max(r.chunk_lens), r.n_ctx, r.n_question, x0, K, V, ratio=r.ratio,
-                                select_layer=r.select_layer)
-    p = out["p"]
-    eng.workspace(eng.request_workspace_bytes(r.n))
+    m, r, p = wl.m, wl.r, wl.p
+    hk = [k.cpu().pin_memory() for k in wl.ck]
+    hv = [v.cpu().pin_memory() for v in wl.cv]
+    hx = wl.x0.cpu().pin_memory()
+    rows_h = torch.empty(p + r.n_question, dtype=torch.int32).pin_memory()
+    x_h = torch.empty((p + r.n_question, m.d_model), dtype=torch.bfloat16).pin_memory()
+    staging = torch.empty(eng.host_staging_bytes(r.n_ctx, r.n), dtype=torch.uint8, device=dev)
+    req_h, out_h = eng.make_request(None, len(hk), 0, r.n_ctx, r.n_question, None, wl.K, wl.V, ratio=wl.ratio, select_layer=r.select_layer)
+    for _ in range(2):
+        eng.fuse_request_host(req_h, hk, hv, hx, rows_h, x_h, staging)
+    barrier()
     torch.cuda.synchronize()
-    stream = torch.cuda.Stream()  # not the default stream: a graph cannot be recorded there
-    torch.cuda.set_stream(stream)
+    t0 = time.perf_counter()
+    sec_dev = timer.run(lambda: eng.fuse_request_host(req_h, hk, hv, hx, rows_h, x_h, staging), steps, sync_ranks=False)
+    wall = time.perf_counter() - t0
+    sec_e = max_over_ranks(max(sec_dev, wall), dev)
+    copied_layers = m.n_layers - r.select_layer - 1  # caches of layers <= select_layer are recomputed, not copied
+    h2d = sum(k.numel() * 2 for k in hk) * 2 * copied_layers // m.n_layers + hx.numel() * 2
+    d2h = rows_h.numel() * 4 + x_h.numel() * 2
+    assert torch.equal(rows_h, wl.out["rows"].cpu()), "host entry selected different rows"
+    return {"value": aggregate_value(r.n_ctx, steps, world, sec_e), "unit": UNIT, "ms_per_step": sec_e / steps * 1e3,
+            "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h),
+            "copied": "in: chunk caches of the layers above the selection layer + embeddings, from pinned host memory; out: R and the final "
+                      "hidden rows; the fused cache stays on the device"}
 
-    for _ in range(max(args.warmup, 3)):
-        eng.fuse_request(req)
+
+def measure_context(eng, wl, timer, peaks, req_ms):
+    """Context for the paper's TTFT comparison, on the same kernels: the full prefill of the concatenated input, the
+    cheaper reading of the selection, the `ex` eviction, and the first token."""
+    import torch
+    m, r, p = wl.m, wl.r, wl.p
+    dev = wl.K.device
+    Kp, Vp = torch.zeros_like(wl.K), torch.zeros_like(wl.V)
+    eng.precompute_chunk(wl.x0.clone(), Kp, Vp)
     torch.cuda.synchronize()
-    assert eng.device_status() == 0, "device status word set during warm-up"
-    a3.launch_count(reset=True)
-    eng.fuse_request(req)
-    torch.cuda.synchronize()
-    launches_per_step = a3.launch_count(reset=True)
+    xs = [wl.x0.clone() for _ in range(2)]
+    it = iter(xs)
+    full_prefill_ms = timer.run(lambda: eng.precompute_chunk(next(it), Kp, Vp), len(xs), sync_ranks=False) / len(xs) * 1e3
+    del Kp, Vp, xs
 
-    # ---- the timed region: K requests through the public call, nothing else on the stream.  By default the call is
-    # a3_graph_launch on a graph that a3_graph_capture recorded once (every kernel of the request runs at every
-    # replay; inputs are read and the fused cache is rebuilt each time); --no-graph times a3_fuse_request itself.
-    # The other of the two is timed the same way right after and reported in `config`.
-    sampler = ClockSampler(local) if rank == 0 else None
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    graph = None if args.no_graph else eng.graph_capture(req)
-    torch.cuda.synchronize()
-
-    def timed(call):
-        barrier()
-        torch.cuda.synchronize()
-        e0.record(stream)
-        for _ in range(args.steps):
-            call()
-        e1.record(stream)
-        torch.cuda.synchronize()
-        barrier()
-        return max_over_ranks(e0.elapsed_time(e1) / 1e3, dev)
-
-    a3.launch_count(reset=True)
-    if graph is not None:
-        graph.launch()  # one untimed replay after the capture
-        torch.cuda.synchronize()
-        a3.launch_count(reset=True)
-        seconds = timed(graph.launch)
-        gpu_launches = a3.launch_count(reset=True)
-        other_seconds = timed(lambda: eng.fuse_request(req))
-    else:
-        seconds = timed(lambda: eng.fuse_request(req))
-        gpu_launches = a3.launch_count(reset=True)
-        other_seconds = None
-    a3.launch_count(reset=True)
-    assert eng.device_status() == 0, "device status word set during the timed region"
-
-    # ---- the same K requests again with the library's per-launch CUDA events on (the clock sampler keeps running):
-    # per-kernel device times for the roofline.  The events themselves cost about 1 ms per request, which is why
-    # this pass is not the one `value` is taken from.
-    eng.profile_enable(launches_per_step * args.steps + 16)
-    e0.record(stream)
-    for _ in range(args.steps):
-        eng.fuse_request(req)
-    e1.record(stream)
-    torch.cuda.synchronize()
-    profiled_ms = e0.elapsed_time(e1) / args.steps
-    clocks = sampler.stop() if sampler else None
-    prof = eng.profile_read()
-    eng.profile_enable(0)
-    a3.launch_count(reset=True)
-
-    if graph is not None:
-        graph.close()
-    value = aggregate_value(r.n_ctx, args.steps, world, seconds)
-    rows = out["rows"].cpu().numpy()
-
-    # ---- roofline of the dominant kernel class (device time from CUDA events around every launch)
-    flops, bts = algorithmic_work(m, r, p, rows)
-    kernels = {}
-    for name, e in prof.items():
-        if not e["launches"]:
-            continue
-        per_step_ms = e["ms"] / args.steps
-        k = {"launches_per_step": e["launches"] / args.steps, "ms_per_step": per_step_ms}
-        if name in flops:
-            k.update(bound="tensor", achieved=flops[name] / (per_step_ms * 1e-3) / 1e12, unit="TFLOP/s")
-            k["frac"] = k["achieved"] / peaks["bf16_tflops_sustained"]
-        elif name in bts:
-            k.update(bound="hbm", achieved=bts[name] / (per_step_ms * 1e-3) / 1e9, unit="GB/s")
-            k["frac"] = k["achieved"] / peaks["hbm_gbs"]
-        kernels[name] = k
-    tot_ms = sum(k["ms_per_step"] for k in kernels.values())
-    for k in kernels.values():
-        k["share"] = k["ms_per_step"] / tot_ms
-    top = max(kernels, key=lambda nm: kernels[nm]["ms_per_step"])
-    tk = kernels[top]
-    traffic = None
-    t = NCU_TRAFFIC.get((args.config, top))
-    if t and not args.layers:
-        n_full = r.select_layer
-        traffic = (t["full"] * n_full + t["sparse"] * (m.n_layers - n_full)) / m.n_layers  # average over the class's launches
-    roofline = {"kernel": top, "bound": tk.get("bound"), "achieved": tk.get("achieved"),
-                "peak": peaks["bf16_tflops_sustained"] if tk.get("bound") == "tensor" else peaks["hbm_gbs"],
-                "unit": tk.get("unit"), "frac": tk.get("frac"), "traffic": traffic, "peak_source": peak_src + " (sustained)",
-                "avg_launch_ms": tk["ms_per_step"] / tk["launches_per_step"], "kernels": kernels}
-    total_flops = sum(flops.values())
-
-    # ---- end to end through the host-buffer entry: pinned chunk caches + embeddings in, rows + hidden rows out
-    e2e = None
-    if not args.no_e2e:
-        hk = [k.cpu().pin_memory() for k in ck]
-        hv = [v.cpu().pin_memory() for v in cv]
-        hx = x0.cpu().pin_memory()
-        rows_h = torch.empty(p + r.n_question, dtype=torch.int32).pin_memory()
-        x_h = torch.empty((p + r.n_question, m.d_model), dtype=torch.bfloat16).pin_memory()
-        staging = torch.empty(eng.host_staging_bytes(r.n_ctx, r.n), dtype=torch.uint8, device=dev)
-        req_h, out_h = eng.make_request(None, len(hk), 0, r.n_ctx, r.n_question, None, K, V, ratio=r.ratio, select_layer=r.select_layer)
+    def variant(**kw):
+        req_v, out_v = eng.make_request(wl.tab, len(wl.ck), max(r.chunk_lens), r.n_ctx, r.n_question, wl.x0, wl.K, wl.V, ratio=wl.ratio,
+                                        select_layer=r.select_layer, **kw)
         for _ in range(2):
-            eng.fuse_request_host(req_h, hk, hv, hx, rows_h, x_h, staging)
-        barrier()
-        torch.cuda.synchronize()
-        t0 = time.perf_counter()
-        e0.record(stream)
-        for _ in range(args.steps):
-            eng.fuse_request_host(req_h, hk, hv, hx, rows_h, x_h, staging)
-        e1.record(stream)
-        torch.cuda.synchronize()
-        wall = time.perf_counter() - t0
-        sec_e = max_over_ranks(max(e0.elapsed_time(e1) / 1e3, wall), dev)
-        copied_layers = m.n_layers - r.select_layer - 1  # caches of layers <= select_layer are recomputed, not copied
-        h2d = sum(k.numel() * 2 for k in hk) * 2 * copied_layers // m.n_layers + hx.numel() * 2
-        d2h = rows_h.numel() * 4 + x_h.numel() * 2
-        e2e = {"value": aggregate_value(r.n_ctx, args.steps, world, sec_e), "unit": UNIT, "ms_per_step": sec_e / args.steps * 1e3,
-               "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h)}
-        assert torch.equal(rows_h, out["rows"].cpu()), "host entry selected different rows"
+            eng.fuse_request(req_v)
+        return timer.run(lambda: eng.fuse_request(req_v), 3, sync_ranks=False) / 3 * 1e3, out_v
 
-    context = {}
-    if not args.no_context:
-        # context for the paper's TTFT comparison: a full prefill of the concatenated input on the same kernels
-        Kp, Vp = torch.zeros_like(K), torch.zeros_like(V)
-        eng.precompute_chunk(x0.clone(), Kp, Vp)
-        torch.cuda.synchronize()
-        xs = [x0.clone() for _ in range(3)]
-        e0.record(stream)
-        for xx in xs:
-            eng.precompute_chunk(xx, Kp, Vp)
-        e1.record(stream)
-        torch.cuda.synchronize()
-        full_prefill_ms = e0.elapsed_time(e1) / len(xs)
-        del Kp, Vp, xs
-
-        # the cheaper reading of the selection (scores against the recovered cached keys, no full block), same request
-        req_c, out_c = eng.make_request(tab, len(ck), max(r.chunk_lens), r.n_ctx, r.n_question, x0, K, V, ratio=r.ratio,
-                                        select_layer=r.select_layer, score_source=1)
-        for _ in range(2):
-            eng.fuse_request(req_c)
-        torch.cuda.synchronize()
-        e0.record(stream)
-        for _ in range(3):
-            eng.fuse_request(req_c)
-        e1.record(stream)
-        torch.cuda.synchronize()
-        cached_ms = e0.elapsed_time(e1) / 3
-        overlap = len(set(out_c["rows"][:p].tolist()) & set(out["rows"][:p].tolist())) / max(p, 1)
-
-        # the `ex` extension on top of the request: compact caches of capacity C = 1024 (the paper's setting) per layer
-        req_e, out_e = eng.make_request(tab, len(ck), max(r.chunk_lens), r.n_ctx, r.n_question, x0, K, V, ratio=r.ratio,
-                                        select_layer=r.select_layer, evict_capacity=1024, evict_pool=7)
-        for _ in range(2):
-            eng.fuse_request(req_e)
-        torch.cuda.synchronize()
-        e0.record(stream)
-        for _ in range(3):
-            eng.fuse_request(req_e)
-        e1.record(stream)
-        torch.cuda.synchronize()
-        evict_ms = e0.elapsed_time(e1) / 3
-        del out_e
-
-        # ... and the first token itself (final norm, vocabulary projection, greedy choice) on the last question row:
-        # HBM-bound, vocab*d*2 bytes read once; synthetic final-norm gains and vocabulary matrix
-        g = torch.Generator(device=dev)
-        g.manual_seed(7)
-        lm_head = (torch.randn((m.vocab, m.d_model), device=dev, generator=g) * 0.02).to(torch.bfloat16)
-        fnorm = torch.ones(m.d_model, dtype=torch.bfloat16, device=dev)
-        x_last = out["x"][-1]
-        for _ in range(3):
-            eng.first_token(x_last, fnorm, lm_head, want_logits=False)
-        torch.cuda.synchronize()
-        e0.record(stream)
-        for _ in range(10):
-            eng.first_token(x_last, fnorm, lm_head, want_logits=False)
-        e1.record(stream)
-        torch.cuda.synchronize()
-        first_token_ms = e0.elapsed_time(e1) / 10
-        first_token_gbs = m.vocab * m.d_model * 2 / (first_token_ms * 1e-3) / 1e9
-        del lm_head
-        req_ms = seconds / args.steps * 1e3
-        context = {
-            "full_prefill_ms": full_prefill_ms, "speedup_vs_full_prefill": full_prefill_ms / req_ms,
+    cached_ms, out_c = variant(score_source=1)
+    overlap = len(set(out_c["rows"][:p].tolist()) & set(wl.out["rows"][:p].tolist())) / max(p, 1)
+    evict_ms, out_e = variant(evict_capacity=1024, evict_pool=7)
+    del out_e
+    g = torch.Generator(device=dev)
+    g.manual_seed(7)
+    lm_head = (torch.randn((m.vocab, m.d_model), device=dev, generator=g) * 0.02).to(torch.bfloat16)
+    fnorm = torch.ones(m.d_model, dtype=torch.bfloat16, device=dev)
+    x_last = wl.out["x"][-1]
+    for _ in range(3):
+        eng.first_token(x_last, fnorm, lm_head, want_logits=False)
+    first_token_ms = timer.run(lambda: eng.first_token(x_last, fnorm, lm_head, want_logits=False), 10, sync_ranks=False) / 10 * 1e3
+    first_token_gbs = m.vocab * m.d_model * 2 / (first_token_ms * 1e-3) / 1e9
+    del lm_head
+    return {"full_prefill_ms": full_prefill_ms, "speedup_vs_full_prefill": full_prefill_ms / req_ms,
             "scores_from_cached_keys": {"request_ms": cached_ms, "tokens_per_s": r.n_ctx / (cached_ms * 1e-3),
                                         "selection_overlap_with_true_keys": overlap},
             "ex_eviction": {"capacity": 1024, "pool": 7, "request_ms": evict_ms, "overhead_ms": evict_ms - req_ms},
@@ -581,36 +625,130 @@ def run_a3(args):
                             "ttft_fused_ms": req_ms + first_token_ms, "ttft_full_prefill_ms": full_prefill_ms + first_token_ms,
                             "ttft_ratio": (full_prefill_ms + first_token_ms) / (req_ms + first_token_ms)}}
 
+
+def run_a3(args):
+    import torch
+    from dataclasses import replace
+    from paper_2511_17560_b200 import a3
+    from paper_2511_17560_b200 import workloads as W
+
+    rank, world, local = dist_setup(args.gpus)
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    peaks, peak_src = load_peaks()
+    suite = args.config is None            # default run: the headline workload plus the other configurations
+    main_name = args.config or HEADLINE
+    stream = torch.cuda.Stream()           # not the default stream: a graph cannot be recorded there
+    torch.cuda.set_stream(stream)
+    timer = Timer(stream, dev)
+    steps, warmup = args.steps, max(args.warmup, 3)
+    sub_steps = max(1, min(steps, 5))
+
+    if main_name == "llama8b_batch16":
+        m = W.LLAMA8B if not args.layers else replace(W.LLAMA8B, n_layers=args.layers)
+        pool_lens, reqs = W.batched_requests(seed=0)
+        n_max = max(sum(pool_lens[i] for i in ids) + nq for ids, nq in reqs)
+        eng = a3.A3(m, W.make_weights_device(m, dev, seed=0), n_max + 8)
+        res = measure_batch(a3, eng, m, dev, timer, peaks, steps, warmup, local, rank, world)
+        if rank == 0:
+            line = {"metric": METRIC, "value": res["value"], "unit": UNIT, "n_gpus": world, "steps": steps, "warmup": warmup,
+                    "ms_per_step": res["ms_per_step"], "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16",
+                    "data": "synthetic", **{k: v for k, v in res.items() if k not in ("value", "unit", "steps", "ms_per_step", "seconds")}}
+            print(json.dumps(line), flush=True)
+        eng.close()
+        return
+
+    m, r = W.request_for(main_name)
+    if args.layers:
+        m = replace(m, n_layers=args.layers)  # profiling captures only: a truncated stack is not a bench result
+    planted = main_name == HEADLINE
+    n_max = r.n
+    if suite:
+        pool_lens, breqs = W.batched_requests(seed=0)
+        n_max = max(n_max, max(sum(pool_lens[i] for i in ids) + nq for ids, nq in breqs))
+    weights = W.make_weights_device(m, dev, seed=0)
+    if planted:
+        W.tie_keys_to_queries(weights[r.select_layer], m, 0.7, 0)  # lets a shared input direction show up as attention
+    eng = a3.A3(m, weights, n_max + 8)
+    wl = RequestWorkload(a3, eng, main_name, m, r, dev, ratio=args.ratio, planted=planted)
+    res = wl.measure(a3, timer, peaks, steps, warmup, local, rank, use_graph=not args.no_graph, want_plain=True)
+    value = aggregate_value(r.n_ctx, steps, world, res["seconds"])
+    roofline = wl.roofline(res, peaks, peak_src)
+    e2e = None if args.no_e2e else measure_e2e(eng, wl, timer, steps, world, dev)
+    context = {} if args.no_context else measure_context(eng, wl, timer, peaks, res["ms_per_step"])
+
+    configs = {}
+    if suite:
+        # ---- the other configurations, same library, same run (sub-results; their own lines with --config NAME)
+        del wl.ck, wl.cv, wl.K, wl.V
+        torch.cuda.empty_cache()
+        m2, r2 = W.request_for("llama8b_10x512")
+        w2 = RequestWorkload(a3, eng, "llama8b_10x512", m2, r2, dev)
+        res2 = w2.measure(a3, timer, peaks, sub_steps, 3, local, rank)
+        configs["llama8b_10x512"] = {**sub_result(res2, world, sub_steps, r2.n_ctx), "config": workload_config("llama8b_10x512", m2, r2, w2.p, world)}
+        del w2
+        torch.cuda.empty_cache()
+        b = measure_batch(a3, eng, m, dev, timer, peaks, max(1, min(steps, 3)), 3, local, rank, world)
+        b.pop("seconds", None)
+        configs["llama8b_batch16"] = b
+        eng.close()
+        del eng, weights
+        torch.cuda.empty_cache()
+        m3, r3 = W.request_for("qwen7b_16xU")
+        eng3 = a3.A3(m3, W.make_weights_device(m3, dev, seed=0), r3.n + 8)
+        sweep, base = {}, None
+        for ratio in SWEEP_RATIOS:
+            w3 = RequestWorkload(a3, eng3, "qwen7b_16xU", m3, r3, dev, ratio=ratio, shared=base)
+            base = base or w3
+            res3 = w3.measure(a3, timer, peaks, sub_steps, 3, local, rank)
+            sweep[f"{int(round(ratio * 100))}%"] = {**sub_result(res3, world, sub_steps, r3.n_ctx), "n_recompute": w3.p}
+        configs["qwen7b_16xU"] = {"config": workload_config("qwen7b_16xU", m3, r3, None, world, ratio=list(SWEEP_RATIOS)), "ratio_sweep": sweep}
+        eng3.close()
+        del eng3, base, w3
+        torch.cuda.empty_cache()
+    else:
+        eng.close()
+
     cpu = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
-        S = oracle_sample(args.config)
-        t, parts = oracle_step(S)
-        cpu = {"value": r.n_ctx / t, "unit": UNIT, "cores": oracle_threads(), "kind": "oracle", "seconds": t,
-               "sample": "one bounded oracle step (fp32): 1 layer of position recovery, a full block and the selection QKV on "
-                         "every 4th row, scores + top-p at full size, one recompute layer; extrapolated to the whole request",
+        S = oracle_sample(main_name)
+        sf, sr = oracle_strides(r.n, wl.p + r.n_question, 4 * args.oracle_rows)
+        t_meas, t_extr, parts = oracle_step(S, sf, sr)
+        cpu = {"value": r.n_ctx / t_extr, "unit": UNIT, "cores": oracle_threads(), "kind": "oracle", "seconds": t_extr, "measured_seconds": t_meas,
+               "extrapolated": True,
+               "sample": f"one bounded oracle step (fp32): 1 layer of position recovery, a full block and the selection QKV on every {sf}-th row, "
+                         f"scores + top-p at full size, one recompute layer on every {sr}-th carried row; extrapolated to the whole request",
                "seconds_by_phase": parts}
+        del S
+        if suite:
+            # the whole Llama-shaped 10 x 512 request on the oracle, every layer and row, not extrapolated
+            sec, rr, phases = oracle_full_request("llama8b_10x512")
+            by = {"position_recovery": phases.get("position_recovery", 0.0), "selection": phases.get("selection", 0.0),
+                  "full_blocks": sum(v for k, v in phases.items() if k.startswith("full_block")),
+                  "recompute_layers": sum(v for k, v in phases.items() if k.startswith("recompute_"))}
+            configs["llama8b_10x512"]["cpu_baseline"] = {"value": rr.n_ctx / sec, "unit": UNIT, "cores": oracle_threads(), "kind": "oracle",
+                                                         "seconds": sec, "extrapolated": False, "seconds_by_phase": by,
+                                                         "sample": "the oracle's fuse_request on the whole request (32 layers, all rows, fp32)"}
     if rank == 0:
-        line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3),
-                "ms_per_step": seconds / args.steps * 1e3, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
-                "dtype": "bf16", "data": "synthetic",
-                "config": {"workload": args.config, "model": m.name, "chunks": len(r.chunk_lens), "n_ctx": r.n_ctx,
-                           "n_question": r.n_question, "recompute_ratio": r.ratio, "n_recompute": p, "select_layer": r.select_layer,
-                           "replicas": world, "layers": m.n_layers, "truncated_for_profiling": bool(args.layers), "l2": "inputs larger than L2: every step streams the stack's weights "
-                                                    f"({sum(t.numel() for w in eng._weights for t in w.values()) * 2 / 2**30:.1f} GiB) and the fused cache"},
-                "request_ms": seconds / args.steps * 1e3,
-                "request_ms_with_profiling_events": profiled_ms,
-                "timed_call": "a3_fuse_request" if graph is None else
-                              "a3_graph_launch (the request recorded once by a3_graph_capture; every kernel runs at every replay)",
-                "plain_launches": None if other_seconds is None else
-                                  {"call": "a3_fuse_request", "ms_per_step": other_seconds / args.steps * 1e3,
-                                   "value": aggregate_value(r.n_ctx, args.steps, world, other_seconds)},
+        cfg = workload_config(main_name, m, r, wl.p, world, ratio=wl.ratio)  # the same object the reference arm prints
+        notes = {"truncated_for_profiling": bool(args.layers), "planted_share_of_Re": res.get("planted_share_of_Re"),
+                 "embeddings": "unit-RMS rows; question and planted chunks share a direction (cosine 0.5); key projection of the "
+                               "selection layer tied to the query projections (rho 0.7)" if planted else "N(0, 0.02^2) rows"}
+        line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": steps, "warmup": warmup,
+                "ms_per_step": res["ms_per_step"], "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+                "dtype": "bf16", "data": "synthetic", "config": cfg, "workload_notes": notes,
+                "request_ms": res["ms_per_step"], "profiled_pass": res["profiled_pass"], "timed_call": res["timed_call"],
+                "plain_launches": None if res["plain_seconds"] is None else
+                                  {"call": "a3_fuse_request", "ms_per_step": res["plain_seconds"] / steps * 1e3,
+                                   "value": aggregate_value(r.n_ctx, steps, world, res["plain_seconds"])},
                 **context,
-                "algorithmic_tflop_per_request": total_flops / 1e12,
-                "request_tflops": total_flops / (seconds / args.steps) / 1e12,
-                "request_frac_of_sustained_peak": total_flops / (seconds / args.steps) / 1e12 / peaks["bf16_tflops_sustained"],
-                "gpu_launches": int(gpu_launches), "clocks": clocks, "roofline": roofline, "e2e": e2e, "cpu_baseline": cpu}
+                "algorithmic_tflop_per_request": res["algorithmic_tflop_per_request"], "request_tflops": res["request_tflops"],
+                "request_frac_of_sustained_peak": res["request_frac_of_sustained_peak"],
+                "request_frac_of_burst_peak": res["request_frac_of_burst_peak"],
+                "request_frac_clock_normalised": res.get("request_frac_clock_normalised"),
+                "gpu_launches": res["gpu_launches"], "clocks": res["clocks"], "roofline": roofline, "e2e": e2e, "cpu_baseline": cpu,
+                "configs": configs or None}
         print(json.dumps(line), flush=True)
-    eng.close()
 
 
 def main():
@@ -619,8 +757,10 @@ def main():
     ap.add_argument("--steps", type=int, default=5)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="a3", choices=["a3", "reference"])
-    ap.add_argument("--config", default="llama8b_10x512")
+    ap.add_argument("--config", default=None, help="one workload only: llama8b_10x512, llama8b_64x512, qwen7b_16xU, llama8b_batch16, tiny, ...")
+    ap.add_argument("--ratio", type=float, default=None, help="recompute ratio of the --config workload (default: the configuration's)")
     ap.add_argument("--layers", type=int, default=0, help="truncate the stack (ncu captures of a small case only)")
+    ap.add_argument("--oracle-rows", type=int, default=384, help="rows per sampled piece of the reference arm's bounded oracle step")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-graph", action="store_true")
     ap.add_argument("--no-context", action="store_true", help="skip the context measurements (full prefill, variants, first token)")
@@ -629,10 +769,7 @@ def main():
     if args.impl == "reference":
         run_reference(args)
     else:
-        if args.config == "llama8b_batch16":
-            run_a3_batch(args)
-        else:
-            run_a3(args)
+        run_a3(args)
 
 
 if __name__ == "__main__":
