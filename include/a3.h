@@ -101,8 +101,8 @@ typedef struct {
 /* What ranks the candidates.  A3_SELECT_ATTENTION is Eq. 3.  A3_SELECT_VALUE_DEVIATION is the comparison method
  * of the Baselines paragraph (CacheBlend): score = squared distance between a token's cached value and its true
  * value at select_layer, over all KV heads and channels (needs A3_SCORES_TRUE_KEYS, which forms the true values);
- * scores_out then holds these distances.  Index-only selections (chunk edges - a3_chunk_edge_rows -, random) are
- * passed through forced_re. */
+ * scores_out then holds these distances.  Index-only selections (chunk edges - a3_chunk_edge_rows -, random -
+ * a3_random_rows -) are passed through forced_re. */
 #define A3_SELECT_ATTENTION 0
 #define A3_SELECT_VALUE_DEVIATION 1
 
@@ -191,6 +191,16 @@ size_t a3_host_staging_bytes(const a3_handle* h, int n_ctx, int n);
  * method of the Baselines paragraph, LegoLink: m = 20).  chunk_len: host [n_chunks].  Writes at most `capacity`
  * slots to rows_out (host; may be NULL) and returns the full count.  Host only. */
 int a3_chunk_edge_rows(const int32_t* chunk_len, int n_chunks, int m, int n_system, int32_t* rows_out, int capacity);
+
+/* k distinct slots of [cand_begin, cand_end) drawn uniformly at random, ascending: the random selection the other
+ * selectors are compared with (Attention Recovery subsection, discussion of Figure 3).  Counter-based and
+ * reproducible: with n = cand_end - cand_begin candidates 0..n-1 in an array, step i = 0..k-1 swaps entry i with
+ * entry i + (mix(seed + i) mod (n - i)), where mix is the SplitMix64 finaliser
+ *   z = x + 0x9E3779B97F4A7C15; z = (z ^ (z >> 30)) * 0xBF58476D1CE4E5B9; z = (z ^ (z >> 27)) * 0x94D049BB133111EB;
+ *   mix = z ^ (z >> 31)                                            (64-bit unsigned arithmetic);
+ * the first k entries, sorted, plus cand_begin are the result.  k is clamped to n.  Writes at most `capacity` slots
+ * to rows_out (host; may be NULL) and returns the count.  Host only. */
+int a3_random_rows(uint64_t seed, int cand_begin, int cand_end, int k, int32_t* rows_out, int capacity);
 
 /* p = min(n_candidates, floor(ratio * n + 1e-9)): the size of Re (Eq. 3, p = r n). Host only. */
 int a3_recompute_count(double ratio, int n, int n_candidates);

@@ -376,6 +376,26 @@ def chunk_edge_rows(chunk_lens: Sequence[int], m: int, n_system: int = 0) -> np.
     return np.array(rows, dtype=np.int64)
 
 
+def random_rows(seed: int, cand_begin: int, cand_end: int, k: int) -> np.ndarray:
+    """The random selection the paper's comparison mentions (Attention Recovery subsection, Figure 3 discussion):
+    k distinct candidate slots drawn uniformly, ascending.  The draw is a counter-based partial shuffle, stated here
+    so that any implementation can reproduce it: candidates 0..n-1 in a list; for i = 0..k-1 swap entry i with entry
+    i + (mix(seed + i) mod (n - i)), mix being the SplitMix64 finaliser on 64-bit unsigned integers; the first k
+    entries, sorted, shifted by cand_begin."""
+    mask = (1 << 64) - 1
+    n = cand_end - cand_begin
+    k = max(0, min(int(k), n))
+    idx = list(range(n))
+    for i in range(k):
+        z = (seed + i + 0x9E3779B97F4A7C15) & mask
+        z = ((z ^ (z >> 30)) * 0xBF58476D1CE4E5B9) & mask
+        z = ((z ^ (z >> 27)) * 0x94D049BB133111EB) & mask
+        z ^= z >> 31
+        j = i + z % (n - i)
+        idx[i], idx[j] = idx[j], idx[i]
+    return np.array(sorted(cand_begin + t for t in idx[:k]), dtype=np.int64)
+
+
 def topk_select(s: np.ndarray, cand_begin: int, cand_end: int, k: int) -> np.ndarray:
     """Re = top_p(s): the k candidate slots with the largest score (Eq. 3).
 

@@ -71,7 +71,7 @@ class HostIO(C.Structure):
 EXPORTS = ("a3_create", "a3_destroy", "a3_set_option", "a3_scores_workspace_bytes", "a3_swiglu_rows", "a3_layer_workspace_bytes", "a3_request_workspace_bytes", "a3_host_staging_bytes",
            "a3_recompute_count", "a3_rope_rerotate", "a3_query_scores", "a3_query_scores_static", "a3_topk_select", "a3_recompute_layer",
            "a3_scatter_kv", "a3_gather_rows", "a3_precompute_chunk", "a3_first_token_workspace_bytes", "a3_first_token",
-           "a3_evict_count", "a3_evict_workspace_bytes", "a3_evict_layer", "a3_chunk_edge_rows", "a3_fuse_request", "a3_fuse_batch", "a3_fuse_request_host",
+           "a3_evict_count", "a3_evict_workspace_bytes", "a3_evict_layer", "a3_chunk_edge_rows", "a3_random_rows", "a3_fuse_request", "a3_fuse_batch", "a3_fuse_request_host",
            "a3_graph_capture", "a3_graph_launch", "a3_graph_kernel_count", "a3_graph_destroy",
            "a3_device_status", "a3_status_string", "a3_last_cuda_error", "a3_launch_count", "a3_profile_enable",
            "a3_profile_read", "a3_kernel_class_name")
@@ -111,6 +111,7 @@ def _load():
     lib.a3_gather_rows.argtypes = [vp, vp, i32, vp, i32, i32, vp, vp]
     lib.a3_precompute_chunk.argtypes = [vp, vp, i32, vp, vp, u64, vp, sz, vp]
     lib.a3_chunk_edge_rows.argtypes = [C.POINTER(C.c_int32), i32, i32, i32, C.POINTER(C.c_int32), i32]
+    lib.a3_random_rows.argtypes = [u64, i32, i32, i32, C.POINTER(C.c_int32), i32]
     lib.a3_evict_count.argtypes = [i32, i32, i32, i32]
     lib.a3_evict_workspace_bytes.argtypes = [vp, i32]
     lib.a3_evict_workspace_bytes.restype = sz
@@ -166,6 +167,14 @@ def chunk_edge_rows(chunk_lens: Sequence[int], m: int, n_system: int = 0) -> np.
     count = int(_load().a3_chunk_edge_rows(lens, len(chunk_lens), int(m), int(n_system), None, 0))
     out = (C.c_int32 * max(1, count))()
     _load().a3_chunk_edge_rows(lens, len(chunk_lens), int(m), int(n_system), out, count)
+    return np.frombuffer(out, dtype=np.int32, count=count).copy()
+
+
+def random_rows(seed: int, cand_begin: int, cand_end: int, k: int) -> np.ndarray:
+    """k distinct candidate slots drawn uniformly at random (ascending), for use as forced_re."""
+    k = max(0, min(int(k), cand_end - cand_begin))
+    out = (C.c_int32 * max(1, k))()
+    count = int(_load().a3_random_rows(int(seed), int(cand_begin), int(cand_end), k, out, k))
     return np.frombuffer(out, dtype=np.int32, count=count).copy()
 
 

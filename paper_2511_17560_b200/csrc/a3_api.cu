@@ -109,6 +109,31 @@ extern "C" int a3_chunk_edge_rows(const int32_t* chunk_len, int n_chunks, int m,
   return count;
 }
 
+extern "C" int a3_random_rows(uint64_t seed, int cand_begin, int cand_end, int k, int32_t* rows_out, int capacity) {
+  if (cand_begin < 0 || cand_end <= cand_begin || k <= 0) return 0;
+  const int n = cand_end - cand_begin;
+  if (k > n) k = n;
+  int32_t* idx = (int32_t*)malloc(sizeof(int32_t) * (size_t)n);
+  if (!idx) return 0;
+  for (int i = 0; i < n; ++i) idx[i] = i;
+  for (int i = 0; i < k; ++i) {
+    uint64_t z = seed + (uint64_t)i + 0x9E3779B97F4A7C15ull;
+    z = (z ^ (z >> 30)) * 0xBF58476D1CE4E5B9ull;
+    z = (z ^ (z >> 27)) * 0x94D049BB133111EBull;
+    z ^= z >> 31;
+    const int j = i + (int)(z % (uint64_t)(n - i));
+    const int32_t t = idx[i];
+    idx[i] = idx[j];
+    idx[j] = t;
+  }
+  // ascending order of the k chosen slots (insertion into a bitmap would do as well; k log k is nothing here)
+  qsort(idx, (size_t)k, sizeof(int32_t), [](const void* a, const void* b) { return (*(const int32_t*)a > *(const int32_t*)b) - (*(const int32_t*)a < *(const int32_t*)b); });
+  if (rows_out)
+    for (int i = 0; i < k && i < capacity; ++i) rows_out[i] = cand_begin + idx[i];
+  free(idx);
+  return k;
+}
+
 extern "C" int a3_recompute_count(double ratio, int n, int n_candidates) {
   if (n_candidates <= 0 || n <= 0 || !(ratio > 0.0)) return 0;
   double p = floor(ratio * (double)n + 1e-9);

@@ -194,6 +194,63 @@ def test_fuse_batch_and_host_entry_match_single_requests(a3mod):
     s.eng.close()
 
 
+def test_fuse_batch_of_different_requests_matches_oracle(a3mod):
+    """Batched serving against the oracle: requests that draw different chunks, in different orders, from one pool of
+    chunk caches (prefilled once, by the oracle, at local positions - Eq. 1) and carry questions of different lengths
+    go through a3_fuse_batch in one call; every request of the batch is then compared with the oracle's fuse_request
+    of that request, the oracle's selection forced on the library, with the gates of the single-request test."""
+    m = W.TINY_GQA
+    dev = torch.device("cuda:0")
+    layers = W.make_weights(m, 3, std=0.05)
+    model, weights = oracle_model(m), oracle_weights(layers)
+    pool_lens = (100, 37, 128, 64, 90)
+    pool_x = [W.make_embeddings(m, t, 3, std=1.0, stream=10 + i) for i, t in enumerate(pool_lens)]
+    pool = [O.precompute_chunk(x, weights, model, rnd=O.round_bf16) for x in pool_x]
+    batch = [((0, 2, 4), 13), ((4, 1, 3, 0), 5), ((2,), 31)]  # (pool chunks in input order, question length)
+    n_max = max(sum(pool_lens[i] for i in ids) + nq for ids, nq in batch)
+    eng = a3mod.A3(m, dev_weights(layers, dev), n_max + 8)
+    dpool = [(to_dev(k, dev), to_dev(v, dev)) for k, v in pool]
+
+    def build(ids, nq, j, forced=None):
+        r = W.RequestShape(tuple(pool_lens[i] for i in ids), nq, 0.2, 1)
+        x0 = np.concatenate([pool_x[i] for i in ids] + [W.make_embeddings(m, nq, 3, std=1.0, stream=50 + j)])
+        tab = a3mod.chunk_table([dpool[i][0] for i in ids], [dpool[i][1] for i in ids], r.offsets)
+        K = torch.zeros((m.n_layers, r.n, m.n_kv_heads, m.head_dim), dtype=torch.bfloat16, device=dev)
+        V = torch.zeros_like(K)
+        fr = None if forced is None else torch.from_numpy(np.asarray(forced, dtype=np.int32)).to(dev)
+        req, out = eng.make_request(tab, len(ids), max(r.chunk_lens), r.n_ctx, nq, to_dev(x0, dev), K, V, ratio=r.ratio, select_layer=1, forced_re=fr)
+        return r, x0, req, out, K, V
+
+    refs = []
+    for j, (ids, nq) in enumerate(batch):
+        r, x0, _, _, _, _ = build(ids, nq, j)
+        refs.append(O.fuse_request([pool[i][0] for i in ids], [pool[i][1] for i in ids], x0, nq, weights, model, r.ratio, select_layer=1, rnd=O.round_bf16))
+    # (a) the batch with the library's own selections: exact top-p of its own scores, scores close to the oracle's
+    own = [build(ids, nq, j) for j, (ids, nq) in enumerate(batch)]
+    eng.fuse_batch([b[2] for b in own])
+    assert eng.device_status() == 0
+    for (r, x0, req, out, K, V), ref in zip(own, refs):
+        p = out["p"]
+        assert p == ref.Re.size
+        gs = out["scores"].cpu().numpy().astype(np.float64)
+        assert out["rows"].cpu().numpy()[:p].tolist() == O.topk_select(gs, 0, r.n_ctx, p).tolist()
+        rel = np.abs(gs[: r.n_ctx] - ref.scores[: r.n_ctx]) / ref.scores[: r.n_ctx]
+        assert rel.max() <= 3e-2, rel.max()
+    # (b) the same batch on the oracle's index sets: fused caches and final rows of every request, layer by layer
+    forced = [build(ids, nq, j, forced=ref.Re) for (j, (ids, nq)), ref in zip(enumerate(batch), refs)]
+    eng.fuse_batch([b[2] for b in forced])
+    assert eng.device_status() == 0
+    for (r, x0, req, out, K, V), ref in zip(forced, refs):
+        assert out["rows"].cpu().numpy()[: out["p"]].tolist() == ref.Re.tolist()
+        gK, gV = f64(K), f64(V)
+        for l in range(m.n_layers):
+            gate = KV_MEAN * 3 ** l  # as in test_fuse_request_matches_oracle for this distribution
+            check_drift(gK[l], ref.K[l], f"fused K layer {l}", gate)
+            check_drift(gV[l], ref.V[l], f"fused V layer {l}", gate)
+        check_drift(f64(out["x"]), ref.X, "final hidden rows", 6e-3 * float(np.abs(ref.X).std()) * 2 ** (m.n_layers - 1))
+    eng.close()
+
+
 def test_fuse_request_rejects_bad_arguments(a3mod):
     s = Setup(a3mod, "tiny")
     r = s.r

@@ -41,6 +41,23 @@ def make_engine(a3mod, m, seed=0, w_std=0.02, max_pos=40000, norm_jitter=0.1):
     return eng, layers, dev
 
 
+def hidden_rows_scale(x_exact) -> float:
+    """Factor on the K/V gates for a layer's hidden rows (which the benchmark spec does not bound), derived from the
+    arithmetic rather than read off a kernel.  The stated K/V gates are the cost of ONE bf16 rounding of values with a
+    spread of about 1.28: a bf16 rounding error is uniform within half an ulp, ulp/|x| averages ln2 * 2^-7, so the
+    mean error is |x| * ln2 * 2^-7 / 4 = 1.35e-3 |x| = 1.08e-3 sigma for normal values (E|x| = 0.8 sigma), and the
+    largest of 1e5..1e6 values (4.5 sigma) is off by up to 2^-8 * 4.5 sigma = 1.8e-2 sigma.  A hidden row x + Wo o +
+    MLP(.) carries, besides that final rounding, what only the kernels do: the probabilities enter the P V product as
+    bf16.  Each p_j is off by a relative error of rms 2^-9 / sqrt(3) = 1.13e-3, independent over j, so the attention
+    output is off by at most rms 1.13e-3 sigma_v (all weight on one key; less for flat rows), i.e. the attention branch
+    carries a relative error of up to 1.13e-3, and so does what the MLP makes of it.  With both branches no larger than
+    the row itself and an MLP gain g <= 2 around its input, the mean error is bounded by
+      1.08e-3 sigma + 0.8 * 1.13e-3 * (1 + g) sigma <= 3.8e-3 sigma,
+    and the maximum by 1.8e-2 sigma + 4.5 * 1.13e-3 * (1 + g) sigma <= 3.3e-2 sigma: twice the K/V gates per unit
+    spread (4e-3 sigma mean, 4e-2 sigma max) cover it with little room, which is what the tests use."""
+    return 2.0 * float(np.asarray(x_exact).std())
+
+
 def check_kv(got, want, what, scale=1.0):
     err = np.abs(got - want)
     assert err.max() <= KV_MAX * scale, f"{what}: max abs {err.max():.3e}"
@@ -413,12 +430,8 @@ def test_recompute_layer_parity(a3mod, shape, kv_len, M, seed):
     mask[pos] = False
     np.testing.assert_array_equal(gK[mask], Kc[layer][mask])  # rows outside R untouched, bit for bit
     np.testing.assert_array_equal(gV[mask], Vc[layer][mask])
-    # Hidden rows are not covered by the stated K/V gates.  Their bound: one bf16 rounding of the result (mean
-    # about 1.2e-3 per unit spread) plus what the one deliberate difference between the pipelines - attention
-    # probabilities enter the P.V tensor-core product as bf16 - becomes after the output projection and the MLP,
-    # whose gains exceed one with these weights (measured 2.5e-3..3e-3 per unit spread).  Gate: twice the K/V
-    # gates per unit spread of the result.
-    check_kv(gX, parts["x_exact"], "hidden rows", scale=2.0 * float(parts["x_exact"].std()))
+    # Hidden rows are not covered by the stated K/V gates; their bound is derived in hidden_rows_scale.
+    check_kv(gX, parts["x_exact"], "hidden rows", scale=hidden_rows_scale(parts["x_exact"]))
     np.testing.assert_allclose(lse.cpu().numpy(), parts["lse"], atol=5e-3)
     eng.close()
 
@@ -466,7 +479,7 @@ def test_recompute_layer_growing_logits(a3mod, shape, kv_len, M, beta):
     gX = f64(dX)
     assert np.isfinite(gX).all()
     check_kv(f64(dK)[pos], parts["k_exact"], "recomputed K rows")
-    check_kv(gX, parts["x_exact"], "hidden rows", scale=2.0 * float(parts["x_exact"].std()))
+    check_kv(gX, parts["x_exact"], "hidden rows", scale=hidden_rows_scale(parts["x_exact"]))
     # The two pipelines round q to bf16 from slightly different fp32 values; an element that lands on the other side
     # of a rounding boundary moves a logit by 2^-9 |q_e| |k_e| / sqrt(D), and the keys are large here: allow two such
     # flips per row on the log-sum-exp (the usual 5e-3 gate assumes keys of unit size).
@@ -686,7 +699,7 @@ def test_attention_two_row_tiles_per_cta(a3mod, shape, kv_len, M, grow):
     assert torch.equal(outs[0][0], outs[1][0]) and torch.equal(outs[0][1], outs[1][1])  # reproducible
     gX = f64(outs[0][0])
     assert np.isfinite(gX).all()
-    check_kv(gX, parts["x_exact"], "hidden rows", scale=2.0 * float(parts["x_exact"].std()))
+    check_kv(gX, parts["x_exact"], "hidden rows", scale=hidden_rows_scale(parts["x_exact"]))
     lse_tol = 2 * 2.0 ** -9 * float(np.abs(parts["q"]).max()) * float(np.abs(Kc).max()) / np.sqrt(m.head_dim)
     np.testing.assert_allclose(outs[0][1].cpu().numpy(), parts["lse"], atol=max(5e-3, lse_tol), rtol=1e-5)
     eng.close()
@@ -731,7 +744,7 @@ def test_qkv_three_head_tiles(a3mod, shape, kv_len, M):
     mask[pos] = False
     np.testing.assert_array_equal(gK[mask], Kc[layer][mask])
     np.testing.assert_array_equal(gV[mask], Vc[layer][mask])
-    check_kv(f64(outs[384][0]), parts["x_exact"], "hidden rows", scale=2.0 * float(parts["x_exact"].std()))
+    check_kv(f64(outs[384][0]), parts["x_exact"], "hidden rows", scale=hidden_rows_scale(parts["x_exact"]))
     eng.close()
 
 
@@ -766,7 +779,7 @@ def test_swiglu_narrow_column_tiles(a3mod, shape, M, g):
     assert torch.equal(outs[g], outs[0])
     Ko, Vo = Kc[layer].astype(np.float64), Vc[layer].astype(np.float64)
     Xo, parts = O.recompute_layer(X.astype(np.float64), pos, weights[layer], model, Ko, Vo, rnd=O.round_bf16, return_parts=True)
-    check_kv(f64(outs[g]), parts["x_exact"], "hidden rows", scale=2.0 * float(parts["x_exact"].std()))
+    check_kv(f64(outs[g]), parts["x_exact"], "hidden rows", scale=hidden_rows_scale(parts["x_exact"]))
     eng.close()
 
 
@@ -801,7 +814,7 @@ def test_swiglu_pair_kernel_matches_one_cta_kernel(a3mod, shape, M):
     assert torch.equal(outs[1][0], outs[0][0])
     Ko, Vo = Kc[layer].astype(np.float64), Vc[layer].astype(np.float64)
     Xo, parts = O.recompute_layer(X.astype(np.float64), pos, weights[layer], model, Ko, Vo, rnd=O.round_bf16, return_parts=True)
-    check_kv(f64(outs[1][0]), parts["x_exact"], "hidden rows", scale=2.0 * float(parts["x_exact"].std()))
+    check_kv(f64(outs[1][0]), parts["x_exact"], "hidden rows", scale=hidden_rows_scale(parts["x_exact"]))
     eng.close()
 
 
@@ -835,7 +848,7 @@ def test_residual_persistent_pair_kernel_matches_tile_kernel(a3mod, shape, M):
     assert torch.equal(outs[2], outs[0])
     Ko, Vo = Kc[layer].astype(np.float64), Vc[layer].astype(np.float64)
     Xo, parts = O.recompute_layer(X.astype(np.float64), pos, weights[layer], model, Ko, Vo, rnd=O.round_bf16, return_parts=True)
-    check_kv(f64(outs[2]), parts["x_exact"], "hidden rows", scale=2.0 * float(parts["x_exact"].std()))
+    check_kv(f64(outs[2]), parts["x_exact"], "hidden rows", scale=hidden_rows_scale(parts["x_exact"]))
     eng.close()
 
 
@@ -916,7 +929,7 @@ def test_attention_logit_spikes(a3mod, pair):
     assert eng.device_status() == 0
     gX = f64(dX)
     assert np.isfinite(gX).all()
-    check_kv(gX, parts["x_exact"], "hidden rows", scale=2.0 * float(parts["x_exact"].std()))
+    check_kv(gX, parts["x_exact"], "hidden rows", scale=hidden_rows_scale(parts["x_exact"]))
     lse_tol = 2 * 2.0 ** -9 * float(np.abs(q).max()) * float(np.abs(Kc).max()) / np.sqrt(m.head_dim)
     np.testing.assert_allclose(lse.cpu().numpy(), parts["lse"], atol=max(5e-3, lse_tol), rtol=1e-5)
     eng.close()
