@@ -416,14 +416,22 @@ extern "C" int a3_query_scores(const a3_handle* h, const void* q_rows, const int
 
 // ------------------------------------------------------------------ the whole request
 namespace a3 {
-// layer_ready (optional, [n_layers]): event after which layer l's chunk caches are in device memory; position
-// recovery of layer l is then queued behind it, just before the layer needs the cache (host-buffer entry).
-static int fuse_impl(const a3_handle* h, const a3_request* r, void* ws, size_t ws_bytes, a3_stream stream,
-                     const cudaEvent_t* layer_ready, cudaEvent_t x0_ready);
+// The host-buffer entry feeds the request: layer_ready[l] is the event after which layer l's chunk caches are in device
+// memory; position recovery of layer l is queued behind it, just before the layer needs the cache.  The copies
+// themselves are queued a few layers ahead of the compute launches that need them (queue_layer), not all up front:
+// thousands of small copies take the host tens of milliseconds to queue, which would otherwise delay the first launch.
+struct HostFeed {
+  const cudaEvent_t* layer_ready;  // [n_layers]
+  cudaEvent_t x0_ready;
+  void* ctx;
+  int (*queue_layer)(void* ctx, int layer);  // queues the copies of one layer on the copy stream, records layer_ready[layer]
+  int next;                                  // first layer whose copies are not queued yet
+};
+static int fuse_impl(const a3_handle* h, const a3_request* r, void* ws, size_t ws_bytes, a3_stream stream, HostFeed* feed);
 }
 
 extern "C" int a3_fuse_request(const a3_handle* h, const a3_request* r, void* ws, size_t ws_bytes, a3_stream stream) {
-  return fuse_impl(h, r, ws, ws_bytes, stream, nullptr, nullptr);
+  return fuse_impl(h, r, ws, ws_bytes, stream, nullptr);
 }
 
 // ---------------------------------------------------------------- the request as a CUDA graph
@@ -487,9 +495,19 @@ extern "C" void a3_graph_destroy(a3_graph* g) {
   free(g);
 }
 
-static int a3::fuse_impl(const a3_handle* h, const a3_request* r, void* ws, size_t ws_bytes, a3_stream stream,
-                         const cudaEvent_t* layer_ready, cudaEvent_t x0_ready) {
+static int a3::fuse_impl(const a3_handle* h, const a3_request* r, void* ws, size_t ws_bytes, a3_stream stream, HostFeed* feed) {
   if (!h || !r || !ws) return A3_EINVAL;
+  const cudaEvent_t* layer_ready = feed ? feed->layer_ready : nullptr;
+  const cudaEvent_t x0_ready = feed ? feed->x0_ready : nullptr;
+  // copies of the layers up to `upto` are on their way (host-buffer entry only)
+  auto feed_to = [&](int upto) -> int {
+    while (feed && feed->next <= upto && feed->next < h->m.n_layers) {
+      A3_TRY(feed->queue_layer(feed->ctx, feed->next));
+      ++feed->next;
+    }
+    return A3_OK;
+  };
+  constexpr int FEED_AHEAD = 3;
   const a3_model_desc& m = h->m;
   if (r->n_ctx < 0 || r->n_question < 0 || r->n_system < 0 || r->n_system > r->n_ctx || r->n_chunks < 0) return A3_EINVAL;
   const int n = r->n_ctx + r->n_question;
@@ -573,7 +591,11 @@ static int a3::fuse_impl(const a3_handle* h, const a3_request* r, void* ws, size
   if (x0_ready) A3_CUDA(cudaStreamWaitEvent(st, x0_ready, 0));
   A3_CUDA(cudaMemcpyAsync(w.x_all, r->x0, (size_t)n * m.d_model * 2, cudaMemcpyDeviceToDevice, st));
   A3_TRY(iota_rows(h, w.all_pos, 0, n, st));
-  for (int l = 0; l < ls; ++l) A3_TRY(layer_step(l, w.x_all, w.all_pos, n));
+  for (int l = 0; l < ls; ++l) {
+    A3_TRY(feed_to(ls + 1 + FEED_AHEAD * (l + 1)));  // a full block is long: several layers' copies fit under it
+    A3_TRY(layer_step(l, w.x_all, w.all_pos, n));
+  }
+  A3_TRY(feed_to(ls + 1 + FEED_AHEAD));
   // selection layer: true K, V for all rows, queries of the question rows, scores, Re (Eq. 3)
   A3_TRY(rmsnorm_rows(h, w.x_all, (const bf16*)h->layers[ls].attn_norm, m.rms_eps, n, m.d_model, lw.a, st));
   A3_TRY(qkv_project(h, ls, lw.a, w.all_pos, n, r->n_ctx, lw.q, kl(ls), vl(ls), n, st));
@@ -590,6 +612,7 @@ static int a3::fuse_impl(const a3_handle* h, const a3_request* r, void* ws, size
   }
   A3_TRY(iota_rows(h, r->rows_out + p, r->n_ctx, nq, st));
   if (M == 0) {
+    A3_TRY(feed_to(m.n_layers));
     if (layer_ready)
       for (int l = ls + 1; l < m.n_layers; ++l) {
         A3_CUDA(cudaStreamWaitEvent(st, layer_ready[l], 0));
@@ -601,6 +624,7 @@ static int a3::fuse_impl(const a3_handle* h, const a3_request* r, void* ws, size
   A3_TRY(a3_gather_rows(h, w.x_all, n, r->rows_out, M, m.d_model, r->x_out, stream));
   // layers select_layer..L-1 on rows [Re, Q] only (Eq. 4, Eq. 5)
   for (int l = ls; l < m.n_layers; ++l) {
+    A3_TRY(feed_to(l + FEED_AHEAD));
     if (layer_ready && l > ls) {
       A3_CUDA(cudaStreamWaitEvent(st, layer_ready[l], 0));
       A3_TRY(a3_rope_rerotate(h, r->chunks, r->n_chunks, r->max_chunk_len, r->k_fused, r->v_fused, r->layer_stride, r->n_ctx, l, l + 1, stream));
@@ -751,19 +775,31 @@ extern "C" int a3_fuse_request_host(const a3_handle* h, const a3_request* req, c
     note(cudaMemcpyAsync(dref, href, sizeof(a3_chunk_ref) * req->n_chunks, cudaMemcpyHostToDevice, cs));
   if (status == A3_OK) note(cudaMemcpyAsync(x0, io->x0, (size_t)n * m.d_model * 2, cudaMemcpyHostToDevice, cs));
   if (status == A3_OK) note(cudaEventRecord(hp->x0_ready, cs));
-  for (int l = req->select_layer + 1; l < m.n_layers && status == A3_OK; ++l) {
-    for (int c = 0; c < req->n_chunks && status == A3_OK; ++c) {
-      const size_t slice = (size_t)href[c].len * row;
-      if (note(cudaMemcpyAsync((char*)href[c].k_src + l * slice, (const char*)io->chunk_k[c] + l * slice, slice, cudaMemcpyHostToDevice, cs)))
-        note(cudaMemcpyAsync((char*)href[c].v_src + l * slice, (const char*)io->chunk_v[c] + l * slice, slice, cudaMemcpyHostToDevice, cs));
-    }
-    if (status == A3_OK) note(cudaEventRecord(hp->layer_ready[l], cs));
-  }
   a3_request r = *req;
   r.chunks = dref;
   r.max_chunk_len = maxlen;
   r.x0 = x0;
-  if (status == A3_OK) status = fuse_impl(h, &r, ws, ws_bytes, stream, hp->layer_ready, hp->x0_ready);
+  struct FeedCtx {
+    const a3_chunk_ref* href;
+    const a3_host_io* io;
+    int n_chunks;
+    size_t row;
+    cudaStream_t cs;
+    cudaEvent_t* layer_ready;
+  } fc{href, io, req->n_chunks, row, cs, hp->layer_ready};
+  HostFeed feed{hp->layer_ready, hp->x0_ready, &fc,
+                [](void* ctx, int l) -> int {
+                  FeedCtx* f = (FeedCtx*)ctx;
+                  for (int c = 0; c < f->n_chunks; ++c) {
+                    const size_t slice = (size_t)f->href[c].len * f->row;
+                    A3_CUDA(cudaMemcpyAsync((char*)f->href[c].k_src + l * slice, (const char*)f->io->chunk_k[c] + l * slice, slice, cudaMemcpyHostToDevice, f->cs));
+                    A3_CUDA(cudaMemcpyAsync((char*)f->href[c].v_src + l * slice, (const char*)f->io->chunk_v[c] + l * slice, slice, cudaMemcpyHostToDevice, f->cs));
+                  }
+                  A3_CUDA(cudaEventRecord(f->layer_ready[l], f->cs));
+                  return A3_OK;
+                },
+                req->select_layer + 1};
+  if (status == A3_OK) status = fuse_impl(h, &r, ws, ws_bytes, stream, &feed);
   const int M = r.n_recompute + r.n_question;
   if (status == A3_OK && M > 0) {
     if (note(cudaMemcpyAsync(io->rows_out, r.rows_out, (size_t)M * 4, cudaMemcpyDeviceToHost, st)))
