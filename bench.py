@@ -33,7 +33,9 @@ if ROOT not in sys.path:
 # DRAM bytes (read + write) per launch of the dominant kernel classes from the ncu captures summarised under profiles/
 # (gemm_kernels_llama8b_2layer.txt: SwiGLU GEMM of a sparse layer, M = 804, and of the full block, M = 5152;
 # attention_kernels_*: see that file).  Used for `roofline.traffic` of the workloads they were captured on.
-NCU_TRAFFIC = {("llama8b_10x512", "gemm_swiglu"): {"sparse": 243.44e6 + 18.51e6, "full": 418.15e6 + 140.63e6}}
+NCU_TRAFFIC = {("llama8b_10x512", "gemm_swiglu"): {"sparse": 243.44e6 + 18.51e6, "full": 418.15e6 + 140.63e6},
+               # attention_and_selection_kernels_llama8b_64x512_2layer.txt: sparse rows (4 952) and the full causal block (32 800)
+               ("llama8b_64x512", "attention"): {"sparse": 419.97e6 + 35.71e6, "full": 2208.55e6 + 265.24e6}}
 
 METRIC = "context_tokens_fused_per_s"
 UNIT = "tokens/s"
@@ -469,7 +471,8 @@ class RequestWorkload:
         t = NCU_TRAFFIC.get((self.name, top))
         if t:
             nf = self.r.select_layer
-            traffic = (t["full"] * nf + t["sparse"] * (self.m.n_layers - nf)) / self.m.n_layers  # average over the class's launches
+            # launch-weighted mean over the class's launches: the leading full blocks, then one sparse-row launch per later layer
+            traffic = (t["full"] * nf + t["sparse"] * (self.m.n_layers - nf)) / self.m.n_layers
         return {"kernel": top, "bound": tk.get("bound"), "achieved": tk.get("achieved"),
                 "peak": peaks["bf16_tflops_sustained"] if tk.get("bound") == "tensor" else peaks["hbm_gbs"],
                 "unit": tk.get("unit"), "frac": tk.get("frac"), "frac_burst": tk.get("frac_burst"),
