@@ -620,7 +620,28 @@ def measure_context(eng, wl, timer, peaks, req_ms):
     first_token_ms = timer.run(lambda: eng.first_token(x_last, fnorm, lm_head, want_logits=False), 10, sync_ranks=False) / 10 * 1e3
     first_token_gbs = m.vocab * m.d_model * 2 / (first_token_ms * 1e-3) / 1e9
     del lm_head
-    return {"full_prefill_ms": full_prefill_ms, "speedup_vs_full_prefill": full_prefill_ms / req_ms,
+    # the standalone HBM-streaming steps of Eq. 4 / Eq. 5 (row gather, K/V scatter) on a synthetic case far beyond the L2:
+    # 65 536 rows into / out of 262 144 slots; bytes = rows read + rows written
+    n_big, m_big = 262144, 65536
+    g.manual_seed(9)
+    slots = torch.sort(torch.randperm(n_big, device=dev, generator=g)[:m_big]).values.to(torch.int32)
+    kr = torch.randn((m_big, m.n_kv_heads, m.head_dim), device=dev, generator=g).to(torch.bfloat16)
+    Kc = torch.zeros((n_big, m.n_kv_heads, m.head_dim), dtype=torch.bfloat16, device=dev)
+    Vc = torch.zeros_like(Kc)
+    eng.scatter_kv(kr, kr, slots, Kc, Vc)
+    scatter_s = timer.run(lambda: eng.scatter_kv(kr, kr, slots, Kc, Vc), 10, sync_ranks=False) / 10
+    scatter_gbs = 4.0 * m_big * m.n_kv_heads * m.head_dim * 2 / scatter_s / 1e9
+    del Vc, kr
+    src = Kc.view(-1)[: (n_big // 4) * m.d_model].view(n_big // 4, m.d_model)  # any rows will do: [65 536][d]
+    rows = torch.sort(torch.randperm(n_big // 4, device=dev, generator=g)[: m_big // 4]).values.to(torch.int32)
+    dst = torch.empty((m_big // 4, m.d_model), dtype=torch.bfloat16, device=dev)
+    eng.gather_rows(src, rows, dst)
+    gather_s = timer.run(lambda: eng.gather_rows(src, rows, dst), 10, sync_ranks=False) / 10
+    gather_gbs = 2.0 * (m_big // 4) * m.d_model * 2 / gather_s / 1e9
+    del Kc, src, dst
+    return {"hbm_steps": {"scatter_kv": {"rows": m_big, "achieved_gbs": scatter_gbs, "frac_of_hbm_peak": scatter_gbs / peaks["hbm_gbs"]},
+                          "gather_rows": {"rows": m_big // 4, "achieved_gbs": gather_gbs, "frac_of_hbm_peak": gather_gbs / peaks["hbm_gbs"]}},
+            "full_prefill_ms": full_prefill_ms, "speedup_vs_full_prefill": full_prefill_ms / req_ms,
             "scores_from_cached_keys": {"request_ms": cached_ms, "tokens_per_s": r.n_ctx / (cached_ms * 1e-3),
                                         "selection_overlap_with_true_keys": overlap},
             "ex_eviction": {"capacity": 1024, "pool": 7, "request_ms": evict_ms, "overhead_ms": evict_ms - req_ms},
