@@ -628,10 +628,11 @@ def measure_context(eng, wl, timer, peaks, req_ms):
     kr = torch.randn((m_big, m.n_kv_heads, m.head_dim), device=dev, generator=g).to(torch.bfloat16)
     Kc = torch.zeros((n_big, m.n_kv_heads, m.head_dim), dtype=torch.bfloat16, device=dev)
     Vc = torch.zeros_like(Kc)
-    eng.scatter_kv(kr, kr, slots, Kc, Vc)
-    scatter_s = timer.run(lambda: eng.scatter_kv(kr, kr, slots, Kc, Vc), 10, sync_ranks=False) / 10
+    vr = torch.randn((m_big, m.n_kv_heads, m.head_dim), device=dev, generator=g).to(torch.bfloat16)
+    eng.scatter_kv(kr, vr, slots, Kc, Vc)
+    scatter_s = timer.run(lambda: eng.scatter_kv(kr, vr, slots, Kc, Vc), 10, sync_ranks=False) / 10
     scatter_gbs = 4.0 * m_big * m.n_kv_heads * m.head_dim * 2 / scatter_s / 1e9
-    del Vc, kr
+    del Vc, kr, vr
     src = Kc.view(-1)[: (n_big // 4) * m.d_model].view(n_big // 4, m.d_model)  # any rows will do: [65 536][d]
     rows = torch.sort(torch.randperm(n_big // 4, device=dev, generator=g)[: m_big // 4]).values.to(torch.int32)
     dst = torch.empty((m_big // 4, m.d_model), dtype=torch.bfloat16, device=dev)

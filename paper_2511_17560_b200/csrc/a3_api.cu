@@ -168,6 +168,7 @@ extern "C" int a3_create(a3_handle** out, const a3_model_desc* m, const a3_layer
   h->opt[A3_OPT_SWIGLU_NARROW] = 1;
   h->opt[A3_OPT_SWIGLU_PAIR] = 1;
   h->opt[A3_OPT_RESIDUAL_T] = 1;
+  h->opt[A3_OPT_QKV_T] = 1;
   h->opt[A3_OPT_GEMM_BN_SWIGLU] = 256;  // the one-CTA gate/up kernel runs two CTAs per SM: 256 columns, 2 stages
   h->opt[A3_OPT_GEMM_STAGES_SWIGLU] = 2;
   h->layers = (a3_layer_weights*)malloc(sizeof(a3_layer_weights) * m->n_layers);

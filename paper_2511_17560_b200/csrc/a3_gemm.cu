@@ -626,6 +626,7 @@ int gemm_bf16(const a3_handle* h, GemmEpilogue epi, const GemmArgs& a, cudaStrea
   int bn = h->opt[A3_OPT_GEMM_BN_RESIDUAL + (int)epi];
   int stages = h->opt[A3_OPT_GEMM_STAGES_RESIDUAL + (int)epi];
   if (epi == EPI_RESIDUAL && bn == 0 && residual_t_usable(h, a)) return gemm_residual_t(h, a, st);
+  if (epi == EPI_QKV && bn == 0 && qkv_t_usable(h, a)) return gemm_qkv_t(h, a, st);
 
   if (bn == 0) {
     const int m_tiles = cdiv(a.M, TC_BM), sms = h->sm_count > 0 ? h->sm_count : 148;

@@ -32,6 +32,9 @@ constexpr int SP_SUB = 2;  // k-blocks of 64 per ring stage: one barrier hand-sh
 constexpr int SP_FEAT = 64;                              // features per CTA (64 gate lanes + 64 up lanes)
 constexpr int SP_A_BYTES = 2 * SP_FEAT * TC_BK * 2;      // 16 KiB: gate rows, then up rows
 constexpr int SP_XCH_BYTES = 2 * 2 * 32 * SP_FEAT * 4;   // per warp set: two buffers of float [32 tokens][64 features]
+constexpr int SP_QKV_SET_FLOATS = 4 * (32 * 32 + 4);            // QKV: per warp set, four quarters of [32 tokens][32 features] fp32, 16 bytes apart in the banks
+constexpr int SP_QKV_XCH_BYTES = 2 * SP_QKV_SET_FLOATS * 4 + 128;  // + room to keep the next field 256-byte aligned
+constexpr int SP_QKV_EXTRA = SP_QKV_XCH_BYTES + 256;              // ... and the checked positions of a chunk's tokens per set
 constexpr int SP_SMEM_LIMIT = 227 * 1024;
 
 struct SpParams {
@@ -42,6 +45,15 @@ struct SpParams {
   bf16* C;
   int ldc;
   uint32_t* status;
+  // EPI_QKV: the concatenated heads of up to three matrices (q, k, v in any subset), 128 features each
+  int n_heads;
+  int seg_heads_end[3];  // cumulative head counts of the segments
+  int kind[3];           // 0 = q, 1 = k, 2 = v
+  const bf16* bias[3];
+  bf16 *q_out, *k_cache, *v_cache;
+  const int32_t* pos;
+  int kv_len, Hq, Hkv, layout, max_pos;
+  const float2* tab;
 };
 
 __device__ __forceinline__ void named_bar_sync(int id, int threads) {
@@ -80,16 +92,20 @@ __device__ __forceinline__ void tc_mma_pair_acc(uint32_t d_tmem, uint64_t a_desc
 
 // EPI_SWIGLU: tmG/tmU are the gate and up matrices (box of 64 rows each); EPI_RESIDUAL: tmG is the one weight matrix
 // (box of 128 rows, tmU unused) and the epilogue adds the accumulator to C in place.
+// EPI_QKV: tmG / tmU / tmW are the matrices of the segments (boxes of 128 rows: one head); a unit is two consecutive
+// heads of the concatenated list, one per CTA of the pair, times one token tile; the epilogue adds the bias, rotates
+// q and k at the tokens' positions (the two halves of a rotation pair sit 64 lanes apart and meet through shared
+// memory, like gate and up) and writes q to its buffer and k, v into the cache rows pos[token] (the scatter of Eq. 5).
 template <int EPI>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(SP_THREADS, 1)
 pair_t_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUtensorMap tmG,
-              const __grid_constant__ CUtensorMap tmU, const SpParams p) {
+              const __grid_constant__ CUtensorMap tmU, const __grid_constant__ CUtensorMap tmW, const SpParams p) {
   constexpr int ROWS = EPI == EPI_SWIGLU ? SP_FEAT : 2 * SP_FEAT;  // output features per CTA
   extern __shared__ unsigned char smem_raw[];
   const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;  // same offset in both CTAs of the pair
   unsigned char* base_ptr = smem_raw + (base - smem_u32(smem_raw));
   const int S = p.stages;
-  const int xch_off = S * p.stage_bytes, bar_off = xch_off + (EPI == EPI_SWIGLU ? SP_XCH_BYTES : 0);
+  const int xch_off = S * p.stage_bytes, bar_off = xch_off + (EPI == EPI_SWIGLU ? SP_XCH_BYTES : (EPI == EPI_QKV ? SP_QKV_EXTRA : 0));
   // barriers (8 bytes each): full[8] (used in the leader), empty[8], tmem_full[2], tmem_empty[2] (used in the leader)
   const uint32_t bars = base + bar_off;
   auto full_bar = [&](int s) { return bars + 8u * s; };
@@ -116,7 +132,7 @@ pair_t_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ C
     }
     for (int b = 0; b < 2; ++b) {
       mbar_init(tmem_full(b), 1);
-      // SwiGLU: the gate warps and the up warps of both warp sets of each CTA; residual: every epilogue warp
+      // SwiGLU: the gate warps and the up warps of both warp sets of each CTA; residual and QKV: every epilogue warp
       mbar_init(tmem_empty(b), EPI == EPI_SWIGLU ? 8 : 16);
     }
     abort_flag[0] = 0;
@@ -146,8 +162,19 @@ pair_t_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ C
       int s = 0;        // ring position and phase, kept by counting: S is a run-time value and a division per
       uint32_t ph = 0;  // k-block is a long dependent chain in a one-thread role
       bool ok = true;
+      if (EPI == EPI_QKV) tmap_prefetch(&tmW);
       for (int u = pair; u < p.n_units && ok; u += p.n_pairs) {
-        const int f0 = (u / p.tok_tiles) * (2 * ROWS) + (int)rank * ROWS;
+        int f0 = (u / p.tok_tiles) * (2 * ROWS) + (int)rank * ROWS;
+        const CUtensorMap* mapA = &tmG;
+        if (EPI == EPI_QKV) {
+          // this CTA's head of the concatenated list -> its matrix and first row there (a pair beyond the last head of
+          // an odd list loads head 0 again; its epilogue stores nothing)
+          int hd = 2 * (u / p.tok_tiles) + (int)rank;
+          if (hd >= p.n_heads) hd = 0;
+          const int sg = (hd >= p.seg_heads_end[0]) + (hd >= p.seg_heads_end[1]);
+          f0 = (hd - (sg == 0 ? 0 : p.seg_heads_end[sg - 1])) * 128;
+          mapA = sg == 0 ? &tmG : (sg == 1 ? &tmU : &tmW);
+        }
         const int t0 = (u % p.tok_tiles) * p.tok_n + (int)rank * half_n;
         for (int kb = 0; kb < KT; kb += SP_SUB, ++kbg) {
           if (!mbar_wait(empty_bar(s), ph ^ 1, abort_flag, p.status)) {
@@ -162,7 +189,7 @@ pair_t_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ C
 #pragma unroll
           for (int j = 0; j < SP_SUB; ++j) {
             const uint32_t sa = base + s * p.stage_bytes + j * p.sub_bytes, sb = sa + SP_A_BYTES;
-            tma_load_2d_pair(sa, &tmG, (kb + j) * TC_BK, f0, full_leader);
+            tma_load_2d_pair(sa, mapA, (kb + j) * TC_BK, f0, full_leader);
             if (EPI == EPI_SWIGLU) tma_load_2d_pair(sa + SP_A_BYTES / 2, &tmU, (kb + j) * TC_BK, f0, full_leader);
             tma_load_2d_pair(sb, &tmX, (kb + j) * TC_BK, t0, full_leader);
           }
@@ -315,6 +342,121 @@ pair_t_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ C
       named_bar_sync(bar_group, 64);
       if (lane == 0 && (quarter == 0 || quarter == 2)) mbar_arrive_in_cta(tmem_empty(b), 0);
     }
+  } else if (EPI == EPI_QKV) {
+    // ---------------- epilogue, q / k / v heads: warps 2..9 of both CTAs; warp w may touch TMEM lanes 32*(w%4) .. +31,
+    // lane = feature of this CTA's head; warp set 0 (warps 2..5) takes the first half of the token columns, set 1 the
+    // second.  32 tokens at a time, in two phases around a named barrier of the set's 128 threads:
+    //   1. feature-major: every warp reads its 32 features x 32 tokens from tensor memory, adds the bias and parks the
+    //      values in shared memory; the first warp also fetches and checks the tokens' positions;
+    //   2. token-major: a thread takes 8 consecutive features of the head's first half and the 8 that lie 64 further of
+    //      ONE token (both halves of its rotation pairs, whichever the pairing), rotates them with 16-byte loads of the
+    //      token's table row and writes two 16-byte vectors: a warp stores 512 contiguous-by-row bytes per instruction
+    //      where a lane-per-feature epilogue stores 64.
+    const int quarter = warp & 3;
+    const int set = (warp - 2) >> 2;
+    const int ep_tid = (warp - 2) * 32 + lane;
+    const int st = quarter * 32 + lane;  // thread within the set
+    const int set_n = p.tok_n >> 1;
+    const int n_chunks = (set_n + 31) >> 5;
+    float* xset = xch + set * SP_QKV_SET_FLOATS;
+    int* posbuf = reinterpret_cast<int*>(base_ptr + xch_off + SP_QKV_XCH_BYTES) + set * 32;
+    const int bar_set = 2 + set;
+    // phase 2 assignment: token e2 (+16 in the second pass), features f0 .. f0 + 7 and 64 + f0 .. 64 + f0 + 7
+    const int e2 = st >> 3, f0 = (st & 7) * 8;
+    const float* xlo = xset + (f0 >> 5) * (32 * 32 + 4) + (f0 & 31);
+    const float* xhi = xset + (2 + (f0 >> 5)) * (32 * 32 + 4) + (f0 & 31);
+    float* xmine = xset + quarter * (32 * 32 + 4) + lane;
+    int it = 0;
+    for (int u = pair; u < p.n_units; u += p.n_pairs, ++it) {
+      const int b = it & 1;
+      const int hd = 2 * (u / p.tok_tiles) + (int)rank;
+      const bool live = hd < p.n_heads;
+      const int hde = live ? hd : 0;
+      const int sg = (hde >= p.seg_heads_end[0]) + (hde >= p.seg_heads_end[1]);
+      const int head_in_seg = hde - (sg == 0 ? 0 : p.seg_heads_end[sg - 1]);
+      const int kind = p.kind[sg];
+      const int t0 = (u % p.tok_tiles) * p.tok_n + set * set_n;
+      const float bias = p.bias[sg] ? __bfloat162float(p.bias[sg][head_in_seg * 128 + quarter * 32 + lane]) : 0.f;
+      const bool rotate = kind != 2;
+      if (ep_tid == 0) ep_ok[0] = mbar_wait(tmem_full(b), (it >> 1) & 1, abort_flag, p.status) ? 1 : 0;
+      named_bar_sync(1, 256);
+      if (!ep_ok[0]) break;  // uniform for the 256 threads
+      tc_fence_after();
+      const uint32_t trow = tmem_base + (uint32_t)b * 256u + (uint32_t)(set * set_n) + ((uint32_t)(quarter * 32) << 16);
+#pragma unroll 1
+      for (int c = 0; c < n_chunks; ++c) {
+        const int w = min(32, set_n - c * 32);
+        const int valid = min(w, p.M - (t0 + c * 32));  // tokens of this chunk that exist (may be <= 0)
+        float v[32];
+        __syncwarp();
+        sp_ld_chunk(trow + c * 32, w, v);
+        if (quarter == 0) {  // positions of the chunk's tokens, checked: -1 where nothing is to be written
+          int ps = -1;
+          if (lane < valid) {
+            ps = p.pos[t0 + c * 32 + lane];
+            if (ps < 0 || ps >= p.kv_len || ps >= p.max_pos) {
+              if (live) atomicOr(p.status, A3_DEV_BAD_POSITION);
+              ps = -1;
+            }
+          }
+          posbuf[lane] = ps;
+        }
+#pragma unroll
+        for (int e = 0; e < 32; ++e) xmine[e * 32] = v[e] + bias;
+        named_bar_sync(bar_set, 128);
+#pragma unroll
+        for (int pass = 0; pass < 2; ++pass) {
+          const int e = e2 + 16 * pass;
+          const int ps = posbuf[e];
+          if (ps < 0 || !live) continue;
+          float a[8], bq[8], ra[8], rb[8];
+          *reinterpret_cast<float4*>(a) = *reinterpret_cast<const float4*>(xlo + e * 32);
+          *reinterpret_cast<float4*>(a + 4) = *reinterpret_cast<const float4*>(xlo + e * 32 + 4);
+          *reinterpret_cast<float4*>(bq) = *reinterpret_cast<const float4*>(xhi + e * 32);
+          *reinterpret_cast<float4*>(bq + 4) = *reinterpret_cast<const float4*>(xhi + e * 32 + 4);
+          if (!rotate) {
+#pragma unroll
+            for (int k = 0; k < 8; ++k) ra[k] = a[k], rb[k] = bq[k];
+          } else if (p.layout == 0) {
+            // pairs (i, i + 64): the thread's first 8 features rotate with the 8 that lie 64 further, frequencies f0 .. f0 + 7
+            const float4* tr = reinterpret_cast<const float4*>(p.tab + (size_t)ps * 64 + f0);
+#pragma unroll
+            for (int k = 0; k < 4; ++k) {
+              const float4 t = __ldg(tr + k);  // (cos, sin) of two frequencies
+              ra[2 * k] = a[2 * k] * t.x - bq[2 * k] * t.y;
+              rb[2 * k] = a[2 * k] * t.y + bq[2 * k] * t.x;
+              ra[2 * k + 1] = a[2 * k + 1] * t.z - bq[2 * k + 1] * t.w;
+              rb[2 * k + 1] = a[2 * k + 1] * t.w + bq[2 * k + 1] * t.z;
+            }
+          } else {
+            // pairs (2i, 2i + 1): both groups of 8 hold four pairs of their own, frequencies f0/2 .. and 32 + f0/2 ..
+            const float4* tl = reinterpret_cast<const float4*>(p.tab + (size_t)ps * 64 + (f0 >> 1));
+            const float4* th = reinterpret_cast<const float4*>(p.tab + (size_t)ps * 64 + 32 + (f0 >> 1));
+#pragma unroll
+            for (int k = 0; k < 2; ++k) {
+              const float4 t = __ldg(tl + k), u4 = __ldg(th + k);
+              ra[4 * k] = a[4 * k] * t.x - a[4 * k + 1] * t.y;
+              ra[4 * k + 1] = a[4 * k] * t.y + a[4 * k + 1] * t.x;
+              ra[4 * k + 2] = a[4 * k + 2] * t.z - a[4 * k + 3] * t.w;
+              ra[4 * k + 3] = a[4 * k + 2] * t.w + a[4 * k + 3] * t.z;
+              rb[4 * k] = bq[4 * k] * u4.x - bq[4 * k + 1] * u4.y;
+              rb[4 * k + 1] = bq[4 * k] * u4.y + bq[4 * k + 1] * u4.x;
+              rb[4 * k + 2] = bq[4 * k + 2] * u4.z - bq[4 * k + 3] * u4.w;
+              rb[4 * k + 3] = bq[4 * k + 2] * u4.w + bq[4 * k + 3] * u4.z;
+            }
+          }
+          bf16* dst = kind == 0 ? p.q_out + (size_t)(t0 + c * 32 + e) * (p.Hq * 128) + head_in_seg * 128
+                    : (kind == 1 ? p.k_cache : p.v_cache) + (size_t)ps * (p.Hkv * 128) + head_in_seg * 128;
+          *reinterpret_cast<uint4*>(dst + f0) = pack8(ra);
+          *reinterpret_cast<uint4*>(dst + 64 + f0) = pack8(rb);
+        }
+        named_bar_sync(bar_set, 128);  // everybody has read this chunk's values and positions
+      }
+      // this warp has read its part of the accumulator (wait::ld in sp_ld_chunk): it goes back to the MMA issuer
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive_in_cta(tmem_empty(b), 0);
+    }
   } else if (EPI == EPI_RESIDUAL) {
     // ---------------- epilogue, C += A B^T: warps 2..9 of both CTAs; warp w may touch TMEM lanes 32*(w%4) .. +31,
     // lane = output feature; warp set 0 (warps 2..5) takes the first half of the token columns, set 1 the second.
@@ -420,7 +562,82 @@ static int launch_pair_t(const a3_handle* h, const GemmArgs& a, cudaStream_t st)
   static SmemAttrOnce attr;
   A3_TRY(smem_attr_once(attr, h->device, pair_t_kernel<EPI>, SP_SMEM_LIMIT));
   ProfScope prof(h, EPI == EPI_SWIGLU ? A3_K_GEMM_SWIGLU : A3_K_GEMM_RESIDUAL, st);
-  A3_CUDA(launch_pdl(pair_t_kernel<EPI>, dim3(2 * p.n_pairs), dim3(SP_THREADS), (size_t)smem_bytes, st, tX, tG, tU, p));
+  A3_CUDA(launch_pdl(pair_t_kernel<EPI>, dim3(2 * p.n_pairs), dim3(SP_THREADS), (size_t)smem_bytes, st, tX, tG, tU, tU, p));
+  A3_LAUNCHED();
+  return A3_OK;
+}
+
+// QKV projection on the same kernel: one head (128 features) per CTA of a pair, token tiles chosen so that the units
+// fill whole rounds of the CTA pairs.  A3_OPT_QKV_T: 0 never, 1 whenever the shape allows (default).
+bool qkv_t_usable(const a3_handle* h, const GemmArgs& a) {
+  if (h->opt[A3_OPT_QKV_T] == 0 || h->m.head_dim != 128 || a.M <= 0 || a.K % (SP_SUB * TC_BK) != 0 || a.nseg < 1 || a.nseg > 3) return false;
+  for (int s = 0; s < a.nseg; ++s)
+    if (a.seg[s].n % 128 != 0 || a.seg[s].n <= 0) return false;
+  return true;
+}
+
+int gemm_qkv_t(const a3_handle* h, const GemmArgs& a, cudaStream_t st) {
+  SpParams p{};
+  p.M = a.M;
+  p.K = a.K;
+  int heads = 0;
+  for (int s = 0; s < 3; ++s) {
+    if (s < a.nseg) {
+      heads += a.seg[s].n / 128;
+      p.kind[s] = a.seg[s].kind;
+      p.bias[s] = a.seg[s].bias;
+    }
+    p.seg_heads_end[s] = heads;
+  }
+  p.n_heads = heads;
+  const int head_pairs = cdiv(heads, 2);
+  const int sms = h->sm_count > 0 ? h->sm_count : 148;
+  const int pairs = sms / 2;
+  // token tiles: the count whose rounds of the CTA pairs cost the fewest token columns (a unit's time follows its
+  // width; 24 columns stand for what a unit costs whatever its width)
+  int best_tt = cdiv(a.M, 256), best_n = 0;
+  long long best_cost = -1;
+  for (int tt = cdiv(a.M, 256); tt <= cdiv(a.M, 64) && tt <= cdiv(a.M, 256) + 64; ++tt) {
+    const int n = cdiv(cdiv(a.M, tt), 16) * 16;
+    if (n > 256) continue;
+    const long long cost = (long long)cdiv((long long)head_pairs * tt, pairs) * (n + 24);
+    if (best_cost < 0 || cost < best_cost) {
+      best_cost = cost;
+      best_tt = tt;
+      best_n = n;
+    }
+  }
+  if (best_n == 0) return A3_EUNSUPPORTED;
+  p.tok_tiles = best_tt;
+  p.tok_n = best_n;
+  p.n_units = head_pairs * p.tok_tiles;
+  p.n_pairs = p.n_units < pairs ? p.n_units : pairs;
+  p.status = h->dev_status;
+  p.q_out = a.q_out;
+  p.k_cache = a.k_cache;
+  p.v_cache = a.v_cache;
+  p.pos = a.pos;
+  p.kv_len = a.kv_len;
+  p.Hq = h->m.n_q_heads;
+  p.Hkv = h->m.n_kv_heads;
+  p.layout = h->m.rope_layout;
+  p.max_pos = h->m.max_positions;
+  p.tab = h->rope_tab;
+  p.sub_bytes = SP_A_BYTES + (int)align_up((size_t)(p.tok_n / 2) * TC_BK * 2, 1024);
+  p.stage_bytes = SP_SUB * p.sub_bytes;
+  p.stages = (SP_SMEM_LIMIT - SP_QKV_EXTRA - 256 - 1024) / p.stage_bytes;
+  if (p.stages > SP_MAX_STAGES) p.stages = SP_MAX_STAGES;
+  const int smem_bytes = p.stages * p.stage_bytes + SP_QKV_EXTRA + 256 + 1024;
+  CUtensorMap tX, tW[3];
+  A3_TRY(make_tmap(&tX, a.A, a.M, a.K, p.tok_n / 2));
+  for (int s = 0; s < 3; ++s) {
+    if (s < a.nseg) A3_TRY(make_tmap(&tW[s], a.seg[s].B, a.seg[s].n, a.K, 128));
+    else tW[s] = tW[0];
+  }
+  static SmemAttrOnce attr;
+  A3_TRY(smem_attr_once(attr, h->device, pair_t_kernel<EPI_QKV>, SP_SMEM_LIMIT));
+  ProfScope prof(h, A3_K_GEMM_QKV, st);
+  A3_CUDA(launch_pdl(pair_t_kernel<EPI_QKV>, dim3(2 * p.n_pairs), dim3(SP_THREADS), (size_t)smem_bytes, st, tX, tW[0], tW[1], tW[2], p));
   A3_LAUNCHED();
   return A3_OK;
 }

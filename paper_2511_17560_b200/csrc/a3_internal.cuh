@@ -160,6 +160,9 @@ int gemm_swiglu_pair(const a3_handle* h, const GemmArgs& a, cudaStream_t st);
 // C += A B^T with the same kernel structure (weights on the M side, persistent CTA pairs).
 bool residual_t_usable(const a3_handle* h, const GemmArgs& a);
 int gemm_residual_t(const a3_handle* h, const GemmArgs& a, cudaStream_t st);
+// QKV projection (bias, RoPE, scatter in the epilogue) with one head per CTA of a pair
+bool qkv_t_usable(const a3_handle* h, const GemmArgs& a);
+int gemm_qkv_t(const a3_handle* h, const GemmArgs& a, cudaStream_t st);
 
 // C-tile GEMM with fused epilogue on the tensor cores; all operands K-major bf16, fp32 accumulate.
 int gemm_bf16(const a3_handle* h, GemmEpilogue epi, const GemmArgs& a, cudaStream_t st);

@@ -872,6 +872,7 @@ def test_persistent_gemms_row_count_sweep(a3mod, shape):
             for sw, rs in ((1, 2), (0, 0)):
                 eng.set_option(a3mod.OPT_SWIGLU_PAIR, sw)
                 eng.set_option(a3mod.OPT_RESIDUAL_T, rs)
+                eng.set_option(a3mod.OPT_QKV_T, sw)
                 X, Kc, Vc = X0.clone(), K.clone(), K.clone()
                 eng.recompute_layer(layer, X, pos, Kc, Vc)
                 assert eng.device_status() == 0, M
@@ -881,6 +882,57 @@ def test_persistent_gemms_row_count_sweep(a3mod, shape):
     finally:
         eng.set_option(a3mod.OPT_SWIGLU_PAIR, 1)
         eng.set_option(a3mod.OPT_RESIDUAL_T, 1)
+        eng.set_option(a3mod.OPT_QKV_T, 1)
+    eng.close()
+
+
+@pytest.mark.parametrize("shape,layout,M", [(W.TINY_GQA, 0, 1), (W.TINY_GQA, 0, 300), (W.TINY_GQA, 1, 131), (W.TINY_G7, 0, 131),
+                                            (W.TINY_G7, 1, 513), (W.TINY_GQA, 0, 1300)])
+def test_qkv_persistent_pair_kernel_matches_tile_kernel(a3mod, shape, layout, M):
+    """The QKV projection in use for head dimension 128 (one head per CTA of a pair, the weights as the M-side operand,
+    bias + RoPE + scatter in an epilogue whose rotation halves meet through shared memory) against the tile kernels it
+    replaced - K/V cache rows, the q buffer through the attention that reads it, and the block output, bit for bit - on
+    head lists of even and odd length (the odd one ends in a pair with an idle CTA), both rotation layouts, with and
+    without bias, one row up to several units per pair; and K/V rows against the oracle."""
+    from dataclasses import replace
+    m = replace(shape, rope_layout=layout)
+    eng, layers, dev = make_engine(a3mod, m, seed=43, w_std=0.05)
+    model, weights = oracle_model(m), oracle_weights(layers)
+    rng = np.random.default_rng(97)
+    kv_len = 2 * M + 50
+    pos = np.sort(rng.choice(kv_len, size=M, replace=False))
+    pos[-1] = kv_len - 1
+    X = W.bf16_round(rng.standard_normal((M, m.d_model), dtype=np.float32))
+    Kc, Vc = W.make_cache_like(m, kv_len, 43, 9, std=1.0)
+    layer = m.n_layers - 1
+    dpos = torch.from_numpy(pos.astype(np.int32)).to(dev)
+    outs = {}
+    try:
+        for mode in (1, 0):
+            eng.set_option(a3mod.OPT_QKV_T, mode)
+            dX, dK, dV = to_dev(X, dev), to_dev(Kc[layer], dev), to_dev(Vc[layer], dev)
+            eng.recompute_layer(layer, dX, dpos, dK, dV)
+            assert eng.device_status() == 0
+            outs[mode] = (dX, dK, dV)
+    finally:
+        eng.set_option(a3mod.OPT_QKV_T, 1)
+    for a, b in zip(outs[1], outs[0]):
+        assert torch.equal(a, b)
+    Ko, Vo = Kc[layer].astype(np.float64), Vc[layer].astype(np.float64)
+    Xo, parts = O.recompute_layer(X.astype(np.float64), pos, weights[layer], model, Ko, Vo, rnd=O.round_bf16, return_parts=True)
+    gK, gV = f64(outs[1][1]), f64(outs[1][2])
+    check_kv(gK[pos], parts["k_exact"], "recomputed K rows")
+    check_kv(gV[pos], parts["v_exact"], "recomputed V rows")
+    mask = np.ones(kv_len, bool)
+    mask[pos] = False
+    np.testing.assert_array_equal(gK[mask], Kc[layer][mask])
+    np.testing.assert_array_equal(gV[mask], Vc[layer][mask])
+    check_kv(f64(outs[1][0]), parts["x_exact"], "hidden rows", scale=hidden_rows_scale(parts["x_exact"]))
+    # an out-of-range position is flagged and its row skipped, as in the tile kernels
+    bad = dpos.clone()
+    bad[0] = -1
+    eng.recompute_layer(layer, to_dev(X, dev), bad, to_dev(Kc[layer], dev), to_dev(Vc[layer], dev))
+    assert eng.device_status() & a3mod.DEV_BAD_POSITION
     eng.close()
 
 
