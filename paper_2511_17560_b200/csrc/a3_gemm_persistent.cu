@@ -40,6 +40,7 @@ constexpr int SP_SMEM_LIMIT = 227 * 1024;
 struct SpParams {
   int M, K, F;
   int tok_tiles, tok_n;  // token tiles and tokens per tile (multiple of 16, at most 256)
+  int n_fblocks;         // feature blocks (one per CTA pair and unit): units = n_fblocks x tok_tiles
   int n_units, n_pairs;
   int stages, stage_bytes, sub_bytes;  // ring depth; bytes per stage = SP_SUB x sub_bytes (A + this CTA's half of the token tile for one k-block, 1024-byte multiple)
   bf16* C;
@@ -78,6 +79,20 @@ __device__ __forceinline__ void sp_ld_chunk(uint32_t taddr, int w, float* v) {
     if (w >= 24) tc_ld8(taddr + 16, v + 16);
   }
   tc_wait_ld();
+}
+
+// Unit u -> (feature block, token tile).  Units are numbered in groups of SP_GROUP feature blocks, token tiles
+// next, the group's blocks innermost: the 74 pairs that work side by side then cover about 8 feature blocks x 9 token
+// tiles, and since they walk the k-blocks at the same pace, what a round pulls from DRAM is 8 weight blocks + 9
+// token tiles instead of 1 + 74 (feature blocks outermost, token tiles innermost: at 32 800 rows the QKV launch read
+// 6.9 GB for 0.3 GB of operands, measured).
+constexpr int SP_GROUP = 8;
+__device__ __forceinline__ void sp_unit(int u, int n_fblocks, int tok_tiles, int& fb, int& tt) {
+  const int per_group = SP_GROUP * tok_tiles;
+  const int g = u / per_group, r = u - g * per_group;
+  const int gsz = min(SP_GROUP, n_fblocks - g * SP_GROUP);
+  tt = r / gsz;
+  fb = g * SP_GROUP + (r - tt * gsz);
 }
 
 // D += A B over the CTA pair (accumulating form: no predicate to set up)
@@ -164,18 +179,20 @@ pair_t_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ C
       bool ok = true;
       if (EPI == EPI_QKV) tmap_prefetch(&tmW);
       for (int u = pair; u < p.n_units && ok; u += p.n_pairs) {
-        int f0 = (u / p.tok_tiles) * (2 * ROWS) + (int)rank * ROWS;
+        int fb, tt;
+        sp_unit(u, p.n_fblocks, p.tok_tiles, fb, tt);
+        int f0 = fb * (2 * ROWS) + (int)rank * ROWS;
         const CUtensorMap* mapA = &tmG;
         if (EPI == EPI_QKV) {
           // this CTA's head of the concatenated list -> its matrix and first row there (a pair beyond the last head of
           // an odd list loads head 0 again; its epilogue stores nothing)
-          int hd = 2 * (u / p.tok_tiles) + (int)rank;
+          int hd = 2 * fb + (int)rank;
           if (hd >= p.n_heads) hd = 0;
           const int sg = (hd >= p.seg_heads_end[0]) + (hd >= p.seg_heads_end[1]);
           f0 = (hd - (sg == 0 ? 0 : p.seg_heads_end[sg - 1])) * 128;
           mapA = sg == 0 ? &tmG : (sg == 1 ? &tmU : &tmW);
         }
-        const int t0 = (u % p.tok_tiles) * p.tok_n + (int)rank * half_n;
+        const int t0 = tt * p.tok_n + (int)rank * half_n;
         for (int kb = 0; kb < KT; kb += SP_SUB, ++kbg) {
           if (!mbar_wait(empty_bar(s), ph ^ 1, abort_flag, p.status)) {
             ok = false;
@@ -299,8 +316,10 @@ pair_t_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ C
       if (!ep_ok[0]) break;  // uniform for the 256 threads
       tc_fence_after();
       const uint32_t trow = tmem_base + (uint32_t)b * 256u + (uint32_t)(set * set_n) + ((uint32_t)(quarter * 32) << 16);
-      const int f = (u / p.tok_tiles) * (2 * SP_FEAT) + (int)rank * SP_FEAT + feat;
-      const int t0 = (u % p.tok_tiles) * p.tok_n + set * set_n;
+      int fb, tt;
+      sp_unit(u, p.n_fblocks, p.tok_tiles, fb, tt);
+      const int f = fb * (2 * SP_FEAT) + (int)rank * SP_FEAT + feat;
+      const int t0 = tt * p.tok_n + set * set_n;
       bf16* out = p.C + f;
 #pragma unroll 1
       for (int c = 0; c < n_chunks; ++c, ++cc) {
@@ -369,13 +388,15 @@ pair_t_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ C
     int it = 0;
     for (int u = pair; u < p.n_units; u += p.n_pairs, ++it) {
       const int b = it & 1;
-      const int hd = 2 * (u / p.tok_tiles) + (int)rank;
+      int fb, tt;
+      sp_unit(u, p.n_fblocks, p.tok_tiles, fb, tt);
+      const int hd = 2 * fb + (int)rank;
       const bool live = hd < p.n_heads;
       const int hde = live ? hd : 0;
       const int sg = (hde >= p.seg_heads_end[0]) + (hde >= p.seg_heads_end[1]);
       const int head_in_seg = hde - (sg == 0 ? 0 : p.seg_heads_end[sg - 1]);
       const int kind = p.kind[sg];
-      const int t0 = (u % p.tok_tiles) * p.tok_n + set * set_n;
+      const int t0 = tt * p.tok_n + set * set_n;
       const float bias = p.bias[sg] ? __bfloat162float(p.bias[sg][head_in_seg * 128 + quarter * 32 + lane]) : 0.f;
       const bool rotate = kind != 2;
       if (ep_tid == 0) ep_ok[0] = mbar_wait(tmem_full(b), (it >> 1) & 1, abort_flag, p.status) ? 1 : 0;
@@ -469,8 +490,10 @@ pair_t_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ C
     int it = 0;
     for (int u = pair; u < p.n_units; u += p.n_pairs, ++it) {
       const int b = it & 1;
-      const int f = (u / p.tok_tiles) * (2 * ROWS) + (int)rank * ROWS + quarter * 32 + lane;
-      const int t0 = (u % p.tok_tiles) * p.tok_n + set * set_n;
+      int fb, tt;
+      sp_unit(u, p.n_fblocks, p.tok_tiles, fb, tt);
+      const int f = fb * (2 * ROWS) + (int)rank * ROWS + quarter * 32 + lane;
+      const int t0 = tt * p.tok_n + set * set_n;
       const bool f_ok = f < p.F;  // the last feature block may reach past the matrix (zero-filled loads)
       bf16* crow = p.C + (size_t)t0 * p.ldc + (f_ok ? f : 0);
       // the old values of the first chunk are on their way while the main loop still runs
@@ -542,7 +565,8 @@ static int launch_pair_t(const a3_handle* h, const GemmArgs& a, cudaStream_t st)
   p.F = a.seg[0].n;
   p.tok_tiles = cdiv(a.M, 256);
   p.tok_n = cdiv(cdiv(a.M, p.tok_tiles), 16) * 16;  // even split, multiple of 16: 804 rows -> 4 x 208
-  p.n_units = cdiv(p.F, 2 * ROWS) * p.tok_tiles;
+  p.n_fblocks = cdiv(p.F, 2 * ROWS);
+  p.n_units = p.n_fblocks * p.tok_tiles;
   const int sms = h->sm_count > 0 ? h->sm_count : 148;
   p.n_pairs = p.n_units < sms / 2 ? p.n_units : sms / 2;
   p.C = a.C;
@@ -610,6 +634,7 @@ int gemm_qkv_t(const a3_handle* h, const GemmArgs& a, cudaStream_t st) {
   if (best_n == 0) return A3_EUNSUPPORTED;
   p.tok_tiles = best_tt;
   p.tok_n = best_n;
+  p.n_fblocks = head_pairs;
   p.n_units = head_pairs * p.tok_tiles;
   p.n_pairs = p.n_units < pairs ? p.n_units : pairs;
   p.status = h->dev_status;
