@@ -165,6 +165,7 @@ typedef enum {
   A3_OPT_GEMM_STAGES_QKV,
   A3_OPT_SCORES_KERNEL,         /* relevance scores: 0 choose (default), 1 the tcgen05 kernel, 2 the warp-level MMA kernel */
   A3_OPT_QKV_T,                 /* persistent CTA-pair QKV projection (one head per CTA): 0 never, 1 whenever the shape allows (default) */
+  A3_OPT_GEMM_TILING,           /* persistent CTA-pair GEMMs, token tiles: 0 widths that balance the pairs' loads (default), 1 even split */
   A3_OPT_COUNT
 } a3_option;
 

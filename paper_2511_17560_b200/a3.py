@@ -66,7 +66,7 @@ class HostIO(C.Structure):
 # a3_option (include/a3.h)
 (OPT_ATTN_SPLIT, OPT_ATTN_PAIR, OPT_ATTN_MAX_CTAS, OPT_SWIGLU_NARROW, OPT_SWIGLU_PAIR, OPT_RESIDUAL_T, OPT_GEMM_BN_RESIDUAL,
  OPT_GEMM_BN_SWIGLU, OPT_GEMM_BN_QKV, OPT_GEMM_STAGES_RESIDUAL, OPT_GEMM_STAGES_SWIGLU, OPT_GEMM_STAGES_QKV,
- OPT_SCORES_KERNEL, OPT_QKV_T, OPT_COUNT) = range(15)
+ OPT_SCORES_KERNEL, OPT_QKV_T, OPT_GEMM_TILING, OPT_COUNT) = range(16)
 
 EXPORTS = ("a3_create", "a3_destroy", "a3_set_option", "a3_scores_workspace_bytes", "a3_swiglu_rows", "a3_layer_workspace_bytes", "a3_request_workspace_bytes", "a3_host_staging_bytes",
            "a3_recompute_count", "a3_rope_rerotate", "a3_query_scores", "a3_query_scores_static", "a3_topk_select", "a3_recompute_layer",

@@ -555,6 +555,39 @@ bool residual_t_usable(const a3_handle* h, const GemmArgs& a) {
   return cdiv(a.seg[0].n, 4 * SP_FEAT) * cdiv(a.M, 256) > sms / 2;
 }
 
+// Token tiling of a launch: `tiles` tiles of `n` tokens (a multiple of 16, at most 256) that divide the row count
+// evenly.  The tile count is the one with the cheapest rounds: the CTA pairs take the units (feature block x token
+// tile) round by round, and a unit of n token columns costs, per k-block, the larger of its tensor time (2 n clocks:
+// four instructions of n / 2) and the time its operands take to arrive (16 KiB of weights + 64 n bytes of tokens per
+// CTA at about 64 bytes per clock: 256 + n clocks), plus a fixed part.  By that measure every unit narrower than 256
+// waits for its operands, and the measurements agree: 804 rows x 112 feature blocks as five tiles of 176 (or as
+// 4 x 176 + 112 with the narrow units last, which a count of token columns alone prefers) took 160-165 us against 147
+// for 4 x 208.  Examples: 4 952 rows x 16 feature blocks -> 23 x 224 (five rounds of 224 instead of five of 256:
+// 536 vs 591 us for both residual GEMMs of a layer), x 112 -> 20 x 256 as before; 804 rows x 24 head pairs -> 6 x 144
+// (two rounds) instead of 4 x 208 (two rounds).  A3_OPT_GEMM_TILING = 1 keeps ceil(M / 256) tiles (comparisons).
+struct SpTiling {
+  int tiles, n;
+};
+static SpTiling choose_tiling(const a3_handle* h, int M, int n_fblocks, int pairs) {
+  SpTiling best{cdiv(M, 256), 0};
+  best.n = cdiv(cdiv(M, best.tiles), 16) * 16;  // 804 rows -> 4 x 208
+  if (h->opt[A3_OPT_GEMM_TILING] == 1) return best;
+  auto load = [&](int tiles, int n) {
+    const long long unit = (long long)(2 * n > 256 + n ? 2 * n : 256 + n) + 32;
+    return (long long)cdiv((long long)n_fblocks * tiles, pairs) * unit;
+  };
+  long long best_load = load(best.tiles, best.n);
+  for (int tiles = best.tiles + 1; tiles <= best.tiles + 64 && tiles <= cdiv(M, 96); ++tiles) {
+    const int n = cdiv(cdiv(M, tiles), 16) * 16;
+    const long long l = load(tiles, n);
+    if (l < best_load) {
+      best_load = l;
+      best = SpTiling{tiles, n};
+    }
+  }
+  return best;
+}
+
 template <int EPI>
 static int launch_pair_t(const a3_handle* h, const GemmArgs& a, cudaStream_t st) {
   constexpr int ROWS = EPI == EPI_SWIGLU ? SP_FEAT : 2 * SP_FEAT;  // output features per CTA
@@ -563,11 +596,12 @@ static int launch_pair_t(const a3_handle* h, const GemmArgs& a, cudaStream_t st)
   p.M = a.M;
   p.K = a.K;
   p.F = a.seg[0].n;
-  p.tok_tiles = cdiv(a.M, 256);
-  p.tok_n = cdiv(cdiv(a.M, p.tok_tiles), 16) * 16;  // even split, multiple of 16: 804 rows -> 4 x 208
-  p.n_fblocks = cdiv(p.F, 2 * ROWS);
-  p.n_units = p.n_fblocks * p.tok_tiles;
   const int sms = h->sm_count > 0 ? h->sm_count : 148;
+  p.n_fblocks = cdiv(p.F, 2 * ROWS);
+  const SpTiling til = choose_tiling(h, a.M, p.n_fblocks, sms / 2);
+  p.tok_tiles = til.tiles;
+  p.tok_n = til.n;
+  p.n_units = p.n_fblocks * p.tok_tiles;
   p.n_pairs = p.n_units < sms / 2 ? p.n_units : sms / 2;
   p.C = a.C;
   p.ldc = a.ldc;
@@ -617,23 +651,9 @@ int gemm_qkv_t(const a3_handle* h, const GemmArgs& a, cudaStream_t st) {
   const int head_pairs = cdiv(heads, 2);
   const int sms = h->sm_count > 0 ? h->sm_count : 148;
   const int pairs = sms / 2;
-  // token tiles: the count whose rounds of the CTA pairs cost the fewest token columns (a unit's time follows its
-  // width; 24 columns stand for what a unit costs whatever its width)
-  int best_tt = cdiv(a.M, 256), best_n = 0;
-  long long best_cost = -1;
-  for (int tt = cdiv(a.M, 256); tt <= cdiv(a.M, 64) && tt <= cdiv(a.M, 256) + 64; ++tt) {
-    const int n = cdiv(cdiv(a.M, tt), 16) * 16;
-    if (n > 256) continue;
-    const long long cost = (long long)cdiv((long long)head_pairs * tt, pairs) * (n + 24);
-    if (best_cost < 0 || cost < best_cost) {
-      best_cost = cost;
-      best_tt = tt;
-      best_n = n;
-    }
-  }
-  if (best_n == 0) return A3_EUNSUPPORTED;
-  p.tok_tiles = best_tt;
-  p.tok_n = best_n;
+  const SpTiling til = choose_tiling(h, a.M, head_pairs, pairs);
+  p.tok_tiles = til.tiles;
+  p.tok_n = til.n;
   p.n_fblocks = head_pairs;
   p.n_units = head_pairs * p.tok_tiles;
   p.n_pairs = p.n_units < pairs ? p.n_units : pairs;

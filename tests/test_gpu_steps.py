@@ -869,20 +869,25 @@ def test_persistent_gemms_row_count_sweep(a3mod, shape):
             X0 = torch.randn((M, m.d_model), device=dev, generator=g).to(torch.bfloat16)
             K = torch.randn((kv_len, m.n_kv_heads, m.head_dim), device=dev, generator=g).to(torch.bfloat16)
             outs = []
-            for sw, rs in ((1, 2), (0, 0)):
+            # persistent kernels with load-balancing token tiles (wide tiles + one narrow), with an even split, and the tile kernels
+            for sw, rs, tiling in ((1, 2, 0), (1, 2, 1), (0, 0, 0)):
                 eng.set_option(a3mod.OPT_SWIGLU_PAIR, sw)
                 eng.set_option(a3mod.OPT_RESIDUAL_T, rs)
                 eng.set_option(a3mod.OPT_QKV_T, sw)
+                eng.set_option(a3mod.OPT_GEMM_TILING, tiling)
                 X, Kc, Vc = X0.clone(), K.clone(), K.clone()
                 eng.recompute_layer(layer, X, pos, Kc, Vc)
                 assert eng.device_status() == 0, M
-                outs.append(X)
-            assert torch.isfinite(outs[0].float()).all(), M
-            assert torch.equal(outs[0], outs[1]), M
+                outs.append((X, Kc, Vc))
+            assert torch.isfinite(outs[0][0].float()).all(), M
+            for other in outs[1:]:
+                for a, b in zip(outs[0], other):
+                    assert torch.equal(a, b), M
     finally:
         eng.set_option(a3mod.OPT_SWIGLU_PAIR, 1)
         eng.set_option(a3mod.OPT_RESIDUAL_T, 1)
         eng.set_option(a3mod.OPT_QKV_T, 1)
+        eng.set_option(a3mod.OPT_GEMM_TILING, 0)
     eng.close()
 
 
