@@ -33,7 +33,7 @@ if ROOT not in sys.path:
 # DRAM bytes (read + write) per launch of the dominant kernel classes from the ncu captures summarised under profiles/
 # (gemm_kernels_llama8b_2layer.txt: SwiGLU GEMM of a sparse layer, M = 804, and of the full block, M = 5152;
 # attention_kernels_*: see that file).  Used for `roofline.traffic` of the workloads they were captured on.
-NCU_TRAFFIC = {("llama8b_10x512", "gemm_swiglu"): {"sparse": 243.44e6 + 18.51e6, "full": 418.15e6 + 140.63e6},
+NCU_TRAFFIC = {("llama8b_10x512", "gemm_swiglu"): {"sparse": 243.87e6 + 18.46e6, "full": 389.03e6 + 140.80e6},
                # attention_and_selection_kernels_llama8b_64x512_2layer.txt: sparse rows (4 952) and the full causal block (32 800)
                ("llama8b_64x512", "attention"): {"sparse": 419.97e6 + 35.71e6, "full": 2208.55e6 + 265.24e6}}
 

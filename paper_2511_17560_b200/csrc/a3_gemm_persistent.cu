@@ -41,6 +41,7 @@ struct SpParams {
   int M, K, F;
   int tok_tiles, tok_n;  // token tiles and tokens per tile (multiple of 16, at most 256)
   int n_fblocks;         // feature blocks (one per CTA pair and unit): units = n_fblocks x tok_tiles
+  int group;             // feature blocks per group of the unit order (1: feature blocks outermost)
   int n_units, n_pairs;
   int stages, stage_bytes, sub_bytes;  // ring depth; bytes per stage = SP_SUB x sub_bytes (A + this CTA's half of the token tile for one k-block, 1024-byte multiple)
   bf16* C;
@@ -81,18 +82,20 @@ __device__ __forceinline__ void sp_ld_chunk(uint32_t taddr, int w, float* v) {
   tc_wait_ld();
 }
 
-// Unit u -> (feature block, token tile).  Units are numbered in groups of SP_GROUP feature blocks, token tiles
-// next, the group's blocks innermost: the 74 pairs that work side by side then cover about 8 feature blocks x 9 token
-// tiles, and since they walk the k-blocks at the same pace, what a round pulls from DRAM is 8 weight blocks + 9
-// token tiles instead of 1 + 74 (feature blocks outermost, token tiles innermost: at 32 800 rows the QKV launch read
-// 6.9 GB for 0.3 GB of operands, measured).
-constexpr int SP_GROUP = 8;
-__device__ __forceinline__ void sp_unit(int u, int n_fblocks, int tok_tiles, int& fb, int& tt) {
-  const int per_group = SP_GROUP * tok_tiles;
+// Unit u -> (feature block, token tile).  Units are numbered in groups of `group` feature blocks, token tiles next,
+// the group's blocks innermost.  With group = 8 the 74 pairs that work side by side cover about 8 feature blocks x 9
+// token tiles, and since they walk the k-blocks at the same pace, what a round pulls through L2 is 8 weight blocks +
+// 9 token tiles: the order for token matrices that do not fit in L2 (with feature blocks outermost a round of the
+// 32 800-row QKV launch pulled 1 weight block + 74 token tiles: 6.9 GB of DRAM reads for 0.3 GB of operands).  With
+// group = 1 (feature blocks outermost) every round walks all token tiles: the order for token matrices that stay in
+// L2, where the weights then stream through exactly once (SwiGLU at 5 152 rows: 418 MB of DRAM reads against 719 MB
+// with groups of 8).
+__device__ __forceinline__ void sp_unit(int u, int n_fblocks, int tok_tiles, int group, int& fb, int& tt) {
+  const int per_group = group * tok_tiles;
   const int g = u / per_group, r = u - g * per_group;
-  const int gsz = min(SP_GROUP, n_fblocks - g * SP_GROUP);
+  const int gsz = min(group, n_fblocks - g * group);
   tt = r / gsz;
-  fb = g * SP_GROUP + (r - tt * gsz);
+  fb = g * group + (r - tt * gsz);
 }
 
 // D += A B over the CTA pair (accumulating form: no predicate to set up)
@@ -180,7 +183,7 @@ pair_t_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ C
       if (EPI == EPI_QKV) tmap_prefetch(&tmW);
       for (int u = pair; u < p.n_units && ok; u += p.n_pairs) {
         int fb, tt;
-        sp_unit(u, p.n_fblocks, p.tok_tiles, fb, tt);
+        sp_unit(u, p.n_fblocks, p.tok_tiles, p.group, fb, tt);
         int f0 = fb * (2 * ROWS) + (int)rank * ROWS;
         const CUtensorMap* mapA = &tmG;
         if (EPI == EPI_QKV) {
@@ -317,7 +320,7 @@ pair_t_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ C
       tc_fence_after();
       const uint32_t trow = tmem_base + (uint32_t)b * 256u + (uint32_t)(set * set_n) + ((uint32_t)(quarter * 32) << 16);
       int fb, tt;
-      sp_unit(u, p.n_fblocks, p.tok_tiles, fb, tt);
+      sp_unit(u, p.n_fblocks, p.tok_tiles, p.group, fb, tt);
       const int f = fb * (2 * SP_FEAT) + (int)rank * SP_FEAT + feat;
       const int t0 = tt * p.tok_n + set * set_n;
       bf16* out = p.C + f;
@@ -389,7 +392,7 @@ pair_t_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ C
     for (int u = pair; u < p.n_units; u += p.n_pairs, ++it) {
       const int b = it & 1;
       int fb, tt;
-      sp_unit(u, p.n_fblocks, p.tok_tiles, fb, tt);
+      sp_unit(u, p.n_fblocks, p.tok_tiles, p.group, fb, tt);
       const int hd = 2 * fb + (int)rank;
       const bool live = hd < p.n_heads;
       const int hde = live ? hd : 0;
@@ -491,7 +494,7 @@ pair_t_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ C
     for (int u = pair; u < p.n_units; u += p.n_pairs, ++it) {
       const int b = it & 1;
       int fb, tt;
-      sp_unit(u, p.n_fblocks, p.tok_tiles, fb, tt);
+      sp_unit(u, p.n_fblocks, p.tok_tiles, p.group, fb, tt);
       const int f = fb * (2 * ROWS) + (int)rank * ROWS + quarter * 32 + lane;
       const int t0 = tt * p.tok_n + set * set_n;
       const bool f_ok = f < p.F;  // the last feature block may reach past the matrix (zero-filled loads)
@@ -565,6 +568,10 @@ bool residual_t_usable(const a3_handle* h, const GemmArgs& a) {
 // for 4 x 208.  Examples: 4 952 rows x 16 feature blocks -> 23 x 224 (five rounds of 224 instead of five of 256:
 // 536 vs 591 us for both residual GEMMs of a layer), x 112 -> 20 x 256 as before; 804 rows x 24 head pairs -> 6 x 144
 // (two rounds) instead of 4 x 208 (two rounds).  A3_OPT_GEMM_TILING = 1 keeps ceil(M / 256) tiles (comparisons).
+// Feature blocks per group of the unit order: 8 when the token matrix (M x K bf16) is too large to stay in L2 beside
+// the weights and the output that stream through it, else 1.
+static int unit_group(int M, int K) { return (long long)M * K * 2 > (64ll << 20) ? 8 : 1; }
+
 struct SpTiling {
   int tiles, n;
 };
@@ -602,6 +609,7 @@ static int launch_pair_t(const a3_handle* h, const GemmArgs& a, cudaStream_t st)
   p.tok_tiles = til.tiles;
   p.tok_n = til.n;
   p.n_units = p.n_fblocks * p.tok_tiles;
+  p.group = unit_group(a.M, a.K);
   p.n_pairs = p.n_units < sms / 2 ? p.n_units : sms / 2;
   p.C = a.C;
   p.ldc = a.ldc;
@@ -655,6 +663,7 @@ int gemm_qkv_t(const a3_handle* h, const GemmArgs& a, cudaStream_t st) {
   p.tok_tiles = til.tiles;
   p.tok_n = til.n;
   p.n_fblocks = head_pairs;
+  p.group = unit_group(a.M, a.K);
   p.n_units = head_pairs * p.tok_tiles;
   p.n_pairs = p.n_units < pairs ? p.n_units : pairs;
   p.status = h->dev_status;
