@@ -347,3 +347,39 @@ def test_first_token_llama_vocabulary():
     # the chosen logit is the largest of the sample in the oracle's arithmetic too (up to the tolerance)
     assert want[np.searchsorted(rows, tok)] >= want.max() - 2 * FT_TOL * scale
     eng.close()
+
+
+@pytest.mark.parametrize("shape,rows", [(W.LLAMA8B, (804, 4952, 7629, 16640)), (W.QWEN7B, (960, 2754, 9404, 16640))])
+def test_persistent_gemms_bit_identical_at_full_width(shape, rows):
+    """One layer at the real widths, row counts of the configs and in between (16 640 rows: the token matrix no longer
+    stays in L2 and the units of the persistent kernels are walked in groups of feature blocks): the persistent CTA-pair
+    GEMMs - gate/up, QKV with its RoPE/scatter epilogue, both residual GEMMs forced onto them, each with the token
+    tiling chosen for its shape - against the tile kernels, bit for bit: hidden rows and the K/V cache."""
+    from paper_2511_17560_b200 import a3
+    m = replace(shape, n_layers=1)
+    eng = a3.A3(m, W.make_weights_device(m, DEV, 0), max(rows) + 128)
+    try:
+        for M in rows:
+            kv_len = M + 64
+            g = torch.Generator(device=DEV)
+            g.manual_seed(M)
+            pos = torch.sort(torch.randperm(kv_len, device=DEV, generator=g)[:M]).values.to(torch.int32)
+            X0 = torch.randn((M, m.d_model), device=DEV, generator=g).to(torch.bfloat16)
+            K = torch.randn((kv_len, m.n_kv_heads, m.head_dim), device=DEV, generator=g).to(torch.bfloat16)
+            outs = []
+            for sw, rs in ((1, 2), (0, 0)):
+                eng.set_option(a3.OPT_SWIGLU_PAIR, sw)
+                eng.set_option(a3.OPT_RESIDUAL_T, rs)
+                eng.set_option(a3.OPT_QKV_T, sw)
+                X, Kc, Vc = X0.clone(), K.clone(), K.clone()
+                eng.recompute_layer(0, X, pos, Kc, Vc)
+                assert eng.device_status() == 0, M
+                outs.append((X, Kc, Vc))
+            assert torch.isfinite(outs[0][0].float()).all(), M
+            for a, b in zip(outs[0], outs[1]):
+                assert torch.equal(a, b), M
+    finally:
+        eng.set_option(a3.OPT_SWIGLU_PAIR, 1)
+        eng.set_option(a3.OPT_RESIDUAL_T, 1)
+        eng.set_option(a3.OPT_QKV_T, 1)
+        eng.close()
