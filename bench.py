@@ -201,13 +201,14 @@ def oracle_strides(n: int, M: int, budget_rows: int):
     return max(1, -(-n // budget_rows)), max(1, -(-M // budget_rows))
 
 
-def oracle_step(S, stride_full: int = 4, stride_rows: int = 1):
+def oracle_step(S, stride_full: int = 4, stride_rows: int = 1, stride_q: int = 1):
     """One bounded sample of the request on the oracle (fp32), with the factors that scale it to the whole request.
 
     Timed pieces, each the oracle's own function: position recovery of one layer (x L); one full block on every
     `stride_full`-th row (x stride_full x select_layer); the selection layer's norm + QKV on every `stride_full`-th row
-    (x stride_full), scores and top-p at full size; one recompute layer on every `stride_rows`-th of the p + |Q| carried
-    rows (x stride_rows x (L - select_layer)).  Returns (measured seconds, extrapolated seconds, parts).
+    (x stride_full), scores (of every `stride_q`-th question row, x stride_q) and top-p at full size; one recompute layer
+    on every `stride_rows`-th of the p + |Q| carried rows (x stride_rows x (L - select_layer)).  Returns (measured
+    seconds, extrapolated seconds, parts).
     """
     O, m, mf, r, model, weights = S["O"], S["m"], S["m_full"], S["r"], S["model"], S["weights"]
     dt = np.float32
@@ -234,14 +235,15 @@ def oracle_step(S, stride_full: int = 4, stride_rows: int = 1):
     t_kv = time.perf_counter() - c0
     c0 = time.perf_counter()
     q_rows = np.arange(r.n_ctx, n)
-    aq = O.rmsnorm(X[q_rows], w.attn_norm, model.rms_eps)
-    q, _, _ = O.project_qkv(aq, w, model, q_rows)
-    s = O.query_scores(q, q_rows, K, model, 0, r.n_ctx)
+    q_sub = q_rows[::stride_q]
+    aq = O.rmsnorm(X[q_sub], w.attn_norm, model.rms_eps)
+    q, _, _ = O.project_qkv(aq, w, model, q_sub)
+    s = O.query_scores(q, q_sub, K, model, 0, r.n_ctx)
     p = O.recompute_count(r.ratio, n, r.n_ctx)
     Re = O.topk_select(s, 0, r.n_ctx, p)
     t_sel = time.perf_counter() - c0
     meas["selection"] = t_kv + t_sel
-    t["selection"] = t_kv * stride_full + t_sel
+    t["selection"] = t_kv * stride_full + t_sel * stride_q
     R = np.concatenate([Re, q_rows])[::stride_rows]
     c0 = time.perf_counter()
     O.recompute_layer(X[R], R, weights[min(ls + 1, m.n_layers - 1)], model, K, V)
@@ -289,18 +291,21 @@ def run_reference(args):
     S = oracle_sample(config)
     m, r = S["m_full"], S["r"]
     p = S["O"].recompute_count(r.ratio, r.n, r.n_ctx)
-    sf, sr = oracle_strides(r.n, p + r.n_question, args.oracle_rows)
+    # the sample shrinks with the number of steps asked for, so that any --steps/--warmup ends within minutes
+    shrink = min(1.0, 25.0 / max(1, args.steps + args.warmup))
+    sf, sr = oracle_strides(r.n, p + r.n_question, max(48, int(args.oracle_rows * shrink)))
+    sq = max(1, min(r.n_question, int(round(1.0 / shrink))))
     for _ in range(args.warmup):
-        oracle_step(S, sf, sr)
+        oracle_step(S, sf, sr, sq)
     meas, extr, parts = [], [], None
     for _ in range(args.steps):
-        a, b, parts = oracle_step(S, sf, sr)
+        a, b, parts = oracle_step(S, sf, sr, sq)
         meas.append(a)
         extr.append(b)
     t_meas, t_extr = float(np.mean(meas)), float(np.mean(extr))
     value = r.n_ctx / t_extr
-    sample = (f"per step: position recovery of 1 layer, one full block and the selection-layer QKV on every {sf}-th row, scores + "
-              f"top-p at full size, one recompute layer on every {sr}-th of the p+|Q| rows; scaled to all layers/rows "
+    sample = (f"per step: position recovery of 1 layer, one full block and the selection-layer QKV on every {sf}-th row, scores "
+              f"of every {sq}-th question row + top-p at full size, one recompute layer on every {sr}-th of the p+|Q| rows; scaled to all layers/rows "
               "(extrapolated); oracle in fp32 with random caches of the workload's shape")
     line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": t_meas * 1e3, "extrapolated": True, "extrapolated_request_ms": t_extr * 1e3,
