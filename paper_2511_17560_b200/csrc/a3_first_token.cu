@@ -3,8 +3,8 @@
 //
 // The projection is a matrix-vector product over a [vocab][d] bf16 matrix read exactly once (1 GiB at
 // Llama-3-8B size): bound by HBM.  Every CTA normalises the row itself (8 KiB, from L2) into shared memory as
-// fp32 holding the bf16-rounded values a bf16 pipeline would store; a warp then walks pairs of vocabulary rows
-// with eight 16-byte streaming loads in flight per lane, reduces with shuffles, writes the fp32 logits and keeps
+// fp32 holding the bf16-rounded values a bf16 pipeline would store; a warp then walks four vocabulary rows at a
+// time with sixteen 16-byte streaming loads in flight per lane, reduces with shuffles, writes the fp32 logits and keeps
 // its best (value, lowest id).  The last CTA to finish (ticket counter) reduces the per-CTA candidates, so the
 // whole step is one launch and its result does not depend on the order in which CTAs finish.
 #include "a3_internal.cuh"
@@ -55,50 +55,54 @@ first_token_kernel(const bf16* __restrict__ x, const bf16* __restrict__ gain, co
   float best_v = -INFINITY;
   int best_i = 0x7fffffff;
   bool bad = false;
-  const int n_pairs = (vocab + 1) / 2;
-  for (int pr = blockIdx.x * FT_WARPS + warp; pr < n_pairs; pr += gridDim.x * FT_WARPS) {
-    const int r0 = 2 * pr, r1 = r0 + 1;
-    const bool has1 = r1 < vocab;
-    const uint4* w0 = w + (size_t)r0 * nchunk;
-    const uint4* w1 = w + (size_t)(has1 ? r1 : r0) * nchunk;
-    float acc0 = 0.f, acc1 = 0.f;
+  constexpr int R = 4;  // vocabulary rows a warp walks together: 4 x 4 loads of 16 bytes in flight per lane
+  const int n_groups = (vocab + R - 1) / R;
+  for (int gr = blockIdx.x * FT_WARPS + warp; gr < n_groups; gr += gridDim.x * FT_WARPS) {
+    const int r0 = R * gr;
+    const uint4* wr[R];
+    float acc[R];
+#pragma unroll
+    for (int j = 0; j < R; ++j) {
+      wr[j] = w + (size_t)min(r0 + j, vocab - 1) * nchunk;  // rows beyond the last repeat it; their results are dropped
+      acc[j] = 0.f;
+    }
     for (int c0 = lane; c0 < nchunk; c0 += 128) {
-      uint4 p0[4], p1[4];
+      uint4 pk[R][4];
 #pragma unroll
       for (int u = 0; u < 4; ++u) {
         const int c = c0 + 32 * u;
-        p0[u] = p1[u] = make_uint4(0, 0, 0, 0);
-        if (c < nchunk) {
-          p0[u] = __ldcs(w0 + c);
-          p1[u] = __ldcs(w1 + c);
-        }
+#pragma unroll
+        for (int j = 0; j < R; ++j) pk[j][u] = c < nchunk ? __ldcs(wr[j] + c) : make_uint4(0, 0, 0, 0);
       }
 #pragma unroll
       for (int u = 0; u < 4; ++u) {
         const int c = c0 + 32 * u;
         if (c < nchunk) {
           const float4 a0 = sa4[2 * c], a1 = sa4[2 * c + 1];
-          float f[8];
-          unpack8(p0[u], f);
-          acc0 += f[0] * a0.x + f[1] * a0.y + f[2] * a0.z + f[3] * a0.w + f[4] * a1.x + f[5] * a1.y + f[6] * a1.z + f[7] * a1.w;
-          unpack8(p1[u], f);
-          acc1 += f[0] * a0.x + f[1] * a0.y + f[2] * a0.z + f[3] * a0.w + f[4] * a1.x + f[5] * a1.y + f[6] * a1.z + f[7] * a1.w;
+#pragma unroll
+          for (int j = 0; j < R; ++j) {
+            float f[8];
+            unpack8(pk[j][u], f);
+            acc[j] += f[0] * a0.x + f[1] * a0.y + f[2] * a0.z + f[3] * a0.w + f[4] * a1.x + f[5] * a1.y + f[6] * a1.z + f[7] * a1.w;
+          }
         }
       }
     }
 #pragma unroll
     for (int o = 16; o; o >>= 1) {
-      acc0 += __shfl_xor_sync(0xffffffffu, acc0, o);
-      acc1 += __shfl_xor_sync(0xffffffffu, acc1, o);
+#pragma unroll
+      for (int j = 0; j < R; ++j) acc[j] += __shfl_xor_sync(0xffffffffu, acc[j], o);
     }
     if (lane == 0) {
-      if (logits) {
-        logits[r0] = acc0;
-        if (has1) logits[r1] = acc1;
+#pragma unroll
+      for (int j = 0; j < R; ++j) {
+        const int rj = r0 + j;
+        if (rj < vocab) {
+          if (logits) logits[rj] = acc[j];
+          bad = bad || !isfinite(acc[j]);
+          if (ft_better(acc[j], rj, best_v, best_i)) best_v = acc[j], best_i = rj;
+        }
       }
-      bad = bad || !isfinite(acc0) || (has1 && !isfinite(acc1));
-      if (ft_better(acc0, r0, best_v, best_i)) best_v = acc0, best_i = r0;
-      if (has1 && ft_better(acc1, r1, best_v, best_i)) best_v = acc1, best_i = r1;
     }
   }
   if (lane == 0) {
@@ -167,7 +171,7 @@ extern "C" int a3_first_token(const a3_handle* h, const void* x_row, const void*
   const size_t smem = (size_t)d * 4;
   if (smem > 48 * 1024) A3_CUDA(cudaFuncSetAttribute(first_token_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 96 * 1024));
   int grid = h->sm_count * 2;
-  const int need = cdiv((vocab + 1) / 2, FT_WARPS);
+  const int need = cdiv((vocab + 3) / 4, FT_WARPS);
   if (grid > need) grid = need;
   {
     ProfScope prof(h, A3_K_FIRST_TOKEN, st);
