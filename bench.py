@@ -435,7 +435,21 @@ class RequestWorkload:
             seconds = timer.run(lambda: eng.fuse_request(req), steps)
         gpu_launches = a3.launch_count(reset=True)
         clocks = sampler.stop() if sampler else None
-        other = timer.run(lambda: eng.fuse_request(req), steps) if (graph is not None and want_plain) else None
+        timed_call = ("a3_fuse_request" if graph is None else
+                      "a3_graph_launch (the request recorded once by a3_graph_capture; every kernel runs at every replay)")
+        other, other_call = None, None
+        if graph is not None and want_plain:
+            # the same K requests through the other public way of issuing them; the faster of the two is the headline
+            # (long kernels: plain launches, whose programmatic dependent launches overlap a kernel's set-up with its
+            # predecessor's tail; short kernels: the graph, which has no launch gaps), the other is reported beside it
+            sampler = ClockSampler(local) if rank == 0 else None
+            other = timer.run(lambda: eng.fuse_request(req), steps)
+            other_clocks = sampler.stop() if sampler else None
+            other_call = "a3_fuse_request"
+            if other < seconds:
+                seconds, other = other, seconds
+                clocks, other_clocks = other_clocks, clocks
+                timed_call, other_call = other_call, timed_call
         a3.launch_count(reset=True)
         assert eng.device_status() == 0, "device status word set during the timed region"
         # second pass: per-launch CUDA events (about 1 ms per request of their own, which is why `value` is not taken here)
@@ -456,10 +470,9 @@ class RequestWorkload:
         tfs = total / (seconds / steps) / 1e12
         res = {"ms_per_step": ms, "tokens_per_s_per_replica": r.n_ctx / (seconds / steps), "seconds": seconds, "gpu_launches": int(gpu_launches),
                "launches_per_step": int(launches_per_step), "clocks": clocks, "profiled_pass": {"request_ms": prof_seconds / steps * 1e3, "clocks": prof_clocks},
-               "plain_seconds": other, "kernels": kernels, "algorithmic_tflop_per_request": total / 1e12, "request_tflops": tfs,
+               "other_seconds": other, "other_call": other_call, "kernels": kernels, "algorithmic_tflop_per_request": total / 1e12, "request_tflops": tfs,
                "request_frac_of_sustained_peak": tfs / peaks["bf16_tflops_sustained"], "request_frac_of_burst_peak": tfs / peaks["bf16_tflops"],
-               "timed_call": "a3_fuse_request" if graph is None else
-                             "a3_graph_launch (the request recorded once by a3_graph_capture; every kernel runs at every replay)"}
+               "timed_call": timed_call}
         if clocks and clocks.get("sm_mhz"):
             res["request_frac_clock_normalised"] = res["request_frac_of_sustained_peak"] * peaks["sustained_mhz"] / clocks["sm_mhz"]
         if self.name == HEADLINE or (self.r.n_ctx == 32768):
@@ -768,9 +781,9 @@ def run_a3(args):
                 "ms_per_step": res["ms_per_step"], "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
                 "dtype": "bf16", "data": "synthetic", "config": cfg, "workload_notes": notes,
                 "request_ms": res["ms_per_step"], "profiled_pass": res["profiled_pass"], "timed_call": res["timed_call"],
-                "plain_launches": None if res["plain_seconds"] is None else
-                                  {"call": "a3_fuse_request", "ms_per_step": res["plain_seconds"] / steps * 1e3,
-                                   "value": aggregate_value(r.n_ctx, steps, world, res["plain_seconds"])},
+                "other_call": None if res["other_seconds"] is None else
+                              {"call": res["other_call"], "ms_per_step": res["other_seconds"] / steps * 1e3,
+                               "value": aggregate_value(r.n_ctx, steps, world, res["other_seconds"])},
                 **context,
                 "algorithmic_tflop_per_request": res["algorithmic_tflop_per_request"], "request_tflops": res["request_tflops"],
                 "request_frac_of_sustained_peak": res["request_frac_of_sustained_peak"],

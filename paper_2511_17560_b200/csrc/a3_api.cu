@@ -421,9 +421,17 @@ namespace a3 {
 // memory; position recovery of layer l is queued behind it, just before the layer needs the cache.  The copies
 // themselves are queued a few layers ahead of the compute launches that need them (queue_layer), not all up front:
 // thousands of small copies take the host tens of milliseconds to queue, which would otherwise delay the first launch.
+// The first full block walks a long input in row panels (same panels whatever the entry point, so that every entry
+// point arrives at the same bits): the host-buffer entry copies the embeddings panel by panel and the block starts
+// on the first panel while the others are still on their way.
+constexpr int X0_PANELS = 4;
+constexpr int X0_PANEL_MIN_ROWS = 16384;  // shorter inputs: one panel
+static inline int x0_panels(int n) { return n >= X0_PANEL_MIN_ROWS ? X0_PANELS : 1; }
+static inline int x0_panel_begin(int n, int i, int panels) { return i >= panels ? n : (int)((long long)n * i / panels) & ~127; }
+
 struct HostFeed {
   const cudaEvent_t* layer_ready;  // [n_layers]
-  cudaEvent_t x0_ready;
+  const cudaEvent_t* x0_ready;     // [x0_panels(n)]: the embeddings of a panel of rows are on the device
   void* ctx;
   int (*queue_layer)(void* ctx, int layer);  // queues the copies of one layer on the copy stream, records layer_ready[layer]
   int next;                                  // first layer whose copies are not queued yet
@@ -499,7 +507,7 @@ extern "C" void a3_graph_destroy(a3_graph* g) {
 static int a3::fuse_impl(const a3_handle* h, const a3_request* r, void* ws, size_t ws_bytes, a3_stream stream, HostFeed* feed) {
   if (!h || !r || !ws) return A3_EINVAL;
   const cudaEvent_t* layer_ready = feed ? feed->layer_ready : nullptr;
-  const cudaEvent_t x0_ready = feed ? feed->x0_ready : nullptr;
+  const cudaEvent_t* x0_ready = feed ? feed->x0_ready : nullptr;
   // copies of the layers up to `upto` are on their way (host-buffer entry only)
   auto feed_to = [&](int upto) -> int {
     while (feed && feed->next <= upto && feed->next < h->m.n_layers) {
@@ -589,11 +597,22 @@ static int a3::fuse_impl(const a3_handle* h, const a3_request* r, void* ws, size
     A3_TRY(a3_rope_rerotate(h, r->chunks, r->n_chunks, r->max_chunk_len, r->k_fused, r->v_fused, r->layer_stride, r->n_ctx, ls + 1,
                             m.n_layers, stream));
   // leading full blocks: the whole input through layers 0..select_layer-1
-  if (x0_ready) A3_CUDA(cudaStreamWaitEvent(st, x0_ready, 0));
-  A3_CUDA(cudaMemcpyAsync(w.x_all, r->x0, (size_t)n * m.d_model * 2, cudaMemcpyDeviceToDevice, st));
+  const int panels = x0_panels(n);
   A3_TRY(iota_rows(h, w.all_pos, 0, n, st));
-  for (int l = 0; l < ls; ++l) {
-    A3_TRY(feed_to(ls + 1 + FEED_AHEAD * (l + 1)));  // a full block is long: several layers' copies fit under it
+  for (int i = 0; i < panels; ++i) {
+    const int r0 = x0_panel_begin(n, i, panels), r1 = x0_panel_begin(n, i + 1, panels);
+    if (x0_ready) A3_CUDA(cudaStreamWaitEvent(st, x0_ready[i], 0));
+    A3_CUDA(cudaMemcpyAsync(w.x_all + (size_t)r0 * m.d_model, (const bf16*)r->x0 + (size_t)r0 * m.d_model, (size_t)(r1 - r0) * m.d_model * 2,
+                            cudaMemcpyDeviceToDevice, st));
+    if (ls > 0) {
+      // block 0 on this panel of rows: they attend to the rows before them, whose K/V the earlier panels have written
+      if (i == 0) A3_TRY(feed_to(ls + 1 + FEED_AHEAD));  // a full block is long: several layers' copies fit under it
+      if (i + 1 < panels) A3_TRY(recompute_layer_impl(h, 0, w.x_all + (size_t)r0 * m.d_model, w.all_pos + r0, r1 - r0, kl(0), vl(0), n, nullptr, lw, st));
+      else A3_TRY(layer_step(0, w.x_all + (size_t)r0 * m.d_model, w.all_pos + r0, r1 - r0));
+    }
+  }
+  for (int l = 1; l < ls; ++l) {
+    A3_TRY(feed_to(ls + 1 + FEED_AHEAD * (l + 1)));
     A3_TRY(layer_step(l, w.x_all, w.all_pos, n));
   }
   A3_TRY(feed_to(ls + 1 + FEED_AHEAD));
@@ -676,7 +695,7 @@ namespace a3 {
 // copy stream and events of the host-buffer entry, created on first use and kept by the handle
 struct HostPipe {
   cudaStream_t copy_stream;
-  cudaEvent_t start, x0_ready;
+  cudaEvent_t start, x0_ready[X0_PANELS];
   cudaEvent_t* layer_ready;
   int n_layers;
   a3_chunk_ref* href;  // host copy of the chunk descriptors of the last call
@@ -691,7 +710,7 @@ static int host_pipe(const a3_handle* h, HostPipe** out) {
     p->layer_ready = (cudaEvent_t*)calloc(p->n_layers, sizeof(cudaEvent_t));
     cudaError_t e = cudaStreamCreateWithFlags(&p->copy_stream, cudaStreamNonBlocking);
     if (e == cudaSuccess) e = cudaEventCreateWithFlags(&p->start, cudaEventDisableTiming);
-    if (e == cudaSuccess) e = cudaEventCreateWithFlags(&p->x0_ready, cudaEventDisableTiming);
+    for (int i = 0; i < X0_PANELS && e == cudaSuccess; ++i) e = cudaEventCreateWithFlags(&p->x0_ready[i], cudaEventDisableTiming);
     for (int l = 0; l < p->n_layers && e == cudaSuccess; ++l) e = cudaEventCreateWithFlags(&p->layer_ready[l], cudaEventDisableTiming);
     if (e != cudaSuccess) return cuda_fail(e);
     hm->host_pipe = p;
@@ -705,7 +724,8 @@ static void host_pipe_destroy(a3_handle* h) {
   for (int l = 0; l < p->n_layers; ++l)
     if (p->layer_ready[l]) cudaEventDestroy(p->layer_ready[l]);
   if (p->start) cudaEventDestroy(p->start);
-  if (p->x0_ready) cudaEventDestroy(p->x0_ready);
+  for (int i = 0; i < X0_PANELS; ++i)
+    if (p->x0_ready[i]) cudaEventDestroy(p->x0_ready[i]);
   if (p->copy_stream) cudaStreamDestroy(p->copy_stream);
   free(p->layer_ready);
   free(p->href);
@@ -774,8 +794,13 @@ extern "C" int a3_fuse_request_host(const a3_handle* h, const a3_request* req, c
   // the descriptor array is pageable host memory: this copy returns only once it has been staged
   if (status == A3_OK && req->n_chunks > 0)
     note(cudaMemcpyAsync(dref, href, sizeof(a3_chunk_ref) * req->n_chunks, cudaMemcpyHostToDevice, cs));
-  if (status == A3_OK) note(cudaMemcpyAsync(x0, io->x0, (size_t)n * m.d_model * 2, cudaMemcpyHostToDevice, cs));
-  if (status == A3_OK) note(cudaEventRecord(hp->x0_ready, cs));
+  const int panels = x0_panels(n);
+  for (int i = 0; i < panels && status == A3_OK; ++i) {
+    const int r0 = x0_panel_begin(n, i, panels), r1 = x0_panel_begin(n, i + 1, panels);
+    if (note(cudaMemcpyAsync(x0 + (size_t)r0 * m.d_model * 2, (const char*)io->x0 + (size_t)r0 * m.d_model * 2, (size_t)(r1 - r0) * m.d_model * 2,
+                             cudaMemcpyHostToDevice, cs)))
+      note(cudaEventRecord(hp->x0_ready[i], cs));
+  }
   a3_request r = *req;
   r.chunks = dref;
   r.max_chunk_len = maxlen;
