@@ -260,6 +260,22 @@ def test_llama8b_32k_planted_relevance():
     assert share >= 3 * len(planted) / 64, share  # the selection concentrates on the planted chunks
     check_position_recovery_samples(c, seed=2)
     check_layer_samples(c, 2, None, n_samples=6, seed=2)
+    # the host-buffer entry on the same request (chunk caches and embeddings in pinned host memory; the embeddings of an
+    # input this long travel in row panels and the first block starts on the first): the same bits as the device entry
+    m, r = c.m, c.r
+    hk = [k.cpu().pin_memory() for k in c.ck]
+    hv = [v.cpu().pin_memory() for v in c.cv]
+    hx = c.x0.cpu().pin_memory()
+    Kh, Vh = c.buffers()
+    rq, oh = c.eng.make_request(None, len(hk), 0, r.n_ctx, r.n_question, None, Kh, Vh, ratio=r.ratio, select_layer=r.select_layer)
+    M = oh["p"] + r.n_question
+    rows_h = torch.empty(M, dtype=torch.int32).pin_memory()
+    x_h = torch.empty((M, m.d_model), dtype=torch.bfloat16).pin_memory()
+    staging = torch.empty(c.eng.host_staging_bytes(r.n_ctx, r.n), dtype=torch.uint8, device=DEV)
+    c.eng.fuse_request_host(rq, hk, hv, hx, rows_h, x_h, staging)
+    assert c.eng.device_status() == 0
+    assert torch.equal(Kh, K) and torch.equal(Vh, V)
+    assert torch.equal(rows_h, out["rows"].cpu()) and torch.equal(x_h, out["x"].cpu())
     c.eng.close()
 
 
